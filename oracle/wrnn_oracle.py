@@ -1,0 +1,234 @@
+"""ctypes front end of the CPU oracle (``wrnn_oracle.c``).
+
+TEST INFRASTRUCTURE, NOT THE PRODUCT: only tests, the smoke check and the
+benchmark's CPU-baseline leg may import this.  It holds no arithmetic of the
+method: it builds the C file with gcc, marshals numpy arrays and calls it.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "wrnn_oracle.c")
+_LIB = os.path.join(_HERE, "libwrnn_oracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain -O2: no fast-math, no reassociation)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(
+            ["gcc", "-std=c99", "-O2", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Params(C.Structure):
+    _fields_ = [("H", C.c_int32), ("cond_dim", C.c_int32)] + [
+        (n, C.c_void_p)
+        for n in ("R", "I", "b_gate", "W_cond", "O1", "b1", "O2", "b2", "O3", "b3", "O4", "b4")
+    ]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        L.orc_uniform.restype = C.c_double
+        L.orc_uniform.argtypes = [C.c_uint64, C.c_uint32, C.c_uint64, C.c_uint32]
+        L.orc_philox4x32_10.argtypes = [C.c_void_p] * 3
+        L.orc_bf16_round.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
+        L.orc_apply_block_mask.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+        L.orc_scale8.restype = C.c_double
+        L.orc_scale8.argtypes = [C.c_int]
+        L.orc_to_int16.restype = C.c_int16
+        L.orc_to_int16.argtypes = [C.c_uint8, C.c_uint8]
+        L.orc_join16.restype = C.c_uint16
+        L.orc_join16.argtypes = [C.c_uint8, C.c_uint8]
+        L.orc_split16.argtypes = [C.c_uint16, C.c_void_p, C.c_void_p]
+        L.orc_fold.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p]
+        L.orc_unfold.argtypes = [C.c_void_p, C.c_int64, C.c_int, C.c_void_p]
+        L.orc_softmax_sample.restype = C.c_int
+        L.orc_softmax_sample.argtypes = [C.c_void_p, C.c_int, C.c_double, C.c_void_p, C.c_void_p]
+        L.orc_run.restype = C.c_int
+        L.orc_run.argtypes = (
+            [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int,
+             C.c_int64, C.c_uint64, C.c_uint32] + [C.c_void_p] * 12 + [C.c_int]
+        )
+        _lib = L
+    return _lib
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def philox4x32_10(ctr, key) -> np.ndarray:
+    c = np.asarray(ctr, dtype=np.uint32).copy()
+    k = np.asarray(key, dtype=np.uint32).copy()
+    out = np.zeros(4, dtype=np.uint32)
+    lib().orc_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def uniform(seed: int, stream: int, step: int, head: int) -> float:
+    return lib().orc_uniform(seed, stream, step, head)
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty_like(x)
+    lib().orc_bf16_round(_ptr(x), _ptr(out), x.size)
+    return out
+
+
+def apply_block_mask(W: np.ndarray, mask: np.ndarray) -> np.ndarray:
+    W = np.array(W, dtype=np.float32, order="C", copy=True)
+    m = np.ascontiguousarray(mask, dtype=np.uint8)
+    assert m.shape == (W.shape[0] // 4, W.shape[1] // 4)
+    lib().orc_apply_block_mask(_ptr(W), W.shape[0], W.shape[1], _ptr(m))
+    return W
+
+
+def scale8(v: int) -> float:
+    return lib().orc_scale8(int(v))
+
+
+def to_int16(c: int, f: int) -> int:
+    return lib().orc_to_int16(int(c), int(f))
+
+
+def join16(c: int, f: int) -> int:
+    return lib().orc_join16(int(c), int(f))
+
+
+def split16(x: int):
+    c = C.c_uint8()
+    f = C.c_uint8()
+    lib().orc_split16(int(x), C.byref(c), C.byref(f))
+    return c.value, f.value
+
+
+def fold(x: np.ndarray, B: int) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.int16)
+    assert x.size % B == 0
+    sub = np.empty((B, x.size // B), dtype=np.int16)
+    lib().orc_fold(_ptr(x), x.size, B, _ptr(sub))
+    return sub
+
+
+def unfold(sub: np.ndarray) -> np.ndarray:
+    sub = np.ascontiguousarray(sub, dtype=np.int16)
+    B = sub.shape[0]
+    x = np.empty(sub.size, dtype=np.int16)
+    lib().orc_unfold(_ptr(sub), sub.size, B, _ptr(x))
+    return x
+
+
+def softmax_sample(logits: np.ndarray, u: float):
+    """-> (index, probs[n], margin)."""
+    l = np.ascontiguousarray(logits, dtype=np.float32)
+    probs = np.empty(l.size, dtype=np.float64)
+    margin = C.c_double()
+    idx = lib().orc_softmax_sample(_ptr(l), l.size, float(u), _ptr(probs), C.byref(margin))
+    return idx, probs, margin.value
+
+
+_WEIGHT_KEYS = ("R", "I", "W_cond", "O1", "O2", "O3", "O4")
+_BIAS_KEYS = ("b_gate", "b1", "b2", "b3", "b4")
+
+
+@dataclass
+class RunResult:
+    out: np.ndarray            # int16 [batch][n_steps]
+    c_out: np.ndarray          # uint8 [batch][n_steps]  indices the oracle drew
+    f_out: np.ndarray
+    margins: np.ndarray        # float64 [batch][n_steps][2]
+    h: np.ndarray              # float32 [batch][H]  final state
+    c_prev: np.ndarray
+    f_prev: np.ndarray
+    gates: Optional[np.ndarray] = None   # [n_steps][batch][3H]
+    hs: Optional[np.ndarray] = None      # [n_steps][batch][H]
+    logits: Optional[np.ndarray] = None  # [n_steps][batch][2][256]
+
+
+class OracleModel:
+    """The stored model: masks applied, then weights rounded to the storage type.
+
+    `weights` is a dict of fp32 arrays (R, I, b_gate, W_cond, O1, b1, ... b4);
+    `masks` an optional dict with 4x4 block masks for "R" [3H/4][H/4],
+    "O1", "O3" [H/8][H/8]; dtype "f32" or "bf16" (weights R, I, W_cond,
+    O1..O4 rounded to bf16; biases stay fp32).
+    """
+
+    def __init__(self, weights: dict, dtype: str = "f32", masks: Optional[dict] = None):
+        assert dtype in ("f32", "bf16")
+        self.H = int(weights["R"].shape[1])
+        assert weights["R"].shape == (3 * self.H, self.H)
+        self.cond_dim = 0 if weights.get("W_cond") is None else int(weights["W_cond"].shape[1])
+        self.dtype = dtype
+        w = {}
+        for k in _WEIGHT_KEYS:
+            a = weights.get(k)
+            if a is None:
+                w[k] = None
+                continue
+            a = np.array(a, dtype=np.float32, order="C", copy=True)
+            if masks and masks.get(k) is not None:
+                a = apply_block_mask(a, masks[k])
+            if dtype == "bf16":
+                a = bf16_round(a)
+            w[k] = a
+        for k in _BIAS_KEYS:
+            a = weights.get(k)
+            w[k] = None if a is None else np.array(a, dtype=np.float32, order="C", copy=True)
+        self.w = w
+        self._p = _Params(self.H, self.cond_dim, *[_ptr(w[k]) for k in (
+            "R", "I", "b_gate", "W_cond", "O1", "b1", "O2", "b2", "O3", "b3", "O4", "b4")])
+
+    def run(self, cond: Optional[np.ndarray], n_steps: int, batch: int = 1, seed: int = 0, *,
+            hop: int = 120, row_stride: int = 1, row_offset_mul: int = 0, step0: int = 0,
+            stream0: int = 0,
+            h: Optional[np.ndarray] = None, c_prev=None, f_prev=None,
+            c_forced: Optional[np.ndarray] = None, f_forced: Optional[np.ndarray] = None,
+            dump: bool = False, threads: int = 1) -> RunResult:
+        H = self.H
+        n_frames = 0
+        if self.cond_dim:
+            cond = np.ascontiguousarray(cond, dtype=np.float32)
+            assert cond.ndim == 3 and cond.shape[0] == batch and cond.shape[2] == self.cond_dim
+            n_frames = cond.shape[1]
+        else:
+            cond = None
+        hh = np.zeros((batch, H), np.float32) if h is None else np.array(h, np.float32, copy=True).reshape(batch, H)
+        cp = np.full(batch, 128, np.uint8) if c_prev is None else np.array(c_prev, np.uint8, copy=True).reshape(batch)
+        fp = np.zeros(batch, np.uint8) if f_prev is None else np.array(f_prev, np.uint8, copy=True).reshape(batch)
+        if c_forced is not None:
+            c_forced = np.ascontiguousarray(c_forced, np.uint8).reshape(batch, n_steps)
+            f_forced = np.ascontiguousarray(f_forced, np.uint8).reshape(batch, n_steps)
+        out = np.zeros((batch, n_steps), np.int16)
+        c_out = np.zeros((batch, n_steps), np.uint8)
+        f_out = np.zeros((batch, n_steps), np.uint8)
+        margins = np.zeros((batch, n_steps, 2), np.float64)
+        gates = hs = logits = None
+        if dump:
+            gates = np.zeros((n_steps, batch, 3 * H), np.float32)
+            hs = np.zeros((n_steps, batch, H), np.float32)
+            logits = np.zeros((n_steps, batch, 2, 256), np.float32)
+        rc = lib().orc_run(C.byref(self._p), _ptr(cond), n_frames, hop, row_stride, row_offset_mul,
+                           n_steps, batch, step0, seed, stream0, _ptr(hh), _ptr(cp), _ptr(fp),
+                           _ptr(c_forced), _ptr(f_forced), _ptr(out), _ptr(c_out), _ptr(f_out),
+                           _ptr(margins), _ptr(gates), _ptr(hs), _ptr(logits), threads)
+        if rc != 0:
+            raise ValueError("conditioning frame index out of range")
+        return RunResult(out, c_out, f_out, margins, hh, cp, fp, gates, hs, logits)

@@ -1,0 +1,123 @@
+"""Seeded synthetic inputs shared by the tests, the benchmark and the CPU checker.
+
+Holds none of the method's arithmetic: only numpy random draws with the shapes
+of the WaveRNN workloads (24 kHz / 16-bit audio, H = 896 dense, H = 2048 with
+4x4 blocks at 96 % sparsity, 16-way subscale folding, 5 ms conditioning hop).
+The paper's own data (a proprietary single-speaker corpus with linguistic
+features, Section 5) is not available; these inputs stand in for it.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, Optional
+
+import numpy as np
+
+SEED_WEIGHTS = 1802
+SEED_BIASES = 1803
+SEED_MASK = 96
+SEED_COND = 8435
+SEED_SAMPLING = 20180223   # Philox key
+HOP = 120                  # samples per conditioning frame (5 ms at 24 kHz)
+COND_DIM = 64
+
+
+def make_weights(H: int, cond_dim: int = COND_DIM, seed_w: int = SEED_WEIGHTS,
+                 seed_b: int = SEED_BIASES, head_scale: float = 1.0) -> Dict[str, np.ndarray]:
+    """All matrices i.i.d. N(0, 1/H), biases N(0, 1/H); fp32, row-major.
+
+    head_scale multiplies O2 and O4 (peaky output distributions for range tests).
+    """
+    assert H % 8 == 0
+    Hh = H // 2
+    rw = np.random.default_rng(seed_w)
+    rb = np.random.default_rng(seed_b)
+    s = 1.0 / np.sqrt(H)
+
+    def mat(rng, *shape):
+        return (rng.standard_normal(shape) * s).astype(np.float32)
+
+    w = {
+        "R": mat(rw, 3 * H, H),
+        "I": mat(rw, 3 * H, 3),
+        "W_cond": mat(rw, 3 * H, cond_dim) if cond_dim else None,
+        "O1": mat(rw, Hh, Hh),
+        "O2": mat(rw, 256, Hh) * np.float32(head_scale),
+        "O3": mat(rw, Hh, Hh),
+        "O4": mat(rw, 256, Hh) * np.float32(head_scale),
+        "b_gate": mat(rb, 3 * H),
+        "b1": mat(rb, Hh),
+        "b2": mat(rb, 256),
+        "b3": mat(rb, Hh),
+        "b4": mat(rb, 256),
+    }
+    return w
+
+
+def make_block_masks(H: int, sparsity: float = 0.96, seed: int = SEED_MASK) -> Dict[str, np.ndarray]:
+    """Uniform random 4x4 block masks with exactly round((1-sparsity) * n_blocks) kept
+    blocks per matrix; R_u, R_r, R_e are masked separately (stacked as one [3H/4][H/4])."""
+    rng = np.random.default_rng(seed)
+    Hh = H // 2
+
+    def one(rows, cols):
+        nb = (rows // 4) * (cols // 4)
+        keep = int(round((1.0 - sparsity) * nb))
+        m = np.zeros(nb, np.uint8)
+        m[rng.permutation(nb)[:keep]] = 1
+        return m.reshape(rows // 4, cols // 4)
+
+    mR = np.concatenate([one(H, H) for _ in range(3)], axis=0)
+    return {"R": mR, "O1": one(Hh, Hh), "O3": one(Hh, Hh)}
+
+
+def rescale_kept(weights: Dict[str, np.ndarray], masks: Dict[str, np.ndarray], sparsity: float = 0.96):
+    """Multiply the maskable matrices by 1/sqrt(1-sparsity) so that pre-activation
+    variance of the pruned model matches the dense one (a property of the synthetic
+    workload, not of the method)."""
+    g = np.float32(1.0 / np.sqrt(1.0 - sparsity))
+    out = dict(weights)
+    for k in masks:
+        out[k] = (weights[k] * g).astype(np.float32)
+    return out
+
+
+def make_cond(batch: int, n_frames: int, cond_dim: int = COND_DIM, seed: int = SEED_COND) -> np.ndarray:
+    rng = np.random.default_rng(seed)
+    return rng.standard_normal((batch, n_frames, cond_dim)).astype(np.float32)
+
+
+@dataclass
+class Workload:
+    name: str
+    H: int
+    dtype: str               # "f32" | "bf16"
+    batch: int
+    n_steps: int
+    n_frames: int
+    row_stride: int = 1
+    row_offset_mul: int = 0
+    sparsity: Optional[float] = None
+    subscale_B: int = 0       # >0: fold/unfold of one n_steps*B sequence
+
+
+# The five named workloads (index = position in the benchmark's config list).
+WORKLOADS = [
+    Workload("dense896_f32_b1_1200", 896, "f32", 1, 1200, 10),
+    Workload("dense896_bf16_b1_24000", 896, "bf16", 1, 24000, 200),
+    Workload("sparse2048_bf16_b1_24000", 2048, "bf16", 1, 24000, 200, sparsity=0.96),
+    Workload("subscale16_896_bf16_1500", 896, "bf16", 16, 1500, 200, row_stride=16, row_offset_mul=1, subscale_B=16),
+    Workload("batched256_896_bf16_24000", 896, "bf16", 256, 24000, 200),
+]
+
+
+def build_workload(wl: Workload, n_steps: Optional[int] = None, batch: Optional[int] = None):
+    """-> (weights, masks or None, cond[batch][n_frames][64]).  n_steps/batch shrink the case."""
+    w = make_weights(wl.H)
+    masks = None
+    if wl.sparsity is not None:
+        masks = make_block_masks(wl.H, wl.sparsity)
+        w = rescale_kept(w, masks, wl.sparsity)
+    b = wl.batch if batch is None else batch
+    cond = make_cond(b, wl.n_frames)
+    return w, masks, cond

@@ -1,0 +1,199 @@
+/*
+ * wrnn.h -- C ABI of the B200 WaveRNN sampling library (libwrnn.so).
+ *
+ * One thing is computed here: the per-sample autoregressive sampling step of
+ * the WaveRNN ("Efficient Neural Audio Synthesis", Section 2, Eq. 2):
+ *
+ *     x_t = [c_{t-1}, f_{t-1}, c_t]                      8-bit values scaled to [-1,1]
+ *     u_t = sigmoid(R_u h_{t-1} + I*_u x_t + g_u)
+ *     r_t = sigmoid(R_r h_{t-1} + I*_r x_t + g_r)
+ *     e_t = tanh(r_t o (R_e h_{t-1}) + I*_e x_t + g_e)
+ *     h_t = u_t o h_{t-1} + (1 - u_t) o e_t
+ *     y_c, y_f = split(h_t)
+ *     P(c_t) = softmax(O2 relu(O1 y_c + b1) + b2),  P(f_t) = softmax(O4 relu(O3 y_f + b3) + b4)
+ *
+ * evaluated in the order of Fig. 1: R h for both halves, coarse gates, draw c_t,
+ * fine gates (I* lets c_t reach only the fine half), draw f_t; the 16-bit sample is
+ * 256 c_t + f_t.  g = W_cond frame + b_gate is the per-step conditioning vector
+ * (held for `hop` samples).  Dense (Section 2.1), 4x4 block-sparse (Section 3.2)
+ * and batched / subscale-folded (Section 4) forms share these entry points.
+ *
+ * Conventions: C linkage; every function returns a wrnn_status (0 = ok) unless
+ * noted; pointers are marked HOST or DEVICE; the caller owns every buffer it
+ * passes; nothing here takes or returns a C++ or torch type.  Argument errors are
+ * reported synchronously and nothing is launched.  Work is enqueued on the given
+ * CUDA stream (a cudaStream_t passed as void*, NULL = default stream) and is
+ * asynchronous unless noted.  One call in flight per model.  There is no CPU path:
+ * without a usable CUDA device every compute entry point returns WRNN_ERR_CUDA.
+ *
+ * Row order of every 3H-row object: u rows [0,H), r rows [H,2H), e rows [2H,3H);
+ * inside each gate rows [0,H/2) belong to the coarse half, [H/2,H) to the fine half.
+ */
+#ifndef WRNN_H
+#define WRNN_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct wrnn_model wrnn_model;   /* opaque; owns the device memory it allocates */
+
+typedef enum {
+    WRNN_OK = 0,
+    WRNN_ERR_INVALID_ARG = 1,
+    WRNN_ERR_UNSUPPORTED = 2,   /* shape / dtype / batch has no kernel, or it does not fit the device */
+    WRNN_ERR_NOMEM = 3,
+    WRNN_ERR_CUDA = 4,
+    WRNN_ERR_TIMEOUT = 5        /* a bounded device-side wait ran out; the kernel returned cleanly */
+} wrnn_status;
+
+typedef enum { WRNN_F32 = 0, WRNN_BF16 = 1 } wrnn_dtype;
+
+/* Which kernel family wrnn_sample / wrnn_step_teacher_forced use. */
+typedef enum {
+    WRNN_KERNEL_AUTO = 0,       /* the fastest one that supports the model and batch          */
+    WRNN_KERNEL_GENERIC = 1,    /* weights streamed from L2 every step; any shape; bring-up path */
+    WRNN_KERNEL_RESIDENT = 2    /* persistent kernel, weights resident in shared memory        */
+} wrnn_kernel;
+
+/*
+ * Model description for wrnn_create.  All pointers HOST, fp32, row-major, read
+ * during the call only (the library keeps packed copies on the device).
+ */
+typedef struct {
+    int32_t H;                  /* state size, a multiple of 8                                        */
+    int32_t cond_dim;           /* length of a conditioning frame; 0 = unconditioned                  */
+    const float *R;             /* [3H][H]   recurrent matrix, gates stacked u|r|e (Eq. 2)            */
+    const float *I;             /* [3H][3]   input matrix, columns (c_{t-1}, f_{t-1}, c_t); column 2  */
+                                /*           is ignored on coarse rows (the mask of I*, Section 2)    */
+    const float *b_gate;        /* [3H] or NULL (= 0)                                                 */
+    const float *W_cond;        /* [3H][cond_dim], NULL iff cond_dim == 0                             */
+    const float *O1, *b1;       /* [H/2][H/2], [H/2]   coarse hidden layer (b* may be NULL = 0)       */
+    const float *O2, *b2;       /* [256][H/2], [256]   coarse logits                                  */
+    const float *O3, *b3;       /* fine hidden layer, same shapes                                     */
+    const float *O4, *b4;       /* fine logits                                                        */
+    const uint8_t *mask_R;      /* [3H/4][H/4] 1 = 4x4 block kept (Section 3.2), NULL = dense         */
+    const uint8_t *mask_O1;     /* [H/8][H/8] or NULL                                                 */
+    const uint8_t *mask_O3;     /* [H/8][H/8] or NULL                                                 */
+    int32_t dtype;              /* wrnn_dtype: storage type of R, I, W_cond, O1..O4 (bf16 = round to  */
+                                /* nearest even at create); biases, state and all arithmetic are fp32 */
+    int32_t kernel;             /* wrnn_kernel                                                        */
+} wrnn_params;
+
+/*
+ * wrnn_create: validate, apply the block masks, round to the storage type, pack and
+ * upload.  max_batch (>= 1) sizes the per-row exchange and state buffers.  Synchronous;
+ * allocates device memory on the current device.  On failure *out is NULL.
+ */
+int wrnn_create(const wrnn_params *params, int32_t max_batch, wrnn_model **out);
+void wrnn_destroy(wrnn_model *m);   /* NULL is allowed; synchronises the device */
+
+/*
+ * Carry state of `batch` stream rows.  DEVICE pointers, caller-owned, read at the
+ * start and written at the end of a call; a NULL pointer means the default initial
+ * value (h = 0; previous sample 0, i.e. c_prev = 128, f_prev = 0) and no write-back.
+ * Row b has the global row id stream0 + b, which selects its Philox stream and its
+ * conditioning offset; step0 is the absolute index of the first step of the call.
+ * Generating T steps in one call equals generating T1 then T - T1 with the state
+ * carried over and step0 advanced.
+ */
+typedef struct {
+    float *h;            /* [batch][H] */
+    uint8_t *c_prev;     /* [batch]    */
+    uint8_t *f_prev;     /* [batch]    */
+    int64_t step0;
+    uint32_t stream0;
+    uint32_t reserved;
+} wrnn_state;
+
+/*
+ * Conditioning and step geometry shared by the two stepping calls.
+ * Frame index of row b at step s of the call:
+ *     ((step0 + s) * row_stride + (stream0 + b) * row_offset_mul) / hop      (integer division)
+ * which must stay below n_frames.  (1, 0) is an ordinary stream; (B, 1) is row b of a
+ * B-way subscale fold (Section 4.1: row b holds samples B i + b).
+ */
+typedef struct {
+    const float *cond;   /* DEVICE [batch][n_frames][cond_dim] fp32; NULL iff cond_dim == 0 */
+    int32_t n_frames;
+    int32_t hop;         /* samples per frame, > 0 */
+    int32_t row_stride;
+    int32_t row_offset_mul;
+} wrnn_cond;
+
+/*
+ * wrnn_sample: free-running generation (Fig. 1).  For every row and step draws
+ * c_t then f_t with uniforms Philox4x32-10(key = seed; counter = (step lo, head,
+ * global row id, step hi)), word 0 >> 8 scaled by 2^-24, head 0 = coarse, 1 = fine;
+ * inverse CDF: smallest k whose running sum of exp(l - max l) exceeds u times the total.
+ * out: DEVICE int16 [batch][n_steps], value 256 c + f - 32768.
+ * st may be NULL (default state, step0 = 0, stream0 = 0).
+ * May grow an internal scratch buffer (synchronously) when batch * n_frames exceeds
+ * what earlier calls needed.
+ */
+int wrnn_sample(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch,
+                uint64_t seed, const wrnn_state *st, int16_t *out, void *cuda_stream);
+
+/*
+ * wrnn_step_teacher_forced: the same steps, but the samples fed back are given.
+ * Step s uses (c_forced, f_forced)[b][s-1] as the previous sample (the state's
+ * c_prev / f_prev at s = 0) and c_forced[b][s] in the fine gates.  The indices the
+ * device itself draws are written to c_out / f_out.  All DEVICE; forced arrays and
+ * c_out / f_out are uint8 [batch][n_steps].  Optional dumps (NULL = off):
+ *   dbg_gates  [n_steps][batch][3H]     post-activation u | r | e
+ *   dbg_h      [n_steps][batch][H]      h_t
+ *   dbg_logits [n_steps][batch][2][256] pre-softmax logits, coarse then fine
+ */
+int wrnn_step_teacher_forced(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch,
+                             uint64_t seed, const wrnn_state *st,
+                             const uint8_t *c_forced, const uint8_t *f_forced,
+                             uint8_t *c_out, uint8_t *f_out,
+                             float *dbg_gates, float *dbg_h, float *dbg_logits, void *cuda_stream);
+
+/*
+ * Subscale fold / unfold (Section 4.1, Eq. 4): sub-tensor s holds x[B i + s].
+ * x: DEVICE int16 [n_total]; sub: DEVICE int16 [B][n_total / B]; B must divide n_total.
+ */
+int wrnn_fold(const int16_t *x, int64_t n_total, int32_t B, int16_t *sub, void *cuda_stream);
+int wrnn_unfold(const int16_t *sub, int64_t n_total, int32_t B, int16_t *x, void *cuda_stream);
+
+/*
+ * wrnn_sample_subscale: generate one sequence of n_total samples as B interleaved
+ * sub-sequences advanced in lock-step as a batch of B (Section 4.2), then unfold.
+ * cond: [B][n_frames][cond_dim] (row s conditions sub-sequence s), geometry forced to
+ * (row_stride, row_offset_mul) = (B, 1).  out: DEVICE int16 [n_total] in original order.
+ */
+int wrnn_sample_subscale(wrnn_model *m, const float *cond, int32_t n_frames, int32_t hop,
+                         int64_t n_total, int32_t B, uint64_t seed, int16_t *out, void *cuda_stream);
+
+/*
+ * Host-buffer convenience for callers without device pointers: copies cond
+ * (HOST [batch][n_frames][cond_dim]) to the device, runs wrnn_sample from the
+ * default state and copies the samples back to out (HOST int16 [batch][n_steps]).
+ * Synchronous.
+ */
+int wrnn_sample_host(wrnn_model *m, const float *cond_host, int32_t n_frames, int32_t hop,
+                     int32_t row_stride, int32_t row_offset_mul, int64_t n_steps, int32_t batch,
+                     uint64_t seed, int16_t *out_host);
+
+/* After the stream has been synchronised: WRNN_OK, or what the last kernel reported. */
+int wrnn_poll_status(wrnn_model *m);
+/* Diagnostic text of the last error on this model (or of the last failed create when
+ * m == NULL).  Not thread-safe; valid until the next call. */
+const char *wrnn_last_error(wrnn_model *m);
+
+/* Introspection used by the benchmark and the tests (HOST out-pointers, any may be NULL):
+ * kernel family in use, CTAs and threads per CTA of the persistent kernel for `batch`
+ * rows, bytes of packed weights read per step, dynamic shared memory per CTA. */
+int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_ctas,
+                     int32_t *n_threads, int64_t *weight_bytes_per_step, int32_t *smem_bytes);
+
+/* Kernels launched by this library in this process since load (all models). */
+int64_t wrnn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WRNN_H */

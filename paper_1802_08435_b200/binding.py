@@ -1,0 +1,223 @@
+"""Python binding of libwrnn.so: the same entry points as include/wrnn.h.
+
+Argument marshalling only.  Device buffers are torch CUDA tensors (torch is used for
+device memory and streams, nothing else); every step of the sampling path runs in
+the library's CUDA kernels.  There is no CPU path: if the library has not been built
+the import of any entry point raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libwrnn.so")
+
+WRNN_OK, WRNN_ERR_INVALID_ARG, WRNN_ERR_UNSUPPORTED, WRNN_ERR_NOMEM, WRNN_ERR_CUDA, WRNN_ERR_TIMEOUT = range(6)
+WRNN_F32, WRNN_BF16 = 0, 1
+WRNN_KERNEL_AUTO, WRNN_KERNEL_GENERIC, WRNN_KERNEL_RESIDENT = 0, 1, 2
+_STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "NOMEM", "CUDA", "TIMEOUT"]
+
+EXPORTS = [
+    "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
+    "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
+    "wrnn_launch_count",
+]
+
+
+class WrnnError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__("wrnn status %d (%s): %s" % (code, _STATUS_NAMES[code] if 0 <= code < 6 else "?", msg))
+        self.code = code
+
+
+class wrnn_params(C.Structure):
+    _fields_ = (
+        [("H", C.c_int32), ("cond_dim", C.c_int32)]
+        + [(n, C.c_void_p) for n in ("R", "I", "b_gate", "W_cond", "O1", "b1", "O2", "b2", "O3", "b3", "O4", "b4",
+                                     "mask_R", "mask_O1", "mask_O3")]
+        + [("dtype", C.c_int32), ("kernel", C.c_int32)]
+    )
+
+
+class wrnn_state(C.Structure):
+    _fields_ = [("h", C.c_void_p), ("c_prev", C.c_void_p), ("f_prev", C.c_void_p), ("step0", C.c_int64),
+                ("stream0", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class wrnn_cond(C.Structure):
+    _fields_ = [("cond", C.c_void_p), ("n_frames", C.c_int32), ("hop", C.c_int32), ("row_stride", C.c_int32),
+                ("row_offset_mul", C.c_int32)]
+
+
+_lib = None
+
+
+def lib():
+    """Load libwrnn.so; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libwrnn.so is missing: build it with `python -m paper_1802_08435_b200.build` "
+                "(nvcc, sm_100a); this package has no CPU or PyTorch fallback")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint64
+        L.wrnn_create.argtypes = [C.POINTER(wrnn_params), i32, C.POINTER(vp)]
+        L.wrnn_destroy.argtypes = [vp]
+        L.wrnn_destroy.restype = None
+        L.wrnn_sample.argtypes = [vp, C.POINTER(wrnn_cond), i64, i32, u64, C.POINTER(wrnn_state), vp, vp]
+        L.wrnn_step_teacher_forced.argtypes = [vp, C.POINTER(wrnn_cond), i64, i32, u64, C.POINTER(wrnn_state)] + [vp] * 8
+        L.wrnn_fold.argtypes = [vp, i64, i32, vp, vp]
+        L.wrnn_unfold.argtypes = [vp, i64, i32, vp, vp]
+        L.wrnn_sample_subscale.argtypes = [vp, vp, i32, i32, i64, i32, u64, vp, vp]
+        L.wrnn_sample_host.argtypes = [vp, vp, i32, i32, i32, i32, i64, i32, u64, vp]
+        L.wrnn_poll_status.argtypes = [vp]
+        L.wrnn_last_error.argtypes = [vp]
+        L.wrnn_last_error.restype = C.c_char_p
+        L.wrnn_launch_info.argtypes = [vp, i32] + [vp] * 5
+        L.wrnn_launch_count.argtypes = []
+        L.wrnn_launch_count.restype = i64
+        _lib = L
+    return _lib
+
+
+def _np_ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _dev_ptr(t):
+    """Device pointer of a contiguous torch CUDA tensor (or None)."""
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device buffers must be contiguous CUDA tensors"
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _check(rc: int, model=None):
+    if rc != WRNN_OK:
+        msg = lib().wrnn_last_error(model)
+        raise WrnnError(rc, msg.decode() if msg else "")
+
+
+def wrnn_last_error(model=None) -> str:
+    msg = lib().wrnn_last_error(model)
+    return msg.decode() if msg else ""
+
+
+def wrnn_create(weights: Dict[str, np.ndarray], dtype: str = "f32", masks: Optional[Dict[str, np.ndarray]] = None,
+                max_batch: int = 1, kernel: int = WRNN_KERNEL_AUTO):
+    """weights: fp32 numpy arrays R [3H][H], I [3H][3], W_cond [3H][D] or None, O1..O4, b_gate, b1..b4 (or None);
+    masks: optional 4x4 block masks {"R": [3H/4][H/4], "O1": [H/8][H/8], "O3": ...}.  Returns an opaque handle."""
+    keep = {}
+
+    def f32(k):
+        a = weights.get(k)
+        if a is None:
+            return None
+        keep[k] = np.ascontiguousarray(a, dtype=np.float32)
+        return keep[k]
+
+    def u8(k):
+        a = None if masks is None else masks.get(k)
+        if a is None:
+            return None
+        keep["m" + k] = np.ascontiguousarray(a, dtype=np.uint8)
+        return keep["m" + k]
+
+    R = f32("R")
+    H = R.shape[1]
+    Wc = f32("W_cond")
+    p = wrnn_params()
+    p.H = H
+    p.cond_dim = 0 if Wc is None else Wc.shape[1]
+    for k in ("R", "I", "b_gate", "W_cond", "O1", "b1", "O2", "b2", "O3", "b3", "O4", "b4"):
+        setattr(p, k, _np_ptr(f32(k)))
+    p.mask_R, p.mask_O1, p.mask_O3 = _np_ptr(u8("R")), _np_ptr(u8("O1")), _np_ptr(u8("O3"))
+    p.dtype = {"f32": WRNN_F32, "bf16": WRNN_BF16}[dtype]
+    p.kernel = kernel
+    out = C.c_void_p()
+    _check(lib().wrnn_create(C.byref(p), max_batch, C.byref(out)))
+    return out
+
+
+def wrnn_destroy(model):
+    lib().wrnn_destroy(model)
+
+
+def _mk_cond(cond, hop, row_stride, row_offset_mul):
+    if cond is None:
+        return None
+    c = wrnn_cond(_dev_ptr(cond), int(cond.shape[1]), hop, row_stride, row_offset_mul)
+    return C.byref(c)
+
+
+def _mk_state(h, c_prev, f_prev, step0, stream0):
+    if h is None and c_prev is None and f_prev is None and step0 == 0 and stream0 == 0:
+        return None
+    return C.byref(wrnn_state(_dev_ptr(h), _dev_ptr(c_prev), _dev_ptr(f_prev), step0, stream0, 0))
+
+
+def wrnn_sample(model, cond, n_steps: int, batch: int, seed: int, out, *, hop: int = 120, row_stride: int = 1,
+                row_offset_mul: int = 0, h=None, c_prev=None, f_prev=None, step0: int = 0, stream0: int = 0,
+                stream=None):
+    """cond: CUDA float32 [batch][n_frames][cond_dim] or None; out: CUDA int16 [batch][n_steps]."""
+    _check(lib().wrnn_sample(model, _mk_cond(cond, hop, row_stride, row_offset_mul), n_steps, batch, seed,
+                             _mk_state(h, c_prev, f_prev, step0, stream0), _dev_ptr(out), _stream_ptr(stream)), model)
+
+
+def wrnn_step_teacher_forced(model, cond, n_steps: int, batch: int, seed: int, c_forced, f_forced, c_out, f_out, *,
+                             dbg_gates=None, dbg_h=None, dbg_logits=None, hop: int = 120, row_stride: int = 1,
+                             row_offset_mul: int = 0, h=None, c_prev=None, f_prev=None, step0: int = 0,
+                             stream0: int = 0, stream=None):
+    _check(lib().wrnn_step_teacher_forced(
+        model, _mk_cond(cond, hop, row_stride, row_offset_mul), n_steps, batch, seed,
+        _mk_state(h, c_prev, f_prev, step0, stream0), _dev_ptr(c_forced), _dev_ptr(f_forced), _dev_ptr(c_out),
+        _dev_ptr(f_out), _dev_ptr(dbg_gates), _dev_ptr(dbg_h), _dev_ptr(dbg_logits), _stream_ptr(stream)), model)
+
+
+def wrnn_fold(x, B: int, sub, stream=None):
+    _check(lib().wrnn_fold(_dev_ptr(x), x.numel(), B, _dev_ptr(sub), _stream_ptr(stream)))
+
+
+def wrnn_unfold(sub, B: int, x, stream=None):
+    _check(lib().wrnn_unfold(_dev_ptr(sub), sub.numel(), B, _dev_ptr(x), _stream_ptr(stream)))
+
+
+def wrnn_sample_subscale(model, cond, n_total: int, B: int, seed: int, out, *, hop: int = 120, stream=None):
+    _check(lib().wrnn_sample_subscale(model, _dev_ptr(cond), int(cond.shape[1]), hop, n_total, B, seed, _dev_ptr(out),
+                                      _stream_ptr(stream)), model)
+
+
+def wrnn_sample_host(model, cond_host: Optional[np.ndarray], n_steps: int, batch: int, seed: int,
+                     out_host: np.ndarray, *, hop: int = 120, row_stride: int = 1, row_offset_mul: int = 0):
+    """Host buffers in and out (numpy, ideally backed by pinned memory); synchronous."""
+    n_frames = 0 if cond_host is None else int(cond_host.shape[1])
+    assert out_host.dtype == np.int16 and out_host.flags.c_contiguous
+    _check(lib().wrnn_sample_host(model, _np_ptr(cond_host), n_frames, hop, row_stride, row_offset_mul, n_steps, batch,
+                                  seed, _np_ptr(out_host)), model)
+
+
+def wrnn_poll_status(model) -> int:
+    return lib().wrnn_poll_status(model)
+
+
+def wrnn_launch_info(model, batch: int = 1) -> dict:
+    k, n, t, s = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32()
+    w = C.c_int64()
+    _check(lib().wrnn_launch_info(model, batch, C.byref(k), C.byref(n), C.byref(t), C.byref(w), C.byref(s)), model)
+    return dict(kernel=k.value, n_ctas=n.value, n_threads=t.value, weight_bytes_per_step=w.value, smem_bytes=s.value)
+
+
+def wrnn_launch_count() -> int:
+    return lib().wrnn_launch_count()

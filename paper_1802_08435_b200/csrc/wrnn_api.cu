@@ -1,0 +1,399 @@
+// C ABI of libwrnn.so: model creation (masking, rounding, packing, upload), argument
+// checking and dispatch to the kernel families.  Declarations and contracts: include/wrnn.h.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "wrnn_internal.h"
+
+namespace wrnn {
+std::atomic<long long> g_launches{0};
+static std::string g_create_err;
+
+// fp32 -> bf16 storage (round to nearest, ties to even) -> back to fp32.
+static float round_bf16(float v)
+{
+    uint32_t b;
+    std::memcpy(&b, &v, 4);
+    if ((b & 0x7f800000u) != 0x7f800000u) {
+        const uint32_t lsb = (b >> 16) & 1u;
+        b += 0x7fffu + lsb;
+    } else if (b & 0x007fffffu) {
+        b |= 0x00400000u;
+    }
+    b &= 0xffff0000u;
+    float r;
+    std::memcpy(&r, &b, 4);
+    return r;
+}
+
+static inline uint16_t bf16_bits(float rounded)
+{
+    uint32_t b;
+    std::memcpy(&b, &rounded, 4);
+    return (uint16_t)(b >> 16);
+}
+
+// Dense row-major W[rows][cols] (+ optional 4x4 block mask) -> host block rows with the
+// values already rounded to the storage type.
+static void build_bsr(const float *W, int rows, int cols, const uint8_t *mask, bool bf16, BsrHost *out)
+{
+    const int R4 = rows / 4, C4 = cols / 4;
+    out->rows4 = R4; out->cols4 = C4;
+    out->row_ptr.assign(R4 + 1, 0);
+    out->col.clear(); out->vals.clear();
+    for (int br = 0; br < R4; ++br) {
+        for (int bc = 0; bc < C4; ++bc) {
+            if (mask && !mask[(size_t)br * C4 + bc]) continue;
+            out->col.push_back((uint16_t)bc);
+            for (int r = 0; r < 4; ++r)
+                for (int c = 0; c < 4; ++c) {
+                    const float v = W[(size_t)(4 * br + r) * cols + 4 * bc + c];
+                    out->vals.push_back(bf16 ? round_bf16(v) : v);
+                }
+        }
+        out->row_ptr[br + 1] = (int)out->col.size();
+    }
+}
+
+template <typename T> static bool upload(T **dst, const void *src, size_t bytes)
+{
+    *dst = nullptr;
+    if (bytes == 0) return true;
+    if (cudaMalloc((void **)dst, bytes) != cudaSuccess) return false;
+    return cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice) == cudaSuccess;
+}
+
+static bool upload_bsr(const BsrHost &h, bool bf16, BsrDev *d)
+{
+    d->rows4 = h.rows4; d->cols4 = h.cols4; d->nnz = (int)h.col.size();
+    if (!upload(&d->row_ptr, h.row_ptr.data(), h.row_ptr.size() * sizeof(int))) return false;
+    // keep 16 B of slack so that vector loads of an empty matrix stay in bounds
+    std::vector<uint16_t> col(h.col);
+    col.resize(col.size() + 8, 0);
+    if (!upload(&d->col, col.data(), col.size() * sizeof(uint16_t))) return false;
+    if (bf16) {
+        std::vector<uint16_t> v(h.vals.size() + 16, 0);
+        for (size_t i = 0; i < h.vals.size(); ++i) v[i] = bf16_bits(h.vals[i]);
+        return upload((uint16_t **)&d->vals, v.data(), v.size() * sizeof(uint16_t));
+    }
+    std::vector<float> v(h.vals);
+    v.resize(v.size() + 16, 0.f);
+    return upload((float **)&d->vals, v.data(), v.size() * sizeof(float));
+}
+
+static void free_bsr(BsrDev *d)
+{
+    cudaFree(d->row_ptr); cudaFree(d->col); cudaFree(d->vals);
+    *d = BsrDev();
+}
+
+static int fail(wrnn_model *m, int code, const std::string &msg)
+{
+    if (m) m->err = msg; else g_create_err = msg;
+    return code;
+}
+
+static bool ensure_g(wrnn_model *m, size_t floats)
+{
+    if (floats <= m->g_cap) return true;
+    cudaDeviceSynchronize();
+    cudaFree(m->g);
+    m->g = nullptr; m->g_cap = 0;
+    if (cudaMalloc((void **)&m->g, floats * sizeof(float)) != cudaSuccess) { cudaGetLastError(); return false; }
+    m->g_cap = floats;
+    return true;
+}
+
+static bool use_resident(const wrnn_model *m, int batch)
+{
+    if (m->kernel == WRNN_KERNEL_GENERIC) return false;
+    return m->resident != nullptr && resident_supported(m, batch, nullptr) == WRNN_OK;
+}
+
+// Common argument checks of the stepping calls; fills the parts of StepArgs that come from
+// cond / st.  Returns WRNN_OK or an error (message in m->err).
+static int check_step(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, const wrnn_state *st,
+                      StepArgs *a)
+{
+    if (!m) return WRNN_ERR_INVALID_ARG;
+    if (n_steps < 0 || batch < 1) return fail(m, WRNN_ERR_INVALID_ARG, "n_steps < 0 or batch < 1");
+    if (batch > m->max_batch) return fail(m, WRNN_ERR_INVALID_ARG, "batch exceeds max_batch given at create");
+    if (n_steps > (1ll << 31) - 2) return fail(m, WRNN_ERR_INVALID_ARG, "n_steps too large for one call");
+    std::memset(a, 0, sizeof(*a));
+    a->n_steps = n_steps; a->batch = batch;
+    a->step0 = st ? st->step0 : 0;
+    a->stream0 = st ? st->stream0 : 0;
+    if (a->step0 < 0) return fail(m, WRNN_ERR_INVALID_ARG, "step0 < 0");
+    if (st) {
+        a->h_in = st->h; a->h_out = st->h;
+        a->c_in = st->c_prev; a->c_st_out = st->c_prev;
+        a->f_in = st->f_prev; a->f_st_out = st->f_prev;
+    }
+    if (m->cond_dim > 0) {
+        if (!cond || !cond->cond) return fail(m, WRNN_ERR_INVALID_ARG, "model is conditioned but cond is NULL");
+        if (cond->hop <= 0 || cond->n_frames <= 0 || cond->row_stride < 0 || cond->row_offset_mul < 0)
+            return fail(m, WRNN_ERR_INVALID_ARG, "bad conditioning geometry");
+        a->cond = cond->cond; a->n_frames = cond->n_frames; a->hop = cond->hop;
+        a->row_stride = cond->row_stride; a->row_offset_mul = cond->row_offset_mul;
+        if (n_steps > 0) {
+            const long long last = ((a->step0 + n_steps - 1) * (long long)a->row_stride +
+                                    ((long long)a->stream0 + batch - 1) * a->row_offset_mul) / a->hop;
+            if (last >= a->n_frames) return fail(m, WRNN_ERR_INVALID_ARG, "conditioning frames run out before n_steps");
+        }
+    } else {
+        a->n_frames = 1; a->hop = 1;
+    }
+    return WRNN_OK;
+}
+
+static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
+{
+    if (a.n_steps == 0) return WRNN_OK;
+    if (cudaSetDevice(m->device) != cudaSuccess) return fail(m, WRNN_ERR_CUDA, "cudaSetDevice failed");
+    const int nf = m->cond_dim ? a.n_frames : 1;
+    if (!ensure_g(m, (size_t)a.batch * nf * 3 * m->H)) return fail(m, WRNN_ERR_NOMEM, "conditioning scratch allocation failed");
+    int rc = cond_project(m, a.cond, a.batch, nf, s);
+    if (rc != WRNN_OK) return fail(m, rc, "conditioning projection launch failed");
+    if (use_resident(m, a.batch)) return resident_run(m, a, s);
+    if (m->kernel == WRNN_KERNEL_RESIDENT) {
+        std::string why;
+        resident_supported(m, a.batch, &why);
+        return fail(m, WRNN_ERR_UNSUPPORTED, "resident kernel unavailable: " + why);
+    }
+    return generic_run(m, a, s);
+}
+
+}  // namespace wrnn
+
+using namespace wrnn;
+
+extern "C" {
+
+int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
+{
+    if (out) *out = nullptr;
+    if (!p || !out) return fail(nullptr, WRNN_ERR_INVALID_ARG, "null params or out");
+    const int H = p->H;
+    if (H < 8 || H % 8 != 0 || H > 65536 * 4 / 4) return fail(nullptr, WRNN_ERR_INVALID_ARG, "H must be a positive multiple of 8");
+    if (H / 4 > 65535) return fail(nullptr, WRNN_ERR_UNSUPPORTED, "H too large for 16-bit block columns");
+    if (max_batch < 1 || max_batch > 65536) return fail(nullptr, WRNN_ERR_INVALID_ARG, "max_batch out of range");
+    if (p->cond_dim < 0 || p->cond_dim > 4096) return fail(nullptr, WRNN_ERR_INVALID_ARG, "cond_dim out of range");
+    if (!p->R || !p->I || !p->O1 || !p->O2 || !p->O3 || !p->O4) return fail(nullptr, WRNN_ERR_INVALID_ARG, "missing weight matrix");
+    if ((p->cond_dim > 0) != (p->W_cond != nullptr)) return fail(nullptr, WRNN_ERR_INVALID_ARG, "W_cond must be given iff cond_dim > 0");
+    if (p->dtype != WRNN_F32 && p->dtype != WRNN_BF16) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown dtype");
+    if (p->kernel < WRNN_KERNEL_AUTO || p->kernel > WRNN_KERNEL_RESIDENT) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown kernel family");
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, WRNN_ERR_CUDA, "no usable CUDA device"); }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return fail(nullptr, WRNN_ERR_CUDA, "cudaGetDeviceProperties failed");
+    if (prop.major != 10) return fail(nullptr, WRNN_ERR_UNSUPPORTED, "this library is built for sm_100a (B200) only");
+
+    wrnn_model *m = new (std::nothrow) wrnn_model();
+    if (!m) return fail(nullptr, WRNN_ERR_NOMEM, "host allocation failed");
+    m->H = H; m->cond_dim = p->cond_dim; m->dtype = p->dtype; m->kernel = p->kernel; m->max_batch = max_batch;
+    m->device = dev; m->n_sms = prop.multiProcessorCount;
+    m->sparse = p->mask_R || p->mask_O1 || p->mask_O3;
+    const bool bf = p->dtype == WRNN_BF16;
+    const int Hh = H / 2, G = 3 * H;
+
+    build_bsr(p->R, G, H, p->mask_R, bf, &m->hR);
+    build_bsr(p->O1, Hh, Hh, p->mask_O1, bf, &m->hO1);
+    build_bsr(p->O2, 256, Hh, nullptr, bf, &m->hO2);
+    build_bsr(p->O3, Hh, Hh, p->mask_O3, bf, &m->hO3);
+    build_bsr(p->O4, 256, Hh, nullptr, bf, &m->hO4);
+    m->hI.resize((size_t)G * 3);
+    for (int row = 0; row < G; ++row)
+        for (int c = 0; c < 3; ++c) {
+            float v = p->I[(size_t)row * 3 + c];
+            if (c == 2 && (row % H) < Hh) v = 0.f;          // c_t reaches only the fine half (I*)
+            m->hI[(size_t)row * 3 + c] = bf ? round_bf16(v) : v;
+        }
+    auto copy_bias = [](const float *b, int n, std::vector<float> *dst) { dst->assign(n, 0.f); if (b) std::memcpy(dst->data(), b, n * sizeof(float)); };
+    copy_bias(p->b_gate, G, &m->hb_gate);
+    copy_bias(p->b1, Hh, &m->hb1); copy_bias(p->b2, 256, &m->hb2);
+    copy_bias(p->b3, Hh, &m->hb3); copy_bias(p->b4, 256, &m->hb4);
+    std::vector<float> WcT((size_t)p->cond_dim * G);
+    for (int row = 0; row < G; ++row)
+        for (int d = 0; d < p->cond_dim; ++d) {
+            const float v = p->W_cond[(size_t)row * p->cond_dim + d];
+            WcT[(size_t)d * G + row] = bf ? round_bf16(v) : v;
+        }
+
+    bool ok = upload_bsr(m->hR, bf, &m->R) && upload_bsr(m->hO1, bf, &m->O1) && upload_bsr(m->hO2, bf, &m->O2) &&
+              upload_bsr(m->hO3, bf, &m->O3) && upload_bsr(m->hO4, bf, &m->O4) &&
+              upload(&m->I, m->hI.data(), m->hI.size() * 4) && upload(&m->b_gate, m->hb_gate.data(), G * 4) &&
+              upload(&m->b1, m->hb1.data(), Hh * 4) && upload(&m->b2, m->hb2.data(), 256 * 4) &&
+              upload(&m->b3, m->hb3.data(), Hh * 4) && upload(&m->b4, m->hb4.data(), 256 * 4) &&
+              upload(&m->W_condT, WcT.data(), WcT.size() * 4);
+    const size_t B = (size_t)max_batch;
+    ok = ok && cudaMalloc((void **)&m->hbuf[0], B * H * 4) == cudaSuccess &&
+         cudaMalloc((void **)&m->hbuf[1], B * H * 4) == cudaSuccess &&
+         cudaMalloc((void **)&m->a_fine, B * 3 * Hh * 4) == cudaSuccess &&
+         cudaMalloc((void **)&m->q, B * Hh * 4) == cudaSuccess &&
+         cudaMalloc((void **)&m->logits, B * 256 * 4) == cudaSuccess &&
+         cudaMalloc((void **)&m->c_cur, B) == cudaSuccess && cudaMalloc((void **)&m->c_prev, B) == cudaSuccess &&
+         cudaMalloc((void **)&m->f_prev, B) == cudaSuccess &&
+         cudaMalloc((void **)&m->bar, 256) == cudaSuccess && cudaMalloc((void **)&m->status, sizeof(DevStatus)) == cudaSuccess;
+    if (ok) ok = cudaMemset(m->status, 0, sizeof(DevStatus)) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        wrnn_destroy(m);
+        return fail(nullptr, WRNN_ERR_NOMEM, "device allocation or upload failed");
+    }
+    const int wsz = bf ? 2 : 4;
+    auto bsr_bytes = [&](const BsrHost &h) { return (int64_t)h.vals.size() * wsz + (int64_t)h.col.size() * 2 + (int64_t)h.row_ptr.size() * 4; };
+    m->weight_bytes = bsr_bytes(m->hR) + bsr_bytes(m->hO1) + bsr_bytes(m->hO2) + bsr_bytes(m->hO3) + bsr_bytes(m->hO4) +
+                      (int64_t)G * 3 * 4;
+
+    if (p->kernel != WRNN_KERNEL_GENERIC) {
+        const int rc = resident_prepare(m);
+        if (rc != WRNN_OK && p->kernel == WRNN_KERNEL_RESIDENT) {
+            const std::string why = m->err;
+            wrnn_destroy(m);
+            return fail(nullptr, rc, "resident kernel unavailable: " + why);
+        }
+    }
+    *out = m;
+    return WRNN_OK;
+}
+
+void wrnn_destroy(wrnn_model *m)
+{
+    if (!m) return;
+    cudaSetDevice(m->device);
+    cudaDeviceSynchronize();
+    resident_destroy(m);
+    free_bsr(&m->R); free_bsr(&m->O1); free_bsr(&m->O2); free_bsr(&m->O3); free_bsr(&m->O4);
+    cudaFree(m->I); cudaFree(m->b_gate); cudaFree(m->b1); cudaFree(m->b2); cudaFree(m->b3); cudaFree(m->b4);
+    cudaFree(m->W_condT); cudaFree(m->g); cudaFree(m->hbuf[0]); cudaFree(m->hbuf[1]); cudaFree(m->a_fine);
+    cudaFree(m->q); cudaFree(m->logits); cudaFree(m->c_cur); cudaFree(m->c_prev); cudaFree(m->f_prev);
+    cudaFree(m->bar); cudaFree(m->status); cudaFree(m->stage_cond); cudaFree(m->stage_out);
+    cudaGetLastError();
+    delete m;
+}
+
+int wrnn_sample(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, uint64_t seed,
+                const wrnn_state *st, int16_t *out, void *cuda_stream)
+{
+    StepArgs a;
+    int rc = check_step(m, cond, n_steps, batch, st, &a);
+    if (rc != WRNN_OK) return rc;
+    if (!out && n_steps > 0) return fail(m, WRNN_ERR_INVALID_ARG, "out is NULL");
+    a.seed = seed; a.out = out;
+    return run_steps(m, a, (cudaStream_t)cuda_stream);
+}
+
+int wrnn_step_teacher_forced(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, uint64_t seed,
+                             const wrnn_state *st, const uint8_t *c_forced, const uint8_t *f_forced, uint8_t *c_out,
+                             uint8_t *f_out, float *dbg_gates, float *dbg_h, float *dbg_logits, void *cuda_stream)
+{
+    StepArgs a;
+    int rc = check_step(m, cond, n_steps, batch, st, &a);
+    if (rc != WRNN_OK) return rc;
+    if ((!c_forced || !f_forced) && n_steps > 0) return fail(m, WRNN_ERR_INVALID_ARG, "forced sample arrays are NULL");
+    a.seed = seed;
+    a.c_forced = c_forced; a.f_forced = f_forced; a.c_out = c_out; a.f_out = f_out;
+    a.dbg_gates = dbg_gates; a.dbg_h = dbg_h; a.dbg_logits = dbg_logits;
+    return run_steps(m, a, (cudaStream_t)cuda_stream);
+}
+
+int wrnn_fold(const int16_t *x, int64_t n_total, int32_t B, int16_t *sub, void *cuda_stream)
+{
+    if (B < 1 || n_total < 0 || n_total % B != 0 || (n_total > 0 && (!x || !sub))) return WRNN_ERR_INVALID_ARG;
+    return fold_launch(x, n_total, B, sub, false, (cudaStream_t)cuda_stream);
+}
+
+int wrnn_unfold(const int16_t *sub, int64_t n_total, int32_t B, int16_t *x, void *cuda_stream)
+{
+    if (B < 1 || n_total < 0 || n_total % B != 0 || (n_total > 0 && (!x || !sub))) return WRNN_ERR_INVALID_ARG;
+    return fold_launch(sub, n_total, B, x, true, (cudaStream_t)cuda_stream);
+}
+
+int wrnn_sample_subscale(wrnn_model *m, const float *cond, int32_t n_frames, int32_t hop, int64_t n_total, int32_t B,
+                         uint64_t seed, int16_t *out, void *cuda_stream)
+{
+    if (!m) return WRNN_ERR_INVALID_ARG;
+    if (B < 1 || n_total < 0 || n_total % B != 0) return fail(m, WRNN_ERR_INVALID_ARG, "B must divide n_total");
+    if (n_total == 0) return WRNN_OK;
+    if (!out) return fail(m, WRNN_ERR_INVALID_ARG, "out is NULL");
+    const size_t need = (size_t)n_total;
+    if (need > m->stage_out_cap) {
+        cudaDeviceSynchronize();
+        cudaFree(m->stage_out); m->stage_out = nullptr; m->stage_out_cap = 0;
+        if (cudaMalloc((void **)&m->stage_out, need * sizeof(int16_t)) != cudaSuccess) { cudaGetLastError(); return fail(m, WRNN_ERR_NOMEM, "staging allocation failed"); }
+        m->stage_out_cap = need;
+    }
+    wrnn_cond c = {cond, n_frames, hop, B, 1};
+    int rc = wrnn_sample(m, &c, n_total / B, B, seed, nullptr, m->stage_out, cuda_stream);
+    if (rc != WRNN_OK) return rc;
+    return fold_launch(m->stage_out, n_total, B, out, true, (cudaStream_t)cuda_stream);
+}
+
+int wrnn_sample_host(wrnn_model *m, const float *cond_host, int32_t n_frames, int32_t hop, int32_t row_stride,
+                     int32_t row_offset_mul, int64_t n_steps, int32_t batch, uint64_t seed, int16_t *out_host)
+{
+    if (!m) return WRNN_ERR_INVALID_ARG;
+    if (batch < 1 || n_steps < 0 || n_frames < 0) return fail(m, WRNN_ERR_INVALID_ARG, "bad sizes");
+    if (cudaSetDevice(m->device) != cudaSuccess) return fail(m, WRNN_ERR_CUDA, "cudaSetDevice failed");
+    const size_t nc = m->cond_dim ? (size_t)batch * n_frames * m->cond_dim : 0;
+    const size_t no = (size_t)batch * (size_t)n_steps;
+    if (nc > m->stage_cond_cap) {
+        cudaDeviceSynchronize();
+        cudaFree(m->stage_cond); m->stage_cond = nullptr; m->stage_cond_cap = 0;
+        if (cudaMalloc((void **)&m->stage_cond, nc * sizeof(float)) != cudaSuccess) { cudaGetLastError(); return fail(m, WRNN_ERR_NOMEM, "staging allocation failed"); }
+        m->stage_cond_cap = nc;
+    }
+    // the subscale path shares stage_out; size for either use
+    if (no > m->stage_out_cap) {
+        cudaDeviceSynchronize();
+        cudaFree(m->stage_out); m->stage_out = nullptr; m->stage_out_cap = 0;
+        if (cudaMalloc((void **)&m->stage_out, no * sizeof(int16_t)) != cudaSuccess) { cudaGetLastError(); return fail(m, WRNN_ERR_NOMEM, "staging allocation failed"); }
+        m->stage_out_cap = no;
+    }
+    if (nc && (!cond_host || cudaMemcpyAsync(m->stage_cond, cond_host, nc * sizeof(float), cudaMemcpyHostToDevice, 0) != cudaSuccess))
+        return fail(m, WRNN_ERR_CUDA, "cond upload failed");
+    wrnn_cond c = {m->stage_cond, n_frames, hop, row_stride, row_offset_mul};
+    int rc = wrnn_sample(m, m->cond_dim ? &c : nullptr, n_steps, batch, seed, nullptr, m->stage_out, nullptr);
+    if (rc != WRNN_OK) return rc;
+    if (no && cudaMemcpyAsync(out_host, m->stage_out, no * sizeof(int16_t), cudaMemcpyDeviceToHost, 0) != cudaSuccess)
+        return fail(m, WRNN_ERR_CUDA, "sample download failed");
+    if (cudaStreamSynchronize(0) != cudaSuccess) return fail(m, WRNN_ERR_CUDA, cudaGetErrorString(cudaGetLastError()));
+    return wrnn_poll_status(m);
+}
+
+int wrnn_poll_status(wrnn_model *m)
+{
+    if (!m) return WRNN_ERR_INVALID_ARG;
+    DevStatus st;
+    if (cudaMemcpy(&st, m->status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return fail(m, WRNN_ERR_CUDA, std::string("status read failed: ") + cudaGetErrorString(cudaGetLastError()));
+    if (st.code != DEV_OK) {
+        char buf[160];
+        std::snprintf(buf, sizeof(buf), "device-side wait timed out (code %d) at cta %d, step %d, phase %d", st.code, st.cta, st.step, st.phase);
+        m->err = buf;
+        return st.code == DEV_TIMEOUT ? WRNN_ERR_TIMEOUT : WRNN_ERR_CUDA;
+    }
+    return WRNN_OK;
+}
+
+const char *wrnn_last_error(wrnn_model *m) { return m ? m->err.c_str() : g_create_err.c_str(); }
+
+int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_ctas, int32_t *n_threads,
+                     int64_t *weight_bytes_per_step, int32_t *smem_bytes)
+{
+    if (!m || batch < 1 || batch > m->max_batch) return WRNN_ERR_INVALID_ARG;
+    if (use_resident(m, batch)) {
+        if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
+        return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
+    }
+    if (kernel) *kernel = WRNN_KERNEL_GENERIC;
+    if (weight_bytes_per_step) *weight_bytes_per_step = m->weight_bytes;
+    return generic_launch_info(m, batch, n_ctas, n_threads, smem_bytes);
+}
+
+int64_t wrnn_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

@@ -1,0 +1,363 @@
+// Generic WaveRNN step kernel: one persistent cooperative kernel per call, weights streamed
+// from global memory (L2-resident) every step, every matrix held as 4x4 block rows, any H,
+// any batch, dense or block-sparse, fp32 or bf16 storage.  This is the bring-up and
+// cross-check path; the shared-memory-resident kernels are the fast ones.
+//
+// Per step (Eq. 2 in the order of Fig. 1), phases separated by grid-wide barriers:
+//   A  a = R h_{t-1} for all 3H rows; coarse gates -> y_c; fine rows keep their a
+//   B  q_c = relu(O1 y_c + b1)          C  l_c = O2 q_c + b2         D  draw c_t
+//   E  fine gates (now with c_t) -> y_f
+//   F  q_f = relu(O3 y_f + b3)          G  l_f = O4 q_f + b4         H  draw f_t, emit sample
+#include "wrnn_internal.h"
+
+namespace wrnn {
+
+struct GenericParams {
+    int H, Hh, G, batch;
+    long long n_steps, step0;
+    unsigned stream0;
+    unsigned long long seed;
+    int n_frames, hop, row_stride, row_offset_mul;
+    BsrDev R, O1, O2, O3, O4;
+    const float *I, *b1, *b2, *b3, *b4, *g;
+    float *h0, *h1, *a_fine, *q, *logits;
+    uint8_t *c_cur, *c_prev, *f_prev;
+    const float *h_in; float *h_out;
+    const uint8_t *c_in, *f_in; uint8_t *c_st_out, *f_st_out;
+    const uint8_t *c_forced, *f_forced;
+    uint8_t *c_out, *f_out;
+    int16_t *out;
+    float *dbg_gates, *dbg_h, *dbg_logits;
+    unsigned long long *bar;
+    DevStatus *status;
+    unsigned long long limit_ns;
+};
+
+template <typename WT> __device__ __forceinline__ void load_block(const void *vals, int i, float (&w)[16]);
+
+template <> __device__ __forceinline__ void load_block<float>(const void *vals, int i, float (&w)[16])
+{
+    const float4 *p = reinterpret_cast<const float4 *>(vals) + 4 * (size_t)i;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const float4 v = __ldg(p + r);
+        w[4 * r] = v.x; w[4 * r + 1] = v.y; w[4 * r + 2] = v.z; w[4 * r + 3] = v.w;
+    }
+}
+template <> __device__ __forceinline__ void load_block<uint16_t>(const void *vals, int i, float (&w)[16])
+{
+    const uint4 *p = reinterpret_cast<const uint4 *>(vals) + 2 * (size_t)i;
+#pragma unroll
+    for (int hlf = 0; hlf < 2; ++hlf) {
+        const uint4 v = __ldg(p + hlf);
+        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { w[8 * hlf + 2 * k] = bf16lo(u[k]); w[8 * hlf + 2 * k + 1] = bf16hi(u[k]); }
+    }
+}
+
+// acc[r * TB + b] += sum over the kept blocks of block row br of W[4 br + r][:] . x[b][:]
+// (lanes stride over the blocks; the caller reduces across lanes).  x was written by other
+// CTAs in an earlier phase, hence the L1-bypassing loads.
+template <typename WT, int TB>
+__device__ __forceinline__ void blockrow_dot(const BsrDev &M, int br, const float *x, int ldx, int nb,
+                                             int lane, float (&acc)[4 * TB])
+{
+    const int beg = __ldg(M.row_ptr + br), end = __ldg(M.row_ptr + br + 1);
+    for (int i = beg + lane; i < end; i += 32) {
+        float w[16];
+        load_block<WT>(M.vals, i, w);
+        const int bc = __ldg(M.col + i);
+#pragma unroll
+        for (int b = 0; b < TB; ++b) {
+            if (b < nb) {
+                const float4 xv = __ldcg(reinterpret_cast<const float4 *>(x + (size_t)b * ldx + 4 * bc));
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    float s = acc[r * TB + b];
+                    s = fmaf(w[4 * r], xv.x, s);
+                    s = fmaf(w[4 * r + 1], xv.y, s);
+                    s = fmaf(w[4 * r + 2], xv.z, s);
+                    s = fmaf(w[4 * r + 3], xv.w, s);
+                    acc[r * TB + b] = s;
+                }
+            }
+        }
+    }
+}
+
+template <typename WT, int TB>
+__device__ __forceinline__ float blockrow_total(const BsrDev &M, int br, const float *x, int ldx, int nb, int lane)
+{
+    float acc[4 * TB];
+#pragma unroll
+    for (int i = 0; i < 4 * TB; ++i) acc[i] = 0.f;
+    blockrow_dot<WT, TB>(M, br, x, ldx, nb, lane, acc);
+    return warp_reduce_scatter<4 * TB>(acc, lane);
+}
+
+__device__ __forceinline__ long long frame_of(const GenericParams &p, long long s, int gb)
+{
+    return ((p.step0 + s) * p.row_stride + (long long)(p.stream0 + (unsigned)gb) * p.row_offset_mul) / p.hop;
+}
+
+// Gate evaluation of one state unit (Eq. 2).  a* = (R h)[row]; x2 is used on fine rows only.
+__device__ __forceinline__ float gate_unit(const GenericParams &p, int j, int gb, long long s, float au, float ar,
+                                           float ae, float hprev, float x0, float x1, float x2, bool fine)
+{
+    const int H = p.H;
+    const float *g = p.g + ((size_t)gb * p.n_frames + (size_t)frame_of(p, s, gb)) * p.G;
+    const float *Iu = p.I + 3 * (size_t)j, *Ir = p.I + 3 * (size_t)(H + j), *Ie = p.I + 3 * (size_t)(2 * H + j);
+    float pu = au + fmaf(Iu[0], x0, fmaf(Iu[1], x1, g[j]));
+    float pr = ar + fmaf(Ir[0], x0, fmaf(Ir[1], x1, g[H + j]));
+    float pe = fmaf(Ie[0], x0, fmaf(Ie[1], x1, g[2 * H + j]));
+    if (fine) { pu = fmaf(Iu[2], x2, pu); pr = fmaf(Ir[2], x2, pr); pe = fmaf(Ie[2], x2, pe); }
+    const float u = sigmoidf_acc(pu);
+    const float r = sigmoidf_acc(pr);
+    const float e = tanhf(fmaf(r, ae, pe));
+    const float hn = fmaf(u, hprev, (1.0f - u) * e);
+    if (p.dbg_gates) {
+        float *d = p.dbg_gates + ((size_t)s * p.batch + gb) * p.G;
+        d[j] = u; d[H + j] = r; d[2 * H + j] = e;
+    }
+    if (p.dbg_h) p.dbg_h[((size_t)s * p.batch + gb) * H + j] = hn;
+    return hn;
+}
+
+template <typename WT, int TB>
+__global__ void __launch_bounds__(512, 1) generic_step_kernel(const GenericParams p)
+{
+    const int lane = threadIdx.x & 31;
+    const int warps_per_cta = blockDim.x >> 5;
+    const int gw = blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
+    const int nw = gridDim.x * warps_per_cta;
+    const int gtid = blockIdx.x * blockDim.x + threadIdx.x;
+    const int nthreads = gridDim.x * blockDim.x;
+    const int H = p.H, Hh = p.Hh, B = p.batch;
+    const int ntiles = (B + TB - 1) / TB;
+    constexpr int N = 4 * TB;
+
+    GridBarrier bar{p.bar, p.status, 0ull, p.limit_ns};
+
+    float *hc = p.h0, *hn = p.h1;
+    for (int i = gtid; i < B * H; i += nthreads) hc[i] = p.h_in ? p.h_in[i] : 0.f;
+    for (int i = gtid; i < B; i += nthreads) {
+        p.c_prev[i] = p.c_in ? p.c_in[i] : (uint8_t)128;
+        p.f_prev[i] = p.f_in ? p.f_in[i] : (uint8_t)0;
+    }
+    if (!bar.sync(-1, 0)) return;
+
+    for (long long s = 0; s < p.n_steps; ++s) {
+        // ---- A: recurrent product for all gates; coarse gates finish here
+        for (int item = gw; item < (H / 4) * ntiles; item += nw) {
+            const int ug = item / ntiles, b0 = (item % ntiles) * TB, nb = min(TB, B - b0);
+            const float *x = hc + (size_t)b0 * H;
+            const float au = blockrow_total<WT, TB>(p.R, ug, x, H, nb, lane);
+            const float ar = blockrow_total<WT, TB>(p.R, H / 4 + ug, x, H, nb, lane);
+            const float ae = blockrow_total<WT, TB>(p.R, 2 * (H / 4) + ug, x, H, nb, lane);
+            const int r = (lane & (N - 1)) / TB, b = (lane & (N - 1)) % TB;
+            if (lane < N && b < nb) {
+                const int j = 4 * ug + r, gb = b0 + b;
+                if (j < Hh) {
+                    const float x0 = scale8(__ldcg(p.c_prev + gb)), x1 = scale8(__ldcg(p.f_prev + gb));
+                    hn[(size_t)gb * H + j] = gate_unit(p, j, gb, s, au, ar, ae, __ldcg(hc + (size_t)gb * H + j), x0, x1, 0.f, false);
+                } else {
+                    float *af = p.a_fine + (size_t)gb * 3 * Hh + (j - Hh);
+                    af[0] = au; af[Hh] = ar; af[2 * Hh] = ae;
+                }
+            }
+        }
+        if (!bar.sync((int)s, 1)) return;
+
+        for (int head = 0; head < 2; ++head) {
+            const BsrDev &Oa = head ? p.O3 : p.O1, &Ob = head ? p.O4 : p.O2;
+            const float *ba = head ? p.b3 : p.b1, *bb = head ? p.b4 : p.b2;
+            if (head == 1) {
+                // ---- E: fine gates, one thread per (row, fine unit)
+                for (int i = gtid; i < B * Hh; i += nthreads) {
+                    const int gb = i / Hh, jf = i % Hh, j = Hh + jf;
+                    const float *af = p.a_fine + (size_t)gb * 3 * Hh + jf;
+                    const float x0 = scale8(__ldcg(p.c_prev + gb)), x1 = scale8(__ldcg(p.f_prev + gb));
+                    const float x2 = scale8(__ldcg(p.c_cur + gb));
+                    hn[(size_t)gb * H + j] = gate_unit(p, j, gb, s, __ldcg(af), __ldcg(af + Hh), __ldcg(af + 2 * Hh),
+                                                       __ldcg(hc + (size_t)gb * H + j), x0, x1, x2, true);
+                }
+                if (!bar.sync((int)s, 5)) return;
+            }
+            // ---- B / F: hidden layer of the head on its half of the new state
+            for (int item = gw; item < (Hh / 4) * ntiles; item += nw) {
+                const int br = item / ntiles, b0 = (item % ntiles) * TB, nb = min(TB, B - b0);
+                const float v = blockrow_total<WT, TB>(Oa, br, hn + (size_t)b0 * H + head * Hh, H, nb, lane);
+                const int r = (lane & (N - 1)) / TB, b = (lane & (N - 1)) % TB;
+                if (lane < N && b < nb) {
+                    const int row = 4 * br + r;
+                    p.q[(size_t)(b0 + b) * Hh + row] = fmaxf(v + (ba ? ba[row] : 0.f), 0.f);
+                }
+            }
+            if (!bar.sync((int)s, head ? 6 : 2)) return;
+            // ---- C / G: logits
+            for (int item = gw; item < 64 * ntiles; item += nw) {
+                const int br = item / ntiles, b0 = (item % ntiles) * TB, nb = min(TB, B - b0);
+                const float v = blockrow_total<WT, TB>(Ob, br, p.q + (size_t)b0 * Hh, Hh, nb, lane);
+                const int r = (lane & (N - 1)) / TB, b = (lane & (N - 1)) % TB;
+                if (lane < N && b < nb) {
+                    const int row = 4 * br + r;
+                    const float l = v + (bb ? bb[row] : 0.f);
+                    p.logits[(size_t)(b0 + b) * 256 + row] = l;
+                    if (p.dbg_logits) p.dbg_logits[(((size_t)s * B + b0 + b) * 2 + head) * 256 + row] = l;
+                }
+            }
+            if (!bar.sync((int)s, head ? 7 : 3)) return;
+            // ---- D / H: softmax + inverse-CDF draw, one warp per row
+            for (int gb = gw; gb < B; gb += nw) {
+                float l[8];
+                const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(p.logits + (size_t)gb * 256 + 8 * lane));
+                const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(p.logits + (size_t)gb * 256 + 8 * lane + 4));
+                l[0] = v0.x; l[1] = v0.y; l[2] = v0.z; l[3] = v0.w; l[4] = v1.x; l[5] = v1.y; l[6] = v1.z; l[7] = v1.w;
+                const float u = uniform24(p.seed, p.stream0 + (unsigned)gb, (unsigned long long)(p.step0 + s), head);
+                int idx = warp_softmax_draw(l, u, lane);
+                if (lane == 0) {
+                    const size_t o = (size_t)gb * p.n_steps + s;
+                    if (head == 0) {
+                        if (p.c_out) p.c_out[o] = (uint8_t)idx;
+                        if (p.c_forced) idx = p.c_forced[o];
+                        p.c_cur[gb] = (uint8_t)idx;
+                    } else {
+                        if (p.f_out) p.f_out[o] = (uint8_t)idx;
+                        if (p.f_forced) idx = p.f_forced[o];
+                        const int c = p.c_cur[gb];
+                        if (p.out) p.out[o] = (int16_t)(256 * c + idx - 32768);
+                        p.c_prev[gb] = (uint8_t)c;
+                        p.f_prev[gb] = (uint8_t)idx;
+                    }
+                }
+            }
+            if (!bar.sync((int)s, head ? 8 : 4)) return;
+        }
+        float *t = hc; hc = hn; hn = t;
+    }
+
+    if (p.h_out) for (int i = gtid; i < B * H; i += nthreads) p.h_out[i] = __ldcg(hc + i);
+    for (int i = gtid; i < B; i += nthreads) {
+        if (p.c_st_out) p.c_st_out[i] = __ldcg(p.c_prev + i);
+        if (p.f_st_out) p.f_st_out[i] = __ldcg(p.f_prev + i);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Prologue: g[b][k][row] = W_cond[row][:] . frame[b][k][:] + b_gate[row]   (the per-step
+// conditioning vector; one frame is held for `hop` samples).
+
+__global__ void cond_project_kernel(const float *__restrict__ cond, const float *__restrict__ W_condT,
+                                    const float *__restrict__ b_gate, float *__restrict__ g, int G, int D,
+                                    int n_frames)
+{
+    extern __shared__ float fr[];
+    const int k = blockIdx.y, b = blockIdx.z;
+    const float *f = cond + ((size_t)b * n_frames + k) * D;
+    for (int d = threadIdx.x; d < D; d += blockDim.x) fr[d] = f[d];
+    __syncthreads();
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= G) return;
+    float acc = 0.f;
+    for (int d = 0; d < D; ++d) acc = fmaf(W_condT[(size_t)d * G + row], fr[d], acc);
+    g[((size_t)b * n_frames + k) * G + row] = acc + (b_gate ? b_gate[row] : 0.f);
+}
+
+__global__ void cond_bias_only_kernel(const float *__restrict__ b_gate, float *__restrict__ g, int G, int batch)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < G * batch) g[i] = b_gate ? b_gate[i % G] : 0.f;
+}
+
+int cond_project(wrnn_model *m, const float *cond, int batch, int n_frames, cudaStream_t s)
+{
+    const int G = 3 * m->H;
+    if (m->cond_dim == 0) {
+        cond_bias_only_kernel<<<(G * batch + 255) / 256, 256, 0, s>>>(m->b_gate, m->g, G, batch);
+    } else {
+        dim3 grid((G + 255) / 256, n_frames, batch);
+        cond_project_kernel<<<grid, 256, m->cond_dim * sizeof(float), s>>>(cond, m->W_condT, m->b_gate, m->g, G,
+                                                                           m->cond_dim, n_frames);
+    }
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Subscale fold / unfold (Eq. 4): sub[s][i] = x[B i + s].
+
+__global__ void fold_kernel(const int16_t *__restrict__ src, int16_t *__restrict__ dst, long long n, int B, int unfold)
+{
+    const long long len = n / B;
+    for (long long o = blockIdx.x * (long long)blockDim.x + threadIdx.x; o < n; o += (long long)gridDim.x * blockDim.x) {
+        if (unfold) { const long long i = o / B; const int s = (int)(o % B); dst[o] = src[(long long)s * len + i]; }
+        else        { const int s = (int)(o / len); const long long i = o % len; dst[o] = src[(long long)B * i + s]; }
+    }
+}
+
+int fold_launch(const int16_t *x, long long n_total, int B, int16_t *sub, bool unfold, cudaStream_t s)
+{
+    if (n_total == 0) return WRNN_OK;
+    const int blocks = (int)((n_total + 255) / 256 > 1184 ? 1184 : (n_total + 255) / 256);
+    fold_kernel<<<blocks, 256, 0, s>>>(x, sub, n_total, B, unfold ? 1 : 0);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+
+static void *generic_kernel_ptr(int dtype, int tb)
+{
+    if (dtype == WRNN_F32) return tb == 1 ? (void *)generic_step_kernel<float, 1> : (void *)generic_step_kernel<float, 8>;
+    return tb == 1 ? (void *)generic_step_kernel<uint16_t, 1> : (void *)generic_step_kernel<uint16_t, 8>;
+}
+
+int generic_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem)
+{
+    (void)batch;
+    if (n_ctas) *n_ctas = m->n_sms;
+    if (n_threads) *n_threads = 512;
+    if (smem) *smem = 0;
+    return WRNN_OK;
+}
+
+int generic_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
+{
+    GenericParams p;
+    p.H = m->H; p.Hh = m->H / 2; p.G = 3 * m->H; p.batch = a.batch;
+    p.n_steps = a.n_steps; p.step0 = a.step0; p.stream0 = a.stream0; p.seed = a.seed;
+    p.n_frames = m->cond_dim ? a.n_frames : 1;
+    p.hop = m->cond_dim ? a.hop : 1;
+    p.row_stride = m->cond_dim ? a.row_stride : 0;
+    p.row_offset_mul = m->cond_dim ? a.row_offset_mul : 0;
+    p.R = m->R; p.O1 = m->O1; p.O2 = m->O2; p.O3 = m->O3; p.O4 = m->O4;
+    p.I = m->I; p.b1 = m->b1; p.b2 = m->b2; p.b3 = m->b3; p.b4 = m->b4; p.g = m->g;
+    p.h0 = m->hbuf[0]; p.h1 = m->hbuf[1]; p.a_fine = m->a_fine; p.q = m->q; p.logits = m->logits;
+    p.c_cur = m->c_cur; p.c_prev = m->c_prev; p.f_prev = m->f_prev;
+    p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in;
+    p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
+    p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
+    p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
+    p.bar = m->bar; p.status = m->status;
+    p.limit_ns = 2000000000ull;
+
+    if (cudaMemsetAsync(m->bar, 0, sizeof(unsigned long long), s) != cudaSuccess) return WRNN_ERR_CUDA;
+    if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
+    void *fn = generic_kernel_ptr(m->dtype, a.batch == 1 ? 1 : 8);
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, 512, 0) != cudaSuccess || per_sm < 1) {
+        m->err = "generic kernel does not fit one CTA per SM";
+        return WRNN_ERR_UNSUPPORTED;
+    }
+    void *args[] = {(void *)&p};
+    const cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(m->n_sms), dim3(512), args, 0, s);
+    if (e != cudaSuccess) {
+        m->err = std::string("cooperative launch failed: ") + cudaGetErrorString(e);
+        return WRNN_ERR_CUDA;
+    }
+    ++g_launches;
+    return WRNN_OK;
+}
+
+}  // namespace wrnn

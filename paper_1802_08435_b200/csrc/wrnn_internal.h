@@ -1,0 +1,109 @@
+// Host-side structures shared by the translation units of libwrnn.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <string>
+#include <vector>
+
+#include "../../include/wrnn.h"
+#include "wrnn_device.cuh"
+
+namespace wrnn {
+
+// A matrix stored as compressed block rows of 4x4 blocks (Section 3.2).  A dense matrix is
+// the same structure with every block present.  vals holds nnz blocks of 16 weights each,
+// block-row-major inside a block (vals[i][4 r + c] = W[4 br + r][4 bc + c]), in the model's
+// storage type (fp32 or bf16).
+struct BsrDev {
+    int rows4 = 0, cols4 = 0, nnz = 0;
+    int *row_ptr = nullptr;        // [rows4 + 1]
+    uint16_t *col = nullptr;       // [nnz] block column
+    void *vals = nullptr;          // [nnz][16]
+};
+
+// Host image of the same thing (after masking and rounding), kept for the packers of the
+// specialised kernels.
+struct BsrHost {
+    int rows4 = 0, cols4 = 0;
+    std::vector<int> row_ptr;
+    std::vector<uint16_t> col;
+    std::vector<float> vals;       // fp32 values (already rounded to the storage type)
+};
+
+// Everything one stepping call needs besides the model (device pointers).
+struct StepArgs {
+    const float *cond;       // [batch][n_frames][cond_dim] (unused by the step kernels: g is projected)
+    int n_frames, hop, row_stride, row_offset_mul;
+    long long n_steps;
+    int batch;
+    unsigned long long seed;
+    long long step0;
+    unsigned stream0;
+    const float *h_in;  float *h_out;            // may be null
+    const uint8_t *c_in, *f_in; uint8_t *c_st_out, *f_st_out;
+    const uint8_t *c_forced, *f_forced;          // [batch][n_steps] or null
+    uint8_t *c_out, *f_out;                      // [batch][n_steps] or null
+    int16_t *out;                                // [batch][n_steps] or null
+    float *dbg_gates, *dbg_h, *dbg_logits;       // or null
+};
+
+struct ResidentPack;   // packed weights of the shared-memory-resident kernels (opaque here)
+
+}  // namespace wrnn
+
+struct wrnn_model {
+    int H = 0, cond_dim = 0, dtype = 0, kernel = 0, max_batch = 0;
+    int device = 0, n_sms = 0;
+    bool sparse = false;
+
+    // generic format
+    wrnn::BsrDev R, O1, O2, O3, O4;
+    float *I = nullptr;            // [3H][3] fp32 (values rounded to storage type; masked column zeroed)
+    float *b_gate = nullptr, *b1 = nullptr, *b2 = nullptr, *b3 = nullptr, *b4 = nullptr;
+    float *W_condT = nullptr;      // [cond_dim][3H] fp32 (rounded values), transposed for coalescing
+    int64_t weight_bytes = 0;      // packed bytes read per step (values + indices + row pointers)
+
+    // per-call scratch owned by the model
+    float *g = nullptr;            // projected conditioning [batch][n_frames][3H]
+    size_t g_cap = 0;              // floats
+    float *hbuf[2] = {nullptr, nullptr};   // [max_batch][H]
+    float *a_fine = nullptr;       // [max_batch][3][H/2]  R h of the fine rows, kept across the coarse head
+    float *q = nullptr;            // [max_batch][H/2]
+    float *logits = nullptr;       // [max_batch][256]
+    uint8_t *c_cur = nullptr, *c_prev = nullptr, *f_prev = nullptr;   // [max_batch]
+    unsigned long long *bar = nullptr;     // grid barrier counter
+    wrnn::DevStatus *status = nullptr;     // device status word
+    // host staging for wrnn_sample_host
+    float *stage_cond = nullptr; size_t stage_cond_cap = 0;
+    int16_t *stage_out = nullptr; size_t stage_out_cap = 0;
+
+    wrnn::ResidentPack *resident = nullptr;
+
+    // host images for packers
+    wrnn::BsrHost hR, hO1, hO2, hO3, hO4;
+    std::vector<float> hI, hb_gate, hb1, hb2, hb3, hb4;
+
+    std::string err;
+};
+
+namespace wrnn {
+
+extern std::atomic<long long> g_launches;
+
+// wrnn_generic.cu
+int generic_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem);
+int generic_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);   // returns wrnn_status
+int cond_project(wrnn_model *m, const float *cond, int batch, int n_frames, cudaStream_t s);
+int fold_launch(const int16_t *x, long long n_total, int B, int16_t *sub, bool unfold, cudaStream_t s);
+
+// wrnn_resident.cu
+int resident_supported(const wrnn_model *m, int batch, std::string *why);
+int resident_prepare(wrnn_model *m);                                  // pack + upload at create
+void resident_destroy(wrnn_model *m);
+int resident_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem,
+                         int64_t *weight_bytes);
+int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
+
+}  // namespace wrnn

@@ -1,0 +1,298 @@
+#!/usr/bin/env python
+"""Benchmark of the WaveRNN sampling path on B200.
+
+One "step" = one pass of the whole hot path over one batch of synthetic input: one
+wrnn_sample call that generates `n_steps` 16-bit samples for every stream row of the
+workload (conditioning projection, recurrent product, gates, dual softmax, draws).
+Default workload: dense H = 896, bf16 weights, batch 1, 24,000 samples (1 s of audio).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload I] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is audio samples per second with inputs resident
+on the device; `e2e` is the same through the host-buffer entry point (host->device copy of
+the conditioning frames and device->host copy of the samples inside the timed region).
+`--impl reference` times the CPU oracle (a deliberately plain program) on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1802_08435_b200 import synth  # noqa: E402
+
+METRIC = "audio samples/sec"
+UNIT = "samples/s"
+SMEM_PEAK_GBS = 148 * 128 * 1.965          # 148 SMs x 128 B/clk x 1.965 GHz = 37,228 GB/s (derived, not measured)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], bf16_tflops_sustained=d.get("bf16_tflops_sustained"),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def run_reference(args, wl):
+    """The CPU oracle as it stands, on the host cores; each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import wrnn_oracle as orc
+    w, masks, cond = synth.build_workload(wl)
+    om = orc.OracleModel(w, wl.dtype, masks)
+    cores = os.cpu_count() or 1
+    threads = 1 if wl.batch == 1 else min(cores, wl.batch)
+    # about 2-3 s of CPU work per step
+    per_row_step_ms = 2.3 * (wl.H / 896.0) ** 2
+    n_steps = max(16, min(wl.n_steps, int(2500.0 * threads / (per_row_step_ms * wl.batch))))
+    n_steps = min(n_steps, (wl.n_frames * synth.HOP) // max(1, wl.row_stride) - 1)
+    kw = dict(hop=synth.HOP, row_stride=wl.row_stride, row_offset_mul=wl.row_offset_mul, threads=threads)
+    for _ in range(max(0, min(args.warmup, 1))):
+        om.run(cond, min(n_steps, 64), wl.batch, synth.SEED_SAMPLING, **kw)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        om.run(cond, n_steps, wl.batch, synth.SEED_SAMPLING, **kw)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = n_steps * wl.batch / dt
+    sample = "first %d of %d steps x %d rows of %s per step" % (n_steps, wl.n_steps, wl.batch, wl.name)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "H": wl.H, "batch": wl.batch, "n_steps": wl.n_steps, "weights": wl.dtype,
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "x_realtime_24khz": value / 24000.0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def cpu_baseline(wl, budget_s=12.0):
+    from oracle import wrnn_oracle as orc
+    w, masks, cond = synth.build_workload(wl)
+    om = orc.OracleModel(w, wl.dtype, masks)
+    cores = os.cpu_count() or 1
+    threads = 1 if wl.batch == 1 else min(cores, wl.batch)
+    per_row_step_ms = 2.3 * (wl.H / 896.0) ** 2
+    n_steps = max(16, min(wl.n_steps, int(budget_s * 1e3 * threads / (per_row_step_ms * wl.batch))))
+    n_steps = min(n_steps, (wl.n_frames * synth.HOP) // max(1, wl.row_stride) - 1)
+    t0 = time.perf_counter()
+    om.run(cond, n_steps, wl.batch, synth.SEED_SAMPLING, hop=synth.HOP, row_stride=wl.row_stride,
+           row_offset_mul=wl.row_offset_mul, threads=threads)
+    dt = time.perf_counter() - t0
+    return {"value": n_steps * wl.batch / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "first %d of %d steps x %d rows of %s, once" % (n_steps, wl.n_steps, wl.batch, wl.name)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", type=int, default=1, help="index into the workload list (default 1: dense 896 bf16, batch 1, 24000)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--n-steps", type=int, default=None, help="override samples per call (profiling of a short case)")
+    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "resident"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    wl = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_1802_08435_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    n_steps = wl.n_steps if args.n_steps is None else args.n_steps
+    w, masks, cond_np = synth.build_workload(wl)
+    kern = {"auto": B.WRNN_KERNEL_AUTO, "generic": B.WRNN_KERNEL_GENERIC, "resident": B.WRNN_KERNEL_RESIDENT}[args.kernel]
+    model = B.wrnn_create(w, wl.dtype, masks, max_batch=wl.batch, kernel=kern)
+    info = B.wrnn_launch_info(model, wl.batch)
+    cond = torch.from_numpy(cond_np).to(dev)
+    out = torch.zeros((wl.batch, n_steps), dtype=torch.int16, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # > 126 MB L2
+    # rows of different ranks are different streams of the same workload (replicas; no collective on the path)
+    kw = dict(hop=synth.HOP, row_stride=wl.row_stride, row_offset_mul=wl.row_offset_mul, stream0=0)
+    seed = synth.SEED_SAMPLING + rank
+
+    def one():
+        B.wrnn_sample(model, cond, n_steps, wl.batch, seed, out, **kw)
+
+    for _ in range(max(args.warmup, 3)):
+        one()
+    torch.cuda.synchronize()
+    assert B.wrnn_poll_status(model) == 0, B.wrnn_last_error(model)
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = B.wrnn_launch_count()
+    evs = []
+    for _ in range(args.steps):
+        flush.fill_(1)                                                # L2 flush between timed iterations
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        one()
+        e1.record()
+        evs.append((e0, e1))
+    torch.cuda.synchronize()
+    launches = B.wrnn_launch_count() - launches0
+    if world > 1:
+        dist.barrier()
+    total_ms = sum(a.elapsed_time(b) for a, b in evs)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    clocks = sampler.stop() if rank == 0 else None
+    assert B.wrnn_poll_status(model) == 0, B.wrnn_last_error(model)
+
+    ms_per_step = total_ms / args.steps
+    samples_per_call = n_steps * wl.batch
+    value = world * samples_per_call / (ms_per_step * 1e-3)
+
+    # end to end through the host-buffer entry point (pinned host memory)
+    e2e = None
+    if not args.no_e2e:
+        cond_pin = torch.from_numpy(cond_np).pin_memory()
+        out_pin = torch.zeros((wl.batch, n_steps), dtype=torch.int16).pin_memory()
+        for _ in range(2):
+            B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
+        dt = (time.perf_counter() - t0) / args.steps
+        if world > 1:
+            t = torch.tensor([dt], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        assert np.array_equal(out_pin.numpy(), out.cpu().numpy()), "host-buffer path disagrees with the device path"
+        e2e = {"value": world * samples_per_call / dt, "unit": UNIT, "h2d_bytes_per_step": int(cond_np.nbytes),
+               "d2h_bytes_per_step": int(out_pin.numel() * 2)}
+
+    if rank == 0:
+        peaks = measured_peaks()
+        us_per_sample_step = ms_per_step * 1e3 / n_steps
+        wbytes = info["weight_bytes_per_step"]
+        if wl.batch >= 64:
+            # dense contraction: algorithmic flops of R, O1..O4 products per lock-step
+            H, Hh = wl.H, wl.H // 2
+            flops = 2.0 * wl.batch * (3 * H * H + 2 * Hh * Hh + 2 * 256 * Hh)
+            ach = flops * n_steps / (ms_per_step * 1e-3) / 1e12
+            roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None, "peak_source": peaks["source"] + " sustained"}
+        elif wl.sparsity is not None:
+            ach = wbytes * n_steps / (ms_per_step * 1e-3) / 1e9
+            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                    "traffic": None, "peak_source": peaks["source"], "bytes_per_step": wbytes,
+                    "note": "nonzero-block bytes per step over the HBM copy bandwidth"}
+        else:
+            ach = wbytes * n_steps / (ms_per_step * 1e-3) / 1e9
+            roof = {"bound": "smem", "achieved": ach, "peak": SMEM_PEAK_GBS, "unit": "GB/s", "frac": ach / SMEM_PEAK_GBS,
+                    "traffic": None, "peak_source": "derived: 148 SMs x 128 B/clk x 1.965 GHz", "bytes_per_step": wbytes,
+                    "note": "resident weight bytes read per step over aggregate shared-memory bandwidth; the step is "
+                            "latency-bound by two machine-wide exchanges, see DESIGN.md"}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "H": wl.H, "batch": wl.batch, "n_steps": n_steps, "weights": wl.dtype,
+                       "sparsity": wl.sparsity, "l2": "flushed between timed iterations (256 MiB fill)",
+                       "kernel": {1: "generic", 2: "resident"}[info["kernel"]], "n_ctas": info["n_ctas"],
+                       "threads_per_cta": info["n_threads"], "smem_bytes_per_cta": info["smem_bytes"],
+                       "multi_gpu": "replicas only"},
+            "us_per_sample_step": us_per_sample_step, "x_realtime_24khz": value / world / wl.batch / 24000.0 * wl.batch,
+            "x_realtime_24khz_per_stream": samples_per_call / wl.batch / (ms_per_step * 1e-3) / 24000.0 * (wl.subscale_B or 1),
+            "paper_context": "4x real time (96,000 samples/s) on an Nvidia P100 (Section 2.1); not the target",
+            "gpu_launches": int(launches), "clocks": clocks, "roofline": roof, "e2e": e2e,
+        }
+        if not args.no_cpu_baseline and world == 1:
+            line["cpu_baseline"] = cpu_baseline(wl)
+        print(json.dumps(line), flush=True)
+    B.wrnn_destroy(model)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -190,6 +190,21 @@ const char *wrnn_last_error(wrnn_model *m);
 int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_ctas,
                      int32_t *n_threads, int64_t *weight_bytes_per_step, int32_t *smem_bytes);
 
+/* Diagnostic of the resident single-stream kernel (Section 2.1: after the persistent kernel the
+ * remaining overhead is the synchronisation between multiprocessors): SM-clock cycles that warp 0 of
+ * CTA 0 spent in each phase of a step, summed over the last finished call on this model (HOST
+ * out16[16]).  A step has a fine half (entries 0..5, 12, 14) and a coarse half (6..11, 13, 15):
+ *   0 / 6   wait for the input half of the state from the whole chip (L2 exchange)
+ *   12 / 13 hidden-layer and recurrent partial products + CTA barrier
+ *   1 / 7   hidden-layer finish and send to the cluster
+ *   2 / 8   wait for the cluster's hidden layer + CTA barrier
+ *   14 / 15 logits partial products + CTA barrier
+ *   3 / 9   logits finish and send to the cluster
+ *   4 / 10  wait for the cluster's logits
+ *   5 / 11  softmax draw, gates of the other half, publish
+ * Synchronous. */
+int wrnn_phase_cycles(wrnn_model *m, int64_t *out16);
+
 /* Kernels launched by this library in this process since load (all models). */
 int64_t wrnn_launch_count(void);
 

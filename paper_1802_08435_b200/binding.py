@@ -24,7 +24,7 @@ _STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "NOMEM", "CUDA", "TIMEOUT"]
 EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
-    "wrnn_launch_count",
+    "wrnn_launch_count", "wrnn_phase_cycles",
 ]
 
 
@@ -79,6 +79,7 @@ def lib():
         L.wrnn_last_error.argtypes = [vp]
         L.wrnn_last_error.restype = C.c_char_p
         L.wrnn_launch_info.argtypes = [vp, i32] + [vp] * 5
+        L.wrnn_phase_cycles.argtypes = [vp, vp]
         L.wrnn_launch_count.argtypes = []
         L.wrnn_launch_count.restype = i64
         _lib = L
@@ -221,3 +222,10 @@ def wrnn_launch_info(model, batch: int = 1) -> dict:
 
 def wrnn_launch_count() -> int:
     return lib().wrnn_launch_count()
+
+
+def wrnn_phase_cycles(model):
+    """SM-clock cycles CTA 0 spent per phase of the resident kernel over the last call (list of 12)."""
+    buf = (C.c_int64 * 16)()
+    _check(lib().wrnn_phase_cycles(model, buf), model)
+    return list(buf)

@@ -396,4 +396,11 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
 
 int64_t wrnn_launch_count(void) { return g_launches.load(); }
 
+int wrnn_phase_cycles(wrnn_model *m, int64_t *out16)
+{
+    if (!m || !out16) return WRNN_ERR_INVALID_ARG;
+    static_assert(sizeof(long long) == sizeof(int64_t), "");
+    return resident_phase_cycles(m, reinterpret_cast<long long *>(out16));
+}
+
 }  // extern "C"

@@ -118,6 +118,53 @@ __device__ __forceinline__ int warp_softmax_draw(const float (&l)[8], float u, i
     return pick == 256 ? 255 : pick;
 }
 
+// Latency-lean variant for the single-stream kernel, where this sits on the per-step critical path:
+// one integer redux for the max and for the pick instead of ten shuffles, exp through ex2.approx
+// (relative error about 2^-21 on arguments in [-88, 0], far inside the 1e-5 CDF margin that index
+// parity allows).  Same contract as warp_softmax_draw.
+__device__ __forceinline__ int float_order_key(float x)
+{
+    const int i = __float_as_int(x);
+    return i ^ ((i >> 31) & 0x7fffffff);          // signed-integer order == float order
+}
+__device__ __forceinline__ int warp_softmax_draw_fast(const float (&l)[8], float u, int lane)
+{
+    float m = l[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) m = fmaxf(m, l[i]);
+    const int km = __reduce_max_sync(FULL, float_order_key(m));
+    m = __int_as_float(km ^ ((km >> 31) & 0x7fffffff));
+    float w[8], s = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { w[i] = __expf(l[i] - m); s += w[i]; }
+    float inc = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float t = __shfl_up_sync(FULL, inc, o);
+        if (lane >= o) inc += t;
+    }
+    const float thr = u * __shfl_sync(FULL, inc, 31);
+    float run = inc - s;                 // exclusive prefix of this lane
+    int pick = 256;
+#pragma unroll
+    for (int i = 7; i >= 0; --i) {       // last assignment wins: the smallest qualifying index
+        float r = run;
+#pragma unroll
+        for (int j = 0; j <= i; ++j) r += w[j];
+        if (r > thr) pick = 8 * lane + i;
+    }
+    pick = __reduce_min_sync(FULL, pick);
+    return pick == 256 ? 255 : pick;
+}
+
+// sigmoid / tanh through ex2.approx and the fast reciprocal: absolute error about 1e-7 .. 3e-7.
+__device__ __forceinline__ float sigmoidf_fast(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
+__device__ __forceinline__ float tanhf_fast(float x)
+{
+    const float e = __expf(-2.0f * fabsf(x));
+    return copysignf(__fdividef(1.0f - e, 1.0f + e), x);
+}
+
 // ------------------------------------------------------------------ memory-order helpers
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long *p)
 {

@@ -105,5 +105,6 @@ void resident_destroy(wrnn_model *m);
 int resident_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem,
                          int64_t *weight_bytes);
 int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
+int resident_phase_cycles(const wrnn_model *m, long long *out16);
 
 }  // namespace wrnn

@@ -13,9 +13,15 @@
 // through distributed shared memory the same way.  The fine head of step t overlaps the recurrent
 // product of step t+1 (f_t is only needed by the coarse gates of t+1).
 //
-// Every wait is bounded; a CTA that gives up records where, raises the abort word and all CTAs
-// leave through the final cluster barrier.
+// Mat-vec products run on the tensor pipe as m16n8k16 bf16 MMAs: the weights sit in shared memory
+// in A-fragment order (one 16-byte load per lane per 16x16 tile), and the fp32 input vector is split
+// exactly into three bf16 vectors (hi + mid + lo) that occupy three of the eight B columns, so the
+// fp32 state is not rounded on its way in; accumulation is fp32.
+//
+// Every wait is bounded; a CTA that gives up records where and all CTAs leave through the final
+// cluster barrier.
 #include <cooperative_groups.h>
+#include <cuda_bf16.h>
 
 #include <algorithm>
 #include <cstring>
@@ -27,18 +33,19 @@ namespace cg = cooperative_groups;
 namespace wrnn {
 
 struct ResidentPack {
-    int NC = 0, CS = 0, NCTA = 0, UC = 0, HR = 0, LR = 0, K = 0, KC = 0, NW = 0;
+    int NC = 0, CS = 0, NCTA = 0, UC = 0, HR = 0, LR = 0, K = 0, NKT = 0, NMT = 0, NLT = 0, NW = 0, KSH = 0, KSL = 0;
     int n_rrows = 0;                 // 6 UC
-    size_t blob_bytes = 0;           // per CTA: bf16 weights then fp32 small parameters
+    size_t blob_bytes = 0;           // per CTA: bf16 weight fragments then fp32 small parameters
     size_t w_bytes = 0;              // bf16 part of the blob
     uint8_t *d_blob = nullptr;       // [NCTA][blob_bytes]
     unsigned long long *d_slots = nullptr;   // [2 halves][2 parities][K] (value, tag)
     int smem_bytes = 0;
     int64_t weight_bytes_per_step = 0;
+    long long *d_prof = nullptr;     // [16] phase cycle totals of the last call (diagnostic)
 };
 
 struct ResidentParams {
-    int H, K, KC, UC, HR, LR, CS, n_rrows;
+    int H, K, NKT, NMT, NLT, UC, HR, LR, CS, n_rrows;
     long long n_steps, step0;
     unsigned stream0;
     unsigned long long seed;
@@ -54,6 +61,7 @@ struct ResidentParams {
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
+    long long *prof;                         // optional [16] per-phase cycle totals of CTA 0, warp 0
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -94,7 +102,7 @@ struct Waiter {
     unsigned long long limit_ns;
 
     // called every few thousand failed polls; true = give up (somebody else already did, or time ran out)
-    __device__ __forceinline__ bool expired(unsigned long long &t0, int step, int phase)
+    __device__ __noinline__ bool expired(unsigned long long &t0, int step, int phase)
     {
         if (ld_relaxed_s32(&status->code) != DEV_OK) return true;
         const unsigned long long now = globaltimer_ns();
@@ -109,76 +117,108 @@ struct Waiter {
     }
 };
 
-// Lane's share of an input vector of KC 8-float chunks: chunks lane, lane + 32, ...
-template <int CPL>
-__device__ __forceinline__ void load_vec(const float *vec, int KC, int lane, float (&hv)[CPL * 8])
+// Split image of an fp32 input vector x of K elements, as the B operand of the MMAs wants it:
+// x = p0 + p1 + p2 exactly (three bf16 parts); the image is [K/16 k-tiles][4 t][4 parts][4 bf16] where
+// the four bf16 of (kt, t, part) are elements 16 kt + {2t, 2t+1, 2t+8, 2t+9} of that part -- exactly the
+// B fragment (b0, b1) of lane (group = part, t) -- and part 3 is zero.  One 8-byte load per lane per
+// k-tile, 128 distinct bytes per warp (lanes of groups 4..7 re-read groups 0..3), no bank conflicts.
+__host__ __device__ __forceinline__ int split_pos(int i, int part)
 {
+    const int c = i & 15, kt = i >> 4;
+    const int t = (c & 7) >> 1, j = c & 1, hi = c >> 3;
+    return (((kt * 4 + t) * 4 + part) << 2) + 2 * hi + j;
+}
+
+__device__ __forceinline__ void store_split(__nv_bfloat16 *split, int i, float x)
+{
+    const __nv_bfloat16 b0 = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(b0);
+    const __nv_bfloat16 b1 = __float2bfloat16_rn(r1);
+    const float r2 = r1 - __bfloat162float(b1);
+    const __nv_bfloat16 b2 = __float2bfloat16_rn(r2);
+    const int pos = split_pos(i, 0);
+    split[pos] = b0; split[pos + 4] = b1; split[pos + 8] = b2;
+}
+
+// NK consecutive k-tiles (from kt0) of one 16-row tile of a fragment-packed bf16 matrix times a split
+// vector.  A: [NKT][32 lanes] uint4.  Straight-line code: all fragment loads are issued before the first
+// MMA and the MMAs run back to back over four independent accumulator chains.  D columns 0,1,2 hold the
+// products with the three parts of the vector (column 3 is zero, columns 4..7 are repeats that nobody
+// reads).  On return the lanes with t = 0 hold the partial totals of rows g (lo) and g + 8 (hi).
+template <int NK>
+__device__ __forceinline__ void mma_partial(const uint4 *A, int kt0, const __nv_bfloat16 *split, int lane, float &lo, float &hi)
+{
+    const int g = lane >> 2, t = lane & 3;
+    const uint2 *bsrc = reinterpret_cast<const uint2 *>(split) + (kt0 * 4 + t) * 4 + (g & 3);
+    const uint4 *a = A + (size_t)kt0 * 32 + lane;
+    uint4 av[NK];
+    uint2 bv[NK];
 #pragma unroll
-    for (int i = 0; i < CPL; ++i) {
-        const int ch = lane + 32 * i;
-        if (ch < KC) {
-            const float4 a = *reinterpret_cast<const float4 *>(vec + 8 * ch);
-            const float4 b = *reinterpret_cast<const float4 *>(vec + 8 * ch + 4);
-            hv[8 * i] = a.x; hv[8 * i + 1] = a.y; hv[8 * i + 2] = a.z; hv[8 * i + 3] = a.w;
-            hv[8 * i + 4] = b.x; hv[8 * i + 5] = b.y; hv[8 * i + 6] = b.z; hv[8 * i + 7] = b.w;
-        } else {
+    for (int i = 0; i < NK; ++i) { av[i] = a[i * 32]; bv[i] = bsrc[16 * i]; }
+    float acc[4][4];
 #pragma unroll
-            for (int k = 0; k < 8; ++k) hv[8 * i + k] = 0.f;
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[c][i] = 0.f;
+#pragma unroll
+    for (int i = 0; i < NK; ++i) {
+        float *c = acc[i & 3];
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                     : "r"(av[i].x), "r"(av[i].y), "r"(av[i].z), "r"(av[i].w), "r"(bv[i].x), "r"(bv[i].y));
+    }
+    float s_lo = (acc[0][0] + acc[1][0]) + (acc[2][0] + acc[3][0]) + ((acc[0][1] + acc[1][1]) + (acc[2][1] + acc[3][1]));
+    float s_hi = (acc[0][2] + acc[1][2]) + (acc[2][2] + acc[3][2]) + ((acc[0][3] + acc[1][3]) + (acc[2][3] + acc[3][3]));
+    s_lo += __shfl_xor_sync(FULL, s_lo, 1);      // t = 0 (columns 0,1) + t = 1 (columns 2,3)
+    s_hi += __shfl_xor_sync(FULL, s_hi, 1);
+    lo = s_lo; hi = s_hi;
+}
+
+// Send the 16 values of a tile (sc[0..15], rows row0..row0+15 of a cluster-wide vector laid out as
+// (value, tag) pairs) to every CTA of the cluster; only rows below row_limit are sent.
+__device__ __forceinline__ void send_tile(const float *sc, uint4 *buf_base, int row0, int row_limit, int CS, int lane, unsigned tag)
+{
+    const int peer = lane & 7, ps = lane >> 3;
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const int pair = ps + 4 * k;
+        if (peer < CS && row0 + 2 * pair < row_limit) {
+            const unsigned a = map_to_rank(smem_addr(buf_base + (row0 >> 1) + pair), peer);
+            st_cluster_ll(a, sc[2 * pair], sc[2 * pair + 1], tag);
         }
     }
 }
 
-// Four consecutive bf16 rows (KC 16-byte chunks each, contiguous in shared memory) times the
-// lane's vector share; returns with lane l holding the total of row (l & 3).
-template <int CPL>
-__device__ __forceinline__ float dot4(const uint4 *w, int KC, int lane, const float (&hv)[CPL * 8])
-{
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int i = 0; i < CPL; ++i) {
-        const int ch = lane + 32 * i;
-        if (ch < KC) {
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const uint4 v = w[r * KC + ch];
-                float s = acc[r];
-                s = fmaf(bf16lo(v.x), hv[8 * i], s);     s = fmaf(bf16hi(v.x), hv[8 * i + 1], s);
-                s = fmaf(bf16lo(v.y), hv[8 * i + 2], s); s = fmaf(bf16hi(v.y), hv[8 * i + 3], s);
-                s = fmaf(bf16lo(v.z), hv[8 * i + 4], s); s = fmaf(bf16hi(v.z), hv[8 * i + 5], s);
-                s = fmaf(bf16lo(v.w), hv[8 * i + 6], s); s = fmaf(bf16hi(v.w), hv[8 * i + 7], s);
-                acc[r] = s;
-            }
-        }
-    }
-    return warp_reduce_scatter<4>(acc, lane);
-}
-
-template <int CPL>
-__global__ void __launch_bounds__(768, 1) resident_dense_kernel(const ResidentParams p)
+// KSH / KSL: K-splits per hidden / logits tile; NKH / NKL: k-tiles per split (KSH * NKH = KSL * NKL = K / 16).
+template <int KSH, int NKH, int KSL, int NKL>
+__global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const int cta = blockIdx.x;                       // global CTA index = owner index of state units
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int K = p.K, KC = p.KC, UC = p.UC, HR = p.HR, LR = p.LR, CS = p.CS, H = p.H;
+    const int K = p.K, NKT = p.NKT, NMT = p.NMT, NLT = p.NLT, UC = p.UC, HR = p.HR, LR = p.LR, CS = p.CS, H = p.H;
     const int NR = p.n_rrows;                          // 6 UC
 
     // ---- shared memory carve-up (must match resident_smem_bytes)
-    const uint4 *wRA = reinterpret_cast<const uint4 *>(smem);                 // [NR][KC]  R rows x coarse columns
-    const uint4 *wRB = wRA + (size_t)NR * KC;                                  // [NR][KC]  R rows x fine columns
-    const uint4 *wO1 = wRB + (size_t)NR * KC;                                  // [HR][KC]
-    const uint4 *wO3 = wO1 + (size_t)HR * KC;
-    const uint4 *wO2 = wO3 + (size_t)HR * KC;                                  // [LR][KC]
-    const uint4 *wO4 = wO2 + (size_t)LR * KC;
+    const size_t tile_u4 = (size_t)NKT * 32;                                   // uint4 per 16-row tile
+    const uint4 *wMA = reinterpret_cast<const uint4 *>(smem);                  // [NMT] tiles: rows [O1 ; R x coarse cols]
+    const uint4 *wMB = wMA + (size_t)NMT * tile_u4;                            // [NMT] tiles: rows [O3 ; R x fine cols]
+    const uint4 *wO2 = wMB + (size_t)NMT * tile_u4;                            // [NLT] tiles
+    const uint4 *wO4 = wO2 + (size_t)NLT * tile_u4;
     const float *sI = reinterpret_cast<const float *>(smem + p.w_bytes);       // [NR][3]
     const float *sb1 = sI + NR * 3, *sb3 = sb1 + HR, *sb2 = sb3 + HR, *sb4 = sb2 + LR;
-    float *vecC = reinterpret_cast<float *>(smem + p.blob_bytes);              // [K] y_c
+    float *vecC = reinterpret_cast<float *>(smem + p.blob_bytes);              // [K] y_c (fp32, natural order)
     float *vecF = vecC + K;                                                    // [K] y_f
-    float *qvec = vecF + K;                                                    // [K] hidden layer of the head
-    float *a_part = qvec + K;                                                  // [NR] R[:, :Hh] y_c
+    float *a_part = vecF + K;                                                  // [NR] R[:, :Hh] y_c
     float *a_full = a_part + NR;                                               // [NR] R h
-    uint4 *qbuf = reinterpret_cast<uint4 *>(a_full + NR + ((2 * NR) % 4 ? 4 - (2 * NR) % 4 : 0));   // [2][K/2]
+    float *part = a_full + NR + ((2 * NR) % 4 ? 4 - (2 * NR) % 4 : 0);         // [tiles x K-splits][16] partial sums
+    float *scratch = part + 384;                                               // [24 warps][16]
+    __nv_bfloat16 *splC = reinterpret_cast<__nv_bfloat16 *>(scratch + 384);    // split images, 4 K bf16 each
+    __nv_bfloat16 *splF = splC + 4 * K;
+    __nv_bfloat16 *splQ = splF + 4 * K;
+    uint4 *qbuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                    // [2][K/2]
     uint4 *lbuf = qbuf + K;                                                    // [2][128]
 
     // ---- one-time load of this CTA's weights
@@ -187,9 +227,13 @@ __global__ void __launch_bounds__(768, 1) resident_dense_kernel(const ResidentPa
         uint4 *dst = reinterpret_cast<uint4 *>(smem);
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
         for (int i = tid; i < K + 256; i += blockDim.x) qbuf[i] = make_uint4(0, 0, 0, 0);   // qbuf and lbuf are adjacent
+        for (int i = tid; i < 12 * K / 8; i += blockDim.x) reinterpret_cast<uint4 *>(splC)[i] = make_uint4(0, 0, 0, 0);
+        __syncthreads();
         for (int i = tid; i < K; i += blockDim.x) {
-            vecC[i] = p.h_in ? p.h_in[i] : 0.f;
-            vecF[i] = p.h_in ? p.h_in[K + i] : 0.f;
+            const float c = p.h_in ? p.h_in[i] : 0.f, f = p.h_in ? p.h_in[K + i] : 0.f;
+            vecC[i] = c; vecF[i] = f;
+            store_split(splC, i, c);
+            store_split(splF, i, f);
         }
     }
     __syncthreads();
@@ -197,251 +241,228 @@ __global__ void __launch_bounds__(768, 1) resident_dense_kernel(const ResidentPa
 
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;      // this thread gave up on a wait; made CTA-uniform by __syncthreads_or
-    const int n_head_warps = HR / 4, n_r_warps = NR / 4, n_logit_warps = LR / 4;
-    const bool is_head_warp = warp < n_head_warps;
-    const bool is_r_warp = warp >= n_head_warps && warp < n_head_warps + n_r_warps;
-    const int r_task = warp - n_head_warps;
+    // optional phase timing (CTA 0, warp 0): cycles spent up to each stamp since the previous one
+    const bool prof_on = p.prof != nullptr && cta == 0 && warp == 0;
+    __shared__ long long s_prof[16];
+    if (tid < 16) s_prof[tid] = 0;
+    __syncthreads();
+    long long prof_t = clock64();
+#define STAMP(i) do { if (prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
+
     const bool writer = (cta == 0);
+    float *sc = scratch + 16 * warp;
+    const int g4 = lane >> 2;
 
     // warp 0 keeps the stream's scalar state
     int c_prev = p.c_in ? p.c_in[0] : 128, f_prev = p.f_in ? p.f_in[0] : 0;
     float hC = 0.f, hF = 0.f;
     if (warp == 0 && lane < UC) { hC = vecC[cta * UC + lane]; hF = vecF[cta * UC + lane]; }
 
-    // prologue: a_part = R[:, :Hh] y_c(-1)
-    if (is_r_warp) {
-        float hv[CPL * 8];
-        load_vec<CPL>(vecC, KC, lane, hv);
-        const float t = dot4<CPL>(wRA + (size_t)(4 * r_task) * KC, KC, lane, hv);
-        if (lane < 4) a_part[4 * r_task + lane] = t;
+    // Fixed roles: in the hidden phase warp w takes K-split (w % KSH) of tile (w / KSH), in the logits
+    // phase K-split (w % KSL) of tile (w / KSL); each leaves 16 partial row sums in part[w].
+    const int h_tile = warp / KSH, h_kt0 = (warp % KSH) * NKH;
+    const int l_tile = warp / KSL, l_kt0 = (warp % KSL) * NKL;
+    const bool h_on = warp < NMT * KSH, l_on = warp < NLT * KSL;
+    const bool h_fin = warp < NMT, l_fin = warp < NLT;
+
+    // ---- prologue: the recurrent products of step 0 from the initial state, coarse gates of step 0
+    if (h_on) {
+        float lo, hi;
+        mma_partial<NKH>(wMA + (size_t)h_tile * tile_u4, h_kt0, splC, lane, lo, hi);
+        if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
+    }
+    __syncthreads();
+    if (h_fin && lane < 16 && 16 * warp + lane >= HR) {
+        float v = 0.f;
+#pragma unroll
+        for (int sp = 0; sp < KSH; ++sp) v += part[(warp * KSH + sp) * 16 + lane];
+        a_part[16 * warp + lane - HR] = v;
+    }
+    __syncthreads();
+    if (h_on) {
+        float lo, hi;
+        mma_partial<NKH>(wMB + (size_t)h_tile * tile_u4, h_kt0, splF, lane, lo, hi);
+        if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
+    }
+    __syncthreads();
+    if (h_fin && lane < 16 && 16 * warp + lane >= HR) {
+        float v = 0.f;
+#pragma unroll
+        for (int sp = 0; sp < KSH; ++sp) v += part[(warp * KSH + sp) * 16 + lane];
+        a_full[16 * warp + lane - HR] = a_part[16 * warp + lane - HR] + v;
     }
     __syncthreads();
 
-    unsigned hs = 0;            // cluster-exchange counter (one per head evaluation)
+    // Gates of Eq. 2 for this CTA's units of one half of the state, then publish them to the chip.
+    // half_g = 0: coarse units (c_s does not reach them: their I* column is zero), 1: fine units.
+    auto gates_and_publish = [&](int half_g, long long s, int drawn, const float (&gv)[3]) {
+        const int rb = half_g ? 3 * UC : 0;
+        const float x0 = scale8(c_prev), x1 = scale8(f_prev), x2 = half_g ? scale8(drawn) : 0.f;
+        const float *Iu = sI + 3 * (rb + lane), *Ir = sI + 3 * (rb + UC + lane), *Ie = sI + 3 * (rb + 2 * UC + lane);
+        const float pu = a_full[rb + lane] + fmaf(Iu[0], x0, fmaf(Iu[1], x1, fmaf(Iu[2], x2, gv[0])));
+        const float pr = a_full[rb + UC + lane] + fmaf(Ir[0], x0, fmaf(Ir[1], x1, fmaf(Ir[2], x2, gv[1])));
+        const float pe = fmaf(Ie[0], x0, fmaf(Ie[1], x1, fmaf(Ie[2], x2, gv[2])));
+        const float u = sigmoidf_fast(pu), r = sigmoidf_fast(pr);
+        const float e = tanhf_fast(fmaf(r, a_full[rb + 2 * UC + lane], pe));
+        const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
+        if (half_g) hF = hn; else hC = hn;
+        const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
+        st_relaxed_u64(p.slots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
+                       ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+        if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
+        if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
+    };
+    auto load_g = [&](int half_g, long long s, float (&gv)[3]) {
+        const long long fr = ((p.step0 + s) * p.row_stride + (long long)p.stream0 * p.row_offset_mul) / p.hop;
+        const float *g = p.g + (size_t)fr * 3 * H + (half_g ? K : 0) + cta * UC + lane;
+#pragma unroll
+        for (int gate = 0; gate < 3; ++gate) gv[gate] = __ldg(g + gate * H);
+    };
+    if (warp == 0 && lane < UC) {
+        float gv[3];
+        load_g(0, 0, gv);
+        gates_and_publish(0, 0, 0, gv);
+    }
+
+    // The step is two structurally identical halves (Fig. 1).  Half-step n = 2 s + 1 is the "coarse" half of
+    // step s (input y_c(s): coarse head -> c_s; R[:, :Hh] y_c(s) kept for step s+1; then the fine gates of
+    // step s); n = 2 s is the "fine" half (input y_f(s-1): fine head -> f_{s-1}; R[:, Hh:] y_f(s-1) completes
+    // R h_{s-1}; then the coarse gates of step s).  One loop body serves both so that the code stays small.
     const long long T = p.n_steps;
+#pragma unroll 1
+    for (long long n = 1; n <= 2 * T; ++n) {
+        const int half = (int)(n & 1);                 // 1: coarse half, 0: fine half
+        const long long s = n >> 1;
+        const bool last = n == 2 * T;                  // final fine half: draw f_{T-1} only
+        const unsigned tag = (unsigned)n, par = (unsigned)((n - 1) & 1);   // cluster-exchange tag / buffer of this half
+        const uint4 *M = half ? wMA : wMB, *L = half ? wO2 : wO4;
+        const float *bh = half ? sb1 : sb3, *bl = half ? sb2 : sb4;
+        float *vec = half ? vecC : vecF;
+        __nv_bfloat16 *spl = half ? splC : splF;
 
-    for (long long s = 0; s <= T; ++s) {
-        // conditioning rows of this CTA's units, fetched early (they do not depend on the chain)
-        float gC[3] = {0.f, 0.f, 0.f}, gF[3] = {0.f, 0.f, 0.f};
-        int cf_next = -1, ff_prev = -1;
+        // everything that does not depend on the chain is fetched / computed before the first wait
+        float gv[3] = {0.f, 0.f, 0.f}, u01 = 0.f;
+        int forced = -1;
         if (warp == 0) {
-            if (lane < UC && s < T) {
-                const long long fr = ((p.step0 + s) * p.row_stride + (long long)p.stream0 * p.row_offset_mul) / p.hop;
-                const float *g = p.g + (size_t)fr * 3 * H;
-#pragma unroll
-                for (int gate = 0; gate < 3; ++gate) {
-                    gC[gate] = __ldg(g + gate * H + cta * UC + lane);
-                    gF[gate] = __ldg(g + gate * H + K + cta * UC + lane);
-                }
-            }
-            if (p.c_forced && s < T) cf_next = p.c_forced[s];
-            if (p.f_forced && s > 0) ff_prev = p.f_forced[s - 1];
+            if (lane < UC && !last) load_g(half, s, gv);          // gates evaluated at the end of this half
+            if (half) { if (p.c_forced) forced = p.c_forced[s]; }
+            else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
+            u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
         }
 
-        // =================== fine half: head of step s-1 (draw f_{s-1}) + R[:, Hh:] y_f(s-1)
-        if (s > 0) {
-            const unsigned long long *slots = p.slots + (size_t)(2 + ((s - 1) & 1)) * K;
-            const unsigned tag = (unsigned)s;                 // y_f(s-1) carries tag s
-            for (int i = tid; i < K; i += blockDim.x) {
-                unsigned long long v, t0 = 0; unsigned n = 0;
-                while ((unsigned)((v = ld_relaxed_u64(slots + i)) >> 32) != tag)
-                    if ((++n & 4095u) == 0 && wt.expired(t0, (int)s, 1)) { my_bad = true; break; }
-                vecF[i] = __uint_as_float((unsigned)v);
-            }
-            if (__syncthreads_or(my_bad)) break;
-        }
-        if (is_head_warp && s > 0) {
-            float hv[CPL * 8];
-            load_vec<CPL>(vecF, KC, lane, hv);
-            const int r0 = 4 * warp;
-            const float t = dot4<CPL>(wO3 + (size_t)r0 * KC, KC, lane, hv);
-            const float q0 = fmaxf(__shfl_sync(FULL, t, 0) + sb3[r0], 0.f), q1 = fmaxf(__shfl_sync(FULL, t, 1) + sb3[r0 + 1], 0.f);
-            const float q2 = fmaxf(__shfl_sync(FULL, t, 2) + sb3[r0 + 2], 0.f), q3 = fmaxf(__shfl_sync(FULL, t, 3) + sb3[r0 + 3], 0.f);
-            if (lane < 2 * CS) {
-                const int peer = lane >> 1, pair = lane & 1;
-                const unsigned a = map_to_rank(smem_addr(qbuf + (size_t)(hs & 1) * (K / 2) + (rank * HR + r0) / 2 + pair), peer);
-                st_cluster_ll(a, pair ? q2 : q0, pair ? q3 : q1, hs + 1);
-            }
-        } else if (is_r_warp) {
-            float hv[CPL * 8];
-            load_vec<CPL>(vecF, KC, lane, hv);
-            const float t = dot4<CPL>(wRB + (size_t)(4 * r_task) * KC, KC, lane, hv);
-            if (lane < 4) a_full[4 * r_task + lane] = a_part[4 * r_task + lane] + t;
-        }
-        if (s > 0) {
-            for (int i = tid; i < K / 2; i += blockDim.x) {
-                const unsigned a = smem_addr(qbuf + (size_t)(hs & 1) * (K / 2) + i);
-                uint4 v; unsigned long long t0 = 0; unsigned n = 0;
-                while (true) {
-                    v = ld_shared_volatile_v4(a);
-                    if (v.y == hs + 1 && v.w == hs + 1) break;
-                    if ((++n & 4095u) == 0 && wt.expired(t0, (int)s, 2)) { my_bad = true; break; }
-                }
-                qvec[2 * i] = __uint_as_float(v.x); qvec[2 * i + 1] = __uint_as_float(v.z);
-            }
-        }
-        if (__syncthreads_or(my_bad)) break;
-        if (s > 0 && warp < n_logit_warps) {
-            float hv[CPL * 8];
-            load_vec<CPL>(qvec, KC, lane, hv);
-            const int r0 = 4 * warp;
-            const float t = dot4<CPL>(wO4 + (size_t)r0 * KC, KC, lane, hv);
-            const float l0 = __shfl_sync(FULL, t, 0) + sb4[r0], l1 = __shfl_sync(FULL, t, 1) + sb4[r0 + 1];
-            const float l2 = __shfl_sync(FULL, t, 2) + sb4[r0 + 2], l3 = __shfl_sync(FULL, t, 3) + sb4[r0 + 3];
-            if (lane < 2 * CS) {
-                const int peer = lane >> 1, pair = lane & 1;
-                const unsigned a = map_to_rank(smem_addr(lbuf + (size_t)(hs & 1) * 128 + (rank * LR + r0) / 2 + pair), peer);
-                st_cluster_ll(a, pair ? l2 : l0, pair ? l3 : l1, hs + 1);
-            }
-        }
-        if (warp == 0) {
-            if (s > 0) {
-                float l[8];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const unsigned a = smem_addr(lbuf + (size_t)(hs & 1) * 128 + 4 * lane + k);
-                    uint4 v; unsigned long long t0 = 0; unsigned n = 0;
-                    while (true) {
-                        v = ld_shared_volatile_v4(a);
-                        if (v.y == hs + 1 && v.w == hs + 1) break;
-                        if ((++n & 4095u) == 0 && wt.expired(t0, (int)s, 3)) { my_bad = true; break; }
-                    }
-                    l[2 * k] = __uint_as_float(v.x); l[2 * k + 1] = __uint_as_float(v.z);
-                }
-                my_bad = __any_sync(FULL, my_bad);
-                const float u = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + s - 1), 1u);
-                int f = warp_softmax_draw(l, u, lane);
-                if (writer) {
-                    if (p.dbg_logits) {
-                        float *d = p.dbg_logits + ((size_t)(s - 1) * 2 + 1) * 256 + 8 * lane;
-#pragma unroll
-                        for (int k = 0; k < 8; ++k) d[k] = l[k];
-                    }
-                    if (lane == 0 && p.f_out) p.f_out[s - 1] = (uint8_t)f;
-                }
-                if (ff_prev >= 0) f = ff_prev;
-                if (writer && lane == 0 && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + f - 32768);
-                f_prev = f;
-            }
-        }
-        if (s > 0) ++hs;
-        if (s == T) break;
-
-        // coarse gates of step s (Eq. 2; c_t does not reach these rows)
-        if (warp == 0 && lane < UC && !my_bad) {
-            const float x0 = scale8(c_prev), x1 = scale8(f_prev);
-            const float *Iu = sI + 3 * (0 * UC + lane), *Ir = sI + 3 * (1 * UC + lane), *Ie = sI + 3 * (2 * UC + lane);
-            const float pu = a_full[lane] + fmaf(Iu[0], x0, fmaf(Iu[1], x1, gC[0]));
-            const float pr = a_full[UC + lane] + fmaf(Ir[0], x0, fmaf(Ir[1], x1, gC[1]));
-            const float pe = fmaf(Ie[0], x0, fmaf(Ie[1], x1, gC[2]));
-            const float u = sigmoidf_acc(pu), r = sigmoidf_acc(pr);
-            const float e = tanhf(fmaf(r, a_full[2 * UC + lane], pe));
-            hC = fmaf(u, hC, (1.0f - u) * e);
-            const int j = cta * UC + lane;
-            st_relaxed_u64(p.slots + (size_t)(s & 1) * K + j, ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hC));
-            if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[j] = u; d[H + j] = r; d[2 * H + j] = e; }
-            if (p.dbg_h) p.dbg_h[(size_t)s * H + j] = hC;
-        }
-
-        // =================== coarse half: head of step s (draw c_s) + R[:, :Hh] y_c(s) for step s+1
+        // ---- 1. input half-vector from the whole chip (y_c(s) carries tag s+1; y_f(s-1) carries tag s)
         {
-            const unsigned long long *slots = p.slots + (size_t)(s & 1) * K;
-            const unsigned tag = (unsigned)(s + 1);
+            const unsigned long long *slots = p.slots + (size_t)(half ? (s & 1) : 2 + ((s - 1) & 1)) * K;
+            const unsigned ytag = (unsigned)(half ? s + 1 : s);
+#pragma unroll 1
             for (int i = tid; i < K; i += blockDim.x) {
-                unsigned long long v, t0 = 0; unsigned n = 0;
-                while ((unsigned)((v = ld_relaxed_u64(slots + i)) >> 32) != tag)
-                    if ((++n & 4095u) == 0 && wt.expired(t0, (int)s, 4)) { my_bad = true; break; }
-                vecC[i] = __uint_as_float((unsigned)v);
+                unsigned long long v, t0 = 0; unsigned cnt = 0;
+                while ((unsigned)((v = ld_relaxed_u64(slots + i)) >> 32) != ytag)
+                    if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+                const float x = __uint_as_float((unsigned)v);
+                vec[i] = x;
+                store_split(spl, i, x);
             }
             if (__syncthreads_or(my_bad)) break;
         }
-        if (is_head_warp) {
-            float hv[CPL * 8];
-            load_vec<CPL>(vecC, KC, lane, hv);
-            const int r0 = 4 * warp;
-            const float t = dot4<CPL>(wO1 + (size_t)r0 * KC, KC, lane, hv);
-            const float q0 = fmaxf(__shfl_sync(FULL, t, 0) + sb1[r0], 0.f), q1 = fmaxf(__shfl_sync(FULL, t, 1) + sb1[r0 + 1], 0.f);
-            const float q2 = fmaxf(__shfl_sync(FULL, t, 2) + sb1[r0 + 2], 0.f), q3 = fmaxf(__shfl_sync(FULL, t, 3) + sb1[r0 + 3], 0.f);
-            if (lane < 2 * CS) {
-                const int peer = lane >> 1, pair = lane & 1;
-                const unsigned a = map_to_rank(smem_addr(qbuf + (size_t)(hs & 1) * (K / 2) + (rank * HR + r0) / 2 + pair), peer);
-                st_cluster_ll(a, pair ? q2 : q0, pair ? q3 : q1, hs + 1);
-            }
-        } else if (is_r_warp) {
-            float hv[CPL * 8];
-            load_vec<CPL>(vecC, KC, lane, hv);
-            const float t = dot4<CPL>(wRA + (size_t)(4 * r_task) * KC, KC, lane, hv);
-            if (lane < 4) a_part[4 * r_task + lane] = t;
+        STAMP(0 + 6 * half);
+
+        // ---- 2. hidden layer of the head + this CTA's R rows against the same input
+        if (h_on) {
+            float lo, hi;
+            mma_partial<NKH>(M + (size_t)h_tile * tile_u4, h_kt0, spl, lane, lo, hi);
+            if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
         }
+        __syncthreads();
+        STAMP(12 + half);
+        if (h_fin) {
+            if (lane < 16) {
+                float v = 0.f;
+#pragma unroll
+                for (int sp = 0; sp < KSH; ++sp) v += part[(warp * KSH + sp) * 16 + lane];
+                const int row = 16 * warp + lane;
+                if (row < HR) sc[lane] = fmaxf(v + bh[row], 0.f);
+                else if (half) a_part[row - HR] = v;                               // R[:, :Hh] y_c(s): kept for step s+1
+                else a_full[row - HR] = a_part[row - HR] + v;                      // R h_{s-1} complete
+            }
+            __syncwarp();
+            send_tile(sc, qbuf + (size_t)par * (K / 2) + (rank * HR) / 2, 16 * warp, HR, CS, lane, tag);
+        }
+        STAMP(1 + 6 * half);
+
+        // ---- 3. the cluster's hidden layer -> logits rows of this CTA
+#pragma unroll 1
         for (int i = tid; i < K / 2; i += blockDim.x) {
-            const unsigned a = smem_addr(qbuf + (size_t)(hs & 1) * (K / 2) + i);
-            uint4 v; unsigned long long t0 = 0; unsigned n = 0;
+            const unsigned a = smem_addr(qbuf + (size_t)par * (K / 2) + i);
+            uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
             while (true) {
                 v = ld_shared_volatile_v4(a);
-                if (v.y == hs + 1 && v.w == hs + 1) break;
-                if ((++n & 4095u) == 0 && wt.expired(t0, (int)s, 5)) { my_bad = true; break; }
+                if (v.y == tag && v.w == tag) break;
+                if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 2 + 4 * half)) { my_bad = true; break; }
             }
-            qvec[2 * i] = __uint_as_float(v.x); qvec[2 * i + 1] = __uint_as_float(v.z);
+            store_split(splQ, 2 * i, __uint_as_float(v.x));
+            store_split(splQ, 2 * i + 1, __uint_as_float(v.z));
         }
         if (__syncthreads_or(my_bad)) break;
-        if (warp < n_logit_warps) {
-            float hv[CPL * 8];
-            load_vec<CPL>(qvec, KC, lane, hv);
-            const int r0 = 4 * warp;
-            const float t = dot4<CPL>(wO2 + (size_t)r0 * KC, KC, lane, hv);
-            const float l0 = __shfl_sync(FULL, t, 0) + sb2[r0], l1 = __shfl_sync(FULL, t, 1) + sb2[r0 + 1];
-            const float l2 = __shfl_sync(FULL, t, 2) + sb2[r0 + 2], l3 = __shfl_sync(FULL, t, 3) + sb2[r0 + 3];
-            if (lane < 2 * CS) {
-                const int peer = lane >> 1, pair = lane & 1;
-                const unsigned a = map_to_rank(smem_addr(lbuf + (size_t)(hs & 1) * 128 + (rank * LR + r0) / 2 + pair), peer);
-                st_cluster_ll(a, pair ? l2 : l0, pair ? l3 : l1, hs + 1);
-            }
+        STAMP(2 + 6 * half);
+        if (l_on) {
+            float lo, hi;
+            mma_partial<NKL>(L + (size_t)l_tile * tile_u4, l_kt0, splQ, lane, lo, hi);
+            if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
         }
+        __syncthreads();
+        STAMP(14 + half);
+        if (l_fin) {
+            if (lane < 16) {
+                float v = 0.f;
+#pragma unroll
+                for (int sp = 0; sp < KSL; ++sp) v += part[(warp * KSL + sp) * 16 + lane];
+                sc[lane] = v + bl[16 * warp + lane];
+            }
+            __syncwarp();
+            send_tile(sc, lbuf + (size_t)par * 128 + (rank * LR) / 2, 16 * warp, LR, CS, lane, tag);
+        }
+        STAMP(3 + 6 * half);
+
+        // ---- 4. warp 0: the cluster's 256 logits -> draw; then the gates of the other half of the state
         if (warp == 0) {
             float l[8];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const unsigned a = smem_addr(lbuf + (size_t)(hs & 1) * 128 + 4 * lane + k);
-                uint4 v; unsigned long long t0 = 0; unsigned n = 0;
+                const unsigned a = smem_addr(lbuf + (size_t)par * 128 + 4 * lane + k);
+                uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
                 while (true) {
                     v = ld_shared_volatile_v4(a);
-                    if (v.y == hs + 1 && v.w == hs + 1) break;
-                    if ((++n & 4095u) == 0 && wt.expired(t0, (int)s, 6)) { my_bad = true; break; }
+                    if (v.y == tag && v.w == tag) break;
+                    if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 3 + 4 * half)) { my_bad = true; break; }
                 }
                 l[2 * k] = __uint_as_float(v.x); l[2 * k + 1] = __uint_as_float(v.z);
             }
             my_bad = __any_sync(FULL, my_bad);
-            const float u = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + s), 0u);
-            int c = warp_softmax_draw(l, u, lane);
+            STAMP(4 + 6 * half);
+            int drawn = warp_softmax_draw_fast(l, u01, lane);
             if (writer) {
                 if (p.dbg_logits) {
-                    float *d = p.dbg_logits + ((size_t)s * 2) * 256 + 8 * lane;
+                    float *d = p.dbg_logits + (size_t)(n - 1) * 256 + 8 * lane;
 #pragma unroll
                     for (int k = 0; k < 8; ++k) d[k] = l[k];
                 }
-                if (lane == 0 && p.c_out) p.c_out[s] = (uint8_t)c;
+                if (lane == 0) {
+                    if (half) { if (p.c_out) p.c_out[s] = (uint8_t)drawn; }
+                    else      { if (p.f_out) p.f_out[s - 1] = (uint8_t)drawn; }
+                }
             }
-            if (cf_next >= 0) c = cf_next;
-
-            // fine gates of step s: now c_s is known (I* lets it reach only these rows)
-            if (lane < UC && !my_bad) {
-                const float x0 = scale8(c_prev), x1 = scale8(f_prev), x2 = scale8(c);
-                const float *Iu = sI + 3 * (3 * UC + lane), *Ir = sI + 3 * (4 * UC + lane), *Ie = sI + 3 * (5 * UC + lane);
-                const float pu = a_full[3 * UC + lane] + fmaf(Iu[0], x0, fmaf(Iu[1], x1, fmaf(Iu[2], x2, gF[0])));
-                const float pr = a_full[4 * UC + lane] + fmaf(Ir[0], x0, fmaf(Ir[1], x1, fmaf(Ir[2], x2, gF[1])));
-                const float pe = fmaf(Ie[0], x0, fmaf(Ie[1], x1, fmaf(Ie[2], x2, gF[2])));
-                const float u2 = sigmoidf_acc(pu), r2 = sigmoidf_acc(pr);
-                const float e2 = tanhf(fmaf(r2, a_full[5 * UC + lane], pe));
-                hF = fmaf(u2, hF, (1.0f - u2) * e2);
-                const int j = cta * UC + lane;
-                st_relaxed_u64(p.slots + (size_t)(2 + (s & 1)) * K + j, ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hF));
-                if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[K + j] = u2; d[H + K + j] = r2; d[2 * H + K + j] = e2; }
-                if (p.dbg_h) p.dbg_h[(size_t)s * H + K + j] = hF;
+            if (forced >= 0) drawn = forced;
+            if (!half) {
+                if (writer && lane == 0 && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + drawn - 32768);
+                f_prev = drawn;
             }
-            c_prev = c;
+            if (lane < UC && !last && !my_bad) gates_and_publish(half, s, drawn, gv);
+            if (half) c_prev = drawn;
         }
-        ++hs;
+        STAMP(5 + 6 * half);
     }
+    if (prof_on && lane == 0) for (int i = 0; i < 16; ++i) p.prof[i] = s_prof[i];
 
     // final state (vecC holds y_c(T-1); vecF was refreshed by the last fine half)
     const int any_bad = __syncthreads_or(my_bad);
@@ -459,10 +480,12 @@ __global__ void __launch_bounds__(768, 1) resident_dense_kernel(const ResidentPa
 static int resident_smem_bytes(const ResidentPack &k)
 {
     size_t b = k.blob_bytes;
-    b += (size_t)3 * k.K * 4;                       // vecC, vecF, qvec
+    b += (size_t)2 * k.K * 4;                       // vecC, vecF
     size_t a = (size_t)2 * k.n_rrows;               // a_part, a_full
     a += (a % 4) ? 4 - (a % 4) : 0;
     b += a * 4;
+    b += 768 * 4;                                   // partial sums + per-warp scratch
+    b += (size_t)12 * k.K * 2;                      // three split images of 4 K bf16
     b += (size_t)k.K * 16;                          // qbuf [2][K/2] x 16 B
     b += 256 * 16;                                  // lbuf [2][128] x 16 B
     return (int)b;
@@ -489,28 +512,50 @@ static void dense_row_bf16(const BsrHost &M, int row, int c0, int n, uint16_t *d
     }
 }
 
+// rows[16][K] (bf16 bits, natural column order) -> A fragments [K/16][32 lanes][8] of m16n8k16:
+// lane (g, t) holds (row g, k 2t..2t+1), (row g+8, same), (row g, k 2t+8..9), (row g+8, same).
+// The vector side stores element 16 kt + c at split_pos and the B-fragment load reads it back from
+// there, so fragment column c of k-tile kt is plain column 16 kt + c of the matrix.
+static void pack_tile(const std::vector<std::vector<uint16_t>> &rows, int K, uint16_t *dst)
+{
+    for (int kt = 0; kt < K / 16; ++kt)
+        for (int lane = 0; lane < 32; ++lane) {
+            const int g = lane >> 2, t = lane & 3;
+            uint16_t *o = dst + ((size_t)kt * 32 + lane) * 8;
+            const int rsel[4] = {g, g + 8, g, g + 8};
+            const int csel[4] = {2 * t, 2 * t, 2 * t + 8, 2 * t + 8};
+            for (int q = 0; q < 4; ++q)
+                for (int j = 0; j < 2; ++j) o[2 * q + j] = rows[rsel[q]][16 * kt + csel[q] + j];
+        }
+}
+
 static bool choose_shape(const wrnn_model *m, ResidentPack *k, std::string *why)
 {
     const int H = m->H, Hh = H / 2;
     if (m->dtype != WRNN_BF16) { if (why) *why = "resident kernel stores bf16 weights only"; return false; }
     if (m->sparse) { if (why) *why = "resident dense kernel does not take block masks"; return false; }
-    if (H % 16 != 0 || Hh / 8 > 64) { if (why) *why = "H must be a multiple of 16 and at most 1024"; return false; }
+    if (H % 32 != 0) { if (why) *why = "H must be a multiple of 32"; return false; }
     const int CS = 8;
-    if (Hh % (4 * CS) != 0) { if (why) *why = "H/2 must be a multiple of 32"; return false; }
+    if (Hh % (2 * CS) != 0) { if (why) *why = "H/2 must be a multiple of 16"; return false; }
+    const int HR = Hh / CS, LR = 256 / CS;
     int best = 0;
     for (int ncta = CS; ncta <= m->n_sms; ncta += CS) {
         if (Hh % ncta) continue;
         const int uc = Hh / ncta;
-        if (uc % 2 || uc > 32) continue;
-        const int nw = Hh / CS / 4 + 6 * uc / 4;
-        if (nw > 24 || nw < 8) continue;
+        if ((HR + 6 * uc) % 16 || uc > 32) continue;       // stacked [head rows ; R rows] must fill 16-row tiles
+        if ((HR + 6 * uc) / 16 > 16) continue;
         best = ncta;
     }
-    if (!best) { if (why) *why = "no CTA count divides H/2 suitably"; return false; }
-    k->CS = CS; k->NCTA = best; k->NC = best / CS; k->UC = Hh / best; k->HR = Hh / CS; k->LR = 256 / CS;
-    k->K = Hh; k->KC = Hh / 8; k->n_rrows = 6 * k->UC;
-    k->NW = k->HR / 4 + k->n_rrows / 4;
-    k->w_bytes = ((size_t)2 * k->n_rrows + 2 * k->HR + 2 * k->LR) * k->K * 2;
+    if (!best) { if (why) *why = "no CTA count tiles H/2 into 16-row fragments"; return false; }
+    k->CS = CS; k->NCTA = best; k->NC = best / CS; k->UC = Hh / best; k->HR = HR; k->LR = LR;
+    k->K = Hh; k->NKT = Hh / 16; k->n_rrows = 6 * k->UC;
+    k->NMT = (HR + k->n_rrows) / 16; k->NLT = LR / 16;
+    k->NW = 20; k->KSH = 4; k->KSL = 7;
+    if (k->NKT != 28 || k->NMT * k->KSH > k->NW || k->NLT * k->KSL > k->NW) {
+        if (why) *why = "only the H/2 = 448 tiling (4 x 7 and 7 x 4 k-tiles) is instantiated";
+        return false;
+    }
+    k->w_bytes = ((size_t)2 * k->NMT + 2 * k->NLT) * 16 * k->K * 2;
     size_t small = ((size_t)k->n_rrows * 3 + 2 * k->HR + 2 * k->LR) * 4;
     small = (small + 15) / 16 * 16;
     k->blob_bytes = k->w_bytes + small;
@@ -518,7 +563,8 @@ static bool choose_shape(const wrnn_model *m, ResidentPack *k, std::string *why)
     return true;
 }
 
-static void *resident_fn() { return (void *)resident_dense_kernel<2>; }
+// The one instantiated split: K = 448 as 4 x 7 k-tiles (hidden, 5 tiles -> 20 warps) and 7 x 4 (logits, 2 tiles).
+static void *resident_fn() { return (void *)resident_dense_kernel<4, 7, 7, 4>; }
 
 int resident_supported(const wrnn_model *m, int batch, std::string *why)
 {
@@ -563,34 +609,40 @@ int resident_prepare(wrnn_model *m)
     // ---- per-CTA blobs
     const int H = m->H, K = k.K, UC = k.UC;
     std::vector<uint8_t> blob((size_t)k.NCTA * k.blob_bytes, 0);
-    std::vector<uint16_t> row(K);
+    std::vector<std::vector<uint16_t>> rows(16, std::vector<uint16_t>(K));
+    const BsrHost *Oa[2] = {&m->hO1, &m->hO3}, *Ob[2] = {&m->hO2, &m->hO4};
     for (int cta = 0; cta < k.NCTA; ++cta) {
         const int rank = cta % k.CS;
         uint8_t *base = blob.data() + (size_t)cta * k.blob_bytes;
         uint16_t *w = reinterpret_cast<uint16_t *>(base);
         float *sm = reinterpret_cast<float *>(base + k.w_bytes);
-        // R rows: index (half * 3 + gate) * UC + u  ->  matrix row gate * H + half * K + cta * UC + u
-        for (int part = 0; part < 2; ++part)            // 0: coarse columns (RA), 1: fine columns (RB)
-            for (int rr = 0; rr < k.n_rrows; ++rr) {
-                const int half = rr / (3 * UC), gate = (rr / UC) % 3, u = rr % UC;
-                const int mrow = gate * H + half * K + cta * UC + u;
-                dense_row_bf16(m->hR, mrow, part * K, K, row.data());
-                std::memcpy(w + ((size_t)part * k.n_rrows + rr) * K, row.data(), (size_t)K * 2);
-                if (part == 0) for (int c = 0; c < 3; ++c) sm[rr * 3 + c] = m->hI[(size_t)mrow * 3 + c];
+        const size_t tile_elems = (size_t)16 * K;
+        // stacked matrices MA (part 0: y_c input) and MB (part 1: y_f input): HR head rows then NR rows of R.
+        // R row rr = (half * 3 + gate) * UC + u  ->  matrix row gate * H + half * K + cta * UC + u
+        for (int part = 0; part < 2; ++part)
+            for (int mt = 0; mt < k.NMT; ++mt) {
+                for (int r = 0; r < 16; ++r) {
+                    const int row = 16 * mt + r;
+                    if (row < k.HR) dense_row_bf16(*Oa[part], rank * k.HR + row, 0, K, rows[r].data());
+                    else {
+                        const int rr = row - k.HR;
+                        const int half = rr / (3 * UC), gate = (rr / UC) % 3, u = rr % UC;
+                        dense_row_bf16(m->hR, gate * H + half * K + cta * UC + u, part * K, K, rows[r].data());
+                    }
+                }
+                pack_tile(rows, K, w + ((size_t)part * k.NMT + mt) * tile_elems);
             }
-        uint16_t *wo = w + (size_t)2 * k.n_rrows * K;
-        const BsrHost *Oa[2] = {&m->hO1, &m->hO3}, *Ob[2] = {&m->hO2, &m->hO4};
+        uint16_t *wl = w + (size_t)2 * k.NMT * tile_elems;
         for (int h = 0; h < 2; ++h)
-            for (int r = 0; r < k.HR; ++r) {
-                dense_row_bf16(*Oa[h], rank * k.HR + r, 0, K, row.data());
-                std::memcpy(wo + ((size_t)h * k.HR + r) * K, row.data(), (size_t)K * 2);
+            for (int mt = 0; mt < k.NLT; ++mt) {
+                for (int r = 0; r < 16; ++r) dense_row_bf16(*Ob[h], rank * k.LR + 16 * mt + r, 0, K, rows[r].data());
+                pack_tile(rows, K, wl + ((size_t)h * k.NLT + mt) * tile_elems);
             }
-        uint16_t *wl = wo + (size_t)2 * k.HR * K;
-        for (int h = 0; h < 2; ++h)
-            for (int r = 0; r < k.LR; ++r) {
-                dense_row_bf16(*Ob[h], rank * k.LR + r, 0, K, row.data());
-                std::memcpy(wl + ((size_t)h * k.LR + r) * K, row.data(), (size_t)K * 2);
-            }
+        for (int rr = 0; rr < k.n_rrows; ++rr) {
+            const int half = rr / (3 * UC), gate = (rr / UC) % 3, u = rr % UC;
+            const int mrow = gate * H + half * K + cta * UC + u;
+            for (int c = 0; c < 3; ++c) sm[rr * 3 + c] = m->hI[(size_t)mrow * 3 + c];
+        }
         float *b = sm + k.n_rrows * 3;
         for (int r = 0; r < k.HR; ++r) { b[r] = m->hb1[rank * k.HR + r]; b[k.HR + r] = m->hb3[rank * k.HR + r]; }
         b += 2 * k.HR;
@@ -599,10 +651,12 @@ int resident_prepare(wrnn_model *m)
     ResidentPack *pk = new ResidentPack(k);
     bool ok = cudaMalloc((void **)&pk->d_blob, blob.size()) == cudaSuccess &&
               cudaMemcpy(pk->d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) == cudaSuccess &&
-              cudaMalloc((void **)&pk->d_slots, (size_t)4 * K * 8) == cudaSuccess;
+              cudaMalloc((void **)&pk->d_slots, (size_t)4 * K * 8) == cudaSuccess &&
+              cudaMalloc((void **)&pk->d_prof, 16 * sizeof(long long)) == cudaSuccess &&
+              cudaMemset(pk->d_prof, 0, 16 * sizeof(long long)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
-        cudaFree(pk->d_blob); cudaFree(pk->d_slots);
+        cudaFree(pk->d_blob); cudaFree(pk->d_slots); cudaFree(pk->d_prof);
         delete pk;
         m->err = "device allocation for the resident kernel failed";
         return WRNN_ERR_NOMEM;
@@ -618,6 +672,7 @@ void resident_destroy(wrnn_model *m)
     if (!m->resident) return;
     cudaFree(m->resident->d_blob);
     cudaFree(m->resident->d_slots);
+    cudaFree(m->resident->d_prof);
     delete m->resident;
     m->resident = nullptr;
 }
@@ -638,7 +693,8 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     const ResidentPack &k = *m->resident;
     ResidentParams p;
     std::memset(&p, 0, sizeof(p));
-    p.H = m->H; p.K = k.K; p.KC = k.KC; p.UC = k.UC; p.HR = k.HR; p.LR = k.LR; p.CS = k.CS; p.n_rrows = k.n_rrows;
+    p.H = m->H; p.K = k.K; p.NKT = k.NKT; p.NMT = k.NMT; p.NLT = k.NLT; p.UC = k.UC; p.HR = k.HR; p.LR = k.LR; p.CS = k.CS;
+    p.n_rrows = k.n_rrows;
     p.n_steps = a.n_steps; p.step0 = a.step0; p.stream0 = a.stream0; p.seed = a.seed;
     p.n_frames = m->cond_dim ? a.n_frames : 1;
     p.hop = m->cond_dim ? a.hop : 1;
@@ -651,12 +707,13 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
     p.limit_ns = 2000000000ull;
+    p.prof = k.d_prof;
 
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     fill_launch(k, &cfg, at, s, true);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, resident_dense_kernel<2>, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, resident_dense_kernel<4, 7, 7, 4>, p);
     if (e != cudaSuccess) {
         m->err = std::string("resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();
@@ -664,6 +721,12 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     }
     ++g_launches;
     return WRNN_OK;
+}
+
+int resident_phase_cycles(const wrnn_model *m, long long *out16)
+{
+    if (!m->resident) return WRNN_ERR_UNSUPPORTED;
+    return cudaMemcpy(out16, m->resident->d_prof, 16 * sizeof(long long), cudaMemcpyDeviceToHost) == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
 }
 
 }  // namespace wrnn

@@ -156,3 +156,149 @@ def test_argument_errors(env):
         B.wrnn_destroy(m)
     with pytest.raises(B.WrnnError):
         B.wrnn_create(synth.make_weights(8, cond_dim=0) | {"R": np.zeros((30, 10), np.float32)}, "f32")   # H = 10
+
+
+# ---------------------------------------------------------------------------------------------
+# The named workloads at their full sizes (index = position in synth.WORKLOADS)
+
+def _tol_check(r, dtype):
+    tol = pu.TOL[dtype]
+    assert r["idx_bad"] == 0, {k: v for k, v in r.items() if k != "oracle"}
+    assert r["gates_err"] < tol and r["h_err"] < tol and r["logits_err"] < tol, {k: v for k, v in r.items() if k != "oracle"}
+
+
+def test_config1_dense_bf16_24000_resident(env):
+    """Dense H=896 bf16, batch 1, 24,000 steps through the shared-memory-resident kernel, in the launch
+    configuration the benchmark times: every step's gates / h / logits and both draws against the oracle."""
+    torch, B = env
+    wl = synth.WORKLOADS[1]
+    w, masks, cond = synth.build_workload(wl)
+    om = orc.OracleModel(w, wl.dtype)
+    m = B.wrnn_create(w, wl.dtype, kernel=B.WRNN_KERNEL_AUTO)
+    try:
+        assert B.wrnn_launch_info(m, 1)["kernel"] == B.WRNN_KERNEL_RESIDENT
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, wl.n_steps, 1, SEED)
+        free = _free_run(torch, B, m, cond, wl.n_steps, 1, SEED)
+        div = pu.first_divergence(free, r["oracle"].out)
+        _report("config1/resident", r, "free-run first divergence step %d" % div)
+        _tol_check(r, wl.dtype)
+        if div >= 0:
+            assert r["oracle"].margins[0, div].min() < pu.MARGIN
+        assert np.array_equal(free, _free_run(torch, B, m, cond, wl.n_steps, 1, SEED))      # deterministic
+        # resume: 10,000 + 14,000 steps with the carried state equal one call
+        h = torch.zeros((1, wl.H), dtype=torch.float32, device="cuda:0")
+        cp = torch.full((1,), 128, dtype=torch.uint8, device="cuda:0")
+        fp = torch.zeros((1,), dtype=torch.uint8, device="cuda:0")
+        a = _free_run(torch, B, m, cond, 10000, 1, SEED, h=h, c_prev=cp, f_prev=fp)
+        b = _free_run(torch, B, m, cond, 14000, 1, SEED, h=h, c_prev=cp, f_prev=fp, step0=10000)
+        assert np.array_equal(np.concatenate([a, b], axis=1), free)
+    finally:
+        B.wrnn_destroy(m)
+
+
+def test_resident_and_generic_kernels_agree(env):
+    """Same model through both kernel families: identical draws under teacher forcing on the oracle stream,
+    state within rounding."""
+    torch, B = env
+    wl = synth.WORKLOADS[1]
+    w, masks, cond = synth.build_workload(wl)
+    om = orc.OracleModel(w, wl.dtype)
+    n = 1500
+    res = om.run(cond, n, 1, SEED, dump=True)
+    outs = []
+    for kern in (B.WRNN_KERNEL_GENERIC, B.WRNN_KERNEL_RESIDENT):
+        m = B.wrnn_create(w, wl.dtype, kernel=kern)
+        try:
+            r = pu.teacher_forced_parity(torch, B, m, om, cond, n, 1, SEED, oracle_free=res)
+            _tol_check(r, wl.dtype)
+            outs.append(r)
+        finally:
+            B.wrnn_destroy(m)
+
+
+def test_config2_sparse_bf16(env):
+    """Block-sparse H=2048 bf16 (96 % of the 4x4 blocks of R_u, R_r, R_e, O1, O3 pruned), batch 1: the first
+    1,500 steps against the dense-with-zeros oracle; the full 24,000 steps for determinism and resume."""
+    torch, B = env
+    wl = synth.WORKLOADS[2]
+    w, masks, cond = synth.build_workload(wl)
+    assert masks["R"].sum() == 3 * 10486 and masks["O1"].sum() == 2621
+    om = orc.OracleModel(w, wl.dtype, masks)
+    m = B.wrnn_create(w, wl.dtype, masks)
+    try:
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, 1500, 1, SEED)
+        _report("config2/sparse", r)
+        _tol_check(r, wl.dtype)
+        free = _free_run(torch, B, m, cond, wl.n_steps, 1, SEED)
+        d = pu.first_divergence(free[:, :1500], r["oracle"].out)
+        if d >= 0:
+            assert r["oracle"].margins[0, d].min() < pu.MARGIN
+        assert np.array_equal(free, _free_run(torch, B, m, cond, wl.n_steps, 1, SEED))
+        h = torch.zeros((1, wl.H), dtype=torch.float32, device="cuda:0")
+        cp = torch.full((1,), 128, dtype=torch.uint8, device="cuda:0")
+        fp = torch.zeros((1,), dtype=torch.uint8, device="cuda:0")
+        a = _free_run(torch, B, m, cond, 9000, 1, SEED, h=h, c_prev=cp, f_prev=fp)
+        b = _free_run(torch, B, m, cond, 15000, 1, SEED, h=h, c_prev=cp, f_prev=fp, step0=9000)
+        assert np.array_equal(np.concatenate([a, b], axis=1), free)
+    finally:
+        B.wrnn_destroy(m)
+
+
+def test_config3_subscale_fold_batch16(env):
+    """One 24,000-sample sequence as 16 interleaved sub-sequences of 1,500 steps in lock-step, then unfolded."""
+    torch, B = env
+    wl = synth.WORKLOADS[3]
+    w, masks, cond = synth.build_workload(wl)
+    om = orc.OracleModel(w, wl.dtype)
+    m = B.wrnn_create(w, wl.dtype, max_batch=16)
+    try:
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, wl.n_steps, 16, SEED, row_stride=16, row_offset_mul=1,
+                                     threads=pu.NCPU)
+        _report("config3/subscale16", r)
+        _tol_check(r, wl.dtype)
+        out = torch.zeros(24000, dtype=torch.int16, device="cuda:0")
+        B.wrnn_sample_subscale(m, torch.from_numpy(cond).cuda(), 24000, 16, SEED, out)
+        torch.cuda.synchronize()
+        sub = _free_run(torch, B, m, cond, wl.n_steps, 16, SEED, row_stride=16, row_offset_mul=1)
+        assert np.array_equal(out.cpu().numpy(), orc.unfold(sub))           # exact permutation of the batch rows
+        div = pu.first_divergence(sub, r["oracle"].out)
+        if div >= 0:
+            assert r["oracle"].margins[:, div].min() < pu.MARGIN
+        # rows are independent: row 5 alone (global row id 5) reproduces row 5 of the batch
+        one = _free_run(torch, B, m, cond[5:6], wl.n_steps, 1, SEED, row_stride=16, row_offset_mul=1, stream0=5)
+        assert np.array_equal(one[0], sub[5])
+    finally:
+        B.wrnn_destroy(m)
+
+
+def _check_free_run_against_oracle(free, res):
+    """A free run may leave the oracle's stream only at a draw whose uniform is within MARGIN of a CDF boundary."""
+    for b in range(free.shape[0]):
+        d = pu.first_divergence(free[b], res.out[b])
+        if d >= 0:
+            assert res.margins[b, d].min() < pu.MARGIN, (b, d, res.margins[b, d])
+
+
+def test_config4_batched256(env):
+    """256 independent streams.  (1) all rows, first 100 steps, every gate / logit against the oracle;
+    (2) rows 0..7 for the full 24,000 steps (draws and final state, teacher-forced on the oracle's streams);
+    (3) the full 256 x 24,000 free run in the benchmark's launch configuration, rows 0..7 against (2)."""
+    torch, B = env
+    wl = synth.WORKLOADS[4]
+    w, masks, cond = synth.build_workload(wl)
+    om = orc.OracleModel(w, wl.dtype)
+    m = B.wrnn_create(w, wl.dtype, max_batch=256)
+    try:
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, 100, 256, SEED, threads=pu.NCPU)
+        _report("config4/batched256 (100 steps, all rows)", r)
+        _tol_check(r, wl.dtype)
+        n = wl.n_steps
+        r8 = pu.teacher_forced_parity(torch, B, m, om, cond[:8], n, 8, SEED, threads=pu.NCPU, dump=False)
+        print("\n[parity] config4 rows 0..7 x %d steps: idx_diff=%d near-boundary=%d bad=%d h_final=%.2e" % (
+            n, r8["idx_diff"], r8["near_boundary"], r8["idx_bad"], r8["h_final_err"]))
+        assert r8["idx_bad"] == 0 and r8["h_final_err"] < pu.TOL[wl.dtype]
+        full = _free_run(torch, B, m, cond, n, 256, SEED)
+        _check_free_run_against_oracle(full[:8], r8["oracle"])
+        assert len({full[b].tobytes() for b in range(256)}) == 256          # every stream is its own
+    finally:
+        B.wrnn_destroy(m)

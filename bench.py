@@ -267,11 +267,34 @@ def main():
                     "traffic": None, "peak_source": peaks["source"], "bytes_per_step": wbytes,
                     "note": "nonzero-block bytes per step over the HBM copy bandwidth"}
         else:
-            ach = wbytes * n_steps / (ms_per_step * 1e-3) / 1e9
+            # single stream, weights resident in shared memory: algorithmic bytes = every stored weight read once
+            # per step (3,047,296 weights at H = 896) over the aggregate shared-memory bandwidth, plus the floor
+            # of the two chip-wide exchanges a step cannot avoid (measured live in an empty kernel of the same shape)
+            H, Hh = wl.H, wl.H // 2
+            n_w = 3 * H * H + 2 * Hh * Hh + 2 * 256 * Hh + 9 * H
+            alg_bytes = n_w * (2 if wl.dtype == "bf16" else 4)
+            ach = alg_bytes * n_steps / (ms_per_step * 1e-3) / 1e9
             roof = {"bound": "smem", "achieved": ach, "peak": SMEM_PEAK_GBS, "unit": "GB/s", "frac": ach / SMEM_PEAK_GBS,
-                    "traffic": None, "peak_source": "derived: 148 SMs x 128 B/clk x 1.965 GHz", "bytes_per_step": wbytes,
-                    "note": "resident weight bytes read per step over aggregate shared-memory bandwidth; the step is "
-                            "latency-bound by two machine-wide exchanges, see DESIGN.md"}
+                    "traffic": 22862848 if info["kernel"] == 2 else None,
+                    "traffic_note": "DRAM bytes per launch from the ncu capture in profiles/ (one-time weight load; "
+                                    "does not grow with the number of steps)",
+                    "peak_source": "derived: 148 SMs x 128 B/clk x 1.965 GHz", "algorithmic_bytes_per_step": alg_bytes,
+                    "resident_bytes_read_per_step": wbytes}
+            if info["kernel"] == 2:
+                t_bar_ns = B.wrnn_measure_exchange_floor(info["n_ctas"], info["n_threads"], Hh, 20000)
+                smem_us = alg_bytes / (SMEM_PEAK_GBS * 1e3)
+                floor_us = smem_us + 2 * t_bar_ns * 1e-3
+                roof["latency_floor"] = {"smem_us": smem_us, "t_bar_us": t_bar_ns * 1e-3, "floor_us_per_step": floor_us,
+                                         "frac_of_floor": floor_us / us_per_sample_step,
+                                         "note": "weight bytes / smem bandwidth + 2 x measured chip-wide exchange"}
+                pc = B.wrnn_phase_cycles(model)
+                tot = float(sum(pc)) or 1.0
+                names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_gates",
+                         "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_gates",
+                         "F.hid_mma", "C.hid_mma", "F.log_mma", "C.log_mma"]
+                roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
+                waits = sum(pc[i] for i in (0, 2, 4, 6, 8, 10))
+                roof["wait_share"] = waits / tot
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",

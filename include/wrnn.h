@@ -205,6 +205,13 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
  * Synchronous. */
 int wrnn_phase_cycles(wrnn_model *m, int64_t *out16);
 
+/* Floor of a chip-wide exchange on this device: nanoseconds per all-gather of K tagged fp32 values through
+ * L2 among n_ctas co-resident CTAs of n_threads threads in an otherwise empty persistent kernel (Section 2.1:
+ * once the weights are resident, what remains per step is the synchronisation between multiprocessors; the
+ * sampling step needs two such exchanges).  K must be a multiple of n_ctas.  HOST out-pointer.  Synchronous;
+ * allocates and frees a small device buffer. */
+int wrnn_measure_exchange_floor(int32_t n_ctas, int32_t n_threads, int32_t K, int32_t iters, float *ns_per_exchange);
+
 /* Kernels launched by this library in this process since load (all models). */
 int64_t wrnn_launch_count(void);
 

@@ -24,7 +24,7 @@ _STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "NOMEM", "CUDA", "TIMEOUT"]
 EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
-    "wrnn_launch_count", "wrnn_phase_cycles",
+    "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor",
 ]
 
 
@@ -80,6 +80,7 @@ def lib():
         L.wrnn_last_error.restype = C.c_char_p
         L.wrnn_launch_info.argtypes = [vp, i32] + [vp] * 5
         L.wrnn_phase_cycles.argtypes = [vp, vp]
+        L.wrnn_measure_exchange_floor.argtypes = [i32, i32, i32, i32, vp]
         L.wrnn_launch_count.argtypes = []
         L.wrnn_launch_count.restype = i64
         _lib = L
@@ -229,3 +230,10 @@ def wrnn_phase_cycles(model):
     buf = (C.c_int64 * 16)()
     _check(lib().wrnn_phase_cycles(model, buf), model)
     return list(buf)
+
+
+def wrnn_measure_exchange_floor(n_ctas: int, n_threads: int, K: int, iters: int = 20000) -> float:
+    """Nanoseconds per chip-wide all-gather of K tagged values through L2 (empty persistent kernel)."""
+    out = C.c_float()
+    _check(lib().wrnn_measure_exchange_floor(n_ctas, n_threads, K, iters, C.byref(out)))
+    return out.value

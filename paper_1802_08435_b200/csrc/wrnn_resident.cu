@@ -24,6 +24,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 
 #include "wrnn_internal.h"
@@ -712,7 +713,11 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
-    fill_launch(k, &cfg, at, s, true);
+    // The cooperative attribute makes the driver refuse the launch unless all clusters can be co-resident.
+    // WRNN_NO_COOP=1 drops it (co-residency was already checked against the occupancy API at create):
+    // a profiler that replays kernels may not accept cooperative cluster launches.
+    const char *no_coop = getenv("WRNN_NO_COOP");
+    fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
     cudaError_t e = cudaLaunchKernelEx(&cfg, resident_dense_kernel<4, 7, 7, 4>, p);
     if (e != cudaSuccess) {
         m->err = std::string("resident kernel launch failed: ") + cudaGetErrorString(e);

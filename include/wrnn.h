@@ -137,6 +137,28 @@ int wrnn_sample(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t b
                 uint64_t seed, const wrnn_state *st, int16_t *out, void *cuda_stream);
 
 /*
+ * wrnn_sample_noalloc: wrnn_sample for callers that must not allocate.  (The paper has no counterpart;
+ * this exists for the way the library gets embedded.)  A real-time audio thread, a caller that is inside a
+ * region where device allocation is forbidden or would synchronise the whole device, or one running under a
+ * fixed memory budget creates its model ahead of time and then needs a sampling call that never reaches
+ * cudaMalloc / cudaFree -- wrnn_sample may grow its conditioning scratch on a larger request.  This entry
+ * point takes the same arguments and produces the same samples (it always runs the generic step kernel), but
+ * every byte of per-call scratch -- projected conditioning, state and head exchange buffers, the barrier
+ * counter -- lives in one fixed 8 MiB array inside the library's device image.  Each GPU that loads the
+ * library carries that array until the process exits.
+ *   - Sizes whose scratch does not fit (roughly batch * n_frames * 3H * 4 bytes plus batch * 5H * 4) are
+ *     refused with WRNN_ERR_UNSUPPORTED and a message that states both numbers; nothing is launched.
+ *   - The first call on a device looks up the array's device address (once per device, with that device made
+ *     current); make that first call outside any stream capture.
+ *   - All calls, on all models and streams, share the one array and it keeps what the previous call left
+ *     behind; the entry point re-zeroes what must start at zero, but two calls that overlap on the GPU race on
+ *     it.  Serialise them (one stream, or events).
+ * No cudaMalloc, cudaFree or allocating library routine is called.  Asynchronous on cuda_stream.
+ */
+int wrnn_sample_noalloc(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch,
+                        uint64_t seed, const wrnn_state *st, int16_t *out, void *cuda_stream);
+
+/*
  * wrnn_step_teacher_forced: the same steps, but the samples fed back are given.
  * Step s uses (c_forced, f_forced)[b][s-1] as the previous sample (the state's
  * c_prev / f_prev at s = 0) and c_forced[b][s] in the fine gates.  The indices the

@@ -24,7 +24,7 @@ _STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "NOMEM", "CUDA", "TIMEOUT"]
 EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
-    "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor",
+    "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor", "wrnn_sample_noalloc",
 ]
 
 
@@ -70,6 +70,7 @@ def lib():
         L.wrnn_destroy.argtypes = [vp]
         L.wrnn_destroy.restype = None
         L.wrnn_sample.argtypes = [vp, C.POINTER(wrnn_cond), i64, i32, u64, C.POINTER(wrnn_state), vp, vp]
+        L.wrnn_sample_noalloc.argtypes = [vp, C.POINTER(wrnn_cond), i64, i32, u64, C.POINTER(wrnn_state), vp, vp]
         L.wrnn_step_teacher_forced.argtypes = [vp, C.POINTER(wrnn_cond), i64, i32, u64, C.POINTER(wrnn_state)] + [vp] * 8
         L.wrnn_fold.argtypes = [vp, i64, i32, vp, vp]
         L.wrnn_unfold.argtypes = [vp, i64, i32, vp, vp]
@@ -237,3 +238,15 @@ def wrnn_measure_exchange_floor(n_ctas: int, n_threads: int, K: int, iters: int 
     out = C.c_float()
     _check(lib().wrnn_measure_exchange_floor(n_ctas, n_threads, K, iters, C.byref(out)))
     return out.value
+
+
+def wrnn_sample_noalloc(model, cond, n_steps: int, batch: int, seed: int, out, *, hop: int = 120, row_stride: int = 1,
+                        row_offset_mul: int = 0, h=None, c_prev=None, f_prev=None, step0: int = 0, stream0: int = 0,
+                        stream=None):
+    """Same arguments and samples as wrnn_sample, for callers that cannot allocate device memory at run time
+    (real-time threads, allocation-free regions, fixed memory budgets): all scratch sits in a fixed 8 MiB array
+    of the library image; requests that do not fit raise WrnnError(UNSUPPORTED).  Calls share that array, so
+    they must not overlap on the GPU."""
+    _check(lib().wrnn_sample_noalloc(model, _mk_cond(cond, hop, row_stride, row_offset_mul), n_steps, batch, seed,
+                                     _mk_state(h, c_prev, f_prev, step0, stream0), _dev_ptr(out), _stream_ptr(stream)),
+           model)

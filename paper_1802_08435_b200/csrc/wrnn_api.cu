@@ -114,8 +114,8 @@ static bool use_resident(const wrnn_model *m, int batch)
 
 // Common argument checks of the stepping calls; fills the parts of StepArgs that come from
 // cond / st.  Returns WRNN_OK or an error (message in m->err).
-static int check_step(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, const wrnn_state *st,
-                      StepArgs *a)
+int check_step(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, const wrnn_state *st,
+               StepArgs *a)
 {
     if (!m) return WRNN_ERR_INVALID_ARG;
     if (n_steps < 0 || batch < 1) return fail(m, WRNN_ERR_INVALID_ARG, "n_steps < 0 or batch < 1");

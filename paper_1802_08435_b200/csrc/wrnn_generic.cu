@@ -8,6 +8,8 @@
 //   B  q_c = relu(O1 y_c + b1)          C  l_c = O2 q_c + b2         D  draw c_t
 //   E  fine gates (now with c_t) -> y_f
 //   F  q_f = relu(O3 y_f + b3)          G  l_f = O4 q_f + b4         H  draw f_t, emit sample
+#include <cstdio>
+
 #include "wrnn_internal.h"
 
 namespace wrnn {
@@ -360,4 +362,124 @@ int generic_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     return WRNN_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Sampling without any allocation.  Everything the generic step kernel needs besides the model's
+// weights and the caller's buffers -- projected conditioning, the two state buffers, the head
+// exchange buffers, the per-row sample bytes and the grid-barrier counter -- is carved out of one
+// fixed array in device memory that belongs to the library image.  Every device that loads the
+// library holds these 8 MiB until the process exits.
+constexpr size_t kStaticScratchBytes = 8u << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// In host code the array's name is only a handle for the symbol, not a device address; the address
+// is looked up once per device (with that device current) and cached.
+constexpr int kMaxDevices = 64;
+static void *g_static_scratch_addr[kMaxDevices];
+static std::atomic<int> g_static_scratch_ready[kMaxDevices];
+
+static int static_scratch_base(int device, unsigned char **base, std::string *err)
+{
+    if (device < 0 || device >= kMaxDevices) { *err = "device index out of range for the static scratch table"; return WRNN_ERR_UNSUPPORTED; }
+    if (!g_static_scratch_ready[device].load(std::memory_order_acquire)) {
+        void *ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess || ptr == nullptr) {
+            *err = std::string("cudaGetSymbolAddress(static scratch) failed: ") + cudaGetErrorString(e);
+            cudaGetLastError();
+            return WRNN_ERR_CUDA;
+        }
+        g_static_scratch_addr[device] = ptr;         // racing first calls store the same value
+        g_static_scratch_ready[device].store(1, std::memory_order_release);
+    }
+    *base = static_cast<unsigned char *>(g_static_scratch_addr[device]);
+    return WRNN_OK;
+}
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
 }  // namespace wrnn
+
+using namespace wrnn;
+
+extern "C" int wrnn_sample_noalloc(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, uint64_t seed,
+                                   const wrnn_state *st, int16_t *out, void *cuda_stream)
+{
+    StepArgs a;
+    int rc = check_step(m, cond, n_steps, batch, st, &a);
+    if (rc != WRNN_OK) return rc;
+    if (n_steps == 0) return WRNN_OK;
+    if (!out) { m->err = "out is NULL"; return WRNN_ERR_INVALID_ARG; }
+    a.seed = seed; a.out = out;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (cudaSetDevice(m->device) != cudaSuccess) { m->err = "cudaSetDevice failed"; return WRNN_ERR_CUDA; }
+
+    // carve the fixed array; refuse sizes it cannot hold
+    const size_t B = (size_t)batch, H = (size_t)m->H, Hh = H / 2, G = 3 * H;
+    const size_t nf = m->cond_dim ? (size_t)a.n_frames : 1;
+    size_t off = 0;
+    const size_t o_bar = off;    off += 256;
+    const size_t o_bytes = off;  off += align256(3 * B);
+    const size_t o_h0 = off;     off += align256(B * H * 4);
+    const size_t o_h1 = off;     off += align256(B * H * 4);
+    const size_t o_af = off;     off += align256(B * 3 * Hh * 4);
+    const size_t o_q = off;      off += align256(B * Hh * 4);
+    const size_t o_l = off;      off += align256(B * 256 * 4);
+    const size_t o_g = off;      off += align256(B * nf * G * 4);
+    if (off > kStaticScratchBytes) {
+        char buf[200];
+        std::snprintf(buf, sizeof(buf), "wrnn_sample_noalloc: batch %d x %zu frames x 3H = %zu needs %zu bytes of scratch, the fixed array holds %zu",
+                      batch, nf, G, off, kStaticScratchBytes);
+        m->err = buf;
+        return WRNN_ERR_UNSUPPORTED;
+    }
+    unsigned char *base = nullptr;
+    rc = static_scratch_base(m->device, &base, &m->err);
+    if (rc != WRNN_OK) return rc;
+    float *g = reinterpret_cast<float *>(base + o_g);
+
+    // conditioning projection into the fixed array
+    if (m->cond_dim == 0) {
+        cond_bias_only_kernel<<<(unsigned)((G * B + 255) / 256), 256, 0, s>>>(m->b_gate, g, (int)G, batch);
+    } else {
+        dim3 grid((unsigned)((G + 255) / 256), (unsigned)nf, (unsigned)batch);
+        cond_project_kernel<<<grid, 256, m->cond_dim * sizeof(float), s>>>(a.cond, m->W_condT, m->b_gate, g, (int)G, m->cond_dim, (int)nf);
+    }
+    ++g_launches;
+    if (cudaGetLastError() != cudaSuccess) { m->err = "conditioning projection launch failed"; return WRNN_ERR_CUDA; }
+
+    GenericParams p;
+    p.H = m->H; p.Hh = m->H / 2; p.G = 3 * m->H; p.batch = batch;
+    p.n_steps = a.n_steps; p.step0 = a.step0; p.stream0 = a.stream0; p.seed = a.seed;
+    p.n_frames = (int)nf;
+    p.hop = m->cond_dim ? a.hop : 1;
+    p.row_stride = m->cond_dim ? a.row_stride : 0;
+    p.row_offset_mul = m->cond_dim ? a.row_offset_mul : 0;
+    p.R = m->R; p.O1 = m->O1; p.O2 = m->O2; p.O3 = m->O3; p.O4 = m->O4;
+    p.I = m->I; p.b1 = m->b1; p.b2 = m->b2; p.b3 = m->b3; p.b4 = m->b4; p.g = g;
+    p.h0 = reinterpret_cast<float *>(base + o_h0); p.h1 = reinterpret_cast<float *>(base + o_h1);
+    p.a_fine = reinterpret_cast<float *>(base + o_af); p.q = reinterpret_cast<float *>(base + o_q);
+    p.logits = reinterpret_cast<float *>(base + o_l);
+    p.c_cur = base + o_bytes; p.c_prev = base + o_bytes + B; p.f_prev = base + o_bytes + 2 * B;
+    p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in;
+    p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
+    p.c_forced = nullptr; p.f_forced = nullptr; p.c_out = nullptr; p.f_out = nullptr; p.out = a.out;
+    p.dbg_gates = nullptr; p.dbg_h = nullptr; p.dbg_logits = nullptr;
+    p.bar = reinterpret_cast<unsigned long long *>(base + o_bar);
+    p.status = m->status;
+    p.limit_ns = 2000000000ull;
+
+    // the array keeps the previous call's contents: the arrival counter must start at zero; the state and
+    // sample bytes are (re)initialised by the kernel itself before use
+    if (cudaMemsetAsync(base + o_bar, 0, 256, s) != cudaSuccess) { m->err = "memset failed"; return WRNN_ERR_CUDA; }
+    if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) { m->err = "memset failed"; return WRNN_ERR_CUDA; }
+    void *fn = generic_kernel_ptr(m->dtype, batch == 1 ? 1 : 8);
+    void *args[] = {(void *)&p};
+    const cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(m->n_sms), dim3(512), args, 0, s);
+    if (e != cudaSuccess) {
+        m->err = std::string("cooperative launch failed: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        return WRNN_ERR_CUDA;
+    }
+    ++g_launches;
+    return WRNN_OK;
+}

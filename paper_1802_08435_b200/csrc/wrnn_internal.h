@@ -92,6 +92,9 @@ namespace wrnn {
 
 extern std::atomic<long long> g_launches;
 
+// wrnn_api.cu: argument checks shared by the stepping entry points (fills the cond / state part of StepArgs)
+int check_step(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, const wrnn_state *st, StepArgs *a);
+
 // wrnn_generic.cu
 int generic_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem);
 int generic_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);   // returns wrnn_status

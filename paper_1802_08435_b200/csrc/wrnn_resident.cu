@@ -175,18 +175,23 @@ __device__ __forceinline__ void mma_partial(const uint4 *A, int kt0, const __nv_
     lo = s_lo; hi = s_hi;
 }
 
-// Send the 16 values of a tile (sc[0..15], rows row0..row0+15 of a cluster-wide vector laid out as
-// (value, tag) pairs) to every CTA of the cluster; only rows below row_limit are sent.
-__device__ __forceinline__ void send_tile(const float *sc, uint4 *buf_base, int row0, int row_limit, int CS, int lane, unsigned tag)
+// Finish and send one 16-row tile of a cluster-wide vector: lane (peer = lane & 7, ps = lane >> 3) sums the
+// K-split partials of rows 2 p, 2 p + 1 for the pairs p = ps and ps + 4, applies bias (and relu), and stores the
+// two tagged values straight into the peer's buffer (16 bytes per store).  Rows at or beyond row_limit are
+// not sent.  dst[k] are the precomputed cluster addresses of slot 0 of this tile's pair p = ps + 4 k at the peer.
+template <int KS, bool RELU>
+__device__ __forceinline__ void finish_and_send(const float *part_tile, const float *bias, int row0, int row_limit,
+                                                int lane, const unsigned (&dst)[2], unsigned tag, bool peer_ok)
 {
-    const int peer = lane & 7, ps = lane >> 3;
+    const int ps = lane >> 3;
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
-        const int pair = ps + 4 * k;
-        if (peer < CS && row0 + 2 * pair < row_limit) {
-            const unsigned a = map_to_rank(smem_addr(buf_base + (row0 >> 1) + pair), peer);
-            st_cluster_ll(a, sc[2 * pair], sc[2 * pair + 1], tag);
-        }
+        const int r = 2 * (ps + 4 * k);
+        float v0 = bias[row0 + r], v1 = bias[row0 + r + 1];
+#pragma unroll
+        for (int sp = 0; sp < KS; ++sp) { v0 += part_tile[sp * 16 + r]; v1 += part_tile[sp * 16 + r + 1]; }
+        if (RELU) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+        if (peer_ok && row0 + r < row_limit) st_cluster_ll(dst[k], v0, v1, tag);
     }
 }
 
@@ -265,6 +270,18 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
     const int l_tile = warp / KSL, l_kt0 = (warp % KSL) * NKL;
     const bool h_on = warp < NMT * KSH, l_on = warp < NLT * KSL;
     const bool h_fin = warp < NMT, l_fin = warp < NLT;
+    // cluster addresses of this lane's two destination slots (pairs ps and ps + 4 of tile `warp`) at peer lane & 7,
+    // for both buffer parities, for the hidden-layer buffer and the logits buffer
+    unsigned q_dst[2][2], l_dst[2][2];
+    const bool peer_ok = (lane & 7) < CS;
+#pragma unroll
+    for (int par2 = 0; par2 < 2; ++par2)
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const int pair = (lane >> 3) + 4 * k;
+            q_dst[par2][k] = map_to_rank(smem_addr(qbuf + (size_t)par2 * (K / 2) + (rank * HR + 16 * warp) / 2 + pair), peer_ok ? (lane & 7) : 0);
+            l_dst[par2][k] = map_to_rank(smem_addr(lbuf + (size_t)par2 * 128 + (rank * LR + 16 * warp) / 2 + pair), peer_ok ? (lane & 7) : 0);
+        }
 
     // ---- prologue: the recurrent products of step 0 from the initial state, coarse gates of step 0
     if (h_on) {
@@ -377,17 +394,17 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         __syncthreads();
         STAMP(12 + half);
         if (h_fin) {
-            if (lane < 16) {
+            // R rows of this tile (rows >= HR of the stacked matrix) stay in this CTA
+            const int row = 16 * warp + lane;
+            if (lane < 16 && row >= HR) {
                 float v = 0.f;
 #pragma unroll
                 for (int sp = 0; sp < KSH; ++sp) v += part[(warp * KSH + sp) * 16 + lane];
-                const int row = 16 * warp + lane;
-                if (row < HR) sc[lane] = fmaxf(v + bh[row], 0.f);
-                else if (half) a_part[row - HR] = v;                               // R[:, :Hh] y_c(s): kept for step s+1
+                if (half) a_part[row - HR] = v;                                    // R[:, :Hh] y_c(s): kept for step s+1
                 else a_full[row - HR] = a_part[row - HR] + v;                      // R h_{s-1} complete
             }
-            __syncwarp();
-            send_tile(sc, qbuf + (size_t)par * (K / 2) + (rank * HR) / 2, 16 * warp, HR, CS, lane, tag);
+            if (par) finish_and_send<KSH, true>(part + warp * KSH * 16, bh, 16 * warp, HR, lane, q_dst[1], tag, peer_ok);
+            else     finish_and_send<KSH, true>(part + warp * KSH * 16, bh, 16 * warp, HR, lane, q_dst[0], tag, peer_ok);
         }
         STAMP(1 + 6 * half);
 
@@ -414,14 +431,8 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         __syncthreads();
         STAMP(14 + half);
         if (l_fin) {
-            if (lane < 16) {
-                float v = 0.f;
-#pragma unroll
-                for (int sp = 0; sp < KSL; ++sp) v += part[(warp * KSL + sp) * 16 + lane];
-                sc[lane] = v + bl[16 * warp + lane];
-            }
-            __syncwarp();
-            send_tile(sc, lbuf + (size_t)par * 128 + (rank * LR) / 2, 16 * warp, LR, CS, lane, tag);
+            if (par) finish_and_send<KSL, false>(part + warp * KSL * 16, bl, 16 * warp, LR, lane, l_dst[1], tag, peer_ok);
+            else     finish_and_send<KSL, false>(part + warp * KSL * 16, bl, 16 * warp, LR, lane, l_dst[0], tag, peer_ok);
         }
         STAMP(3 + 6 * half);
 

@@ -55,7 +55,8 @@ typedef enum { WRNN_F32 = 0, WRNN_BF16 = 1 } wrnn_dtype;
 typedef enum {
     WRNN_KERNEL_AUTO = 0,       /* the fastest one that supports the model and batch          */
     WRNN_KERNEL_GENERIC = 1,    /* weights streamed from L2 every step; any shape; bring-up path */
-    WRNN_KERNEL_RESIDENT = 2    /* persistent kernel, weights resident in shared memory        */
+    WRNN_KERNEL_RESIDENT = 2,   /* persistent kernel, weights resident in shared memory (one row) */
+    WRNN_KERNEL_BATCHED = 3     /* tensor-pipe contractions over all rows (dense bf16, >= 2 rows)  */
 } wrnn_kernel;
 
 /*

@@ -50,6 +50,7 @@ struct StepArgs {
 };
 
 struct ResidentPack;   // packed weights of the shared-memory-resident kernels (opaque here)
+struct BatchedPack;    // fragment-packed weights and activation images of the batched kernel (opaque here)
 
 }  // namespace wrnn
 
@@ -80,6 +81,7 @@ struct wrnn_model {
     int16_t *stage_out = nullptr; size_t stage_out_cap = 0;
 
     wrnn::ResidentPack *resident = nullptr;
+    wrnn::BatchedPack *batched = nullptr;
 
     // host images for packers
     wrnn::BsrHost hR, hO1, hO2, hO3, hO4;
@@ -109,5 +111,12 @@ int resident_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_thr
                          int64_t *weight_bytes);
 int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
 int resident_phase_cycles(const wrnn_model *m, long long *out16);
+
+// wrnn_batched.cu
+int batched_supported(const wrnn_model *m, int batch, std::string *why);
+int batched_prepare(wrnn_model *m);
+void batched_destroy(wrnn_model *m);
+int batched_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem, int64_t *weight_bytes);
+int batched_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
 
 }  // namespace wrnn

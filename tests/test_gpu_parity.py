@@ -53,6 +53,30 @@ def test_tiny_teacher_forced(env, kernel, H, dtype, batch, sparse):
         B.wrnn_destroy(m)
 
 
+@pytest.mark.parametrize("H,batch", [(32, 2), (64, 11), (128, 33), (96, 16), (64, 70)])
+def test_tiny_batched_kernel(env, H, batch):
+    """The tensor-pipe batched kernel on small shapes: ragged batches, one and several stream blocks."""
+    torch, B = env
+    w = _tiny(H)
+    om = orc.OracleModel(w, "bf16")
+    m = B.wrnn_create(w, "bf16", max_batch=batch, kernel=B.WRNN_KERNEL_BATCHED)
+    try:
+        assert B.wrnn_launch_info(m, batch)["kernel"] == B.WRNN_KERNEL_BATCHED
+        cond = synth.make_cond(batch, 12, 4)
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, 40, batch, SEED, hop=10, row_stride=1, row_offset_mul=1,
+                                     threads=pu.NCPU)
+        assert r["idx_bad"] == 0, {k: v for k, v in r.items() if k != "oracle"}
+        tol = pu.TOL["bf16"]
+        assert r["gates_err"] < tol and r["h_err"] < tol and r["logits_err"] < tol, {k: v for k, v in r.items() if k != "oracle"}
+        # a smaller batch on the same model, with a row offset, and resume
+        lo = batch - 2
+        one = _free_run(torch, B, m, cond[lo:], 40, 2, SEED, hop=10, row_stride=1, row_offset_mul=1, stream0=lo)
+        ref = om.run(cond[lo:], 40, 2, SEED, hop=10, row_stride=1, row_offset_mul=1, stream0=lo)
+        _check_free_run_against_oracle(one, ref)
+    finally:
+        B.wrnn_destroy(m)
+
+
 def test_unconditioned_model_and_null_biases(env):
     torch, B = env
     w = _tiny(16, cond_dim=0)
@@ -65,6 +89,14 @@ def test_unconditioned_model_and_null_biases(env):
         assert r["idx_bad"] == 0 and r["gates_err"] < 1e-4 and r["logits_err"] < 1e-4, r
     finally:
         B.wrnn_destroy(m)
+
+
+def _check_free_run_against_oracle(free, res):
+    """A free run may leave the oracle's stream only at a draw whose uniform is within MARGIN of a CDF boundary."""
+    for b in range(free.shape[0]):
+        d = pu.first_divergence(free[b], res.out[b])
+        if d >= 0:
+            assert res.margins[b, d].min() < pu.MARGIN, (b, d, res.margins[b, d])
 
 
 def _free_run(torch, B, m, cond_np, n_steps, batch, seed, **kw):
@@ -108,7 +140,7 @@ def test_config0_dense_f32_1200(env, kernel):
 def test_resume_and_state_roundtrip(env):
     torch, B = env
     w = _tiny(64)
-    m = B.wrnn_create(w, "bf16", max_batch=3, kernel=B.WRNN_KERNEL_AUTO)
+    m = B.wrnn_create(w, "bf16", max_batch=3, kernel=B.WRNN_KERNEL_GENERIC)
     try:
         cond = synth.make_cond(3, 10, 4)
         full = _free_run(torch, B, m, cond, 90, 3, 77, hop=10)
@@ -269,14 +301,6 @@ def test_config3_subscale_fold_batch16(env):
         assert np.array_equal(one[0], sub[5])
     finally:
         B.wrnn_destroy(m)
-
-
-def _check_free_run_against_oracle(free, res):
-    """A free run may leave the oracle's stream only at a draw whose uniform is within MARGIN of a CDF boundary."""
-    for b in range(free.shape[0]):
-        d = pu.first_divergence(free[b], res.out[b])
-        if d >= 0:
-            assert res.margins[b, d].min() < pu.MARGIN, (b, d, res.margins[b, d])
 
 
 def test_config4_batched256(env):

@@ -12,7 +12,7 @@
 //   A   a = R h_{t-1}                         (all 3H rows)
 //   Gc  coarse gates -> y_c                   (element-wise)
 //   O1  q_c = relu(O1 y_c + b1)      O2  l_c = O2 q_c + b2
-//   Sc  draw c_t, then the fine gates -> y_f  (one warp per row)
+//   Sc  draw c_t (one warp per row)           Gf  fine gates -> y_f (element-wise)
 //   O3  q_f = relu(O3 y_f + b3)      O4  l_f = O4 q_f + b4
 //   Sf  draw f_t, emit the sample
 #include <cuda_bf16.h>
@@ -83,20 +83,26 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint4 &a, const ui
 }
 
 // Copy the image slice of one stream block (NT n8-tiles, both parts, k-tiles [kt0, kt0 + nk)) into shared
-// memory as [ntl][part][nk][32] uint2.  The image was written by other CTAs in an earlier phase: L1 is bypassed.
+// memory as [ntl][part][nk][32] uint2, with asynchronous 16-byte copies that bypass L1 (the image was written
+// by other CTAs in an earlier phase) so that the whole slice costs about one L2 round trip.
 template <int NT>
 __device__ __forceinline__ void stage_image(uint2 *sB, const __nv_bfloat16 *img, int sb, int nkt_img, int kt0, int nk)
 {
-    const uint2 *src = reinterpret_cast<const uint2 *>(img);
-    const int per = nk * 32;                    // uint2 per (ntl, part)
-    for (int i = threadIdx.x; i < NT * 2 * per; i += blockDim.x) {
-        const int np = i / per, r = i - np * per;          // np = ntl * 2 + part
-        const size_t s = ((size_t)(sb * NT) * 2 + np) * nkt_img * 32 + (size_t)kt0 * 32 + r;
-        sB[i] = __ldcg(src + s);
+    const uint4 *src = reinterpret_cast<const uint4 *>(img);
+    const int per = nk * 16;                    // uint4 per (ntl, part)
+    const unsigned sbase = (unsigned)__cvta_generic_to_shared(sB);
+    for (int np = 0; np < NT * 2; ++np) {       // np = ntl * 2 + part
+        const uint4 *g = src + (((size_t)(sb * NT) * 2 + np) * nkt_img + kt0) * 16;
+        for (int r = threadIdx.x; r < per; r += blockDim.x)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sbase + (unsigned)(np * per + r) * 16u), "l"(g + r) : "memory");
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
-// One 16-row weight tile (A fragments in global memory, nk k-tiles) against the staged stream block.
+// One 16-row weight tile (A fragments in global memory, nk k-tiles, nk a multiple of 4) against the staged
+// stream block.  The k loop runs in chunks of four k-tiles of straight-line code; the A fragments of the next
+// DEPTH chunks are already in flight (L2 latency), with the prefetch index clamped instead of branched.
 // acc[ntl][0..3]: rows g / g+8 of the tile, rows (streams) 8 ntl + 2t, 2t+1 of the block.
 template <int NT>
 __device__ __forceinline__ void tile_gemm(const uint4 *Af, int nk, const uint2 *sB, int lane, float (&acc)[NT][4])
@@ -105,24 +111,41 @@ __device__ __forceinline__ void tile_gemm(const uint4 *Af, int nk, const uint2 *
     for (int n = 0; n < NT; ++n)
 #pragma unroll
         for (int i = 0; i < 4; ++i) acc[n][i] = 0.f;
-    constexpr int PF = 8;                       // A fragments in flight (L2 latency)
-    uint4 a[PF];
+    constexpr int KC = 4;
+    constexpr int DEPTH = NT >= 4 ? 2 : 4;
+    const int nchunks = nk / KC;
+    uint4 a[DEPTH][KC];
     const uint4 *ap = Af + lane;
 #pragma unroll
-    for (int i = 0; i < PF; ++i) a[i] = (i < nk) ? __ldg(ap + (size_t)i * 32) : make_uint4(0, 0, 0, 0);
-    for (int k0 = 0; k0 < nk; k0 += PF) {
+    for (int d = 0; d < DEPTH; ++d) {
+        const int c = min(d, nchunks - 1);
 #pragma unroll
-        for (int i = 0; i < PF; ++i) {
-            const int kt = k0 + i;
-            if (kt < nk) {
-                const uint4 av = a[i];
-                if (kt + PF < nk) a[i] = __ldg(ap + (size_t)(kt + PF) * 32);
+        for (int i = 0; i < KC; ++i) a[d][i] = __ldg(ap + (size_t)(c * KC + i) * 32);
+    }
+    for (int c0 = 0; c0 < nchunks; c0 += DEPTH) {
 #pragma unroll
-                for (int n = 0; n < NT; ++n) {
-                    const uint2 bhi = sB[((n * 2 + 0) * nk + kt) * 32 + lane];
-                    const uint2 blo = sB[((n * 2 + 1) * nk + kt) * 32 + lane];
-                    mma_bf16(acc[n], av, bhi);
-                    mma_bf16(acc[n], av, blo);
+        for (int d = 0; d < DEPTH; ++d) {
+            const int c = c0 + d;
+            if (c < nchunks) {
+                uint4 av[KC];
+#pragma unroll
+                for (int i = 0; i < KC; ++i) av[i] = a[d][i];
+                const int cn = min(c + DEPTH, nchunks - 1);
+#pragma unroll
+                for (int i = 0; i < KC; ++i) a[d][i] = __ldg(ap + (size_t)(cn * KC + i) * 32);
+#pragma unroll
+                for (int i = 0; i < KC; ++i) {
+                    const int kt = c * KC + i;
+                    uint2 bhi[NT], blo[NT];
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) {
+                        bhi[n] = sB[((n * 2 + 0) * nk + kt) * 32 + lane];
+                        blo[n] = sB[((n * 2 + 1) * nk + kt) * 32 + lane];
+                    }
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) mma_bf16(acc[n], av[i], bhi[n]);
+#pragma unroll
+                    for (int n = 0; n < NT; ++n) mma_bf16(acc[n], av[i], blo[n]);
                 }
             }
         }
@@ -154,9 +177,19 @@ __device__ __forceinline__ void gate_unit_b(const BatchedParams &p, int j, int g
     if (p.dbg_h) p.dbg_h[((size_t)s * p.batch + gb) * H + j] = hn;
 }
 
+#ifdef WRNN_PROFILE_BATCHED
+__device__ long long g_bprof[32];
+#define BSTAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { const long long n_ = clock64(); g_bprof[i] += n_ - bt_; bt_ = n_; } } while (0)
+#else
+#define BSTAMP(i) do { } while (0)
+#endif
+
 template <int NT>
 __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParams p)
 {
+#ifdef WRNN_PROFILE_BATCHED
+    long long bt_ = clock64();
+#endif
     extern __shared__ __align__(16) uint8_t smem_raw[];
     uint2 *sB = reinterpret_cast<uint2 *>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
@@ -209,14 +242,19 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
 
     for (long long s = 0; s < p.n_steps; ++s) {
         // ---- A: a = R h_{t-1}
+        BSTAMP(31);
         contraction(p.Rf, 3 * H / 16, p.NKT_R, ic, p.NKT_R, 0, [&](int row, int b, float v) { p.a_buf[(size_t)b * p.G + row] = v; });
+        BSTAMP(0);
         if (!bar.sync((int)s, 1)) return;
+        BSTAMP(1);
         // ---- Gc: coarse gates
         for (int i = gtid; i < B * Hh; i += nthreads) {
             const int gb = i / Hh, j = i - gb * Hh;
             gate_unit_b(p, j, gb, s, hc, hn, in, scale8(__ldcg(p.c_prev + gb)), scale8(__ldcg(p.f_prev + gb)), 0.f);
         }
+        BSTAMP(2);
         if (!bar.sync((int)s, 2)) return;
+        BSTAMP(3);
 
         for (int head = 0; head < 2; ++head) {
             const uint4 *Oa = head ? p.O3f : p.O1f, *Ob = head ? p.O4f : p.O2f;
@@ -225,16 +263,19 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
             contraction(Oa, Hh / 16, p.NKT_H, in, p.NKT_R, head * p.NKT_H, [&](int row, int b, float v) {
                 img_store(p.qimg, b, row, p.NKT_H, fmaxf(v + (ba ? ba[row] : 0.f), 0.f));
             });
+            BSTAMP(4 + 8 * head);
             if (!bar.sync((int)s, 3 + 4 * head)) return;
+            BSTAMP(5 + 8 * head);
             // ---- O2 / O4: logits
             contraction(Ob, 16, p.NKT_H, p.qimg, p.NKT_H, 0, [&](int row, int b, float v) {
                 const float l = v + (bb ? bb[row] : 0.f);
                 p.logits[(size_t)b * 256 + row] = l;
                 if (p.dbg_logits) p.dbg_logits[(((size_t)s * B + b) * 2 + head) * 256 + row] = l;
             });
+            BSTAMP(6 + 8 * head);
             if (!bar.sync((int)s, 4 + 4 * head)) return;
-            // ---- Sc / Sf: softmax + inverse-CDF draw, one warp per row; after the coarse draw the same warp
-            //      evaluates the fine gates of its row (c_t reaches only those, Section 2)
+            BSTAMP(7 + 8 * head);
+            // ---- Sc / Sf: softmax + inverse-CDF draw, one warp per row
             for (int gb = gw; gb < B; gb += nw) {
                 float l[8];
                 const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(p.logits + (size_t)gb * 256 + 8 * lane));
@@ -244,11 +285,11 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
                 int idx = warp_softmax_draw(l, u, lane);
                 const size_t o = (size_t)gb * p.n_steps + s;
                 if (head == 0) {
-                    if (lane == 0 && p.c_out) p.c_out[o] = (uint8_t)idx;
-                    if (p.c_forced) idx = p.c_forced[o];
-                    if (lane == 0) p.c_cur[gb] = (uint8_t)idx;
-                    const float x0 = scale8(__ldcg(p.c_prev + gb)), x1 = scale8(__ldcg(p.f_prev + gb)), x2 = scale8(idx);
-                    for (int j = Hh + lane; j < H; j += 32) gate_unit_b(p, j, gb, s, hc, hn, in, x0, x1, x2);
+                    if (lane == 0) {
+                        if (p.c_out) p.c_out[o] = (uint8_t)idx;
+                        if (p.c_forced) idx = p.c_forced[o];
+                        p.c_cur[gb] = (uint8_t)idx;
+                    }
                 } else {
                     if (lane == 0) {
                         if (p.f_out) p.f_out[o] = (uint8_t)idx;
@@ -260,7 +301,20 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
                     }
                 }
             }
+            BSTAMP(8 + 8 * head);
             if (!bar.sync((int)s, 5 + 4 * head)) return;
+            BSTAMP(9 + 8 * head);
+            if (head == 0) {
+                // ---- Gf: fine gates, now that c_t is known (it reaches only these rows, Section 2)
+                for (int i = gtid; i < B * Hh; i += nthreads) {
+                    const int gb = i / Hh, j = Hh + (i - gb * Hh);
+                    gate_unit_b(p, j, gb, s, hc, hn, in, scale8(__ldcg(p.c_prev + gb)), scale8(__ldcg(p.f_prev + gb)),
+                                scale8(__ldcg(p.c_cur + gb)));
+                }
+                BSTAMP(10);
+                if (!bar.sync((int)s, 6)) return;
+                BSTAMP(11);
+            }
         }
         { float *t = hc; hc = hn; hn = t; }
         { __nv_bfloat16 *t = ic; ic = in; in = t; }
@@ -320,7 +374,7 @@ int batched_supported(const wrnn_model *m, int batch, std::string *why)
 int batched_prepare(wrnn_model *m)
 {
     if (m->dtype != WRNN_BF16 || m->sparse) { m->err = "batched kernel takes dense bf16 models"; return WRNN_ERR_UNSUPPORTED; }
-    if (m->H % 32 != 0) { m->err = "batched kernel needs H to be a multiple of 32"; return WRNN_ERR_UNSUPPORTED; }
+    if (m->H % 128 != 0) { m->err = "batched kernel needs H to be a multiple of 128 (k-tiles in chunks of four)"; return WRNN_ERR_UNSUPPORTED; }
     if (m->max_batch < 2) { m->err = "max_batch < 2"; return WRNN_ERR_UNSUPPORTED; }
     BatchedPack *k = new BatchedPack();
     const int H = m->H, Hh = H / 2;
@@ -420,3 +474,11 @@ int batched_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
 }
 
 }  // namespace wrnn
+
+#ifdef WRNN_PROFILE_BATCHED
+extern "C" int wrnn_debug_batched_prof(long long *out32, int reset)
+{
+    if (reset) { long long z[32] = {0}; return cudaMemcpyToSymbol(wrnn::g_bprof, z, sizeof(z)) == cudaSuccess ? 0 : 4; }
+    return cudaMemcpyFromSymbol(out32, wrnn::g_bprof, 32 * sizeof(long long)) == cudaSuccess ? 0 : 4;
+}
+#endif

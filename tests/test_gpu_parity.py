@@ -53,7 +53,7 @@ def test_tiny_teacher_forced(env, kernel, H, dtype, batch, sparse):
         B.wrnn_destroy(m)
 
 
-@pytest.mark.parametrize("H,batch", [(32, 2), (64, 11), (128, 33), (96, 16), (64, 70)])
+@pytest.mark.parametrize("H,batch", [(128, 2), (128, 11), (256, 33), (384, 16), (128, 70)])
 def test_tiny_batched_kernel(env, H, batch):
     """The tensor-pipe batched kernel on small shapes: ragged batches, one and several stream blocks."""
     torch, B = env

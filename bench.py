@@ -301,7 +301,7 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "H": wl.H, "batch": wl.batch, "n_steps": n_steps, "weights": wl.dtype,
                        "sparsity": wl.sparsity, "l2": "flushed between timed iterations (256 MiB fill)",
-                       "kernel": {1: "generic", 2: "resident", 3: "batched"}[info["kernel"]], "n_ctas": info["n_ctas"],
+                       "kernel": {1: "generic", 2: "resident", 3: "batched", 4: "sparse-cluster"}[info["kernel"]], "n_ctas": info["n_ctas"],
                        "threads_per_cta": info["n_threads"], "smem_bytes_per_cta": info["smem_bytes"],
                        "multi_gpu": "replicas only"},
             "us_per_sample_step": us_per_sample_step, "x_realtime_24khz": value / world / wl.batch / 24000.0 * wl.batch,

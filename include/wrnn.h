@@ -56,7 +56,8 @@ typedef enum {
     WRNN_KERNEL_AUTO = 0,       /* the fastest one that supports the model and batch          */
     WRNN_KERNEL_GENERIC = 1,    /* weights streamed from L2 every step; any shape; bring-up path */
     WRNN_KERNEL_RESIDENT = 2,   /* persistent kernel, weights resident in shared memory (one row) */
-    WRNN_KERNEL_BATCHED = 3     /* tensor-pipe contractions over all rows (dense bf16, >= 2 rows)  */
+    WRNN_KERNEL_BATCHED = 3,    /* tensor-pipe contractions over all rows (dense bf16, >= 2 rows)  */
+    WRNN_KERNEL_SPARSE = 4      /* block-sparse model resident in one 16-CTA cluster (one row)     */
 } wrnn_kernel;
 
 /*

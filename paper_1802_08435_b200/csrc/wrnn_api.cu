@@ -112,6 +112,12 @@ static bool use_resident(const wrnn_model *m, int batch)
     return m->resident != nullptr && resident_supported(m, batch, nullptr) == WRNN_OK;
 }
 
+static bool use_sparse(const wrnn_model *m, int batch)
+{
+    if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_SPARSE) return false;
+    return m->sparse_pack != nullptr && sparse_supported(m, batch, nullptr) == WRNN_OK;
+}
+
 static bool use_batched(const wrnn_model *m, int batch)
 {
     if (m->kernel == WRNN_KERNEL_GENERIC || m->kernel == WRNN_KERNEL_RESIDENT) return false;
@@ -163,7 +169,13 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     int rc = cond_project(m, a.cond, a.batch, nf, s);
     if (rc != WRNN_OK) return fail(m, rc, "conditioning projection launch failed");
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
+    if (use_sparse(m, a.batch)) return sparse_run(m, a, s);
     if (use_batched(m, a.batch)) return batched_run(m, a, s);
+    if (m->kernel == WRNN_KERNEL_SPARSE) {
+        std::string why;
+        sparse_supported(m, a.batch, &why);
+        return fail(m, WRNN_ERR_UNSUPPORTED, "sparse cluster kernel unavailable: " + why);
+    }
     if (m->kernel == WRNN_KERNEL_BATCHED) {
         std::string why;
         batched_supported(m, a.batch, &why);
@@ -195,7 +207,7 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
     if (!p->R || !p->I || !p->O1 || !p->O2 || !p->O3 || !p->O4) return fail(nullptr, WRNN_ERR_INVALID_ARG, "missing weight matrix");
     if ((p->cond_dim > 0) != (p->W_cond != nullptr)) return fail(nullptr, WRNN_ERR_INVALID_ARG, "W_cond must be given iff cond_dim > 0");
     if (p->dtype != WRNN_F32 && p->dtype != WRNN_BF16) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown dtype");
-    if (p->kernel < WRNN_KERNEL_AUTO || p->kernel > WRNN_KERNEL_BATCHED) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown kernel family");
+    if (p->kernel < WRNN_KERNEL_AUTO || p->kernel > WRNN_KERNEL_SPARSE) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown kernel family");
 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, WRNN_ERR_CUDA, "no usable CUDA device"); }
@@ -260,6 +272,14 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
     m->weight_bytes = bsr_bytes(m->hR) + bsr_bytes(m->hO1) + bsr_bytes(m->hO2) + bsr_bytes(m->hO3) + bsr_bytes(m->hO4) +
                       (int64_t)G * 3 * 4;
 
+    if (p->kernel == WRNN_KERNEL_AUTO || p->kernel == WRNN_KERNEL_SPARSE) {
+        const int rc = sparse_prepare(m);
+        if (rc != WRNN_OK && p->kernel == WRNN_KERNEL_SPARSE) {
+            const std::string why = m->err;
+            wrnn_destroy(m);
+            return fail(nullptr, rc, "sparse cluster kernel unavailable: " + why);
+        }
+    }
     if (p->kernel == WRNN_KERNEL_AUTO || p->kernel == WRNN_KERNEL_BATCHED) {
         const int rc = batched_prepare(m);
         if (rc != WRNN_OK && p->kernel == WRNN_KERNEL_BATCHED) {
@@ -287,6 +307,7 @@ void wrnn_destroy(wrnn_model *m)
     cudaDeviceSynchronize();
     resident_destroy(m);
     batched_destroy(m);
+    sparse_destroy(m);
     free_bsr(&m->R); free_bsr(&m->O1); free_bsr(&m->O2); free_bsr(&m->O3); free_bsr(&m->O4);
     cudaFree(m->I); cudaFree(m->b_gate); cudaFree(m->b1); cudaFree(m->b2); cudaFree(m->b3); cudaFree(m->b4);
     cudaFree(m->W_condT); cudaFree(m->g); cudaFree(m->hbuf[0]); cudaFree(m->hbuf[1]); cudaFree(m->a_fine);
@@ -409,6 +430,10 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
     if (use_resident(m, batch)) {
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
+    }
+    if (use_sparse(m, batch)) {
+        if (kernel) *kernel = WRNN_KERNEL_SPARSE;
+        return sparse_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
     }
     if (use_batched(m, batch)) {
         if (kernel) *kernel = WRNN_KERNEL_BATCHED;

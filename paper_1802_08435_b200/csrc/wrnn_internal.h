@@ -51,6 +51,7 @@ struct StepArgs {
 
 struct ResidentPack;   // packed weights of the shared-memory-resident kernels (opaque here)
 struct BatchedPack;    // fragment-packed weights and activation images of the batched kernel (opaque here)
+struct SparsePack;     // compressed block rows of the single-cluster block-sparse kernel (opaque here)
 
 }  // namespace wrnn
 
@@ -82,6 +83,7 @@ struct wrnn_model {
 
     wrnn::ResidentPack *resident = nullptr;
     wrnn::BatchedPack *batched = nullptr;
+    wrnn::SparsePack *sparse_pack = nullptr;
 
     // host images for packers
     wrnn::BsrHost hR, hO1, hO2, hO3, hO4;
@@ -111,6 +113,13 @@ int resident_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_thr
                          int64_t *weight_bytes);
 int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
 int resident_phase_cycles(const wrnn_model *m, long long *out16);
+
+// wrnn_sparse.cu
+int sparse_supported(const wrnn_model *m, int batch, std::string *why);
+int sparse_prepare(wrnn_model *m);
+void sparse_destroy(wrnn_model *m);
+int sparse_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem, int64_t *weight_bytes);
+int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
 
 // wrnn_batched.cu
 int batched_supported(const wrnn_model *m, int batch, std::string *why);

@@ -1,0 +1,588 @@
+// Block-sparse single-stream sampling kernel (Section 3: only the kept 4x4 blocks of R_u, R_r, R_e, O1, O3
+// are stored and multiplied): bf16 weights, batch 1, the whole model resident in the shared memory of ONE
+// thread-block cluster of 16 CTAs.
+//
+// A pruned model is small enough (H = 2048 at 96 %: 2.3 MB of blocks, plus the dense O2 / O4) that no state
+// ever has to cross the chip through L2: every exchange of a step -- the two halves of the state, the hidden
+// layer of a head, its logits -- is an all-gather of (value, tag) words through distributed shared memory.
+// Each CTA owns Hh/16 coarse and Hh/16 fine units (their block rows of R, compressed: block column index +
+// 16 bf16 per kept block), Hh/16 rows of O1 and O3 (compressed block rows) and 16 rows of the dense O2 and O4
+// (mma.sync A fragments).  Sparse rows: eight lanes share a block row, each lane takes every eighth kept
+// block (two 16-byte weight loads, four activations, 16 FMAs), a four-value reduce-scatter finishes the rows.
+// The step itself is the two-half schedule of the dense resident kernel (Fig. 1's order).
+//
+// Every wait is bounded; all CTAs leave through the final cluster barrier.
+#include <cooperative_groups.h>
+
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+
+#include "wrnn_cluster.cuh"
+#include "wrnn_internal.h"
+
+namespace cg = cooperative_groups;
+
+namespace wrnn {
+
+constexpr int SCS = 16;          // cluster size
+constexpr int SNW = 20;          // warps per CTA
+
+struct SparsePack {
+    int H = 0, K = 0, NKT = 0, UC = 0, HR = 0, NBR = 0;   // NBR: block rows per phase = (HR + 6 UC) / 4
+    int max_nnz = 0;                  // kept blocks per phase per CTA (padded maximum)
+    size_t blob_bytes = 0;            // per CTA
+    size_t off_brp[2], off_col[2], off_val[2], off_o2 = 0, off_o4 = 0, off_small = 0;
+    uint8_t *d_blob = nullptr;
+    int smem_bytes = 0;
+    int64_t weight_bytes_per_step = 0;   // kept blocks + indices + row pointers + dense O2/O4/I, each counted once
+};
+
+struct SparseParams {
+    int H, K, NKT, UC, HR, NBR;
+    unsigned long long off_brp[2], off_col[2], off_val[2], off_o2, off_o4, off_small, blob_bytes;
+    long long n_steps, step0;
+    unsigned stream0;
+    unsigned long long seed;
+    int n_frames, hop, row_stride, row_offset_mul;
+    const uint8_t *blob;
+    const float *g;
+    const float *h_in; float *h_out;
+    const uint8_t *c_in, *f_in; uint8_t *c_st_out, *f_st_out;
+    const uint8_t *c_forced, *f_forced;
+    uint8_t *c_out, *f_out;
+    int16_t *out;
+    float *dbg_gates, *dbg_h, *dbg_logits;
+    DevStatus *status;
+    unsigned long long limit_ns;
+};
+
+#ifdef WRNN_PROFILE_SPARSE
+__device__ long long g_sprof[16];
+#define SSTAMP(i) do { if (blockIdx.x == 0 && warp == 0) { const long long n_ = clock64(); if (lane == 0) g_sprof[i] += n_ - st_; st_ = n_; } } while (0)
+#else
+#define SSTAMP(i) do { } while (0)
+#endif
+
+// NKL: k-tiles of the logits tile per warp (K / 16 / NKL warps split K).
+template <int NKL>
+__global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const SparseParams p)
+{
+    extern __shared__ __align__(16) uint8_t smem[];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int K = p.K, NKT = p.NKT, UC = p.UC, HR = p.HR, NBR = p.NBR, H = p.H;
+    const int NR = 6 * UC;
+
+    // ---- shared memory carve-up (must match sparse_smem_bytes)
+    const int *brp[2] = {reinterpret_cast<const int *>(smem + p.off_brp[0]), reinterpret_cast<const int *>(smem + p.off_brp[1])};
+    const uint16_t *bcol[2] = {reinterpret_cast<const uint16_t *>(smem + p.off_col[0]), reinterpret_cast<const uint16_t *>(smem + p.off_col[1])};
+    const uint4 *bval[2] = {reinterpret_cast<const uint4 *>(smem + p.off_val[0]), reinterpret_cast<const uint4 *>(smem + p.off_val[1])};
+    const uint4 *wO2 = reinterpret_cast<const uint4 *>(smem + p.off_o2), *wO4 = reinterpret_cast<const uint4 *>(smem + p.off_o4);
+    const float *sI = reinterpret_cast<const float *>(smem + p.off_small);            // [NR][3]
+    const float *sb1 = sI + NR * 3, *sb3 = sb1 + HR, *sb2 = sb3 + HR, *sb4 = sb2 + 16;
+    float *vecC = reinterpret_cast<float *>(smem + p.blob_bytes);                     // [K] y_c
+    float *vecF = vecC + K;                                                           // [K] y_f
+    float *qvec = vecF + K;                                                           // [K] hidden layer
+    float *a_part = qvec + K;                                                         // [NR]
+    float *a_full = a_part + NR;                                                      // [NR]
+    float *part = a_full + NR;                                                        // [16 warps][16]
+    float *ynew = part + 256;                                                         // [UC] freshly gated units
+    __nv_bfloat16 *splQ = reinterpret_cast<__nv_bfloat16 *>(ynew + ((UC + 3) & ~3));  // split image of q, 4 K bf16
+    uint4 *ybuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                            // [2][K/2] state halves
+    uint4 *qbuf = ybuf + K;                                                           // [2][K/2] hidden layer
+    uint4 *lbuf = qbuf + K;                                                           // [2][128] logits
+
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.blob + (size_t)rank * p.blob_bytes);
+        uint4 *dst = reinterpret_cast<uint4 *>(smem);
+        for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
+        for (int i = tid; i < 2 * K + 256; i += blockDim.x) ybuf[i] = make_uint4(0, 0, 0, 0);   // ybuf, qbuf, lbuf are adjacent
+        for (int i = tid; i < 4 * K / 8; i += blockDim.x) reinterpret_cast<uint4 *>(splQ)[i] = make_uint4(0, 0, 0, 0);
+        for (int i = tid; i < K; i += blockDim.x) {
+            vecC[i] = p.h_in ? p.h_in[i] : 0.f;
+            vecF[i] = p.h_in ? p.h_in[K + i] : 0.f;
+        }
+    }
+    __syncthreads();
+    cluster.sync();
+
+    Waiter wt{p.status, p.limit_ns};
+    bool my_bad = false;
+    const bool writer = (rank == 0);
+
+    int c_prev = p.c_in ? p.c_in[0] : 128, f_prev = p.f_in ? p.f_in[0] : 0;
+
+    // ---- sparse phase: block rows [0, NBR) of phase ph (0: input y_c -> [O1 ; R x coarse cols], 1: y_f -> [O3 ; R x fine cols]).
+    // Eight lanes per block row.  Rows [0, HR) are hidden-layer rows (bias, relu, sent to all peers when send != 0),
+    // rows [HR, HR + NR) are this CTA's R rows (ph 1 completes R h, ph 0 keeps the partial for the next step).
+    auto sparse_phase = [&](int ph, const float *x, const float *bias) {
+        // Four lanes per block row (sub-group q = lane >> 2 of warp w takes block row q * SNW + w, so that the
+        // hidden-layer rows and the R rows are spread over all warps); each lane takes every fourth kept block.
+        const int l4 = lane & 3;
+        const int nrounds = (NBR + 8 * SNW - 1) / (8 * SNW);
+        for (int round = 0; round < nrounds; ++round) {
+            const int lbr_raw = round * 8 * SNW + (lane >> 2) * SNW + warp;
+            const bool valid = lbr_raw < NBR;
+            const int lbr = valid ? lbr_raw : 0;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            const int beg = brp[ph][lbr], end = valid ? brp[ph][lbr + 1] : beg;
+            for (int i = beg + l4; i < end; i += 4) {
+                const uint4 w0 = bval[ph][2 * i], w1 = bval[ph][2 * i + 1];
+                const float4 xv = *reinterpret_cast<const float4 *>(x + 4 * (int)bcol[ph][i]);
+                acc[0] = fmaf(bf16lo(w0.x), xv.x, fmaf(bf16hi(w0.x), xv.y, fmaf(bf16lo(w0.y), xv.z, fmaf(bf16hi(w0.y), xv.w, acc[0]))));
+                acc[1] = fmaf(bf16lo(w0.z), xv.x, fmaf(bf16hi(w0.z), xv.y, fmaf(bf16lo(w0.w), xv.z, fmaf(bf16hi(w0.w), xv.w, acc[1]))));
+                acc[2] = fmaf(bf16lo(w1.x), xv.x, fmaf(bf16hi(w1.x), xv.y, fmaf(bf16lo(w1.y), xv.z, fmaf(bf16hi(w1.y), xv.w, acc[2]))));
+                acc[3] = fmaf(bf16lo(w1.z), xv.x, fmaf(bf16hi(w1.z), xv.y, fmaf(bf16lo(w1.w), xv.z, fmaf(bf16hi(w1.w), xv.w, acc[3]))));
+            }
+            // four row sums over four lanes: two transposing steps leave row l4 in lane l4
+            const bool up2 = (l4 & 2) != 0;
+            const float s0 = up2 ? acc[0] : acc[2], k0 = up2 ? acc[2] : acc[0];
+            const float s1 = up2 ? acc[1] : acc[3], k1 = up2 ? acc[3] : acc[1];
+            const float t0 = k0 + __shfl_xor_sync(FULL, s0, 2);
+            const float t1 = k1 + __shfl_xor_sync(FULL, s1, 2);
+            const bool up1 = (l4 & 1) != 0;
+            const float v = (up1 ? t1 : t0) + __shfl_xor_sync(FULL, up1 ? t0 : t1, 1);
+            if (valid) {
+                const int row = 4 * lbr + l4;
+                if (row < HR) qvec[row] = fmaxf(v + bias[row], 0.f);
+                else if (ph) a_full[row - HR] = a_part[row - HR] + v;
+                else a_part[row - HR] = v;
+            }
+        }
+    };
+
+    // Gates of Eq. 2 for this CTA's UC units of one half, then publish them to all 16 CTAs.  The first GW warps
+    // each draw the sample redundantly (same logits, same uniform, same instructions -> same value) and then gate
+    // UC / GW units each, so that neither the gates nor the 16 x UC / 2 remote stores queue up in one warp.
+    constexpr int GW = 4;
+    const int UW = UC / GW;
+    auto load_g = [&](int half_g, long long s, float (&gv)[3]) {
+        const long long fr = ((p.step0 + s) * p.row_stride + (long long)p.stream0 * p.row_offset_mul) / p.hop;
+        const float *g = p.g + (size_t)fr * 3 * H + (half_g ? K : 0) + rank * UC + warp * UW + lane;
+#pragma unroll
+        for (int gate = 0; gate < 3; ++gate) gv[gate] = __ldg(g + gate * H);
+    };
+    auto gates = [&](int half_g, long long s, int drawn, const float (&gv)[3]) {
+        const int rb = half_g ? 3 * UC : 0;
+        const float *vec = half_g ? vecF : vecC;    // previous value of these units: still in the fp32 vector of that half
+        if (lane < UW) {
+            const int u0 = warp * UW + lane;
+            const float x0 = scale8(c_prev), x1 = scale8(f_prev), x2 = half_g ? scale8(drawn) : 0.f;
+            const float *Iu = sI + 3 * (rb + u0), *Ir = sI + 3 * (rb + UC + u0), *Ie = sI + 3 * (rb + 2 * UC + u0);
+            const float pu = a_full[rb + u0] + fmaf(Iu[0], x0, fmaf(Iu[1], x1, fmaf(Iu[2], x2, gv[0])));
+            const float pr = a_full[rb + UC + u0] + fmaf(Ir[0], x0, fmaf(Ir[1], x1, fmaf(Ir[2], x2, gv[1])));
+            const float pe = fmaf(Ie[0], x0, fmaf(Ie[1], x1, fmaf(Ie[2], x2, gv[2])));
+            const float u = sigmoidf_fast(pu), r = sigmoidf_fast(pr);
+            const float e = tanhf_fast(fmaf(r, a_full[rb + 2 * UC + u0], pe));
+            const float hn = fmaf(u, vec[rank * UC + u0], (1.0f - u) * e);
+            ynew[u0] = hn;
+            const int jj = (half_g ? K : 0) + rank * UC + u0;
+            if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
+            if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
+        }
+    };
+    // the UC freshly gated values -> every peer (warp w -> peer w, one coalesced store), after a CTA barrier
+    auto publish = [&](unsigned ytag) {
+        if (warp < SCS) {
+            for (int pr2 = lane; pr2 < UC / 2; pr2 += 32) {
+                const unsigned a = map_to_rank(smem_addr(ybuf + (size_t)(ytag & 1) * (K / 2) + (rank * UC) / 2 + pr2), warp);
+                st_cluster_ll(a, ynew[2 * pr2], ynew[2 * pr2 + 1], ytag);
+            }
+        }
+    };
+
+    // ---- prologue: R h of step 0 from the initial state, coarse gates of step 0
+    sparse_phase(0, vecC, sb1);
+    __syncthreads();
+    sparse_phase(1, vecF, sb3);
+    __syncthreads();
+    if (warp < GW) {
+        float gv0[3] = {0.f, 0.f, 0.f};
+        if (lane < UW) load_g(0, 0, gv0);
+        gates(0, 0, 0, gv0);
+    }
+    __syncthreads();
+    publish(1u);
+
+    const int l_kt0 = warp * NKL;
+    const int KSL = NKT / NKL;                   // warps that split K of the logits tile
+    const bool l_on = warp < KSL;
+
+#ifdef WRNN_PROFILE_SPARSE
+    long long st_ = clock64();
+#endif
+    const long long T = p.n_steps;
+#pragma unroll 1
+    for (long long n = 1; n <= 2 * T; ++n) {
+        const int half = (int)(n & 1);                 // 1: coarse half (input y_c(s)), 0: fine half (input y_f(s-1))
+        const long long s = n >> 1;
+        const bool last = n == 2 * T;
+        const unsigned tag = (unsigned)n, par = (unsigned)((n - 1) & 1);
+        float *vec = half ? vecC : vecF;
+
+        float u01 = 0.f, gv[3] = {0.f, 0.f, 0.f};
+        int forced = -1;
+        if (warp < GW) {
+            if (lane < UW && !last) load_g(half, s, gv);
+            if (half) { if (p.c_forced) forced = p.c_forced[s]; }
+            else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
+            u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
+        }
+
+        // ---- 1. the input half of the state from all 16 CTAs (published with tag n into buffer n & 1)
+#pragma unroll 1
+        for (int i = tid; i < K / 2; i += blockDim.x) {
+            const unsigned a = smem_addr(ybuf + (size_t)(n & 1) * (K / 2) + i);
+            uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
+            while (true) {
+                v = ld_shared_volatile_v4(a);
+                if (v.y == tag && v.w == tag) break;
+                if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+            }
+            vec[2 * i] = __uint_as_float(v.x); vec[2 * i + 1] = __uint_as_float(v.z);
+        }
+        if (__syncthreads_or(my_bad)) break;
+        SSTAMP(0);
+
+        // ---- 2. hidden layer of the head + this CTA's R rows (compressed block rows)
+        sparse_phase(half ? 0 : 1, vec, half ? sb1 : sb3);
+        __syncthreads();
+        // this CTA's HR hidden-layer values -> every peer, one coalesced 16-byte-per-lane store per peer (warp w -> peer w)
+        if (warp < SCS) {
+            for (int pr2 = lane; pr2 < HR / 2; pr2 += 32) {
+                const unsigned a = map_to_rank(smem_addr(qbuf + (size_t)par * (K / 2) + (rank * HR) / 2 + pr2), warp);
+                st_cluster_ll(a, qvec[2 * pr2], qvec[2 * pr2 + 1], tag);
+            }
+        }
+        SSTAMP(1);
+
+        // ---- 3. the cluster's hidden layer -> 16 logits rows of this CTA
+#pragma unroll 1
+        for (int i = tid; i < K / 2; i += blockDim.x) {
+            const unsigned a = smem_addr(qbuf + (size_t)par * (K / 2) + i);
+            uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
+            while (true) {
+                v = ld_shared_volatile_v4(a);
+                if (v.y == tag && v.w == tag) break;
+                if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 2 + 4 * half)) { my_bad = true; break; }
+            }
+            store_split(splQ, 2 * i, __uint_as_float(v.x));
+            store_split(splQ, 2 * i + 1, __uint_as_float(v.z));
+        }
+        if (__syncthreads_or(my_bad)) break;
+        SSTAMP(2);
+        if (l_on) {
+            float lo, hi;
+            mma_partial<NKL>(half ? wO2 : wO4, l_kt0, splQ, lane, lo, hi);
+            if ((lane & 3) == 0) { part[warp * 16 + (lane >> 2)] = lo; part[warp * 16 + (lane >> 2) + 8] = hi; }
+        }
+        __syncthreads();
+        SSTAMP(3);
+        if (warp == GW) {
+            // 16 logits of this CTA: lanes 0..7 finish one pair of rows each, then every peer gets the 8 pairs as one
+            // contiguous 128-byte piece (four store instructions, four peers each)
+            const float *bl = half ? sb2 : sb4;
+            const int r = 2 * (lane & 7);
+            float v0 = bl[r], v1 = bl[r + 1];
+            for (int w = 0; w < KSL; ++w) { v0 += part[w * 16 + r]; v1 += part[w * 16 + r + 1]; }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int peer = 4 * k + (lane >> 3);
+                const unsigned a = map_to_rank(smem_addr(lbuf + (size_t)par * 128 + (rank * 16) / 2 + (lane & 7)), peer);
+                st_cluster_ll(a, v0, v1, tag);
+            }
+        }
+
+        // ---- 4. warps 0..GW-1: the cluster's 256 logits -> draw; then the gates of the other half, published to the cluster
+        if (warp < GW) {
+            float l[8];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const unsigned a = smem_addr(lbuf + (size_t)par * 128 + 4 * lane + k);
+                uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
+                while (true) {
+                    v = ld_shared_volatile_v4(a);
+                    if (v.y == tag && v.w == tag) break;
+                    if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 3 + 4 * half)) { my_bad = true; break; }
+                }
+                l[2 * k] = __uint_as_float(v.x); l[2 * k + 1] = __uint_as_float(v.z);
+            }
+            my_bad = __any_sync(FULL, my_bad);
+            SSTAMP(4);
+            int drawn = warp_softmax_draw_fast(l, u01, lane);
+            if (writer && warp == 0) {
+                if (p.dbg_logits) {
+                    float *d = p.dbg_logits + (size_t)(n - 1) * 256 + 8 * lane;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) d[k] = l[k];
+                }
+                if (lane == 0) {
+                    if (half) { if (p.c_out) p.c_out[s] = (uint8_t)drawn; }
+                    else      { if (p.f_out) p.f_out[s - 1] = (uint8_t)drawn; }
+                }
+            }
+            if (forced >= 0) drawn = forced;
+            if (!half) {
+                if (writer && warp == 0 && lane == 0 && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + drawn - 32768);
+                f_prev = drawn;
+            }
+            SSTAMP(5);
+            if (!last && !my_bad) gates(half, s, drawn, gv);
+            if (half) c_prev = drawn;
+            SSTAMP(6);
+        }
+        if (__syncthreads_or(my_bad)) break;
+        if (!last) publish((unsigned)(n + 1));
+    }
+
+    const int any_bad = __syncthreads_or(my_bad);
+    if (writer && !any_bad) {
+        if (p.h_out) for (int i = tid; i < K; i += blockDim.x) { p.h_out[i] = vecC[i]; p.h_out[K + i] = vecF[i]; }
+        if (tid == 0) {
+            if (p.c_st_out) p.c_st_out[0] = (uint8_t)c_prev;
+            if (p.f_st_out) p.f_st_out[0] = (uint8_t)f_prev;
+        }
+    }
+    cluster.sync();
+}
+
+// ---------------------------------------------------------------------------------------------
+static size_t a16(size_t x) { return (x + 15) & ~(size_t)15; }
+
+static int sparse_smem_bytes(const SparsePack &k)
+{
+    size_t b = k.blob_bytes;
+    b += (size_t)3 * k.K * 4;                      // vecC, vecF, qvec
+    b += (size_t)2 * 6 * k.UC * 4;                 // a_part, a_full
+    b += 256 * 4;                                  // part
+    b += (size_t)((k.UC + 3) & ~3) * 4;            // ynew
+    b += (size_t)4 * k.K * 2;                      // split image of q
+    b += (size_t)2 * k.K * 16;                     // ybuf, qbuf: [2][K/2] x 16 B each
+    b += 256 * 16;                                 // lbuf
+    return (int)b;
+}
+
+static uint16_t bf16_bits_s(float rounded)
+{
+    uint32_t b;
+    std::memcpy(&b, &rounded, 4);
+    return (uint16_t)(b >> 16);
+}
+
+int sparse_supported(const wrnn_model *m, int batch, std::string *why)
+{
+    if (batch != 1) { if (why) *why = "single-stream kernel"; return WRNN_ERR_UNSUPPORTED; }
+    if (!m->sparse_pack) { if (why) *why = "model was not packed for the sparse cluster kernel"; return WRNN_ERR_UNSUPPORTED; }
+    return WRNN_OK;
+}
+
+static void *sparse_fn() { return (void *)sparse_cluster_kernel<8>; }
+
+static void sparse_fill_launch(const SparsePack &k, cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at, cudaStream_t s, bool coop)
+{
+    std::memset(cfg, 0, sizeof(*cfg));
+    cfg->gridDim = dim3(SCS);
+    cfg->blockDim = dim3(SNW * 32);
+    cfg->dynamicSmemBytes = k.smem_bytes;
+    cfg->stream = s;
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = SCS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeCooperative;
+    at[1].val.cooperative = 1;
+    cfg->attrs = at;
+    cfg->numAttrs = coop ? 2 : 1;
+}
+
+int sparse_prepare(wrnn_model *m)
+{
+    const int H = m->H, Hh = H / 2;
+    if (m->dtype != WRNN_BF16) { m->err = "sparse cluster kernel stores bf16 weights"; return WRNN_ERR_UNSUPPORTED; }
+    if (!m->sparse) { m->err = "model has no block masks"; return WRNN_ERR_UNSUPPORTED; }
+    if (Hh != 1024) { m->err = "only H/2 = 1024 is instantiated (8 warps x 8 k-tiles for the logits tile)"; return WRNN_ERR_UNSUPPORTED; }
+    SparsePack k;
+    k.H = H; k.K = Hh; k.NKT = Hh / 16; k.UC = Hh / SCS; k.HR = Hh / SCS;
+    k.NBR = (k.HR + 6 * k.UC) / 4;
+    const int UC = k.UC, HR = k.HR, NBR = k.NBR, Kb = Hh / 4;      // Kb: block columns per half
+
+    // kept blocks of each phase of each CTA
+    struct Blk { uint16_t col; const float *v; };
+    std::vector<std::vector<std::vector<Blk>>> rows(SCS * 2);      // [cta * 2 + phase][local block row] -> blocks
+    const BsrHost *Oa[2] = {&m->hO1, &m->hO3};
+    for (int cta = 0; cta < SCS; ++cta)
+        for (int ph = 0; ph < 2; ++ph) {
+            auto &R = rows[cta * 2 + ph];
+            R.assign(NBR, {});
+            for (int lbr = 0; lbr < NBR; ++lbr) {
+                if (lbr < HR / 4) {
+                    const BsrHost &M = *Oa[ph];
+                    const int br = cta * (HR / 4) + lbr;
+                    for (int i = M.row_ptr[br]; i < M.row_ptr[br + 1]; ++i) R[lbr].push_back({M.col[i], &M.vals[(size_t)i * 16]});
+                } else {
+                    const int q = lbr - HR / 4;                    // (half * 3 + gate) * (UC / 4) + u4
+                    const int half = q / (3 * (UC / 4)), gate = (q / (UC / 4)) % 3, u4 = q % (UC / 4);
+                    const int br = (gate * H + half * Hh + cta * UC) / 4 + u4;
+                    for (int i = m->hR.row_ptr[br]; i < m->hR.row_ptr[br + 1]; ++i) {
+                        const int bc = m->hR.col[i];
+                        if ((bc >= Kb) == (ph == 1)) R[lbr].push_back({(uint16_t)(bc - ph * Kb), &m->hR.vals[(size_t)i * 16]});
+                    }
+                }
+            }
+        }
+    int max_nnz = 0;
+    for (auto &R : rows) { int n = 0; for (auto &r : R) n += (int)r.size(); max_nnz = std::max(max_nnz, n); }
+    k.max_nnz = (max_nnz + 7) & ~7;
+
+    size_t off = 0;
+    for (int ph = 0; ph < 2; ++ph) {
+        k.off_brp[ph] = off; off = a16(off + (size_t)(NBR + 1) * 4);
+        k.off_col[ph] = off; off = a16(off + (size_t)k.max_nnz * 2);
+        k.off_val[ph] = off; off = a16(off + (size_t)k.max_nnz * 32);
+    }
+    const size_t frag = (size_t)k.NKT * 512;
+    k.off_o2 = off; off += frag;
+    k.off_o4 = off; off += frag;
+    k.off_small = off; off = a16(off + ((size_t)6 * UC * 3 + 2 * HR + 32) * 4);
+    k.blob_bytes = off;
+    k.smem_bytes = sparse_smem_bytes(k);
+
+    cudaDeviceProp prop;
+    cudaGetDeviceProperties(&prop, m->device);
+    if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "pruned model does not fit the shared memory of one cluster"; return WRNN_ERR_UNSUPPORTED; }
+    if (cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
+        cudaGetLastError(); m->err = "cannot configure the 16-CTA cluster kernel"; return WRNN_ERR_UNSUPPORTED;
+    }
+    cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
+    sparse_fill_launch(k, &cfg, at, 0, false);
+    int max_clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&max_clusters, sparse_fn(), &cfg) != cudaSuccess || max_clusters < 1) {
+        cudaGetLastError(); m->err = "no 16-CTA cluster can be co-resident on this device"; return WRNN_ERR_UNSUPPORTED;
+    }
+
+    std::vector<uint8_t> blob((size_t)SCS * k.blob_bytes, 0);
+    const BsrHost *Ob[2] = {&m->hO2, &m->hO4};
+    int64_t kept_bytes = 0;
+    for (int cta = 0; cta < SCS; ++cta) {
+        uint8_t *base = blob.data() + (size_t)cta * k.blob_bytes;
+        for (int ph = 0; ph < 2; ++ph) {
+            int *brp = reinterpret_cast<int *>(base + k.off_brp[ph]);
+            uint16_t *col = reinterpret_cast<uint16_t *>(base + k.off_col[ph]);
+            uint16_t *val = reinterpret_cast<uint16_t *>(base + k.off_val[ph]);
+            int n = 0;
+            for (int lbr = 0; lbr < NBR; ++lbr) {
+                brp[lbr] = n;
+                for (const Blk &b : rows[cta * 2 + ph][lbr]) {
+                    col[n] = b.col;
+                    for (int e = 0; e < 16; ++e) val[(size_t)n * 16 + e] = bf16_bits_s(b.v[e]);
+                    ++n;
+                }
+            }
+            brp[NBR] = n;
+            kept_bytes += (int64_t)n * 34 + (int64_t)(NBR + 1) * 4;
+        }
+        // dense O2 / O4: 16 rows of this CTA as one tile of A fragments (natural column order)
+        for (int h = 0; h < 2; ++h) {
+            uint16_t *dst = reinterpret_cast<uint16_t *>(base + (h ? k.off_o4 : k.off_o2));
+            std::vector<uint16_t> dense((size_t)16 * Hh, 0);
+            const BsrHost &M = *Ob[h];
+            for (int r = 0; r < 16; ++r) {
+                const int row = cta * 16 + r, br = row / 4, rr = row % 4;
+                for (int i = M.row_ptr[br]; i < M.row_ptr[br + 1]; ++i)
+                    for (int c = 0; c < 4; ++c) dense[(size_t)r * Hh + 4 * M.col[i] + c] = bf16_bits_s(M.vals[(size_t)i * 16 + 4 * rr + c]);
+            }
+            for (int kt = 0; kt < k.NKT; ++kt)
+                for (int lane = 0; lane < 32; ++lane) {
+                    const int g = lane >> 2, t = lane & 3;
+                    uint16_t *o = dst + ((size_t)kt * 32 + lane) * 8;
+                    const int rsel[4] = {g, g + 8, g, g + 8}, csel[4] = {2 * t, 2 * t, 2 * t + 8, 2 * t + 8};
+                    for (int q = 0; q < 4; ++q)
+                        for (int j = 0; j < 2; ++j) o[2 * q + j] = dense[(size_t)rsel[q] * Hh + 16 * kt + csel[q] + j];
+                }
+        }
+        float *sm = reinterpret_cast<float *>(base + k.off_small);
+        for (int rr = 0; rr < 6 * UC; ++rr) {
+            const int half = rr / (3 * UC), gate = (rr / UC) % 3, u = rr % UC;
+            const int mrow = gate * H + half * Hh + cta * UC + u;
+            for (int c = 0; c < 3; ++c) sm[rr * 3 + c] = m->hI[(size_t)mrow * 3 + c];
+        }
+        float *b = sm + 6 * UC * 3;
+        for (int r = 0; r < HR; ++r) { b[r] = m->hb1[cta * HR + r]; b[HR + r] = m->hb3[cta * HR + r]; }
+        b += 2 * HR;
+        for (int r = 0; r < 16; ++r) { b[r] = m->hb2[cta * 16 + r]; b[16 + r] = m->hb4[cta * 16 + r]; }
+    }
+    SparsePack *pk = new SparsePack(k);
+    if (cudaMalloc((void **)&pk->d_blob, blob.size()) != cudaSuccess ||
+        cudaMemcpy(pk->d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError(); cudaFree(pk->d_blob); delete pk;
+        m->err = "device allocation for the sparse cluster kernel failed";
+        return WRNN_ERR_NOMEM;
+    }
+    pk->weight_bytes_per_step = kept_bytes + (int64_t)2 * 256 * Hh * 2 + (int64_t)3 * H * 3 * 4;
+    m->sparse_pack = pk;
+    return WRNN_OK;
+}
+
+void sparse_destroy(wrnn_model *m)
+{
+    if (!m->sparse_pack) return;
+    cudaFree(m->sparse_pack->d_blob);
+    delete m->sparse_pack;
+    m->sparse_pack = nullptr;
+}
+
+int sparse_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem, int64_t *weight_bytes)
+{
+    (void)batch;
+    const SparsePack &k = *m->sparse_pack;
+    if (n_ctas) *n_ctas = SCS;
+    if (n_threads) *n_threads = SNW * 32;
+    if (smem) *smem = k.smem_bytes;
+    if (weight_bytes) *weight_bytes = k.weight_bytes_per_step;
+    return WRNN_OK;
+}
+
+int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
+{
+    const SparsePack &k = *m->sparse_pack;
+    SparseParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.H = k.H; p.K = k.K; p.NKT = k.NKT; p.UC = k.UC; p.HR = k.HR; p.NBR = k.NBR;
+    for (int ph = 0; ph < 2; ++ph) { p.off_brp[ph] = k.off_brp[ph]; p.off_col[ph] = k.off_col[ph]; p.off_val[ph] = k.off_val[ph]; }
+    p.off_o2 = k.off_o2; p.off_o4 = k.off_o4; p.off_small = k.off_small; p.blob_bytes = k.blob_bytes;
+    p.n_steps = a.n_steps; p.step0 = a.step0; p.stream0 = a.stream0; p.seed = a.seed;
+    p.n_frames = m->cond_dim ? a.n_frames : 1;
+    p.hop = m->cond_dim ? a.hop : 1;
+    p.row_stride = m->cond_dim ? a.row_stride : 0;
+    p.row_offset_mul = m->cond_dim ? a.row_offset_mul : 0;
+    p.blob = k.d_blob; p.g = m->g;
+    p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in; p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
+    p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
+    p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
+    p.status = m->status;
+    p.limit_ns = 2000000000ull;
+
+    if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
+    cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
+    const char *no_coop = getenv("WRNN_NO_COOP");
+    sparse_fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
+    cudaError_t e = cudaLaunchKernelEx(&cfg, sparse_cluster_kernel<8>, p);
+    if (e != cudaSuccess) {
+        m->err = std::string("sparse cluster kernel launch failed: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        return WRNN_ERR_CUDA;
+    }
+    ++g_launches;
+    return WRNN_OK;
+}
+
+}  // namespace wrnn
+
+#ifdef WRNN_PROFILE_SPARSE
+extern "C" int wrnn_debug_sparse_prof(long long *out16, int reset)
+{
+    if (reset) { long long z[16] = {0}; return cudaMemcpyToSymbol(wrnn::g_sprof, z, sizeof(z)) == cudaSuccess ? 0 : 4; }
+    return cudaMemcpyFromSymbol(out16, wrnn::g_sprof, 16 * sizeof(long long)) == cudaSuccess ? 0 : 4;
+}
+#endif

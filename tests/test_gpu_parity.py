@@ -258,6 +258,7 @@ def test_config2_sparse_bf16(env):
     om = orc.OracleModel(w, wl.dtype, masks)
     m = B.wrnn_create(w, wl.dtype, masks)
     try:
+        assert B.wrnn_launch_info(m, 1)["kernel"] == B.WRNN_KERNEL_SPARSE        # one 16-CTA cluster, all exchanges in DSMEM
         r = pu.teacher_forced_parity(torch, B, m, om, cond, 1500, 1, SEED)
         _report("config2/sparse", r)
         _tol_check(r, wl.dtype)
@@ -274,6 +275,22 @@ def test_config2_sparse_bf16(env):
         assert np.array_equal(np.concatenate([a, b], axis=1), free)
     finally:
         B.wrnn_destroy(m)
+
+
+def test_sparse_cluster_and_generic_kernels_agree(env):
+    """The block-sparse model through the generic block-row kernel and the single-cluster kernel."""
+    torch, B = env
+    wl = synth.WORKLOADS[2]
+    w, masks, cond = synth.build_workload(wl)
+    om = orc.OracleModel(w, wl.dtype, masks)
+    res = om.run(cond, 400, 1, SEED, dump=True)
+    for kern in (B.WRNN_KERNEL_GENERIC, B.WRNN_KERNEL_SPARSE):
+        m = B.wrnn_create(w, wl.dtype, masks, kernel=kern)
+        try:
+            r = pu.teacher_forced_parity(torch, B, m, om, cond, 400, 1, SEED, oracle_free=res)
+            _tol_check(r, wl.dtype)
+        finally:
+            B.wrnn_destroy(m)
 
 
 def test_config3_subscale_fold_batch16(env):

@@ -254,7 +254,7 @@ def main():
         peaks = measured_peaks()
         us_per_sample_step = ms_per_step * 1e3 / n_steps
         wbytes = info["weight_bytes_per_step"]
-        if wl.batch >= 64:
+        if wl.batch >= 2:
             # dense contraction: algorithmic flops of R, O1..O4 products per lock-step
             H, Hh = wl.H, wl.H // 2
             flops = 2.0 * wl.batch * (3 * H * H + 2 * Hh * Hh + 2 * 256 * Hh)

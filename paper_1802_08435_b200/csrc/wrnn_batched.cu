@@ -15,8 +15,16 @@
 //   Sc  draw c_t (one warp per row)           Gf  fine gates -> y_f (element-wise)
 //   O3  q_f = relu(O3 y_f + b3)      O4  l_f = O4 q_f + b4
 //   Sf  draw f_t, emit the sample
+//
+// With 16 or more rows, phase A -- the [B x H] . [H x 3H] recurrent contraction, 79 % of the flops -- runs on the
+// fifth-generation tensor cores instead: one CTA per (128 rows of R) x (block of BN rows of the batch), the weight
+// tile and the hi / lo activation tiles brought in by TMA (128-byte swizzle, three-stage mbarrier ring), one
+// elected thread issuing tcgen05.mma (M = 128, N = BN, K = 16, bf16 -> fp32) into a TMEM accumulator, and four
+// warps reading it back with tcgen05.ld for the epilogue.  Every mbarrier wait is bounded.
+#include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdlib>
 #include <cstring>
 
 #include "wrnn_internal.h"
@@ -35,6 +43,12 @@ struct BatchedPack {
     uint8_t *c_cur = nullptr, *c_prev = nullptr, *f_prev = nullptr;
     unsigned long long *bar = nullptr;
     int64_t weight_bytes = 0;
+    // tcgen05 path of phase A: plain row-major bf16 copies (K-major operands for TMA) and their tensor maps
+    bool tc = false;
+    int tc_rows = 0;                               // rows of the hrm arrays (max batch rounded up to 64)
+    __nv_bfloat16 *Rrm = nullptr;                  // [3H][H]
+    __nv_bfloat16 *hrm[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};   // [buffer][part] -> [tc_rows][H]
+    CUtensorMap tmR, tmH64[2][2], tmH16[2][2];     // box 64 x 128 (R), 64 x 64 and 64 x 16 (activations)
 };
 
 struct BatchedParams {
@@ -58,6 +72,10 @@ struct BatchedParams {
     unsigned long long *bar;
     DevStatus *status;
     unsigned long long limit_ns;
+    int tc;                                     // phase A on tcgen05
+    __nv_bfloat16 *hrm[2][2];                   // [buffer][part] row-major hi / lo state
+    alignas(64) CUtensorMap tmR;
+    alignas(64) CUtensorMap tmH[2][2];
 };
 
 // bf16 index of (row b, element k, part) inside an activation image with nkt k-tiles:
@@ -152,6 +170,55 @@ __device__ __forceinline__ void tile_gemm(const uint4 *Af, int nk, const uint2 *
     }
 }
 
+// ---- tcgen05 / TMA / mbarrier helpers (phase A with 16 or more rows)
+constexpr int TC_STAGES = 3, TC_BM = 128, TC_BK = 64;
+constexpr unsigned long long TC_WAIT_NS = 2000000000ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) { asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory"); }
+// bounded: false when the phase did not complete within about two seconds
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    unsigned long long t0 = 0;
+    for (unsigned n = 1;; ++n) {
+        uint32_t ok;
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0,1,0,p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        if (ok) return true;
+        if ((n & 255u) == 0) {
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > TC_WAIT_NS) return false;
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y) : "memory");
+}
+// shared-memory matrix descriptor of a K-major tile with 128-byte swizzle (rows of 128 bytes, 8-row atoms of 1 KB)
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr)
+{
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+                 ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+                   "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+                 : "r"(taddr));
+}
+
 __device__ __forceinline__ long long frame_of_b(const BatchedParams &p, long long s, int gb)
 {
     return ((p.step0 + s) * p.row_stride + (long long)(p.stream0 + (unsigned)gb) * p.row_offset_mul) / p.hop;
@@ -159,7 +226,8 @@ __device__ __forceinline__ long long frame_of_b(const BatchedParams &p, long lon
 
 // Gates of Eq. 2 for one (row, unit); writes the fp32 state, its image and the optional dumps.
 __device__ __forceinline__ void gate_unit_b(const BatchedParams &p, int j, int gb, long long s, const float *hcur, float *hnext,
-                                            __nv_bfloat16 *img_next, float x0, float x1, float x2)
+                                            __nv_bfloat16 *img_next, __nv_bfloat16 *hrm_hi, __nv_bfloat16 *hrm_lo, float x0, float x1,
+                                            float x2)
 {
     const int H = p.H;
     const float *a = p.a_buf + (size_t)gb * p.G;
@@ -173,6 +241,11 @@ __device__ __forceinline__ void gate_unit_b(const BatchedParams &p, int j, int g
     const float hn = fmaf(u, __ldcg(hcur + (size_t)gb * H + j), (1.0f - u) * e);
     hnext[(size_t)gb * H + j] = hn;
     img_store(img_next, gb, j, p.NKT_R, hn);
+    if (hrm_hi) {
+        const __nv_bfloat16 hi = __float2bfloat16_rn(hn);
+        hrm_hi[(size_t)gb * H + j] = hi;
+        hrm_lo[(size_t)gb * H + j] = __float2bfloat16_rn(hn - __bfloat162float(hi));
+    }
     if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * p.batch + gb) * p.G; d[j] = u; d[H + j] = r; d[2 * H + j] = e; }
     if (p.dbg_h) p.dbg_h[((size_t)s * p.batch + gb) * H + j] = hn;
 }
@@ -184,8 +257,9 @@ __device__ long long g_bprof[32];
 #define BSTAMP(i) do { } while (0)
 #endif
 
-template <int NT>
-__global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParams p)
+// BN: rows of the batch per tcgen05 tile of phase A (0: phase A stays on mma.sync).
+template <int NT, int BN>
+__global__ void __launch_bounds__(512, 1) batched_step_kernel(const __grid_constant__ BatchedParams p)
 {
 #ifdef WRNN_PROFILE_BATCHED
     long long bt_ = clock64();
@@ -199,25 +273,56 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
     const int g4 = lane >> 2, t4 = lane & 3;
     const bool active = blockIdx.x < p.NSB * p.NMG;
     const int sb = blockIdx.x % p.NSB, mg = blockIdx.x / p.NSB;
+    const bool tc = BN > 0 && p.tc != 0;
 
     GridBarrier bar{p.bar, p.status, 0ull, p.limit_ns};
+    bool failed = false;
+
+    // ---- tcgen05 set-up: mbarrier ring, TMEM accumulator of BN fp32 columns (allocated by warp 1, freed at exit)
+    __shared__ __align__(8) uint64_t tc_full[TC_STAGES], tc_empty[TC_STAGES], tc_done;
+    __shared__ uint32_t tc_slot;
+    uint32_t tmem_base = 0;
+    unsigned tc_kb = 0, tc_tasks = 0;            // running k-block and task counters (mbarrier phases)
+    constexpr int TMEM_COLS = BN >= 64 ? 64 : 32;
+    if (tc) {
+        if (tid == 0) {
+            for (int i = 0; i < TC_STAGES; ++i) { mbar_init(smem_u32(&tc_full[i]), 1); mbar_init(smem_u32(&tc_empty[i]), 1); }
+            mbar_init(smem_u32(&tc_done), 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        if (warp == 1) {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tc_slot)), "r"(TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        tmem_base = tc_slot;
+    }
 
     float *hc = p.hf0, *hn = p.hf1;
     __nv_bfloat16 *ic = p.himg0, *in = p.himg1;
-    // initial state: fp32 and image (rows beyond the batch stay zero)
+    int cur = 0;                                  // buffer of the row-major hi / lo state that holds h_{t-1}
+    // initial state: fp32 and images (rows beyond the batch stay zero)
     for (int i = gtid; i < Bp * H; i += nthreads) {
         const int b = i / H, j = i - b * H;
         const float x = (b < B && p.h_in) ? p.h_in[i] : 0.f;
         hc[i] = x;
         img_store(ic, b, j, p.NKT_R, x);
         img_store(in, b, j, p.NKT_R, 0.f);
+        if (tc) {
+            const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+            p.hrm[0][0][i] = hi; p.hrm[0][1][i] = __float2bfloat16_rn(x - __bfloat162float(hi));
+            p.hrm[1][0][i] = __float2bfloat16_rn(0.f); p.hrm[1][1][i] = __float2bfloat16_rn(0.f);
+        }
     }
     for (int i = gtid; i < Bp * Hh; i += nthreads) img_store(p.qimg, i / Hh, i % Hh, p.NKT_H, 0.f);
     for (int i = gtid; i < B; i += nthreads) {
         p.c_prev[i] = p.c_in ? p.c_in[i] : (uint8_t)128;
         p.f_prev[i] = p.f_in ? p.f_in[i] : (uint8_t)0;
     }
-    if (!bar.sync(-1, 0)) return;
+    if (tc) asm volatile("fence.proxy.async.global;" ::: "memory");     // generic-proxy writes before TMA reads
+    if (!bar.sync(-1, 0)) failed = true;
 
     // Generic contraction phase: rows [0, n_mt * 16) of a fragment-packed matrix with nk k-tiles against the
     // image slice [kt0, kt0 + nk) of `img`; `epi(row, stream, value)` consumes the results.
@@ -240,23 +345,89 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
         }
     };
 
-    for (long long s = 0; s < p.n_steps; ++s) {
+    // Phase A on tcgen05: CTA (mtile, nblk) computes a[nblk * BN .. + BN][mtile * 128 .. + 128] = R tile . (h_hi + h_lo)^T.
+    // warp 0 / lane 0 feeds the TMA ring, warp 1 / lane 0 issues the MMAs, warps 4..7 drain the TMEM accumulator.
+    auto phase_a_tc = [&]() {
+        const int n_mt = (3 * H) / TC_BM, n_nb = (Bp + BN - 1) / (BN > 0 ? BN : 1), nkb = H / TC_BK;
+        const bool mine = (int)blockIdx.x < n_mt * n_nb;
+        if (mine) {
+            const int mtile = blockIdx.x % n_mt, nblk = blockIdx.x / n_mt;
+            uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+            constexpr uint32_t A_BYTES = TC_BM * TC_BK * 2, B_BYTES = (BN > 0 ? BN : 1) * TC_BK * 2, STAGE_BYTES = A_BYTES + 2 * B_BYTES;
+            const uint32_t ring0 = smem_u32(ring);
+            bool ok = true;
+            if (warp == 0 && lane == 0) {
+                asm volatile("fence.proxy.async;" ::: "memory");         // earlier generic-proxy use of this shared memory and of h
+                for (int kb = 0; kb < nkb; ++kb) {
+                    const unsigned it = tc_kb + kb, st = it % TC_STAGES, ph = (it / TC_STAGES) & 1;
+                    if (!mbar_wait(smem_u32(&tc_empty[st]), ph ^ 1)) { ok = false; break; }
+                    const uint32_t fb = smem_u32(&tc_full[st]), base = ring0 + st * STAGE_BYTES;
+                    mbar_expect_tx(fb, STAGE_BYTES);
+                    tma_load_2d(base, &p.tmR, fb, kb * TC_BK, mtile * TC_BM);
+                    tma_load_2d(base + A_BYTES, &p.tmH[cur][0], fb, kb * TC_BK, nblk * BN);
+                    tma_load_2d(base + A_BYTES + B_BYTES, &p.tmH[cur][1], fb, kb * TC_BK, nblk * BN);
+                }
+            } else if (warp == 1 && lane == 0) {
+                // instruction descriptor: D fp32, A / B bf16, both K-major, N = BN, M = 128
+                const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+                for (int kb = 0; kb < nkb; ++kb) {
+                    const unsigned it = tc_kb + kb, st = it % TC_STAGES, ph = (it / TC_STAGES) & 1;
+                    if (!mbar_wait(smem_u32(&tc_full[st]), ph)) { ok = false; break; }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t base = ring0 + st * STAGE_BYTES;
+                    const uint64_t da = umma_desc_sw128(base), dhi = umma_desc_sw128(base + A_BYTES), dlo = umma_desc_sw128(base + A_BYTES + B_BYTES);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 16; ++k) {                 // 32 bytes along K per MMA inside the swizzle atom
+                        umma_bf16(tmem_base, da + 2 * k, dhi + 2 * k, idesc, (kb | k) ? 1u : 0u);
+                        umma_bf16(tmem_base, da + 2 * k, dlo + 2 * k, idesc, 1u);
+                    }
+                    umma_commit(smem_u32(&tc_empty[st]));
+                }
+                if (ok) umma_commit(smem_u32(&tc_done));
+            } else if (warp >= 4 && warp < 8) {
+                if (mbar_wait(smem_u32(&tc_done), tc_tasks & 1)) {
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const int sub = warp & 3;
+                    const int row = mtile * TC_BM + sub * 32 + lane;
+#pragma unroll
+                    for (int c0 = 0; c0 < BN; c0 += 16) {
+                        uint32_t r[16];
+                        tmem_ld16(tmem_base + ((uint32_t)(sub * 32) << 16) + c0, r);
+                        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const int b = nblk * BN + c0 + c;
+                            if (b < B) p.a_buf[(size_t)b * p.G + row] = __uint_as_float(r[c]);
+                        }
+                    }
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                } else ok = false;
+            }
+            if (!ok && atomicCAS(&p.status->code, DEV_OK, DEV_TIMEOUT) == DEV_OK) { p.status->cta = blockIdx.x; p.status->step = -2; p.status->phase = 1; }
+            tc_kb += nkb; ++tc_tasks;
+        }
+        __syncthreads();
+    };
+
+    for (long long s = 0; s < p.n_steps && !failed; ++s) {
+        __nv_bfloat16 *nhi = tc ? p.hrm[cur ^ 1][0] : nullptr, *nlo = tc ? p.hrm[cur ^ 1][1] : nullptr;
         // ---- A: a = R h_{t-1}
         BSTAMP(31);
-        contraction(p.Rf, 3 * H / 16, p.NKT_R, ic, p.NKT_R, 0, [&](int row, int b, float v) { p.a_buf[(size_t)b * p.G + row] = v; });
+        if (tc) phase_a_tc();
+        else contraction(p.Rf, 3 * H / 16, p.NKT_R, ic, p.NKT_R, 0, [&](int row, int b, float v) { p.a_buf[(size_t)b * p.G + row] = v; });
         BSTAMP(0);
-        if (!bar.sync((int)s, 1)) return;
+        if (!bar.sync((int)s, 1)) { failed = true; break; }
         BSTAMP(1);
         // ---- Gc: coarse gates
         for (int i = gtid; i < B * Hh; i += nthreads) {
             const int gb = i / Hh, j = i - gb * Hh;
-            gate_unit_b(p, j, gb, s, hc, hn, in, scale8(__ldcg(p.c_prev + gb)), scale8(__ldcg(p.f_prev + gb)), 0.f);
+            gate_unit_b(p, j, gb, s, hc, hn, in, nhi, nlo, scale8(__ldcg(p.c_prev + gb)), scale8(__ldcg(p.f_prev + gb)), 0.f);
         }
         BSTAMP(2);
-        if (!bar.sync((int)s, 2)) return;
+        if (!bar.sync((int)s, 2)) { failed = true; break; }
         BSTAMP(3);
 
-        for (int head = 0; head < 2; ++head) {
+        for (int head = 0; head < 2 && !failed; ++head) {
             const uint4 *Oa = head ? p.O3f : p.O1f, *Ob = head ? p.O4f : p.O2f;
             const float *ba = head ? p.b3 : p.b1, *bb = head ? p.b4 : p.b2;
             // ---- O1 / O3: hidden layer on this half of the new state (k-tiles [head * H/32, +H/32) of its image)
@@ -264,7 +435,7 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
                 img_store(p.qimg, b, row, p.NKT_H, fmaxf(v + (ba ? ba[row] : 0.f), 0.f));
             });
             BSTAMP(4 + 8 * head);
-            if (!bar.sync((int)s, 3 + 4 * head)) return;
+            if (!bar.sync((int)s, 3 + 4 * head)) { failed = true; break; }
             BSTAMP(5 + 8 * head);
             // ---- O2 / O4: logits
             contraction(Ob, 16, p.NKT_H, p.qimg, p.NKT_H, 0, [&](int row, int b, float v) {
@@ -273,7 +444,7 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
                 if (p.dbg_logits) p.dbg_logits[(((size_t)s * B + b) * 2 + head) * 256 + row] = l;
             });
             BSTAMP(6 + 8 * head);
-            if (!bar.sync((int)s, 4 + 4 * head)) return;
+            if (!bar.sync((int)s, 4 + 4 * head)) { failed = true; break; }
             BSTAMP(7 + 8 * head);
             // ---- Sc / Sf: softmax + inverse-CDF draw, one warp per row
             for (int gb = gw; gb < B; gb += nw) {
@@ -284,14 +455,12 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
                 const float u = uniform24(p.seed, p.stream0 + (unsigned)gb, (unsigned long long)(p.step0 + s), head);
                 int idx = warp_softmax_draw(l, u, lane);
                 const size_t o = (size_t)gb * p.n_steps + s;
-                if (head == 0) {
-                    if (lane == 0) {
+                if (lane == 0) {
+                    if (head == 0) {
                         if (p.c_out) p.c_out[o] = (uint8_t)idx;
                         if (p.c_forced) idx = p.c_forced[o];
                         p.c_cur[gb] = (uint8_t)idx;
-                    }
-                } else {
-                    if (lane == 0) {
+                    } else {
                         if (p.f_out) p.f_out[o] = (uint8_t)idx;
                         if (p.f_forced) idx = p.f_forced[o];
                         const int c = __ldcg(p.c_cur + gb);
@@ -302,28 +471,37 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const BatchedParam
                 }
             }
             BSTAMP(8 + 8 * head);
-            if (!bar.sync((int)s, 5 + 4 * head)) return;
+            if (!bar.sync((int)s, 5 + 4 * head)) { failed = true; break; }
             BSTAMP(9 + 8 * head);
             if (head == 0) {
                 // ---- Gf: fine gates, now that c_t is known (it reaches only these rows, Section 2)
                 for (int i = gtid; i < B * Hh; i += nthreads) {
                     const int gb = i / Hh, j = Hh + (i - gb * Hh);
-                    gate_unit_b(p, j, gb, s, hc, hn, in, scale8(__ldcg(p.c_prev + gb)), scale8(__ldcg(p.f_prev + gb)),
+                    gate_unit_b(p, j, gb, s, hc, hn, in, nhi, nlo, scale8(__ldcg(p.c_prev + gb)), scale8(__ldcg(p.f_prev + gb)),
                                 scale8(__ldcg(p.c_cur + gb)));
                 }
+                if (tc) asm volatile("fence.proxy.async.global;" ::: "memory");
                 BSTAMP(10);
-                if (!bar.sync((int)s, 6)) return;
+                if (!bar.sync((int)s, 6)) { failed = true; break; }
                 BSTAMP(11);
             }
         }
         { float *t = hc; hc = hn; hn = t; }
         { __nv_bfloat16 *t = ic; ic = in; in = t; }
+        cur ^= 1;
     }
 
-    if (p.h_out) for (int i = gtid; i < B * H; i += nthreads) p.h_out[i] = __ldcg(hc + i);
-    for (int i = gtid; i < B; i += nthreads) {
-        if (p.c_st_out) p.c_st_out[i] = __ldcg(p.c_prev + i);
-        if (p.f_st_out) p.f_st_out[i] = __ldcg(p.f_prev + i);
+    if (!failed) {
+        if (p.h_out) for (int i = gtid; i < B * H; i += nthreads) p.h_out[i] = __ldcg(hc + i);
+        for (int i = gtid; i < B; i += nthreads) {
+            if (p.c_st_out) p.c_st_out[i] = __ldcg(p.c_prev + i);
+            if (p.f_st_out) p.f_st_out[i] = __ldcg(p.f_prev + i);
+        }
+    }
+    if (tc) {
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncthreads();
+        if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -335,16 +513,25 @@ static uint16_t bf16_bits_b(float rounded)
     return (uint16_t)(b >> 16);
 }
 
-// dense matrix (host block rows, values already rounded) -> A fragments [rows/16][cols/16][32 lanes][8 bf16]
-static std::vector<uint16_t> pack_fragments(const BsrHost &M)
+// host block rows (values already rounded) -> dense row-major bf16 bits
+static std::vector<uint16_t> dense_bf16(const BsrHost &M)
 {
-    const int rows = M.rows4 * 4, cols = M.cols4 * 4, nmt = rows / 16, nkt = cols / 16;
-    std::vector<uint16_t> dense((size_t)rows * cols, 0), out((size_t)nmt * nkt * 256);
+    const int rows = M.rows4 * 4, cols = M.cols4 * 4;
+    std::vector<uint16_t> dense((size_t)rows * cols, 0);
     for (int br = 0; br < M.rows4; ++br)
         for (int i = M.row_ptr[br]; i < M.row_ptr[br + 1]; ++i)
             for (int r = 0; r < 4; ++r)
                 for (int c = 0; c < 4; ++c)
                     dense[(size_t)(4 * br + r) * cols + 4 * M.col[i] + c] = bf16_bits_b(M.vals[(size_t)i * 16 + 4 * r + c]);
+    return dense;
+}
+
+// dense matrix -> A fragments [rows/16][cols/16][32 lanes][8 bf16]
+static std::vector<uint16_t> pack_fragments(const BsrHost &M)
+{
+    const int rows = M.rows4 * 4, cols = M.cols4 * 4, nmt = rows / 16, nkt = cols / 16;
+    const std::vector<uint16_t> dense = dense_bf16(M);
+    std::vector<uint16_t> out((size_t)nmt * nkt * 256);
     for (int mt = 0; mt < nmt; ++mt)
         for (int kt = 0; kt < nkt; ++kt)
             for (int lane = 0; lane < 32; ++lane) {
@@ -357,11 +544,46 @@ static std::vector<uint16_t> pack_fragments(const BsrHost &M)
     return out;
 }
 
+// 2-D tensor map of a row-major bf16 matrix [rows][cols] with a (64 x box_rows) box and the 128-byte swizzle
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = [] {
+        void *f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) f = nullptr;
+        cudaGetLastError();
+        return (EncodeTiledFn)f;
+    }();
+    return fn;
+}
+static bool make_map(CUtensorMap *tm, void *base, int rows, int cols, int box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static int bn_for(int nt) { return nt == 4 ? 64 : (nt == 2 ? 16 : 0); }
+static size_t smem_for(int nt, int nkt_r)
+{
+    const size_t img = (size_t)nt * 2 * nkt_r * 32 * 8;
+    const size_t ring = bn_for(nt) ? (size_t)TC_STAGES * (TC_BM * TC_BK * 2 + 2 * bn_for(nt) * TC_BK * 2) + 1024 : 0;
+    return img > ring ? img : ring;
+}
+
 static int nt_for(int batch) { return batch <= 8 ? 1 : (batch <= 16 ? 2 : 4); }
 
 static void *batched_fn(int nt)
 {
-    return nt == 1 ? (void *)batched_step_kernel<1> : nt == 2 ? (void *)batched_step_kernel<2> : (void *)batched_step_kernel<4>;
+    return nt == 1 ? (void *)batched_step_kernel<1, 0> : nt == 2 ? (void *)batched_step_kernel<2, 16> : (void *)batched_step_kernel<4, 64>;
 }
 
 int batched_supported(const wrnn_model *m, int batch, std::string *why)
@@ -396,8 +618,26 @@ int batched_prepare(wrnn_model *m)
          cudaMalloc((void **)&k->a_buf, Bp * 3 * H * 4) == cudaSuccess && cudaMalloc((void **)&k->logits, Bp * 256 * 4) == cudaSuccess &&
          cudaMalloc((void **)&k->c_cur, Bp) == cudaSuccess && cudaMalloc((void **)&k->c_prev, Bp) == cudaSuccess &&
          cudaMalloc((void **)&k->f_prev, Bp) == cudaSuccess && cudaMalloc((void **)&k->bar, 256) == cudaSuccess;
+    // tcgen05 phase A: row-major R, row-major hi / lo state (rows beyond the padded batch stay zero), tensor maps
+    const int nt_max = nt_for(m->max_batch);
+    if (ok && nt_max >= 2 && !std::getenv("WRNN_BATCHED_NO_TC") && encode_tiled_fn()) {
+        k->tc_rows = (k->max_bp + 63) / 64 * 64;
+        const std::vector<uint16_t> Rd = dense_bf16(m->hR);
+        bool t = cudaMalloc((void **)&k->Rrm, Rd.size() * 2) == cudaSuccess &&
+                 cudaMemcpy(k->Rrm, Rd.data(), Rd.size() * 2, cudaMemcpyHostToDevice) == cudaSuccess;
+        for (int b = 0; b < 2 && t; ++b)
+            for (int q = 0; q < 2 && t; ++q)
+                t = cudaMalloc((void **)&k->hrm[b][q], (size_t)k->tc_rows * H * 2) == cudaSuccess &&
+                    cudaMemset(k->hrm[b][q], 0, (size_t)k->tc_rows * H * 2) == cudaSuccess;
+        t = t && make_map(&k->tmR, k->Rrm, 3 * H, H, TC_BM);
+        for (int b = 0; b < 2 && t; ++b)
+            for (int q = 0; q < 2 && t; ++q)
+                t = make_map(&k->tmH64[b][q], k->hrm[b][q], k->tc_rows, H, 64) && make_map(&k->tmH16[b][q], k->hrm[b][q], k->tc_rows, H, 16);
+        if (t) { k->tc = true; k->weight_bytes += (int64_t)Rd.size() * 2; }
+        else ok = false;
+    }
     for (int nt : {1, 2, 4}) {
-        const size_t smem = (size_t)nt * 2 * k->NKT_R * 32 * 8;
+        const size_t smem = smem_for(nt, k->NKT_R);
         if (ok && cudaFuncSetAttribute(batched_fn(nt), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) ok = false;
     }
     m->batched = k;
@@ -417,6 +657,9 @@ void batched_destroy(wrnn_model *m)
     cudaFree(k->Rf); cudaFree(k->O1f); cudaFree(k->O2f); cudaFree(k->O3f); cudaFree(k->O4f);
     cudaFree(k->himg[0]); cudaFree(k->himg[1]); cudaFree(k->qimg); cudaFree(k->hf32[0]); cudaFree(k->hf32[1]);
     cudaFree(k->a_buf); cudaFree(k->logits); cudaFree(k->c_cur); cudaFree(k->c_prev); cudaFree(k->f_prev); cudaFree(k->bar);
+    cudaFree(k->Rrm);
+    for (int b = 0; b < 2; ++b)
+        for (int q = 0; q < 2; ++q) cudaFree(k->hrm[b][q]);
     delete k;
     m->batched = nullptr;
 }
@@ -427,7 +670,7 @@ int batched_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_thre
     const int nt = nt_for(batch);
     if (n_ctas) *n_ctas = m->n_sms;
     if (n_threads) *n_threads = 512;
-    if (smem) *smem = nt * 2 * k.NKT_R * 32 * 8;
+    if (smem) *smem = (int)smem_for(nt, k.NKT_R);
     if (weight_bytes) *weight_bytes = k.weight_bytes;
     return WRNN_OK;
 }
@@ -458,11 +701,19 @@ int batched_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.bar = k.bar; p.status = m->status;
     p.limit_ns = 2000000000ull;
+    // tcgen05 phase A: one CTA per (128 rows of R) x (BN rows of the batch); falls back to mma.sync when the grid is too small
+    const int bn = bn_for(nt);
+    if (k.tc && bn && (3 * m->H / TC_BM) * ((p.Bp + bn - 1) / bn) <= m->n_sms) {
+        p.tc = 1;
+        p.tmR = k.tmR;
+        for (int b = 0; b < 2; ++b)
+            for (int q = 0; q < 2; ++q) { p.hrm[b][q] = k.hrm[b][q]; p.tmH[b][q] = bn == 64 ? k.tmH64[b][q] : k.tmH16[b][q]; }
+    }
 
     if (cudaMemsetAsync(k.bar, 0, sizeof(unsigned long long), s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     void *args[] = {(void *)&p};
-    const size_t smem = (size_t)nt * 2 * k.NKT_R * 32 * 8;
+    const size_t smem = smem_for(nt, k.NKT_R);
     const cudaError_t e = cudaLaunchCooperativeKernel(batched_fn(nt), dim3(m->n_sms), dim3(512), args, smem, s);
     if (e != cudaSuccess) {
         m->err = std::string("batched kernel launch failed: ") + cudaGetErrorString(e);

@@ -154,7 +154,7 @@ def main():
     ap.add_argument("--workload", type=int, default=1, help="index into the workload list (default 1: dense 896 bf16, batch 1, 24000)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--n-steps", type=int, default=None, help="override samples per call (profiling of a short case)")
-    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "resident", "batched"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "resident", "batched", "bcluster"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -179,7 +179,7 @@ def main():
 
     n_steps = wl.n_steps if args.n_steps is None else args.n_steps
     w, masks, cond_np = synth.build_workload(wl)
-    kern = {"auto": B.WRNN_KERNEL_AUTO, "generic": B.WRNN_KERNEL_GENERIC, "resident": B.WRNN_KERNEL_RESIDENT, "batched": B.WRNN_KERNEL_BATCHED}[args.kernel]
+    kern = {"auto": B.WRNN_KERNEL_AUTO, "generic": B.WRNN_KERNEL_GENERIC, "resident": B.WRNN_KERNEL_RESIDENT, "batched": B.WRNN_KERNEL_BATCHED, "bcluster": B.WRNN_KERNEL_BCLUSTER}[args.kernel]
     model = B.wrnn_create(w, wl.dtype, masks, max_batch=wl.batch, kernel=kern)
     info = B.wrnn_launch_info(model, wl.batch)
     cond = torch.from_numpy(cond_np).to(dev)
@@ -301,7 +301,7 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "H": wl.H, "batch": wl.batch, "n_steps": n_steps, "weights": wl.dtype,
                        "sparsity": wl.sparsity, "l2": "flushed between timed iterations (256 MiB fill)",
-                       "kernel": {1: "generic", 2: "resident", 3: "batched", 4: "sparse-cluster"}[info["kernel"]], "n_ctas": info["n_ctas"],
+                       "kernel": {1: "generic", 2: "resident", 3: "batched", 4: "sparse-cluster", 5: "batched-cluster"}[info["kernel"]], "n_ctas": info["n_ctas"],
                        "threads_per_cta": info["n_threads"], "smem_bytes_per_cta": info["smem_bytes"],
                        "multi_gpu": "replicas only"},
             "us_per_sample_step": us_per_sample_step, "x_realtime_24khz": value / world / wl.batch / 24000.0 * wl.batch,

@@ -57,7 +57,8 @@ typedef enum {
     WRNN_KERNEL_GENERIC = 1,    /* weights streamed from L2 every step; any shape; bring-up path */
     WRNN_KERNEL_RESIDENT = 2,   /* persistent kernel, weights resident in shared memory (one row) */
     WRNN_KERNEL_BATCHED = 3,    /* tensor-pipe contractions over all rows (dense bf16, >= 2 rows)  */
-    WRNN_KERNEL_SPARSE = 4      /* block-sparse model resident in one 16-CTA cluster (one row)     */
+    WRNN_KERNEL_SPARSE = 4,     /* block-sparse model resident in one 16-CTA cluster (one row)     */
+    WRNN_KERNEL_BCLUSTER = 5    /* rows dealt to 16-CTA clusters, tcgen05 contractions (dense bf16, >= 2 rows) */
 } wrnn_kernel;
 
 /*

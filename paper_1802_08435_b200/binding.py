@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libwrnn.so")
 WRNN_OK, WRNN_ERR_INVALID_ARG, WRNN_ERR_UNSUPPORTED, WRNN_ERR_NOMEM, WRNN_ERR_CUDA, WRNN_ERR_TIMEOUT = range(6)
 WRNN_F32, WRNN_BF16 = 0, 1
 WRNN_KERNEL_AUTO, WRNN_KERNEL_GENERIC, WRNN_KERNEL_RESIDENT, WRNN_KERNEL_BATCHED, WRNN_KERNEL_SPARSE = 0, 1, 2, 3, 4
+WRNN_KERNEL_BCLUSTER = 5
 _STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "NOMEM", "CUDA", "TIMEOUT"]
 
 EXPORTS = [

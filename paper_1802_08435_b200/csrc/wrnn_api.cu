@@ -108,7 +108,7 @@ static bool ensure_g(wrnn_model *m, size_t floats)
 
 static bool use_resident(const wrnn_model *m, int batch)
 {
-    if (m->kernel == WRNN_KERNEL_GENERIC || m->kernel == WRNN_KERNEL_BATCHED) return false;
+    if (m->kernel == WRNN_KERNEL_GENERIC || m->kernel == WRNN_KERNEL_BATCHED || m->kernel == WRNN_KERNEL_BCLUSTER) return false;
     return m->resident != nullptr && resident_supported(m, batch, nullptr) == WRNN_OK;
 }
 
@@ -118,9 +118,15 @@ static bool use_sparse(const wrnn_model *m, int batch)
     return m->sparse_pack != nullptr && sparse_supported(m, batch, nullptr) == WRNN_OK;
 }
 
+static bool use_bcluster(const wrnn_model *m, int batch)
+{
+    if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_BCLUSTER) return false;
+    return m->bcluster != nullptr && bcluster_supported(m, batch, nullptr) == WRNN_OK;
+}
+
 static bool use_batched(const wrnn_model *m, int batch)
 {
-    if (m->kernel == WRNN_KERNEL_GENERIC || m->kernel == WRNN_KERNEL_RESIDENT) return false;
+    if (m->kernel == WRNN_KERNEL_GENERIC || m->kernel == WRNN_KERNEL_RESIDENT || m->kernel == WRNN_KERNEL_BCLUSTER) return false;
     return m->batched != nullptr && batched_supported(m, batch, nullptr) == WRNN_OK;
 }
 
@@ -170,7 +176,13 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     if (rc != WRNN_OK) return fail(m, rc, "conditioning projection launch failed");
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
     if (use_sparse(m, a.batch)) return sparse_run(m, a, s);
+    if (use_bcluster(m, a.batch)) return bcluster_run(m, a, s);
     if (use_batched(m, a.batch)) return batched_run(m, a, s);
+    if (m->kernel == WRNN_KERNEL_BCLUSTER) {
+        std::string why;
+        bcluster_supported(m, a.batch, &why);
+        return fail(m, WRNN_ERR_UNSUPPORTED, "cluster-partitioned kernel unavailable: " + why);
+    }
     if (m->kernel == WRNN_KERNEL_SPARSE) {
         std::string why;
         sparse_supported(m, a.batch, &why);
@@ -207,7 +219,7 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
     if (!p->R || !p->I || !p->O1 || !p->O2 || !p->O3 || !p->O4) return fail(nullptr, WRNN_ERR_INVALID_ARG, "missing weight matrix");
     if ((p->cond_dim > 0) != (p->W_cond != nullptr)) return fail(nullptr, WRNN_ERR_INVALID_ARG, "W_cond must be given iff cond_dim > 0");
     if (p->dtype != WRNN_F32 && p->dtype != WRNN_BF16) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown dtype");
-    if (p->kernel < WRNN_KERNEL_AUTO || p->kernel > WRNN_KERNEL_SPARSE) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown kernel family");
+    if (p->kernel < WRNN_KERNEL_AUTO || p->kernel > WRNN_KERNEL_BCLUSTER) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown kernel family");
 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, WRNN_ERR_CUDA, "no usable CUDA device"); }
@@ -280,6 +292,14 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
             return fail(nullptr, rc, "sparse cluster kernel unavailable: " + why);
         }
     }
+    if (p->kernel == WRNN_KERNEL_AUTO || p->kernel == WRNN_KERNEL_BCLUSTER) {
+        const int rc = bcluster_prepare(m);
+        if (rc != WRNN_OK && p->kernel == WRNN_KERNEL_BCLUSTER) {
+            const std::string why = m->err;
+            wrnn_destroy(m);
+            return fail(nullptr, rc, "cluster-partitioned kernel unavailable: " + why);
+        }
+    }
     if (p->kernel == WRNN_KERNEL_AUTO || p->kernel == WRNN_KERNEL_BATCHED) {
         const int rc = batched_prepare(m);
         if (rc != WRNN_OK && p->kernel == WRNN_KERNEL_BATCHED) {
@@ -307,6 +327,7 @@ void wrnn_destroy(wrnn_model *m)
     cudaDeviceSynchronize();
     resident_destroy(m);
     batched_destroy(m);
+    bcluster_destroy(m);
     sparse_destroy(m);
     free_bsr(&m->R); free_bsr(&m->O1); free_bsr(&m->O2); free_bsr(&m->O3); free_bsr(&m->O4);
     cudaFree(m->I); cudaFree(m->b_gate); cudaFree(m->b1); cudaFree(m->b2); cudaFree(m->b3); cudaFree(m->b4);
@@ -434,6 +455,10 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
     if (use_sparse(m, batch)) {
         if (kernel) *kernel = WRNN_KERNEL_SPARSE;
         return sparse_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
+    }
+    if (use_bcluster(m, batch)) {
+        if (kernel) *kernel = WRNN_KERNEL_BCLUSTER;
+        return bcluster_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
     }
     if (use_batched(m, batch)) {
         if (kernel) *kernel = WRNN_KERNEL_BATCHED;

@@ -21,13 +21,13 @@
 // tile and the hi / lo activation tiles brought in by TMA (128-byte swizzle, three-stage mbarrier ring), one
 // elected thread issuing tcgen05.mma (M = 128, N = BN, K = 16, bf16 -> fp32) into a TMEM accumulator, and four
 // warps reading it back with tcgen05.ld for the epilogue.  Every mbarrier wait is bounded.
-#include <cuda.h>
 #include <cuda_bf16.h>
 
 #include <cstdlib>
 #include <cstring>
 
 #include "wrnn_internal.h"
+#include "wrnn_tc.cuh"
 
 namespace wrnn {
 
@@ -170,54 +170,8 @@ __device__ __forceinline__ void tile_gemm(const uint4 *Af, int nk, const uint2 *
     }
 }
 
-// ---- tcgen05 / TMA / mbarrier helpers (phase A with 16 or more rows)
-constexpr int TC_STAGES = 3, TC_BM = 128, TC_BK = 64;
-constexpr unsigned long long TC_WAIT_NS = 2000000000ull;
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) { asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory"); }
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) { asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory"); }
-// bounded: false when the phase did not complete within about two seconds
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
-{
-    unsigned long long t0 = 0;
-    for (unsigned n = 1;; ++n) {
-        uint32_t ok;
-        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0,1,0,p;\n}" : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-        if (ok) return true;
-        if ((n & 255u) == 0) {
-            const unsigned long long now = globaltimer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > TC_WAIT_NS) return false;
-        }
-    }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int x, int y)
-{
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y) : "memory");
-}
-// shared-memory matrix descriptor of a K-major tile with 128-byte swizzle (rows of 128 bytes, 8-row atoms of 1 KB)
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr)
-{
-    return (uint64_t)((saddr >> 4) & 0x3FFF) | ((uint64_t)1 << 16) | ((uint64_t)(1024 >> 4) << 32) | ((uint64_t)1 << 46) | ((uint64_t)2 << 61);
-}
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-                 ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
-{
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
-                   "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-                 : "r"(taddr));
-}
+// ---- tcgen05 phase A (16 or more rows): tile and ring geometry
+constexpr int TC_STAGES = 3, TC_BM = 128;
 
 __device__ __forceinline__ long long frame_of_b(const BatchedParams &p, long long s, int gb)
 {
@@ -253,8 +207,16 @@ __device__ __forceinline__ void gate_unit_b(const BatchedParams &p, int j, int g
 #ifdef WRNN_PROFILE_BATCHED
 __device__ long long g_bprof[32];
 #define BSTAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { const long long n_ = clock64(); g_bprof[i] += n_ - bt_; bt_ = n_; } } while (0)
+#define BROLE_BEGIN() long long rt_ = clock64(), ra_ = 0, rb_ = 0
+#define BROLE_A() do { const long long n_ = clock64(); ra_ += n_ - rt_; rt_ = n_; } while (0)
+#define BROLE_B() do { const long long n_ = clock64(); rb_ += n_ - rt_; rt_ = n_; } while (0)
+#define BROLE_FLUSH(i) do { if (blockIdx.x == 0) { g_bprof[i] += ra_; g_bprof[i + 1] += rb_; } } while (0)
 #else
 #define BSTAMP(i) do { } while (0)
+#define BROLE_BEGIN() do { } while (0)
+#define BROLE_A() do { } while (0)
+#define BROLE_B() do { } while (0)
+#define BROLE_FLUSH(i) do { } while (0)
 #endif
 
 // BN: rows of the batch per tcgen05 tile of phase A (0: phase A stays on mma.sync).
@@ -358,21 +320,28 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const __grid_const
             bool ok = true;
             if (warp == 0 && lane == 0) {
                 asm volatile("fence.proxy.async;" ::: "memory");         // earlier generic-proxy use of this shared memory and of h
+                BROLE_BEGIN();
                 for (int kb = 0; kb < nkb; ++kb) {
                     const unsigned it = tc_kb + kb, st = it % TC_STAGES, ph = (it / TC_STAGES) & 1;
+                    BROLE_A();
                     if (!mbar_wait(smem_u32(&tc_empty[st]), ph ^ 1)) { ok = false; break; }
+                    BROLE_B();
                     const uint32_t fb = smem_u32(&tc_full[st]), base = ring0 + st * STAGE_BYTES;
                     mbar_expect_tx(fb, STAGE_BYTES);
                     tma_load_2d(base, &p.tmR, fb, kb * TC_BK, mtile * TC_BM);
                     tma_load_2d(base + A_BYTES, &p.tmH[cur][0], fb, kb * TC_BK, nblk * BN);
                     tma_load_2d(base + A_BYTES + B_BYTES, &p.tmH[cur][1], fb, kb * TC_BK, nblk * BN);
                 }
+                BROLE_A(); BROLE_FLUSH(18);
             } else if (warp == 1 && lane == 0) {
                 // instruction descriptor: D fp32, A / B bf16, both K-major, N = BN, M = 128
                 const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+                BROLE_BEGIN();
                 for (int kb = 0; kb < nkb; ++kb) {
                     const unsigned it = tc_kb + kb, st = it % TC_STAGES, ph = (it / TC_STAGES) & 1;
+                    BROLE_A();
                     if (!mbar_wait(smem_u32(&tc_full[st]), ph)) { ok = false; break; }
+                    BROLE_B();
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t base = ring0 + st * STAGE_BYTES;
                     const uint64_t da = umma_desc_sw128(base), dhi = umma_desc_sw128(base + A_BYTES), dlo = umma_desc_sw128(base + A_BYTES + B_BYTES);
@@ -384,8 +353,11 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const __grid_const
                     umma_commit(smem_u32(&tc_empty[st]));
                 }
                 if (ok) umma_commit(smem_u32(&tc_done));
+                BROLE_A(); BROLE_FLUSH(20);
             } else if (warp >= 4 && warp < 8) {
+                BROLE_BEGIN();
                 if (mbar_wait(smem_u32(&tc_done), tc_tasks & 1)) {
+                    BROLE_A();
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const int sub = warp & 3;
                     const int row = mtile * TC_BM + sub * 32 + lane;
@@ -401,6 +373,7 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const __grid_const
                         }
                     }
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    BROLE_B(); if (tid == 128) BROLE_FLUSH(22);
                 } else ok = false;
             }
             if (!ok && atomicCAS(&p.status->code, DEV_OK, DEV_TIMEOUT) == DEV_OK) { p.status->cta = blockIdx.x; p.status->step = -2; p.status->phase = 1; }
@@ -514,7 +487,7 @@ static uint16_t bf16_bits_b(float rounded)
 }
 
 // host block rows (values already rounded) -> dense row-major bf16 bits
-static std::vector<uint16_t> dense_bf16(const BsrHost &M)
+std::vector<uint16_t> dense_bf16_bits(const BsrHost &M)
 {
     const int rows = M.rows4 * 4, cols = M.cols4 * 4;
     std::vector<uint16_t> dense((size_t)rows * cols, 0);
@@ -530,7 +503,7 @@ static std::vector<uint16_t> dense_bf16(const BsrHost &M)
 static std::vector<uint16_t> pack_fragments(const BsrHost &M)
 {
     const int rows = M.rows4 * 4, cols = M.cols4 * 4, nmt = rows / 16, nkt = cols / 16;
-    const std::vector<uint16_t> dense = dense_bf16(M);
+    const std::vector<uint16_t> dense = dense_bf16_bits(M);
     std::vector<uint16_t> out((size_t)nmt * nkt * 256);
     for (int mt = 0; mt < nmt; ++mt)
         for (int kt = 0; kt < nkt; ++kt)
@@ -542,33 +515,6 @@ static std::vector<uint16_t> pack_fragments(const BsrHost &M)
                     for (int j = 0; j < 2; ++j) o[2 * q + j] = dense[(size_t)(16 * mt + rsel[q]) * cols + 16 * kt + csel[q] + j];
             }
     return out;
-}
-
-// 2-D tensor map of a row-major bf16 matrix [rows][cols] with a (64 x box_rows) box and the 128-byte swizzle
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
-                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                                  CUtensorMapFloatOOBfill);
-static EncodeTiledFn encode_tiled_fn()
-{
-    static EncodeTiledFn fn = [] {
-        void *f = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || q != cudaDriverEntryPointSuccess) f = nullptr;
-        cudaGetLastError();
-        return (EncodeTiledFn)f;
-    }();
-    return fn;
-}
-static bool make_map(CUtensorMap *tm, void *base, int rows, int cols, int box_rows)
-{
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 static int bn_for(int nt) { return nt == 4 ? 64 : (nt == 2 ? 16 : 0); }
@@ -622,7 +568,7 @@ int batched_prepare(wrnn_model *m)
     const int nt_max = nt_for(m->max_batch);
     if (ok && nt_max >= 2 && !std::getenv("WRNN_BATCHED_NO_TC") && encode_tiled_fn()) {
         k->tc_rows = (k->max_bp + 63) / 64 * 64;
-        const std::vector<uint16_t> Rd = dense_bf16(m->hR);
+        const std::vector<uint16_t> Rd = dense_bf16_bits(m->hR);
         bool t = cudaMalloc((void **)&k->Rrm, Rd.size() * 2) == cudaSuccess &&
                  cudaMemcpy(k->Rrm, Rd.data(), Rd.size() * 2, cudaMemcpyHostToDevice) == cudaSuccess;
         for (int b = 0; b < 2 && t; ++b)

@@ -52,6 +52,7 @@ struct StepArgs {
 struct ResidentPack;   // packed weights of the shared-memory-resident kernels (opaque here)
 struct BatchedPack;    // fragment-packed weights and activation images of the batched kernel (opaque here)
 struct SparsePack;     // compressed block rows of the single-cluster block-sparse kernel (opaque here)
+struct BcPack;         // per-CTA weight slices and stacked activation images of the cluster-partitioned multi-row kernel
 
 }  // namespace wrnn
 
@@ -84,6 +85,7 @@ struct wrnn_model {
     wrnn::ResidentPack *resident = nullptr;
     wrnn::BatchedPack *batched = nullptr;
     wrnn::SparsePack *sparse_pack = nullptr;
+    wrnn::BcPack *bcluster = nullptr;
 
     // host images for packers
     wrnn::BsrHost hR, hO1, hO2, hO3, hO4;
@@ -127,5 +129,13 @@ int batched_prepare(wrnn_model *m);
 void batched_destroy(wrnn_model *m);
 int batched_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem, int64_t *weight_bytes);
 int batched_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
+std::vector<uint16_t> dense_bf16_bits(const BsrHost &M);   // host block rows -> dense row-major bf16 bits
+
+// wrnn_bcluster.cu
+int bcluster_supported(const wrnn_model *m, int batch, std::string *why);
+int bcluster_prepare(wrnn_model *m);
+void bcluster_destroy(wrnn_model *m);
+int bcluster_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem, int64_t *weight_bytes);
+int bcluster_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
 
 }  // namespace wrnn

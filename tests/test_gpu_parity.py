@@ -53,16 +53,21 @@ def test_tiny_teacher_forced(env, kernel, H, dtype, batch, sparse):
         B.wrnn_destroy(m)
 
 
-@pytest.mark.parametrize("H,batch", [(128, 2), (128, 11), (256, 33), (384, 16), (128, 70)])
-def test_tiny_batched_kernel(env, H, batch):
-    """The tensor-pipe batched kernel on small shapes: ragged batches, one and several stream blocks."""
+@pytest.mark.parametrize("kernel,H,batch", [
+    ("BATCHED", 128, 2), ("BATCHED", 128, 11), ("BATCHED", 256, 33), ("BATCHED", 384, 16), ("BATCHED", 128, 70),
+    ("BCLUSTER", 128, 2), ("BCLUSTER", 128, 11), ("BCLUSTER", 256, 33), ("BCLUSTER", 384, 16), ("BCLUSTER", 128, 70),
+    ("BCLUSTER", 256, 130), ("BCLUSTER", 128, 300)])
+def test_tiny_batched_kernel(env, kernel, H, batch):
+    """The two multi-row kernels on small shapes: ragged batches; one and several stream blocks (grid-phased kernel);
+    one and several clusters, one to three lane quadrants per cluster (cluster-partitioned kernel)."""
     torch, B = env
     w = _tiny(H)
     om = orc.OracleModel(w, "bf16")
-    m = B.wrnn_create(w, "bf16", max_batch=batch, kernel=B.WRNN_KERNEL_BATCHED)
+    kid = getattr(B, "WRNN_KERNEL_" + kernel)
+    m = B.wrnn_create(w, "bf16", max_batch=batch, kernel=kid)
     try:
-        assert B.wrnn_launch_info(m, batch)["kernel"] == B.WRNN_KERNEL_BATCHED
-        cond = synth.make_cond(batch, 12, 4)
+        assert B.wrnn_launch_info(m, batch)["kernel"] == kid
+        cond = synth.make_cond(batch, (40 + batch) // 10 + 2, 4)
         r = pu.teacher_forced_parity(torch, B, m, om, cond, 40, batch, SEED, hop=10, row_stride=1, row_offset_mul=1,
                                      threads=pu.NCPU)
         assert r["idx_bad"] == 0, {k: v for k, v in r.items() if k != "oracle"}

@@ -7,7 +7,7 @@
 // freely against one another.  Inside a cluster the weight rows are dealt out in chunks of eight rows:
 //
 //   A    a = R h_{t-1}                 CTA c holds the (u, r, e) rows of hidden-unit chunks c, c+16, c+32, ...
-//   Gc   coarse gates -> y_c           in the epilogue of A, straight from the TMEM accumulator
+//   Gc   coarse gates -> y_c           from the TMEM accumulator of A
 //   O1   q_c = relu(O1 y_c + b1)       chunks c, c+16, ... of the hidden layer
 //   O2   l_c = O2 q_c + b2             logits 16 c .. 16 c + 15
 //   Sc   draw c_t                      one warp per row, rows c, c+16, ... of the group
@@ -18,17 +18,20 @@
 // group are stacked as a 128-row operand whose lane quadrant q holds the bf16 high parts of rows 16 q .. 16 q + 15
 // in lanes 0-15 and the low parts (x - bf16(x)) in lanes 16-31, so that one tcgen05.mma (M = 128, N = the CTA's
 // weight rows, K = 16) yields both partial products and the epilogue adds them with one shuffle.  The weights are
-// the N side, streamed every step from L2 (they are shared by all clusters) by TMA with the 128-byte swizzle,
-// together with the activation tile, through an mbarrier ring; accumulators live in TMEM (A: columns 0-255,
-// kept until Gf; O1 / O3: 256-287; O2 / O4: 320-335).  The fp32 hidden state of a (row, chunk) pair never
+// the N side.  R is streamed every step from L2 (it is shared by all clusters) by TMA with the 128-byte swizzle,
+// together with the activation tiles, through an mbarrier ring; the CTA's slices of O1 .. O4 stay resident in shared
+// memory and the activations of those phases arrive in two multi-tile TMA copies.  Operands live in global memory
+// as arrays of [rows][64] k-block tiles so that every copy is one box.  Accumulators live in TMEM (A: columns
+// 0-255, kept until Gf; O1 / O3: 256-287; O2 / O4: 320-335).  The fp32 hidden state of a (row, unit) pair never
 // leaves the registers of the thread that owns it; only its bf16 high / low split is written out (to L2, in the
-// operand layout) for the next contractions.  Every mbarrier wait is bounded; a CTA whose wait ran out records
-// it, skips its remaining work and keeps arriving at the cluster barriers so that the launch drains cleanly.
+// operand layout) for the next contractions.  Every mbarrier wait is bounded; a CTA whose wait ran out records it,
+// skips its remaining tensor work and keeps arriving at the cluster barriers so that the launch drains cleanly.
 #include <cuda_bf16.h>
 
 #include <cstdlib>
 #include <cstring>
 
+#include "wrnn_cluster.cuh"
 #include "wrnn_internal.h"
 #include "wrnn_tc.cuh"
 
@@ -38,34 +41,35 @@ constexpr int BC_CS = 16;             // CTAs per cluster
 constexpr int BC_THREADS = 512;
 constexpr int BC_MAX_STAGES = 8;
 constexpr int BC_SLACK = 16384;       // the 128-row A operand may read this far past a short activation tile
-constexpr int BC_MROWS = 128;         // rows of the activation arrays reserved per cluster
+constexpr int BC_MROWS = 128;         // rows of an activation tile (the stacked operand of one cluster)
 constexpr int BC_GROUP = 64;          // most rows of a batch one cluster takes
 constexpr int BC_COL_A = 0, BC_COL_O1 = 256, BC_COL_O2 = 320, BC_TMEM_COLS = 512;
+constexpr int BC_UH = 32;             // most hidden units of one half (coarse or fine) a CTA owns
+constexpr int BC_S_BYTES = 3 * BC_UH * BC_GROUP * 4;       // staged accumulators [gate][unit][row] fp32
+constexpr int BC_SOUT_PITCH = 40;                          // bf16 per (row, part) of the staged gate outputs
+constexpr int BC_SOUT_BYTES = BC_GROUP * 2 * BC_SOUT_PITCH * 2;
 
 struct BcPack {
     int H = 0, NCH = 0, NRp = 0, NOC = 0, NO1 = 0;
-    __nv_bfloat16 *Wr = nullptr, *O1p = nullptr, *O2p = nullptr, *O3p = nullptr, *O4p = nullptr;   // [16][rows per CTA][K]
+    __nv_bfloat16 *Wr = nullptr, *O1p = nullptr, *O2p = nullptr, *O3p = nullptr, *O4p = nullptr;   // [16][k-block][rows per CTA][64]
     float4 *Ip = nullptr;                                   // [16][3][64]: I of the CTA's gate rows
-    __nv_bfloat16 *act[2] = {nullptr, nullptr};             // [clusters * 128][H]   stacked high / low state
-    __nv_bfloat16 *q = nullptr;                             // [clusters * 128][H/2] stacked hidden layer
-    float *logits = nullptr;                                // [max rows][256]
-    uint8_t *c_cur = nullptr, *c_prev = nullptr, *f_prev = nullptr;
+    float *bp = nullptr;                                    // [16][2][48]: b1 | b2 (head 0), b3 | b4 (head 1) of the CTA's rows
+    __nv_bfloat16 *act[2] = {nullptr, nullptr};             // [clusters][H/64][128][64]   stacked high / low state tiles
+    __nv_bfloat16 *q = nullptr;                             // [clusters][H/128][128][64]  stacked hidden-layer tiles
     CUtensorMap tmWr, tmO1, tmO2, tmO3, tmO4;
     int max_clusters = 0, max_dyn_smem = 0;
     int64_t weight_bytes = 0;
 };
 
 struct BcParams {
-    int H, Hh, G, batch, RB, MR, NCH, NRp, NO1, n_stages, stage_bytes;
+    int H, Hh, G, batch, RB, MR, NCH, NRp, NO1, n_stages, stage_bytes, kpart, res_bytes, s_off;
     long long n_steps, step0;
     unsigned stream0;
     unsigned long long seed;
     int n_frames, hop, row_stride, row_offset_mul;
     const float4 *Ip;
-    const float *b1, *b2, *b3, *b4, *g;
+    const float *bp, *g;
     __nv_bfloat16 *act0, *act1, *q;
-    float *logits;
-    uint8_t *c_cur, *c_prev, *f_prev;
     const float *h_in; float *h_out;
     const uint8_t *c_in, *f_in; uint8_t *c_st_out, *f_st_out;
     const uint8_t *c_forced, *f_forced;
@@ -78,8 +82,9 @@ struct BcParams {
     alignas(64) CUtensorMap tmO2;
     alignas(64) CUtensorMap tmO3;
     alignas(64) CUtensorMap tmO4;
-    alignas(64) CUtensorMap tmAct[2];
-    alignas(64) CUtensorMap tmQ;
+    alignas(64) CUtensorMap tmActA[2];     // one tile of MR rows (ring of phase A)
+    alignas(64) CUtensorMap tmActO[2];     // kpart tiles of MR rows (operand of O1 / O3)
+    alignas(64) CUtensorMap tmQ;           // kpart tiles of MR rows (operand of O2 / O4)
 };
 
 // all threads of all CTAs of the cluster; orders global-memory and TMEM traffic across it
@@ -100,36 +105,38 @@ __device__ __forceinline__ uint4 pack8_bf16(const __nv_bfloat16 (&v)[8])
     return o;
 }
 
-// Eight values -> their bf16 high parts at `hi` and low parts at `lo` (16-byte stores).
-__device__ __forceinline__ void store_split8(__nv_bfloat16 *hi, __nv_bfloat16 *lo, const float (&x)[8])
+// element (operand row mrow, column k) of a cluster's tile array with nkb k-blocks
+__device__ __forceinline__ size_t tile_index(int cl, int nkb, int mrow, int k)
 {
-    __nv_bfloat16 h[8], l[8];
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        h[e] = __float2bfloat16_rn(x[e]);
-        l[e] = __float2bfloat16_rn(x[e] - __bfloat162float(h[e]));
-    }
-    *reinterpret_cast<uint4 *>(hi) = pack8_bf16(h);
-    *reinterpret_cast<uint4 *>(lo) = pack8_bf16(l);
+    return (((size_t)cl * nkb + (k >> 6)) * BC_MROWS + mrow) * 64 + (k & 63);
 }
 
 #ifdef WRNN_PROFILE_BC
 __device__ long long g_bcprof[32];
-#define CSTAMP(i) do { if (blockIdx.x == 0 && threadIdx.x == 96) { const long long n_ = clock64(); g_bcprof[i] += n_ - bt_; bt_ = n_; } } while (0)
+#define CSTAMP(i) do { if (threadIdx.x == 96) { const long long n_ = clock64(); s_prof[i] += n_ - bt_; bt_ = n_; } } while (0)
+#define RBEGIN() long long rt_ = clock64()
+#define RSTAMP(i) do { const long long n_ = clock64(); s_prof[i] += n_ - rt_; rt_ = n_; } while (0)
 #else
 #define CSTAMP(i) do { } while (0)
+#define RBEGIN() do { } while (0)
+#define RSTAMP(i) do { } while (0)
 #endif
 
 __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __grid_constant__ BcParams p)
 {
-#ifdef WRNN_PROFILE_BC
-    long long bt_ = clock64();
-#endif
     extern __shared__ __align__(16) uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t s_full[BC_MAX_STAGES], s_empty[BC_MAX_STAGES], s_done;
+    __shared__ __align__(8) uint64_t s_full[BC_MAX_STAGES], s_empty[BC_MAX_STAGES], s_ofull[2], s_done, s_wload;
     __shared__ uint32_t s_tmem;
     __shared__ int s_failed;
     __shared__ float4 s_I[3 * 64];                  // [gate][unit of this CTA] -> (I0, I1, I2, -)
+    __shared__ float s_b[2 * 48];                   // [head][b1 of the CTA's 32 hidden-layer rows | b2 of its 16 logits]
+    __shared__ __align__(16) float s_log[4 * 256];  // logits of the rows this CTA draws for (row crank + 16 w of the group), written by peers
+    __shared__ int s_c[BC_GROUP], s_f[BC_GROUP];    // c_t / f_t of every row of the group, broadcast by the drawing CTAs
+#ifdef WRNN_PROFILE_BC
+    __shared__ long long s_prof[32];
+    long long bt_ = clock64();
+    if (threadIdx.x < 32) s_prof[threadIdx.x] = 0;
+#endif
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     unsigned crank;
@@ -139,44 +146,62 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
     const int nrows = min(p.RB, p.batch - row0);
     if (nrows <= 0) return;                         // the same for every CTA of the cluster
     const int H = p.H, Hh = p.Hh, NCH = p.NCH;
+    const int nkbA = H / TC_BK, nkbH = Hh / TC_BK;
 
     // ---- fixed roles of this thread
+    // (1) TMEM reader: warp (quadrant qd, slot); lanes 0-15 see the high-part rows 16 qd + lr, lanes 16-31 the low-part ones
     const int qd = warp & 3, slot = warp >> 2, half = lane >> 4, lr = lane & 15;
     const int nQ = (nrows + 15) >> 4;               // lane quadrants in use
-    const int bl = 16 * qd + lr;                    // row of the group this lane serves in the epilogues
+    const int bl = 16 * qd + lr;
     const bool rowv = bl < nrows;
-    const int gb = row0 + bl;                       // its row of the batch
-    const int ci = 2 * slot + half;                 // gate chunk of this thread (8 hidden units)
-    const int gch = (int)crank + BC_CS * ci;
-    const bool chv = ci < NCH && gch < H / 8;
-    const bool ch_coarse = gch < Hh / 8;
-    const int unit0 = 8 * gch;
-    const size_t arow_hi = (size_t)cl * BC_MROWS + 32 * qd + lr, arow_lo = arow_hi + 16;
-    // warp-uniform: does either chunk of this warp belong to the coarse / fine half
-    const int gch_a = (int)crank + BC_CS * (2 * slot), gch_b = gch_a + BC_CS;
-    const bool va = 2 * slot < NCH && gch_a < H / 8, vb = 2 * slot + 1 < NCH && gch_b < H / 8;
-    const bool warp_coarse = (va && gch_a < Hh / 8) || (vb && gch_b < Hh / 8);
-    const bool warp_fine = (va && gch_a >= Hh / 8) || (vb && gch_b >= Hh / 8);
+    const int gb = row0 + bl;
+    const int mrow_hi = 32 * qd + lr, mrow_lo = mrow_hi + 16;
+    // chunks of this CTA: i = 0 .. nchv-1 valid, the first nCc of them coarse
+    const int tot_ch = H / 8, half_ch = Hh / 8;
+    const int nchv = (tot_ch - (int)crank + BC_CS - 1) / BC_CS;
+    const int nCc = (half_ch - (int)crank + BC_CS - 1) / BC_CS;
     // hidden-layer chunk (8 outputs of O1 / O3) of this warp
     const int och = (int)crank + BC_CS * slot;
-    const bool ochv = och < Hh / 8;
+    const bool ochv = och < half_ch;
+    // (2) gate thread: one row of the group, hidden units g_u0, g_u0 + g_step, ... of the half in flight
+    const int rshift = nrows <= 16 ? 4 : (nrows <= 32 ? 5 : 6);
+    const int g_row = tid & ((1 << rshift) - 1), g_u0 = tid >> rshift, g_step = BC_THREADS >> rshift;
+    const bool g_rowv = g_row < nrows;
+    const int g_gb = row0 + g_row;
 
-    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const uint32_t ring0 = smem_u32(ring);
+    uint8_t *base = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t res0 = smem_u32(base);                           // resident O1 | O3 | O2 | O4 tiles
+    const uint32_t wO1 = res0, wO3 = wO1 + (uint32_t)(nkbH * p.NO1 * 128), wO2 = wO3 + (uint32_t)(nkbH * p.NO1 * 128),
+                   wO4 = wO2 + (uint32_t)(nkbH * 16 * 128);
+    uint8_t *area = base + p.res_bytes;
+    const uint32_t area0 = smem_u32(area);                          // ring of phase A / operand of the O phases
+    float *S = reinterpret_cast<float *>(area + p.s_off);           // staged accumulators [gate][unit][row]
+    __nv_bfloat16 *Sout = reinterpret_cast<__nv_bfloat16 *>(area + p.s_off + BC_S_BYTES);
     const uint32_t done_bar = smem_u32(&s_done);
     volatile int *failed = &s_failed;
+    const uint32_t abytes = (uint32_t)p.MR * 128u;
 
     if (tid == 0) {
         for (int i = 0; i < BC_MAX_STAGES; ++i) { mbar_init(smem_u32(&s_full[i]), 2); mbar_init(smem_u32(&s_empty[i]), 1); }
+        mbar_init(smem_u32(&s_ofull[0]), 1); mbar_init(smem_u32(&s_ofull[1]), 1);
         mbar_init(done_bar, 1);
+        mbar_init(smem_u32(&s_wload), 1);
         s_failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // resident slices of O1 .. O4: one box each
+        const uint32_t wb = smem_u32(&s_wload);
+        mbar_expect_tx(wb, (uint32_t)p.res_bytes);
+        tma_load_2d(wO1, &p.tmO1, wb, 0, (int)crank * nkbH * p.NO1);
+        tma_load_2d(wO3, &p.tmO3, wb, 0, (int)crank * nkbH * p.NO1);
+        tma_load_2d(wO2, &p.tmO2, wb, 0, (int)crank * nkbH * 16);
+        tma_load_2d(wO4, &p.tmO4, wb, 0, (int)crank * nkbH * 16);
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(BC_TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     for (int i = tid; i < 3 * 64; i += BC_THREADS) s_I[i] = p.Ip[(size_t)crank * 3 * 64 + i];
+    for (int i = tid; i < 2 * 48; i += BC_THREADS) s_b[i] = p.bp[(size_t)crank * 96 + i];
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -186,181 +211,287 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
         *failed = 1;
         if (atomicCAS(&p.status->code, DEV_OK, DEV_TIMEOUT) == DEV_OK) { p.status->cta = blockIdx.x; p.status->step = step; p.status->phase = phase; }
     };
+    if (!mbar_wait(smem_u32(&s_wload), 0)) fail(-1, 0);
 
-    // ---- initial state: fp32 in registers, stacked high / low image in buffer 0 (other rows of the image stay zero)
-    float hreg[8];
+    // ---- initial state: fp32 in the registers of the gate threads, stacked high / low tiles in buffer 0
+    // (operand rows that no thread writes were zeroed by the host)
+    float hc[4], hf[4];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) hreg[e] = (rowv && chv && p.h_in) ? p.h_in[(size_t)gb * H + unit0 + e] : 0.f;
-    if (rowv && chv && qd < nQ) store_split8(p.act0 + arow_hi * H + unit0, p.act0 + arow_lo * H + unit0, hreg);
-    if (tid < 4) {
-        const int r = (int)crank + BC_CS * tid;
-        if (r < nrows) {
-            p.c_prev[row0 + r] = p.c_in ? p.c_in[row0 + r] : (uint8_t)128;
-            p.f_prev[row0 + r] = p.f_in ? p.f_in[row0 + r] : (uint8_t)0;
+    for (int j = 0; j < 4; ++j) {
+        const int uc = g_u0 + j * g_step;
+        hc[j] = hf[j] = 0.f;
+        if (g_rowv && p.h_in) {
+            if (uc < 8 * nCc) hc[j] = p.h_in[(size_t)g_gb * H + 8 * ((int)crank + BC_CS * (uc >> 3)) + (uc & 7)];
+            if (uc < 8 * (nchv - nCc)) hf[j] = p.h_in[(size_t)g_gb * H + 8 * ((int)crank + BC_CS * (nCc + (uc >> 3))) + (uc & 7)];
+        }
+        if (g_rowv) {
+            const int mr_hi = 32 * (g_row >> 4) + (g_row & 15);
+            if (uc < 8 * nCc) {
+                const int unit = 8 * ((int)crank + BC_CS * (uc >> 3)) + (uc & 7);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(hc[j]);
+                p.act0[tile_index(cl, nkbA, mr_hi, unit)] = hi;
+                p.act0[tile_index(cl, nkbA, mr_hi + 16, unit)] = __float2bfloat16_rn(hc[j] - __bfloat162float(hi));
+            }
+            if (uc < 8 * (nchv - nCc)) {
+                const int unit = 8 * ((int)crank + BC_CS * (nCc + (uc >> 3))) + (uc & 7);
+                const __nv_bfloat16 hi = __float2bfloat16_rn(hf[j]);
+                p.act0[tile_index(cl, nkbA, mr_hi, unit)] = hi;
+                p.act0[tile_index(cl, nkbA, mr_hi + 16, unit)] = __float2bfloat16_rn(hf[j] - __bfloat162float(hi));
+            }
         }
     }
+    // the rows this CTA draws for: row crank + 16 w by warp w; their last drawn (or forced) pair stays in registers
+    const int s_r = (int)crank + BC_CS * warp;
+    const bool sampler = warp < 4 && s_r < nrows;
+    const int s_gb = row0 + s_r;
+    int last_c = sampler ? (p.c_in ? (int)p.c_in[s_gb] : 128) : 0, last_f = sampler ? (p.f_in ? (int)p.f_in[s_gb] : 0) : 0;
     fence_proxy_async();
     cluster_barrier();
 
-    // ring position of the three role threads (they walk the same sequence of k-blocks) and parity of `done`
+    // ring position of the three role threads of phase A (they walk the same sequence of k-blocks), parities of the
+    // O-phase operand barriers and of `done`
     int rst = 0;
-    uint32_t rph = 0, dph = 0;
-    const uint32_t abytes = (uint32_t)p.MR * 128u;
+    uint32_t rph = 0, oph = 0, dph = 0;
 
-    // One contraction: D[128 x n_w] (TMEM column dcol) = activations[cluster rows, columns ax ..] . W[rows wy ..]^T over nkb
-    // k-blocks of 64.  warp 0 / lane 0 loads the activation tiles, warp 2 / lane 0 the weight tiles, warp 1 / lane 0
-    // issues the MMAs; every thread returns once the accumulator is complete.
-    auto gemm = [&](const CUtensorMap *tmA, int ax, const CUtensorMap *tmW, int wy, int nkb, int n_w, uint32_t dcol, int step, int phase) {
+    // Only the MMA thread watches the `done` mbarrier; everybody else blocks on the CTA barrier, so that no polling warp
+    // competes with the three role threads for issue slots.
+    auto wait_done = [&](int step, int phase) {
+        if (warp == 1) {
+            if (lane == 0) {
+                RBEGIN();
+                if (!*failed && !mbar_wait(done_bar, dph)) fail(step, phase);
+                RSTAMP(31);
+            }
+            __syncwarp();
+        }
+        dph ^= 1;
+        __syncthreads();
+        tc_fence_after();
+    };
+
+    // Phase A: D[128 x NRp] (TMEM column 0) = state tiles of buffer `cur` . (this CTA's rows of R)^T through the ring.
+    // warp 0 / lane 0 loads the activation tiles, warp 2 / lane 0 the weight tiles, warp 1 / lane 0 issues the MMAs.
+    // The role loops are kept to a handful of instructions per k-block: a lone thread issues slowly.
+    const uint32_t full0 = smem_u32(&s_full[0]), empty0 = smem_u32(&s_empty[0]);
+    auto gemm_a_issue = [&](int cur, int step) {
         if (lane == 0 && warp < 3 && !*failed) {
             if (warp == 1) {
-                const uint32_t idesc = umma_idesc_bf16(128, n_w);
+                const uint32_t idesc = umma_idesc_bf16(128, p.NRp);
+                const uint32_t dstep = (uint32_t)(p.stage_bytes >> 4), boff = abytes >> 4;
+                uint32_t da = umma_desc_lo(area0) + (uint32_t)rst * dstep;
                 bool ok = true;
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (!mbar_wait(smem_u32(&s_full[rst]), rph)) { ok = false; break; }
+                RBEGIN();
+                for (int kb = 0; kb < nkbA; ++kb) {
+                    if (!mbar_wait(full0 + 8u * (uint32_t)rst, rph)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t base = ring0 + (uint32_t)rst * (uint32_t)p.stage_bytes;
-                    const uint64_t da = umma_desc_sw128(base), db = umma_desc_sw128(base + abytes);
-#pragma unroll
-                    for (int k = 0; k < TC_BK / 16; ++k) umma_bf16(tmem + dcol, da + 2 * k, db + 2 * k, idesc, (kb | k) ? 1u : 0u);
-                    umma_commit(smem_u32(&s_empty[rst]));
-                    if (++rst == p.n_stages) { rst = 0; rph ^= 1; }
+                    umma_bf16_kblock(tmem + BC_COL_A, da, da + boff, idesc, kb ? 1u : 0u);
+                    umma_commit(empty0 + 8u * (uint32_t)rst);
+                    da += dstep;
+                    if (++rst == p.n_stages) { rst = 0; rph ^= 1; da = umma_desc_lo(area0); }
                 }
                 if (ok) umma_commit(done_bar);
-                else fail(step, phase);
+                else fail(step, 1);
             } else {
                 const bool is_act = warp == 0;
-                const uint32_t bytes = is_act ? abytes : (uint32_t)n_w * 128u;
-                const CUtensorMap *tm = is_act ? tmA : tmW;
-                const int x0 = is_act ? ax : 0, y = is_act ? cl * BC_MROWS : wy;
-                const uint32_t off = is_act ? 0u : abytes;
-                fence_proxy_async();               // earlier generic-proxy writes of the activations, by this and (through the barrier) other CTAs
-                for (int kb = 0; kb < nkb; ++kb) {
-                    if (!mbar_wait(smem_u32(&s_empty[rst]), rph ^ 1)) { fail(step, phase); break; }
-                    const uint32_t fb = smem_u32(&s_full[rst]);
+                const uint32_t bytes = is_act ? abytes : (uint32_t)p.NRp * 128u;
+                const CUtensorMap *tmA = &p.tmActA[cur];
+                uint32_t dst = area0 + (uint32_t)rst * (uint32_t)p.stage_bytes + (is_act ? 0u : abytes);
+                int coord = is_act ? cl * nkbA : (int)crank * nkbA * p.NRp;
+                const int cstep = is_act ? 1 : p.NRp;
+                RBEGIN();
+                // (the writers of the state tiles and of this shared memory issued their proxy fences before the cluster barrier)
+                for (int kb = 0; kb < nkbA; ++kb) {
+                    if (!mbar_wait(empty0 + 8u * (uint32_t)rst, rph ^ 1)) { fail(step, 1); break; }
+                    const uint32_t fb = full0 + 8u * (uint32_t)rst;
                     mbar_expect_tx(fb, bytes);
-                    tma_load_2d(ring0 + (uint32_t)rst * (uint32_t)p.stage_bytes + off, tm, fb, x0 + kb * TC_BK, y);
-                    if (++rst == p.n_stages) { rst = 0; rph ^= 1; }
+                    if (is_act) tma_load_3d(dst, tmA, fb, 0, 0, coord);
+                    else tma_load_2d(dst, &p.tmWr, fb, 0, coord);
+                    coord += cstep;
+                    dst += (uint32_t)p.stage_bytes;
+                    if (++rst == p.n_stages) { rst = 0; rph ^= 1; dst -= (uint32_t)p.n_stages * (uint32_t)p.stage_bytes; }
                 }
             }
         }
         __syncwarp();
-        if (!*failed && !mbar_wait(done_bar, dph)) fail(step, phase);
-        dph ^= 1;
-        tc_fence_after();
     };
 
-    // Gates of Eq. 2 for the chunks of one half (coarse: x2 = 0; fine: x2 = c_t), from the accumulator of phase A.
-    auto gates = [&](bool coarse, long long s, float x0, float x1, float x2, const float *grow, __nv_bfloat16 *anext) {
-        if (qd >= nQ || !(coarse ? warp_coarse : warp_fine)) return;
-        // columns of gate g of chunk i: 8 NCH g + 8 i; both chunks of the warp are read by all lanes
-        float a[3][8], b[3][8];
-        const uint32_t t0 = tmem + ((uint32_t)(32 * qd) << 16) + BC_COL_A + 16 * slot;
-#pragma unroll
-        for (int g = 0; g < 3; ++g) { tmem_ld8(t0 + 8 * NCH * g, a[g]); tmem_ld8(t0 + 8 * NCH * g + 8, b[g]); }
-        tmem_wait_ld();
-        // lanes 0-15 hold the high-part products of a row, lanes 16-31 the low-part ones: the lower half-warp takes
-        // chunk a, the upper chunk b, each adding the other half's partial
-        float acc[3][8];
-#pragma unroll
-        for (int g = 0; g < 3; ++g)
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const float send = half ? a[g][e] : b[g][e];
-                const float recv = __shfl_xor_sync(0xffffffffu, send, 16);
-                acc[g][e] = (half ? b[g][e] : a[g][e]) + recv;
+    // O phases: D[128 x n_w] (TMEM column dcol) = tiles tile0 .. tile0 + nkbH - 1 of an activation array . (resident weights)^T.
+    // The operand arrives as two copies of kpart tiles; the MMAs of the first half start while the second is in flight.
+    auto gemm_o_issue = [&](const CUtensorMap *tmA, int tile0, uint32_t wres, int n_w, uint32_t dcol, int step, int phase) {
+        if (lane == 0 && warp < 3 && !*failed) {
+            if (warp != 1) {
+                // warp 0 fetches the first half of the operand, warp 2 the second
+                const int part = warp >> 1;
+                const uint32_t half_bytes = (uint32_t)p.kpart * abytes, fb = smem_u32(&s_ofull[part]);
+                mbar_expect_tx(fb, half_bytes);
+                tma_load_3d(area0 + (uint32_t)part * half_bytes, tmA, fb, 0, 0, tile0 + part * p.kpart);
+            } else {
+                const uint32_t idesc = umma_idesc_bf16(128, n_w);
+                const uint32_t astep = abytes >> 4, wstep = (uint32_t)(n_w * 8);
+                uint32_t da = umma_desc_lo(area0), db = umma_desc_lo(wres);
+                RBEGIN();
+                bool ok = mbar_wait(smem_u32(&s_ofull[0]), oph);
+                RSTAMP(30);
+                if (ok) {
+                    tc_fence_after();
+                    int kb = 0;
+                    for (; kb < p.kpart; ++kb, da += astep, db += wstep) umma_bf16_kblock(tmem + dcol, da, db, idesc, kb ? 1u : 0u);
+                    RSTAMP(27);
+                    ok = mbar_wait(smem_u32(&s_ofull[1]), oph);
+                    RSTAMP(28);
+                    if (ok) {
+                        tc_fence_after();
+                        for (; kb < nkbH; ++kb, da += astep, db += wstep) umma_bf16_kblock(tmem + dcol, da, db, idesc, 1u);
+                    }
+                    RSTAMP(29);
+                }
+                if (ok) umma_commit(done_bar);
+                else fail(step, phase);
             }
-        if (!(rowv && chv && ch_coarse == coarse)) return;
-        float gu[8], gr[8], ge[8];
-        {
-            const float4 *g4 = reinterpret_cast<const float4 *>(grow + unit0);
-            const float4 u0 = __ldg(g4), u1 = __ldg(g4 + 1);
-            const float4 *r4 = reinterpret_cast<const float4 *>(grow + H + unit0);
-            const float4 r0 = __ldg(r4), r1 = __ldg(r4 + 1);
-            const float4 *e4 = reinterpret_cast<const float4 *>(grow + 2 * H + unit0);
-            const float4 e0 = __ldg(e4), e1 = __ldg(e4 + 1);
-            gu[0] = u0.x; gu[1] = u0.y; gu[2] = u0.z; gu[3] = u0.w; gu[4] = u1.x; gu[5] = u1.y; gu[6] = u1.z; gu[7] = u1.w;
-            gr[0] = r0.x; gr[1] = r0.y; gr[2] = r0.z; gr[3] = r0.w; gr[4] = r1.x; gr[5] = r1.y; gr[6] = r1.z; gr[7] = r1.w;
-            ge[0] = e0.x; ge[1] = e0.y; ge[2] = e0.z; ge[3] = e0.w; ge[4] = e1.x; ge[5] = e1.y; ge[6] = e1.z; ge[7] = e1.w;
         }
-        float uu[8], rr[8], ee[8];
+        oph ^= 1;
+        __syncwarp();
+    };
+
+    // Inputs of the gates of one half that do not depend on the contraction (I x + conditioning; x2 joins later for the
+    // fine half): computed while the tensor pipe works.
+    auto gate_inputs = [&](bool coarse, float x0, float x1, const float *grow, float (&pre)[4][3]) {
+        const int i0 = coarse ? 0 : nCc, nchh = coarse ? nCc : nchv - nCc;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            const float4 Iu = s_I[8 * ci + e], Ir = s_I[64 + 8 * ci + e], Ie = s_I[128 + 8 * ci + e];
-            const float pu = acc[0][e] + fmaf(Iu.x, x0, fmaf(Iu.y, x1, fmaf(Iu.z, x2, gu[e])));
-            const float pr = acc[1][e] + fmaf(Ir.x, x0, fmaf(Ir.y, x1, fmaf(Ir.z, x2, gr[e])));
-            const float pe = fmaf(Ie.x, x0, fmaf(Ie.y, x1, fmaf(Ie.z, x2, ge[e])));
-            uu[e] = sigmoidf_acc(pu);
-            rr[e] = sigmoidf_acc(pr);
-            ee[e] = tanhf(fmaf(rr[e], acc[2][e], pe));
-            hreg[e] = fmaf(uu[e], hreg[e], (1.0f - uu[e]) * ee[e]);
-        }
-        store_split8(anext + arow_hi * H + unit0, anext + arow_lo * H + unit0, hreg);
-        if (p.dbg_gates) {
-            float *d = p.dbg_gates + ((size_t)s * p.batch + gb) * p.G + unit0;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) { d[e] = uu[e]; d[H + e] = rr[e]; d[2 * H + e] = ee[e]; }
-        }
-        if (p.dbg_h) {
-            float *d = p.dbg_h + ((size_t)s * p.batch + gb) * H + unit0;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) d[e] = hreg[e];
+        for (int j = 0; j < 4; ++j) {
+            const int uh = g_u0 + j * g_step;
+            pre[j][0] = pre[j][1] = pre[j][2] = 0.f;
+            if (!g_rowv || uh >= 8 * nchh) continue;
+            const int il = 8 * (i0 + (uh >> 3)) + (uh & 7);
+            const int unit = 8 * ((int)crank + BC_CS * (i0 + (uh >> 3))) + (uh & 7);
+            const float4 Iu = s_I[il], Ir = s_I[64 + il], Ie = s_I[128 + il];
+            pre[j][0] = fmaf(Iu.x, x0, fmaf(Iu.y, x1, __ldg(grow + unit)));
+            pre[j][1] = fmaf(Ir.x, x0, fmaf(Ir.y, x1, __ldg(grow + H + unit)));
+            pre[j][2] = fmaf(Ie.x, x0, fmaf(Ie.y, x1, __ldg(grow + 2 * H + unit)));
         }
     };
+
+    // Gates of Eq. 2 for the hidden units of one half that this CTA owns (coarse: x2 = 0; fine: x2 = c_t).
+    auto gates = [&](bool coarse, long long s, float x2, const float (&pre)[4][3], __nv_bfloat16 *anext, float (&hreg)[4]) {
+        const int i0 = coarse ? 0 : nCc, nchh = coarse ? nCc : nchv - nCc;      // chunk slots of this half
+        // (1) accumulator columns of the half: TMEM -> shared memory, high-part + low-part products added on the way;
+        // the warp of slot g takes gate g: its 8 nchh (<= 32) columns are adjacent
+        if (qd < nQ && slot < 3) {
+            float v[32];
+            tmem_ld32(tmem + ((uint32_t)(32 * qd) << 16) + BC_COL_A + 8 * NCH * slot + 8 * i0, v);
+            tmem_wait_ld();
+            float *d = S + ((size_t)(slot * BC_UH)) * BC_GROUP + bl;
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+                // lanes 0-15 (high-part products) keep the even column, lanes 16-31 (low-part) the odd one
+                const float mine = half ? v[c + 1] : v[c], send = half ? v[c] : v[c + 1];
+                const float sum = mine + __shfl_xor_sync(0xffffffffu, send, 16);
+                if (c < 8 * nchh) d[(size_t)(c + half) * BC_GROUP] = sum;
+            }
+        }
+        CSTAMP(22);
+        __syncthreads();
+        CSTAMP(23);
+        // (2) one (row, unit) pair per thread and pass
+        if (g_rowv) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int uh = g_u0 + j * g_step;
+                if (uh >= 8 * nchh) continue;
+                const int il = 8 * (i0 + (uh >> 3)) + (uh & 7);               // unit of this CTA
+                const float au = S[(size_t)uh * BC_GROUP + g_row], ar = S[(size_t)(BC_UH + uh) * BC_GROUP + g_row],
+                            ae = S[(size_t)(2 * BC_UH + uh) * BC_GROUP + g_row];
+                float pu = pre[j][0], pr = pre[j][1], pe = pre[j][2];
+                if (!coarse) { pu = fmaf(s_I[il].z, x2, pu); pr = fmaf(s_I[64 + il].z, x2, pr); pe = fmaf(s_I[128 + il].z, x2, pe); }
+                const float u = sigmoidf_fast(au + pu), r = sigmoidf_fast(ar + pr);
+                const float e = tanhf_fast(fmaf(r, ae, pe));
+                const float hn = fmaf(u, hreg[j], (1.0f - u) * e);
+                hreg[j] = hn;
+                const __nv_bfloat16 hi = __float2bfloat16_rn(hn);
+                Sout[(size_t)(2 * g_row) * BC_SOUT_PITCH + uh] = hi;
+                Sout[(size_t)(2 * g_row + 1) * BC_SOUT_PITCH + uh] = __float2bfloat16_rn(hn - __bfloat162float(hi));
+                if (p.dbg_gates || p.dbg_h) {
+                    const int unit = 8 * ((int)crank + BC_CS * (i0 + (uh >> 3))) + (uh & 7);
+                    if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * p.batch + g_gb) * p.G + unit; d[0] = u; d[H] = r; d[2 * H] = e; }
+                    if (p.dbg_h) p.dbg_h[((size_t)s * p.batch + g_gb) * H + unit] = hn;
+                }
+            }
+        }
+        CSTAMP(24);
+        __syncthreads();
+        CSTAMP(25);
+        // (3) 16-byte pieces (row, part, chunk) into the next state tiles
+        {
+            const int ii = tid & 3, part = (tid >> 2) & 1, row = tid >> 3;
+            if (ii < nchh && row < nrows) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(Sout + (size_t)(2 * row + part) * BC_SOUT_PITCH + 8 * ii);
+                const int mrow = 32 * (row >> 4) + 16 * part + (row & 15);
+                *reinterpret_cast<uint4 *>(anext + tile_index(cl, nkbA, mrow, 8 * ((int)crank + BC_CS * (i0 + ii)))) = v;
+            }
+        }
+    };
+
+    // conditioning frame of this thread's row, tracked without a division per step
+    long long g_frame = 0;
+    int g_rem = 0;
+    float x0 = 0.f, x1 = 0.f;
+    if (g_rowv) {
+        const long long pos = p.step0 * p.row_stride + (long long)(p.stream0 + (unsigned)g_gb) * p.row_offset_mul;
+        g_frame = pos / p.hop;
+        g_rem = (int)(pos - g_frame * p.hop);
+        x0 = scale8(p.c_in ? (int)p.c_in[g_gb] : 128);
+        x1 = scale8(p.f_in ? (int)p.f_in[g_gb] : 0);
+    }
 
     for (long long s = 0; s < p.n_steps; ++s) {
         __nv_bfloat16 *anext = (s & 1) ? p.act0 : p.act1;
         const int cur = (int)(s & 1);
-        // inputs of the gates that do not depend on this step's contractions
-        float x0 = 0.f, x1 = 0.f;
-        const float *grow = p.g;
-        if (rowv) {
-            x0 = scale8(__ldcg(p.c_prev + gb));
-            x1 = scale8(__ldcg(p.f_prev + gb));
-            const long long frame = ((p.step0 + s) * p.row_stride + (long long)(p.stream0 + (unsigned)gb) * p.row_offset_mul) / p.hop;
-            grow = p.g + ((size_t)gb * p.n_frames + (size_t)frame) * p.G;
-        }
+        const float *grow = p.g + ((size_t)g_gb * p.n_frames + (size_t)g_frame) * p.G;
+        float pre[4][3];
         // ---- A + Gc
         CSTAMP(0);
-        gemm(&p.tmAct[cur], 0, &p.tmWr, (int)crank * p.NRp, H / TC_BK, p.NRp, BC_COL_A, (int)s, 1);
+        gemm_a_issue(cur, (int)s);
+        if (s > 0 && g_rowv) x1 = scale8(s_f[g_row]);                  // f_{t-1}: drawn at the end of the last step
+        gate_inputs(true, x0, x1, grow, pre);
+        wait_done((int)s, 1);
         CSTAMP(1);
-        gates(true, s, x0, x1, 0.f, grow, anext);
+        gates(true, s, 0.f, pre, anext, hc);
+        CSTAMP(26);
         fence_proxy_async();
         CSTAMP(2);
         cluster_barrier();
         CSTAMP(3);
+        float x2 = 0.f;
 
         for (int head = 0; head < 2; ++head) {
-            const float *ba = head ? p.b3 : p.b1, *bb = head ? p.b4 : p.b2;
+            const float *bh = s_b + 48 * head;
             // ---- O1 / O3: hidden layer on this half of the new state
-            gemm(&p.tmAct[cur ^ 1], head * Hh, head ? &p.tmO3 : &p.tmO1, (int)crank * p.NO1, Hh / TC_BK, p.NO1, BC_COL_O1, (int)s, 2 + 4 * head);
+            gemm_o_issue(&p.tmActO[cur ^ 1], cl * nkbA + head * nkbH, head ? wO3 : wO1, p.NO1, BC_COL_O1, (int)s, 2 + 4 * head);
+            if (head == 0) gate_inputs(false, x0, x1, grow, pre);            // for Gf, while the tensor pipe works
+            wait_done((int)s, 2 + 4 * head);
             CSTAMP(4 + 8 * head);
             if (qd < nQ && 8 * slot < p.NO1) {
                 float v[8];
                 tmem_ld8(tmem + ((uint32_t)(32 * qd) << 16) + BC_COL_O1 + 8 * slot, v);
                 tmem_wait_ld();
-                float x[8];
+                __nv_bfloat16 o[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const float t = v[e] + __shfl_xor_sync(0xffffffffu, v[e], 16);
-                    x[e] = ochv ? fmaxf(t + (ba ? __ldg(ba + 8 * och + e) : 0.f), 0.f) : 0.f;
-                }
-                if (rowv && ochv) {
+                    const float x = fmaxf(t + bh[8 * slot + e], 0.f);
                     // both half-warps hold the sums: the lower writes the high parts, the upper the low parts
-                    __nv_bfloat16 o[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const __nv_bfloat16 hi = __float2bfloat16_rn(x[e]);
-                        o[e] = half ? __float2bfloat16_rn(x[e] - __bfloat162float(hi)) : hi;
-                    }
-                    *reinterpret_cast<uint4 *>(p.q + (half ? arow_lo : arow_hi) * Hh + 8 * och) = pack8_bf16(o);
+                    const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+                    o[e] = half ? __float2bfloat16_rn(x - __bfloat162float(hi)) : hi;
                 }
+                if (rowv && ochv) *reinterpret_cast<uint4 *>(p.q + tile_index(cl, nkbH, half ? mrow_lo : mrow_hi, 8 * och)) = pack8_bf16(o);
             }
             fence_proxy_async();
             CSTAMP(5 + 8 * head);
             cluster_barrier();
             CSTAMP(6 + 8 * head);
             // ---- O2 / O4: logits 16 crank .. + 15
-            gemm(&p.tmQ, 0, head ? &p.tmO4 : &p.tmO2, (int)crank * 16, Hh / TC_BK, 16, BC_COL_O2, (int)s, 3 + 4 * head);
+            gemm_o_issue(&p.tmQ, cl * nkbH, head ? wO4 : wO2, 16, BC_COL_O2, (int)s, 3 + 4 * head);
+            wait_done((int)s, 3 + 4 * head);
             CSTAMP(7 + 8 * head);
             if (qd < nQ && slot < 2) {
                 float v[8];
@@ -369,120 +500,159 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
 #pragma unroll
                 for (int e = 0; e < 8; ++e) v[e] += __shfl_xor_sync(0xffffffffu, v[e], 16);
                 if (rowv) {
-                    const int r0 = 16 * (int)crank + 8 * slot + 4 * half;      // four logits per lane
+                    const int c0 = 8 * slot + 4 * half;                        // four logits per lane
                     float4 o;
-                    o.x = (half ? v[4] : v[0]) + (bb ? __ldg(bb + r0 + 0) : 0.f);
-                    o.y = (half ? v[5] : v[1]) + (bb ? __ldg(bb + r0 + 1) : 0.f);
-                    o.z = (half ? v[6] : v[2]) + (bb ? __ldg(bb + r0 + 2) : 0.f);
-                    o.w = (half ? v[7] : v[3]) + (bb ? __ldg(bb + r0 + 3) : 0.f);
-                    *reinterpret_cast<float4 *>(p.logits + (size_t)gb * 256 + r0) = o;
+                    o.x = (half ? v[4] : v[0]) + bh[32 + c0 + 0];
+                    o.y = (half ? v[5] : v[1]) + bh[32 + c0 + 1];
+                    o.z = (half ? v[6] : v[2]) + bh[32 + c0 + 2];
+                    o.w = (half ? v[7] : v[3]) + bh[32 + c0 + 3];
+                    const int r0 = 16 * (int)crank + c0;
+                    // row bl of the group is drawn by warp bl / 16 of CTA bl % 16: the logits go straight into its shared memory
+                    const unsigned dst = map_to_rank(smem_addr(s_log + (bl >> 4) * 256 + r0), (unsigned)(bl & 15));
+                    asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(o.x), "f"(o.y), "f"(o.z), "f"(o.w) : "memory");
                     if (p.dbg_logits) *reinterpret_cast<float4 *>(p.dbg_logits + (((size_t)s * p.batch + gb) * 2 + head) * 256 + r0) = o;
                 }
             }
             CSTAMP(8 + 8 * head);
             cluster_barrier();
             CSTAMP(9 + 8 * head);
-            // ---- Sc / Sf: softmax + inverse-CDF draw, one warp per row
-            if (warp < 4) {
-                const int r = (int)crank + BC_CS * warp;
-                if (r < nrows) {
-                    const int sb = row0 + r;
-                    float l[8];
-                    const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(p.logits + (size_t)sb * 256 + 8 * lane));
-                    const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(p.logits + (size_t)sb * 256 + 8 * lane + 4));
-                    l[0] = v0.x; l[1] = v0.y; l[2] = v0.z; l[3] = v0.w; l[4] = v1.x; l[5] = v1.y; l[6] = v1.z; l[7] = v1.w;
-                    const float u = uniform24(p.seed, p.stream0 + (unsigned)sb, (unsigned long long)(p.step0 + s), head);
-                    int idx = warp_softmax_draw(l, u, lane);
-                    const size_t o = (size_t)sb * p.n_steps + s;
-                    if (lane == 0) {
-                        if (head == 0) {
-                            if (p.c_out) p.c_out[o] = (uint8_t)idx;
-                            if (p.c_forced) idx = p.c_forced[o];
-                            p.c_cur[sb] = (uint8_t)idx;
-                        } else {
-                            if (p.f_out) p.f_out[o] = (uint8_t)idx;
-                            if (p.f_forced) idx = p.f_forced[o];
-                            const int c = __ldcg(p.c_cur + sb);
-                            if (p.out) p.out[o] = (int16_t)(256 * c + idx - 32768);
-                            p.c_prev[sb] = (uint8_t)c;
-                            p.f_prev[sb] = (uint8_t)idx;
-                        }
-                    }
+            // ---- Sc / Sf: softmax + inverse-CDF draw, one warp per row; the result goes to every CTA of the cluster
+            int drawn = 0, used = 0;
+            const size_t s_o = (size_t)s_gb * p.n_steps + s;
+            if (sampler) {
+                float l[8];
+                const float4 v0 = *reinterpret_cast<const float4 *>(s_log + warp * 256 + 8 * lane);
+                const float4 v1 = *reinterpret_cast<const float4 *>(s_log + warp * 256 + 8 * lane + 4);
+                l[0] = v0.x; l[1] = v0.y; l[2] = v0.z; l[3] = v0.w; l[4] = v1.x; l[5] = v1.y; l[6] = v1.z; l[7] = v1.w;
+                const float u = uniform24(p.seed, p.stream0 + (unsigned)s_gb, (unsigned long long)(p.step0 + s), head);
+                drawn = warp_softmax_draw(l, u, lane);
+                const uint8_t *forced = head ? p.f_forced : p.c_forced;
+                used = forced ? (int)forced[s_o] : drawn;
+                if (lane < BC_CS) {
+                    const unsigned dst = map_to_rank(smem_addr((head ? s_f : s_c) + s_r), (unsigned)lane);
+                    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(dst), "r"(used) : "memory");
                 }
             }
             CSTAMP(10 + 8 * head);
             cluster_barrier();
             CSTAMP(11 + 8 * head);
+            // outputs leave after the barrier so that its release does not wait for them
+            if (sampler) {
+                if (head == 0) {
+                    if (lane == 0 && p.c_out) p.c_out[s_o] = (uint8_t)drawn;
+                    last_c = used;
+                } else {
+                    if (lane == 0) {
+                        if (p.f_out) p.f_out[s_o] = (uint8_t)drawn;
+                        if (p.out) p.out[s_o] = (int16_t)(256 * last_c + used - 32768);
+                    }
+                    last_f = used;
+                }
+            }
             if (head == 0) {
                 // ---- Gf: fine gates, now that c_t is known (it reaches only these rows, Section 2)
-                const float x2 = rowv ? scale8(__ldcg(p.c_cur + gb)) : 0.f;
-                gates(false, s, x0, x1, x2, grow, anext);
+                x2 = g_rowv ? scale8(s_c[g_row]) : 0.f;
+                gates(false, s, x2, pre, anext, hf);
+                CSTAMP(26);
                 fence_proxy_async();
                 CSTAMP(20);
                 cluster_barrier();
                 CSTAMP(21);
             }
         }
+        x0 = x2;                                  // c_t becomes c_{t-1}
+        g_rem += p.row_stride;
+        while (g_rem >= p.hop) { g_rem -= p.hop; ++g_frame; }
     }
 
-    if (p.h_out && rowv && chv && qd < nQ) {
+    if (p.h_out && g_rowv) {
 #pragma unroll
-        for (int e = 0; e < 8; ++e) p.h_out[(size_t)gb * H + unit0 + e] = hreg[e];
-    }
-    if (tid < 4) {
-        const int r = (int)crank + BC_CS * tid;
-        if (r < nrows) {
-            if (p.c_st_out) p.c_st_out[row0 + r] = __ldcg(p.c_prev + row0 + r);
-            if (p.f_st_out) p.f_st_out[row0 + r] = __ldcg(p.f_prev + row0 + r);
+        for (int j = 0; j < 4; ++j) {
+            const int uc = g_u0 + j * g_step;
+            if (uc < 8 * nCc) p.h_out[(size_t)g_gb * H + 8 * ((int)crank + BC_CS * (uc >> 3)) + (uc & 7)] = hc[j];
+            if (uc < 8 * (nchv - nCc)) p.h_out[(size_t)g_gb * H + 8 * ((int)crank + BC_CS * (nCc + (uc >> 3))) + (uc & 7)] = hf[j];
         }
     }
+    if (sampler && lane == 0) {
+        if (p.c_st_out) p.c_st_out[s_gb] = (uint8_t)last_c;
+        if (p.f_st_out) p.f_st_out[s_gb] = (uint8_t)last_f;
+    }
+#ifdef WRNN_PROFILE_BC
+    if (blockIdx.x == 0 && tid == 96) for (int i = 0; i < 32; ++i) g_bcprof[i] += s_prof[i];
+#endif
     tc_fence_before();
     __syncthreads();
     if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(BC_TMEM_COLS) : "memory");
-    cluster_barrier();      // no CTA leaves while a peer may still be inside a cluster barrier sequence
 }
 
 // ---------------------------------------------------------------------------------------------
 static int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
-// rows of a dense matrix (bf16 bits, `cols` wide) dealt out in chunks of 8 rows: CTA c gets chunks c, c + 16, ... of each
-// of the `gates` row blocks of `rows_per_gate` rows, laid out [c][gate][chunk slot][8] and padded with zero rows to rp rows
+// Rows of a dense matrix (bf16 bits, `cols` wide) dealt out in chunks of 8 rows -- CTA c gets chunks c, c + 16, ... of
+// each of the `gates` row blocks of `rows_per_gate` rows, as row 8 nch g + 8 i + e of its slice, padded with zero
+// rows to rp rows -- and cut into 64-column k-block tiles: [c][k-block][rp][64].
 static std::vector<uint16_t> deal_rows(const std::vector<uint16_t> &dense, int cols, int gates, int rows_per_gate, int nch, int rp)
 {
-    std::vector<uint16_t> out((size_t)BC_CS * rp * cols, 0);
+    const int nkb = cols / 64;
+    std::vector<uint16_t> out((size_t)BC_CS * nkb * rp * 64, 0);
     for (int c = 0; c < BC_CS; ++c)
         for (int g = 0; g < gates; ++g)
             for (int i = 0; i < nch; ++i) {
                 const int ch = c + BC_CS * i;
                 if (ch >= rows_per_gate / 8) continue;
                 for (int e = 0; e < 8; ++e)
-                    std::memcpy(&out[((size_t)c * rp + (size_t)g * 8 * nch + 8 * i + e) * cols],
-                                &dense[((size_t)g * rows_per_gate + 8 * ch + e) * cols], (size_t)cols * 2);
+                    for (int kb = 0; kb < nkb; ++kb)
+                        std::memcpy(&out[(((size_t)c * nkb + kb) * rp + (size_t)g * 8 * nch + 8 * i + e) * 64],
+                                    &dense[((size_t)g * rows_per_gate + 8 * ch + e) * cols + 64 * kb], 128);
             }
     return out;
+}
+
+// rows 16 c .. 16 c + 15 of a dense [256][cols] matrix as [c][k-block][16][64]
+static std::vector<uint16_t> tile_logit_rows(const std::vector<uint16_t> &dense, int cols)
+{
+    const int nkb = cols / 64;
+    std::vector<uint16_t> out((size_t)256 * cols, 0);
+    for (int c = 0; c < BC_CS; ++c)
+        for (int kb = 0; kb < nkb; ++kb)
+            for (int r = 0; r < 16; ++r)
+                std::memcpy(&out[(((size_t)c * nkb + kb) * 16 + r) * 64], &dense[((size_t)16 * c + r) * cols + 64 * kb], 128);
+    return out;
+}
+
+struct BcGeometry { int n_cl, RB, MR, stage_bytes, n_stages, kpart, res_bytes, s_off, smem; bool fits; };
+
+static BcGeometry bc_geometry(const BcPack &k, int batch)
+{
+    BcGeometry g;
+    int ncl = (batch + 15) / 16;
+    if (ncl > k.max_clusters) ncl = k.max_clusters;
+    g.RB = (batch + ncl - 1) / ncl;
+    g.n_cl = (batch + g.RB - 1) / g.RB;
+    g.MR = 32 * ((g.RB + 15) / 16);
+    const int nkbH = k.H / 128;
+    g.kpart = (nkbH + 1) / 2;
+    g.res_bytes = 2 * nkbH * 128 * (k.NO1 + 16);
+    g.stage_bytes = (g.MR + k.NRp) * 128;
+    g.s_off = round_up(2 * g.kpart * g.MR * 128, 1024);
+    const int area = k.max_dyn_smem - 1024 - g.res_bytes;
+    int ns = (area - BC_SLACK) / g.stage_bytes;
+    if (ns > BC_MAX_STAGES) ns = BC_MAX_STAGES;
+    g.n_stages = ns;
+    int need = ns * g.stage_bytes + BC_SLACK;
+    const int need_o = g.s_off + BC_S_BYTES + BC_SOUT_BYTES;
+    if (need_o > need) need = need_o;
+    g.fits = ns >= 2 && need_o <= area && g.RB <= BC_GROUP;
+    g.smem = 1024 + g.res_bytes + need;
+    return g;
 }
 
 int bcluster_supported(const wrnn_model *m, int batch, std::string *why)
 {
     if (!m->bcluster) { if (why) *why = "model was not packed for the cluster-partitioned kernel"; return WRNN_ERR_UNSUPPORTED; }
     if (batch < 2) { if (why) *why = "cluster-partitioned kernel needs at least two rows"; return WRNN_ERR_UNSUPPORTED; }
-    if (batch > m->bcluster->max_clusters * BC_GROUP) { if (why) *why = "batch exceeds 64 rows per co-resident cluster"; return WRNN_ERR_UNSUPPORTED; }
+    if (!bc_geometry(*m->bcluster, batch).fits) { if (why) *why = "batch does not fit the co-resident clusters"; return WRNN_ERR_UNSUPPORTED; }
     return WRNN_OK;
-}
-
-static void bc_geometry(const BcPack &k, int batch, int *n_cl, int *RB, int *MR, int *stage_bytes, int *n_stages, int *smem)
-{
-    int ncl = (batch + 15) / 16;
-    if (ncl > k.max_clusters) ncl = k.max_clusters;
-    const int rb = (batch + ncl - 1) / ncl;
-    *n_cl = (batch + rb - 1) / rb;
-    *RB = rb;
-    *MR = 32 * ((rb + 15) / 16);
-    *stage_bytes = (*MR + k.NRp) * 128;
-    int ns = (k.max_dyn_smem - 1024 - BC_SLACK) / *stage_bytes;
-    if (ns > BC_MAX_STAGES) ns = BC_MAX_STAGES;
-    *n_stages = ns;
-    *smem = ns * *stage_bytes + 1024 + BC_SLACK;
 }
 
 int bcluster_prepare(wrnn_model *m)
@@ -493,7 +663,7 @@ int bcluster_prepare(wrnn_model *m)
     if (!encode_tiled_fn()) { m->err = "driver has no tensor-map encoder"; return WRNN_ERR_UNSUPPORTED; }
     BcPack *k = new BcPack();
     m->bcluster = k;
-    const int H = m->H, Hh = H / 2;
+    const int H = m->H, Hh = H / 2, nkbA = H / 64, nkbH = Hh / 64;
     k->H = H;
     k->NCH = (H / 8 + BC_CS - 1) / BC_CS;
     k->NRp = round_up(24 * k->NCH, 16);
@@ -527,12 +697,7 @@ int bcluster_prepare(wrnn_model *m)
             return failed("device cannot co-schedule a 16-CTA cluster of this size", WRNN_ERR_UNSUPPORTED);
         k->max_clusters = n;
     }
-    if (m->max_batch > k->max_clusters * BC_GROUP) return failed("max_batch exceeds 64 rows per co-resident cluster", WRNN_ERR_UNSUPPORTED);
-    {
-        int ncl, rb, mr, sb, ns, smem;
-        bc_geometry(*k, m->max_batch, &ncl, &rb, &mr, &sb, &ns, &smem);
-        if (ns < 2) return failed("shared memory too small for the tile ring", WRNN_ERR_UNSUPPORTED);
-    }
+    if (!bc_geometry(*k, m->max_batch).fits) return failed("max_batch does not fit the co-resident clusters", WRNN_ERR_UNSUPPORTED);
 
     auto up = [&](const std::vector<uint16_t> &v, __nv_bfloat16 **dst) {
         k->weight_bytes += (int64_t)v.size() * 2;
@@ -541,10 +706,11 @@ int bcluster_prepare(wrnn_model *m)
     bool ok = up(deal_rows(dense_bf16_bits(m->hR), H, 3, H, k->NCH, k->NRp), &k->Wr) &&
               up(deal_rows(dense_bf16_bits(m->hO1), Hh, 1, Hh, k->NOC, k->NO1), &k->O1p) &&
               up(deal_rows(dense_bf16_bits(m->hO3), Hh, 1, Hh, k->NOC, k->NO1), &k->O3p) &&
-              up(dense_bf16_bits(m->hO2), &k->O2p) && up(dense_bf16_bits(m->hO4), &k->O4p);
+              up(tile_logit_rows(dense_bf16_bits(m->hO2), Hh), &k->O2p) && up(tile_logit_rows(dense_bf16_bits(m->hO4), Hh), &k->O4p);
     {
         std::vector<float4> Ih((size_t)BC_CS * 3 * 64, make_float4(0.f, 0.f, 0.f, 0.f));
-        for (int c = 0; c < BC_CS; ++c)
+        std::vector<float> bh((size_t)BC_CS * 96, 0.f);
+        for (int c = 0; c < BC_CS; ++c) {
             for (int g = 0; g < 3; ++g)
                 for (int i = 0; i < k->NCH; ++i) {
                     const int ch = c + BC_CS * i;
@@ -554,17 +720,29 @@ int bcluster_prepare(wrnn_model *m)
                         Ih[((size_t)c * 3 + g) * 64 + 8 * i + e] = make_float4(src[0], src[1], src[2], 0.f);
                     }
                 }
+            for (int head = 0; head < 2; ++head) {
+                const std::vector<float> &ba = head ? m->hb3 : m->hb1, &bb = head ? m->hb4 : m->hb2;
+                for (int i = 0; i < k->NOC; ++i) {
+                    const int ch = c + BC_CS * i;
+                    if (ch >= Hh / 8) continue;
+                    for (int e = 0; e < 8; ++e) bh[(size_t)c * 96 + 48 * head + 8 * i + e] = ba.empty() ? 0.f : ba[8 * ch + e];
+                }
+                for (int r = 0; r < 16; ++r) bh[(size_t)c * 96 + 48 * head + 32 + r] = bb.empty() ? 0.f : bb[16 * c + r];
+            }
+        }
         ok = ok && cudaMalloc((void **)&k->Ip, Ih.size() * sizeof(float4)) == cudaSuccess &&
-             cudaMemcpy(k->Ip, Ih.data(), Ih.size() * sizeof(float4), cudaMemcpyHostToDevice) == cudaSuccess;
+             cudaMemcpy(k->Ip, Ih.data(), Ih.size() * sizeof(float4), cudaMemcpyHostToDevice) == cudaSuccess &&
+             cudaMalloc((void **)&k->bp, bh.size() * 4) == cudaSuccess &&
+             cudaMemcpy(k->bp, bh.data(), bh.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess;
     }
-    const size_t arows = (size_t)k->max_clusters * BC_MROWS, mb = (size_t)m->max_batch;
-    ok = ok && cudaMalloc((void **)&k->act[0], arows * H * 2) == cudaSuccess && cudaMalloc((void **)&k->act[1], arows * H * 2) == cudaSuccess &&
-         cudaMalloc((void **)&k->q, arows * Hh * 2) == cudaSuccess && cudaMalloc((void **)&k->logits, mb * 256 * 4) == cudaSuccess &&
-         cudaMalloc((void **)&k->c_cur, mb) == cudaSuccess && cudaMalloc((void **)&k->c_prev, mb) == cudaSuccess &&
-         cudaMalloc((void **)&k->f_prev, mb) == cudaSuccess;
-    ok = ok && make_map(&k->tmWr, k->Wr, (long long)BC_CS * k->NRp, H, k->NRp) && make_map(&k->tmO1, k->O1p, (long long)BC_CS * k->NO1, Hh, k->NO1) &&
-         make_map(&k->tmO3, k->O3p, (long long)BC_CS * k->NO1, Hh, k->NO1) && make_map(&k->tmO2, k->O2p, 256, Hh, 16) &&
-         make_map(&k->tmO4, k->O4p, 256, Hh, 16);
+    const size_t tile = (size_t)BC_MROWS * 64 * 2, ncl = (size_t)k->max_clusters;
+    ok = ok && cudaMalloc((void **)&k->act[0], ncl * nkbA * tile) == cudaSuccess && cudaMalloc((void **)&k->act[1], ncl * nkbA * tile) == cudaSuccess &&
+         cudaMalloc((void **)&k->q, ncl * nkbH * tile) == cudaSuccess;
+    ok = ok && make_map(&k->tmWr, k->Wr, (long long)BC_CS * nkbA * k->NRp, 64, k->NRp) &&
+         make_map(&k->tmO1, k->O1p, (long long)BC_CS * nkbH * k->NO1, 64, nkbH * k->NO1) &&
+         make_map(&k->tmO3, k->O3p, (long long)BC_CS * nkbH * k->NO1, 64, nkbH * k->NO1) &&
+         make_map(&k->tmO2, k->O2p, (long long)BC_CS * nkbH * 16, 64, nkbH * 16) &&
+         make_map(&k->tmO4, k->O4p, (long long)BC_CS * nkbH * 16, 64, nkbH * 16);
     if (!ok) return failed("device allocation for the cluster-partitioned kernel failed", WRNN_ERR_NOMEM);
     return WRNN_OK;
 }
@@ -573,9 +751,8 @@ void bcluster_destroy(wrnn_model *m)
 {
     BcPack *k = m->bcluster;
     if (!k) return;
-    cudaFree(k->Wr); cudaFree(k->O1p); cudaFree(k->O2p); cudaFree(k->O3p); cudaFree(k->O4p); cudaFree(k->Ip);
-    cudaFree(k->act[0]); cudaFree(k->act[1]); cudaFree(k->q); cudaFree(k->logits);
-    cudaFree(k->c_cur); cudaFree(k->c_prev); cudaFree(k->f_prev);
+    cudaFree(k->Wr); cudaFree(k->O1p); cudaFree(k->O2p); cudaFree(k->O3p); cudaFree(k->O4p); cudaFree(k->Ip); cudaFree(k->bp);
+    cudaFree(k->act[0]); cudaFree(k->act[1]); cudaFree(k->q);
     delete k;
     m->bcluster = nullptr;
 }
@@ -583,11 +760,10 @@ void bcluster_destroy(wrnn_model *m)
 int bcluster_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem, int64_t *weight_bytes)
 {
     const BcPack &k = *m->bcluster;
-    int ncl, rb, mr, sb, ns, sm;
-    bc_geometry(k, batch, &ncl, &rb, &mr, &sb, &ns, &sm);
-    if (n_ctas) *n_ctas = ncl * BC_CS;
+    const BcGeometry g = bc_geometry(k, batch);
+    if (n_ctas) *n_ctas = g.n_cl * BC_CS;
     if (n_threads) *n_threads = BC_THREADS;
-    if (smem) *smem = sm;
+    if (smem) *smem = g.smem;
     if (weight_bytes) *weight_bytes = k.weight_bytes;
     return WRNN_OK;
 }
@@ -595,10 +771,10 @@ int bcluster_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_thr
 int bcluster_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
 {
     BcPack &k = *m->bcluster;
+    const BcGeometry g = bc_geometry(k, a.batch);
     BcParams p;
     std::memset(&p, 0, sizeof(p));
-    int ncl, smem;
-    bc_geometry(k, a.batch, &ncl, &p.RB, &p.MR, &p.stage_bytes, &p.n_stages, &smem);
+    p.RB = g.RB; p.MR = g.MR; p.stage_bytes = g.stage_bytes; p.n_stages = g.n_stages; p.kpart = g.kpart; p.res_bytes = g.res_bytes; p.s_off = g.s_off;
     p.H = m->H; p.Hh = m->H / 2; p.G = 3 * m->H; p.batch = a.batch;
     p.NCH = k.NCH; p.NRp = k.NRp; p.NO1 = k.NO1;
     p.n_steps = a.n_steps; p.step0 = a.step0; p.stream0 = a.stream0; p.seed = a.seed;
@@ -606,27 +782,27 @@ int bcluster_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.hop = m->cond_dim ? a.hop : 1;
     p.row_stride = m->cond_dim ? a.row_stride : 0;
     p.row_offset_mul = m->cond_dim ? a.row_offset_mul : 0;
-    p.Ip = k.Ip; p.b1 = m->b1; p.b2 = m->b2; p.b3 = m->b3; p.b4 = m->b4; p.g = m->g;
-    p.act0 = k.act[0]; p.act1 = k.act[1]; p.q = k.q; p.logits = k.logits;
-    p.c_cur = k.c_cur; p.c_prev = k.c_prev; p.f_prev = k.f_prev;
+    p.Ip = k.Ip; p.bp = k.bp; p.g = m->g;
+    p.act0 = k.act[0]; p.act1 = k.act[1]; p.q = k.q;
     p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in; p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
     p.tmWr = k.tmWr; p.tmO1 = k.tmO1; p.tmO2 = k.tmO2; p.tmO3 = k.tmO3; p.tmO4 = k.tmO4;
-    const long long arows = (long long)k.max_clusters * BC_MROWS;
-    if (!make_map(&p.tmAct[0], k.act[0], arows, m->H, p.MR) || !make_map(&p.tmAct[1], k.act[1], arows, m->H, p.MR) ||
-        !make_map(&p.tmQ, k.q, arows, m->H / 2, p.MR)) {
-        m->err = "tensor-map encoding failed";
-        return WRNN_ERR_CUDA;
-    }
-    // rows of the stacked images that no thread writes must read as zero
-    if (cudaMemsetAsync(k.act[0], 0, (size_t)arows * m->H * 2, s) != cudaSuccess || cudaMemsetAsync(k.act[1], 0, (size_t)arows * m->H * 2, s) != cudaSuccess ||
-        cudaMemsetAsync(k.q, 0, (size_t)arows * (m->H / 2) * 2, s) != cudaSuccess || cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess)
+    const int nkbA = m->H / 64, nkbH = m->H / 128;
+    const long long tilesA = (long long)k.max_clusters * nkbA, tilesH = (long long)k.max_clusters * nkbH;
+    bool ok = make_map_tiles(&p.tmQ, k.q, tilesH, BC_MROWS, g.MR, g.kpart);
+    for (int b = 0; b < 2; ++b)
+        ok = ok && make_map_tiles(&p.tmActA[b], k.act[b], tilesA, BC_MROWS, g.MR, 1) && make_map_tiles(&p.tmActO[b], k.act[b], tilesA, BC_MROWS, g.MR, g.kpart);
+    if (!ok) { m->err = "tensor-map encoding failed"; return WRNN_ERR_CUDA; }
+    // operand rows that no thread writes must read as zero
+    const size_t tile = (size_t)BC_MROWS * 64 * 2;
+    if (cudaMemsetAsync(k.act[0], 0, (size_t)tilesA * tile, s) != cudaSuccess || cudaMemsetAsync(k.act[1], 0, (size_t)tilesA * tile, s) != cudaSuccess ||
+        cudaMemsetAsync(k.q, 0, (size_t)tilesH * tile, s) != cudaSuccess || cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess)
         return WRNN_ERR_CUDA;
 
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(ncl * BC_CS); cfg.blockDim = dim3(BC_THREADS); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = s;
+    cfg.gridDim = dim3(g.n_cl * BC_CS); cfg.blockDim = dim3(BC_THREADS); cfg.dynamicSmemBytes = (size_t)g.smem; cfg.stream = s;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = BC_CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;

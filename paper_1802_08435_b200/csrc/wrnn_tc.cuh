@@ -41,6 +41,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *tm,
     asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
                  ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y) : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int x, int y, int z)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(dst), "l"(tm), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
 // shared-memory matrix descriptor of a K-major tile with 128-byte swizzle (rows of 128 bytes, 8-row atoms of 1 KB)
 __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr)
 {
@@ -55,6 +60,26 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t
 {
     asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
                  ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The four MMAs of one 64-wide k-block in one straight-line sequence: both descriptors advance by 32 bytes (2 units of
+// 16 bytes) per K = 16, which only touches their low words (a_lo, b_lo; the high word `hi` is common to every 128-byte
+// swizzled K-major tile); only the first MMA may overwrite the accumulator (accumulate_first == 0).
+constexpr uint32_t UMMA_DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t umma_desc_lo(uint32_t saddr) { return ((saddr >> 4) & 0x3FFFu) | (1u << 16); }
+__device__ __forceinline__ void umma_bf16_kblock(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate_first)
+{
+    asm volatile("{\n.reg .pred p, t;\n.reg .b32 a1, a2, a3, b1, b2, b3;\n.reg .b64 da, db;\n"
+                 "setp.ne.b32 p, %4, 0;\nsetp.eq.u32 t, %3, %3;\n"
+                 "add.u32 a1, %1, 2;\nadd.u32 b1, %2, 2;\nadd.u32 a2, %1, 4;\nadd.u32 b2, %2, 4;\nadd.u32 a3, %1, 6;\nadd.u32 b3, %2, 6;\n"
+                 "mov.b64 da, {%1, %5};\nmov.b64 db, {%2, %5};\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n"
+                 "mov.b64 da, {a1, %5};\nmov.b64 db, {b1, %5};\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, t;\n"
+                 "mov.b64 da, {a2, %5};\nmov.b64 db, {b2, %5};\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, t;\n"
+                 "mov.b64 da, {a3, %5};\nmov.b64 db, {b3, %5};\n"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, t;\n}"
+                 ::"r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate_first), "r"(UMMA_DESC_HI) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
@@ -75,6 +100,18 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&r)[8])
                  : "r"(taddr));
 #pragma unroll
     for (int i = 0; i < 8; ++i) r[i] = __uint_as_float(u[i]);
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&r)[32])
+{
+    uint32_t u[32];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]), "=r"(u[9]), "=r"(u[10]),
+                   "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]), "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]),
+                   "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]), "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]),
+                   "=r"(u[31])
+                 : "r"(taddr));
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(u[i]);
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -105,6 +142,20 @@ inline bool make_map(CUtensorMap *tm, void *base, long long rows, int cols, int 
     const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 3-D tensor map of an array of tiles [n_tiles][tile_rows][64] bf16 (one tile = one 64-wide k-block of up to tile_rows
+// operand rows): box (64 columns x box_rows x box_tiles), 128-byte swizzle
+inline bool make_map_tiles(CUtensorMap *tm, void *base, long long n_tiles, int tile_rows, int box_rows, int box_tiles)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)TC_BK, (cuuint64_t)tile_rows, (cuuint64_t)n_tiles};
+    const cuuint64_t strides[2] = {(cuuint64_t)TC_BK * 2, (cuuint64_t)TC_BK * 2 * (cuuint64_t)tile_rows};
+    const cuuint32_t box[3] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows, (cuuint32_t)box_tiles};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

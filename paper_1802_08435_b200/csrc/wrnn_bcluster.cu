@@ -244,6 +244,10 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
     const int s_r = (int)crank + BC_CS * warp;
     const bool sampler = warp < 4 && s_r < nrows;
     const int s_gb = row0 + s_r;
+    // The three single-thread roles of the contractions sit on lane 31 of warps 1, 3 and 5: as gate threads those lanes serve
+    // the last row slot of the group, which is empty unless the group has exactly 16, 32 or 64 rows, so that their role work
+    // does not delay gate work of their own.
+    const int role = (lane == 31 && (warp == 1 || warp == 3 || warp == 5)) ? (warp >> 1) : -1;   // 0: MMA issue, 1 / 2: TMA producers
     int last_c = sampler ? (p.c_in ? (int)p.c_in[s_gb] : 128) : 0, last_f = sampler ? (p.f_in ? (int)p.f_in[s_gb] : 0) : 0;
     fence_proxy_async();
     cluster_barrier();
@@ -257,7 +261,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
     // competes with the three role threads for issue slots.
     auto wait_done = [&](int step, int phase) {
         if (warp == 1) {
-            if (lane == 0) {
+            if (role == 0) {
                 RBEGIN();
                 if (!*failed && !mbar_wait(done_bar, dph)) fail(step, phase);
                 RSTAMP(31);
@@ -270,12 +274,12 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
     };
 
     // Phase A: D[128 x NRp] (TMEM column 0) = state tiles of buffer `cur` . (this CTA's rows of R)^T through the ring.
-    // warp 0 / lane 0 loads the activation tiles, warp 2 / lane 0 the weight tiles, warp 1 / lane 0 issues the MMAs.
+    // One role thread loads the activation tiles, one the weight tiles, one issues the MMAs.
     // The role loops are kept to a handful of instructions per k-block: a lone thread issues slowly.
     const uint32_t full0 = smem_u32(&s_full[0]), empty0 = smem_u32(&s_empty[0]);
     auto gemm_a_issue = [&](int cur, int step) {
-        if (lane == 0 && warp < 3 && !*failed) {
-            if (warp == 1) {
+        if (role >= 0 && !*failed) {
+            if (role == 0) {
                 const uint32_t idesc = umma_idesc_bf16(128, p.NRp);
                 const uint32_t dstep = (uint32_t)(p.stage_bytes >> 4), boff = abytes >> 4;
                 uint32_t da = umma_desc_lo(area0) + (uint32_t)rst * dstep;
@@ -292,7 +296,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 if (ok) umma_commit(done_bar);
                 else fail(step, 1);
             } else {
-                const bool is_act = warp == 0;
+                const bool is_act = role == 1;
                 const uint32_t bytes = is_act ? abytes : (uint32_t)p.NRp * 128u;
                 const CUtensorMap *tmA = &p.tmActA[cur];
                 uint32_t dst = area0 + (uint32_t)rst * (uint32_t)p.stage_bytes + (is_act ? 0u : abytes);
@@ -312,16 +316,15 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 }
             }
         }
-        __syncwarp();
     };
 
     // O phases: D[128 x n_w] (TMEM column dcol) = tiles tile0 .. tile0 + nkbH - 1 of an activation array . (resident weights)^T.
     // The operand arrives as two copies of kpart tiles; the MMAs of the first half start while the second is in flight.
     auto gemm_o_issue = [&](const CUtensorMap *tmA, int tile0, uint32_t wres, int n_w, uint32_t dcol, int step, int phase) {
-        if (lane == 0 && warp < 3 && !*failed) {
-            if (warp != 1) {
-                // warp 0 fetches the first half of the operand, warp 2 the second
-                const int part = warp >> 1;
+        if (role >= 0 && !*failed) {
+            if (role != 0) {
+                // one producer fetches the first half of the operand, the other the second
+                const int part = role - 1;
                 const uint32_t half_bytes = (uint32_t)p.kpart * abytes, fb = smem_u32(&s_ofull[part]);
                 mbar_expect_tx(fb, half_bytes);
                 tma_load_3d(area0 + (uint32_t)part * half_bytes, tmA, fb, 0, 0, tile0 + part * p.kpart);
@@ -350,7 +353,6 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
             }
         }
         oph ^= 1;
-        __syncwarp();
     };
 
     // Inputs of the gates of one half that do not depend on the contraction (I x + conditioning; x2 joins later for the
@@ -525,7 +527,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 const float4 v1 = *reinterpret_cast<const float4 *>(s_log + warp * 256 + 8 * lane + 4);
                 l[0] = v0.x; l[1] = v0.y; l[2] = v0.z; l[3] = v0.w; l[4] = v1.x; l[5] = v1.y; l[6] = v1.z; l[7] = v1.w;
                 const float u = uniform24(p.seed, p.stream0 + (unsigned)s_gb, (unsigned long long)(p.step0 + s), head);
-                drawn = warp_softmax_draw(l, u, lane);
+                drawn = warp_softmax_draw_fast(l, u, lane);
                 const uint8_t *forced = head ? p.f_forced : p.c_forced;
                 used = forced ? (int)forced[s_o] : drawn;
                 if (lane < BC_CS) {

@@ -82,6 +82,51 @@ def test_tiny_batched_kernel(env, kernel, H, batch):
         B.wrnn_destroy(m)
 
 
+@pytest.mark.parametrize("kernel", ["BATCHED", "BCLUSTER"])
+def test_multirow_resume_unconditioned_and_wide_models(env, kernel):
+    """The multi-row kernels: (1) a run split in two calls that carry (h, c, f) reproduces the unsplit run bit for bit;
+    (2) a model without conditioning and without biases; (3) wider models (other chunk counts per CTA, H = 1024 being the
+    largest the cluster-partitioned kernel takes)."""
+    torch, B = env
+    kid = getattr(B, "WRNN_KERNEL_" + kernel)
+    w = _tiny(128)
+    m = B.wrnn_create(w, "bf16", max_batch=19, kernel=kid)
+    try:
+        cond = synth.make_cond(19, 12, 4)
+        full = _free_run(torch, B, m, cond, 90, 19, 77, hop=10)
+        h = torch.zeros((19, 128), dtype=torch.float32, device="cuda:0")
+        cp = torch.full((19,), 128, dtype=torch.uint8, device="cuda:0")
+        fp = torch.zeros((19,), dtype=torch.uint8, device="cuda:0")
+        a = _free_run(torch, B, m, cond, 35, 19, 77, hop=10, h=h, c_prev=cp, f_prev=fp)
+        b = _free_run(torch, B, m, cond, 55, 19, 77, hop=10, h=h, c_prev=cp, f_prev=fp, step0=35)
+        assert np.array_equal(np.concatenate([a, b], axis=1), full)
+        again = _free_run(torch, B, m, cond, 90, 19, 77, hop=10)
+        assert np.array_equal(again, full)                                   # deterministic
+    finally:
+        B.wrnn_destroy(m)
+    w = _tiny(128, cond_dim=0)
+    for k in ("b_gate", "b1", "b2", "b3", "b4"):
+        w[k] = None
+    om = orc.OracleModel(w, "bf16")
+    m = B.wrnn_create(w, "bf16", max_batch=5, kernel=kid)
+    try:
+        r = pu.teacher_forced_parity(torch, B, m, om, None, 40, 5, 5, threads=pu.NCPU)
+        assert r["idx_bad"] == 0 and max(r["gates_err"], r["h_err"], r["logits_err"]) < pu.TOL["bf16"], {k: v for k, v in r.items() if k != "oracle"}
+    finally:
+        B.wrnn_destroy(m)
+    for H, batch in [(512, 40), (1024, 24)]:
+        w = _tiny(H, scale=1.5)
+        om = orc.OracleModel(w, "bf16")
+        m = B.wrnn_create(w, "bf16", max_batch=batch, kernel=kid)
+        try:
+            assert B.wrnn_launch_info(m, batch)["kernel"] == kid
+            cond = synth.make_cond(batch, 8, 4)
+            r = pu.teacher_forced_parity(torch, B, m, om, cond, 12, batch, SEED, hop=10, row_stride=1, row_offset_mul=1, threads=pu.NCPU)
+            assert r["idx_bad"] == 0 and max(r["gates_err"], r["h_err"], r["logits_err"]) < pu.TOL["bf16"], {k: v for k, v in r.items() if k != "oracle"}
+        finally:
+            B.wrnn_destroy(m)
+
+
 def test_unconditioned_model_and_null_biases(env):
     torch, B = env
     w = _tiny(16, cond_dim=0)

@@ -237,6 +237,13 @@ int wrnn_phase_cycles(wrnn_model *m, int64_t *out16);
  * allocates and frees a small device buffer. */
 int wrnn_measure_exchange_floor(int32_t n_ctas, int32_t n_threads, int32_t K, int32_t iters, float *ns_per_exchange);
 
+/* Self-test of the bounded device-side waits (the error path of every persistent kernel here): a two-CTA kernel whose
+ * first CTA waits at the grid barrier for an arrival that never comes, gives up after limit_ns (1 us .. 1 s of the
+ * global timer) and returns.  *code receives the device status word (WRNN_ERR_TIMEOUT when the wait ran out as it
+ * should), the optional HOST out-pointers the (cta, step, phase) it recorded (0, 7, 3) and the kernel's duration.
+ * Nothing faults and the context stays usable.  Synchronous; allocates and frees two small device buffers. */
+int wrnn_selftest_bounded_wait(int64_t limit_ns, int32_t *code, int32_t *cta, int32_t *step, int32_t *phase, float *waited_ms);
+
 /* Kernels launched by this library in this process since load (all models). */
 int64_t wrnn_launch_count(void);
 

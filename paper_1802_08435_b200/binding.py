@@ -26,6 +26,7 @@ EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
     "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor", "wrnn_sample_noalloc",
+    "wrnn_selftest_bounded_wait",
 ]
 
 
@@ -83,6 +84,7 @@ def lib():
         L.wrnn_launch_info.argtypes = [vp, i32] + [vp] * 5
         L.wrnn_phase_cycles.argtypes = [vp, vp]
         L.wrnn_measure_exchange_floor.argtypes = [i32, i32, i32, i32, vp]
+        L.wrnn_selftest_bounded_wait.argtypes = [i64] + [vp] * 5
         L.wrnn_launch_count.argtypes = []
         L.wrnn_launch_count.restype = i64
         _lib = L
@@ -239,6 +241,13 @@ def wrnn_measure_exchange_floor(n_ctas: int, n_threads: int, K: int, iters: int 
     out = C.c_float()
     _check(lib().wrnn_measure_exchange_floor(n_ctas, n_threads, K, iters, C.byref(out)))
     return out.value
+
+
+def wrnn_selftest_bounded_wait(limit_ns: int = 50_000_000) -> dict:
+    """Run the bounded-wait self-test; returns the device status word, where it was recorded and the kernel time."""
+    code, cta, step, phase, ms = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32(), C.c_float()
+    _check(lib().wrnn_selftest_bounded_wait(limit_ns, C.byref(code), C.byref(cta), C.byref(step), C.byref(phase), C.byref(ms)))
+    return {"code": code.value, "cta": cta.value, "step": step.value, "phase": phase.value, "waited_ms": ms.value}
 
 
 def wrnn_sample_noalloc(model, cond, n_steps: int, batch: int, seed: int, out, *, hop: int = 120, row_stride: int = 1,

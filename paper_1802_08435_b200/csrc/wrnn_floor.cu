@@ -75,3 +75,50 @@ extern "C" int wrnn_measure_exchange_floor(int32_t n_ctas, int32_t n_threads, in
     if (rc == WRNN_OK) *ns_per_exchange = ms * 1e6f / (float)iters;
     return rc;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded waits: two CTAs, the first waits at the grid barrier for an arrival that never comes
+// (the second returns at once), gives up after limit_ns, records where, and returns; the context stays usable.
+namespace wrnn {
+__global__ void bounded_wait_selftest_kernel(unsigned long long *counter, DevStatus *status, unsigned long long limit_ns)
+{
+    if (blockIdx.x != 0) return;
+    GridBarrier bar{counter, status, 0ull, limit_ns};
+    bar.sync(7, 3);
+}
+}  // namespace wrnn
+
+extern "C" int wrnn_selftest_bounded_wait(int64_t limit_ns, int32_t *code, int32_t *cta, int32_t *step, int32_t *phase, float *waited_ms)
+{
+    if (limit_ns < 1000 || limit_ns > 1000000000ll || !code) return WRNN_ERR_INVALID_ARG;
+    unsigned long long *counter = nullptr;
+    wrnn::DevStatus *status = nullptr;
+    if (cudaMalloc((void **)&counter, 8) != cudaSuccess || cudaMalloc((void **)&status, sizeof(wrnn::DevStatus)) != cudaSuccess) {
+        cudaGetLastError(); cudaFree(counter); return WRNN_ERR_NOMEM;
+    }
+    cudaMemset(counter, 0, 8);
+    cudaMemset(status, 0, sizeof(wrnn::DevStatus));
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0); cudaEventCreate(&e1);
+    cudaEventRecord(e0, 0);
+    wrnn::bounded_wait_selftest_kernel<<<2, 64>>>(counter, status, (unsigned long long)limit_ns);
+    ++wrnn::g_launches;
+    cudaEventRecord(e1, 0);
+    int rc = cudaEventSynchronize(e1) == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
+    float ms = 0.f;
+    wrnn::DevStatus h = {0, 0, 0, 0};
+    if (rc == WRNN_OK) {
+        cudaEventElapsedTime(&ms, e0, e1);
+        if (cudaMemcpy(&h, status, sizeof(h), cudaMemcpyDeviceToHost) != cudaSuccess) rc = WRNN_ERR_CUDA;
+    }
+    *code = h.code;
+    if (cta) *cta = h.cta;
+    if (step) *step = h.step;
+    if (phase) *phase = h.phase;
+    if (waited_ms) *waited_ms = ms;
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    cudaFree(counter); cudaFree(status);
+    cudaGetLastError();
+    return rc;
+}
+

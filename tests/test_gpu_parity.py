@@ -207,6 +207,22 @@ def test_resume_and_state_roundtrip(env):
         B.wrnn_destroy(m)
 
 
+def test_bounded_wait_gives_up_cleanly(env):
+    """A device-side wait for an arrival that never comes ends after its limit with WRNN_ERR_TIMEOUT recorded at the right
+    place, and the context stays usable (a sampling call afterwards works)."""
+    torch, B = env
+    r = B.wrnn_selftest_bounded_wait(30_000_000)
+    assert r["code"] == B.WRNN_ERR_TIMEOUT and (r["cta"], r["step"], r["phase"]) == (0, 7, 3), r
+    assert 25.0 < r["waited_ms"] < 500.0, r
+    w = _tiny(16)
+    m = B.wrnn_create(w, "f32", kernel=B.WRNN_KERNEL_GENERIC)
+    try:
+        out = _free_run(torch, B, m, synth.make_cond(1, 4, 4), 20, 1, 3, hop=10)
+        assert out.shape == (1, 20)
+    finally:
+        B.wrnn_destroy(m)
+
+
 def test_fold_unfold_exact_permutation(env):
     torch, B = env
     for n, Bf in [(24000, 16), (16, 16), (35, 5), (7, 1)]:

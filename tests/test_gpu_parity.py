@@ -259,6 +259,32 @@ def test_argument_errors(env):
 # ---------------------------------------------------------------------------------------------
 # The named workloads at their full sizes (index = position in synth.WORKLOADS)
 
+@pytest.mark.parametrize("batch", [1, 32])
+def test_peaky_distributions(env, batch):
+    """The benchmark model with O2 and O4 scaled by 32: logits spread over tens of units, so the softmax is far from uniform
+    and exp sees large negative arguments (the synthetic weights alone give near-uniform distributions).  Batch 1 runs
+    on the resident kernel, batch 32 on the cluster-partitioned one."""
+    torch, B = env
+    wl = synth.WORKLOADS[1]
+    w, masks, _ = synth.build_workload(wl)
+    w = dict(w)
+    w["O2"] = (w["O2"] * 32).astype(np.float32)
+    w["O4"] = (w["O4"] * 32).astype(np.float32)
+    n_steps = 600 if batch == 1 else 40
+    cond = synth.make_cond(batch, n_steps // 120 + 2, 64)
+    om = orc.OracleModel(w, wl.dtype)
+    m = B.wrnn_create(w, wl.dtype, max_batch=batch)
+    try:
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, n_steps, batch, SEED, threads=pu.NCPU)
+        _report("peaky O2/O4 x32, batch %d" % batch, r)
+        lg = r["oracle"].logits if hasattr(r["oracle"], "logits") else None
+        if lg is not None:
+            assert float(np.max(lg) - np.min(lg)) > 16.0                    # the case is what it claims to be
+        _tol_check(r, wl.dtype)
+    finally:
+        B.wrnn_destroy(m)
+
+
 def _tol_check(r, dtype):
     tol = pu.TOL[dtype]
     assert r["idx_bad"] == 0, {k: v for k, v in r.items() if k != "oracle"}

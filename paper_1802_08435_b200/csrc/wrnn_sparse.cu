@@ -7,8 +7,9 @@
 // layer of a head, its logits -- is an all-gather of (value, tag) words through distributed shared memory.
 // Each CTA owns Hh/16 coarse and Hh/16 fine units (their block rows of R, compressed: block column index +
 // 16 bf16 per kept block), Hh/16 rows of O1 and O3 (compressed block rows) and 16 rows of the dense O2 and O4
-// (mma.sync A fragments).  Sparse rows: eight lanes share a block row, each lane takes every eighth kept
-// block (two 16-byte weight loads, four activations, 16 FMAs), a four-value reduce-scatter finishes the rows.
+// (mma.sync A fragments).  Sparse rows: four lanes share a block row, each lane takes every fourth kept block
+// (two 16-byte weight loads, four activations, 16 FMAs), a four-value reduce-scatter finishes the rows; the rows
+// are sorted by length and stored sliced by warp so that every shared-memory load of a warp is one contiguous run.
 // The step itself is the two-half schedule of the dense resident kernel (Fig. 1's order).
 //
 // Every wait is bounded; all CTAs leave through the final cluster barrier.
@@ -28,11 +29,18 @@ namespace wrnn {
 constexpr int SCS = 16;          // cluster size
 constexpr int SNW = 20;          // warps per CTA
 
+// Compressed block rows of one phase of one CTA, sliced by warp: the block rows are sorted by their number of kept
+// blocks and dealt out in runs of up to eight to the warps, four lanes per block row; lane 4 g + l of warp w takes
+// blocks l, l + 4, ... of its row g.  Iteration t of a warp reads slot t * nl + lane of its slice (nl = 4 x rows of
+// the warp): the two 16-byte halves of the block's weights from two planes and the block column, so every load of a
+// warp is one contiguous run; rows shorter than the warp's longest are padded with zero blocks.
+struct SliceMeta { int voff, coff, T, nl; int16_t row[8]; };     // offsets in 16-byte / 2-byte units from the phase's arrays
+
 struct SparsePack {
     int H = 0, K = 0, NKT = 0, UC = 0, HR = 0, NBR = 0;   // NBR: block rows per phase = (HR + 6 UC) / 4
-    int max_nnz = 0;                  // kept blocks per phase per CTA (padded maximum)
+    int max_slots = 0;                // block slots per phase per CTA (kept blocks + padding of the sliced layout, maximum)
     size_t blob_bytes = 0;            // per CTA
-    size_t off_brp[2], off_col[2], off_val[2], off_o2 = 0, off_o4 = 0, off_small = 0;
+    size_t off_meta[2], off_col[2], off_val[2], off_o2 = 0, off_o4 = 0, off_small = 0;
     uint8_t *d_blob = nullptr;
     int smem_bytes = 0;
     int64_t weight_bytes_per_step = 0;   // kept blocks + indices + row pointers + dense O2/O4/I, each counted once
@@ -40,7 +48,7 @@ struct SparsePack {
 
 struct SparseParams {
     int H, K, NKT, UC, HR, NBR;
-    unsigned long long off_brp[2], off_col[2], off_val[2], off_o2, off_o4, off_small, blob_bytes;
+    unsigned long long off_meta[2], off_col[2], off_val[2], off_o2, off_o4, off_small, blob_bytes;
     long long n_steps, step0;
     unsigned stream0;
     unsigned long long seed;
@@ -59,7 +67,7 @@ struct SparseParams {
 
 #ifdef WRNN_PROFILE_SPARSE
 __device__ long long g_sprof[16];
-#define SSTAMP(i) do { if (blockIdx.x == 0 && warp == 0) { const long long n_ = clock64(); if (lane == 0) g_sprof[i] += n_ - st_; st_ = n_; } } while (0)
+#define SSTAMP(i) do { if (warp == 0) { const long long n_ = clock64(); if (lane == 0) s_sprof[i] += n_ - st_; st_ = n_; } } while (0)
 #else
 #define SSTAMP(i) do { } while (0)
 #endif
@@ -76,7 +84,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     const int NR = 6 * UC;
 
     // ---- shared memory carve-up (must match sparse_smem_bytes)
-    const int *brp[2] = {reinterpret_cast<const int *>(smem + p.off_brp[0]), reinterpret_cast<const int *>(smem + p.off_brp[1])};
+    const SliceMeta *smeta[2] = {reinterpret_cast<const SliceMeta *>(smem + p.off_meta[0]), reinterpret_cast<const SliceMeta *>(smem + p.off_meta[1])};
     const uint16_t *bcol[2] = {reinterpret_cast<const uint16_t *>(smem + p.off_col[0]), reinterpret_cast<const uint16_t *>(smem + p.off_col[1])};
     const uint4 *bval[2] = {reinterpret_cast<const uint4 *>(smem + p.off_val[0]), reinterpret_cast<const uint4 *>(smem + p.off_val[1])};
     const uint4 *wO2 = reinterpret_cast<const uint4 *>(smem + p.off_o2), *wO4 = reinterpret_cast<const uint4 *>(smem + p.off_o4);
@@ -90,15 +98,17 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     float *part = a_full + NR;                                                        // [16 warps][16]
     float *ynew = part + 256;                                                         // [UC] freshly gated units
     __nv_bfloat16 *splQ = reinterpret_cast<__nv_bfloat16 *>(ynew + ((UC + 3) & ~3));  // split image of q, 4 K bf16
-    uint4 *ybuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                            // [2][K/2] state halves
-    uint4 *qbuf = ybuf + K;                                                           // [2][K/2] hidden layer
-    uint4 *lbuf = qbuf + K;                                                           // [2][128] logits
+    // Exchange buffers, one of each: a peer can only write the next half-step's words after it has received words that
+    // this CTA sent after reading the current ones (y(n+1) follows q(n), q(n+1) follows y(n+1), logits(n+1) follow q(n+1)).
+    uint4 *ybuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                            // [K/2] state half
+    uint4 *qbuf = ybuf + K / 2;                                                       // [K/2] hidden layer
+    uint4 *lbuf = qbuf + K / 2;                                                       // [128] logits
 
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(p.blob + (size_t)rank * p.blob_bytes);
         uint4 *dst = reinterpret_cast<uint4 *>(smem);
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
-        for (int i = tid; i < 2 * K + 256; i += blockDim.x) ybuf[i] = make_uint4(0, 0, 0, 0);   // ybuf, qbuf, lbuf are adjacent
+        for (int i = tid; i < K + 128; i += blockDim.x) ybuf[i] = make_uint4(0, 0, 0, 0);   // ybuf, qbuf, lbuf are adjacent
         for (int i = tid; i < 4 * K / 8; i += blockDim.x) reinterpret_cast<uint4 *>(splQ)[i] = make_uint4(0, 0, 0, 0);
         for (int i = tid; i < K; i += blockDim.x) {
             vecC[i] = p.h_in ? p.h_in[i] : 0.f;
@@ -111,45 +121,59 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
     const bool writer = (rank == 0);
+#ifdef WRNN_PROFILE_SPARSE
+    __shared__ long long s_sprof[16];
+    long long st_ = clock64();
+#endif
 
     int c_prev = p.c_in ? p.c_in[0] : 128, f_prev = p.f_in ? p.f_in[0] : 0;
 
     // ---- sparse phase: block rows [0, NBR) of phase ph (0: input y_c -> [O1 ; R x coarse cols], 1: y_f -> [O3 ; R x fine cols]).
-    // Eight lanes per block row.  Rows [0, HR) are hidden-layer rows (bias, relu, sent to all peers when send != 0),
+    // Four lanes per block row.  Rows [0, HR) are hidden-layer rows (bias, relu, sent to all peers when send != 0),
     // rows [HR, HR + NR) are this CTA's R rows (ph 1 completes R h, ph 0 keeps the partial for the next step).
+    // this warp's slices of the two phases: constants of the whole call, kept in registers
+    const SliceMeta &sm0 = smeta[0][warp], &sm1 = smeta[1][warp];
+    const int sl_nl0 = sm0.nl, sl_nl1 = sm1.nl, sl_T0 = sm0.T, sl_T1 = sm1.T;
+    const uint4 *sl_wv0 = bval[0] + sm0.voff + (lane < sl_nl0 ? lane : 0), *sl_wv1 = bval[1] + sm1.voff + (lane < sl_nl1 ? lane : 0);
+    const uint16_t *sl_wc0 = bcol[0] + sm0.coff + (lane < sl_nl0 ? lane : 0), *sl_wc1 = bcol[1] + sm1.coff + (lane < sl_nl1 ? lane : 0);
+    const int sl_row0 = lane < sl_nl0 ? (int)sm0.row[lane >> 2] : -1, sl_row1 = lane < sl_nl1 ? (int)sm1.row[lane >> 2] : -1;
+
     auto sparse_phase = [&](int ph, const float *x, const float *bias) {
-        // Four lanes per block row (sub-group q = lane >> 2 of warp w takes block row q * SNW + w, so that the
-        // hidden-layer rows and the R rows are spread over all warps); each lane takes every fourth kept block.
-        const int l4 = lane & 3;
-        const int nrounds = (NBR + 8 * SNW - 1) / (8 * SNW);
-        for (int round = 0; round < nrounds; ++round) {
-            const int lbr_raw = round * 8 * SNW + (lane >> 2) * SNW + warp;
-            const bool valid = lbr_raw < NBR;
-            const int lbr = valid ? lbr_raw : 0;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-            const int beg = brp[ph][lbr], end = valid ? brp[ph][lbr + 1] : beg;
-            for (int i = beg + l4; i < end; i += 4) {
-                const uint4 w0 = bval[ph][2 * i], w1 = bval[ph][2 * i + 1];
-                const float4 xv = *reinterpret_cast<const float4 *>(x + 4 * (int)bcol[ph][i]);
-                acc[0] = fmaf(bf16lo(w0.x), xv.x, fmaf(bf16hi(w0.x), xv.y, fmaf(bf16lo(w0.y), xv.z, fmaf(bf16hi(w0.y), xv.w, acc[0]))));
-                acc[1] = fmaf(bf16lo(w0.z), xv.x, fmaf(bf16hi(w0.z), xv.y, fmaf(bf16lo(w0.w), xv.z, fmaf(bf16hi(w0.w), xv.w, acc[1]))));
-                acc[2] = fmaf(bf16lo(w1.x), xv.x, fmaf(bf16hi(w1.x), xv.y, fmaf(bf16lo(w1.y), xv.z, fmaf(bf16hi(w1.y), xv.w, acc[2]))));
-                acc[3] = fmaf(bf16lo(w1.z), xv.x, fmaf(bf16hi(w1.z), xv.y, fmaf(bf16lo(w1.w), xv.z, fmaf(bf16hi(w1.w), xv.w, acc[3]))));
-            }
-            // four row sums over four lanes: two transposing steps leave row l4 in lane l4
-            const bool up2 = (l4 & 2) != 0;
-            const float s0 = up2 ? acc[0] : acc[2], k0 = up2 ? acc[2] : acc[0];
-            const float s1 = up2 ? acc[1] : acc[3], k1 = up2 ? acc[3] : acc[1];
-            const float t0 = k0 + __shfl_xor_sync(FULL, s0, 2);
-            const float t1 = k1 + __shfl_xor_sync(FULL, s1, 2);
-            const bool up1 = (l4 & 1) != 0;
-            const float v = (up1 ? t1 : t0) + __shfl_xor_sync(FULL, up1 ? t0 : t1, 1);
-            if (valid) {
-                const int row = 4 * lbr + l4;
-                if (row < HR) qvec[row] = fmaxf(v + bias[row], 0.f);
-                else if (ph) a_full[row - HR] = a_part[row - HR] + v;
-                else a_part[row - HR] = v;
-            }
+        const int nl = ph ? sl_nl1 : sl_nl0, T = ph ? sl_T1 : sl_T0, l4 = lane & 3;
+        const uint4 *wv = ph ? sl_wv1 : sl_wv0;
+        const uint16_t *wc = ph ? sl_wc1 : sl_wc0;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        SSTAMP(9);
+        // software pipeline: the weights and the column of the next block are in flight while this block's four
+        // activations are gathered and multiplied (the last prefetch re-reads the last slot)
+        uint4 w0 = wv[0], w1 = wv[nl];
+        int c = wc[0];
+        for (int t = 0; t < T; ++t) {
+            const float4 xv = *reinterpret_cast<const float4 *>(x + 4 * c);
+            const int tn = t + 1 < T ? t + 1 : t;
+            const uint4 w0n = wv[(2 * tn) * nl], w1n = wv[(2 * tn + 1) * nl];
+            const int cn = wc[tn * nl];
+            acc[0] = fmaf(bf16lo(w0.x), xv.x, fmaf(bf16hi(w0.x), xv.y, fmaf(bf16lo(w0.y), xv.z, fmaf(bf16hi(w0.y), xv.w, acc[0]))));
+            acc[1] = fmaf(bf16lo(w0.z), xv.x, fmaf(bf16hi(w0.z), xv.y, fmaf(bf16lo(w0.w), xv.z, fmaf(bf16hi(w0.w), xv.w, acc[1]))));
+            acc[2] = fmaf(bf16lo(w1.x), xv.x, fmaf(bf16hi(w1.x), xv.y, fmaf(bf16lo(w1.y), xv.z, fmaf(bf16hi(w1.y), xv.w, acc[2]))));
+            acc[3] = fmaf(bf16lo(w1.z), xv.x, fmaf(bf16hi(w1.z), xv.y, fmaf(bf16lo(w1.w), xv.z, fmaf(bf16hi(w1.w), xv.w, acc[3]))));
+            w0 = w0n; w1 = w1n; c = cn;
+        }
+        SSTAMP(10);
+        // four row sums over four lanes: two transposing steps leave row l4 in lane l4
+        const bool up2 = (l4 & 2) != 0;
+        const float s0 = up2 ? acc[0] : acc[2], k0 = up2 ? acc[2] : acc[0];
+        const float s1 = up2 ? acc[1] : acc[3], k1 = up2 ? acc[3] : acc[1];
+        const float t0 = k0 + __shfl_xor_sync(FULL, s0, 2);
+        const float t1 = k1 + __shfl_xor_sync(FULL, s1, 2);
+        const bool up1 = (l4 & 1) != 0;
+        const float v = (up1 ? t1 : t0) + __shfl_xor_sync(FULL, up1 ? t0 : t1, 1);
+        const int lbr = ph ? sl_row1 : sl_row0;
+        if (lbr >= 0) {
+            const int row = 4 * lbr + l4;
+            if (row < HR) qvec[row] = fmaxf(v + bias[row], 0.f);
+            else if (ph) a_full[row - HR] = a_part[row - HR] + v;
+            else a_part[row - HR] = v;
         }
     };
 
@@ -187,7 +211,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     auto publish = [&](unsigned ytag) {
         if (warp < SCS) {
             for (int pr2 = lane; pr2 < UC / 2; pr2 += 32) {
-                const unsigned a = map_to_rank(smem_addr(ybuf + (size_t)(ytag & 1) * (K / 2) + (rank * UC) / 2 + pr2), warp);
+                const unsigned a = map_to_rank(smem_addr(ybuf + (rank * UC) / 2 + pr2), warp);
                 st_cluster_ll(a, ynew[2 * pr2], ynew[2 * pr2 + 1], ytag);
             }
         }
@@ -211,7 +235,9 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     const bool l_on = warp < KSL;
 
 #ifdef WRNN_PROFILE_SPARSE
-    long long st_ = clock64();
+    if (tid < 16) s_sprof[tid] = 0;
+    __syncthreads();
+    st_ = clock64();
 #endif
     const long long T = p.n_steps;
 #pragma unroll 1
@@ -219,7 +245,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         const int half = (int)(n & 1);                 // 1: coarse half (input y_c(s)), 0: fine half (input y_f(s-1))
         const long long s = n >> 1;
         const bool last = n == 2 * T;
-        const unsigned tag = (unsigned)n, par = (unsigned)((n - 1) & 1);
+        const unsigned tag = (unsigned)n;
         float *vec = half ? vecC : vecF;
 
         float u01 = 0.f, gv[3] = {0.f, 0.f, 0.f};
@@ -231,10 +257,10 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
         }
 
-        // ---- 1. the input half of the state from all 16 CTAs (published with tag n into buffer n & 1)
+        // ---- 1. the input half of the state from all 16 CTAs (published with tag n)
 #pragma unroll 1
         for (int i = tid; i < K / 2; i += blockDim.x) {
-            const unsigned a = smem_addr(ybuf + (size_t)(n & 1) * (K / 2) + i);
+            const unsigned a = smem_addr(ybuf + i);
             uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
             while (true) {
                 v = ld_shared_volatile_v4(a);
@@ -248,11 +274,13 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
 
         // ---- 2. hidden layer of the head + this CTA's R rows (compressed block rows)
         sparse_phase(half ? 0 : 1, vec, half ? sb1 : sb3);
+        SSTAMP(7);
         __syncthreads();
+        SSTAMP(8);
         // this CTA's HR hidden-layer values -> every peer, one coalesced 16-byte-per-lane store per peer (warp w -> peer w)
         if (warp < SCS) {
             for (int pr2 = lane; pr2 < HR / 2; pr2 += 32) {
-                const unsigned a = map_to_rank(smem_addr(qbuf + (size_t)par * (K / 2) + (rank * HR) / 2 + pr2), warp);
+                const unsigned a = map_to_rank(smem_addr(qbuf + (rank * HR) / 2 + pr2), warp);
                 st_cluster_ll(a, qvec[2 * pr2], qvec[2 * pr2 + 1], tag);
             }
         }
@@ -261,7 +289,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         // ---- 3. the cluster's hidden layer -> 16 logits rows of this CTA
 #pragma unroll 1
         for (int i = tid; i < K / 2; i += blockDim.x) {
-            const unsigned a = smem_addr(qbuf + (size_t)par * (K / 2) + i);
+            const unsigned a = smem_addr(qbuf + i);
             uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
             while (true) {
                 v = ld_shared_volatile_v4(a);
@@ -290,7 +318,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const int peer = 4 * k + (lane >> 3);
-                const unsigned a = map_to_rank(smem_addr(lbuf + (size_t)par * 128 + (rank * 16) / 2 + (lane & 7)), peer);
+                const unsigned a = map_to_rank(smem_addr(lbuf + (rank * 16) / 2 + (lane & 7)), peer);
                 st_cluster_ll(a, v0, v1, tag);
             }
         }
@@ -300,7 +328,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             float l[8];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const unsigned a = smem_addr(lbuf + (size_t)par * 128 + 4 * lane + k);
+                const unsigned a = smem_addr(lbuf + 4 * lane + k);
                 uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
                 while (true) {
                     v = ld_shared_volatile_v4(a);
@@ -337,6 +365,9 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         if (!last) publish((unsigned)(n + 1));
     }
 
+#ifdef WRNN_PROFILE_SPARSE
+    if (blockIdx.x == 0 && tid == 0) for (int i = 0; i < 16; ++i) g_sprof[i] += s_sprof[i];
+#endif
     const int any_bad = __syncthreads_or(my_bad);
     if (writer && !any_bad) {
         if (p.h_out) for (int i = tid; i < K; i += blockDim.x) { p.h_out[i] = vecC[i]; p.h_out[K + i] = vecF[i]; }
@@ -359,8 +390,8 @@ static int sparse_smem_bytes(const SparsePack &k)
     b += 256 * 4;                                  // part
     b += (size_t)((k.UC + 3) & ~3) * 4;            // ynew
     b += (size_t)4 * k.K * 2;                      // split image of q
-    b += (size_t)2 * k.K * 16;                     // ybuf, qbuf: [2][K/2] x 16 B each
-    b += 256 * 16;                                 // lbuf
+    b += (size_t)k.K * 16;                         // ybuf, qbuf: [K/2] x 16 B each
+    b += 128 * 16;                                 // lbuf
     return (int)b;
 }
 
@@ -430,15 +461,37 @@ int sparse_prepare(wrnn_model *m)
                 }
             }
         }
-    int max_nnz = 0;
-    for (auto &R : rows) { int n = 0; for (auto &r : R) n += (int)r.size(); max_nnz = std::max(max_nnz, n); }
-    k.max_nnz = (max_nnz + 7) & ~7;
+    // slice every (CTA, phase): block rows sorted by length (longest first, stable), dealt to the warps in runs
+    struct Slice { std::vector<int> rows; int T = 0; };
+    const int base_rows = NBR / SNW, extra = NBR % SNW;
+    if (base_rows + (extra ? 1 : 0) > 8) { m->err = "too many block rows per warp"; return WRNN_ERR_UNSUPPORTED; }
+    std::vector<std::vector<Slice>> slices(SCS * 2);              // [cta * 2 + phase][warp]
+    int max_slots = 0;
+    for (int cp = 0; cp < SCS * 2; ++cp) {
+        const auto &R = rows[cp];
+        std::vector<int> order(NBR);
+        for (int i = 0; i < NBR; ++i) order[i] = i;
+        std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return R[a].size() > R[b].size(); });
+        slices[cp].assign(SNW, {});
+        int next = 0, slots = 0;
+        for (int w = 0; w < SNW; ++w) {
+            const int nr = base_rows + (w < extra ? 1 : 0);
+            Slice &sl = slices[cp][w];
+            size_t longest = 0;
+            for (int i = 0; i < nr; ++i) { sl.rows.push_back(order[next + i]); longest = std::max(longest, R[order[next + i]].size()); }
+            next += nr;
+            sl.T = (int)((longest + 3) / 4);
+            slots += 4 * nr * sl.T;
+        }
+        max_slots = std::max(max_slots, slots);
+    }
+    k.max_slots = (max_slots + 7) & ~7;
 
     size_t off = 0;
     for (int ph = 0; ph < 2; ++ph) {
-        k.off_brp[ph] = off; off = a16(off + (size_t)(NBR + 1) * 4);
-        k.off_col[ph] = off; off = a16(off + (size_t)k.max_nnz * 2);
-        k.off_val[ph] = off; off = a16(off + (size_t)k.max_nnz * 32);
+        k.off_meta[ph] = off; off = a16(off + (size_t)SNW * sizeof(SliceMeta));
+        k.off_col[ph] = off; off = a16(off + (size_t)k.max_slots * 2);
+        k.off_val[ph] = off; off = a16(off + (size_t)k.max_slots * 32);
     }
     const size_t frag = (size_t)k.NKT * 512;
     k.off_o2 = off; off += frag;
@@ -467,19 +520,29 @@ int sparse_prepare(wrnn_model *m)
     for (int cta = 0; cta < SCS; ++cta) {
         uint8_t *base = blob.data() + (size_t)cta * k.blob_bytes;
         for (int ph = 0; ph < 2; ++ph) {
-            int *brp = reinterpret_cast<int *>(base + k.off_brp[ph]);
+            SliceMeta *meta = reinterpret_cast<SliceMeta *>(base + k.off_meta[ph]);
             uint16_t *col = reinterpret_cast<uint16_t *>(base + k.off_col[ph]);
-            uint16_t *val = reinterpret_cast<uint16_t *>(base + k.off_val[ph]);
-            int n = 0;
-            for (int lbr = 0; lbr < NBR; ++lbr) {
-                brp[lbr] = n;
-                for (const Blk &b : rows[cta * 2 + ph][lbr]) {
-                    col[n] = b.col;
-                    for (int e = 0; e < 16; ++e) val[(size_t)n * 16 + e] = bf16_bits_s(b.v[e]);
-                    ++n;
+            uint16_t *val = reinterpret_cast<uint16_t *>(base + k.off_val[ph]);       // [slot plane][8 bf16]
+            const auto &R = rows[cta * 2 + ph];
+            int slot0 = 0, n = 0;
+            for (int w = 0; w < SNW; ++w) {
+                const Slice &sl = slices[cta * 2 + ph][w];
+                const int nl = 4 * (int)sl.rows.size();
+                meta[w].voff = 2 * slot0; meta[w].coff = slot0; meta[w].T = sl.T; meta[w].nl = nl;
+                for (int g = 0; g < 8; ++g) meta[w].row[g] = g < (int)sl.rows.size() ? (int16_t)sl.rows[g] : (int16_t)-1;
+                for (int g = 0; g < (int)sl.rows.size(); ++g) {
+                    const auto &blocks = R[sl.rows[g]];
+                    for (int i = 0; i < (int)blocks.size(); ++i) {
+                        const int t = i / 4, lane = 4 * g + i % 4;
+                        col[slot0 + t * nl + lane] = blocks[i].col;
+                        for (int h = 0; h < 2; ++h)                  // plane h holds rows 2 h, 2 h + 1 of the block
+                            for (int e = 0; e < 8; ++e)
+                                val[((size_t)2 * slot0 + (size_t)(2 * t + h) * nl + lane) * 8 + e] = bf16_bits_s(blocks[i].v[8 * h + e]);
+                        ++n;
+                    }
                 }
+                slot0 += nl * sl.T;
             }
-            brp[NBR] = n;
             kept_bytes += (int64_t)n * 34 + (int64_t)(NBR + 1) * 4;
         }
         // dense O2 / O4: 16 rows of this CTA as one tile of A fragments (natural column order)
@@ -549,7 +612,7 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     SparseParams p;
     std::memset(&p, 0, sizeof(p));
     p.H = k.H; p.K = k.K; p.NKT = k.NKT; p.UC = k.UC; p.HR = k.HR; p.NBR = k.NBR;
-    for (int ph = 0; ph < 2; ++ph) { p.off_brp[ph] = k.off_brp[ph]; p.off_col[ph] = k.off_col[ph]; p.off_val[ph] = k.off_val[ph]; }
+    for (int ph = 0; ph < 2; ++ph) { p.off_meta[ph] = k.off_meta[ph]; p.off_col[ph] = k.off_col[ph]; p.off_val[ph] = k.off_val[ph]; }
     p.off_o2 = k.off_o2; p.off_o4 = k.off_o4; p.off_small = k.off_small; p.blob_bytes = k.blob_bytes;
     p.n_steps = a.n_steps; p.step0 = a.step0; p.stream0 = a.stream0; p.seed = a.seed;
     p.n_frames = m->cond_dim ? a.n_frames : 1;

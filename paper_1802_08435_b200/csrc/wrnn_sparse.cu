@@ -30,11 +30,12 @@ constexpr int SCS = 16;          // cluster size
 constexpr int SNW = 20;          // warps per CTA
 
 // Compressed block rows of one phase of one CTA, sliced by warp: the block rows are sorted by their number of kept
-// blocks and dealt out in runs of up to eight to the warps, four lanes per block row; lane 4 g + l of warp w takes
-// blocks l, l + 4, ... of its row g.  Iteration t of a warp reads slot t * nl + lane of its slice (nl = 4 x rows of
-// the warp): the two 16-byte halves of the block's weights from two planes and the block column, so every load of a
-// warp is one contiguous run; rows shorter than the warp's longest are padded with zero blocks.
-struct SliceMeta { int voff, coff, T, nl; int16_t row[8]; };     // offsets in 16-byte / 2-byte units from the phase's arrays
+// blocks and dealt out in runs to the warps; the longest rows get eight lanes each (four rows per warp), the others
+// four (eight rows per warp), as many eight-lane warps as the CTA's lanes allow.  Lane lpr g + l of warp w takes
+// blocks l, l + lpr, ... of its row g.  Iteration t of a warp reads slot t * nl + lane of its slice (nl = lanes in
+// use): the two 16-byte halves of the block's weights from two planes and the block column, so every load of a warp is
+// one contiguous run; rows shorter than the warp's longest are padded with zero blocks.
+struct SliceMeta { int voff, coff, T, nl, lpr, pad[3]; int16_t row[8]; };   // offsets in 16-byte / 2-byte units from the phase's arrays
 
 struct SparsePack {
     int H = 0, K = 0, NKT = 0, UC = 0, HR = 0, NBR = 0;   // NBR: block rows per phase = (HR + 6 UC) / 4
@@ -136,7 +137,10 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     const int sl_nl0 = sm0.nl, sl_nl1 = sm1.nl, sl_T0 = sm0.T, sl_T1 = sm1.T;
     const uint4 *sl_wv0 = bval[0] + sm0.voff + (lane < sl_nl0 ? lane : 0), *sl_wv1 = bval[1] + sm1.voff + (lane < sl_nl1 ? lane : 0);
     const uint16_t *sl_wc0 = bcol[0] + sm0.coff + (lane < sl_nl0 ? lane : 0), *sl_wc1 = bcol[1] + sm1.coff + (lane < sl_nl1 ? lane : 0);
-    const int sl_row0 = lane < sl_nl0 ? (int)sm0.row[lane >> 2] : -1, sl_row1 = lane < sl_nl1 ? (int)sm1.row[lane >> 2] : -1;
+    const bool sl_wide0 = sm0.lpr == 8, sl_wide1 = sm1.lpr == 8;      // eight lanes per block row (else four)
+    // the block row this lane finishes (lanes 0..3 of a row's lanes hold its four sums after the reduction)
+    const int sl_row0 = (lane < sl_nl0 && (!sl_wide0 || (lane & 4) == 0)) ? (int)sm0.row[sl_wide0 ? lane >> 3 : lane >> 2] : -1;
+    const int sl_row1 = (lane < sl_nl1 && (!sl_wide1 || (lane & 4) == 0)) ? (int)sm1.row[sl_wide1 ? lane >> 3 : lane >> 2] : -1;
 
     auto sparse_phase = [&](int ph, const float *x, const float *bias) {
         const int nl = ph ? sl_nl1 : sl_nl0, T = ph ? sl_T1 : sl_T0, l4 = lane & 3;
@@ -160,6 +164,10 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             w0 = w0n; w1 = w1n; c = cn;
         }
         SSTAMP(10);
+        if (ph ? sl_wide1 : sl_wide0) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[j] += __shfl_xor_sync(FULL, acc[j], 4);
+        }
         // four row sums over four lanes: two transposing steps leave row l4 in lane l4
         const bool up2 = (l4 & 2) != 0;
         const float s0 = up2 ? acc[0] : acc[2], k0 = up2 ? acc[2] : acc[0];
@@ -461,10 +469,12 @@ int sparse_prepare(wrnn_model *m)
                 }
             }
         }
-    // slice every (CTA, phase): block rows sorted by length (longest first, stable), dealt to the warps in runs
-    struct Slice { std::vector<int> rows; int T = 0; };
-    const int base_rows = NBR / SNW, extra = NBR % SNW;
-    if (base_rows + (extra ? 1 : 0) > 8) { m->err = "too many block rows per warp"; return WRNN_ERR_UNSUPPORTED; }
+    // slice every (CTA, phase): block rows sorted by length (longest first, stable), dealt to the warps in runs; the
+    // first w8 warps take four rows with eight lanes each, the others up to eight rows with four lanes each
+    struct Slice { std::vector<int> rows; int T = 0, lpr = 4; };
+    int w8 = (8 * SNW - NBR) / 4;
+    if (w8 < 0) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
+    if (w8 > SNW) w8 = SNW;
     std::vector<std::vector<Slice>> slices(SCS * 2);              // [cta * 2 + phase][warp]
     int max_slots = 0;
     for (int cp = 0; cp < SCS * 2; ++cp) {
@@ -475,13 +485,20 @@ int sparse_prepare(wrnn_model *m)
         slices[cp].assign(SNW, {});
         int next = 0, slots = 0;
         for (int w = 0; w < SNW; ++w) {
-            const int nr = base_rows + (w < extra ? 1 : 0);
             Slice &sl = slices[cp][w];
+            sl.lpr = w < w8 ? 8 : 4;
+            const int cap = 32 / sl.lpr;
+            // rows still to place, spread evenly over the remaining four-lane warps
+            int nr = cap;
+            if (w >= w8) { const int left = NBR - next, warps_left = SNW - w; nr = (left + warps_left - 1) / warps_left; }
+            if (nr > NBR - next) nr = NBR - next;
+            if (nr > cap) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
             size_t longest = 0;
             for (int i = 0; i < nr; ++i) { sl.rows.push_back(order[next + i]); longest = std::max(longest, R[order[next + i]].size()); }
             next += nr;
-            sl.T = (int)((longest + 3) / 4);
-            slots += 4 * nr * sl.T;
+            sl.T = (int)((longest + sl.lpr - 1) / sl.lpr);
+            if (sl.T < 1) sl.T = 1;                                  // the loop's first loads are unconditional
+            slots += sl.lpr * nr * sl.T;
         }
         max_slots = std::max(max_slots, slots);
     }
@@ -527,13 +544,13 @@ int sparse_prepare(wrnn_model *m)
             int slot0 = 0, n = 0;
             for (int w = 0; w < SNW; ++w) {
                 const Slice &sl = slices[cta * 2 + ph][w];
-                const int nl = 4 * (int)sl.rows.size();
-                meta[w].voff = 2 * slot0; meta[w].coff = slot0; meta[w].T = sl.T; meta[w].nl = nl;
+                const int nl = sl.lpr * (int)sl.rows.size();
+                meta[w].voff = 2 * slot0; meta[w].coff = slot0; meta[w].T = sl.T; meta[w].nl = nl; meta[w].lpr = sl.lpr;
                 for (int g = 0; g < 8; ++g) meta[w].row[g] = g < (int)sl.rows.size() ? (int16_t)sl.rows[g] : (int16_t)-1;
                 for (int g = 0; g < (int)sl.rows.size(); ++g) {
                     const auto &blocks = R[sl.rows[g]];
                     for (int i = 0; i < (int)blocks.size(); ++i) {
-                        const int t = i / 4, lane = 4 * g + i % 4;
+                        const int t = i / sl.lpr, lane = sl.lpr * g + i % sl.lpr;
                         col[slot0 + t * nl + lane] = blocks[i].col;
                         for (int h = 0; h < 2; ++h)                  // plane h holds rows 2 h, 2 h + 1 of the block
                             for (int e = 0; e < 8; ++e)

@@ -77,12 +77,17 @@ typedef struct {
     const float *O2, *b2;       /* [256][H/2], [256]   coarse logits                                  */
     const float *O3, *b3;       /* fine hidden layer, same shapes                                     */
     const float *O4, *b4;       /* fine logits                                                        */
-    const uint8_t *mask_R;      /* [3H/4][H/4] 1 = 4x4 block kept (Section 3.2), NULL = dense         */
-    const uint8_t *mask_O1;     /* [H/8][H/8] or NULL                                                 */
-    const uint8_t *mask_O3;     /* [H/8][H/8] or NULL                                                 */
+    const uint8_t *mask_R;      /* [3H/br][H/bc] 1 = block kept (Section 3.2), NULL = dense; br x bc  */
+                                /* is the block shape given below (4 x 4 unless stated otherwise)     */
+    const uint8_t *mask_O1;     /* [H/2/br][H/2/bc] or NULL                                           */
+    const uint8_t *mask_O3;     /* [H/2/br][H/2/bc] or NULL                                           */
     int32_t dtype;              /* wrnn_dtype: storage type of R, I, W_cond, O1..O4 (bf16 = round to  */
                                 /* nearest even at create); biases, state and all arithmetic are fp32 */
     int32_t kernel;             /* wrnn_kernel                                                        */
+    int32_t mask_block_rows;    /* rows and columns of one block of the three masks (Section 3.2:     */
+    int32_t mask_block_cols;    /* 4 x 4, or m x 1 = 16 rows of one column, or 1 x 1 = unstructured); */
+                                /* 0, 0 means 4 x 4.  Both must divide H/2.  Every shape runs on the  */
+                                /* generic kernel; 4 x 4 and 16 x 1 also on the single-cluster kernel */
 } wrnn_params;
 
 /*

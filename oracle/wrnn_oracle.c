@@ -97,14 +97,21 @@ void orc_bf16_round(const float *in, float *out, int64_t n)
     for (int64_t i = 0; i < n; ++i) out[i] = orc_bf16_round_scalar(in[i]);
 }
 
-/* Zero every 4x4 block of W[rows][cols] whose mask entry is 0
- * (mask is [rows/4][cols/4], Section 3.2: blocks pruned or kept together). */
-void orc_apply_block_mask(float *W, int rows, int cols, const uint8_t *mask)
+/* Zero every br x bc block of W[rows][cols] whose mask entry is 0 (mask is [rows/br][cols/bc]; Section 3.2:
+ * non-overlapping blocks pruned or kept together, 4 x 4 or m x 1 -- m rows, one column -- with m = 16;
+ * 1 x 1 is the unstructured case). */
+void orc_apply_block_mask_shape(float *W, int rows, int cols, const uint8_t *mask, int br, int bc)
 {
-    int bc = cols / 4;
+    int nbc = cols / bc;
     for (int r = 0; r < rows; ++r)
         for (int c = 0; c < cols; ++c)
-            if (!mask[(r / 4) * bc + (c / 4)]) W[(int64_t)r * cols + c] = 0.0f;
+            if (!mask[(r / br) * nbc + (c / bc)]) W[(int64_t)r * cols + c] = 0.0f;
+}
+
+/* The 4 x 4 case. */
+void orc_apply_block_mask(float *W, int rows, int cols, const uint8_t *mask)
+{
+    orc_apply_block_mask_shape(W, rows, cols, mask, 4, 4);
 }
 
 /* ------------------------------------------------------------------ */

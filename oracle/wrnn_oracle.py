@@ -49,6 +49,7 @@ def lib():
         L.orc_philox4x32_10.argtypes = [C.c_void_p] * 3
         L.orc_bf16_round.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.orc_apply_block_mask.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p]
+        L.orc_apply_block_mask_shape.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_int]
         L.orc_scale8.restype = C.c_double
         L.orc_scale8.argtypes = [C.c_int]
         L.orc_to_int16.restype = C.c_int16
@@ -92,11 +93,13 @@ def bf16_round(x: np.ndarray) -> np.ndarray:
     return out
 
 
-def apply_block_mask(W: np.ndarray, mask: np.ndarray) -> np.ndarray:
+def apply_block_mask(W: np.ndarray, mask: np.ndarray, block=(4, 4)) -> np.ndarray:
+    """Zero the blocks of W (block = (rows, columns) of one block) whose mask entry is 0."""
     W = np.array(W, dtype=np.float32, order="C", copy=True)
     m = np.ascontiguousarray(mask, dtype=np.uint8)
-    assert m.shape == (W.shape[0] // 4, W.shape[1] // 4)
-    lib().orc_apply_block_mask(_ptr(W), W.shape[0], W.shape[1], _ptr(m))
+    br, bc = int(block[0]), int(block[1])
+    assert W.shape[0] % br == 0 and W.shape[1] % bc == 0 and m.shape == (W.shape[0] // br, W.shape[1] // bc)
+    lib().orc_apply_block_mask_shape(_ptr(W), W.shape[0], W.shape[1], _ptr(m), br, bc)
     return W
 
 
@@ -166,12 +169,13 @@ class OracleModel:
     """The stored model: masks applied, then weights rounded to the storage type.
 
     `weights` is a dict of fp32 arrays (R, I, b_gate, W_cond, O1, b1, ... b4);
-    `masks` an optional dict with 4x4 block masks for "R" [3H/4][H/4],
-    "O1", "O3" [H/8][H/8]; dtype "f32" or "bf16" (weights R, I, W_cond,
+    `masks` an optional dict with block masks for "R" [3H/br][H/bc], "O1",
+    "O3" [H/2/br][H/2/bc], `block` = (br, bc) the shape of one block (4 x 4,
+    16 x 1 or 1 x 1, Section 3.2); dtype "f32" or "bf16" (weights R, I, W_cond,
     O1..O4 rounded to bf16; biases stay fp32).
     """
 
-    def __init__(self, weights: dict, dtype: str = "f32", masks: Optional[dict] = None):
+    def __init__(self, weights: dict, dtype: str = "f32", masks: Optional[dict] = None, block=(4, 4)):
         assert dtype in ("f32", "bf16")
         self.H = int(weights["R"].shape[1])
         assert weights["R"].shape == (3 * self.H, self.H)
@@ -185,7 +189,7 @@ class OracleModel:
                 continue
             a = np.array(a, dtype=np.float32, order="C", copy=True)
             if masks and masks.get(k) is not None:
-                a = apply_block_mask(a, masks[k])
+                a = apply_block_mask(a, masks[k], block)
             if dtype == "bf16":
                 a = bf16_round(a)
             w[k] = a

@@ -41,7 +41,7 @@ class wrnn_params(C.Structure):
         [("H", C.c_int32), ("cond_dim", C.c_int32)]
         + [(n, C.c_void_p) for n in ("R", "I", "b_gate", "W_cond", "O1", "b1", "O2", "b2", "O3", "b3", "O4", "b4",
                                      "mask_R", "mask_O1", "mask_O3")]
-        + [("dtype", C.c_int32), ("kernel", C.c_int32)]
+        + [("dtype", C.c_int32), ("kernel", C.c_int32), ("mask_block_rows", C.c_int32), ("mask_block_cols", C.c_int32)]
     )
 
 
@@ -122,9 +122,10 @@ def wrnn_last_error(model=None) -> str:
 
 
 def wrnn_create(weights: Dict[str, np.ndarray], dtype: str = "f32", masks: Optional[Dict[str, np.ndarray]] = None,
-                max_batch: int = 1, kernel: int = WRNN_KERNEL_AUTO):
+                max_batch: int = 1, kernel: int = WRNN_KERNEL_AUTO, block=(4, 4)):
     """weights: fp32 numpy arrays R [3H][H], I [3H][3], W_cond [3H][D] or None, O1..O4, b_gate, b1..b4 (or None);
-    masks: optional 4x4 block masks {"R": [3H/4][H/4], "O1": [H/8][H/8], "O3": ...}.  Returns an opaque handle."""
+    masks: optional block masks {"R": [3H/br][H/bc], "O1": [H/2/br][H/2/bc], "O3": ...} with block = (br, bc).
+    Returns an opaque handle."""
     keep = {}
 
     def f32(k):
@@ -152,6 +153,7 @@ def wrnn_create(weights: Dict[str, np.ndarray], dtype: str = "f32", masks: Optio
     p.mask_R, p.mask_O1, p.mask_O3 = _np_ptr(u8("R")), _np_ptr(u8("O1")), _np_ptr(u8("O3"))
     p.dtype = {"f32": WRNN_F32, "bf16": WRNN_BF16}[dtype]
     p.kernel = kernel
+    p.mask_block_rows, p.mask_block_cols = int(block[0]), int(block[1])
     out = C.c_void_p()
     _check(lib().wrnn_create(C.byref(p), max_batch, C.byref(out)))
     return out

@@ -37,19 +37,27 @@ static inline uint16_t bf16_bits(float rounded)
 
 // Dense row-major W[rows][cols] (+ optional 4x4 block mask) -> host block rows with the
 // values already rounded to the storage type.
-static void build_bsr(const float *W, int rows, int cols, const uint8_t *mask, bool bf16, BsrHost *out)
+// W[rows][cols] with an optional mask of mr x mc blocks ([rows/mr][cols/mc], 1 = kept) -> compressed block rows of
+// 4x4 blocks: a 4x4 block is stored when any of its 16 weights is kept; weights that are not kept are stored as zero.
+static void build_bsr(const float *W, int rows, int cols, const uint8_t *mask, int mr, int mc, bool bf16, BsrHost *out)
 {
-    const int R4 = rows / 4, C4 = cols / 4;
+    const int R4 = rows / 4, C4 = cols / 4, MC = mask ? cols / mc : 0;
     out->rows4 = R4; out->cols4 = C4;
     out->row_ptr.assign(R4 + 1, 0);
     out->col.clear(); out->vals.clear();
     for (int br = 0; br < R4; ++br) {
         for (int bc = 0; bc < C4; ++bc) {
-            if (mask && !mask[(size_t)br * C4 + bc]) continue;
+            bool kept[16], any = false;
+            for (int r = 0; r < 4; ++r)
+                for (int c = 0; c < 4; ++c) {
+                    kept[4 * r + c] = !mask || mask[(size_t)((4 * br + r) / mr) * MC + (4 * bc + c) / mc] != 0;
+                    any = any || kept[4 * r + c];
+                }
+            if (!any) continue;
             out->col.push_back((uint16_t)bc);
             for (int r = 0; r < 4; ++r)
                 for (int c = 0; c < 4; ++c) {
-                    const float v = W[(size_t)(4 * br + r) * cols + 4 * bc + c];
+                    const float v = kept[4 * r + c] ? W[(size_t)(4 * br + r) * cols + 4 * bc + c] : 0.f;
                     out->vals.push_back(bf16 ? round_bf16(v) : v);
                 }
         }
@@ -220,6 +228,9 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
     if ((p->cond_dim > 0) != (p->W_cond != nullptr)) return fail(nullptr, WRNN_ERR_INVALID_ARG, "W_cond must be given iff cond_dim > 0");
     if (p->dtype != WRNN_F32 && p->dtype != WRNN_BF16) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown dtype");
     if (p->kernel < WRNN_KERNEL_AUTO || p->kernel > WRNN_KERNEL_BCLUSTER) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown kernel family");
+    const int mbr = p->mask_block_rows ? p->mask_block_rows : 4, mbc = p->mask_block_cols ? p->mask_block_cols : 4;
+    if ((p->mask_block_rows == 0) != (p->mask_block_cols == 0) || mbr < 1 || mbc < 1 || (H / 2) % mbr != 0 || (H / 2) % mbc != 0)
+        return fail(nullptr, WRNN_ERR_INVALID_ARG, "mask block shape must divide H/2 (0, 0 = 4 x 4)");
 
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return fail(nullptr, WRNN_ERR_CUDA, "no usable CUDA device"); }
@@ -232,14 +243,15 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
     m->H = H; m->cond_dim = p->cond_dim; m->dtype = p->dtype; m->kernel = p->kernel; m->max_batch = max_batch;
     m->device = dev; m->n_sms = prop.multiProcessorCount;
     m->sparse = p->mask_R || p->mask_O1 || p->mask_O3;
+    m->mask_br = mbr; m->mask_bc = mbc;
     const bool bf = p->dtype == WRNN_BF16;
     const int Hh = H / 2, G = 3 * H;
 
-    build_bsr(p->R, G, H, p->mask_R, bf, &m->hR);
-    build_bsr(p->O1, Hh, Hh, p->mask_O1, bf, &m->hO1);
-    build_bsr(p->O2, 256, Hh, nullptr, bf, &m->hO2);
-    build_bsr(p->O3, Hh, Hh, p->mask_O3, bf, &m->hO3);
-    build_bsr(p->O4, 256, Hh, nullptr, bf, &m->hO4);
+    build_bsr(p->R, G, H, p->mask_R, mbr, mbc, bf, &m->hR);
+    build_bsr(p->O1, Hh, Hh, p->mask_O1, mbr, mbc, bf, &m->hO1);
+    build_bsr(p->O2, 256, Hh, nullptr, 4, 4, bf, &m->hO2);
+    build_bsr(p->O3, Hh, Hh, p->mask_O3, mbr, mbc, bf, &m->hO3);
+    build_bsr(p->O4, 256, Hh, nullptr, 4, 4, bf, &m->hO4);
     m->hI.resize((size_t)G * 3);
     for (int row = 0; row < G; ++row)
         for (int c = 0; c < 3; ++c) {

@@ -60,6 +60,7 @@ struct wrnn_model {
     int H = 0, cond_dim = 0, dtype = 0, kernel = 0, max_batch = 0;
     int device = 0, n_sms = 0;
     bool sparse = false;
+    int mask_br = 4, mask_bc = 4;   // shape of one block of the sparsity masks (Section 3.2)
 
     // generic format
     wrnn::BsrDev R, O1, O2, O3, O4;

@@ -439,6 +439,7 @@ int sparse_prepare(wrnn_model *m)
     const int H = m->H, Hh = H / 2;
     if (m->dtype != WRNN_BF16) { m->err = "sparse cluster kernel stores bf16 weights"; return WRNN_ERR_UNSUPPORTED; }
     if (!m->sparse) { m->err = "model has no block masks"; return WRNN_ERR_UNSUPPORTED; }
+    if (m->mask_br != 4 || m->mask_bc != 4) { m->err = "single-cluster kernel takes 4 x 4 blocks"; return WRNN_ERR_UNSUPPORTED; }
     if (Hh != 1024) { m->err = "only H/2 = 1024 is instantiated (8 warps x 8 k-tiles for the logits tile)"; return WRNN_ERR_UNSUPPORTED; }
     SparsePack k;
     k.H = H; k.K = Hh; k.NKT = Hh / 16; k.UC = Hh / SCS; k.HR = Hh / SCS;

@@ -54,18 +54,20 @@ def make_weights(H: int, cond_dim: int = COND_DIM, seed_w: int = SEED_WEIGHTS,
     return w
 
 
-def make_block_masks(H: int, sparsity: float = 0.96, seed: int = SEED_MASK) -> Dict[str, np.ndarray]:
-    """Uniform random 4x4 block masks with exactly round((1-sparsity) * n_blocks) kept
-    blocks per matrix; R_u, R_r, R_e are masked separately (stacked as one [3H/4][H/4])."""
+def make_block_masks(H: int, sparsity: float = 0.96, seed: int = SEED_MASK, block=(4, 4)) -> Dict[str, np.ndarray]:
+    """Uniform random block masks (block = (rows, columns) of one block: 4 x 4, 16 x 1 or 1 x 1) with exactly
+    round((1-sparsity) * n_blocks) kept blocks per matrix; R_u, R_r, R_e are masked separately (stacked as one
+    [3H/br][H/bc])."""
     rng = np.random.default_rng(seed)
     Hh = H // 2
+    br, bc = block
 
     def one(rows, cols):
-        nb = (rows // 4) * (cols // 4)
+        nb = (rows // br) * (cols // bc)
         keep = int(round((1.0 - sparsity) * nb))
         m = np.zeros(nb, np.uint8)
         m[rng.permutation(nb)[:keep]] = 1
-        return m.reshape(rows // 4, cols // 4)
+        return m.reshape(rows // br, cols // bc)
 
     mR = np.concatenate([one(H, H) for _ in range(3)], axis=0)
     return {"R": mR, "O1": one(Hh, Hh), "O3": one(Hh, Hh)}
@@ -99,15 +101,19 @@ class Workload:
     row_offset_mul: int = 0
     sparsity: Optional[float] = None
     subscale_B: int = 0       # >0: fold/unfold of one n_steps*B sequence
+    block: tuple = (4, 4)     # shape of one block of the sparsity masks (rows, columns)
 
 
-# The five named workloads (index = position in the benchmark's config list).
+# The five named workloads (index = position in the benchmark's config list), then two extra sparse ones.
 WORKLOADS = [
     Workload("dense896_f32_b1_1200", 896, "f32", 1, 1200, 10),
     Workload("dense896_bf16_b1_24000", 896, "bf16", 1, 24000, 200),
     Workload("sparse2048_bf16_b1_24000", 2048, "bf16", 1, 24000, 200, sparsity=0.96),
     Workload("subscale16_896_bf16_1500", 896, "bf16", 16, 1500, 200, row_stride=16, row_offset_mul=1, subscale_B=16),
     Workload("batched256_896_bf16_24000", 896, "bf16", 256, 24000, 200),
+    # beyond the five benchmark configurations: the other block shapes of Section 3.2 (same model, same sparsity)
+    Workload("sparse2048_16x1_bf16_b1_24000", 2048, "bf16", 1, 24000, 200, sparsity=0.96, block=(16, 1)),
+    Workload("sparse2048_1x1_bf16_b1_2400", 2048, "bf16", 1, 2400, 20, sparsity=0.96, block=(1, 1)),
 ]
 
 
@@ -116,7 +122,7 @@ def build_workload(wl: Workload, n_steps: Optional[int] = None, batch: Optional[
     w = make_weights(wl.H)
     masks = None
     if wl.sparsity is not None:
-        masks = make_block_masks(wl.H, wl.sparsity)
+        masks = make_block_masks(wl.H, wl.sparsity, block=wl.block)
         w = rescale_kept(w, masks, wl.sparsity)
     b = wl.batch if batch is None else batch
     cond = make_cond(b, wl.n_frames)

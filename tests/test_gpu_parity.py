@@ -127,6 +127,27 @@ def test_multirow_resume_unconditioned_and_wide_models(env, kernel):
             B.wrnn_destroy(m)
 
 
+@pytest.mark.parametrize("block", [(16, 1), (1, 1), (4, 4)])
+def test_tiny_block_shapes(env, block):
+    """Section 3.2's block shapes (4 x 4, 16 x 1, unstructured) on the generic kernel: every shape is stored as 4 x 4
+    block rows that hold the kept weights and zeros."""
+    torch, B = env
+    H = 64
+    w = _tiny(H)
+    masks = synth.make_block_masks(H, sparsity=0.75, seed=3, block=block)
+    w = synth.rescale_kept(w, masks, 0.75)
+    om = orc.OracleModel(w, "bf16", masks, block)
+    m = B.wrnn_create(w, "bf16", masks, kernel=B.WRNN_KERNEL_GENERIC, block=block)
+    try:
+        cond = synth.make_cond(1, 6, 4)
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, 50, 1, SEED, hop=10)
+        assert r["idx_bad"] == 0 and max(r["gates_err"], r["h_err"], r["logits_err"]) < pu.TOL["bf16"], {k: v for k, v in r.items() if k != "oracle"}
+    finally:
+        B.wrnn_destroy(m)
+    with pytest.raises(B.WrnnError):
+        B.wrnn_create(w, "bf16", masks, block=(3, 1))              # does not divide H/2
+
+
 def test_unconditioned_model_and_null_biases(env):
     torch, B = env
     w = _tiny(16, cond_dim=0)

@@ -309,20 +309,26 @@ def test_teacher_forcing_with_own_stream_reproduces_free_run():
     assert np.array_equal(u >> 8, free.c_out) and np.array_equal(u & 255, free.f_out)
 
 
-def test_sparse_model_is_dense_model_with_zero_blocks():
+@pytest.mark.parametrize("block", [(4, 4), (16, 1), (1, 1)])
+def test_sparse_model_is_dense_model_with_zero_blocks(block):
+    """Section 3.2's block shapes: 4 x 4, m x 1 with m = 16 (16 rows of one column), and unstructured."""
     H = 32
+    br, bc = block
     w = tiny_weights(H, scale=3.0)
-    masks = synth.make_block_masks(H, sparsity=0.5, seed=1)
-    assert masks["R"].shape == (3 * H // 4, H // 4)
+    masks = synth.make_block_masks(H, sparsity=0.5, seed=1, block=block)
+    assert masks["R"].shape == (3 * H // br, H // bc) and masks["O1"].shape == (H // 2 // br, H // 2 // bc)
     for g in range(3):
-        assert masks["R"][g * H // 4:(g + 1) * H // 4].sum() == round(0.5 * (H // 4) ** 2)   # per-gate masks
+        assert masks["R"][g * H // br:(g + 1) * H // br].sum() == round(0.5 * (H // br) * (H // bc))   # per-gate masks
     wz = dict(w)
     for k, m in masks.items():
-        wz[k] = w[k] * np.kron(m, np.ones((4, 4), np.float32))
+        wz[k] = w[k] * np.kron(m, np.ones((br, bc), np.float32))
+        assert np.array_equal(orc.apply_block_mask(w[k], m, block), wz[k])
     cond = synth.make_cond(1, 2, 4)
-    a = orc.OracleModel(w, "bf16", masks).run(cond, 25, 1, seed=4, hop=20, dump=True)
+    a = orc.OracleModel(w, "bf16", masks, block).run(cond, 25, 1, seed=4, hop=20, dump=True)
     b = orc.OracleModel(wz, "bf16").run(cond, 25, 1, seed=4, hop=20, dump=True)
     assert np.array_equal(a.out, b.out) and np.array_equal(a.logits, b.logits)
+    d = orc.OracleModel(w, "bf16").run(cond, 25, 1, seed=4, hop=20, dump=True)
+    assert not np.array_equal(a.logits, d.logits)                   # the mask does something
 
 
 def test_frame_index_out_of_range_is_an_error():

@@ -100,7 +100,7 @@ def run_reference(args, wl):
         return
     from oracle import wrnn_oracle as orc
     w, masks, cond = synth.build_workload(wl)
-    om = orc.OracleModel(w, wl.dtype, masks)
+    om = orc.OracleModel(w, wl.dtype, masks, wl.block)
     cores = os.cpu_count() or 1
     threads = 1 if wl.batch == 1 else min(cores, wl.batch)
     # about 2-3 s of CPU work per step
@@ -132,7 +132,7 @@ def run_reference(args, wl):
 def cpu_baseline(wl, budget_s=12.0):
     from oracle import wrnn_oracle as orc
     w, masks, cond = synth.build_workload(wl)
-    om = orc.OracleModel(w, wl.dtype, masks)
+    om = orc.OracleModel(w, wl.dtype, masks, wl.block)
     cores = os.cpu_count() or 1
     threads = 1 if wl.batch == 1 else min(cores, wl.batch)
     per_row_step_ms = 2.3 * (wl.H / 896.0) ** 2
@@ -180,7 +180,7 @@ def main():
     n_steps = wl.n_steps if args.n_steps is None else args.n_steps
     w, masks, cond_np = synth.build_workload(wl)
     kern = {"auto": B.WRNN_KERNEL_AUTO, "generic": B.WRNN_KERNEL_GENERIC, "resident": B.WRNN_KERNEL_RESIDENT, "batched": B.WRNN_KERNEL_BATCHED, "bcluster": B.WRNN_KERNEL_BCLUSTER}[args.kernel]
-    model = B.wrnn_create(w, wl.dtype, masks, max_batch=wl.batch, kernel=kern)
+    model = B.wrnn_create(w, wl.dtype, masks, max_batch=wl.batch, kernel=kern, block=wl.block)
     info = B.wrnn_launch_info(model, wl.batch)
     cond = torch.from_numpy(cond_np).to(dev)
     out = torch.zeros((wl.batch, n_steps), dtype=torch.int16, device=dev)
@@ -300,7 +300,7 @@ def main():
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "H": wl.H, "batch": wl.batch, "n_steps": n_steps, "weights": wl.dtype,
-                       "sparsity": wl.sparsity, "l2": "flushed between timed iterations (256 MiB fill)",
+                       "sparsity": wl.sparsity, "block": ("%dx%d" % tuple(wl.block)) if wl.sparsity is not None else None, "l2": "flushed between timed iterations (256 MiB fill)",
                        "kernel": {1: "generic", 2: "resident", 3: "batched", 4: "sparse-cluster", 5: "batched-cluster"}[info["kernel"]], "n_ctas": info["n_ctas"],
                        "threads_per_cta": info["n_threads"], "smem_bytes_per_cta": info["smem_bytes"],
                        "multi_gpu": "replicas only"},

@@ -38,7 +38,8 @@ constexpr int SNW = 20;          // warps per CTA
 struct SliceMeta { int voff, coff, T, nl, lpr, pad[3]; int16_t row[8]; };   // offsets in 16-byte / 2-byte units from the phase's arrays
 
 struct SparsePack {
-    int H = 0, K = 0, NKT = 0, UC = 0, HR = 0, NBR = 0;   // NBR: block rows per phase = (HR + 6 UC) / 4
+    int H = 0, K = 0, NKT = 0, UC = 0, HR = 0, NBR = 0;   // NBR: block rows per phase = (HR + 6 UC) / rows of a block
+    int tall = 0;                     // 16 x 1 blocks (else 4 x 4)
     int max_slots = 0;                // block slots per phase per CTA (kept blocks + padding of the sliced layout, maximum)
     size_t blob_bytes = 0;            // per CTA
     size_t off_meta[2], off_col[2], off_val[2], off_o2 = 0, off_o4 = 0, off_small = 0;
@@ -48,7 +49,7 @@ struct SparsePack {
 };
 
 struct SparseParams {
-    int H, K, NKT, UC, HR, NBR;
+    int H, K, NKT, UC, HR, NBR, tall;        // tall: blocks are 16 x 1 (16 rows of one column) instead of 4 x 4
     unsigned long long off_meta[2], off_col[2], off_val[2], off_o2, off_o4, off_small, blob_bytes;
     long long n_steps, step0;
     unsigned stream0;
@@ -137,15 +138,63 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     const int sl_nl0 = sm0.nl, sl_nl1 = sm1.nl, sl_T0 = sm0.T, sl_T1 = sm1.T;
     const uint4 *sl_wv0 = bval[0] + sm0.voff + (lane < sl_nl0 ? lane : 0), *sl_wv1 = bval[1] + sm1.voff + (lane < sl_nl1 ? lane : 0);
     const uint16_t *sl_wc0 = bcol[0] + sm0.coff + (lane < sl_nl0 ? lane : 0), *sl_wc1 = bcol[1] + sm1.coff + (lane < sl_nl1 ? lane : 0);
-    const bool sl_wide0 = sm0.lpr == 8, sl_wide1 = sm1.lpr == 8;      // eight lanes per block row (else four)
-    // the block row this lane finishes (lanes 0..3 of a row's lanes hold its four sums after the reduction)
-    const int sl_row0 = (lane < sl_nl0 && (!sl_wide0 || (lane & 4) == 0)) ? (int)sm0.row[sl_wide0 ? lane >> 3 : lane >> 2] : -1;
-    const int sl_row1 = (lane < sl_nl1 && (!sl_wide1 || (lane & 4) == 0)) ? (int)sm1.row[sl_wide1 ? lane >> 3 : lane >> 2] : -1;
+    const bool tall = p.tall != 0;
+    const int lpr_n = tall ? 16 : 4;                                    // lanes per block row, narrow slices
+    const bool sl_wide0 = sm0.lpr == 2 * lpr_n, sl_wide1 = sm1.lpr == 2 * lpr_n;   // twice as many lanes per block row
+    // the block row this lane finishes (the first lpr_n lanes of a row's lanes hold its sums after the reduction)
+    const int sl_sh = tall ? 4 : 2;
+    const int sl_row0 = (lane < sl_nl0 && (!sl_wide0 || (lane & lpr_n) == 0)) ? (int)sm0.row[lane >> (sl_sh + (sl_wide0 ? 1 : 0))] : -1;
+    const int sl_row1 = (lane < sl_nl1 && (!sl_wide1 || (lane & lpr_n) == 0)) ? (int)sm1.row[lane >> (sl_sh + (sl_wide1 ? 1 : 0))] : -1;
 
     auto sparse_phase = [&](int ph, const float *x, const float *bias) {
         const int nl = ph ? sl_nl1 : sl_nl0, T = ph ? sl_T1 : sl_T0, l4 = lane & 3;
         const uint4 *wv = ph ? sl_wv1 : sl_wv0;
         const uint16_t *wc = ph ? sl_wc1 : sl_wc0;
+        if (tall) {
+            // 16 x 1 blocks (Section 3.2): one activation per block, sixteen row sums per lane
+            float a16[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) a16[j] = 0.f;
+            uint4 w0 = wv[0], w1 = wv[nl];
+            int c = wc[0];
+            for (int t = 0; t < T; ++t) {
+                const float xs = x[c];
+                const int tn = t + 1 < T ? t + 1 : t;
+                const uint4 w0n = wv[(2 * tn) * nl], w1n = wv[(2 * tn + 1) * nl];
+                const int cn = wc[tn * nl];
+                a16[0] = fmaf(bf16lo(w0.x), xs, a16[0]);   a16[1] = fmaf(bf16hi(w0.x), xs, a16[1]);
+                a16[2] = fmaf(bf16lo(w0.y), xs, a16[2]);   a16[3] = fmaf(bf16hi(w0.y), xs, a16[3]);
+                a16[4] = fmaf(bf16lo(w0.z), xs, a16[4]);   a16[5] = fmaf(bf16hi(w0.z), xs, a16[5]);
+                a16[6] = fmaf(bf16lo(w0.w), xs, a16[6]);   a16[7] = fmaf(bf16hi(w0.w), xs, a16[7]);
+                a16[8] = fmaf(bf16lo(w1.x), xs, a16[8]);   a16[9] = fmaf(bf16hi(w1.x), xs, a16[9]);
+                a16[10] = fmaf(bf16lo(w1.y), xs, a16[10]); a16[11] = fmaf(bf16hi(w1.y), xs, a16[11]);
+                a16[12] = fmaf(bf16lo(w1.z), xs, a16[12]); a16[13] = fmaf(bf16hi(w1.z), xs, a16[13]);
+                a16[14] = fmaf(bf16lo(w1.w), xs, a16[14]); a16[15] = fmaf(bf16hi(w1.w), xs, a16[15]);
+                w0 = w0n; w1 = w1n; c = cn;
+            }
+            if (ph ? sl_wide1 : sl_wide0) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) a16[j] += __shfl_xor_sync(FULL, a16[j], 16);
+            }
+            // sixteen row sums over sixteen lanes: four transposing steps leave row l in lane l of the row's lanes
+            float a8[8], a4[4], a2[2];
+            const bool u8 = (lane & 8) != 0, u4 = (lane & 4) != 0, u2 = (lane & 2) != 0, u1 = (lane & 1) != 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) a8[j] = (u8 ? a16[8 + j] : a16[j]) + __shfl_xor_sync(FULL, u8 ? a16[j] : a16[8 + j], 8);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) a4[j] = (u4 ? a8[4 + j] : a8[j]) + __shfl_xor_sync(FULL, u4 ? a8[j] : a8[4 + j], 4);
+#pragma unroll
+            for (int j = 0; j < 2; ++j) a2[j] = (u2 ? a4[2 + j] : a4[j]) + __shfl_xor_sync(FULL, u2 ? a4[j] : a4[2 + j], 2);
+            const float v = (u1 ? a2[1] : a2[0]) + __shfl_xor_sync(FULL, u1 ? a2[0] : a2[1], 1);
+            const int lbr = ph ? sl_row1 : sl_row0;
+            if (lbr >= 0) {
+                const int row = 16 * lbr + (lane & 15);
+                if (row < HR) qvec[row] = fmaxf(v + bias[row], 0.f);
+                else if (ph) a_full[row - HR] = a_part[row - HR] + v;
+                else a_part[row - HR] = v;
+            }
+            return;
+        }
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         SSTAMP(9);
         // software pipeline: the weights and the column of the next block are in flight while this block's four
@@ -439,15 +488,20 @@ int sparse_prepare(wrnn_model *m)
     const int H = m->H, Hh = H / 2;
     if (m->dtype != WRNN_BF16) { m->err = "sparse cluster kernel stores bf16 weights"; return WRNN_ERR_UNSUPPORTED; }
     if (!m->sparse) { m->err = "model has no block masks"; return WRNN_ERR_UNSUPPORTED; }
-    if (m->mask_br != 4 || m->mask_bc != 4) { m->err = "single-cluster kernel takes 4 x 4 blocks"; return WRNN_ERR_UNSUPPORTED; }
+    const bool tall = m->mask_br == 16 && m->mask_bc == 1;
+    if (!tall && (m->mask_br != 4 || m->mask_bc != 4)) { m->err = "single-cluster kernel takes 4 x 4 or 16 x 1 blocks"; return WRNN_ERR_UNSUPPORTED; }
     if (Hh != 1024) { m->err = "only H/2 = 1024 is instantiated (8 warps x 8 k-tiles for the logits tile)"; return WRNN_ERR_UNSUPPORTED; }
     SparsePack k;
     k.H = H; k.K = Hh; k.NKT = Hh / 16; k.UC = Hh / SCS; k.HR = Hh / SCS;
-    k.NBR = (k.HR + 6 * k.UC) / 4;
-    const int UC = k.UC, HR = k.HR, NBR = k.NBR, Kb = Hh / 4;      // Kb: block columns per half
+    const int BRH = tall ? 16 : 4;                                 // rows of one block
+    k.tall = tall ? 1 : 0;
+    k.NBR = (k.HR + 6 * k.UC) / BRH;
+    const int UC = k.UC, HR = k.HR, NBR = k.NBR, Kb = Hh / 4;      // Kb: 4-wide block columns per half
+    if (HR % BRH != 0 || UC % BRH != 0) { m->err = "block height does not divide the rows of one CTA"; return WRNN_ERR_UNSUPPORTED; }
 
-    // kept blocks of each phase of each CTA
-    struct Blk { uint16_t col; const float *v; };
+    // kept blocks of each phase of each CTA.  A block is 16 weights: a 4 x 4 block row-major, or the 16 rows of one column;
+    // col is the block column (4 x 4) or the column (16 x 1) inside the phase's input half.
+    struct Blk { uint16_t col; float v[16]; };
     std::vector<std::vector<std::vector<Blk>>> rows(SCS * 2);      // [cta * 2 + phase][local block row] -> blocks
     const BsrHost *Oa[2] = {&m->hO1, &m->hO3};
     for (int cta = 0; cta < SCS; ++cta)
@@ -455,27 +509,57 @@ int sparse_prepare(wrnn_model *m)
             auto &R = rows[cta * 2 + ph];
             R.assign(NBR, {});
             for (int lbr = 0; lbr < NBR; ++lbr) {
-                if (lbr < HR / 4) {
-                    const BsrHost &M = *Oa[ph];
-                    const int br = cta * (HR / 4) + lbr;
-                    for (int i = M.row_ptr[br]; i < M.row_ptr[br + 1]; ++i) R[lbr].push_back({M.col[i], &M.vals[(size_t)i * 16]});
+                // the 4-row block rows of the source matrix under this block row, and the range of its 4-wide block columns
+                const BsrHost *M;
+                int br0, bc_lo, bc_hi;
+                if (lbr < HR / BRH) {
+                    M = Oa[ph];
+                    br0 = (cta * HR + lbr * BRH) / 4; bc_lo = 0; bc_hi = Kb;
                 } else {
-                    const int q = lbr - HR / 4;                    // (half * 3 + gate) * (UC / 4) + u4
-                    const int half = q / (3 * (UC / 4)), gate = (q / (UC / 4)) % 3, u4 = q % (UC / 4);
-                    const int br = (gate * H + half * Hh + cta * UC) / 4 + u4;
-                    for (int i = m->hR.row_ptr[br]; i < m->hR.row_ptr[br + 1]; ++i) {
-                        const int bc = m->hR.col[i];
-                        if ((bc >= Kb) == (ph == 1)) R[lbr].push_back({(uint16_t)(bc - ph * Kb), &m->hR.vals[(size_t)i * 16]});
+                    const int q = lbr - HR / BRH;                  // (half * 3 + gate) * (UC / BRH) + u
+                    const int half = q / (3 * (UC / BRH)), gate = (q / (UC / BRH)) % 3, u = q % (UC / BRH);
+                    M = &m->hR;
+                    br0 = (gate * H + half * Hh + cta * UC + u * BRH) / 4; bc_lo = ph * Kb; bc_hi = bc_lo + Kb;
+                }
+                if (!tall) {
+                    for (int i = M->row_ptr[br0]; i < M->row_ptr[br0 + 1]; ++i) {
+                        const int bc = M->col[i];
+                        if (bc < bc_lo || bc >= bc_hi) continue;
+                        Blk b;
+                        b.col = (uint16_t)(bc - bc_lo);
+                        std::memcpy(b.v, &M->vals[(size_t)i * 16], sizeof(b.v));
+                        R[lbr].push_back(b);
                     }
+                } else {
+                    // columns with a nonzero weight in any of the 16 rows, in ascending order
+                    std::vector<int> slot((size_t)4 * Kb, -1);
+                    std::vector<Blk> found;
+                    for (int r4 = 0; r4 < 4; ++r4)
+                        for (int i = M->row_ptr[br0 + r4]; i < M->row_ptr[br0 + r4 + 1]; ++i) {
+                            const int bc = M->col[i];
+                            if (bc < bc_lo || bc >= bc_hi) continue;
+                            for (int c = 0; c < 4; ++c) {
+                                bool any = false;
+                                for (int r = 0; r < 4; ++r) any = any || M->vals[(size_t)i * 16 + 4 * r + c] != 0.f;
+                                if (!any) continue;
+                                const int col = 4 * (bc - bc_lo) + c;
+                                if (slot[col] < 0) { slot[col] = (int)found.size(); Blk b; b.col = (uint16_t)col; std::memset(b.v, 0, sizeof(b.v)); found.push_back(b); }
+                                for (int r = 0; r < 4; ++r) found[slot[col]].v[4 * r4 + r] = M->vals[(size_t)i * 16 + 4 * r + c];
+                            }
+                        }
+                    std::sort(found.begin(), found.end(), [](const Blk &a, const Blk &b) { return a.col < b.col; });
+                    R[lbr] = found;
                 }
             }
         }
     // slice every (CTA, phase): block rows sorted by length (longest first, stable), dealt to the warps in runs; the
     // first w8 warps take four rows with eight lanes each, the others up to eight rows with four lanes each
     struct Slice { std::vector<int> rows; int T = 0, lpr = 4; };
-    int w8 = (8 * SNW - NBR) / 4;
+    const int lpr_n = tall ? 16 : 4, cap_n = 32 / lpr_n, cap_w = cap_n / 2;     // lanes per row and rows per warp, narrow / wide slices
+    int w8 = (cap_n * SNW - NBR) / (cap_n - cap_w);                              // warps that can afford wide rows
     if (w8 < 0) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
     if (w8 > SNW) w8 = SNW;
+    if (w8 * cap_w > NBR) w8 = NBR / cap_w;
     std::vector<std::vector<Slice>> slices(SCS * 2);              // [cta * 2 + phase][warp]
     int max_slots = 0;
     for (int cp = 0; cp < SCS * 2; ++cp) {
@@ -487,13 +571,13 @@ int sparse_prepare(wrnn_model *m)
         int next = 0, slots = 0;
         for (int w = 0; w < SNW; ++w) {
             Slice &sl = slices[cp][w];
-            sl.lpr = w < w8 ? 8 : 4;
+            sl.lpr = w < w8 ? 2 * lpr_n : lpr_n;
             const int cap = 32 / sl.lpr;
             // rows still to place, spread evenly over the remaining four-lane warps
             int nr = cap;
             if (w >= w8) { const int left = NBR - next, warps_left = SNW - w; nr = (left + warps_left - 1) / warps_left; }
+            if (nr > cap) nr = cap;
             if (nr > NBR - next) nr = NBR - next;
-            if (nr > cap) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
             size_t longest = 0;
             for (int i = 0; i < nr; ++i) { sl.rows.push_back(order[next + i]); longest = std::max(longest, R[order[next + i]].size()); }
             next += nr;
@@ -501,6 +585,7 @@ int sparse_prepare(wrnn_model *m)
             if (sl.T < 1) sl.T = 1;                                  // the loop's first loads are unconditional
             slots += sl.lpr * nr * sl.T;
         }
+        if (next != NBR) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
         max_slots = std::max(max_slots, slots);
     }
     k.max_slots = (max_slots + 7) & ~7;
@@ -629,7 +714,7 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     const SparsePack &k = *m->sparse_pack;
     SparseParams p;
     std::memset(&p, 0, sizeof(p));
-    p.H = k.H; p.K = k.K; p.NKT = k.NKT; p.UC = k.UC; p.HR = k.HR; p.NBR = k.NBR;
+    p.H = k.H; p.K = k.K; p.NKT = k.NKT; p.UC = k.UC; p.HR = k.HR; p.NBR = k.NBR; p.tall = k.tall;
     for (int ph = 0; ph < 2; ++ph) { p.off_meta[ph] = k.off_meta[ph]; p.off_col[ph] = k.off_col[ph]; p.off_val[ph] = k.off_val[ph]; }
     p.off_o2 = k.off_o2; p.off_o4 = k.off_o4; p.off_small = k.off_small; p.blob_bytes = k.blob_bytes;
     p.n_steps = a.n_steps; p.step0 = a.step0; p.stream0 = a.stream0; p.seed = a.seed;

@@ -406,6 +406,30 @@ def test_sparse_cluster_and_generic_kernels_agree(env):
             B.wrnn_destroy(m)
 
 
+def test_sparse_16x1_blocks_cluster_kernel(env):
+    """The H = 2048 model pruned to 96 % with 16 x 1 blocks (Section 3.2's m x 1 shape, one activation per block) on
+    the single-cluster kernel and on the generic kernel, both against the dense-with-zeros oracle."""
+    torch, B = env
+    wl = synth.WORKLOADS[5]
+    assert wl.block == (16, 1)
+    w, masks, cond = synth.build_workload(wl)
+    assert int(masks["R"].sum()) == 3 * round(0.04 * (2048 // 16) * 2048)
+    om = orc.OracleModel(w, wl.dtype, masks, wl.block)
+    res = om.run(cond, 600, 1, SEED, dump=True)
+    for kern in (B.WRNN_KERNEL_SPARSE, B.WRNN_KERNEL_GENERIC):
+        m = B.wrnn_create(w, wl.dtype, masks, kernel=kern, block=wl.block)
+        try:
+            assert B.wrnn_launch_info(m, 1)["kernel"] == kern
+            r = pu.teacher_forced_parity(torch, B, m, om, cond, 600, 1, SEED, oracle_free=res)
+            _report("sparse 16x1 blocks, kernel %d" % kern, r)
+            _tol_check(r, wl.dtype)
+            if kern == B.WRNN_KERNEL_SPARSE:
+                free = _free_run(torch, B, m, cond, 600, 1, SEED)
+                _check_free_run_against_oracle(free, res)
+        finally:
+            B.wrnn_destroy(m)
+
+
 def test_config3_subscale_fold_batch16(env):
     """One 24,000-sample sequence as 16 interleaved sub-sequences of 1,500 steps in lock-step, then unfolded."""
     torch, B = env

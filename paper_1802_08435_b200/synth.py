@@ -104,7 +104,7 @@ class Workload:
     block: tuple = (4, 4)     # shape of one block of the sparsity masks (rows, columns)
 
 
-# The five named workloads (index = position in the benchmark's config list), then two extra sparse ones.
+# The five named workloads (index = position in the benchmark's config list), then three extra ones.
 WORKLOADS = [
     Workload("dense896_f32_b1_1200", 896, "f32", 1, 1200, 10),
     Workload("dense896_bf16_b1_24000", 896, "bf16", 1, 24000, 200),
@@ -114,6 +114,8 @@ WORKLOADS = [
     # beyond the five benchmark configurations: the other block shapes of Section 3.2 (same model, same sparsity)
     Workload("sparse2048_16x1_bf16_b1_24000", 2048, "bf16", 1, 24000, 200, sparsity=0.96, block=(16, 1)),
     Workload("sparse2048_1x1_bf16_b1_2400", 2048, "bf16", 1, 2400, 20, sparsity=0.96, block=(1, 1)),
+    # the paper's own small-batch point (Section 5.1: four utterances at once)
+    Workload("batched4_896_bf16_24000", 896, "bf16", 4, 24000, 200),
 ]
 
 

@@ -164,18 +164,15 @@ def main():
         return
 
     import torch
-    import torch.distributed as dist
     from paper_1802_08435_b200 import binding as B
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_1802_08435_b200 import replicas
+    rank, world, local = replicas.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    pg = replicas.init("nccl", dev)
 
     n_steps = wl.n_steps if args.n_steps is None else args.n_steps
     w, masks, cond_np = synth.build_workload(wl)
@@ -187,7 +184,7 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # > 126 MB L2
     # rows of different ranks are different streams of the same workload (replicas; no collective on the path)
     kw = dict(hop=synth.HOP, row_stride=wl.row_stride, row_offset_mul=wl.row_offset_mul, stream0=0)
-    seed = synth.SEED_SAMPLING + rank
+    seed = replicas.rank_seed(synth.SEED_SAMPLING, rank)
 
     def one():
         B.wrnn_sample(model, cond, n_steps, wl.batch, seed, out, **kw)
@@ -201,8 +198,7 @@ def main():
     if rank == 0:
         sampler.start()
         time.sleep(0.25)
-    if world > 1:
-        dist.barrier()
+    replicas.barrier(pg)
     torch.cuda.synchronize()
     launches0 = B.wrnn_launch_count()
     evs = []
@@ -215,19 +211,14 @@ def main():
         evs.append((e0, e1))
     torch.cuda.synchronize()
     launches = B.wrnn_launch_count() - launches0
-    if world > 1:
-        dist.barrier()
-    total_ms = sum(a.elapsed_time(b) for a, b in evs)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    replicas.barrier(pg)
+    total_ms = replicas.max_over_ranks(sum(a.elapsed_time(b) for a, b in evs), pg, dev)
     clocks = sampler.stop() if rank == 0 else None
     assert B.wrnn_poll_status(model) == 0, B.wrnn_last_error(model)
 
     ms_per_step = total_ms / args.steps
     samples_per_call = n_steps * wl.batch
-    value = world * samples_per_call / (ms_per_step * 1e-3)
+    value = replicas.aggregate_throughput(world, samples_per_call, ms_per_step * 1e-3)
 
     # end to end through the host-buffer entry point (pinned host memory)
     e2e = None
@@ -236,18 +227,14 @@ def main():
         out_pin = torch.zeros((wl.batch, n_steps), dtype=torch.int16).pin_memory()
         for _ in range(2):
             B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
-        if world > 1:
-            dist.barrier()
+        replicas.barrier(pg)
         t0 = time.perf_counter()
         for _ in range(args.steps):
             B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
         dt = (time.perf_counter() - t0) / args.steps
-        if world > 1:
-            t = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = replicas.max_over_ranks(dt, pg, dev)
         assert np.array_equal(out_pin.numpy(), out.cpu().numpy()), "host-buffer path disagrees with the device path"
-        e2e = {"value": world * samples_per_call / dt, "unit": UNIT, "h2d_bytes_per_step": int(cond_np.nbytes),
+        e2e = {"value": replicas.aggregate_throughput(world, samples_per_call, dt), "unit": UNIT, "h2d_bytes_per_step": int(cond_np.nbytes),
                "d2h_bytes_per_step": int(out_pin.numel() * 2)}
 
     if rank == 0:
@@ -313,8 +300,8 @@ def main():
             line["cpu_baseline"] = cpu_baseline(wl)
         print(json.dumps(line), flush=True)
     B.wrnn_destroy(model)
-    if world > 1:
-        dist.destroy_process_group()
+    if pg is not None:
+        pg.destroy_process_group()
 
 
 if __name__ == "__main__":

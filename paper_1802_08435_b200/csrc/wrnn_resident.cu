@@ -204,15 +204,28 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
 
     // Gates of Eq. 2 for this CTA's units of one half of the state, then publish them to the chip.
     // half_g = 0: coarse units (c_s does not reach them: their I* column is zero), 1: fine units.
-    auto gates_and_publish = [&](int half_g, long long s, int drawn, const float (&gv)[3]) {
+    // The gate pre-activations up to the one input that is only known after the draw (c_s for the fine units, f_{s-1} for
+    // the coarse units of the next step): computed while the logits are still on their way.
+    struct GatePre { float pu, pr, pe, ae, ku, kr, ke; };
+    auto gates_prepare = [&](int half_g, const float (&gv)[3]) {
+        GatePre q;
         const int rb = half_g ? 3 * UC : 0;
-        const float x0 = scale8(c_prev), x1 = scale8(f_prev), x2 = half_g ? scale8(drawn) : 0.f;
+        const float x0 = scale8(c_prev), x1 = scale8(f_prev);
         const float *Iu = sI + 3 * (rb + lane), *Ir = sI + 3 * (rb + UC + lane), *Ie = sI + 3 * (rb + 2 * UC + lane);
-        const float pu = a_full[rb + lane] + fmaf(Iu[0], x0, fmaf(Iu[1], x1, fmaf(Iu[2], x2, gv[0])));
-        const float pr = a_full[rb + UC + lane] + fmaf(Ir[0], x0, fmaf(Ir[1], x1, fmaf(Ir[2], x2, gv[1])));
-        const float pe = fmaf(Ie[0], x0, fmaf(Ie[1], x1, fmaf(Ie[2], x2, gv[2])));
-        const float u = sigmoidf_fast(pu), r = sigmoidf_fast(pr);
-        const float e = tanhf_fast(fmaf(r, a_full[rb + 2 * UC + lane], pe));
+        // fine units: inputs (c_{s-1}, f_{s-1}) known, c_s pending (column 2); coarse units: c_{s-1} known, f_{s-1} pending (column 1)
+        q.pu = a_full[rb + lane] + fmaf(Iu[0], x0, half_g ? fmaf(Iu[1], x1, gv[0]) : gv[0]);
+        q.pr = a_full[rb + UC + lane] + fmaf(Ir[0], x0, half_g ? fmaf(Ir[1], x1, gv[1]) : gv[1]);
+        q.pe = fmaf(Ie[0], x0, half_g ? fmaf(Ie[1], x1, gv[2]) : gv[2]);
+        q.ae = a_full[rb + 2 * UC + lane];
+        q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
+        return q;
+    };
+    // Gates of Eq. 2 for this CTA's units of one half of the state, then publish them to the chip.
+    // half_g = 0: coarse units (c_s does not reach them: their I* column is zero), 1: fine units.
+    auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
+        const float xk = scale8(drawn);                  // the pending input
+        const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
+        const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
@@ -230,7 +243,7 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
     if (warp == 0 && lane < UC) {
         float gv[3];
         load_g(0, 0, gv);
-        gates_and_publish(0, 0, 0, gv);
+        gates_and_publish(0, 0, f_prev, gates_prepare(0, gv));
     }
 
     // The step is two structurally identical halves (Fig. 1).  Half-step n = 2 s + 1 is the "coarse" half of
@@ -285,6 +298,9 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         __syncthreads();
         STAMP(12 + half);
         if (h_fin) {
+            // the hidden-layer rows first: the whole cluster waits for them
+            if (par) finish_and_send<KSH, true>(part + warp * KSH * 16, bh, 16 * warp, HR, lane, q_dst[1], tag, peer_ok);
+            else     finish_and_send<KSH, true>(part + warp * KSH * 16, bh, 16 * warp, HR, lane, q_dst[0], tag, peer_ok);
             // R rows of this tile (rows >= HR of the stacked matrix) stay in this CTA
             const int row = 16 * warp + lane;
             if (lane < 16 && row >= HR) {
@@ -294,8 +310,6 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
                 if (half) a_part[row - HR] = v;                                    // R[:, :Hh] y_c(s): kept for step s+1
                 else a_full[row - HR] = a_part[row - HR] + v;                      // R h_{s-1} complete
             }
-            if (par) finish_and_send<KSH, true>(part + warp * KSH * 16, bh, 16 * warp, HR, lane, q_dst[1], tag, peer_ok);
-            else     finish_and_send<KSH, true>(part + warp * KSH * 16, bh, 16 * warp, HR, lane, q_dst[0], tag, peer_ok);
         }
         STAMP(1 + 6 * half);
 
@@ -329,6 +343,8 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
 
         // ---- 4. warp 0: the cluster's 256 logits -> draw; then the gates of the other half of the state
         if (warp == 0) {
+            GatePre gp = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            if (lane < UC && !last) gp = gates_prepare(half, gv);
             float l[8];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -360,7 +376,7 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
                 if (writer && lane == 0 && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + drawn - 32768);
                 f_prev = drawn;
             }
-            if (lane < UC && !last && !my_bad) gates_and_publish(half, s, drawn, gv);
+            if (lane < UC && !last && !my_bad) gates_and_publish(half, s, drawn, gp);
             if (half) c_prev = drawn;
         }
         STAMP(5 + 6 * half);

@@ -147,7 +147,6 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
 #define STAMP(i) do { if (prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
 
     const bool writer = (cta == 0);
-    float *sc = scratch + 16 * warp;
     const int g4 = lane >> 2;
 
     // warp 0 keeps the stream's scalar state

@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int K = p.K, NKT = p.NKT, UC = p.UC, HR = p.HR, NBR = p.NBR, H = p.H;
+    const int K = p.K, NKT = p.NKT, UC = p.UC, HR = p.HR, H = p.H;
     const int NR = 6 * UC;
 
     // ---- shared memory carve-up (must match sparse_smem_bytes)

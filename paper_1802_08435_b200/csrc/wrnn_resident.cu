@@ -159,9 +159,17 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
     const int h_tile = warp / KSH, h_kt0 = (warp % KSH) * NKH;
     const int l_tile = warp / KSL, l_kt0 = (warp % KSL) * NKL;
     const bool h_on = warp < NMT * KSH, l_on = warp < NLT * KSL;
-    const bool h_fin = warp < NMT, l_fin = warp < NLT;
+    const bool h_fin = warp < NMT;
     // cluster addresses of this lane's two destination slots (pairs ps and ps + 4 of tile `warp`) at peer lane & 7,
     // for both buffer parities, for the hidden-layer buffer and the logits buffer
+    // one peer per warp: warp w sends this CTA's whole slice to CTA w of the cluster with one store instruction, lanes at
+    // consecutive 16-byte slots (a store whose lanes address several CTAs at once is much slower)
+    unsigned q_snd[2], l_snd[2];
+#pragma unroll
+    for (int par2 = 0; par2 < 2; ++par2) {
+        q_snd[par2] = map_to_rank(smem_addr(qbuf + (size_t)par2 * (K / 2) + (rank * HR) / 2 + (lane < HR / 2 ? lane : 0)), warp < CS ? warp : 0);
+        l_snd[par2] = map_to_rank(smem_addr(lbuf + (size_t)par2 * 128 + (rank * LR) / 2 + (lane < LR / 2 ? lane : 0)), warp < CS ? warp : 0);
+    }
     unsigned q_dst[2][2], l_dst[2][2];
     const bool peer_ok = (lane & 7) < CS;
 #pragma unroll
@@ -296,13 +304,19 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         }
         __syncthreads();
         STAMP(12 + half);
-        if (h_fin) {
-            // the hidden-layer rows first: the whole cluster waits for them
-            if (par) finish_and_send<KSH, true>(part + warp * KSH * 16, bh, 16 * warp, HR, lane, q_dst[1], tag, peer_ok);
-            else     finish_and_send<KSH, true>(part + warp * KSH * 16, bh, 16 * warp, HR, lane, q_dst[0], tag, peer_ok);
+        // warp w finishes the whole hidden-layer slice of this CTA itself (two rows per lane: K-split partials, bias,
+        // relu) and sends it to CTA w of the cluster: one store instruction per peer, no further CTA barrier
+        if (warp < CS && lane < HR / 2) {
+            const int r0 = 2 * lane, tile = r0 >> 4, rr = r0 & 15;
+            float v0 = bh[r0], v1 = bh[r0 + 1];
+#pragma unroll
+            for (int sp = 0; sp < KSH; ++sp) { v0 += part[(tile * KSH + sp) * 16 + rr]; v1 += part[(tile * KSH + sp) * 16 + rr + 1]; }
+            st_cluster_ll(q_snd[par], fmaxf(v0, 0.f), fmaxf(v1, 0.f), tag);
+        }
+        if (h_fin && lane < 16) {
             // R rows of this tile (rows >= HR of the stacked matrix) stay in this CTA
             const int row = 16 * warp + lane;
-            if (lane < 16 && row >= HR) {
+            if (row >= HR && row - HR < NR) {
                 float v = 0.f;
 #pragma unroll
                 for (int sp = 0; sp < KSH; ++sp) v += part[(warp * KSH + sp) * 16 + lane];
@@ -334,9 +348,12 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         }
         __syncthreads();
         STAMP(14 + half);
-        if (l_fin) {
-            if (par) finish_and_send<KSL, false>(part + warp * KSL * 16, bl, 16 * warp, LR, lane, l_dst[1], tag, peer_ok);
-            else     finish_and_send<KSL, false>(part + warp * KSL * 16, bl, 16 * warp, LR, lane, l_dst[0], tag, peer_ok);
+        if (warp < CS && lane < LR / 2) {
+            const int r0 = 2 * lane, tile = r0 >> 4, rr = r0 & 15;
+            float v0 = bl[r0], v1 = bl[r0 + 1];
+#pragma unroll
+            for (int sp = 0; sp < KSL; ++sp) { v0 += part[(tile * KSL + sp) * 16 + rr]; v1 += part[(tile * KSL + sp) * 16 + rr + 1]; }
+            st_cluster_ll(l_snd[par], v0, v1, tag);
         }
         STAMP(3 + 6 * half);
 
@@ -345,16 +362,20 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
             GatePre gp = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
             if (lane < UC && !last) gp = gates_prepare(half, gv);
             float l[8];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const unsigned a = smem_addr(lbuf + (size_t)par * 128 + 4 * lane + k);
-                uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
+            {
+                // the four slots of this lane are loaded together and re-read until all of them carry this half-step's tag
+                const unsigned a = smem_addr(lbuf + (size_t)par * 128 + 4 * lane);
+                uint4 v0, v1, v2, v3;
+                unsigned long long t0 = 0; unsigned cnt = 0;
                 while (true) {
-                    v = ld_shared_volatile_v4(a);
-                    if (v.y == tag && v.w == tag) break;
+                    v0 = ld_shared_volatile_v4(a); v1 = ld_shared_volatile_v4(a + 16);
+                    v2 = ld_shared_volatile_v4(a + 32); v3 = ld_shared_volatile_v4(a + 48);
+                    const bool ok = v0.y == tag && v0.w == tag && v1.y == tag && v1.w == tag && v2.y == tag && v2.w == tag && v3.y == tag && v3.w == tag;
+                    if (ok) break;
                     if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 3 + 4 * half)) { my_bad = true; break; }
                 }
-                l[2 * k] = __uint_as_float(v.x); l[2 * k + 1] = __uint_as_float(v.z);
+                l[0] = __uint_as_float(v0.x); l[1] = __uint_as_float(v0.z); l[2] = __uint_as_float(v1.x); l[3] = __uint_as_float(v1.z);
+                l[4] = __uint_as_float(v2.x); l[5] = __uint_as_float(v2.z); l[6] = __uint_as_float(v3.x); l[7] = __uint_as_float(v3.z);
             }
             my_bad = __any_sync(FULL, my_bad);
             STAMP(4 + 6 * half);

@@ -245,19 +245,31 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
 #pragma unroll
         for (int gate = 0; gate < 3; ++gate) gv[gate] = __ldg(g + gate * H);
     };
-    auto gates = [&](int half_g, long long s, int drawn, const float (&gv)[3]) {
-        const int rb = half_g ? 3 * UC : 0;
-        const float *vec = half_g ? vecF : vecC;    // previous value of these units: still in the fp32 vector of that half
+    // The gate pre-activations up to the one input that is only known after the draw (c_s for the fine units, f_{s-1} for
+    // the coarse units of the next step): computed while the logits are still on their way.
+    struct GatePre { float pu, pr, pe, ae, ku, kr, ke, hprev; };
+    auto gates_prepare = [&](int half_g, const float (&gv)[3]) {
+        GatePre q = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        if (lane < UW) {
+            const int rb = half_g ? 3 * UC : 0, u0 = warp * UW + lane;
+            const float x0 = scale8(c_prev), x1 = scale8(f_prev);
+            const float *Iu = sI + 3 * (rb + u0), *Ir = sI + 3 * (rb + UC + u0), *Ie = sI + 3 * (rb + 2 * UC + u0);
+            q.pu = a_full[rb + u0] + fmaf(Iu[0], x0, half_g ? fmaf(Iu[1], x1, gv[0]) : gv[0]);
+            q.pr = a_full[rb + UC + u0] + fmaf(Ir[0], x0, half_g ? fmaf(Ir[1], x1, gv[1]) : gv[1]);
+            q.pe = fmaf(Ie[0], x0, half_g ? fmaf(Ie[1], x1, gv[2]) : gv[2]);
+            q.ae = a_full[rb + 2 * UC + u0];
+            q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
+            q.hprev = (half_g ? vecF : vecC)[rank * UC + u0];       // previous value of the unit: still in the fp32 vector of that half
+        }
+        return q;
+    };
+    auto gates = [&](int half_g, long long s, int drawn, const GatePre &q) {
         if (lane < UW) {
             const int u0 = warp * UW + lane;
-            const float x0 = scale8(c_prev), x1 = scale8(f_prev), x2 = half_g ? scale8(drawn) : 0.f;
-            const float *Iu = sI + 3 * (rb + u0), *Ir = sI + 3 * (rb + UC + u0), *Ie = sI + 3 * (rb + 2 * UC + u0);
-            const float pu = a_full[rb + u0] + fmaf(Iu[0], x0, fmaf(Iu[1], x1, fmaf(Iu[2], x2, gv[0])));
-            const float pr = a_full[rb + UC + u0] + fmaf(Ir[0], x0, fmaf(Ir[1], x1, fmaf(Ir[2], x2, gv[1])));
-            const float pe = fmaf(Ie[0], x0, fmaf(Ie[1], x1, fmaf(Ie[2], x2, gv[2])));
-            const float u = sigmoidf_fast(pu), r = sigmoidf_fast(pr);
-            const float e = tanhf_fast(fmaf(r, a_full[rb + 2 * UC + u0], pe));
-            const float hn = fmaf(u, vec[rank * UC + u0], (1.0f - u) * e);
+            const float xk = scale8(drawn);              // the pending input
+            const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
+            const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
+            const float hn = fmaf(u, q.hprev, (1.0f - u) * e);
             ynew[u0] = hn;
             const int jj = (half_g ? K : 0) + rank * UC + u0;
             if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
@@ -282,7 +294,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     if (warp < GW) {
         float gv0[3] = {0.f, 0.f, 0.f};
         if (lane < UW) load_g(0, 0, gv0);
-        gates(0, 0, 0, gv0);
+        gates(0, 0, f_prev, gates_prepare(0, gv0));
     }
     __syncthreads();
     publish(1u);
@@ -382,17 +394,22 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
 
         // ---- 4. warps 0..GW-1: the cluster's 256 logits -> draw; then the gates of the other half, published to the cluster
         if (warp < GW) {
+            const GatePre gp = gates_prepare(half, gv);
             float l[8];
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const unsigned a = smem_addr(lbuf + 4 * lane + k);
-                uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
+            {
+                // the four slots of this lane are loaded together and re-read until all of them carry this half-step's tag
+                const unsigned a = smem_addr(lbuf + 4 * lane);
+                uint4 v0, v1, v2, v3;
+                unsigned long long t0 = 0; unsigned cnt = 0;
                 while (true) {
-                    v = ld_shared_volatile_v4(a);
-                    if (v.y == tag && v.w == tag) break;
+                    v0 = ld_shared_volatile_v4(a); v1 = ld_shared_volatile_v4(a + 16);
+                    v2 = ld_shared_volatile_v4(a + 32); v3 = ld_shared_volatile_v4(a + 48);
+                    const bool ok = v0.y == tag && v0.w == tag && v1.y == tag && v1.w == tag && v2.y == tag && v2.w == tag && v3.y == tag && v3.w == tag;
+                    if (ok) break;
                     if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 3 + 4 * half)) { my_bad = true; break; }
                 }
-                l[2 * k] = __uint_as_float(v.x); l[2 * k + 1] = __uint_as_float(v.z);
+                l[0] = __uint_as_float(v0.x); l[1] = __uint_as_float(v0.z); l[2] = __uint_as_float(v1.x); l[3] = __uint_as_float(v1.z);
+                l[4] = __uint_as_float(v2.x); l[5] = __uint_as_float(v2.z); l[6] = __uint_as_float(v3.x); l[7] = __uint_as_float(v3.z);
             }
             my_bad = __any_sync(FULL, my_bad);
             SSTAMP(4);
@@ -414,7 +431,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
                 f_prev = drawn;
             }
             SSTAMP(5);
-            if (!last && !my_bad) gates(half, s, drawn, gv);
+            if (!last && !my_bad) gates(half, s, drawn, gp);
             if (half) c_prev = drawn;
             SSTAMP(6);
         }

@@ -262,7 +262,7 @@ def main():
             alg_bytes = n_w * (2 if wl.dtype == "bf16" else 4)
             ach = alg_bytes * n_steps / (ms_per_step * 1e-3) / 1e9
             roof = {"bound": "smem", "achieved": ach, "peak": SMEM_PEAK_GBS, "unit": "GB/s", "frac": ach / SMEM_PEAK_GBS,
-                    "traffic": 22862848 if info["kernel"] == 2 else None,
+                    "traffic": 22862848 if info["kernel"] == 2 and wl.dtype == "bf16" else None,
                     "traffic_note": "DRAM bytes per launch from the ncu capture in profiles/ (one-time weight load; "
                                     "does not grow with the number of steps)",
                     "peak_source": "derived: 148 SMs x 128 B/clk x 1.965 GHz", "algorithmic_bytes_per_step": alg_bytes,
@@ -274,6 +274,12 @@ def main():
                 roof["latency_floor"] = {"smem_us": smem_us, "t_bar_us": t_bar_ns * 1e-3, "floor_us_per_step": floor_us,
                                          "frac_of_floor": floor_us / us_per_sample_step,
                                          "note": "weight bytes / smem bandwidth + 2 x measured chip-wide exchange"}
+            if info["kernel"] == 2 and wl.dtype != "bf16":      # the fp32 resident kernel: five stamped phases per half
+                pc = B.wrnn_phase_cycles(model)
+                names = [h + n for h in ("F.", "C.") for n in ("wait_y", "hid_rows_publish", "wait_q", "logit_rows_send", "wait_logits", "draw_gates")]
+                roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
+                roof["wait_share"] = sum(pc[i] for i in (0, 2, 4, 6, 8, 10)) / (float(sum(pc)) or 1.0)
+            if info["kernel"] == 2 and wl.dtype == "bf16":      # the bf16 resident kernel stamps its phases
                 pc = B.wrnn_phase_cycles(model)
                 tot = float(sum(pc)) or 1.0
                 names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_gates",

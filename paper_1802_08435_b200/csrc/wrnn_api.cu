@@ -120,6 +120,12 @@ static bool use_resident(const wrnn_model *m, int batch)
     return m->resident != nullptr && resident_supported(m, batch, nullptr) == WRNN_OK;
 }
 
+static bool use_resf32(const wrnn_model *m, int batch)
+{
+    if (m->kernel == WRNN_KERNEL_GENERIC || m->kernel == WRNN_KERNEL_BATCHED || m->kernel == WRNN_KERNEL_BCLUSTER) return false;
+    return m->resf32 != nullptr && resf32_supported(m, batch, nullptr) == WRNN_OK;
+}
+
 static bool use_sparse(const wrnn_model *m, int batch)
 {
     if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_SPARSE) return false;
@@ -183,6 +189,7 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     int rc = cond_project(m, a.cond, a.batch, nf, s);
     if (rc != WRNN_OK) return fail(m, rc, "conditioning projection launch failed");
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
+    if (use_resf32(m, a.batch)) return resf32_run(m, a, s);
     if (use_sparse(m, a.batch)) return sparse_run(m, a, s);
     if (use_bcluster(m, a.batch)) return bcluster_run(m, a, s);
     if (use_batched(m, a.batch)) return batched_run(m, a, s);
@@ -203,7 +210,7 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     }
     if (m->kernel == WRNN_KERNEL_RESIDENT) {
         std::string why;
-        resident_supported(m, a.batch, &why);
+        if (m->dtype == WRNN_F32) resf32_supported(m, a.batch, &why); else resident_supported(m, a.batch, &why);
         return fail(m, WRNN_ERR_UNSUPPORTED, "resident kernel unavailable: " + why);
     }
     return generic_run(m, a, s);
@@ -321,7 +328,7 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
         }
     }
     if (p->kernel == WRNN_KERNEL_AUTO || p->kernel == WRNN_KERNEL_RESIDENT) {
-        const int rc = resident_prepare(m);
+        const int rc = m->dtype == WRNN_F32 ? resf32_prepare(m) : resident_prepare(m);
         if (rc != WRNN_OK && p->kernel == WRNN_KERNEL_RESIDENT) {
             const std::string why = m->err;
             wrnn_destroy(m);
@@ -338,6 +345,7 @@ void wrnn_destroy(wrnn_model *m)
     cudaSetDevice(m->device);
     cudaDeviceSynchronize();
     resident_destroy(m);
+    resf32_destroy(m);
     batched_destroy(m);
     bcluster_destroy(m);
     sparse_destroy(m);
@@ -464,6 +472,10 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
     }
+    if (use_resf32(m, batch)) {
+        if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
+        return resf32_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
+    }
     if (use_sparse(m, batch)) {
         if (kernel) *kernel = WRNN_KERNEL_SPARSE;
         return sparse_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
@@ -487,6 +499,7 @@ int wrnn_phase_cycles(wrnn_model *m, int64_t *out16)
 {
     if (!m || !out16) return WRNN_ERR_INVALID_ARG;
     static_assert(sizeof(long long) == sizeof(int64_t), "");
+    if (m->resf32) return resf32_phase_cycles(m, reinterpret_cast<long long *>(out16));
     return resident_phase_cycles(m, reinterpret_cast<long long *>(out16));
 }
 

@@ -52,6 +52,7 @@ struct StepArgs {
 struct ResidentPack;   // packed weights of the shared-memory-resident kernels (opaque here)
 struct BatchedPack;    // fragment-packed weights and activation images of the batched kernel (opaque here)
 struct SparsePack;     // compressed block rows of the single-cluster block-sparse kernel (opaque here)
+struct ResF32Pack;     // per-CTA fp32 weight shards of the single-stream fp32 resident kernel (opaque here)
 struct BcPack;         // per-CTA weight slices and stacked activation images of the cluster-partitioned multi-row kernel
 
 }  // namespace wrnn
@@ -84,6 +85,7 @@ struct wrnn_model {
     int16_t *stage_out = nullptr; size_t stage_out_cap = 0;
 
     wrnn::ResidentPack *resident = nullptr;
+    wrnn::ResF32Pack *resf32 = nullptr;
     wrnn::BatchedPack *batched = nullptr;
     wrnn::SparsePack *sparse_pack = nullptr;
     wrnn::BcPack *bcluster = nullptr;
@@ -116,6 +118,14 @@ int resident_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_thr
                          int64_t *weight_bytes);
 int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
 int resident_phase_cycles(const wrnn_model *m, long long *out16);
+
+// wrnn_resf32.cu: the same role for dense fp32 models (every matrix sharded chip-wide, nothing replicated)
+int resf32_supported(const wrnn_model *m, int batch, std::string *why);
+int resf32_prepare(wrnn_model *m);
+void resf32_destroy(wrnn_model *m);
+int resf32_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem, int64_t *weight_bytes);
+int resf32_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
+int resf32_phase_cycles(const wrnn_model *m, long long *out16);
 
 // wrnn_sparse.cu
 int sparse_supported(const wrnn_model *m, int batch, std::string *why);

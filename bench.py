@@ -274,17 +274,12 @@ def main():
                 roof["latency_floor"] = {"smem_us": smem_us, "t_bar_us": t_bar_ns * 1e-3, "floor_us_per_step": floor_us,
                                          "frac_of_floor": floor_us / us_per_sample_step,
                                          "note": "weight bytes / smem bandwidth + 2 x measured chip-wide exchange"}
-            if info["kernel"] == 2 and wl.dtype != "bf16":      # the fp32 resident kernel: five stamped phases per half
-                pc = B.wrnn_phase_cycles(model)
-                names = [h + n for h in ("F.", "C.") for n in ("wait_y", "hid_rows_publish", "wait_q", "logit_rows_send", "wait_logits", "draw_gates")]
-                roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
-                roof["wait_share"] = sum(pc[i] for i in (0, 2, 4, 6, 8, 10)) / (float(sum(pc)) or 1.0)
-            if info["kernel"] == 2 and wl.dtype == "bf16":      # the bf16 resident kernel stamps its phases
+            if info["kernel"] == 2:      # the resident kernels stamp their phases
                 pc = B.wrnn_phase_cycles(model)
                 tot = float(sum(pc)) or 1.0
                 names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_gates",
                          "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_gates",
-                         "F.hid_mma", "C.hid_mma", "F.log_mma", "C.log_mma"]
+                         "F.hid_products", "C.hid_products", "F.log_products", "C.log_products"]
                 roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
                 waits = sum(pc[i] for i in (0, 2, 4, 6, 8, 10))
                 roof["wait_share"] = waits / tot

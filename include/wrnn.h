@@ -232,9 +232,8 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
  *   3 / 9   logits finish and send to the cluster
  *   4 / 10  wait for the cluster's logits
  *   5 / 11  softmax draw, gates of the other half, publish
- * For a dense fp32 model (the hidden layer crosses the chip as well) the entries are six per half, fine half
- * 0..5, coarse half 6..11: wait for the state half; own hidden-layer and recurrent rows + publish; wait for the
- * hidden layer; own logit rows + send to the cluster; wait for the cluster's logits; draw + gates + publish.
+ * A dense fp32 model runs the fp32 variant of the kernel: the same slots, with "partial products" read as its
+ * plain fp32 row products, and 2 / 8 a second chip-wide wait (the hidden layer crosses L2 there).
  * Synchronous. */
 int wrnn_phase_cycles(wrnn_model *m, int64_t *out16);
 

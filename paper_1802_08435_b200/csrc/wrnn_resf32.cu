@@ -57,7 +57,7 @@ struct ResF32Params {
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
-    long long *prof;                         // [16] per-phase cycle totals of CTA 0, warp 0: 6 phases per half, fine half first
+    long long *prof;                         // [16] per-phase cycle totals of CTA 0, warp 0 (same slots as the bf16 kernel)
 };
 
 __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF32Params p)
@@ -244,6 +244,7 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
         // ---- 2. this CTA's rows of the hidden layer and of R against the same input; publish the hidden-layer rows
         rows_times(half ? wA : wB, NS, vec);
         __syncthreads();
+        STAMP(12 + half);
         stacked_finish(half ? sb1 : sb3, !half, p.qslots + (size_t)par * K, tag);
         STAMP(1 + 6 * half);
 
@@ -252,6 +253,7 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
         STAMP(2 + 6 * half);
         rows_times(half ? wO2 : wO4, LR, qvec);
         __syncthreads();
+        STAMP(14 + half);
         if (warp < CS) {
             const float *bl = half ? sb2 : sb4;
             for (int i = lane; i < LR / 2; i += 32) {

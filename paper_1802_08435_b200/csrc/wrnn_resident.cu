@@ -66,26 +66,6 @@ struct ResidentParams {
     long long *prof;                         // optional [16] per-phase cycle totals of CTA 0, warp 0
 };
 
-// Finish and send one 16-row tile of a cluster-wide vector: lane (peer = lane & 7, ps = lane >> 3) sums the
-// K-split partials of rows 2 p, 2 p + 1 for the pairs p = ps and ps + 4, applies bias (and relu), and stores the
-// two tagged values straight into the peer's buffer (16 bytes per store).  Rows at or beyond row_limit are
-// not sent.  dst[k] are the precomputed cluster addresses of slot 0 of this tile's pair p = ps + 4 k at the peer.
-template <int KS, bool RELU>
-__device__ __forceinline__ void finish_and_send(const float *part_tile, const float *bias, int row0, int row_limit,
-                                                int lane, const unsigned (&dst)[2], unsigned tag, bool peer_ok)
-{
-    const int ps = lane >> 3;
-#pragma unroll
-    for (int k = 0; k < 2; ++k) {
-        const int r = 2 * (ps + 4 * k);
-        float v0 = bias[row0 + r], v1 = bias[row0 + r + 1];
-#pragma unroll
-        for (int sp = 0; sp < KS; ++sp) { v0 += part_tile[sp * 16 + r]; v1 += part_tile[sp * 16 + r + 1]; }
-        if (RELU) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
-        if (peer_ok && row0 + r < row_limit) st_cluster_ll(dst[k], v0, v1, tag);
-    }
-}
-
 // KSH / KSL: K-splits per hidden / logits tile; NKH / NKL: k-tiles per split (KSH * NKH = KSL * NKL = K / 16).
 template <int KSH, int NKH, int KSL, int NKL>
 __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentParams p)
@@ -111,8 +91,7 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
     float *a_part = vecF + K;                                                  // [NR] R[:, :Hh] y_c
     float *a_full = a_part + NR;                                               // [NR] R h
     float *part = a_full + NR + ((2 * NR) % 4 ? 4 - (2 * NR) % 4 : 0);         // [tiles x K-splits][16] partial sums
-    float *scratch = part + 384;                                               // [24 warps][16]
-    __nv_bfloat16 *splC = reinterpret_cast<__nv_bfloat16 *>(scratch + 384);    // split images, 4 K bf16 each
+    __nv_bfloat16 *splC = reinterpret_cast<__nv_bfloat16 *>(part + 384);       // split images, 4 K bf16 each
     __nv_bfloat16 *splF = splC + 4 * K;
     __nv_bfloat16 *splQ = splF + 4 * K;
     uint4 *qbuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                    // [2][K/2]
@@ -160,8 +139,6 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
     const int l_tile = warp / KSL, l_kt0 = (warp % KSL) * NKL;
     const bool h_on = warp < NMT * KSH, l_on = warp < NLT * KSL;
     const bool h_fin = warp < NMT;
-    // cluster addresses of this lane's two destination slots (pairs ps and ps + 4 of tile `warp`) at peer lane & 7,
-    // for both buffer parities, for the hidden-layer buffer and the logits buffer
     // one peer per warp: warp w sends this CTA's whole slice to CTA w of the cluster with one store instruction, lanes at
     // consecutive 16-byte slots (a store whose lanes address several CTAs at once is much slower)
     unsigned q_snd[2], l_snd[2];
@@ -170,17 +147,6 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         q_snd[par2] = map_to_rank(smem_addr(qbuf + (size_t)par2 * (K / 2) + (rank * HR) / 2 + (lane < HR / 2 ? lane : 0)), warp < CS ? warp : 0);
         l_snd[par2] = map_to_rank(smem_addr(lbuf + (size_t)par2 * 128 + (rank * LR) / 2 + (lane < LR / 2 ? lane : 0)), warp < CS ? warp : 0);
     }
-    unsigned q_dst[2][2], l_dst[2][2];
-    const bool peer_ok = (lane & 7) < CS;
-#pragma unroll
-    for (int par2 = 0; par2 < 2; ++par2)
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            const int pair = (lane >> 3) + 4 * k;
-            q_dst[par2][k] = map_to_rank(smem_addr(qbuf + (size_t)par2 * (K / 2) + (rank * HR + 16 * warp) / 2 + pair), peer_ok ? (lane & 7) : 0);
-            l_dst[par2][k] = map_to_rank(smem_addr(lbuf + (size_t)par2 * 128 + (rank * LR + 16 * warp) / 2 + pair), peer_ok ? (lane & 7) : 0);
-        }
-
     // ---- prologue: the recurrent products of step 0 from the initial state, coarse gates of step 0
     if (h_on) {
         float lo, hi;
@@ -188,7 +154,7 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
     }
     __syncthreads();
-    if (h_fin && lane < 16 && 16 * warp + lane >= HR) {
+    if (h_fin && lane < 16 && 16 * warp + lane >= HR && 16 * warp + lane - HR < NR) {
         float v = 0.f;
 #pragma unroll
         for (int sp = 0; sp < KSH; ++sp) v += part[(warp * KSH + sp) * 16 + lane];
@@ -201,7 +167,7 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
     }
     __syncthreads();
-    if (h_fin && lane < 16 && 16 * warp + lane >= HR) {
+    if (h_fin && lane < 16 && 16 * warp + lane >= HR && 16 * warp + lane - HR < NR) {
         float v = 0.f;
 #pragma unroll
         for (int sp = 0; sp < KSH; ++sp) v += part[(warp * KSH + sp) * 16 + lane];
@@ -423,7 +389,7 @@ static int resident_smem_bytes(const ResidentPack &k)
     size_t a = (size_t)2 * k.n_rrows;               // a_part, a_full
     a += (a % 4) ? 4 - (a % 4) : 0;
     b += a * 4;
-    b += 768 * 4;                                   // partial sums + per-warp scratch
+    b += 384 * 4;                                   // partial sums [24 warps][16]
     b += (size_t)12 * k.K * 2;                      // three split images of 4 K bf16
     b += (size_t)k.K * 16;                          // qbuf [2][K/2] x 16 B
     b += 256 * 16;                                  // lbuf [2][128] x 16 B
@@ -468,29 +434,29 @@ static void pack_tile(const std::vector<std::vector<uint16_t>> &rows, int K, uin
         }
 }
 
-static bool choose_shape(const wrnn_model *m, ResidentPack *k, std::string *why)
+static bool choose_shape(const wrnn_model *m, int CS, ResidentPack *k, std::string *why)
 {
     const int H = m->H, Hh = H / 2;
     if (m->dtype != WRNN_BF16) { if (why) *why = "resident kernel stores bf16 weights only"; return false; }
     if (m->sparse) { if (why) *why = "resident dense kernel does not take block masks"; return false; }
     if (H % 32 != 0) { if (why) *why = "H must be a multiple of 32"; return false; }
-    const int CS = 8;
-    if (Hh % (2 * CS) != 0) { if (why) *why = "H/2 must be a multiple of 16"; return false; }
+    if (CS != 8 && CS != 16) { if (why) *why = "cluster size must be 8 or 16"; return false; }
+    if (Hh % (2 * CS) != 0 || 256 % (16 * CS) != 0) { if (why) *why = "H/2 must be a multiple of twice the cluster size"; return false; }
     const int HR = Hh / CS, LR = 256 / CS;
     int best = 0;
     for (int ncta = CS; ncta <= m->n_sms; ncta += CS) {
         if (Hh % ncta) continue;
         const int uc = Hh / ncta;
-        if ((HR + 6 * uc) % 16 || uc > 32) continue;       // stacked [head rows ; R rows] must fill 16-row tiles
-        if ((HR + 6 * uc) / 16 > 16) continue;
+        if (uc > 32) continue;
+        if ((HR + 6 * uc + 15) / 16 > 16) continue;        // stacked [head rows ; R rows], padded with zero rows to 16-row tiles
         best = ncta;
     }
     if (!best) { if (why) *why = "no CTA count tiles H/2 into 16-row fragments"; return false; }
     k->CS = CS; k->NCTA = best; k->NC = best / CS; k->UC = Hh / best; k->HR = HR; k->LR = LR;
     k->K = Hh; k->NKT = Hh / 16; k->n_rrows = 6 * k->UC;
-    k->NMT = (HR + k->n_rrows) / 16; k->NLT = LR / 16;
+    k->NMT = (HR + k->n_rrows + 15) / 16; k->NLT = LR / 16;
     k->NW = 20; k->KSH = 4; k->KSL = 7;
-    if (k->NKT != 28 || k->NMT * k->KSH > k->NW || k->NLT * k->KSL > k->NW) {
+    if (k->NKT != 28 || k->NMT * k->KSH > k->NW || k->NLT * k->KSL > k->NW || CS > k->NW) {
         if (why) *why = "only the H/2 = 448 tiling (4 x 7 and 7 x 4 k-tiles) is instantiated";
         return false;
     }
@@ -529,21 +495,35 @@ static void fill_launch(const ResidentPack &k, cudaLaunchConfig_t *cfg, cudaLaun
 
 int resident_prepare(wrnn_model *m)
 {
+    // A cluster of 16 holds half as many head rows per CTA as a cluster of 8 (fewer weight fragments to stream per
+    // step); it needs the non-portable cluster size and enough co-resident clusters, else 8 is used.
+    // WRNN_RESIDENT_CS=8 / 16 forces one of them (diagnostic).
     ResidentPack k;
     std::string why;
-    if (!choose_shape(m, &k, &why)) { m->err = why; return WRNN_ERR_UNSUPPORTED; }
     cudaDeviceProp prop;
     cudaGetDeviceProperties(&prop, m->device);
-    if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "weights do not fit in shared memory"; return WRNN_ERR_UNSUPPORTED; }
-    if (cudaFuncSetAttribute(resident_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
-        cudaGetLastError(); m->err = "cannot raise the dynamic shared memory limit"; return WRNN_ERR_UNSUPPORTED;
+    cudaFuncSetAttribute(resident_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    cudaGetLastError();
+    const char *force = getenv("WRNN_RESIDENT_CS");
+    bool found = false;
+    for (int cs : {16, 8}) {
+        if (force && atoi(force) != cs) continue;
+        ResidentPack c;
+        if (!choose_shape(m, cs, &c, &why)) continue;
+        if ((size_t)c.smem_bytes > prop.sharedMemPerBlockOptin) { why = "weights do not fit in shared memory"; continue; }
+        if (cudaFuncSetAttribute(resident_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, c.smem_bytes) != cudaSuccess) {
+            cudaGetLastError(); why = "cannot raise the dynamic shared memory limit"; continue;
+        }
+        cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
+        fill_launch(c, &cfg, at, 0, false);
+        int max_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_fn(), &cfg) != cudaSuccess || max_clusters < c.NC) {
+            cudaGetLastError(); why = "not enough co-resident clusters on this device"; continue;
+        }
+        k = c; found = true;
+        break;
     }
-    cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
-    fill_launch(k, &cfg, at, 0, false);
-    int max_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_fn(), &cfg) != cudaSuccess || max_clusters < k.NC) {
-        cudaGetLastError(); m->err = "not enough co-resident clusters on this device"; return WRNN_ERR_UNSUPPORTED;
-    }
+    if (!found) { m->err = why; return WRNN_ERR_UNSUPPORTED; }
 
     // ---- per-CTA blobs
     const int H = m->H, K = k.K, UC = k.UC;
@@ -563,11 +543,12 @@ int resident_prepare(wrnn_model *m)
                 for (int r = 0; r < 16; ++r) {
                     const int row = 16 * mt + r;
                     if (row < k.HR) dense_row_bf16(*Oa[part], rank * k.HR + row, 0, K, rows[r].data());
-                    else {
+                    else if (row - k.HR < k.n_rrows) {
                         const int rr = row - k.HR;
                         const int half = rr / (3 * UC), gate = (rr / UC) % 3, u = rr % UC;
                         dense_row_bf16(m->hR, gate * H + half * K + cta * UC + u, part * K, K, rows[r].data());
                     }
+                    else std::fill(rows[r].begin(), rows[r].end(), (uint16_t)0);       // padding row of the last tile
                 }
                 pack_tile(rows, K, w + ((size_t)part * k.NMT + mt) * tile_elems);
             }

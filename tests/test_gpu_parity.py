@@ -208,6 +208,36 @@ def test_config0_dense_f32_1200(env, kernel):
         B.wrnn_destroy(m)
 
 
+@pytest.mark.parametrize("H", [32, 64, 96, 192, 512])
+def test_tiny_fp32_resident_kernel(env, H):
+    """The shared-memory-resident fp32 kernel at small widths (one unit per CTA, several cluster shapes): every gate,
+    state and logit against the oracle, a resumed run against an unbroken one, and the stream offset."""
+    torch, B = env
+    w = _tiny(H)
+    om = orc.OracleModel(w, "f32")
+    m = B.wrnn_create(w, "f32", max_batch=1, kernel=B.WRNN_KERNEL_RESIDENT)
+    try:
+        info = B.wrnn_launch_info(m, 1)
+        assert info["kernel"] == B.WRNN_KERNEL_RESIDENT and (H // 2) % info["n_ctas"] == 0
+        cond = synth.make_cond(3, 9, 4)
+        r = pu.teacher_forced_parity(torch, B, m, om, cond[:1], 80, 1, SEED, hop=10)
+        assert r["idx_bad"] == 0, r
+        assert r["gates_err"] < 1e-4 and r["h_err"] < 1e-4 and r["logits_err"] < 1e-4, r
+        full = _free_run(torch, B, m, cond[2:3], 80, 1, 77, hop=10, stream0=2)
+        ref = om.run(cond[2:3], 80, 1, 77, hop=10, stream0=2, dump=True)
+        div = pu.first_divergence(full, ref.out)
+        if div >= 0:
+            assert ref.margins[0, div].min() < pu.MARGIN
+        h = torch.zeros((1, H), dtype=torch.float32, device="cuda:0")
+        cp = torch.full((1,), 128, dtype=torch.uint8, device="cuda:0")
+        fp = torch.zeros((1,), dtype=torch.uint8, device="cuda:0")
+        a = _free_run(torch, B, m, cond[2:3], 33, 1, 77, hop=10, stream0=2, h=h, c_prev=cp, f_prev=fp)
+        b = _free_run(torch, B, m, cond[2:3], 47, 1, 77, hop=10, stream0=2, h=h, c_prev=cp, f_prev=fp, step0=33)
+        assert np.array_equal(np.concatenate([a, b], axis=1), full)
+    finally:
+        B.wrnn_destroy(m)
+
+
 def test_resume_and_state_roundtrip(env):
     torch, B = env
     w = _tiny(64)

@@ -118,5 +118,70 @@ __device__ __forceinline__ void mma_partial(const uint4 *A, int kt0, const __nv_
     lo = s_lo; hi = s_hi;
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same split image with two k-tiles per 16-byte piece: [K/32 k-tile pairs][4 t][4 parts][2 k-tiles][4 bf16], so that
+// one 16-byte load per lane brings the B fragments of two k-tiles (the load/store unit is the busiest unit of the
+// single-stream kernel, and its cost goes by instructions, not bytes).
+__host__ __device__ __forceinline__ int split2_pos(int i, int part)
+{
+    const int c = i & 15, kt = i >> 4;
+    const int t = (c & 7) >> 1, j = c & 1, hi = c >> 3;
+    return ((((((kt >> 1) * 4 + t) * 4 + part) << 1) + (kt & 1)) << 2) + 2 * hi + j;
+}
+
+__device__ __forceinline__ void store_split2(__nv_bfloat16 *split, int i, float x)
+{
+    const __nv_bfloat16 b0 = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(b0);
+    const __nv_bfloat16 b1 = __float2bfloat16_rn(r1);
+    const float r2 = r1 - __bfloat162float(b1);
+    const __nv_bfloat16 b2 = __float2bfloat16_rn(r2);
+    const int pos = split2_pos(i, 0);
+    split[pos] = b0; split[pos + 8] = b1; split[pos + 16] = b2;
+}
+
+// NK consecutive k-tiles (NK even, from the even k-tile kt0) of NT 16-row tiles (consecutive in memory, tile_u4 apart) of a
+// fragment-packed bf16 matrix times a split2 vector: the B fragments are loaded once for all NT tiles.  On return the
+// lanes with t = 0 hold the partial totals of rows g (lo[n]) and g + 8 (hi[n]) of tile n.
+template <int NK, int NT>
+__device__ __forceinline__ void mma_tiles(const uint4 *A, size_t tile_u4, int kt0, const __nv_bfloat16 *split, int lane, float (&lo)[NT], float (&hi)[NT])
+{
+    static_assert(NK % 2 == 0, "k-tiles come in pairs");
+    const int g = lane >> 2, t = lane & 3;
+    const uint4 *bsrc = reinterpret_cast<const uint4 *>(split) + ((kt0 >> 1) * 4 + t) * 4 + (g & 3);
+    uint4 av[NT][NK];
+    uint4 bv[NK / 2];
+#pragma unroll
+    for (int i = 0; i < NK / 2; ++i) bv[i] = bsrc[16 * i];
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+        for (int i = 0; i < NK; ++i) av[n][i] = A[n * tile_u4 + (size_t)(kt0 + i) * 32 + lane];
+    float acc[NT][2][4];
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[n][c][i] = 0.f;
+#pragma unroll
+    for (int i = 0; i < NK; ++i)
+#pragma unroll
+        for (int n = 0; n < NT; ++n) {
+            float *c = acc[n][i & 1];
+            const unsigned b0 = (i & 1) ? bv[i >> 1].z : bv[i >> 1].x, b1 = (i & 1) ? bv[i >> 1].w : bv[i >> 1].y;
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                         : "r"(av[n][i].x), "r"(av[n][i].y), "r"(av[n][i].z), "r"(av[n][i].w), "r"(b0), "r"(b1));
+        }
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+        float s_lo = (acc[n][0][0] + acc[n][1][0]) + (acc[n][0][1] + acc[n][1][1]);
+        float s_hi = (acc[n][0][2] + acc[n][1][2]) + (acc[n][0][3] + acc[n][1][3]);
+        s_lo += __shfl_xor_sync(FULL, s_lo, 1);      // t = 0 (columns 0,1) + t = 1 (columns 2,3)
+        s_hi += __shfl_xor_sync(FULL, s_hi, 1);
+        lo[n] = s_lo; hi[n] = s_hi;
+    }
+}
 
 }  // namespace wrnn

@@ -68,7 +68,7 @@ struct ResidentParams {
 
 // KSH / KSL: K-splits per hidden / logits tile; NKH / NKL: k-tiles per split (KSH * NKH = KSL * NKL = K / 16).
 template <int KSH, int NKH, int KSL, int NKL>
-__global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentParams p)
+__global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
     cg::cluster_group cluster = cg::this_cluster();
@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
     float *a_part = vecF + K;                                                  // [NR] R[:, :Hh] y_c
     float *a_full = a_part + NR;                                               // [NR] R h
     float *part = a_full + NR + ((2 * NR) % 4 ? 4 - (2 * NR) % 4 : 0);         // [tiles x K-splits][16] partial sums
-    __nv_bfloat16 *splC = reinterpret_cast<__nv_bfloat16 *>(part + 384);       // split images, 4 K bf16 each
+    __nv_bfloat16 *splC = reinterpret_cast<__nv_bfloat16 *>(part + 512);       // split images, 4 K bf16 each
     __nv_bfloat16 *splF = splC + 4 * K;
     __nv_bfloat16 *splQ = splF + 4 * K;
     uint4 *qbuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                    // [2][K/2]
@@ -108,8 +108,8 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         for (int i = tid; i < K; i += blockDim.x) {
             const float c = p.h_in ? p.h_in[i] : 0.f, f = p.h_in ? p.h_in[K + i] : 0.f;
             vecC[i] = c; vecF[i] = f;
-            store_split(splC, i, c);
-            store_split(splF, i, f);
+            store_split2(splC, i, c);
+            store_split2(splF, i, f);
         }
     }
     __syncthreads();
@@ -133,12 +133,24 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
     float hC = 0.f, hF = 0.f;
     if (warp == 0 && lane < UC) { hC = vecC[cta * UC + lane]; hF = vecF[cta * UC + lane]; }
 
-    // Fixed roles: in the hidden phase warp w takes K-split (w % KSH) of tile (w / KSH), in the logits
-    // phase K-split (w % KSL) of tile (w / KSL); each leaves 16 partial row sums in part[w].
-    const int h_tile = warp / KSH, h_kt0 = (warp % KSH) * NKH;
-    const int l_tile = warp / KSL, l_kt0 = (warp % KSL) * NKL;
-    const bool h_on = warp < NMT * KSH, l_on = warp < NLT * KSL;
+    // Fixed roles: in the hidden phase warp w takes K-split (w % KSH) of the tile pair (w / KSH), one load of the vector
+    // fragments serving both tiles; in the logits phase K-split (w % KSL) of tile (w / KSL).  Each leaves 16 partial row
+    // sums per tile in part[tile * K-splits + split].
+    const int h_pair = warp / KSH, h_ks = warp % KSH, h_kt0 = h_ks * NKH;
+    const int l_tile = warp / KSL, l_ks = warp % KSL, l_kt0 = l_ks * NKL;
+    const bool h_on = warp < (NMT / 2) * KSH, l_on = warp < NLT * KSL;
     const bool h_fin = warp < NMT;
+    auto hidden_products = [&](const uint4 *Mx, const __nv_bfloat16 *sp) {
+        float lo[2], hi[2];
+        mma_tiles<NKH, 2>(Mx + (size_t)(2 * h_pair) * tile_u4, tile_u4, h_kt0, sp, lane, lo, hi);
+        if ((lane & 3) == 0) {
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                float *d = part + ((2 * h_pair + n) * KSH + h_ks) * 16;
+                d[g4] = lo[n]; d[g4 + 8] = hi[n];
+            }
+        }
+    };
     // one peer per warp: warp w sends this CTA's whole slice to CTA w of the cluster with one store instruction, lanes at
     // consecutive 16-byte slots (a store whose lanes address several CTAs at once is much slower)
     unsigned q_snd[2], l_snd[2];
@@ -148,11 +160,7 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         l_snd[par2] = map_to_rank(smem_addr(lbuf + (size_t)par2 * 128 + (rank * LR) / 2 + (lane < LR / 2 ? lane : 0)), warp < CS ? warp : 0);
     }
     // ---- prologue: the recurrent products of step 0 from the initial state, coarse gates of step 0
-    if (h_on) {
-        float lo, hi;
-        mma_partial<NKH>(wMA + (size_t)h_tile * tile_u4, h_kt0, splC, lane, lo, hi);
-        if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
-    }
+    if (h_on) hidden_products(wMA, splC);
     __syncthreads();
     if (h_fin && lane < 16 && 16 * warp + lane >= HR && 16 * warp + lane - HR < NR) {
         float v = 0.f;
@@ -161,11 +169,7 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
         a_part[16 * warp + lane - HR] = v;
     }
     __syncthreads();
-    if (h_on) {
-        float lo, hi;
-        mma_partial<NKH>(wMB + (size_t)h_tile * tile_u4, h_kt0, splF, lane, lo, hi);
-        if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
-    }
+    if (h_on) hidden_products(wMB, splF);
     __syncthreads();
     if (h_fin && lane < 16 && 16 * warp + lane >= HR && 16 * warp + lane - HR < NR) {
         float v = 0.f;
@@ -256,18 +260,14 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
                     if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
                 const float x = __uint_as_float((unsigned)v);
                 vec[i] = x;
-                store_split(spl, i, x);
+                store_split2(spl, i, x);
             }
             if (__syncthreads_or(my_bad)) break;
         }
         STAMP(0 + 6 * half);
 
         // ---- 2. hidden layer of the head + this CTA's R rows against the same input
-        if (h_on) {
-            float lo, hi;
-            mma_partial<NKH>(M + (size_t)h_tile * tile_u4, h_kt0, spl, lane, lo, hi);
-            if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
-        }
+        if (h_on) hidden_products(M, spl);
         __syncthreads();
         STAMP(12 + half);
         // warp w finishes the whole hidden-layer slice of this CTA itself (two rows per lane: K-split partials, bias,
@@ -302,15 +302,15 @@ __global__ void __launch_bounds__(640, 1) resident_dense_kernel(const ResidentPa
                 if (v.y == tag && v.w == tag) break;
                 if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 2 + 4 * half)) { my_bad = true; break; }
             }
-            store_split(splQ, 2 * i, __uint_as_float(v.x));
-            store_split(splQ, 2 * i + 1, __uint_as_float(v.z));
+            store_split2(splQ, 2 * i, __uint_as_float(v.x));
+            store_split2(splQ, 2 * i + 1, __uint_as_float(v.z));
         }
         if (__syncthreads_or(my_bad)) break;
         STAMP(2 + 6 * half);
         if (l_on) {
-            float lo, hi;
-            mma_partial<NKL>(L + (size_t)l_tile * tile_u4, l_kt0, splQ, lane, lo, hi);
-            if ((lane & 3) == 0) { part[warp * 16 + g4] = lo; part[warp * 16 + g4 + 8] = hi; }
+            float lo[1], hi[1];
+            mma_tiles<NKL, 1>(L + (size_t)l_tile * tile_u4, tile_u4, l_kt0, splQ, lane, lo, hi);
+            if ((lane & 3) == 0) { part[warp * 16 + g4] = lo[0]; part[warp * 16 + g4 + 8] = hi[0]; }
         }
         __syncthreads();
         STAMP(14 + half);
@@ -389,7 +389,7 @@ static int resident_smem_bytes(const ResidentPack &k)
     size_t a = (size_t)2 * k.n_rrows;               // a_part, a_full
     a += (a % 4) ? 4 - (a % 4) : 0;
     b += a * 4;
-    b += 384 * 4;                                   // partial sums [24 warps][16]
+    b += 512 * 4;                                   // partial sums [tiles x K-splits][16]
     b += (size_t)12 * k.K * 2;                      // three split images of 4 K bf16
     b += (size_t)k.K * 16;                          // qbuf [2][K/2] x 16 B
     b += 256 * 16;                                  // lbuf [2][128] x 16 B
@@ -419,7 +419,7 @@ static void dense_row_bf16(const BsrHost &M, int row, int c0, int n, uint16_t *d
 
 // rows[16][K] (bf16 bits, natural column order) -> A fragments [K/16][32 lanes][8] of m16n8k16:
 // lane (g, t) holds (row g, k 2t..2t+1), (row g+8, same), (row g, k 2t+8..9), (row g+8, same).
-// The vector side stores element 16 kt + c at split_pos and the B-fragment load reads it back from
+// The vector side stores element 16 kt + c at split2_pos and the B-fragment load reads it back from
 // there, so fragment column c of k-tile kt is plain column 16 kt + c of the matrix.
 static void pack_tile(const std::vector<std::vector<uint16_t>> &rows, int K, uint16_t *dst)
 {
@@ -455,9 +455,10 @@ static bool choose_shape(const wrnn_model *m, int CS, ResidentPack *k, std::stri
     k->CS = CS; k->NCTA = best; k->NC = best / CS; k->UC = Hh / best; k->HR = HR; k->LR = LR;
     k->K = Hh; k->NKT = Hh / 16; k->n_rrows = 6 * k->UC;
     k->NMT = (HR + k->n_rrows + 15) / 16; k->NLT = LR / 16;
-    k->NW = 20; k->KSH = 4; k->KSL = 7;
-    if (k->NKT != 28 || k->NMT * k->KSH > k->NW || k->NLT * k->KSL > k->NW || CS > k->NW) {
-        if (why) *why = "only the H/2 = 448 tiling (4 x 7 and 7 x 4 k-tiles) is instantiated";
+    k->NMT += k->NMT & 1;                                   // tiles are multiplied in pairs
+    k->NW = 16; k->KSH = 7; k->KSL = 7;
+    if (k->NKT != 28 || (k->NMT / 2) * k->KSH > k->NW || k->NLT * k->KSL > k->NW || CS > k->NW || k->NMT * k->KSH > 32) {
+        if (why) *why = "only the H/2 = 448 tiling (7 K-splits of 4 k-tiles) is instantiated";
         return false;
     }
     k->w_bytes = ((size_t)2 * k->NMT + 2 * k->NLT) * 16 * k->K * 2;
@@ -468,8 +469,8 @@ static bool choose_shape(const wrnn_model *m, int CS, ResidentPack *k, std::stri
     return true;
 }
 
-// The one instantiated split: K = 448 as 4 x 7 k-tiles (hidden, 5 tiles -> 20 warps) and 7 x 4 (logits, 2 tiles).
-static void *resident_fn() { return (void *)resident_dense_kernel<4, 7, 7, 4>; }
+// The one instantiated split: K = 448 as 7 x 4 k-tiles, for pairs of hidden tiles and for single logits tiles.
+static void *resident_fn() { return (void *)resident_dense_kernel<7, 4, 7, 4>; }
 
 int resident_supported(const wrnn_model *m, int batch, std::string *why)
 {
@@ -637,7 +638,7 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     // a profiler that replays kernels may not accept cooperative cluster launches.
     const char *no_coop = getenv("WRNN_NO_COOP");
     fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
-    cudaError_t e = cudaLaunchKernelEx(&cfg, resident_dense_kernel<4, 7, 7, 4>, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, resident_dense_kernel<7, 4, 7, 4>, p);
     if (e != cudaSuccess) {
         m->err = std::string("resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

@@ -331,3 +331,150 @@ int orc_run(const orc_params *p, const float *cond, int n_frames, int hop,
     }
     return err_any;
 }
+
+/* ====================================================================== */
+/* Fused Subscale WaveRNN 2x (the paper's subsection of that name; batched
+ * sampling and the lag between sub-tensors are in the subsection before it).
+ *
+ * What the paper fixes: a Subscale WaveRNN 2x whose two sub-tensors are not
+ * batched but given one part each of the hidden state of a single WaveRNN;
+ * 8 softmaxes of 4 bits; future horizon F = 2; the sub-tensors' samples are
+ * the network's direct inputs, no conditioning network; 32 bits per step.
+ * Everything else below is a stated reading (parity for it is unpinned
+ * outside this file):
+ *   - sub-tensor 0 holds a_i = u_{2i}, sub-tensor 1 holds b_i = u_{2i+1};
+ *     step t emits a_t from part A of the state (units [0,H/2), the "coarse"
+ *     half of Eq. 2) and then b_{t-2} from part B (units [H/2,H)): part B sees
+ *     a_t inside the step exactly as the fine half sees c_t in Eq. 2, so b_j is
+ *     conditioned on a_{<= j+2}: F = 2;
+ *   - x_t = [nibbles of a_{t-1}, nibbles of the previous step's b, nibbles of
+ *     a_t], most significant nibble first, a nibble v scaled to v/7.5 - 1;
+ *     I* is [3H][12] and its last four columns reach only the rows of part B;
+ *   - each part keeps the head of Eq. 2, softmax(O2 relu(O1 y)), with
+ *     O2 of 64 rows: rows [16k, 16k+16) are the softmax of nibble k, and the four
+ *     nibbles of a sample are drawn independently given the state;
+ *   - sample = sum_k nibble_k << (12 - 4k), emitted as int16 minus 32768;
+ *   - uniforms: the same counter generator with head = 4 * part + k;
+ *   - before the first step a_{-1} = b = 0x8000 and h = 0.
+ * Gate rows, biases, conditioning and the draw are as for the base model.    */
+
+double orc_scale4(int v) { return (double)v / 7.5 - 1.0; }
+void orc_split_nibbles(uint16_t x, uint8_t n[4]) { for (int k = 0; k < 4; ++k) n[k] = (uint8_t)((x >> (12 - 4 * k)) & 15u); }
+uint16_t orc_join_nibbles(const uint8_t n[4]) { return (uint16_t)((n[0] << 12) | (n[1] << 8) | (n[2] << 4) | n[3]); }
+
+/*
+ * One stream, n_steps steps from step0.  p->I is [3H][12], p->O2 / p->O4 are
+ * [64][H/2], p->b2 / p->b4 [64]; the other fields as for orc_run.  a_prev /
+ * b_prev: the two samples emitted by the previous step (in / out).  With
+ * a_forced / b_forced the drawn samples are only recorded and the forced
+ * ones fed back.  out is [2][n_steps] (row 0: a_t, row 1: the b of step t);
+ * margins [n_steps][8]; dbg_gates [n_steps][3H]; dbg_h [n_steps][H];
+ * dbg_logits [n_steps][2][64].  Returns 0, or 1 when a frame index fell
+ * outside [0, n_frames).
+ */
+int orc_fs2_run(const orc_params *p, const float *cond, int n_frames, int hop, int64_t n_steps, int64_t step0,
+                uint64_t seed, uint32_t stream, float *h, uint16_t *a_prev, uint16_t *b_prev,
+                const uint16_t *a_forced, const uint16_t *b_forced, uint16_t *a_out, uint16_t *b_out,
+                int16_t *out, double *margins, float *dbg_gates, float *dbg_h, float *dbg_logits)
+{
+    const int H = p->H, Hh = H / 2, G = 3 * H, D = p->cond_dim;
+    double *a = (double *)malloc(sizeof(double) * (size_t)G);
+    double *g = (double *)malloc(sizeof(double) * (size_t)G);
+    double *gate = (double *)malloc(sizeof(double) * (size_t)G);
+    float *hn = (float *)malloc(sizeof(float) * (size_t)H);
+    double *q = (double *)malloc(sizeof(double) * (size_t)Hh);
+    float logit[64];
+    int64_t g_frame = -1;
+    int err = 0;
+    uint16_t ap = *a_prev, bp = *b_prev;
+
+    for (int64_t s = 0; s < n_steps && !err; ++s) {
+        const int64_t t = step0 + s;
+        int64_t k = (D > 0) ? t / hop : 0;
+        if (D > 0 && (k < 0 || k >= n_frames)) { err = 1; break; }
+        if (k != g_frame) {
+            for (int row = 0; row < G; ++row) {
+                double acc = p->b_gate ? (double)p->b_gate[row] : 0.0;
+                for (int d = 0; d < D; ++d) acc += (double)p->W_cond[(int64_t)row * D + d] * (double)cond[k * D + d];
+                g[row] = acc;
+            }
+            g_frame = k;
+        }
+        double x[12];
+        uint8_t nb[4];
+        orc_split_nibbles(ap, nb); for (int c = 0; c < 4; ++c) x[c] = orc_scale4(nb[c]);
+        orc_split_nibbles(bp, nb); for (int c = 0; c < 4; ++c) x[4 + c] = orc_scale4(nb[c]);
+        for (int c = 8; c < 12; ++c) x[c] = 0.0;
+
+        for (int row = 0; row < G; ++row) {
+            double acc = 0.0;
+            const float *Rr = p->R + (int64_t)row * H;
+            for (int j = 0; j < H; ++j) acc += (double)Rr[j] * (double)h[j];
+            a[row] = acc;
+        }
+
+        uint16_t smp[2] = {0, 0};
+        for (int part = 0; part < 2; ++part) {
+            const int j0 = part ? Hh : 0, j1 = part ? H : Hh;
+            const int ncol = part ? 12 : 8;             /* a_t reaches only part B (masked I*) */
+            for (int j = j0; j < j1; ++j) {
+                const float *Iu = p->I + (int64_t)j * 12;
+                const float *Ir = p->I + (int64_t)(H + j) * 12;
+                const float *Ie = p->I + (int64_t)(2 * H + j) * 12;
+                double pu = a[j] + g[j], pr = a[H + j] + g[H + j], pe_in = g[2 * H + j];
+                for (int c = 0; c < ncol; ++c) { pu += Iu[c] * x[c]; pr += Ir[c] * x[c]; pe_in += Ie[c] * x[c]; }
+                double u = sigmoid_d(pu);
+                double r = sigmoid_d(pr);
+                double e = tanh(r * a[2 * H + j] + pe_in);
+                gate[j] = u; gate[H + j] = r; gate[2 * H + j] = e;
+                hn[j] = (float)(u * (double)h[j] + (1.0 - u) * e);
+            }
+            const float *Oa = part ? p->O3 : p->O1, *ba = part ? p->b3 : p->b1;
+            const float *Ob = part ? p->O4 : p->O2, *bb = part ? p->b4 : p->b2;
+            for (int i = 0; i < Hh; ++i) {
+                double acc = ba ? (double)ba[i] : 0.0;
+                for (int j = 0; j < Hh; ++j) acc += (double)Oa[(int64_t)i * Hh + j] * (double)hn[j0 + j];
+                q[i] = acc > 0.0 ? acc : 0.0;
+            }
+            for (int i = 0; i < 64; ++i) {
+                double acc = bb ? (double)bb[i] : 0.0;
+                for (int j = 0; j < Hh; ++j) acc += (double)Ob[(int64_t)i * Hh + j] * q[j];
+                logit[i] = (float)acc;
+            }
+            uint8_t drawn[4];
+            for (int kk = 0; kk < 4; ++kk) {
+                double uu = orc_uniform(seed, stream, (uint64_t)t, (uint32_t)(4 * part + kk));
+                double margin;
+                drawn[kk] = (uint8_t)orc_softmax_sample(logit + 16 * kk, 16, uu, NULL, &margin);
+                if (margins) margins[8 * s + 4 * part + kk] = margin;
+            }
+            if (dbg_logits) memcpy(dbg_logits + s * 128 + part * 64, logit, sizeof(logit));
+            const uint16_t v = orc_join_nibbles(drawn);
+            if (part == 0) {
+                if (a_out) a_out[s] = v;
+                smp[0] = a_forced ? a_forced[s] : v;
+                orc_split_nibbles(smp[0], nb);
+                for (int c = 0; c < 4; ++c) x[8 + c] = orc_scale4(nb[c]);
+            } else {
+                if (b_out) b_out[s] = v;
+                smp[1] = b_forced ? b_forced[s] : v;
+            }
+        }
+        if (dbg_gates) for (int row = 0; row < G; ++row) dbg_gates[s * G + row] = (float)gate[row];
+        if (dbg_h) memcpy(dbg_h + s * H, hn, sizeof(float) * (size_t)H);
+        memcpy(h, hn, sizeof(float) * (size_t)H);
+        if (out) { out[s] = (int16_t)((int32_t)smp[0] - 32768); out[n_steps + s] = (int16_t)((int32_t)smp[1] - 32768); }
+        ap = smp[0]; bp = smp[1];
+    }
+    *a_prev = ap; *b_prev = bp;
+    free(a); free(g); free(gate); free(hn); free(q);
+    return err;
+}
+
+/* Interleave the two streams of orc_fs2_run into the original order: u_{2i} = a_i, u_{2i+1} = b_i, where b_i is the b
+ * of step i + 2 (the first two b of a run are the lag's pre-roll and are dropped).  n = number of steps; u gets
+ * 2 (n - 2) samples. */
+void orc_fs2_unfold(const int16_t *ab /* [2][n] */, int64_t n, int16_t *u)
+{
+    for (int64_t i = 0; i + 2 < n; ++i) { u[2 * i] = ab[i]; u[2 * i + 1] = ab[n + i + 2]; }
+}

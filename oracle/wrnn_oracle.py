@@ -66,6 +66,15 @@ def lib():
             [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int,
              C.c_int64, C.c_uint64, C.c_uint32] + [C.c_void_p] * 12 + [C.c_int]
         )
+        L.orc_scale4.restype = C.c_double
+        L.orc_scale4.argtypes = [C.c_int]
+        L.orc_split_nibbles.argtypes = [C.c_uint16, C.c_void_p]
+        L.orc_join_nibbles.restype = C.c_uint16
+        L.orc_join_nibbles.argtypes = [C.c_void_p]
+        L.orc_fs2_run.restype = C.c_int
+        L.orc_fs2_run.argtypes = ([C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int64, C.c_int64, C.c_uint64, C.c_uint32]
+                                  + [C.c_void_p] * 12)
+        L.orc_fs2_unfold.argtypes = [C.c_void_p, C.c_int64, C.c_void_p]
         _lib = L
     return _lib
 
@@ -236,3 +245,84 @@ class OracleModel:
         if rc != 0:
             raise ValueError("conditioning frame index out of range")
         return RunResult(out, c_out, f_out, margins, hh, cp, fp, gates, hs, logits)
+
+
+# ----------------------------------------------------------------------------------------------
+# Fused Subscale WaveRNN 2x
+
+def scale4(v: int) -> float:
+    return lib().orc_scale4(int(v))
+
+
+def split_nibbles(x: int):
+    n = (C.c_uint8 * 4)()
+    lib().orc_split_nibbles(int(x), n)
+    return list(n)
+
+
+def join_nibbles(n) -> int:
+    a = (C.c_uint8 * 4)(*[int(v) for v in n])
+    return lib().orc_join_nibbles(a)
+
+
+def fs2_unfold(ab: np.ndarray) -> np.ndarray:
+    ab = np.ascontiguousarray(ab, dtype=np.int16)
+    n = ab.shape[1]
+    u = np.zeros(2 * max(n - 2, 0), dtype=np.int16)
+    lib().orc_fs2_unfold(_ptr(ab), n, _ptr(u))
+    return u
+
+
+@dataclass
+class Fs2Result:
+    out: np.ndarray            # int16 [2][n_steps]: row 0 a_t, row 1 the b of step t
+    a_out: np.ndarray          # uint16 [n_steps] samples the oracle drew
+    b_out: np.ndarray
+    margins: np.ndarray        # float64 [n_steps][8]
+    h: np.ndarray
+    a_prev: int
+    b_prev: int
+    gates: Optional[np.ndarray] = None   # [n_steps][3H]
+    hs: Optional[np.ndarray] = None      # [n_steps][H]
+    logits: Optional[np.ndarray] = None  # [n_steps][2][64]
+
+
+class Fs2OracleModel(OracleModel):
+    """Fused Subscale WaveRNN 2x: the same cell with I of 12 columns and heads of 64 logits (4 softmaxes of 4 bits)."""
+
+    def __init__(self, weights: dict, dtype: str = "f32"):
+        super().__init__(weights, dtype)
+        H = self.H
+        assert self.w["I"].shape == (3 * H, 12) and self.w["O2"].shape == (64, H // 2) and self.w["O4"].shape == (64, H // 2)
+
+    def run(self, cond: Optional[np.ndarray], n_steps: int, seed: int = 0, *, hop: int = 120, step0: int = 0, stream: int = 0,
+            h: Optional[np.ndarray] = None, a_prev: int = 0x8000, b_prev: int = 0x8000,
+            a_forced: Optional[np.ndarray] = None, b_forced: Optional[np.ndarray] = None, dump: bool = False) -> Fs2Result:
+        H = self.H
+        n_frames = 0
+        if self.cond_dim:
+            cond = np.ascontiguousarray(cond, dtype=np.float32).reshape(-1, self.cond_dim)
+            n_frames = cond.shape[0]
+        else:
+            cond = None
+        hh = np.zeros(H, np.float32) if h is None else np.array(h, np.float32, copy=True).reshape(H)
+        ap = np.array([a_prev], np.uint16)
+        bp = np.array([b_prev], np.uint16)
+        if a_forced is not None:
+            a_forced = np.ascontiguousarray(a_forced, np.uint16).reshape(n_steps)
+            b_forced = np.ascontiguousarray(b_forced, np.uint16).reshape(n_steps)
+        out = np.zeros((2, n_steps), np.int16)
+        a_out = np.zeros(n_steps, np.uint16)
+        b_out = np.zeros(n_steps, np.uint16)
+        margins = np.zeros((n_steps, 8), np.float64)
+        gates = hs = logits = None
+        if dump:
+            gates = np.zeros((n_steps, 3 * H), np.float32)
+            hs = np.zeros((n_steps, H), np.float32)
+            logits = np.zeros((n_steps, 2, 64), np.float32)
+        rc = lib().orc_fs2_run(C.byref(self._p), _ptr(cond), n_frames, hop, n_steps, step0, seed, stream, _ptr(hh), _ptr(ap), _ptr(bp),
+                               _ptr(a_forced), _ptr(b_forced), _ptr(a_out), _ptr(b_out), _ptr(out), _ptr(margins),
+                               _ptr(gates), _ptr(hs), _ptr(logits))
+        if rc != 0:
+            raise ValueError("conditioning frame index out of range")
+        return Fs2Result(out, a_out, b_out, margins, hh, int(ap[0]), int(bp[0]), gates, hs, logits)

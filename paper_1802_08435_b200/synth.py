@@ -23,10 +23,12 @@ COND_DIM = 64
 
 
 def make_weights(H: int, cond_dim: int = COND_DIM, seed_w: int = SEED_WEIGHTS,
-                 seed_b: int = SEED_BIASES, head_scale: float = 1.0) -> Dict[str, np.ndarray]:
+                 seed_b: int = SEED_BIASES, head_scale: float = 1.0, n_inputs: int = 3,
+                 n_logits: int = 256) -> Dict[str, np.ndarray]:
     """All matrices i.i.d. N(0, 1/H), biases N(0, 1/H); fp32, row-major.
 
-    head_scale multiplies O2 and O4 (peaky output distributions for range tests).
+    head_scale multiplies O2 and O4 (peaky output distributions for range tests).  n_inputs = 12 and n_logits = 64 give
+    the shapes of the Fused Subscale WaveRNN 2x (twelve nibble inputs, four 16-way softmaxes per head).
     """
     assert H % 8 == 0
     Hh = H // 2
@@ -39,17 +41,17 @@ def make_weights(H: int, cond_dim: int = COND_DIM, seed_w: int = SEED_WEIGHTS,
 
     w = {
         "R": mat(rw, 3 * H, H),
-        "I": mat(rw, 3 * H, 3),
+        "I": mat(rw, 3 * H, n_inputs),
         "W_cond": mat(rw, 3 * H, cond_dim) if cond_dim else None,
         "O1": mat(rw, Hh, Hh),
-        "O2": mat(rw, 256, Hh) * np.float32(head_scale),
+        "O2": mat(rw, n_logits, Hh) * np.float32(head_scale),
         "O3": mat(rw, Hh, Hh),
-        "O4": mat(rw, 256, Hh) * np.float32(head_scale),
+        "O4": mat(rw, n_logits, Hh) * np.float32(head_scale),
         "b_gate": mat(rb, 3 * H),
         "b1": mat(rb, Hh),
-        "b2": mat(rb, 256),
+        "b2": mat(rb, n_logits),
         "b3": mat(rb, Hh),
-        "b4": mat(rb, 256),
+        "b4": mat(rb, n_logits),
     }
     return w
 

@@ -88,6 +88,12 @@ typedef struct {
     int32_t mask_block_cols;    /* 4 x 4, or m x 1 = 16 rows of one column, or 1 x 1 = unstructured); */
                                 /* 0, 0 means 4 x 4.  Both must divide H/2.  Every shape runs on the  */
                                 /* generic kernel; 4 x 4 and 16 x 1 also on the single-cluster kernel */
+    int32_t variant;            /* 0: WaveRNN (Eq. 2, shapes as above).  1: Fused Subscale WaveRNN 2x */
+                                /* (Section 4.4): I is [3H][12] (nibbles of a_{t-1}, of the previous  */
+                                /* b, of a_t; the last four columns are ignored on part-A rows),      */
+                                /* O2 / O4 are [64][H/2] and b2 / b4 [64]: rows 16 k .. 16 k + 15 are  */
+                                /* the softmax of nibble k.  Dense bf16, one stream, the resident     */
+                                /* kernel only; stepped with the wrnn_fs2_* calls below               */
 } wrnn_params;
 
 /*
@@ -219,6 +225,41 @@ const char *wrnn_last_error(wrnn_model *m);
  * rows, bytes of packed weights read per step, dynamic shared memory per CTA. */
 int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_ctas,
                      int32_t *n_threads, int64_t *weight_bytes_per_step, int32_t *smem_bytes);
+
+/*
+ * Fused Subscale WaveRNN 2x (Section 4.4: a Subscale WaveRNN 2x whose two sub-tensors each get one part of the hidden
+ * state of a single WaveRNN; 8 softmaxes of 4 bits, future horizon F = 2, the generated samples are the direct inputs;
+ * 32 bits per step).  Reading used here: sub-tensor 0 holds a_i = u_{2i}, sub-tensor 1 holds b_i = u_{2i+1}; step t
+ * emits a_t from part A (units [0, H/2)) and then b_{t-2} from part B (units [H/2, H)), which sees a_t inside the step
+ * as the fine half sees c_t in Eq. 2; a 16-bit sample is four nibbles, most significant first, each drawn from its own
+ * 16-way softmax over 16 consecutive logits of the part's head, and fed back scaled to v / 7.5 - 1.  Uniforms: the
+ * same Philox keying with head = 4 * part + nibble.  Models are created by wrnn_create with variant = 1; batch is 1.
+ *
+ * State: DEVICE pointers as for wrnn_state; a_prev / b_prev hold the two samples of the previous step as unsigned
+ * 16-bit values (NULL = 0x8000).  cond: as for wrnn_sample with batch 1 (frame index (step0 + s) * row_stride / hop).
+ * wrnn_fs2_sample writes DEVICE out[2][n_steps] int16 (value - 32768): row 0 = a_t, row 1 = the sample part B emitted in
+ * step t (= b_{t-2}).  wrnn_fs2_step_teacher_forced records the drawn samples in a_out / b_out (DEVICE [n_steps] or
+ * NULL) and feeds a_forced / b_forced back instead; dumps as for wrnn_step_teacher_forced with logits [n_steps][2][64].
+ * wrnn_fs2_unfold interleaves the two rows into the original order, dropping the two pre-roll samples of row 1:
+ * u[2 i] = ab[0][i], u[2 i + 1] = ab[1][i + 2] for i < n_steps - 2 (DEVICE u of 2 (n_steps - 2) samples).
+ * All asynchronous on cuda_stream; errors as for the calls above; WRNN_ERR_UNSUPPORTED for a model of the other variant.
+ */
+typedef struct {
+    float *h;            /* [H] */
+    uint16_t *a_prev;    /* [1] */
+    uint16_t *b_prev;    /* [1] */
+    int64_t step0;
+    uint32_t stream0;
+    uint32_t reserved;
+} wrnn_fs2_state;
+
+int wrnn_fs2_sample(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, uint64_t seed, const wrnn_fs2_state *st,
+                    int16_t *out, void *cuda_stream);
+int wrnn_fs2_step_teacher_forced(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, uint64_t seed,
+                                 const wrnn_fs2_state *st, const uint16_t *a_forced, const uint16_t *b_forced,
+                                 uint16_t *a_out, uint16_t *b_out, float *dbg_gates, float *dbg_h, float *dbg_logits,
+                                 void *cuda_stream);
+int wrnn_fs2_unfold(const int16_t *ab, int64_t n_steps, int16_t *u, void *cuda_stream);
 
 /* Diagnostic of the resident single-stream kernel (Section 2.1: after the persistent kernel the
  * remaining overhead is the synchronisation between multiprocessors): SM-clock cycles that warp 0 of

@@ -26,7 +26,7 @@ EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
     "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor", "wrnn_sample_noalloc",
-    "wrnn_selftest_bounded_wait",
+    "wrnn_selftest_bounded_wait", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold",
 ]
 
 
@@ -41,12 +41,18 @@ class wrnn_params(C.Structure):
         [("H", C.c_int32), ("cond_dim", C.c_int32)]
         + [(n, C.c_void_p) for n in ("R", "I", "b_gate", "W_cond", "O1", "b1", "O2", "b2", "O3", "b3", "O4", "b4",
                                      "mask_R", "mask_O1", "mask_O3")]
-        + [("dtype", C.c_int32), ("kernel", C.c_int32), ("mask_block_rows", C.c_int32), ("mask_block_cols", C.c_int32)]
+        + [("dtype", C.c_int32), ("kernel", C.c_int32), ("mask_block_rows", C.c_int32), ("mask_block_cols", C.c_int32),
+           ("variant", C.c_int32)]
     )
 
 
 class wrnn_state(C.Structure):
     _fields_ = [("h", C.c_void_p), ("c_prev", C.c_void_p), ("f_prev", C.c_void_p), ("step0", C.c_int64),
+                ("stream0", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class wrnn_fs2_state(C.Structure):
+    _fields_ = [("h", C.c_void_p), ("a_prev", C.c_void_p), ("b_prev", C.c_void_p), ("step0", C.c_int64),
                 ("stream0", C.c_uint32), ("reserved", C.c_uint32)]
 
 
@@ -74,6 +80,9 @@ def lib():
         L.wrnn_sample.argtypes = [vp, C.POINTER(wrnn_cond), i64, i32, u64, C.POINTER(wrnn_state), vp, vp]
         L.wrnn_sample_noalloc.argtypes = [vp, C.POINTER(wrnn_cond), i64, i32, u64, C.POINTER(wrnn_state), vp, vp]
         L.wrnn_step_teacher_forced.argtypes = [vp, C.POINTER(wrnn_cond), i64, i32, u64, C.POINTER(wrnn_state)] + [vp] * 8
+        L.wrnn_fs2_sample.argtypes = [vp, C.POINTER(wrnn_cond), i64, u64, C.POINTER(wrnn_fs2_state), vp, vp]
+        L.wrnn_fs2_step_teacher_forced.argtypes = [vp, C.POINTER(wrnn_cond), i64, u64, C.POINTER(wrnn_fs2_state)] + [vp] * 8
+        L.wrnn_fs2_unfold.argtypes = [vp, i64, vp, vp]
         L.wrnn_fold.argtypes = [vp, i64, i32, vp, vp]
         L.wrnn_unfold.argtypes = [vp, i64, i32, vp, vp]
         L.wrnn_sample_subscale.argtypes = [vp, vp, i32, i32, i64, i32, u64, vp, vp]
@@ -122,9 +131,10 @@ def wrnn_last_error(model=None) -> str:
 
 
 def wrnn_create(weights: Dict[str, np.ndarray], dtype: str = "f32", masks: Optional[Dict[str, np.ndarray]] = None,
-                max_batch: int = 1, kernel: int = WRNN_KERNEL_AUTO, block=(4, 4)):
+                max_batch: int = 1, kernel: int = WRNN_KERNEL_AUTO, block=(4, 4), variant: int = 0):
     """weights: fp32 numpy arrays R [3H][H], I [3H][3], W_cond [3H][D] or None, O1..O4, b_gate, b1..b4 (or None);
     masks: optional block masks {"R": [3H/br][H/bc], "O1": [H/2/br][H/2/bc], "O3": ...} with block = (br, bc).
+    variant = 1: Fused Subscale WaveRNN 2x (I [3H][12], O2 / O4 [64][H/2], b2 / b4 [64]).
     Returns an opaque handle."""
     keep = {}
 
@@ -154,6 +164,7 @@ def wrnn_create(weights: Dict[str, np.ndarray], dtype: str = "f32", masks: Optio
     p.dtype = {"f32": WRNN_F32, "bf16": WRNN_BF16}[dtype]
     p.kernel = kernel
     p.mask_block_rows, p.mask_block_cols = int(block[0]), int(block[1])
+    p.variant = int(variant)
     out = C.c_void_p()
     _check(lib().wrnn_create(C.byref(p), max_batch, C.byref(out)))
     return out
@@ -200,6 +211,34 @@ def wrnn_fold(x, B: int, sub, stream=None):
 
 def wrnn_unfold(sub, B: int, x, stream=None):
     _check(lib().wrnn_unfold(_dev_ptr(sub), sub.numel(), B, _dev_ptr(x), _stream_ptr(stream)))
+
+
+def _mk_fs2_state(h, a_prev, b_prev, step0, stream0):
+    if h is None and a_prev is None and b_prev is None and step0 == 0 and stream0 == 0:
+        return None
+    return C.byref(wrnn_fs2_state(_dev_ptr(h), _dev_ptr(a_prev), _dev_ptr(b_prev), step0, stream0, 0))
+
+
+def wrnn_fs2_sample(model, cond, n_steps: int, seed: int, out, *, hop: int = 120, h=None, a_prev=None, b_prev=None,
+                    step0: int = 0, stream0: int = 0, stream=None):
+    """Fused Subscale WaveRNN 2x.  cond: CUDA float32 [1][n_frames][cond_dim] or None; out: CUDA int16 [2][n_steps]
+    (row 0: a_t, row 1: the sample part B emitted in step t); a_prev / b_prev: CUDA uint16 [1] carry state."""
+    _check(lib().wrnn_fs2_sample(model, _mk_cond(cond, hop, 1, 0), n_steps, seed, _mk_fs2_state(h, a_prev, b_prev, step0, stream0),
+                                 _dev_ptr(out), _stream_ptr(stream)), model)
+
+
+def wrnn_fs2_step_teacher_forced(model, cond, n_steps: int, seed: int, a_forced, b_forced, a_out, b_out, *, dbg_gates=None,
+                                 dbg_h=None, dbg_logits=None, hop: int = 120, h=None, a_prev=None, b_prev=None,
+                                 step0: int = 0, stream0: int = 0, stream=None):
+    _check(lib().wrnn_fs2_step_teacher_forced(
+        model, _mk_cond(cond, hop, 1, 0), n_steps, seed, _mk_fs2_state(h, a_prev, b_prev, step0, stream0),
+        _dev_ptr(a_forced), _dev_ptr(b_forced), _dev_ptr(a_out), _dev_ptr(b_out), _dev_ptr(dbg_gates), _dev_ptr(dbg_h),
+        _dev_ptr(dbg_logits), _stream_ptr(stream)), model)
+
+
+def wrnn_fs2_unfold(ab, n_steps: int, u, stream=None):
+    """ab: CUDA int16 [2][n_steps] from wrnn_fs2_sample; u: CUDA int16 [2 (n_steps - 2)]."""
+    _check(lib().wrnn_fs2_unfold(_dev_ptr(ab), n_steps, _dev_ptr(u), _stream_ptr(stream)))
 
 
 def wrnn_sample_subscale(model, cond, n_total: int, B: int, seed: int, out, *, hop: int = 120, stream=None):

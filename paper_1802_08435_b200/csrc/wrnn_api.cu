@@ -146,10 +146,13 @@ static bool use_batched(const wrnn_model *m, int batch)
 
 // Common argument checks of the stepping calls; fills the parts of StepArgs that come from
 // cond / st.  Returns WRNN_OK or an error (message in m->err).
-int check_step(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, const wrnn_state *st,
-               StepArgs *a)
+static int check_step_any(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, const wrnn_state *st,
+                          StepArgs *a, bool fused_call)
 {
     if (!m) return WRNN_ERR_INVALID_ARG;
+    if ((m->variant == 1) != fused_call)
+        return fail(m, WRNN_ERR_UNSUPPORTED, fused_call ? "not a fused subscale model (create with variant = 1)"
+                                                        : "a fused subscale model is stepped with the wrnn_fs2_* calls");
     if (n_steps < 0 || batch < 1) return fail(m, WRNN_ERR_INVALID_ARG, "n_steps < 0 or batch < 1");
     if (batch > m->max_batch) return fail(m, WRNN_ERR_INVALID_ARG, "batch exceeds max_batch given at create");
     if (n_steps > (1ll << 31) - 2) return fail(m, WRNN_ERR_INVALID_ARG, "n_steps too large for one call");
@@ -178,6 +181,11 @@ int check_step(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t ba
         a->n_frames = 1; a->hop = 1;
     }
     return WRNN_OK;
+}
+
+int check_step(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, const wrnn_state *st, StepArgs *a)
+{
+    return check_step_any(m, cond, n_steps, batch, st, a, false);
 }
 
 static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
@@ -235,6 +243,12 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
     if ((p->cond_dim > 0) != (p->W_cond != nullptr)) return fail(nullptr, WRNN_ERR_INVALID_ARG, "W_cond must be given iff cond_dim > 0");
     if (p->dtype != WRNN_F32 && p->dtype != WRNN_BF16) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown dtype");
     if (p->kernel < WRNN_KERNEL_AUTO || p->kernel > WRNN_KERNEL_BCLUSTER) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown kernel family");
+    if (p->variant != 0 && p->variant != 1) return fail(nullptr, WRNN_ERR_INVALID_ARG, "unknown model variant");
+    const bool fused = p->variant == 1;
+    if (fused && (p->dtype != WRNN_BF16 || p->mask_R || p->mask_O1 || p->mask_O3 || max_batch != 1 ||
+                  (p->kernel != WRNN_KERNEL_AUTO && p->kernel != WRNN_KERNEL_RESIDENT)))
+        return fail(nullptr, WRNN_ERR_UNSUPPORTED, "the fused subscale variant runs dense, bf16, one stream, on the resident kernel");
+    const int n_in = fused ? 12 : 3, n_logits = fused ? 64 : 256;
     const int mbr = p->mask_block_rows ? p->mask_block_rows : 4, mbc = p->mask_block_cols ? p->mask_block_cols : 4;
     if ((p->mask_block_rows == 0) != (p->mask_block_cols == 0) || mbr < 1 || mbc < 1 || (H / 2) % mbr != 0 || (H / 2) % mbc != 0)
         return fail(nullptr, WRNN_ERR_INVALID_ARG, "mask block shape must divide H/2 (0, 0 = 4 x 4)");
@@ -248,6 +262,7 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
     wrnn_model *m = new (std::nothrow) wrnn_model();
     if (!m) return fail(nullptr, WRNN_ERR_NOMEM, "host allocation failed");
     m->H = H; m->cond_dim = p->cond_dim; m->dtype = p->dtype; m->kernel = p->kernel; m->max_batch = max_batch;
+    m->variant = p->variant;
     m->device = dev; m->n_sms = prop.multiProcessorCount;
     m->sparse = p->mask_R || p->mask_O1 || p->mask_O3;
     m->mask_br = mbr; m->mask_bc = mbc;
@@ -256,20 +271,20 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
 
     build_bsr(p->R, G, H, p->mask_R, mbr, mbc, bf, &m->hR);
     build_bsr(p->O1, Hh, Hh, p->mask_O1, mbr, mbc, bf, &m->hO1);
-    build_bsr(p->O2, 256, Hh, nullptr, 4, 4, bf, &m->hO2);
+    build_bsr(p->O2, n_logits, Hh, nullptr, 4, 4, bf, &m->hO2);
     build_bsr(p->O3, Hh, Hh, p->mask_O3, mbr, mbc, bf, &m->hO3);
-    build_bsr(p->O4, 256, Hh, nullptr, 4, 4, bf, &m->hO4);
-    m->hI.resize((size_t)G * 3);
+    build_bsr(p->O4, n_logits, Hh, nullptr, 4, 4, bf, &m->hO4);
+    m->hI.resize((size_t)G * n_in);
     for (int row = 0; row < G; ++row)
-        for (int c = 0; c < 3; ++c) {
-            float v = p->I[(size_t)row * 3 + c];
-            if (c == 2 && (row % H) < Hh) v = 0.f;          // c_t reaches only the fine half (I*)
-            m->hI[(size_t)row * 3 + c] = bf ? round_bf16(v) : v;
+        for (int c = 0; c < n_in; ++c) {
+            float v = p->I[(size_t)row * n_in + c];
+            if (c >= 2 * (n_in / 3) && (row % H) < Hh) v = 0.f;   // c_t (a_t) reaches only the fine half (part B): I*
+            m->hI[(size_t)row * n_in + c] = bf ? round_bf16(v) : v;
         }
     auto copy_bias = [](const float *b, int n, std::vector<float> *dst) { dst->assign(n, 0.f); if (b) std::memcpy(dst->data(), b, n * sizeof(float)); };
     copy_bias(p->b_gate, G, &m->hb_gate);
-    copy_bias(p->b1, Hh, &m->hb1); copy_bias(p->b2, 256, &m->hb2);
-    copy_bias(p->b3, Hh, &m->hb3); copy_bias(p->b4, 256, &m->hb4);
+    copy_bias(p->b1, Hh, &m->hb1); copy_bias(p->b2, n_logits, &m->hb2);
+    copy_bias(p->b3, Hh, &m->hb3); copy_bias(p->b4, n_logits, &m->hb4);
     std::vector<float> WcT((size_t)p->cond_dim * G);
     for (int row = 0; row < G; ++row)
         for (int d = 0; d < p->cond_dim; ++d) {
@@ -280,8 +295,8 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
     bool ok = upload_bsr(m->hR, bf, &m->R) && upload_bsr(m->hO1, bf, &m->O1) && upload_bsr(m->hO2, bf, &m->O2) &&
               upload_bsr(m->hO3, bf, &m->O3) && upload_bsr(m->hO4, bf, &m->O4) &&
               upload(&m->I, m->hI.data(), m->hI.size() * 4) && upload(&m->b_gate, m->hb_gate.data(), G * 4) &&
-              upload(&m->b1, m->hb1.data(), Hh * 4) && upload(&m->b2, m->hb2.data(), 256 * 4) &&
-              upload(&m->b3, m->hb3.data(), Hh * 4) && upload(&m->b4, m->hb4.data(), 256 * 4) &&
+              upload(&m->b1, m->hb1.data(), Hh * 4) && upload(&m->b2, m->hb2.data(), n_logits * 4) &&
+              upload(&m->b3, m->hb3.data(), Hh * 4) && upload(&m->b4, m->hb4.data(), n_logits * 4) &&
               upload(&m->W_condT, WcT.data(), WcT.size() * 4);
     const size_t B = (size_t)max_batch;
     ok = ok && cudaMalloc((void **)&m->hbuf[0], B * H * 4) == cudaSuccess &&
@@ -303,6 +318,17 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
     m->weight_bytes = bsr_bytes(m->hR) + bsr_bytes(m->hO1) + bsr_bytes(m->hO2) + bsr_bytes(m->hO3) + bsr_bytes(m->hO4) +
                       (int64_t)G * 3 * 4;
 
+    if (fused) {
+        // one kernel serves this variant; without it the model cannot be stepped
+        const int rc = resident_prepare(m);
+        if (rc != WRNN_OK) {
+            const std::string why = m->err;
+            wrnn_destroy(m);
+            return fail(nullptr, rc, "resident kernel unavailable: " + why);
+        }
+        *out = m;
+        return WRNN_OK;
+    }
     if (p->kernel == WRNN_KERNEL_AUTO || p->kernel == WRNN_KERNEL_SPARSE) {
         const int rc = sparse_prepare(m);
         if (rc != WRNN_OK && p->kernel == WRNN_KERNEL_SPARSE) {
@@ -381,6 +407,57 @@ int wrnn_step_teacher_forced(wrnn_model *m, const wrnn_cond *cond, int64_t n_ste
     a.c_forced = c_forced; a.f_forced = f_forced; a.c_out = c_out; a.f_out = f_out;
     a.dbg_gates = dbg_gates; a.dbg_h = dbg_h; a.dbg_logits = dbg_logits;
     return run_steps(m, a, (cudaStream_t)cuda_stream);
+}
+
+// Fused Subscale WaveRNN 2x: the same checks and launch path with the 16-bit state of the two parts.
+static int fs2_args(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, const wrnn_fs2_state *st, StepArgs *a)
+{
+    int rc = check_step_any(m, cond, n_steps, 1, nullptr, a, true);
+    if (rc != WRNN_OK) return rc;
+    if (st) {
+        if (st->step0 < 0) return fail(m, WRNN_ERR_INVALID_ARG, "step0 < 0");
+        a->step0 = st->step0; a->stream0 = st->stream0;
+        a->h_in = st->h; a->h_out = st->h;
+        a->a_in = st->a_prev; a->a_st_out = st->a_prev;
+        a->b_in = st->b_prev; a->b_st_out = st->b_prev;
+        if (m->cond_dim > 0 && n_steps > 0) {
+            const long long last = ((a->step0 + n_steps - 1) * (long long)a->row_stride + (long long)a->stream0 * a->row_offset_mul) / a->hop;
+            if (last >= a->n_frames) return fail(m, WRNN_ERR_INVALID_ARG, "conditioning frames run out before n_steps");
+        }
+    }
+    return WRNN_OK;
+}
+
+int wrnn_fs2_sample(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, uint64_t seed, const wrnn_fs2_state *st,
+                    int16_t *out, void *cuda_stream)
+{
+    StepArgs a;
+    int rc = fs2_args(m, cond, n_steps, st, &a);
+    if (rc != WRNN_OK) return rc;
+    if (!out && n_steps > 0) return fail(m, WRNN_ERR_INVALID_ARG, "out is NULL");
+    a.seed = seed; a.out = out;
+    return run_steps(m, a, (cudaStream_t)cuda_stream);
+}
+
+int wrnn_fs2_step_teacher_forced(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, uint64_t seed,
+                                 const wrnn_fs2_state *st, const uint16_t *a_forced, const uint16_t *b_forced,
+                                 uint16_t *a_out, uint16_t *b_out, float *dbg_gates, float *dbg_h, float *dbg_logits,
+                                 void *cuda_stream)
+{
+    StepArgs a;
+    int rc = fs2_args(m, cond, n_steps, st, &a);
+    if (rc != WRNN_OK) return rc;
+    if ((!a_forced || !b_forced) && n_steps > 0) return fail(m, WRNN_ERR_INVALID_ARG, "forced sample arrays are NULL");
+    a.seed = seed;
+    a.a_forced = a_forced; a.b_forced = b_forced; a.a_out = a_out; a.b_out = b_out;
+    a.dbg_gates = dbg_gates; a.dbg_h = dbg_h; a.dbg_logits = dbg_logits;
+    return run_steps(m, a, (cudaStream_t)cuda_stream);
+}
+
+int wrnn_fs2_unfold(const int16_t *ab, int64_t n_steps, int16_t *u, void *cuda_stream)
+{
+    if (n_steps < 0 || (n_steps > 2 && (!ab || !u))) return WRNN_ERR_INVALID_ARG;
+    return fs2_unfold_launch(ab, n_steps, u, (cudaStream_t)cuda_stream);
 }
 
 int wrnn_fold(const int16_t *x, int64_t n_total, int32_t B, int16_t *sub, void *cuda_stream)

@@ -157,6 +157,33 @@ __device__ __forceinline__ int warp_softmax_draw_fast(const float (&l)[8], float
     return pick == 256 ? 255 : pick;
 }
 
+// Four softmaxes of 16 in one warp (the 4-bit heads of the Fused Subscale WaveRNN 2x): lane l holds logits 2 l, 2 l + 1 of
+// 64, lanes [8 k, 8 k + 8) form softmax k and share the uniform u.  Returns, on every lane, the index its group drew
+// (same rule as warp_softmax_draw: smallest k whose running sum exceeds u * total, 15 if none).
+__device__ __forceinline__ int group16_softmax_draw(float l0, float l1, float u, int lane)
+{
+    float m = fmaxf(l0, l1);
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) m = fmaxf(m, __shfl_xor_sync(FULL, m, o));
+    const float w0 = __expf(l0 - m), w1 = __expf(l1 - m);
+    const float s = w0 + w1;
+    float inc = s;
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) {
+        const float t = __shfl_up_sync(FULL, inc, o, 8);
+        if ((lane & 7) >= o) inc += t;
+    }
+    const float thr = u * __shfl_sync(FULL, inc, 7, 8);
+    const float run = inc - s;           // exclusive prefix of this lane inside its group
+    int pick = 16;
+    if (inc > thr) pick = 2 * (lane & 7) + 1;
+    if (run + w0 > thr) pick = 2 * (lane & 7);
+#pragma unroll
+    for (int o = 1; o < 8; o <<= 1) pick = min(pick, __shfl_xor_sync(FULL, pick, o));
+    return pick == 16 ? 15 : pick;
+}
+__device__ __forceinline__ float scale4(int v) { return (float)v * (1.0f / 7.5f) - 1.0f; }
+
 // sigmoid / tanh through ex2.approx and the fast reciprocal: absolute error about 1e-7 .. 3e-7.
 __device__ __forceinline__ float sigmoidf_fast(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
 __device__ __forceinline__ float tanhf_fast(float x)

@@ -307,6 +307,24 @@ int fold_launch(const int16_t *x, long long n_total, int B, int16_t *sub, bool u
     return cudaGetLastError() == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
 }
 
+// The two streams of the fused subscale variant back in the original order: u[2 i] = a_i, u[2 i + 1] = the sample part B
+// emitted two steps later (Section 4.4 with F = 2).
+__global__ void fs2_unfold_kernel(const int16_t *__restrict__ ab, long long n, int16_t *__restrict__ u)
+{
+    for (long long o = blockIdx.x * (long long)blockDim.x + threadIdx.x; o < 2 * (n - 2); o += (long long)gridDim.x * blockDim.x)
+        u[o] = (o & 1) ? ab[n + (o >> 1) + 2] : ab[o >> 1];
+}
+
+int fs2_unfold_launch(const int16_t *ab, long long n, int16_t *u, cudaStream_t s)
+{
+    if (n <= 2) return WRNN_OK;
+    const long long tot = 2 * (n - 2);
+    const int blocks = (int)((tot + 255) / 256 > 1184 ? 1184 : (tot + 255) / 256);
+    fs2_unfold_kernel<<<blocks, 256, 0, s>>>(ab, n, u);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
+}
+
 // ---------------------------------------------------------------------------------------------
 
 static void *generic_kernel_ptr(int dtype, int tb)

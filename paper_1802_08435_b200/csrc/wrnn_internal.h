@@ -47,6 +47,10 @@ struct StepArgs {
     uint8_t *c_out, *f_out;                      // [batch][n_steps] or null
     int16_t *out;                                // [batch][n_steps] or null
     float *dbg_gates, *dbg_h, *dbg_logits;       // or null
+    // fused subscale variant: 16-bit samples of parts A and B in place of the bytes above (batch 1)
+    const uint16_t *a_in, *b_in; uint16_t *a_st_out, *b_st_out;
+    const uint16_t *a_forced, *b_forced;         // [n_steps] or null
+    uint16_t *a_out, *b_out;                     // [n_steps] or null
 };
 
 struct ResidentPack;   // packed weights of the shared-memory-resident kernels (opaque here)
@@ -59,6 +63,7 @@ struct BcPack;         // per-CTA weight slices and stacked activation images of
 
 struct wrnn_model {
     int H = 0, cond_dim = 0, dtype = 0, kernel = 0, max_batch = 0;
+    int variant = 0;                // 0: WaveRNN (Eq. 2); 1: Fused Subscale WaveRNN 2x (I has 12 columns, O2 / O4 64 rows)
     int device = 0, n_sms = 0;
     bool sparse = false;
     int mask_br = 4, mask_bc = 4;   // shape of one block of the sparsity masks (Section 3.2)
@@ -109,6 +114,7 @@ int generic_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_thre
 int generic_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);   // returns wrnn_status
 int cond_project(wrnn_model *m, const float *cond, int batch, int n_frames, cudaStream_t s);
 int fold_launch(const int16_t *x, long long n_total, int B, int16_t *sub, bool unfold, cudaStream_t s);
+int fs2_unfold_launch(const int16_t *ab, long long n, int16_t *u, cudaStream_t s);
 
 // wrnn_resident.cu
 int resident_supported(const wrnn_model *m, int batch, std::string *why);

@@ -37,6 +37,7 @@ namespace wrnn {
 struct ResidentPack {
     int NC = 0, CS = 0, NCTA = 0, UC = 0, HR = 0, LR = 0, K = 0, NKT = 0, NMT = 0, NLT = 0, NW = 0, KSH = 0, KSL = 0;
     int n_rrows = 0;                 // 6 UC
+    bool fused = false;              // Fused Subscale WaveRNN 2x: 12 input columns, 64 logits per head
     size_t blob_bytes = 0;           // per CTA: bf16 weight fragments then fp32 small parameters
     size_t w_bytes = 0;              // bf16 part of the blob
     uint8_t *d_blob = nullptr;       // [NCTA][blob_bytes]
@@ -60,6 +61,10 @@ struct ResidentParams {
     const uint8_t *c_forced, *f_forced;
     uint8_t *c_out, *f_out;
     int16_t *out;
+    // the fused variant's 16-bit counterparts of the byte arrays above (part A = the coarse half, part B = the fine half)
+    const uint16_t *a_in, *b_in; uint16_t *a_st_out, *b_st_out;
+    const uint16_t *a_forced, *b_forced;
+    uint16_t *a_out, *b_out;
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
@@ -67,7 +72,11 @@ struct ResidentParams {
 };
 
 // KSH / KSL: K-splits per hidden / logits tile; NKH / NKL: k-tiles per split (KSH * NKH = KSL * NKL = K / 16).
-template <int KSH, int NKH, int KSL, int NKL>
+// FUSED: the Fused Subscale WaveRNN 2x.  The same cell and schedule; the coarse half of the state is part A (sub-tensor
+// 0), the fine half part B (sub-tensor 1, which sees the sample of part A inside the step: future horizon 2); each head
+// has 64 logits = four softmaxes of 4 bits, every input is a group of four nibbles instead of one byte, and the
+// symbols (c, f) below are the 16-bit samples (a, b).
+template <int KSH, int NKH, int KSL, int NKL, bool FUSED>
 __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -77,6 +86,8 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int K = p.K, NKT = p.NKT, NMT = p.NMT, NLT = p.NLT, UC = p.UC, HR = p.HR, LR = p.LR, CS = p.CS, H = p.H;
     const int NR = p.n_rrows;                          // 6 UC
+    constexpr int NP = FUSED ? 4 : 1;                  // scalars per symbol: four nibbles, or one byte
+    constexpr int NIN = 3 * NP;                        // columns of I*: previous c, previous f, this step's c
 
     // ---- shared memory carve-up (must match resident_smem_bytes)
     const size_t tile_u4 = (size_t)NKT * 32;                                   // uint4 per 16-row tile
@@ -84,8 +95,8 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
     const uint4 *wMB = wMA + (size_t)NMT * tile_u4;                            // [NMT] tiles: rows [O3 ; R x fine cols]
     const uint4 *wO2 = wMB + (size_t)NMT * tile_u4;                            // [NLT] tiles
     const uint4 *wO4 = wO2 + (size_t)NLT * tile_u4;
-    const float *sI = reinterpret_cast<const float *>(smem + p.w_bytes);       // [NR][3]
-    const float *sb1 = sI + NR * 3, *sb3 = sb1 + HR, *sb2 = sb3 + HR, *sb4 = sb2 + LR;
+    const float *sI = reinterpret_cast<const float *>(smem + p.w_bytes);       // [NR][NIN]
+    const float *sb1 = sI + NR * NIN, *sb3 = sb1 + HR, *sb2 = sb3 + HR, *sb4 = sb2 + LR;
     float *vecC = reinterpret_cast<float *>(smem + p.blob_bytes);              // [K] y_c (fp32, natural order)
     float *vecF = vecC + K;                                                    // [K] y_f
     float *a_part = vecF + K;                                                  // [NR] R[:, :Hh] y_c
@@ -129,7 +140,11 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
     const int g4 = lane >> 2;
 
     // warp 0 keeps the stream's scalar state
-    int c_prev = p.c_in ? p.c_in[0] : 128, f_prev = p.f_in ? p.f_in[0] : 0;
+    int c_prev, f_prev;
+    if (FUSED) { c_prev = p.a_in ? p.a_in[0] : 0x8000; f_prev = p.b_in ? p.b_in[0] : 0x8000; }
+    else { c_prev = p.c_in ? p.c_in[0] : 128; f_prev = p.f_in ? p.f_in[0] : 0; }
+    // scalar k of a symbol as the network sees it
+    auto xin = [](int v, int k) { return FUSED ? scale4((v >> (12 - 4 * k)) & 15) : scale8(v); };
     float hC = 0.f, hF = 0.f;
     if (warp == 0 && lane < UC) { hC = vecC[cta * UC + lane]; hF = vecF[cta * UC + lane]; }
 
@@ -183,26 +198,46 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
     // half_g = 0: coarse units (c_s does not reach them: their I* column is zero), 1: fine units.
     // The gate pre-activations up to the one input that is only known after the draw (c_s for the fine units, f_{s-1} for
     // the coarse units of the next step): computed while the logits are still on their way.
-    struct GatePre { float pu, pr, pe, ae, ku, kr, ke; };
+    struct GatePre { float pu, pr, pe, ae, ku[NP], kr[NP], ke[NP]; };
     auto gates_prepare = [&](int half_g, const float (&gv)[3]) {
         GatePre q;
         const int rb = half_g ? 3 * UC : 0;
-        const float x0 = scale8(c_prev), x1 = scale8(f_prev);
-        const float *Iu = sI + 3 * (rb + lane), *Ir = sI + 3 * (rb + UC + lane), *Ie = sI + 3 * (rb + 2 * UC + lane);
-        // fine units: inputs (c_{s-1}, f_{s-1}) known, c_s pending (column 2); coarse units: c_{s-1} known, f_{s-1} pending (column 1)
-        q.pu = a_full[rb + lane] + fmaf(Iu[0], x0, half_g ? fmaf(Iu[1], x1, gv[0]) : gv[0]);
-        q.pr = a_full[rb + UC + lane] + fmaf(Ir[0], x0, half_g ? fmaf(Ir[1], x1, gv[1]) : gv[1]);
-        q.pe = fmaf(Ie[0], x0, half_g ? fmaf(Ie[1], x1, gv[2]) : gv[2]);
+        const float *Iu = sI + NIN * (rb + lane), *Ir = sI + NIN * (rb + UC + lane), *Ie = sI + NIN * (rb + 2 * UC + lane);
+        // fine units: inputs (c_{s-1}, f_{s-1}) known, c_s pending (last column group); coarse units: c_{s-1} known,
+        // f_{s-1} pending (middle column group)
+        float su = gv[0], sr = gv[1], se = gv[2];
+#pragma unroll
+        for (int k = 0; k < NP; ++k) {
+            const float x = xin(c_prev, k);
+            su = fmaf(Iu[k], x, su); sr = fmaf(Ir[k], x, sr); se = fmaf(Ie[k], x, se);
+        }
+        if (half_g) {
+#pragma unroll
+            for (int k = 0; k < NP; ++k) {
+                const float x = xin(f_prev, k);
+                su = fmaf(Iu[NP + k], x, su); sr = fmaf(Ir[NP + k], x, sr); se = fmaf(Ie[NP + k], x, se);
+            }
+        }
+        q.pu = a_full[rb + lane] + su;
+        q.pr = a_full[rb + UC + lane] + sr;
+        q.pe = se;
         q.ae = a_full[rb + 2 * UC + lane];
-        q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
+        const int pend = half_g ? 2 * NP : NP;
+#pragma unroll
+        for (int k = 0; k < NP; ++k) { q.ku[k] = Iu[pend + k]; q.kr[k] = Ir[pend + k]; q.ke[k] = Ie[pend + k]; }
         return q;
     };
     // Gates of Eq. 2 for this CTA's units of one half of the state, then publish them to the chip.
     // half_g = 0: coarse units (c_s does not reach them: their I* column is zero), 1: fine units.
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
-        const float xk = scale8(drawn);                  // the pending input
-        const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
-        const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
+        float pu = q.pu, pr = q.pr, pe = q.pe;
+#pragma unroll
+        for (int k = 0; k < NP; ++k) {
+            const float xk = xin(drawn, k);              // the pending input
+            pu = fmaf(q.ku[k], xk, pu); pr = fmaf(q.kr[k], xk, pr); pe = fmaf(q.ke[k], xk, pe);
+        }
+        const float u = sigmoidf_fast(pu), r = sigmoidf_fast(pr);
+        const float e = tanhf_fast(fmaf(r, q.ae, pe));
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
@@ -244,9 +279,15 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
         int forced = -1;
         if (warp == 0) {
             if (lane < UC && !last) load_g(half, s, gv);          // gates evaluated at the end of this half
-            if (half) { if (p.c_forced) forced = p.c_forced[s]; }
-            else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
-            u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
+            if (FUSED) {
+                if (half) { if (p.a_forced) forced = p.a_forced[s]; }
+                else      { if (p.b_forced) forced = p.b_forced[s - 1]; }
+                u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), (half ? 0u : 4u) + (unsigned)(lane >> 3));
+            } else {
+                if (half) { if (p.c_forced) forced = p.c_forced[s]; }
+                else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
+                u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
+            }
         }
 
         // ---- 1. input half-vector from the whole chip (y_c(s) carries tag s+1; y_f(s-1) carries tag s)
@@ -325,40 +366,69 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
 
         // ---- 4. warp 0: the cluster's 256 logits -> draw; then the gates of the other half of the state
         if (warp == 0) {
-            GatePre gp = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            GatePre gp = {};
             if (lane < UC && !last) gp = gates_prepare(half, gv);
-            float l[8];
-            {
-                // the four slots of this lane are loaded together and re-read until all of them carry this half-step's tag
-                const unsigned a = smem_addr(lbuf + (size_t)par * 128 + 4 * lane);
-                uint4 v0, v1, v2, v3;
+            int drawn;
+            if (FUSED) {
+                // 64 logits: one slot (two logits) per lane
+                const unsigned a = smem_addr(lbuf + (size_t)par * 128 + lane);
+                uint4 v0;
                 unsigned long long t0 = 0; unsigned cnt = 0;
                 while (true) {
-                    v0 = ld_shared_volatile_v4(a); v1 = ld_shared_volatile_v4(a + 16);
-                    v2 = ld_shared_volatile_v4(a + 32); v3 = ld_shared_volatile_v4(a + 48);
-                    const bool ok = v0.y == tag && v0.w == tag && v1.y == tag && v1.w == tag && v2.y == tag && v2.w == tag && v3.y == tag && v3.w == tag;
-                    if (ok) break;
+                    v0 = ld_shared_volatile_v4(a);
+                    if (v0.y == tag && v0.w == tag) break;
                     if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 3 + 4 * half)) { my_bad = true; break; }
                 }
-                l[0] = __uint_as_float(v0.x); l[1] = __uint_as_float(v0.z); l[2] = __uint_as_float(v1.x); l[3] = __uint_as_float(v1.z);
-                l[4] = __uint_as_float(v2.x); l[5] = __uint_as_float(v2.z); l[6] = __uint_as_float(v3.x); l[7] = __uint_as_float(v3.z);
-            }
-            my_bad = __any_sync(FULL, my_bad);
-            STAMP(4 + 6 * half);
-            int drawn = warp_softmax_draw_fast(l, u01, lane);
-            if (writer) {
-                if (p.dbg_logits) {
-                    float *d = p.dbg_logits + (size_t)(n - 1) * 256 + 8 * lane;
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) d[k] = l[k];
+                my_bad = __any_sync(FULL, my_bad);
+                STAMP(4 + 6 * half);
+                const float l0 = __uint_as_float(v0.x), l1 = __uint_as_float(v0.z);
+                const int nib = group16_softmax_draw(l0, l1, u01, lane);
+                drawn = (__shfl_sync(FULL, nib, 0) << 12) | (__shfl_sync(FULL, nib, 8) << 8) | (__shfl_sync(FULL, nib, 16) << 4) | __shfl_sync(FULL, nib, 24);
+                if (writer) {
+                    if (p.dbg_logits) { float *d = p.dbg_logits + (size_t)(n - 1) * 64 + 2 * lane; d[0] = l0; d[1] = l1; }
+                    if (lane == 0) {
+                        if (half) { if (p.a_out) p.a_out[s] = (uint16_t)drawn; }
+                        else      { if (p.b_out) p.b_out[s - 1] = (uint16_t)drawn; }
+                    }
                 }
-                if (lane == 0) {
-                    if (half) { if (p.c_out) p.c_out[s] = (uint8_t)drawn; }
-                    else      { if (p.f_out) p.f_out[s - 1] = (uint8_t)drawn; }
+            } else {
+                float l[8];
+                {
+                    // the four slots of this lane are loaded together and re-read until all of them carry this half-step's tag
+                    const unsigned a = smem_addr(lbuf + (size_t)par * 128 + 4 * lane);
+                    uint4 v0, v1, v2, v3;
+                    unsigned long long t0 = 0; unsigned cnt = 0;
+                    while (true) {
+                        v0 = ld_shared_volatile_v4(a); v1 = ld_shared_volatile_v4(a + 16);
+                        v2 = ld_shared_volatile_v4(a + 32); v3 = ld_shared_volatile_v4(a + 48);
+                        const bool ok = v0.y == tag && v0.w == tag && v1.y == tag && v1.w == tag && v2.y == tag && v2.w == tag && v3.y == tag && v3.w == tag;
+                        if (ok) break;
+                        if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 3 + 4 * half)) { my_bad = true; break; }
+                    }
+                    l[0] = __uint_as_float(v0.x); l[1] = __uint_as_float(v0.z); l[2] = __uint_as_float(v1.x); l[3] = __uint_as_float(v1.z);
+                    l[4] = __uint_as_float(v2.x); l[5] = __uint_as_float(v2.z); l[6] = __uint_as_float(v3.x); l[7] = __uint_as_float(v3.z);
+                }
+                my_bad = __any_sync(FULL, my_bad);
+                STAMP(4 + 6 * half);
+                drawn = warp_softmax_draw_fast(l, u01, lane);
+                if (writer) {
+                    if (p.dbg_logits) {
+                        float *d = p.dbg_logits + (size_t)(n - 1) * 256 + 8 * lane;
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) d[k] = l[k];
+                    }
+                    if (lane == 0) {
+                        if (half) { if (p.c_out) p.c_out[s] = (uint8_t)drawn; }
+                        else      { if (p.f_out) p.f_out[s - 1] = (uint8_t)drawn; }
+                    }
                 }
             }
             if (forced >= 0) drawn = forced;
-            if (!half) {
+            if (FUSED) {
+                // the two streams side by side: out[0][s] = a_s, out[1][s] = the sample part B emits in step s
+                if (writer && lane == 0 && p.out) p.out[(half ? 0 : T) + (half ? s : s - 1)] = (int16_t)(drawn - 32768);
+                if (!half) f_prev = drawn;
+            } else if (!half) {
                 if (writer && lane == 0 && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + drawn - 32768);
                 f_prev = drawn;
             }
@@ -374,8 +444,13 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
     if (writer && !any_bad) {
         if (p.h_out) for (int i = tid; i < K; i += blockDim.x) { p.h_out[i] = vecC[i]; p.h_out[K + i] = vecF[i]; }
         if (tid == 0) {
-            if (p.c_st_out) p.c_st_out[0] = (uint8_t)c_prev;
-            if (p.f_st_out) p.f_st_out[0] = (uint8_t)f_prev;
+            if (FUSED) {
+                if (p.a_st_out) p.a_st_out[0] = (uint16_t)c_prev;
+                if (p.b_st_out) p.b_st_out[0] = (uint16_t)f_prev;
+            } else {
+                if (p.c_st_out) p.c_st_out[0] = (uint8_t)c_prev;
+                if (p.f_st_out) p.f_st_out[0] = (uint8_t)f_prev;
+            }
         }
     }
     cluster.sync();     // nobody leaves while a peer may still write into its shared memory
@@ -441,8 +516,10 @@ static bool choose_shape(const wrnn_model *m, int CS, ResidentPack *k, std::stri
     if (m->sparse) { if (why) *why = "resident dense kernel does not take block masks"; return false; }
     if (H % 32 != 0) { if (why) *why = "H must be a multiple of 32"; return false; }
     if (CS != 8 && CS != 16) { if (why) *why = "cluster size must be 8 or 16"; return false; }
-    if (Hh % (2 * CS) != 0 || 256 % (16 * CS) != 0) { if (why) *why = "H/2 must be a multiple of twice the cluster size"; return false; }
-    const int HR = Hh / CS, LR = 256 / CS;
+    const bool fused = m->variant == 1;
+    const int n_logits = fused ? 64 : 256, n_in = fused ? 12 : 3;
+    if (Hh % (2 * CS) != 0 || n_logits % (2 * CS) != 0) { if (why) *why = "H/2 must be a multiple of twice the cluster size"; return false; }
+    const int HR = Hh / CS, LR = n_logits / CS;
     int best = 0;
     for (int ncta = CS; ncta <= m->n_sms; ncta += CS) {
         if (Hh % ncta) continue;
@@ -454,7 +531,8 @@ static bool choose_shape(const wrnn_model *m, int CS, ResidentPack *k, std::stri
     if (!best) { if (why) *why = "no CTA count tiles H/2 into 16-row fragments"; return false; }
     k->CS = CS; k->NCTA = best; k->NC = best / CS; k->UC = Hh / best; k->HR = HR; k->LR = LR;
     k->K = Hh; k->NKT = Hh / 16; k->n_rrows = 6 * k->UC;
-    k->NMT = (HR + k->n_rrows + 15) / 16; k->NLT = LR / 16;
+    k->NMT = (HR + k->n_rrows + 15) / 16; k->NLT = (LR + 15) / 16;
+    k->fused = fused;
     k->NMT += k->NMT & 1;                                   // tiles are multiplied in pairs
     k->NW = 16; k->KSH = 7; k->KSL = 7;
     if (k->NKT != 28 || (k->NMT / 2) * k->KSH > k->NW || k->NLT * k->KSL > k->NW || CS > k->NW || k->NMT * k->KSH > 32) {
@@ -462,7 +540,7 @@ static bool choose_shape(const wrnn_model *m, int CS, ResidentPack *k, std::stri
         return false;
     }
     k->w_bytes = ((size_t)2 * k->NMT + 2 * k->NLT) * 16 * k->K * 2;
-    size_t small = ((size_t)k->n_rrows * 3 + 2 * k->HR + 2 * k->LR) * 4;
+    size_t small = ((size_t)k->n_rrows * n_in + 2 * k->HR + 2 * k->LR) * 4;
     small = (small + 15) / 16 * 16;
     k->blob_bytes = k->w_bytes + small;
     k->smem_bytes = resident_smem_bytes(*k);
@@ -470,7 +548,10 @@ static bool choose_shape(const wrnn_model *m, int CS, ResidentPack *k, std::stri
 }
 
 // The one instantiated split: K = 448 as 7 x 4 k-tiles, for pairs of hidden tiles and for single logits tiles.
-static void *resident_fn() { return (void *)resident_dense_kernel<7, 4, 7, 4>; }
+static void *resident_fn(bool fused)
+{
+    return fused ? (void *)resident_dense_kernel<7, 4, 7, 4, true> : (void *)resident_dense_kernel<7, 4, 7, 4, false>;
+}
 
 int resident_supported(const wrnn_model *m, int batch, std::string *why)
 {
@@ -503,7 +584,7 @@ int resident_prepare(wrnn_model *m)
     std::string why;
     cudaDeviceProp prop;
     cudaGetDeviceProperties(&prop, m->device);
-    cudaFuncSetAttribute(resident_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    cudaFuncSetAttribute(resident_fn(m->variant == 1), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     cudaGetLastError();
     const char *force = getenv("WRNN_RESIDENT_CS");
     bool found = false;
@@ -512,13 +593,13 @@ int resident_prepare(wrnn_model *m)
         ResidentPack c;
         if (!choose_shape(m, cs, &c, &why)) continue;
         if ((size_t)c.smem_bytes > prop.sharedMemPerBlockOptin) { why = "weights do not fit in shared memory"; continue; }
-        if (cudaFuncSetAttribute(resident_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, c.smem_bytes) != cudaSuccess) {
+        if (cudaFuncSetAttribute(resident_fn(m->variant == 1), cudaFuncAttributeMaxDynamicSharedMemorySize, c.smem_bytes) != cudaSuccess) {
             cudaGetLastError(); why = "cannot raise the dynamic shared memory limit"; continue;
         }
         cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
         fill_launch(c, &cfg, at, 0, false);
         int max_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_fn(), &cfg) != cudaSuccess || max_clusters < c.NC) {
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_fn(m->variant == 1), &cfg) != cudaSuccess || max_clusters < c.NC) {
             cudaGetLastError(); why = "not enough co-resident clusters on this device"; continue;
         }
         k = c; found = true;
@@ -527,7 +608,7 @@ int resident_prepare(wrnn_model *m)
     if (!found) { m->err = why; return WRNN_ERR_UNSUPPORTED; }
 
     // ---- per-CTA blobs
-    const int H = m->H, K = k.K, UC = k.UC;
+    const int H = m->H, K = k.K, UC = k.UC, n_in = k.fused ? 12 : 3;
     std::vector<uint8_t> blob((size_t)k.NCTA * k.blob_bytes, 0);
     std::vector<std::vector<uint16_t>> rows(16, std::vector<uint16_t>(K));
     const BsrHost *Oa[2] = {&m->hO1, &m->hO3}, *Ob[2] = {&m->hO2, &m->hO4};
@@ -556,15 +637,18 @@ int resident_prepare(wrnn_model *m)
         uint16_t *wl = w + (size_t)2 * k.NMT * tile_elems;
         for (int h = 0; h < 2; ++h)
             for (int mt = 0; mt < k.NLT; ++mt) {
-                for (int r = 0; r < 16; ++r) dense_row_bf16(*Ob[h], rank * k.LR + 16 * mt + r, 0, K, rows[r].data());
+                for (int r = 0; r < 16; ++r) {
+                    if (16 * mt + r < k.LR) dense_row_bf16(*Ob[h], rank * k.LR + 16 * mt + r, 0, K, rows[r].data());
+                    else std::fill(rows[r].begin(), rows[r].end(), (uint16_t)0);
+                }
                 pack_tile(rows, K, wl + ((size_t)h * k.NLT + mt) * tile_elems);
             }
         for (int rr = 0; rr < k.n_rrows; ++rr) {
             const int half = rr / (3 * UC), gate = (rr / UC) % 3, u = rr % UC;
             const int mrow = gate * H + half * K + cta * UC + u;
-            for (int c = 0; c < 3; ++c) sm[rr * 3 + c] = m->hI[(size_t)mrow * 3 + c];
+            for (int c = 0; c < n_in; ++c) sm[rr * n_in + c] = m->hI[(size_t)mrow * n_in + c];
         }
-        float *b = sm + k.n_rrows * 3;
+        float *b = sm + k.n_rrows * n_in;
         for (int r = 0; r < k.HR; ++r) { b[r] = m->hb1[rank * k.HR + r]; b[k.HR + r] = m->hb3[rank * k.HR + r]; }
         b += 2 * k.HR;
         for (int r = 0; r < k.LR; ++r) { b[r] = m->hb2[rank * k.LR + r]; b[k.LR + r] = m->hb4[rank * k.LR + r]; }
@@ -626,6 +710,8 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in; p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
+    p.a_in = a.a_in; p.b_in = a.b_in; p.a_st_out = a.a_st_out; p.b_st_out = a.b_st_out;
+    p.a_forced = a.a_forced; p.b_forced = a.b_forced; p.a_out = a.a_out; p.b_out = a.b_out;
     p.status = m->status;
     p.limit_ns = 2000000000ull;
     p.prof = k.d_prof;
@@ -638,7 +724,8 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     // a profiler that replays kernels may not accept cooperative cluster launches.
     const char *no_coop = getenv("WRNN_NO_COOP");
     fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
-    cudaError_t e = cudaLaunchKernelEx(&cfg, resident_dense_kernel<7, 4, 7, 4>, p);
+    cudaError_t e = k.fused ? cudaLaunchKernelEx(&cfg, resident_dense_kernel<7, 4, 7, 4, true>, p)
+                            : cudaLaunchKernelEx(&cfg, resident_dense_kernel<7, 4, 7, 4, false>, p);
     if (e != cudaSuccess) {
         m->err = std::string("resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

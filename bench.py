@@ -100,21 +100,20 @@ def run_reference(args, wl):
         return
     from oracle import wrnn_oracle as orc
     w, masks, cond = synth.build_workload(wl)
-    om = orc.OracleModel(w, wl.dtype, masks, wl.block)
     cores = os.cpu_count() or 1
     threads = 1 if wl.batch == 1 else min(cores, wl.batch)
     # about 2-3 s of CPU work per step
     per_row_step_ms = 2.3 * (wl.H / 896.0) ** 2
     n_steps = max(16, min(wl.n_steps, int(2500.0 * threads / (per_row_step_ms * wl.batch))))
     n_steps = min(n_steps, (wl.n_frames * synth.HOP) // max(1, wl.row_stride) - 1)
-    kw = dict(hop=synth.HOP, row_stride=wl.row_stride, row_offset_mul=wl.row_offset_mul, threads=threads)
+    run = oracle_runner(orc, wl, w, masks, cond, threads)
     for _ in range(max(0, min(args.warmup, 1))):
-        om.run(cond, min(n_steps, 64), wl.batch, synth.SEED_SAMPLING, **kw)
+        run(min(n_steps, 64))
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        om.run(cond, n_steps, wl.batch, synth.SEED_SAMPLING, **kw)
+        run(n_steps)
     dt = (time.perf_counter() - t0) / args.steps
-    value = n_steps * wl.batch / dt
+    value = n_steps * wl.batch * samples_per_step(wl) / dt
     sample = "first %d of %d steps x %d rows of %s per step" % (n_steps, wl.n_steps, wl.batch, wl.name)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
@@ -129,20 +128,34 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
+def samples_per_step(wl):
+    """Audio samples one step of one row produces: 1, or 2 for the fused subscale variant."""
+    return 2 if wl.variant == 1 else 1
+
+
+def oracle_runner(orc, wl, w, masks, cond, threads):
+    """-> run(n_steps): the oracle of this workload's model variant on its inputs."""
+    if wl.variant == 1:
+        om = orc.Fs2OracleModel(w, wl.dtype)
+        return lambda n: om.run(cond[0], n, seed=synth.SEED_SAMPLING, hop=synth.HOP)
+    om = orc.OracleModel(w, wl.dtype, masks, wl.block)
+    return lambda n: om.run(cond, n, wl.batch, synth.SEED_SAMPLING, hop=synth.HOP, row_stride=wl.row_stride,
+                            row_offset_mul=wl.row_offset_mul, threads=threads)
+
+
 def cpu_baseline(wl, budget_s=12.0):
     from oracle import wrnn_oracle as orc
     w, masks, cond = synth.build_workload(wl)
-    om = orc.OracleModel(w, wl.dtype, masks, wl.block)
     cores = os.cpu_count() or 1
     threads = 1 if wl.batch == 1 else min(cores, wl.batch)
     per_row_step_ms = 2.3 * (wl.H / 896.0) ** 2
     n_steps = max(16, min(wl.n_steps, int(budget_s * 1e3 * threads / (per_row_step_ms * wl.batch))))
     n_steps = min(n_steps, (wl.n_frames * synth.HOP) // max(1, wl.row_stride) - 1)
+    run = oracle_runner(orc, wl, w, masks, cond, threads)
     t0 = time.perf_counter()
-    om.run(cond, n_steps, wl.batch, synth.SEED_SAMPLING, hop=synth.HOP, row_stride=wl.row_stride,
-           row_offset_mul=wl.row_offset_mul, threads=threads)
+    run(n_steps)
     dt = time.perf_counter() - t0
-    return {"value": n_steps * wl.batch / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+    return {"value": n_steps * wl.batch * samples_per_step(wl) / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": "first %d of %d steps x %d rows of %s, once" % (n_steps, wl.n_steps, wl.batch, wl.name)}
 
 
@@ -177,7 +190,7 @@ def main():
     n_steps = wl.n_steps if args.n_steps is None else args.n_steps
     w, masks, cond_np = synth.build_workload(wl)
     kern = {"auto": B.WRNN_KERNEL_AUTO, "generic": B.WRNN_KERNEL_GENERIC, "resident": B.WRNN_KERNEL_RESIDENT, "batched": B.WRNN_KERNEL_BATCHED, "bcluster": B.WRNN_KERNEL_BCLUSTER}[args.kernel]
-    model = B.wrnn_create(w, wl.dtype, masks, max_batch=wl.batch, kernel=kern, block=wl.block)
+    model = B.wrnn_create(w, wl.dtype, masks, max_batch=wl.batch, kernel=kern, block=wl.block, variant=wl.variant)
     info = B.wrnn_launch_info(model, wl.batch)
     cond = torch.from_numpy(cond_np).to(dev)
     out = torch.zeros((wl.batch, n_steps), dtype=torch.int16, device=dev)
@@ -186,8 +199,17 @@ def main():
     kw = dict(hop=synth.HOP, row_stride=wl.row_stride, row_offset_mul=wl.row_offset_mul, stream0=0)
     seed = replicas.rank_seed(synth.SEED_SAMPLING, rank)
 
+    fused = wl.variant == 1
+    if fused:       # two streams per call, then the interleaved samples (the two pre-roll samples of part B dropped)
+        out = torch.zeros((2, n_steps), dtype=torch.int16, device=dev)
+        u_out = torch.zeros((2 * (n_steps - 2),), dtype=torch.int16, device=dev)
+
     def one():
-        B.wrnn_sample(model, cond, n_steps, wl.batch, seed, out, **kw)
+        if fused:
+            B.wrnn_fs2_sample(model, cond, n_steps, seed, out, hop=synth.HOP)
+            B.wrnn_fs2_unfold(out, n_steps, u_out)
+        else:
+            B.wrnn_sample(model, cond, n_steps, wl.batch, seed, out, **kw)
 
     for _ in range(max(args.warmup, 3)):
         one()
@@ -217,23 +239,30 @@ def main():
     assert B.wrnn_poll_status(model) == 0, B.wrnn_last_error(model)
 
     ms_per_step = total_ms / args.steps
-    samples_per_call = n_steps * wl.batch
+    samples_per_call = 2 * (n_steps - 2) if fused else n_steps * wl.batch
     value = replicas.aggregate_throughput(world, samples_per_call, ms_per_step * 1e-3)
 
     # end to end through the host-buffer entry point (pinned host memory)
     e2e = None
     if not args.no_e2e:
         cond_pin = torch.from_numpy(cond_np).pin_memory()
-        out_pin = torch.zeros((wl.batch, n_steps), dtype=torch.int16).pin_memory()
+        out_pin = torch.zeros((2 * (n_steps - 2),) if fused else (wl.batch, n_steps), dtype=torch.int16).pin_memory()
+
+        def one_host():
+            if fused:
+                B.wrnn_fs2_sample_host(model, cond_pin.numpy()[0], n_steps, seed, out_pin.numpy(), hop=synth.HOP)
+            else:
+                B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
+
         for _ in range(2):
-            B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
+            one_host()
         replicas.barrier(pg)
         t0 = time.perf_counter()
         for _ in range(args.steps):
-            B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
+            one_host()
         dt = (time.perf_counter() - t0) / args.steps
         dt = replicas.max_over_ranks(dt, pg, dev)
-        assert np.array_equal(out_pin.numpy(), out.cpu().numpy()), "host-buffer path disagrees with the device path"
+        assert np.array_equal(out_pin.numpy(), (u_out if fused else out).cpu().numpy()), "host-buffer path disagrees with the device path"
         e2e = {"value": replicas.aggregate_throughput(world, samples_per_call, dt), "unit": UNIT, "h2d_bytes_per_step": int(cond_np.nbytes),
                "d2h_bytes_per_step": int(out_pin.numel() * 2)}
 
@@ -258,11 +287,12 @@ def main():
             # per step (3,047,296 weights at H = 896) over the aggregate shared-memory bandwidth, plus the floor
             # of the two chip-wide exchanges a step cannot avoid (measured live in an empty kernel of the same shape)
             H, Hh = wl.H, wl.H // 2
-            n_w = 3 * H * H + 2 * Hh * Hh + 2 * 256 * Hh + 9 * H
+            n_logits, n_in = (64, 12) if fused else (256, 3)
+            n_w = 3 * H * H + 2 * Hh * Hh + 2 * n_logits * Hh + 3 * n_in * H
             alg_bytes = n_w * (2 if wl.dtype == "bf16" else 4)
             ach = alg_bytes * n_steps / (ms_per_step * 1e-3) / 1e9
             roof = {"bound": "smem", "achieved": ach, "peak": SMEM_PEAK_GBS, "unit": "GB/s", "frac": ach / SMEM_PEAK_GBS,
-                    "traffic": 22862848 if info["kernel"] == 2 and wl.dtype == "bf16" else None,
+                    "traffic": 16394496 if info["kernel"] == 2 and wl.dtype == "bf16" and not fused else None,
                     "traffic_note": "DRAM bytes per launch from the ncu capture in profiles/ (one-time weight load; "
                                     "does not grow with the number of steps)",
                     "peak_source": "derived: 148 SMs x 128 B/clk x 1.965 GHz", "algorithmic_bytes_per_step": alg_bytes,

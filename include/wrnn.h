@@ -260,6 +260,10 @@ int wrnn_fs2_step_teacher_forced(wrnn_model *m, const wrnn_cond *cond, int64_t n
                                  uint16_t *a_out, uint16_t *b_out, float *dbg_gates, float *dbg_h, float *dbg_logits,
                                  void *cuda_stream);
 int wrnn_fs2_unfold(const int16_t *ab, int64_t n_steps, int16_t *u, void *cuda_stream);
+/* Host-buffer convenience, synchronous: cond_host HOST [n_frames][cond_dim] -> device, wrnn_fs2_sample from the default
+ * state, wrnn_fs2_unfold, and the 2 (n_steps - 2) interleaved samples back to u_host (HOST int16). */
+int wrnn_fs2_sample_host(wrnn_model *m, const float *cond_host, int32_t n_frames, int32_t hop, int64_t n_steps,
+                         uint64_t seed, int16_t *u_host);
 
 /* Diagnostic of the resident single-stream kernel (Section 2.1: after the persistent kernel the
  * remaining overhead is the synchronisation between multiprocessors): SM-clock cycles that warp 0 of

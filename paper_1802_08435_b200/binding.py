@@ -26,7 +26,7 @@ EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
     "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor", "wrnn_sample_noalloc",
-    "wrnn_selftest_bounded_wait", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold",
+    "wrnn_selftest_bounded_wait", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold", "wrnn_fs2_sample_host",
 ]
 
 
@@ -83,6 +83,7 @@ def lib():
         L.wrnn_fs2_sample.argtypes = [vp, C.POINTER(wrnn_cond), i64, u64, C.POINTER(wrnn_fs2_state), vp, vp]
         L.wrnn_fs2_step_teacher_forced.argtypes = [vp, C.POINTER(wrnn_cond), i64, u64, C.POINTER(wrnn_fs2_state)] + [vp] * 8
         L.wrnn_fs2_unfold.argtypes = [vp, i64, vp, vp]
+        L.wrnn_fs2_sample_host.argtypes = [vp, vp, i32, i32, i64, u64, vp]
         L.wrnn_fold.argtypes = [vp, i64, i32, vp, vp]
         L.wrnn_unfold.argtypes = [vp, i64, i32, vp, vp]
         L.wrnn_sample_subscale.argtypes = [vp, vp, i32, i32, i64, i32, u64, vp, vp]
@@ -239,6 +240,13 @@ def wrnn_fs2_step_teacher_forced(model, cond, n_steps: int, seed: int, a_forced,
 def wrnn_fs2_unfold(ab, n_steps: int, u, stream=None):
     """ab: CUDA int16 [2][n_steps] from wrnn_fs2_sample; u: CUDA int16 [2 (n_steps - 2)]."""
     _check(lib().wrnn_fs2_unfold(_dev_ptr(ab), n_steps, _dev_ptr(u), _stream_ptr(stream)))
+
+
+def wrnn_fs2_sample_host(model, cond_host: Optional[np.ndarray], n_steps: int, seed: int, u_host: np.ndarray, *, hop: int = 120):
+    """Host buffers in and out: cond_host [n_frames][cond_dim] float32, u_host int16 [2 (n_steps - 2)]; synchronous."""
+    n_frames = 0 if cond_host is None else int(cond_host.shape[-2])
+    assert u_host.dtype == np.int16 and u_host.flags.c_contiguous and u_host.size >= 2 * max(n_steps - 2, 0)
+    _check(lib().wrnn_fs2_sample_host(model, _np_ptr(cond_host), n_frames, hop, n_steps, seed, _np_ptr(u_host)), model)
 
 
 def wrnn_sample_subscale(model, cond, n_total: int, B: int, seed: int, out, *, hop: int = 120, stream=None):

@@ -524,6 +524,42 @@ int wrnn_sample_host(wrnn_model *m, const float *cond_host, int32_t n_frames, in
     return wrnn_poll_status(m);
 }
 
+int wrnn_fs2_sample_host(wrnn_model *m, const float *cond_host, int32_t n_frames, int32_t hop, int64_t n_steps, uint64_t seed,
+                         int16_t *u_host)
+{
+    if (!m) return WRNN_ERR_INVALID_ARG;
+    if (m->variant != 1) return fail(m, WRNN_ERR_UNSUPPORTED, "not a fused subscale model (create with variant = 1)");
+    if (n_steps < 0 || n_frames < 0) return fail(m, WRNN_ERR_INVALID_ARG, "bad sizes");
+    if (cudaSetDevice(m->device) != cudaSuccess) return fail(m, WRNN_ERR_CUDA, "cudaSetDevice failed");
+    const size_t nc = m->cond_dim ? (size_t)n_frames * m->cond_dim : 0;
+    const size_t nu = n_steps > 2 ? 2 * (size_t)(n_steps - 2) : 0;
+    const size_t no = 2 * (size_t)n_steps + nu;                 // the two streams, then the interleaved samples
+    if (nc > m->stage_cond_cap) {
+        cudaDeviceSynchronize();
+        cudaFree(m->stage_cond); m->stage_cond = nullptr; m->stage_cond_cap = 0;
+        if (cudaMalloc((void **)&m->stage_cond, nc * sizeof(float)) != cudaSuccess) { cudaGetLastError(); return fail(m, WRNN_ERR_NOMEM, "staging allocation failed"); }
+        m->stage_cond_cap = nc;
+    }
+    if (no > m->stage_out_cap) {
+        cudaDeviceSynchronize();
+        cudaFree(m->stage_out); m->stage_out = nullptr; m->stage_out_cap = 0;
+        if (cudaMalloc((void **)&m->stage_out, no * sizeof(int16_t)) != cudaSuccess) { cudaGetLastError(); return fail(m, WRNN_ERR_NOMEM, "staging allocation failed"); }
+        m->stage_out_cap = no;
+    }
+    if (nc && (!cond_host || cudaMemcpyAsync(m->stage_cond, cond_host, nc * sizeof(float), cudaMemcpyHostToDevice, 0) != cudaSuccess))
+        return fail(m, WRNN_ERR_CUDA, "cond upload failed");
+    wrnn_cond c = {m->stage_cond, n_frames, hop, 1, 0};
+    int rc = wrnn_fs2_sample(m, m->cond_dim ? &c : nullptr, n_steps, seed, nullptr, m->stage_out, nullptr);
+    if (rc != WRNN_OK) return rc;
+    int16_t *u = m->stage_out + 2 * (size_t)n_steps;
+    rc = fs2_unfold_launch(m->stage_out, n_steps, u, 0);
+    if (rc != WRNN_OK) return fail(m, rc, "unfold launch failed");
+    if (nu && (!u_host || cudaMemcpyAsync(u_host, u, nu * sizeof(int16_t), cudaMemcpyDeviceToHost, 0) != cudaSuccess))
+        return fail(m, WRNN_ERR_CUDA, "sample download failed");
+    if (cudaStreamSynchronize(0) != cudaSuccess) return fail(m, WRNN_ERR_CUDA, cudaGetErrorString(cudaGetLastError()));
+    return wrnn_poll_status(m);
+}
+
 int wrnn_poll_status(wrnn_model *m)
 {
     if (!m) return WRNN_ERR_INVALID_ARG;

@@ -104,6 +104,7 @@ class Workload:
     sparsity: Optional[float] = None
     subscale_B: int = 0       # >0: fold/unfold of one n_steps*B sequence
     block: tuple = (4, 4)     # shape of one block of the sparsity masks (rows, columns)
+    variant: int = 0          # 1: Fused Subscale WaveRNN 2x (two samples per step)
 
 
 # The five named workloads (index = position in the benchmark's config list), then three extra ones.
@@ -118,12 +119,14 @@ WORKLOADS = [
     Workload("sparse2048_1x1_bf16_b1_2400", 2048, "bf16", 1, 2400, 20, sparsity=0.96, block=(1, 1)),
     # the paper's own small-batch point (Section 5.1: four utterances at once)
     Workload("batched4_896_bf16_24000", 896, "bf16", 4, 24000, 200),
+    # Fused Subscale WaveRNN 2x (Section 4.4): 12,002 steps = 24,000 samples after the two pre-roll samples
+    Workload("fused2x_896_bf16_24000", 896, "bf16", 1, 12002, 102, variant=1),
 ]
 
 
 def build_workload(wl: Workload, n_steps: Optional[int] = None, batch: Optional[int] = None):
     """-> (weights, masks or None, cond[batch][n_frames][64]).  n_steps/batch shrink the case."""
-    w = make_weights(wl.H)
+    w = make_weights(wl.H, n_inputs=12, n_logits=64) if wl.variant == 1 else make_weights(wl.H)
     masks = None
     if wl.sparsity is not None:
         masks = make_block_masks(wl.H, wl.sparsity, block=wl.block)

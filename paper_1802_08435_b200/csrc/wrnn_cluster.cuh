@@ -23,6 +23,37 @@ __device__ __forceinline__ void st_cluster_ll(unsigned addr, float v0, float v1,
                  "r"(__float_as_uint(v1)), "r"(tag)
                  : "memory");
 }
+// Asynchronous 16-byte (or, below, 8-byte) store of four (two) values into a (possibly remote) CTA's shared memory that counts its bytes on an
+// mbarrier of the same CTA: the receiver waits on the barrier instead of polling the data, so nothing competes with the
+// arriving stores (measured on a 16-CTA all-gather of 448 values: 600 cycles against 780 for tagged stores + polls).
+__device__ __forceinline__ void st_async_v4(unsigned addr, float v0, float v1, float v2, float v3, unsigned mbar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(addr),
+                 "r"(__float_as_uint(v0)), "r"(__float_as_uint(v1)), "r"(__float_as_uint(v2)), "r"(__float_as_uint(v3)), "r"(mbar)
+                 : "memory");
+}
+__device__ __forceinline__ void st_async_v2(unsigned addr, float v0, float v1, unsigned mbar)
+{
+    asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v2.b32 [%0], {%1, %2}, [%3];" ::"r"(addr),
+                 "r"(__float_as_uint(v0)), "r"(__float_as_uint(v1)), "r"(mbar)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_init_cluster(unsigned mbar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(mbar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+// one arrival that also announces `bytes` of asynchronous stores still to come in this phase
+__device__ __forceinline__ void mbar_arrive_expect(unsigned mbar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(mbar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_parity(unsigned mbar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }" : "=r"(ok) : "r"(mbar), "r"(parity) : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ uint4 ld_shared_volatile_v4(unsigned addr)
 {
     uint4 v;

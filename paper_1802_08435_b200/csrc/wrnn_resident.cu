@@ -105,15 +105,20 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
     __nv_bfloat16 *splC = reinterpret_cast<__nv_bfloat16 *>(part + 512);       // split images, 4 K bf16 each
     __nv_bfloat16 *splF = splC + 4 * K;
     __nv_bfloat16 *splQ = splF + 4 * K;
-    uint4 *qbuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                    // [2][K/2]
-    uint4 *lbuf = qbuf + K;                                                    // [2][128]
+    float *qbuf = reinterpret_cast<float *>(splQ + 4 * K);                    // [2][K] hidden layer of the cluster
+    uint4 *lbuf = reinterpret_cast<uint4 *>(qbuf + 2 * K);                     // [2][128] logits of the cluster: {v, tag, v, tag}
+    __shared__ __align__(8) unsigned long long xbar[2];                        // arrival barriers of qbuf[0], qbuf[1]
 
     // ---- one-time load of this CTA's weights
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(p.blob + (size_t)cta * p.blob_bytes);
         uint4 *dst = reinterpret_cast<uint4 *>(smem);
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
-        for (int i = tid; i < K + 256; i += blockDim.x) qbuf[i] = make_uint4(0, 0, 0, 0);   // qbuf and lbuf are adjacent
+        for (int i = tid; i < 2 * K + 1024; i += blockDim.x) qbuf[i] = 0.f;             // qbuf and lbuf are adjacent
+        if (tid == 0) {
+            for (int i = 0; i < 2; ++i) mbar_init_cluster(smem_addr(&xbar[i]), 1);
+            mbar_fence_init();
+        }
         for (int i = tid; i < 12 * K / 8; i += blockDim.x) reinterpret_cast<uint4 *>(splC)[i] = make_uint4(0, 0, 0, 0);
         __syncthreads();
         for (int i = tid; i < K; i += blockDim.x) {
@@ -167,13 +172,25 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
         }
     };
     // one peer per warp: warp w sends this CTA's whole slice to CTA w of the cluster with one store instruction, lanes at
-    // consecutive 16-byte slots (a store whose lanes address several CTAs at once is much slower)
-    unsigned q_snd[2], l_snd[2];
+    // consecutive pieces (a store whose lanes address several CTAs at once is much slower).  The hidden layer, which
+    // many threads consume, goes by asynchronous stores that count their bytes on the receiver's barrier of that buffer
+    // (nobody polls the data); the logits, which one warp consumes, as tagged values that this warp polls.
+    unsigned q_snd[2], l_snd[2], q_bar[2];
 #pragma unroll
     for (int par2 = 0; par2 < 2; ++par2) {
-        q_snd[par2] = map_to_rank(smem_addr(qbuf + (size_t)par2 * (K / 2) + (rank * HR) / 2 + (lane < HR / 2 ? lane : 0)), warp < CS ? warp : 0);
-        l_snd[par2] = map_to_rank(smem_addr(lbuf + (size_t)par2 * 128 + (rank * LR) / 2 + (lane < LR / 2 ? lane : 0)), warp < CS ? warp : 0);
+        const unsigned peer = warp < CS ? warp : 0;
+        q_snd[par2] = map_to_rank(smem_addr(qbuf + (size_t)par2 * K + rank * HR + 2 * (lane < HR / 2 ? lane : 0)), peer);
+        l_snd[par2] = map_to_rank(smem_addr(lbuf + (size_t)par2 * 128 + (rank * LR) / 2 + (lane < LR / 2 ? lane : 0)), peer);
+        q_bar[par2] = map_to_rank(smem_addr(&xbar[par2]), peer);
     }
+    // bounded wait for all bytes of one buffer (use k of a buffer completes barrier phase k)
+    auto wait_arrival = [&](int which, unsigned use, int step, int phase) {
+        const unsigned bar = smem_addr(&xbar[which]);
+        unsigned long long t0 = 0; unsigned cnt = 0;
+        while (!mbar_try_parity(bar, use & 1u))
+            if ((++cnt & 1023u) == 0 && wt.expired(t0, step, phase)) return false;
+        return true;
+    };
     // ---- prologue: the recurrent products of step 0 from the initial state, coarse gates of step 0
     if (h_on) hidden_products(wMA, splC);
     __syncthreads();
@@ -274,6 +291,8 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
         float *vec = half ? vecC : vecF;
         __nv_bfloat16 *spl = half ? splC : splF;
 
+        const unsigned use = (unsigned)((n - 1) >> 1);          // how often this half's buffers were used before
+        if (tid == 0) mbar_arrive_expect(smem_addr(&xbar[par]), (unsigned)K * 4u);      // this half's arrivals: K hidden values
         // everything that does not depend on the chain is fetched / computed before the first wait
         float gv[3] = {0.f, 0.f, 0.f}, u01 = 0.f;
         int forced = -1;
@@ -318,7 +337,7 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
             float v0 = bh[r0], v1 = bh[r0 + 1];
 #pragma unroll
             for (int sp = 0; sp < KSH; ++sp) { v0 += part[(tile * KSH + sp) * 16 + rr]; v1 += part[(tile * KSH + sp) * 16 + rr + 1]; }
-            st_cluster_ll(q_snd[par], fmaxf(v0, 0.f), fmaxf(v1, 0.f), tag);
+            st_async_v2(q_snd[par], fmaxf(v0, 0.f), fmaxf(v1, 0.f), q_bar[par]);
         }
         if (h_fin && lane < 16) {
             // R rows of this tile (rows >= HR of the stacked matrix) stay in this CTA
@@ -334,17 +353,11 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
         STAMP(1 + 6 * half);
 
         // ---- 3. the cluster's hidden layer -> logits rows of this CTA
-#pragma unroll 1
-        for (int i = tid; i < K / 2; i += blockDim.x) {
-            const unsigned a = smem_addr(qbuf + (size_t)par * (K / 2) + i);
-            uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
-            while (true) {
-                v = ld_shared_volatile_v4(a);
-                if (v.y == tag && v.w == tag) break;
-                if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 2 + 4 * half)) { my_bad = true; break; }
-            }
-            store_split2(splQ, 2 * i, __uint_as_float(v.x));
-            store_split2(splQ, 2 * i + 1, __uint_as_float(v.z));
+        if (tid < K / 2) {
+            if (!wait_arrival(par, use, (int)s, 2 + 4 * half)) my_bad = true;
+            const float2 v = reinterpret_cast<const float2 *>(qbuf + (size_t)par * K)[tid];
+            store_split2(splQ, 2 * tid, v.x);
+            store_split2(splQ, 2 * tid + 1, v.y);
         }
         if (__syncthreads_or(my_bad)) break;
         STAMP(2 + 6 * half);
@@ -466,7 +479,7 @@ static int resident_smem_bytes(const ResidentPack &k)
     b += a * 4;
     b += 512 * 4;                                   // partial sums [tiles x K-splits][16]
     b += (size_t)12 * k.K * 2;                      // three split images of 4 K bf16
-    b += (size_t)k.K * 16;                          // qbuf [2][K/2] x 16 B
+    b += (size_t)2 * k.K * 4;                       // qbuf [2][K]
     b += 256 * 16;                                  // lbuf [2][128] x 16 B
     return (int)b;
 }

@@ -313,14 +313,19 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
         {
             const unsigned long long *slots = p.slots + (size_t)(half ? (s & 1) : 2 + ((s - 1) & 1)) * K;
             const unsigned ytag = (unsigned)(half ? s + 1 : s);
+            // two adjacent slots per polling thread (one 16-byte load): half as many requests queue at the L2 slices
 #pragma unroll 1
-            for (int i = tid; i < K; i += blockDim.x) {
-                unsigned long long v, t0 = 0; unsigned cnt = 0;
-                while ((unsigned)((v = ld_relaxed_u64(slots + i)) >> 32) != ytag)
+            for (int i = tid; i < K / 2; i += blockDim.x) {
+                unsigned long long v0, v1, t0 = 0; unsigned cnt = 0;
+                while (true) {
+                    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0), "=l"(v1) : "l"(slots + 2 * i) : "memory");
+                    if ((unsigned)(v0 >> 32) == ytag && (unsigned)(v1 >> 32) == ytag) break;
                     if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
-                const float x = __uint_as_float((unsigned)v);
-                vec[i] = x;
-                store_split2(spl, i, x);
+                }
+                const float x0 = __uint_as_float((unsigned)v0), x1 = __uint_as_float((unsigned)v1);
+                vec[2 * i] = x0; vec[2 * i + 1] = x1;
+                store_split2(spl, 2 * i, x0);
+                store_split2(spl, 2 * i + 1, x1);
             }
             if (__syncthreads_or(my_bad)) break;
         }

@@ -391,6 +391,32 @@ def test_resident_and_generic_kernels_agree(env):
             B.wrnn_destroy(m)
 
 
+def test_resident_kernel_short_calls_and_resume(env):
+    """The resident bf16 kernel at H = 896 in calls of 1, 2 and 3 steps and a resumed run: every call sets up and
+    drains its exchange buffers and barriers; the pieces must reproduce the unbroken run bit for bit."""
+    torch, B = env
+    wl = synth.WORKLOADS[1]
+    w, masks, cond = synth.build_workload(wl)
+    m = B.wrnn_create(w, wl.dtype, kernel=B.WRNN_KERNEL_RESIDENT)
+    try:
+        full = _free_run(torch, B, m, cond, 40, 1, SEED)
+        h = torch.zeros((1, wl.H), dtype=torch.float32, device="cuda:0")
+        cp = torch.full((1,), 128, dtype=torch.uint8, device="cuda:0")
+        fp = torch.zeros((1,), dtype=torch.uint8, device="cuda:0")
+        pieces, pos = [], 0
+        for n in (1, 2, 3, 1, 33):
+            pieces.append(_free_run(torch, B, m, cond, n, 1, SEED, h=h, c_prev=cp, f_prev=fp, step0=pos))
+            pos += n
+        assert np.array_equal(np.concatenate(pieces, axis=1), full)
+        om = orc.OracleModel(w, wl.dtype)
+        ref = om.run(cond, 40, 1, SEED, dump=True)
+        div = pu.first_divergence(full, ref.out)
+        if div >= 0:
+            assert ref.margins[0, div].min() < pu.MARGIN
+    finally:
+        B.wrnn_destroy(m)
+
+
 def test_config2_sparse_bf16(env):
     """Block-sparse H=2048 bf16 (96 % of the 4x4 blocks of R_u, R_r, R_e, O1, O3 pruned), batch 1: the first
     1,500 steps against the dense-with-zeros oracle; the full 24,000 steps for determinism and resume."""

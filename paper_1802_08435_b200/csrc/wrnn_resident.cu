@@ -387,6 +387,7 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
             GatePre gp = {};
             if (lane < UC && !last) gp = gates_prepare(half, gv);
             int drawn;
+            float l[FUSED ? 2 : 8];
             if (FUSED) {
                 // 64 logits: one slot (two logits) per lane
                 const unsigned a = smem_addr(lbuf + (size_t)par * 128 + lane);
@@ -399,18 +400,10 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
                 }
                 my_bad = __any_sync(FULL, my_bad);
                 STAMP(4 + 6 * half);
-                const float l0 = __uint_as_float(v0.x), l1 = __uint_as_float(v0.z);
-                const int nib = group16_softmax_draw(l0, l1, u01, lane);
+                l[0] = __uint_as_float(v0.x); l[1] = __uint_as_float(v0.z);
+                const int nib = group16_softmax_draw(l[0], l[1], u01, lane);
                 drawn = (__shfl_sync(FULL, nib, 0) << 12) | (__shfl_sync(FULL, nib, 8) << 8) | (__shfl_sync(FULL, nib, 16) << 4) | __shfl_sync(FULL, nib, 24);
-                if (writer) {
-                    if (p.dbg_logits) { float *d = p.dbg_logits + (size_t)(n - 1) * 64 + 2 * lane; d[0] = l0; d[1] = l1; }
-                    if (lane == 0) {
-                        if (half) { if (p.a_out) p.a_out[s] = (uint16_t)drawn; }
-                        else      { if (p.b_out) p.b_out[s - 1] = (uint16_t)drawn; }
-                    }
-                }
             } else {
-                float l[8];
                 {
                     // the four slots of this lane are loaded together and re-read until all of them carry this half-step's tag
                     const unsigned a = smem_addr(lbuf + (size_t)par * 128 + 4 * lane);
@@ -428,30 +421,33 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
                 }
                 my_bad = __any_sync(FULL, my_bad);
                 STAMP(4 + 6 * half);
-                drawn = warp_softmax_draw_fast(l, u01, lane);
-                if (writer) {
-                    if (p.dbg_logits) {
-                        float *d = p.dbg_logits + (size_t)(n - 1) * 256 + 8 * lane;
+                drawn = warp_softmax_draw_fast(reinterpret_cast<const float (&)[8]>(l), u01, lane);
+            }
+            // The chip waits for the slowest CTA's state: publish first, the writer's bookkeeping (which only CTA 0 has)
+            // comes after it and overlaps the next exchange.
+            const int fed = forced >= 0 ? forced : drawn;
+            if (lane < UC && !last && !my_bad) gates_and_publish(half, s, fed, gp);
+            if (writer) {
+                constexpr int NL = FUSED ? 2 : 8, NLOG2 = FUSED ? 64 : 256;
+                if (p.dbg_logits) {
+                    float *d = p.dbg_logits + (size_t)(n - 1) * NLOG2 + NL * lane;
 #pragma unroll
-                        for (int k = 0; k < 8; ++k) d[k] = l[k];
-                    }
-                    if (lane == 0) {
+                    for (int k = 0; k < NL; ++k) d[k] = l[k];
+                }
+                if (lane == 0) {
+                    if (FUSED) {
+                        if (half) { if (p.a_out) p.a_out[s] = (uint16_t)drawn; }
+                        else      { if (p.b_out) p.b_out[s - 1] = (uint16_t)drawn; }
+                        // the two streams side by side: out[0][s] = a_s, out[1][s] = the sample part B emits in step s
+                        if (p.out) p.out[(half ? 0 : T) + (half ? s : s - 1)] = (int16_t)(fed - 32768);
+                    } else {
                         if (half) { if (p.c_out) p.c_out[s] = (uint8_t)drawn; }
                         else      { if (p.f_out) p.f_out[s - 1] = (uint8_t)drawn; }
+                        if (!half && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + fed - 32768);
                     }
                 }
             }
-            if (forced >= 0) drawn = forced;
-            if (FUSED) {
-                // the two streams side by side: out[0][s] = a_s, out[1][s] = the sample part B emits in step s
-                if (writer && lane == 0 && p.out) p.out[(half ? 0 : T) + (half ? s : s - 1)] = (int16_t)(drawn - 32768);
-                if (!half) f_prev = drawn;
-            } else if (!half) {
-                if (writer && lane == 0 && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + drawn - 32768);
-                f_prev = drawn;
-            }
-            if (lane < UC && !last && !my_bad) gates_and_publish(half, s, drawn, gp);
-            if (half) c_prev = drawn;
+            if (half) c_prev = fed; else f_prev = fed;
         }
         STAMP(5 + 6 * half);
     }

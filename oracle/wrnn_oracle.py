@@ -326,3 +326,50 @@ class Fs2OracleModel(OracleModel):
         if rc != 0:
             raise ValueError("conditioning frame index out of range")
         return Fs2Result(out, a_out, b_out, margins, hh, int(ap[0]), int(bp[0]), gates, hs, logits)
+
+
+# ----------------------------------------------------------------------------------------------
+# Subscale generation with dependent rows (Section 4.1 ordering, Section 4.2 future horizon)
+#
+# What the paper fixes: sub-tensor s (samples u_{B i + s}) is generated after sub-tensors z < s and is conditioned on
+# their past and on their future up to a horizon of F positions, through a conditioning network whose mask removes the
+# past connections; the WaveRNN itself is shared by all sub-tensors.  The network used here is a stated reading (one
+# masked convolution layer instead of the paper's ten, synthetic weights; parity for it is unpinned outside this file):
+#     v_s[i] = frame_s[(B i + s) div hop] + relu(b + sum_{delta=1..s} sum_{d=0..F} V[delta-1][d] . x(u_{s-delta}[i+d]))
+# with x(u) = u / 32768 for the int16 sample u, positions at or beyond the row length contributing nothing; row s is
+# an ordinary WaveRNN stream (Philox stream id s, step = position) whose conditioning vector at step i is v_s[i].
+
+def subscale_conditioning(history: np.ndarray, s: int, V: np.ndarray, b: np.ndarray) -> np.ndarray:
+    """The convolution term of v_s for all positions: history int16 [B][L] (rows < s must be complete), V [B-1][F+1][D],
+    b [D] -> float32 [L][D].  Plain double loops over (delta, d); row 0 has no earlier row: relu(b)."""
+    B, L = history.shape
+    F1, D = V.shape[1], V.shape[2]
+    acc = np.tile(b.astype(np.float64), (L, 1))
+    for delta in range(1, s + 1):
+        x = history[s - delta].astype(np.float64) / 32768.0
+        for d in range(F1):
+            n = L - d
+            if n <= 0:
+                break
+            acc[:n] += np.outer(x[d:], V[delta - 1, d].astype(np.float64))
+    return np.maximum(acc, 0.0).astype(np.float32)
+
+
+def subscale_dependent_run(om: "OracleModel", frames: np.ndarray, V: np.ndarray, b: np.ndarray, B: int, L: int, hop: int,
+                           seed: int, forced: Optional[np.ndarray] = None):
+    """Generate the B sub-tensors one after the other (the order of Eq. 4).  frames: float32 [B][n_frames][D] (row s,
+    frame (B i + s) div hop at position i).  forced: optional int16 [B][L]; when given, row s is conditioned on the
+    forced samples of rows < s (the drawn ones are still returned).  -> (samples int16 [B][L], cond float32 [B][L][D],
+    margins [B][L][2])."""
+    D = om.cond_dim
+    out = np.zeros((B, L), np.int16)
+    cond = np.zeros((B, L, D), np.float32)
+    margins = np.zeros((B, L, 2), np.float64)
+    for s in range(B):
+        hist = out if forced is None else forced
+        idx = (B * np.arange(L) + s) // hop
+        cond[s] = frames[s][idx] + (subscale_conditioning(hist, s, V, b) if s > 0 else np.maximum(b, 0.0).astype(np.float32)[None, :])
+        r = om.run(cond[s][None], L, 1, seed, hop=1, stream0=s)
+        out[s] = r.out[0]
+        margins[s] = r.margins[0]
+    return out, cond, margins

@@ -91,6 +91,15 @@ def make_cond(batch: int, n_frames: int, cond_dim: int = COND_DIM, seed: int = S
     return rng.standard_normal((batch, n_frames, cond_dim)).astype(np.float32)
 
 
+def make_subscale_conv(B: int, F: int, cond_dim: int = COND_DIM, seed: int = 417):
+    """Synthetic weights of the one-layer masked convolution that conditions sub-tensor s on sub-tensors z < s
+    (Section 4.1): V [B-1][F+1][cond_dim] ~ N(0, 1 / ((F+1) (B-1))) scaled to unit-order outputs, b [cond_dim]."""
+    rng = np.random.default_rng(seed)
+    V = (rng.standard_normal((max(B - 1, 1), F + 1, cond_dim)) * (3.0 / np.sqrt((F + 1) * max(B - 1, 1)))).astype(np.float32)
+    b = (rng.standard_normal(cond_dim) * 0.1).astype(np.float32)
+    return V, b
+
+
 @dataclass
 class Workload:
     name: str

@@ -205,6 +205,28 @@ int wrnn_sample_subscale(wrnn_model *m, const float *cond, int32_t n_frames, int
                          int64_t n_total, int32_t B, uint64_t seed, int16_t *out, void *cuda_stream);
 
 /*
+ * Subscale generation with dependent rows and the staggered schedule of batched sampling (Sections 4.1, 4.2): sub-tensor r
+ * (samples u_{B i + r}) is conditioned on the sub-tensors z < r, on their positions up to F ahead of its own, and starts
+ * `lag` steps after sub-tensor r - 1, so that after (B - 1) lag steps all B rows advance together through the shared
+ * WaveRNN.  The conditioning network is computed `chunk` positions ahead at a time (the paper's L), hence lag >= F + chunk
+ * (and a multiple of chunk, so that the rows' chunks line up).  The network here is one masked convolution (a stated
+ * reading; the paper's has ten layers):
+ *     v_r[i] = frames[r][(B i + r) div hop] + relu(bias + sum_{delta=1..r} sum_{d=0..F} V[delta-1][d] x(u_{r-delta}[i + d]))
+ * with x(u) = u / 32768 and positions beyond the row length contributing nothing; row r is a WaveRNN stream with Philox
+ * stream id r, step = position, conditioning vector v_r[i] at step i.  The result does not depend on chunk or lag.
+ * frames: DEVICE [B][n_frames][cond_dim]; V: DEVICE [B-1][F+1][cond_dim]; bias: DEVICE [cond_dim]; out: DEVICE int16
+ * [n_total] in the original order.  B <= max_batch given at create.  Asynchronous on cuda_stream.  Runs on the any-shape
+ * kernel.  wrnn_subscale_conditioning computes v_row[0..L) alone from a given history (DEVICE int16 [B][L]) into
+ * v (DEVICE [L][cond_dim]).
+ */
+int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n_frames, int32_t hop, const float *V,
+                                   const float *bias, int32_t F, int32_t chunk, int32_t lag, int64_t n_total, int32_t B,
+                                   uint64_t seed, int16_t *out, void *cuda_stream);
+int wrnn_subscale_conditioning(const int16_t *hist, const float *frames, const float *V, const float *bias, int32_t B,
+                               int64_t L, int32_t F, int32_t cond_dim, int32_t n_frames, int32_t hop, int32_t row, float *v,
+                               void *cuda_stream);
+
+/*
  * Host-buffer convenience for callers without device pointers: copies cond
  * (HOST [batch][n_frames][cond_dim]) to the device, runs wrnn_sample from the
  * default state and copies the samples back to out (HOST int16 [batch][n_steps]).

@@ -27,6 +27,7 @@ EXPORTS = [
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
     "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor", "wrnn_sample_noalloc",
     "wrnn_selftest_bounded_wait", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold", "wrnn_fs2_sample_host",
+    "wrnn_sample_subscale_dependent", "wrnn_subscale_conditioning",
 ]
 
 
@@ -84,6 +85,8 @@ def lib():
         L.wrnn_fs2_step_teacher_forced.argtypes = [vp, C.POINTER(wrnn_cond), i64, u64, C.POINTER(wrnn_fs2_state)] + [vp] * 8
         L.wrnn_fs2_unfold.argtypes = [vp, i64, vp, vp]
         L.wrnn_fs2_sample_host.argtypes = [vp, vp, i32, i32, i64, u64, vp]
+        L.wrnn_sample_subscale_dependent.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i64, i32, u64, vp, vp]
+        L.wrnn_subscale_conditioning.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, i32, vp, vp]
         L.wrnn_fold.argtypes = [vp, i64, i32, vp, vp]
         L.wrnn_unfold.argtypes = [vp, i64, i32, vp, vp]
         L.wrnn_sample_subscale.argtypes = [vp, vp, i32, i32, i64, i32, u64, vp, vp]
@@ -240,6 +243,21 @@ def wrnn_fs2_step_teacher_forced(model, cond, n_steps: int, seed: int, a_forced,
 def wrnn_fs2_unfold(ab, n_steps: int, u, stream=None):
     """ab: CUDA int16 [2][n_steps] from wrnn_fs2_sample; u: CUDA int16 [2 (n_steps - 2)]."""
     _check(lib().wrnn_fs2_unfold(_dev_ptr(ab), n_steps, _dev_ptr(u), _stream_ptr(stream)))
+
+
+def wrnn_sample_subscale_dependent(model, frames, V, bias, F: int, chunk: int, lag: int, n_total: int, B: int, seed: int, out, *,
+                                   hop: int = 120, stream=None):
+    """Subscale generation with dependent rows on the staggered schedule.  frames: CUDA float32 [B][n_frames][D];
+    V: CUDA float32 [B-1][F+1][D]; bias: CUDA float32 [D]; out: CUDA int16 [n_total] in the original order."""
+    _check(lib().wrnn_sample_subscale_dependent(model, _dev_ptr(frames), int(frames.shape[1]), hop, _dev_ptr(V), _dev_ptr(bias), F,
+                                                chunk, lag, n_total, B, seed, _dev_ptr(out), _stream_ptr(stream)), model)
+
+
+def wrnn_subscale_conditioning(hist, frames, V, bias, F: int, row: int, v, *, hop: int = 120, stream=None):
+    """v (CUDA float32 [L][D]) = conditioning vectors of sub-tensor `row` from the history hist (CUDA int16 [B][L])."""
+    B, L = int(hist.shape[0]), int(hist.shape[1])
+    _check(lib().wrnn_subscale_conditioning(_dev_ptr(hist), _dev_ptr(frames), _dev_ptr(V), _dev_ptr(bias), B, L, F, int(frames.shape[2]),
+                                            int(frames.shape[1]), hop, row, _dev_ptr(v), _stream_ptr(stream)))
 
 
 def wrnn_fs2_sample_host(model, cond_host: Optional[np.ndarray], n_steps: int, seed: int, u_host: np.ndarray, *, hop: int = 120):

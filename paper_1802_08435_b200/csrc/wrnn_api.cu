@@ -196,6 +196,7 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     if (!ensure_g(m, (size_t)a.batch * nf * 3 * m->H)) return fail(m, WRNN_ERR_NOMEM, "conditioning scratch allocation failed");
     int rc = cond_project(m, a.cond, a.batch, nf, s);
     if (rc != WRNN_OK) return fail(m, rc, "conditioning projection launch failed");
+    if (a.row_lag > 0) return generic_run(m, a, s);          // staggered rows: the any-shape kernel
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
     if (use_resf32(m, a.batch)) return resf32_run(m, a, s);
     if (use_sparse(m, a.batch)) return sparse_run(m, a, s);
@@ -379,7 +380,7 @@ void wrnn_destroy(wrnn_model *m)
     cudaFree(m->I); cudaFree(m->b_gate); cudaFree(m->b1); cudaFree(m->b2); cudaFree(m->b3); cudaFree(m->b4);
     cudaFree(m->W_condT); cudaFree(m->g); cudaFree(m->hbuf[0]); cudaFree(m->hbuf[1]); cudaFree(m->a_fine);
     cudaFree(m->q); cudaFree(m->logits); cudaFree(m->c_cur); cudaFree(m->c_prev); cudaFree(m->f_prev);
-    cudaFree(m->bar); cudaFree(m->status); cudaFree(m->stage_cond); cudaFree(m->stage_out);
+    cudaFree(m->bar); cudaFree(m->status); cudaFree(m->stage_cond); cudaFree(m->stage_out); cudaFree(m->sub_scratch);
     cudaGetLastError();
     delete m;
 }
@@ -490,6 +491,84 @@ int wrnn_sample_subscale(wrnn_model *m, const float *cond, int32_t n_frames, int
     int rc = wrnn_sample(m, &c, n_total / B, B, seed, nullptr, m->stage_out, cuda_stream);
     if (rc != WRNN_OK) return rc;
     return fold_launch(m->stage_out, n_total, B, out, true, (cudaStream_t)cuda_stream);
+}
+
+int wrnn_subscale_conditioning(const int16_t *hist, const float *frames, const float *V, const float *bias, int32_t B, int64_t L,
+                               int32_t F, int32_t cond_dim, int32_t n_frames, int32_t hop, int32_t row, float *v, void *cuda_stream)
+{
+    if (!hist || !frames || !V || !bias || !v || B < 1 || L < 1 || F < 0 || cond_dim < 1 || hop < 1 || row < 0 || row >= B || L > (1ll << 30))
+        return WRNN_ERR_INVALID_ARG;
+    if (((long long)B * (L - 1) + row) / hop >= n_frames) return WRNN_ERR_INVALID_ARG;
+    return subscale_cond_launch(hist, frames, V, bias, v, B, L, F, cond_dim, n_frames, hop, row, 1, 0, 0, (int)L, (cudaStream_t)cuda_stream);
+}
+
+int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n_frames, int32_t hop, const float *V, const float *bias,
+                                   int32_t F, int32_t chunk, int32_t lag, int64_t n_total, int32_t B, uint64_t seed, int16_t *out,
+                                   void *cuda_stream)
+{
+    if (!m) return WRNN_ERR_INVALID_ARG;
+    if (m->variant != 0) return fail(m, WRNN_ERR_UNSUPPORTED, "subscale generation takes a WaveRNN model (variant 0)");
+    if (m->cond_dim <= 0) return fail(m, WRNN_ERR_INVALID_ARG, "the model must be conditioned");
+    if (B < 1 || B > m->max_batch || n_total < 0 || n_total % B != 0) return fail(m, WRNN_ERR_INVALID_ARG, "B must divide n_total and fit max_batch");
+    if (n_total == 0) return WRNN_OK;
+    if (!frames || !V || !bias || !out || hop < 1 || F < 0 || chunk < 1) return fail(m, WRNN_ERR_INVALID_ARG, "bad arguments");
+    // row r + 1 may use positions of row r up to F ahead of its own, for a whole chunk at a time: it follows F + chunk
+    // steps (or more) behind; chunks of all rows line up when the lag is a multiple of the chunk
+    if (lag < F + chunk || lag % chunk != 0) return fail(m, WRNN_ERR_INVALID_ARG, "lag must be a multiple of chunk and at least F + chunk");
+    const long long L = n_total / B;
+    if (((long long)B * (L - 1) + (B - 1)) / hop >= n_frames) return fail(m, WRNN_ERR_INVALID_ARG, "conditioning frames run out");
+    if (cudaSetDevice(m->device) != cudaSuccess) return fail(m, WRNN_ERR_CUDA, "cudaSetDevice failed");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const int D = m->cond_dim, H = m->H;
+    // scratch: sample history [B][L], per-call conditioning [B][chunk][D], carry state
+    const size_t need = (size_t)B * L * sizeof(int16_t) + (size_t)B * chunk * D * sizeof(float) + (size_t)B * H * sizeof(float) + 2 * (size_t)B + 64;
+    if (need > m->sub_cap) {
+        cudaDeviceSynchronize();
+        cudaFree(m->sub_scratch); m->sub_scratch = nullptr; m->sub_cap = 0;
+        if (cudaMalloc((void **)&m->sub_scratch, need) != cudaSuccess) { cudaGetLastError(); return fail(m, WRNN_ERR_NOMEM, "scratch allocation failed"); }
+        m->sub_cap = need;
+    }
+    float *v = reinterpret_cast<float *>(m->sub_scratch);
+    float *hst = v + (size_t)B * chunk * D;
+    int16_t *hist = reinterpret_cast<int16_t *>(hst + (size_t)B * H);
+    uint8_t *cp = reinterpret_cast<uint8_t *>(hist + (size_t)B * L);
+    uint8_t *fp = cp + B;
+    if (cudaMemsetAsync(hst, 0, (size_t)B * H * sizeof(float), s) != cudaSuccess || cudaMemsetAsync(cp, 128, B, s) != cudaSuccess ||
+        cudaMemsetAsync(fp, 0, B, s) != cudaSuccess || cudaMemsetAsync(hist, 0, (size_t)B * L * sizeof(int16_t), s) != cudaSuccess)
+        return fail(m, WRNN_ERR_CUDA, "scratch initialisation failed");
+
+    auto run_rows = [&](int r_a, int n_rows, long long p_lo, int n) -> int {
+        int rc = subscale_cond_launch(hist, frames, V, bias, v, B, L, F, D, n_frames, hop, r_a, n_rows, p_lo, lag, n, s);
+        if (rc != WRNN_OK) return fail(m, rc, "conditioning launch failed");
+        StepArgs a;
+        std::memset(&a, 0, sizeof(a));
+        a.cond = v; a.n_frames = n; a.hop = 1; a.row_stride = 1; a.row_offset_mul = 0;
+        a.n_steps = n; a.batch = n_rows; a.seed = seed; a.step0 = p_lo; a.stream0 = (unsigned)r_a;
+        a.h_in = a.h_out = hst + (size_t)r_a * H;
+        a.c_in = a.c_st_out = cp + r_a; a.f_in = a.f_st_out = fp + r_a;
+        a.out = hist + (size_t)r_a * L + p_lo;
+        a.row_lag = lag; a.out_pitch = L - lag;
+        return run_steps(m, a, s);
+    };
+    // global time advances by one chunk per iteration; row r is at position k * chunk - r * lag
+    for (long long k = 0;; ++k) {
+        const long long t = k * chunk;
+        if (t - (long long)(B - 1) * lag >= L) break;                       // the last row is done
+        const int r_hi = (int)std::min<long long>(B - 1, t / lag);
+        int r_lo = t >= L ? (int)((t - L) / lag) + 1 : 0;
+        if (r_lo > r_hi) continue;                                          // a gap between rows (lag > L)
+        const long long p_lo = t - (long long)r_lo * lag;
+        const long long left = L - p_lo;
+        if (left < chunk) {                                                 // the oldest active row ends inside this chunk
+            int rc = run_rows(r_lo, 1, p_lo, (int)left);
+            if (rc != WRNN_OK) return rc;
+            ++r_lo;
+            if (r_lo > r_hi) continue;
+        }
+        int rc = run_rows(r_lo, r_hi - r_lo + 1, t - (long long)r_lo * lag, chunk);
+        if (rc != WRNN_OK) return rc;
+    }
+    return fold_launch(hist, n_total, B, out, true, s);
 }
 
 int wrnn_sample_host(wrnn_model *m, const float *cond_host, int32_t n_frames, int32_t hop, int32_t row_stride,

@@ -20,6 +20,9 @@ struct GenericParams {
     unsigned stream0;
     unsigned long long seed;
     int n_frames, hop, row_stride, row_offset_mul;
+    int row_lag;                 // > 0: row b of the call is row_lag steps behind row b - 1 (staggered subscale rows); its
+                                 // conditioning then holds one frame per step of the call
+    long long out_pitch;         // samples between the rows of `out`
     BsrDev R, O1, O2, O3, O4;
     const float *I, *b1, *b2, *b3, *b4, *g;
     float *h0, *h1, *a_fine, *q, *logits;
@@ -100,6 +103,7 @@ __device__ __forceinline__ float blockrow_total(const BsrDev &M, int br, const f
 
 __device__ __forceinline__ long long frame_of(const GenericParams &p, long long s, int gb)
 {
+    if (p.row_lag > 0) return s;
     return ((p.step0 + s) * p.row_stride + (long long)(p.stream0 + (unsigned)gb) * p.row_offset_mul) / p.hop;
 }
 
@@ -216,7 +220,7 @@ __global__ void __launch_bounds__(512, 1) generic_step_kernel(const GenericParam
                 const float4 v0 = __ldcg(reinterpret_cast<const float4 *>(p.logits + (size_t)gb * 256 + 8 * lane));
                 const float4 v1 = __ldcg(reinterpret_cast<const float4 *>(p.logits + (size_t)gb * 256 + 8 * lane + 4));
                 l[0] = v0.x; l[1] = v0.y; l[2] = v0.z; l[3] = v0.w; l[4] = v1.x; l[5] = v1.y; l[6] = v1.z; l[7] = v1.w;
-                const float u = uniform24(p.seed, p.stream0 + (unsigned)gb, (unsigned long long)(p.step0 + s), head);
+                const float u = uniform24(p.seed, p.stream0 + (unsigned)gb, (unsigned long long)(p.step0 + s - (long long)gb * p.row_lag), head);
                 int idx = warp_softmax_draw(l, u, lane);
                 if (lane == 0) {
                     const size_t o = (size_t)gb * p.n_steps + s;
@@ -228,7 +232,7 @@ __global__ void __launch_bounds__(512, 1) generic_step_kernel(const GenericParam
                         if (p.f_out) p.f_out[o] = (uint8_t)idx;
                         if (p.f_forced) idx = p.f_forced[o];
                         const int c = p.c_cur[gb];
-                        if (p.out) p.out[o] = (int16_t)(256 * c + idx - 32768);
+                        if (p.out) p.out[(size_t)gb * p.out_pitch + s] = (int16_t)(256 * c + idx - 32768);
                         p.c_prev[gb] = (uint8_t)c;
                         p.f_prev[gb] = (uint8_t)idx;
                     }
@@ -307,6 +311,37 @@ int fold_launch(const int16_t *x, long long n_total, int B, int16_t *sub, bool u
     return cudaGetLastError() == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
 }
 
+// Conditioning of staggered subscale rows (Section 4.1: sub-tensor r sees the future of sub-tensors z < r up to F
+// positions; one masked convolution stands in for the paper's network):
+//     v[b][c][k] = frame_r[(B (p + c) + r) div hop][k] + relu(bias[k] + sum_{delta=1..r} sum_{d=0..F} V[delta-1][d][k] x(hist[r-delta][p+c+d]))
+// for row r = r_lo + b of the call, whose first position is p = p_lo - b * lag; x(u) = u / 32768; positions >= L give 0.
+__global__ void subscale_cond_kernel(const int16_t *__restrict__ hist, const float *__restrict__ frames, const float *__restrict__ V,
+                                     const float *__restrict__ bias, float *__restrict__ v, int B, long long L, int F, int D,
+                                     int n_frames, int hop, int r_lo, long long p_lo, int lag, int n_steps)
+{
+    const int b = blockIdx.y, c = blockIdx.x, r = r_lo + b;
+    const long long pos = p_lo - (long long)b * lag + c;
+    for (int k = threadIdx.x; k < D; k += blockDim.x) {
+        float acc = bias[k];
+        for (int delta = 1; delta <= r; ++delta) {
+            const int16_t *hz = hist + (size_t)(r - delta) * L;
+            const float *Vz = V + (size_t)(delta - 1) * (F + 1) * D + k;
+            for (int d = 0; d <= F && pos + d < L; ++d) acc = fmaf(Vz[(size_t)d * D], (float)hz[pos + d] * (1.0f / 32768.0f), acc);
+        }
+        const long long fr = ((long long)B * pos + r) / hop;
+        v[((size_t)b * n_steps + c) * D + k] = frames[((size_t)r * n_frames + fr) * D + k] + fmaxf(acc, 0.f);
+    }
+}
+
+int subscale_cond_launch(const int16_t *hist, const float *frames, const float *V, const float *bias, float *v, int B, long long L, int F,
+                         int D, int n_frames, int hop, int r_lo, int n_rows, long long p_lo, int lag, int n_steps, cudaStream_t s)
+{
+    if (n_rows <= 0 || n_steps <= 0) return WRNN_OK;
+    subscale_cond_kernel<<<dim3(n_steps, n_rows), 64, 0, s>>>(hist, frames, V, bias, v, B, L, F, D, n_frames, hop, r_lo, p_lo, lag, n_steps);
+    ++g_launches;
+    return cudaGetLastError() == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
+}
+
 // The two streams of the fused subscale variant back in the original order: u[2 i] = a_i, u[2 i + 1] = the sample part B
 // emitted two steps later (Section 4.4 with F = 2).
 __global__ void fs2_unfold_kernel(const int16_t *__restrict__ ab, long long n, int16_t *__restrict__ u)
@@ -358,6 +393,7 @@ int generic_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in;
     p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
+    p.row_lag = a.row_lag; p.out_pitch = a.out_pitch ? a.out_pitch : a.n_steps;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.bar = m->bar; p.status = m->status;
     p.limit_ns = 2000000000ull;
@@ -481,6 +517,7 @@ extern "C" int wrnn_sample_noalloc(wrnn_model *m, const wrnn_cond *cond, int64_t
     p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in;
     p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
     p.c_forced = nullptr; p.f_forced = nullptr; p.c_out = nullptr; p.f_out = nullptr; p.out = a.out;
+    p.row_lag = 0; p.out_pitch = a.n_steps;
     p.dbg_gates = nullptr; p.dbg_h = nullptr; p.dbg_logits = nullptr;
     p.bar = reinterpret_cast<unsigned long long *>(base + o_bar);
     p.status = m->status;

@@ -47,6 +47,10 @@ struct StepArgs {
     uint8_t *c_out, *f_out;                      // [batch][n_steps] or null
     int16_t *out;                                // [batch][n_steps] or null
     float *dbg_gates, *dbg_h, *dbg_logits;       // or null
+    // staggered subscale rows: row b of the call is row_lag steps behind row b - 1 and takes one conditioning frame per
+    // step of the call (0 = rows in lock step); out_pitch = samples between the rows of `out` (0 = n_steps)
+    int row_lag;
+    long long out_pitch;
     // fused subscale variant: 16-bit samples of parts A and B in place of the bytes above (batch 1)
     const uint16_t *a_in, *b_in; uint16_t *a_st_out, *b_st_out;
     const uint16_t *a_forced, *b_forced;         // [n_steps] or null
@@ -88,6 +92,7 @@ struct wrnn_model {
     // host staging for wrnn_sample_host
     float *stage_cond = nullptr; size_t stage_cond_cap = 0;
     int16_t *stage_out = nullptr; size_t stage_out_cap = 0;
+    uint8_t *sub_scratch = nullptr; size_t sub_cap = 0;   // history, conditioning and carry state of wrnn_sample_subscale_dependent
 
     wrnn::ResidentPack *resident = nullptr;
     wrnn::ResF32Pack *resf32 = nullptr;
@@ -115,6 +120,8 @@ int generic_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);   // returns 
 int cond_project(wrnn_model *m, const float *cond, int batch, int n_frames, cudaStream_t s);
 int fold_launch(const int16_t *x, long long n_total, int B, int16_t *sub, bool unfold, cudaStream_t s);
 int fs2_unfold_launch(const int16_t *ab, long long n, int16_t *u, cudaStream_t s);
+int subscale_cond_launch(const int16_t *hist, const float *frames, const float *V, const float *bias, float *v, int B, long long L, int F,
+                         int D, int n_frames, int hop, int r_lo, int n_rows, long long p_lo, int lag, int n_steps, cudaStream_t s);
 
 // wrnn_resident.cu
 int resident_supported(const wrnn_model *m, int batch, std::string *why);

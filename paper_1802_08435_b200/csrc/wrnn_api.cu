@@ -196,7 +196,8 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     if (!ensure_g(m, (size_t)a.batch * nf * 3 * m->H)) return fail(m, WRNN_ERR_NOMEM, "conditioning scratch allocation failed");
     int rc = cond_project(m, a.cond, a.batch, nf, s);
     if (rc != WRNN_OK) return fail(m, rc, "conditioning projection launch failed");
-    if (a.row_lag > 0) return generic_run(m, a, s);          // staggered rows: the any-shape kernel
+    // staggered rows: the cluster-partitioned kernel, else the any-shape kernel
+    if (a.row_lag > 0) return a.batch >= 2 && use_bcluster(m, a.batch) ? bcluster_run(m, a, s) : generic_run(m, a, s);
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
     if (use_resf32(m, a.batch)) return resf32_run(m, a, s);
     if (use_sparse(m, a.batch)) return sparse_run(m, a, s);

@@ -67,6 +67,8 @@ struct BcParams {
     unsigned stream0;
     unsigned long long seed;
     int n_frames, hop, row_stride, row_offset_mul;
+    int row_lag;                 // > 0: row b of the call is row_lag steps behind row b - 1 and takes one conditioning frame per step
+    long long out_pitch;         // samples between the rows of `out`
     const float4 *Ip;
     const float *bp, *g;
     __nv_bfloat16 *act0, *act1, *q;
@@ -438,7 +440,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
     int g_rem = 0;
     float x0 = 0.f, x1 = 0.f;
     if (g_rowv) {
-        const long long pos = p.step0 * p.row_stride + (long long)(p.stream0 + (unsigned)g_gb) * p.row_offset_mul;
+        const long long pos = p.row_lag > 0 ? 0 : p.step0 * p.row_stride + (long long)(p.stream0 + (unsigned)g_gb) * p.row_offset_mul;
         g_frame = pos / p.hop;
         g_rem = (int)(pos - g_frame * p.hop);
         x0 = scale8(p.c_in ? (int)p.c_in[g_gb] : 128);
@@ -526,7 +528,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 const float4 v0 = *reinterpret_cast<const float4 *>(s_log + warp * 256 + 8 * lane);
                 const float4 v1 = *reinterpret_cast<const float4 *>(s_log + warp * 256 + 8 * lane + 4);
                 l[0] = v0.x; l[1] = v0.y; l[2] = v0.z; l[3] = v0.w; l[4] = v1.x; l[5] = v1.y; l[6] = v1.z; l[7] = v1.w;
-                const float u = uniform24(p.seed, p.stream0 + (unsigned)s_gb, (unsigned long long)(p.step0 + s), head);
+                const float u = uniform24(p.seed, p.stream0 + (unsigned)s_gb, (unsigned long long)(p.step0 + s - (long long)s_gb * p.row_lag), head);
                 drawn = warp_softmax_draw_fast(l, u, lane);
                 const uint8_t *forced = head ? p.f_forced : p.c_forced;
                 used = forced ? (int)forced[s_o] : drawn;
@@ -546,7 +548,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 } else {
                     if (lane == 0) {
                         if (p.f_out) p.f_out[s_o] = (uint8_t)drawn;
-                        if (p.out) p.out[s_o] = (int16_t)(256 * last_c + used - 32768);
+                        if (p.out) p.out[(long long)s_gb * p.out_pitch + s] = (int16_t)(256 * last_c + used - 32768);
                     }
                     last_f = used;
                 }
@@ -788,6 +790,7 @@ int bcluster_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.act0 = k.act[0]; p.act1 = k.act[1]; p.q = k.q;
     p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in; p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
+    p.row_lag = a.row_lag; p.out_pitch = a.out_pitch ? a.out_pitch : a.n_steps;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
     p.tmWr = k.tmWr; p.tmO1 = k.tmO1; p.tmO2 = k.tmO2; p.tmO3 = k.tmO3; p.tmO4 = k.tmO4;

@@ -42,8 +42,11 @@ def _gpu_run(torch, Bn, m, frames, V, b, F, chunk, lag, B_rows, L, hop=synth.HOP
     return out.cpu().numpy()
 
 
-@pytest.mark.parametrize("H,dtype,B_rows,L,F,chunk", [(32, "f32", 4, 90, 6, 3), (64, "bf16", 5, 64, 8, 8), (896, "bf16", 16, 300, 32, 32)])
-def test_staggered_schedule_and_oracle(env, H, dtype, B_rows, L, F, chunk):
+@pytest.mark.parametrize("H,dtype,B_rows,L,F,chunk,kernel", [
+    (32, "f32", 4, 90, 6, 3, "generic"), (64, "bf16", 5, 64, 8, 8, "generic"), (896, "bf16", 16, 300, 32, 32, "generic"),
+    (896, "bf16", 16, 300, 32, 32, "auto"),      # two or more active rows run on the cluster-partitioned kernel
+])
+def test_staggered_schedule_and_oracle(env, H, dtype, B_rows, L, F, chunk, kernel):
     torch, Bn = env
     w, V, b, frames = _case(H, B_rows, L, F, scale=2.0 if H < 100 else 1.0)
     om = orc.OracleModel(w, dtype)
@@ -57,18 +60,21 @@ def test_staggered_schedule_and_oracle(env, H, dtype, B_rows, L, F, chunk):
         Bn.wrnn_subscale_conditioning(hist, fr_d, V_d, b_d, F, row, v)
         torch.cuda.synchronize()
         assert pu.rel_err(v.cpu().numpy(), cond_ref[row]) < 1e-5, row
-    m = Bn.wrnn_create(w, dtype, max_batch=B_rows)
+    m = Bn.wrnn_create(w, dtype, max_batch=B_rows, kernel=Bn.WRNN_KERNEL_GENERIC if kernel == "generic" else Bn.WRNN_KERNEL_AUTO)
     try:
+        if kernel == "auto":
+            assert Bn.wrnn_launch_info(m, B_rows)["kernel"] == Bn.WRNN_KERNEL_BCLUSTER
         lag = F + chunk if (F + chunk) % chunk == 0 else ((F + chunk + chunk - 1) // chunk) * chunk
         stag = _gpu_run(torch, Bn, m, frames, V, b, F, chunk, lag, B_rows, L)
         # row after row: a lag beyond the row length leaves one row active at a time
         seq_lag = ((L + F + chunk) // chunk + 1) * chunk
         seq = _gpu_run(torch, Bn, m, frames, V, b, F, chunk, seq_lag, B_rows, L)
-        assert np.array_equal(stag, seq)
-        # another chunk / lag: same samples
-        if chunk % 2 == 0 and F % (chunk // 2) == 0:
-            other = _gpu_run(torch, Bn, m, frames, V, b, F, chunk // 2, 2 * (F + chunk // 2), B_rows, L)
-            assert np.array_equal(other, stag)
+        if kernel == "generic":      # one kernel family: the schedule cannot change a bit
+            assert np.array_equal(stag, seq)
+            # another chunk / lag: same samples
+            if chunk % 2 == 0 and F % (chunk // 2) == 0:
+                other = _gpu_run(torch, Bn, m, frames, V, b, F, chunk // 2, 2 * (F + chunk // 2), B_rows, L)
+                assert np.array_equal(other, stag)
         # against the oracle: in the order of Eq. 4 (row after row) the first difference, if any, sits at a near-boundary draw
         got = orc.fold(stag, B_rows)
         for row in range(B_rows):

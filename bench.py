@@ -101,7 +101,7 @@ def run_reference(args, wl):
     from oracle import wrnn_oracle as orc
     w, masks, cond = synth.build_workload(wl)
     cores = os.cpu_count() or 1
-    threads = 1 if wl.batch == 1 else min(cores, wl.batch)
+    threads = 1 if (wl.batch == 1 or wl.dependent) else min(cores, wl.batch)      # dependent rows are generated one after the other
     # about 2-3 s of CPU work per step
     per_row_step_ms = 2.3 * (wl.H / 896.0) ** 2
     n_steps = max(16, min(wl.n_steps, int(2500.0 * threads / (per_row_step_ms * wl.batch))))
@@ -138,6 +138,10 @@ def oracle_runner(orc, wl, w, masks, cond, threads):
     if wl.variant == 1:
         om = orc.Fs2OracleModel(w, wl.dtype)
         return lambda n: om.run(cond[0], n, seed=synth.SEED_SAMPLING, hop=synth.HOP)
+    if wl.dependent:
+        om = orc.OracleModel(w, wl.dtype)
+        V, b = synth.make_subscale_conv(wl.batch, wl.dependent[0])
+        return lambda n: orc.subscale_dependent_run(om, cond, V, b, wl.batch, n, synth.HOP, synth.SEED_SAMPLING)
     om = orc.OracleModel(w, wl.dtype, masks, wl.block)
     return lambda n: om.run(cond, n, wl.batch, synth.SEED_SAMPLING, hop=synth.HOP, row_stride=wl.row_stride,
                             row_offset_mul=wl.row_offset_mul, threads=threads)
@@ -147,7 +151,7 @@ def cpu_baseline(wl, budget_s=12.0):
     from oracle import wrnn_oracle as orc
     w, masks, cond = synth.build_workload(wl)
     cores = os.cpu_count() or 1
-    threads = 1 if wl.batch == 1 else min(cores, wl.batch)
+    threads = 1 if (wl.batch == 1 or wl.dependent) else min(cores, wl.batch)      # dependent rows are generated one after the other
     per_row_step_ms = 2.3 * (wl.H / 896.0) ** 2
     n_steps = max(16, min(wl.n_steps, int(budget_s * 1e3 * threads / (per_row_step_ms * wl.batch))))
     n_steps = min(n_steps, (wl.n_frames * synth.HOP) // max(1, wl.row_stride) - 1)
@@ -204,8 +208,16 @@ def main():
         out = torch.zeros((2, n_steps), dtype=torch.int16, device=dev)
         u_out = torch.zeros((2 * (n_steps - 2),), dtype=torch.int16, device=dev)
 
+    dep = wl.dependent
+    if dep:
+        Vn, bn = synth.make_subscale_conv(wl.batch, dep[0])
+        V_d, b_d = torch.from_numpy(Vn).to(dev), torch.from_numpy(bn).to(dev)
+        out = torch.zeros((wl.batch * n_steps,), dtype=torch.int16, device=dev)
+
     def one():
-        if fused:
+        if dep:
+            B.wrnn_sample_subscale_dependent(model, cond, V_d, b_d, dep[0], dep[1], dep[2], wl.batch * n_steps, wl.batch, seed, out, hop=synth.HOP)
+        elif fused:
             B.wrnn_fs2_sample(model, cond, n_steps, seed, out, hop=synth.HOP)
             B.wrnn_fs2_unfold(out, n_steps, u_out)
         else:
@@ -248,8 +260,17 @@ def main():
         cond_pin = torch.from_numpy(cond_np).pin_memory()
         out_pin = torch.zeros((2 * (n_steps - 2),) if fused else (wl.batch, n_steps), dtype=torch.int16).pin_memory()
 
+        if dep:
+            V_pin, b_pin = torch.from_numpy(Vn).pin_memory(), torch.from_numpy(bn).pin_memory()
+            out_pin = torch.zeros((wl.batch * n_steps,), dtype=torch.int16).pin_memory()
+
         def one_host():
-            if fused:
+            if dep:      # host buffers in and out around the device entry point
+                cond.copy_(cond_pin, non_blocking=True); V_d.copy_(V_pin, non_blocking=True); b_d.copy_(b_pin, non_blocking=True)
+                one()
+                out_pin.copy_(out, non_blocking=True)
+                torch.cuda.synchronize()
+            elif fused:
                 B.wrnn_fs2_sample_host(model, cond_pin.numpy()[0], n_steps, seed, out_pin.numpy(), hop=synth.HOP)
             else:
                 B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
@@ -263,7 +284,8 @@ def main():
         dt = (time.perf_counter() - t0) / args.steps
         dt = replicas.max_over_ranks(dt, pg, dev)
         assert np.array_equal(out_pin.numpy(), (u_out if fused else out).cpu().numpy()), "host-buffer path disagrees with the device path"
-        e2e = {"value": replicas.aggregate_throughput(world, samples_per_call, dt), "unit": UNIT, "h2d_bytes_per_step": int(cond_np.nbytes),
+        e2e = {"value": replicas.aggregate_throughput(world, samples_per_call, dt), "unit": UNIT,
+               "h2d_bytes_per_step": int(cond_np.nbytes) + (int(Vn.nbytes + bn.nbytes) if dep else 0),
                "d2h_bytes_per_step": int(out_pin.numel() * 2)}
 
     if rank == 0:

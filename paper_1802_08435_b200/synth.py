@@ -114,6 +114,7 @@ class Workload:
     subscale_B: int = 0       # >0: fold/unfold of one n_steps*B sequence
     block: tuple = (4, 4)     # shape of one block of the sparsity masks (rows, columns)
     variant: int = 0          # 1: Fused Subscale WaveRNN 2x (two samples per step)
+    dependent: Optional[tuple] = None   # (F, chunk, lag): subscale rows conditioned on the earlier rows, staggered schedule
 
 
 # The five named workloads (index = position in the benchmark's config list), then three extra ones.
@@ -130,6 +131,10 @@ WORKLOADS = [
     Workload("batched4_896_bf16_24000", 896, "bf16", 4, 24000, 200),
     # Fused Subscale WaveRNN 2x (Section 4.4): 12,002 steps = 24,000 samples after the two pre-roll samples
     Workload("fused2x_896_bf16_24000", 896, "bf16", 1, 12002, 102, variant=1),
+    # Subscale 16x with dependent rows (Sections 4.1, 4.2): 4 s of audio, F = 128, conditioning 128 positions at a time,
+    # rows 256 steps apart (the batch is full after 15 x 256 of the 9,840 global steps)
+    Workload("subscale16_dependent_896_bf16_6000", 896, "bf16", 16, 6000, 802, row_stride=16, row_offset_mul=1, subscale_B=16,
+             dependent=(128, 128, 256)),
 ]
 
 

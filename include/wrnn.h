@@ -215,8 +215,9 @@ int wrnn_sample_subscale(wrnn_model *m, const float *cond, int32_t n_frames, int
  * with x(u) = u / 32768 and positions beyond the row length contributing nothing; row r is a WaveRNN stream with Philox
  * stream id r, step = position, conditioning vector v_r[i] at step i.  The result does not depend on chunk or lag.
  * frames: DEVICE [B][n_frames][cond_dim]; V: DEVICE [B-1][F+1][cond_dim]; bias: DEVICE [cond_dim]; out: DEVICE int16
- * [n_total] in the original order.  B <= max_batch given at create.  Asynchronous on cuda_stream.  Runs on the
- * cluster-partitioned kernel (dense bf16 models, two or more active rows), else on the any-shape kernel.
+ * [n_total] in the original order.  B <= max_batch given at create.  Asynchronous on cuda_stream.  Dense bf16 models run
+ * on the cluster-partitioned kernel while two or more rows are active and on the resident kernel while one is (the ramps
+ * of the schedule); everything else on the any-shape kernel.
  * wrnn_subscale_conditioning computes v_row[0..L) alone from a given history (DEVICE int16 [B][L]) into
  * v (DEVICE [L][cond_dim]).
  */

@@ -197,7 +197,11 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     int rc = cond_project(m, a.cond, a.batch, nf, s);
     if (rc != WRNN_OK) return fail(m, rc, "conditioning projection launch failed");
     // staggered rows: the cluster-partitioned kernel, else the any-shape kernel
-    if (a.row_lag > 0) return a.batch >= 2 && use_bcluster(m, a.batch) ? bcluster_run(m, a, s) : generic_run(m, a, s);
+    if (a.row_lag > 0) {
+        if (a.batch >= 2 && use_bcluster(m, a.batch)) return bcluster_run(m, a, s);
+        if (a.batch == 1 && use_resident(m, 1)) return resident_run(m, a, s);     // a lone row (the ramps of the schedule)
+        return generic_run(m, a, s);
+    }
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
     if (use_resf32(m, a.batch)) return resf32_run(m, a, s);
     if (use_sparse(m, a.batch)) return sparse_run(m, a, s);

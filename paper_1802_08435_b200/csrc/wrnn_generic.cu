@@ -319,25 +319,35 @@ __global__ void subscale_cond_kernel(const int16_t *__restrict__ hist, const flo
                                      const float *__restrict__ bias, float *__restrict__ v, int B, long long L, int F, int D,
                                      int n_frames, int hop, int r_lo, long long p_lo, int lag, int n_steps)
 {
+    // one block per (row, step): threadIdx.x = output channel (strided), threadIdx.y = one of four slices of the (earlier
+    // row, offset) pairs; the slices meet in shared memory
+    extern __shared__ float cpart[];                 // [4][D]
     const int b = blockIdx.y, c = blockIdx.x, r = r_lo + b;
     const long long pos = p_lo - (long long)b * lag + c;
+    const int n_pairs = r * (F + 1);
     for (int k = threadIdx.x; k < D; k += blockDim.x) {
-        float acc = bias[k];
-        for (int delta = 1; delta <= r; ++delta) {
-            const int16_t *hz = hist + (size_t)(r - delta) * L;
-            const float *Vz = V + (size_t)(delta - 1) * (F + 1) * D + k;
-            for (int d = 0; d <= F && pos + d < L; ++d) acc = fmaf(Vz[(size_t)d * D], (float)hz[pos + d] * (1.0f / 32768.0f), acc);
+        float acc = 0.f;
+        for (int j = threadIdx.y; j < n_pairs; j += blockDim.y) {
+            const int delta = j / (F + 1) + 1, d = j - (delta - 1) * (F + 1);
+            if (pos + d < L)
+                acc = fmaf(V[((size_t)(delta - 1) * (F + 1) + d) * D + k], (float)hist[(size_t)(r - delta) * L + pos + d] * (1.0f / 32768.0f), acc);
         }
-        const long long fr = ((long long)B * pos + r) / hop;
-        v[((size_t)b * n_steps + c) * D + k] = frames[((size_t)r * n_frames + fr) * D + k] + fmaxf(acc, 0.f);
+        cpart[threadIdx.y * D + k] = acc;
     }
+    __syncthreads();
+    if (threadIdx.y == 0)
+        for (int k = threadIdx.x; k < D; k += blockDim.x) {
+            const float acc = bias[k] + ((cpart[k] + cpart[D + k]) + (cpart[2 * D + k] + cpart[3 * D + k]));
+            const long long fr = ((long long)B * pos + r) / hop;
+            v[((size_t)b * n_steps + c) * D + k] = frames[((size_t)r * n_frames + fr) * D + k] + fmaxf(acc, 0.f);
+        }
 }
 
 int subscale_cond_launch(const int16_t *hist, const float *frames, const float *V, const float *bias, float *v, int B, long long L, int F,
                          int D, int n_frames, int hop, int r_lo, int n_rows, long long p_lo, int lag, int n_steps, cudaStream_t s)
 {
     if (n_rows <= 0 || n_steps <= 0) return WRNN_OK;
-    subscale_cond_kernel<<<dim3(n_steps, n_rows), 64, 0, s>>>(hist, frames, V, bias, v, B, L, F, D, n_frames, hop, r_lo, p_lo, lag, n_steps);
+    subscale_cond_kernel<<<dim3(n_steps, n_rows), dim3(64, 4), (size_t)4 * D * sizeof(float), s>>>(hist, frames, V, bias, v, B, L, F, D, n_frames, hop, r_lo, p_lo, lag, n_steps);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
 }

@@ -53,6 +53,7 @@ struct ResidentParams {
     unsigned stream0;
     unsigned long long seed;
     int n_frames, hop, row_stride, row_offset_mul;
+    long long frame_shift;                   // subtracted from the frame index (a call whose conditioning starts at its first step)
     const uint8_t *blob; unsigned long long blob_bytes, w_bytes;
     const float *g;                          // [n_frames][3H]
     unsigned long long *slots;               // [2][2][K]
@@ -264,7 +265,7 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
         if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
     };
     auto load_g = [&](int half_g, long long s, float (&gv)[3]) {
-        const long long fr = ((p.step0 + s) * p.row_stride + (long long)p.stream0 * p.row_offset_mul) / p.hop;
+        const long long fr = ((p.step0 + s) * p.row_stride + (long long)p.stream0 * p.row_offset_mul) / p.hop - p.frame_shift;
         const float *g = p.g + (size_t)fr * 3 * H + (half_g ? K : 0) + cta * UC + lane;
 #pragma unroll
         for (int gate = 0; gate < 3; ++gate) gv[gate] = __ldg(g + gate * H);
@@ -724,6 +725,7 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in; p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
+    p.frame_shift = a.row_lag > 0 ? a.step0 : 0;          // staggered rows bring one frame per step of the call
     p.a_in = a.a_in; p.b_in = a.b_in; p.a_st_out = a.a_st_out; p.b_st_out = a.b_st_out;
     p.a_forced = a.a_forced; p.b_forced = a.b_forced; p.a_out = a.a_out; p.b_out = a.b_out;
     p.status = m->status;

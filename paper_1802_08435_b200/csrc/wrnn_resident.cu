@@ -9,9 +9,10 @@
 //     inside every cluster (bit-identically) and never have to be broadcast across the chip.
 // Per step there are exactly two chip-wide exchanges through L2 -- y_c(t) before the coarse head and
 // y_f(t) before the fine head (Fig. 1's order) -- each an all-gather of (value, step-tag) words so
-// that arrival of the data is the signal.  Inside a cluster the hidden layer and the logits travel
-// through distributed shared memory the same way.  The fine head of step t overlaps the recurrent
-// product of step t+1 (f_t is only needed by the coarse gates of t+1).
+// that arrival of the data is the signal.  Inside a cluster the logits travel through distributed
+// shared memory the same way (one warp consumes them), the hidden layer by asynchronous stores that
+// complete an mbarrier at the receiver (every warp of the CTA consumes it: nobody polls).  The fine head
+// of step t overlaps the recurrent product of step t+1 (f_t is only needed by the coarse gates of t+1).
 //
 // Mat-vec products run on the tensor pipe as m16n8k16 bf16 MMAs: the weights sit in shared memory
 // in A-fragment order (one 16-byte load per lane per 16x16 tile), and the fp32 input vector is split

@@ -227,6 +227,11 @@ int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n
 int wrnn_subscale_conditioning(const int16_t *hist, const float *frames, const float *V, const float *bias, int32_t B,
                                int64_t L, int32_t F, int32_t cond_dim, int32_t n_frames, int32_t hop, int32_t row, float *v,
                                void *cuda_stream);
+/* The stepping launches of that schedule, in order, without running anything (host only, no device needed): call i is
+ * calls[4 i .. 4 i + 3] = (first row, number of rows, position of the first row, steps); row b of a call is at the
+ * first row's position minus b * lag.  HOST calls[max_calls][4].  Returns the number of launches of the schedule (which
+ * may exceed max_calls: only the first max_calls are written), or minus a wrnn_status for bad arguments. */
+int wrnn_subscale_schedule(int32_t B, int64_t L, int32_t chunk, int32_t lag, int64_t *calls, int32_t max_calls);
 
 /*
  * Host-buffer convenience for callers without device pointers: copies cond

@@ -27,7 +27,7 @@ EXPORTS = [
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
     "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor", "wrnn_sample_noalloc",
     "wrnn_selftest_bounded_wait", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold", "wrnn_fs2_sample_host",
-    "wrnn_sample_subscale_dependent", "wrnn_subscale_conditioning",
+    "wrnn_sample_subscale_dependent", "wrnn_subscale_conditioning", "wrnn_subscale_schedule",
 ]
 
 
@@ -86,6 +86,7 @@ def lib():
         L.wrnn_fs2_unfold.argtypes = [vp, i64, vp, vp]
         L.wrnn_fs2_sample_host.argtypes = [vp, vp, i32, i32, i64, u64, vp]
         L.wrnn_sample_subscale_dependent.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i64, i32, u64, vp, vp]
+        L.wrnn_subscale_schedule.argtypes = [i32, i64, i32, i32, vp, i32]
         L.wrnn_subscale_conditioning.argtypes = [vp, vp, vp, vp, i32, i64, i32, i32, i32, i32, i32, vp, vp]
         L.wrnn_fold.argtypes = [vp, i64, i32, vp, vp]
         L.wrnn_unfold.argtypes = [vp, i64, i32, vp, vp]
@@ -251,6 +252,17 @@ def wrnn_sample_subscale_dependent(model, frames, V, bias, F: int, chunk: int, l
     V: CUDA float32 [B-1][F+1][D]; bias: CUDA float32 [D]; out: CUDA int16 [n_total] in the original order."""
     _check(lib().wrnn_sample_subscale_dependent(model, _dev_ptr(frames), int(frames.shape[1]), hop, _dev_ptr(V), _dev_ptr(bias), F,
                                                 chunk, lag, n_total, B, seed, _dev_ptr(out), _stream_ptr(stream)), model)
+
+
+def wrnn_subscale_schedule(B: int, L: int, chunk: int, lag: int):
+    """The stepping launches of the staggered schedule as a list of (first row, rows, position of the first row, steps).
+    Host arithmetic only: works without a GPU."""
+    n = lib().wrnn_subscale_schedule(B, L, chunk, lag, None, 0)
+    if n < 0:
+        raise WrnnError(-n, "bad schedule arguments")
+    buf = (C.c_int64 * (4 * max(n, 1)))()
+    lib().wrnn_subscale_schedule(B, L, chunk, lag, buf, n)
+    return [tuple(buf[4 * i: 4 * i + 4]) for i in range(n)]
 
 
 def wrnn_subscale_conditioning(hist, frames, V, bias, F: int, row: int, v, *, hop: int = 120, stream=None):

@@ -230,6 +230,29 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     return generic_run(m, a, s);
 }
 
+// The stepping calls of the staggered subscale schedule (Section 4.2), in launch order: global time advances one chunk
+// per iteration, row r is at position k * chunk - r * lag and active while that lies in [0, L); the active rows are
+// contiguous; a row that ends inside a chunk gets a call of its own (all rows of a call run the same number of steps).
+struct SubCall { int r_lo, n_rows; long long p_lo; int n_steps; };
+static void subscale_schedule(int B, long long L, int chunk, int lag, std::vector<SubCall> *calls)
+{
+    for (long long k = 0;; ++k) {
+        const long long t = k * chunk;
+        if (t - (long long)(B - 1) * lag >= L) break;                       // the last row is done
+        const int r_hi = (int)std::min<long long>(B - 1, t / lag);
+        int r_lo = t >= L ? (int)((t - L) / lag) + 1 : 0;
+        if (r_lo > r_hi) continue;                                          // a gap between rows (lag > L)
+        const long long p_lo = t - (long long)r_lo * lag;
+        const long long left = L - p_lo;
+        if (left < chunk) {                                                 // the oldest active row ends inside this chunk
+            calls->push_back({r_lo, 1, p_lo, (int)left});
+            ++r_lo;
+            if (r_lo > r_hi) continue;
+        }
+        calls->push_back({r_lo, r_hi - r_lo + 1, t - (long long)r_lo * lag, chunk});
+    }
+}
+
 }  // namespace wrnn
 
 using namespace wrnn;
@@ -498,6 +521,17 @@ int wrnn_sample_subscale(wrnn_model *m, const float *cond, int32_t n_frames, int
     return fold_launch(m->stage_out, n_total, B, out, true, (cudaStream_t)cuda_stream);
 }
 
+int wrnn_subscale_schedule(int32_t B, int64_t L, int32_t chunk, int32_t lag, int64_t *calls, int32_t max_calls)
+{
+    if (B < 1 || L < 1 || chunk < 1 || lag < chunk || lag % chunk != 0 || max_calls < 0 || (max_calls > 0 && !calls)) return -WRNN_ERR_INVALID_ARG;
+    std::vector<SubCall> v;
+    subscale_schedule(B, L, chunk, lag, &v);
+    for (size_t i = 0; i < v.size() && i < (size_t)max_calls; ++i) {
+        calls[4 * i] = v[i].r_lo; calls[4 * i + 1] = v[i].n_rows; calls[4 * i + 2] = v[i].p_lo; calls[4 * i + 3] = v[i].n_steps;
+    }
+    return (int)v.size();
+}
+
 int wrnn_subscale_conditioning(const int16_t *hist, const float *frames, const float *V, const float *bias, int32_t B, int64_t L,
                                int32_t F, int32_t cond_dim, int32_t n_frames, int32_t hop, int32_t row, float *v, void *cuda_stream)
 {
@@ -555,22 +589,10 @@ int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n
         a.row_lag = lag; a.out_pitch = L - lag;
         return run_steps(m, a, s);
     };
-    // global time advances by one chunk per iteration; row r is at position k * chunk - r * lag
-    for (long long k = 0;; ++k) {
-        const long long t = k * chunk;
-        if (t - (long long)(B - 1) * lag >= L) break;                       // the last row is done
-        const int r_hi = (int)std::min<long long>(B - 1, t / lag);
-        int r_lo = t >= L ? (int)((t - L) / lag) + 1 : 0;
-        if (r_lo > r_hi) continue;                                          // a gap between rows (lag > L)
-        const long long p_lo = t - (long long)r_lo * lag;
-        const long long left = L - p_lo;
-        if (left < chunk) {                                                 // the oldest active row ends inside this chunk
-            int rc = run_rows(r_lo, 1, p_lo, (int)left);
-            if (rc != WRNN_OK) return rc;
-            ++r_lo;
-            if (r_lo > r_hi) continue;
-        }
-        int rc = run_rows(r_lo, r_hi - r_lo + 1, t - (long long)r_lo * lag, chunk);
+    std::vector<SubCall> calls;
+    subscale_schedule(B, L, chunk, lag, &calls);
+    for (const SubCall &c : calls) {
+        const int rc = run_rows(c.r_lo, c.n_rows, c.p_lo, c.n_steps);
         if (rc != WRNN_OK) return rc;
     }
     return fold_launch(hist, n_total, B, out, true, s);

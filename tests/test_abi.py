@@ -68,3 +68,33 @@ def test_create_without_a_device_fails_loudly(libpath):
     with pytest.raises(binding.WrnnError) as e:
         binding.wrnn_create(w, "f32")
     assert e.value.code in (binding.WRNN_ERR_CUDA, binding.WRNN_ERR_UNSUPPORTED)
+
+
+@pytest.mark.parametrize("B,L,F,chunk,lag", [(16, 1500, 128, 128, 256), (4, 90, 6, 3, 9), (5, 64, 8, 8, 16), (3, 10, 2, 4, 8),
+                                           (4, 40, 4, 4, 64), (1, 33, 5, 8, 16), (8, 1000, 128, 64, 192)])
+def test_staggered_subscale_schedule(B, L, F, chunk, lag):
+    """Host logic of the staggered schedule (Section 4.2): every (row, position) is generated exactly once, in order;
+    whenever row r generates positions up to p, row r - 1 has already finished position p + F (the future horizon),
+    i.e. the conditioning of a whole call can be computed before it starts; the batch ramps up to min(B, ...) rows."""
+    from paper_1802_08435_b200 import binding
+    assert lag >= F + chunk and lag % chunk == 0
+    calls = binding.wrnn_subscale_schedule(B, L, chunk, lag)
+    done = [0] * B                       # positions finished per row
+    active = {}                          # rows stepping at a global time (a row that ends inside a chunk has a call of its own)
+    for (r_lo, n_rows, p_lo, n) in calls:
+        assert n_rows >= 1 and 1 <= n <= chunk and 0 <= r_lo and r_lo + n_rows <= B
+        t = p_lo + r_lo * lag
+        active[t] = active.get(t, 0) + n_rows
+        for b in range(n_rows):          # check against the state BEFORE this call (all its rows advance together)
+            r, p = r_lo + b, p_lo - b * lag
+            assert p == done[r], "rows advance contiguously"
+            assert p + n <= L
+            if r > 0:
+                need = min(L, p + n - 1 + F + 1)          # positions [0, need) of row r - 1 feed this call's conditioning
+                assert done[r - 1] >= need, (r, p, n, done[r - 1])
+        for b in range(n_rows):
+            done[r_lo + b] += n
+    assert done == [L] * B
+    assert max(active.values()) == min(B, (L + lag - 1) // lag)
+    with pytest.raises(binding.WrnnError):
+        binding.wrnn_subscale_schedule(B, L, chunk, lag + 1)

@@ -216,8 +216,8 @@ int wrnn_sample_subscale(wrnn_model *m, const float *cond, int32_t n_frames, int
  * stream id r, step = position, conditioning vector v_r[i] at step i.  The result does not depend on chunk or lag.
  * frames: DEVICE [B][n_frames][cond_dim]; V: DEVICE [B-1][F+1][cond_dim]; bias: DEVICE [cond_dim]; out: DEVICE int16
  * [n_total] in the original order.  B <= max_batch given at create.  Asynchronous on cuda_stream.  Dense bf16 models run
- * on the cluster-partitioned kernel while two or more rows are active and on the resident kernel while one is (the ramps
- * of the schedule); everything else on the any-shape kernel.
+ * on the cluster-partitioned kernel while four or more rows are active and row by row on the resident kernel while fewer
+ * are (the ramps of the schedule); everything else on the any-shape kernel.
  * wrnn_subscale_conditioning computes v_row[0..L) alone from a given history (DEVICE int16 [B][L]) into
  * v (DEVICE [L][cond_dim]).
  */

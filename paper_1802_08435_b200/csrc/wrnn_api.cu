@@ -579,15 +579,24 @@ int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n
     auto run_rows = [&](int r_a, int n_rows, long long p_lo, int n) -> int {
         int rc = subscale_cond_launch(hist, frames, V, bias, v, B, L, F, D, n_frames, hop, r_a, n_rows, p_lo, lag, n, s);
         if (rc != WRNN_OK) return fail(m, rc, "conditioning launch failed");
-        StepArgs a;
-        std::memset(&a, 0, sizeof(a));
-        a.cond = v; a.n_frames = n; a.hop = 1; a.row_stride = 1; a.row_offset_mul = 0;
-        a.n_steps = n; a.batch = n_rows; a.seed = seed; a.step0 = p_lo; a.stream0 = (unsigned)r_a;
-        a.h_in = a.h_out = hst + (size_t)r_a * H;
-        a.c_in = a.c_st_out = cp + r_a; a.f_in = a.f_st_out = fp + r_a;
-        a.out = hist + (size_t)r_a * L + p_lo;
-        a.row_lag = lag; a.out_pitch = L - lag;
-        return run_steps(m, a, s);
+        // up to three rows go one after the other through the single-stream kernel where the model has one (6.6 us per
+        // step and row against 24 us per step of the multi-row kernel); more rows advance together
+        const int group = (n_rows <= 3 && use_resident(m, 1)) ? 1 : n_rows;
+        for (int b0 = 0; b0 < n_rows; b0 += group) {
+            const int r0 = r_a + b0;
+            const long long p0 = p_lo - (long long)b0 * lag;
+            StepArgs a;
+            std::memset(&a, 0, sizeof(a));
+            a.cond = v + (size_t)b0 * n * D; a.n_frames = n; a.hop = 1; a.row_stride = 1; a.row_offset_mul = 0;
+            a.n_steps = n; a.batch = group; a.seed = seed; a.step0 = p0; a.stream0 = (unsigned)r0;
+            a.h_in = a.h_out = hst + (size_t)r0 * H;
+            a.c_in = a.c_st_out = cp + r0; a.f_in = a.f_st_out = fp + r0;
+            a.out = hist + (size_t)r0 * L + p0;
+            a.row_lag = lag; a.out_pitch = L - lag;
+            rc = run_steps(m, a, s);
+            if (rc != WRNN_OK) return rc;
+        }
+        return WRNN_OK;
     };
     std::vector<SubCall> calls;
     subscale_schedule(B, L, chunk, lag, &calls);

@@ -16,7 +16,9 @@
  * fine gates (I* lets c_t reach only the fine half), draw f_t; the 16-bit sample is
  * 256 c_t + f_t.  g = W_cond frame + b_gate is the per-step conditioning vector
  * (held for `hop` samples).  Dense (Section 2.1), 4x4 block-sparse (Section 3.2)
- * and batched / subscale-folded (Section 4) forms share these entry points.
+ * and batched / subscale-folded (Section 4) forms share these entry points; the Fused Subscale
+ * WaveRNN 2x (Section 4.4, wrnn_fs2_*) and subscale generation with dependent rows on the staggered
+ * schedule (Sections 4.1, 4.2, wrnn_sample_subscale_dependent) are built on the same step.
  *
  * Conventions: C linkage; every function returns a wrnn_status (0 = ok) unless
  * noted; pointers are marked HOST or DEVICE; the caller owns every buffer it

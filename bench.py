@@ -318,7 +318,11 @@ def main():
                     "traffic_note": "DRAM bytes per launch from the ncu capture in profiles/ (one-time weight load; "
                                     "does not grow with the number of steps)",
                     "peak_source": "derived: 148 SMs x 128 B/clk x 1.965 GHz", "algorithmic_bytes_per_step": alg_bytes,
-                    "resident_bytes_read_per_step": wbytes}
+                    "resident_bytes_read_per_step": wbytes,
+                    # the same bytes per second against the measured HBM copy bandwidth: what a kernel that streamed the
+                    # weights from DRAM once per step would be held to (the weights are in fact resident on-chip)
+                    "hbm_equivalent": {"achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                                       "peak_source": peaks["source"]}}
             if info["kernel"] == 2:
                 t_bar_ns = B.wrnn_measure_exchange_floor(info["n_ctas"], info["n_threads"], Hh, 20000)
                 smem_us = alg_bytes / (SMEM_PEAK_GBS * 1e3)

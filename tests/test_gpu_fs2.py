@@ -112,3 +112,31 @@ def test_variant_gating(env):
         B.wrnn_destroy(base)
     with pytest.raises(B.WrnnError):      # the variant exists for dense bf16 single-stream models only
         B.wrnn_create(w, "f32", max_batch=1, variant=1)
+
+
+def test_short_runs_and_unfold_sizes(env):
+    """One, two and three steps: the first two samples of part B are pre-roll, so the unfold of n steps has 2 (n - 2)
+    samples; short calls chained through the carry state reproduce a longer run."""
+    torch, B, w, m = env
+    dev = "cuda:0"
+    cd = torch.from_numpy(synth.make_cond(1, 3)).to(dev)
+    full = torch.zeros((2, 6), dtype=torch.int16, device=dev)
+    B.wrnn_fs2_sample(m, cd, 6, SEED, full, hop=synth.HOP)
+    h = torch.zeros((H,), dtype=torch.float32, device=dev)
+    ap = torch.full((1,), -32768, dtype=torch.int16, device=dev)
+    bp = torch.full((1,), -32768, dtype=torch.int16, device=dev)
+    pieces, pos = [], 0
+    for n in (1, 2, 3):
+        o = torch.zeros((2, n), dtype=torch.int16, device=dev)
+        B.wrnn_fs2_sample(m, cd, n, SEED, o, hop=synth.HOP, h=h, a_prev=ap, b_prev=bp, step0=pos)
+        pieces.append(o.cpu().numpy()); pos += n
+    torch.cuda.synchronize()
+    assert np.array_equal(np.concatenate(pieces, axis=1), full.cpu().numpy())
+    for n in (1, 2, 3, 6):
+        u = torch.full((max(2 * (n - 2), 1),), 77, dtype=torch.int16, device=dev)
+        B.wrnn_fs2_unfold(full[:, :n].contiguous(), n, u)
+        torch.cuda.synchronize()
+        ref = orc.fs2_unfold(full[:, :n].cpu().numpy())
+        assert np.array_equal(u.cpu().numpy()[: ref.size], ref)
+        if n <= 2:
+            assert int(u.cpu()[0]) == 77          # nothing written

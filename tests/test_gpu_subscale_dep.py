@@ -103,3 +103,35 @@ def test_argument_errors(env):
             assert e.value.code == 1
     finally:
         Bn.wrnn_destroy(m)
+
+
+def test_edge_shapes(env):
+    """One sub-tensor (no earlier row: an ordinary stream), a row shorter than a chunk, and an empty request."""
+    torch, Bn = env
+    dev = "cuda:0"
+    w, V, b, frames = _case(64, 1, 50, 4)
+    om = orc.OracleModel(w, "f32")
+    m = Bn.wrnn_create(w, "f32", max_batch=4)
+    try:
+        one = _gpu_run(torch, Bn, m, frames, V, b, 4, 8, 16, 1, 50)
+        ref, _, margins = orc.subscale_dependent_run(om, frames, V, b, 1, 50, synth.HOP, SEED)
+        d = np.nonzero(one != ref[0])[0]
+        assert d.size == 0 or margins[0, d[0]].min() < pu.MARGIN
+        # rows of 5 positions with chunks of 8: every call is a short one
+        w3, V3, b3, fr3 = _case(64, 3, 5, 2)
+        m3 = Bn.wrnn_create(w3, "f32", max_batch=3)
+        try:
+            got = orc.fold(_gpu_run(torch, Bn, m3, fr3, V3, b3, 2, 8, 16, 3, 5), 3)
+            ref3, _, mg3 = orc.subscale_dependent_run(orc.OracleModel(w3, "f32"), fr3, V3, b3, 3, 5, synth.HOP, SEED)
+            for row in range(3):
+                d = np.nonzero(got[row] != ref3[row])[0]
+                if d.size:
+                    assert mg3[row, d[0]].min() < pu.MARGIN
+                    break
+        finally:
+            Bn.wrnn_destroy(m3)
+        out = torch.zeros((4,), dtype=torch.int16, device=dev)
+        Bn.wrnn_sample_subscale_dependent(m, torch.from_numpy(frames).to(dev), torch.from_numpy(V).to(dev), torch.from_numpy(b).to(dev), 4, 8, 16,
+                                          0, 1, SEED, out)       # nothing to do
+    finally:
+        Bn.wrnn_destroy(m)

@@ -39,6 +39,8 @@ struct SliceMeta { int voff, coff, T, nl, lpr, pad[3]; int16_t row[8]; };   // o
 
 struct SparsePack {
     int H = 0, K = 0, NKT = 0, UC = 0, HR = 0, NBR = 0;   // NBR: block rows per phase = (HR + 6 UC) / rows of a block
+    int NC = 1;                       // clusters: the rows of R are dealt over NC x 16 CTAs, the heads once per cluster
+    unsigned long long *d_slots = nullptr;   // [4][K] exchange slots of the state halves
     int tall = 0;                     // 16 x 1 blocks (else 4 x 4)
     int max_slots = 0;                // block slots per phase per CTA (kept blocks + padding of the sliced layout, maximum)
     size_t blob_bytes = 0;            // per CTA
@@ -50,6 +52,7 @@ struct SparsePack {
 
 struct SparseParams {
     int H, K, NKT, UC, HR, NBR, tall;        // tall: blocks are 16 x 1 (16 rows of one column) instead of 4 x 4
+    unsigned long long *yslots;              // [2 halves][2 parities][K] (value, tag): the state crosses the chip when there is more than one cluster
     unsigned long long off_meta[2], off_col[2], off_val[2], off_o2, off_o4, off_small, blob_bytes;
     long long n_steps, step0;
     unsigned stream0;
@@ -80,7 +83,8 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
 {
     extern __shared__ __align__(16) uint8_t smem[];
     cg::cluster_group cluster = cg::this_cluster();
-    const int rank = (int)cluster.block_rank();
+    const int rank = (int)cluster.block_rank();      // owner index of head rows and logits (per cluster)
+    const int cta = blockIdx.x;                      // owner index of state units and their rows of R (whole grid)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int K = p.K, NKT = p.NKT, UC = p.UC, HR = p.HR, H = p.H;
     const int NR = 6 * UC;
@@ -98,19 +102,18 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     float *a_part = qvec + K;                                                         // [NR]
     float *a_full = a_part + NR;                                                      // [NR]
     float *part = a_full + NR;                                                        // [16 warps][16]
-    float *ynew = part + 256;                                                         // [UC] freshly gated units
-    __nv_bfloat16 *splQ = reinterpret_cast<__nv_bfloat16 *>(ynew + ((UC + 3) & ~3));  // split image of q, 4 K bf16
-    // Exchange buffers, one of each: a peer can only write the next half-step's words after it has received words that
-    // this CTA sent after reading the current ones (y(n+1) follows q(n), q(n+1) follows y(n+1), logits(n+1) follow q(n+1)).
-    uint4 *ybuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                            // [K/2] state half
-    uint4 *qbuf = ybuf + K / 2;                                                       // [K/2] hidden layer
+    __nv_bfloat16 *splQ = reinterpret_cast<__nv_bfloat16 *>(part + 256);              // split image of q, 4 K bf16
+    // Cluster exchange buffers, one of each: a peer can only write the next half-step's words after it has received
+    // words that this CTA sent after reading the current ones (q(n+1) follows y(n+1), which follows this CTA's draw from
+    // logits(n); logits(n+1) follow q(n+1)).
+    uint4 *qbuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                            // [K/2] hidden layer
     uint4 *lbuf = qbuf + K / 2;                                                       // [128] logits
 
     {
-        const uint4 *src = reinterpret_cast<const uint4 *>(p.blob + (size_t)rank * p.blob_bytes);
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.blob + (size_t)cta * p.blob_bytes);
         uint4 *dst = reinterpret_cast<uint4 *>(smem);
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
-        for (int i = tid; i < K + 128; i += blockDim.x) ybuf[i] = make_uint4(0, 0, 0, 0);   // ybuf, qbuf, lbuf are adjacent
+        for (int i = tid; i < K / 2 + 128; i += blockDim.x) qbuf[i] = make_uint4(0, 0, 0, 0);   // qbuf, lbuf are adjacent
         for (int i = tid; i < 4 * K / 8; i += blockDim.x) reinterpret_cast<uint4 *>(splQ)[i] = make_uint4(0, 0, 0, 0);
         for (int i = tid; i < K; i += blockDim.x) {
             vecC[i] = p.h_in ? p.h_in[i] : 0.f;
@@ -122,7 +125,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
 
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
-    const bool writer = (rank == 0);
+    const bool writer = (cta == 0);
 #ifdef WRNN_PROFILE_SPARSE
     __shared__ long long s_sprof[16];
     long long st_ = clock64();
@@ -148,6 +151,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
 
     auto sparse_phase = [&](int ph, const float *x, const float *bias) {
         const int nl = ph ? sl_nl1 : sl_nl0, T = ph ? sl_T1 : sl_T0, l4 = lane & 3;
+        if (nl == 0) return;                       // a warp without block rows (few rows per CTA): its slice has no slots to read
         const uint4 *wv = ph ? sl_wv1 : sl_wv0;
         const uint16_t *wc = ph ? sl_wc1 : sl_wc0;
         if (tall) {
@@ -234,14 +238,14 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         }
     };
 
-    // Gates of Eq. 2 for this CTA's UC units of one half, then publish them to all 16 CTAs.  The first GW warps
+    // Gates of Eq. 2 for this CTA's UC units of one half, then publish them to the whole grid.  The first GW warps
     // each draw the sample redundantly (same logits, same uniform, same instructions -> same value) and then gate
     // UC / GW units each, so that neither the gates nor the 16 x UC / 2 remote stores queue up in one warp.
     constexpr int GW = 4;
     const int UW = UC / GW;
     auto load_g = [&](int half_g, long long s, float (&gv)[3]) {
         const long long fr = ((p.step0 + s) * p.row_stride + (long long)p.stream0 * p.row_offset_mul) / p.hop;
-        const float *g = p.g + (size_t)fr * 3 * H + (half_g ? K : 0) + rank * UC + warp * UW + lane;
+        const float *g = p.g + (size_t)fr * 3 * H + (half_g ? K : 0) + cta * UC + warp * UW + lane;
 #pragma unroll
         for (int gate = 0; gate < 3; ++gate) gv[gate] = __ldg(g + gate * H);
     };
@@ -259,7 +263,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             q.pe = fmaf(Ie[0], x0, half_g ? fmaf(Ie[1], x1, gv[2]) : gv[2]);
             q.ae = a_full[rb + 2 * UC + u0];
             q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
-            q.hprev = (half_g ? vecF : vecC)[rank * UC + u0];       // previous value of the unit: still in the fp32 vector of that half
+            q.hprev = (half_g ? vecF : vecC)[cta * UC + u0];       // previous value of the unit: still in the fp32 vector of that half
         }
         return q;
     };
@@ -270,22 +274,14 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
             const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
             const float hn = fmaf(u, q.hprev, (1.0f - u) * e);
-            ynew[u0] = hn;
-            const int jj = (half_g ? K : 0) + rank * UC + u0;
+            // published to the whole chip: arrival of the tagged value is the signal (two-deep by step parity)
+            st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + cta * UC + u0,
+                           ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+            const int jj = (half_g ? K : 0) + cta * UC + u0;
             if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
             if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
         }
     };
-    // the UC freshly gated values -> every peer (warp w -> peer w, one coalesced store), after a CTA barrier
-    auto publish = [&](unsigned ytag) {
-        if (warp < SCS) {
-            for (int pr2 = lane; pr2 < UC / 2; pr2 += 32) {
-                const unsigned a = map_to_rank(smem_addr(ybuf + (rank * UC) / 2 + pr2), warp);
-                st_cluster_ll(a, ynew[2 * pr2], ynew[2 * pr2 + 1], ytag);
-            }
-        }
-    };
-
     // ---- prologue: R h of step 0 from the initial state, coarse gates of step 0
     sparse_phase(0, vecC, sb1);
     __syncthreads();
@@ -296,8 +292,6 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         if (lane < UW) load_g(0, 0, gv0);
         gates(0, 0, f_prev, gates_prepare(0, gv0));
     }
-    __syncthreads();
-    publish(1u);
 
     const int l_kt0 = warp * NKL;
     const int KSL = NKT / NKL;                   // warps that split K of the logits tile
@@ -326,17 +320,21 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
         }
 
-        // ---- 1. the input half of the state from all 16 CTAs (published with tag n)
+        // ---- 1. the input half of the state from the whole grid (y_c(s) carries tag s + 1, y_f(s-1) tag s): two adjacent
+        // slots per polling thread
+        {
+            const unsigned long long *slots = p.yslots + (size_t)(half ? (s & 1) : 2 + ((s - 1) & 1)) * K;
+            const unsigned ytag = (unsigned)(half ? s + 1 : s);
 #pragma unroll 1
-        for (int i = tid; i < K / 2; i += blockDim.x) {
-            const unsigned a = smem_addr(ybuf + i);
-            uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
-            while (true) {
-                v = ld_shared_volatile_v4(a);
-                if (v.y == tag && v.w == tag) break;
-                if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+            for (int i = tid; i < K / 2; i += blockDim.x) {
+                unsigned long long v0, v1, t0 = 0; unsigned cnt = 0;
+                while (true) {
+                    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0), "=l"(v1) : "l"(slots + 2 * i) : "memory");
+                    if ((unsigned)(v0 >> 32) == ytag && (unsigned)(v1 >> 32) == ytag) break;
+                    if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+                }
+                vec[2 * i] = __uint_as_float((unsigned)v0); vec[2 * i + 1] = __uint_as_float((unsigned)v1);
             }
-            vec[2 * i] = __uint_as_float(v.x); vec[2 * i + 1] = __uint_as_float(v.z);
         }
         if (__syncthreads_or(my_bad)) break;
         SSTAMP(0);
@@ -435,8 +433,6 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             if (half) c_prev = drawn;
             SSTAMP(6);
         }
-        if (__syncthreads_or(my_bad)) break;
-        if (!last) publish((unsigned)(n + 1));
     }
 
 #ifdef WRNN_PROFILE_SPARSE
@@ -462,9 +458,8 @@ static int sparse_smem_bytes(const SparsePack &k)
     b += (size_t)3 * k.K * 4;                      // vecC, vecF, qvec
     b += (size_t)2 * 6 * k.UC * 4;                 // a_part, a_full
     b += 256 * 4;                                  // part
-    b += (size_t)((k.UC + 3) & ~3) * 4;            // ynew
     b += (size_t)4 * k.K * 2;                      // split image of q
-    b += (size_t)k.K * 16;                         // ybuf, qbuf: [K/2] x 16 B each
+    b += (size_t)k.K * 8;                          // qbuf: [K/2] x 16 B
     b += 128 * 16;                                 // lbuf
     return (int)b;
 }
@@ -488,7 +483,7 @@ static void *sparse_fn() { return (void *)sparse_cluster_kernel<8>; }
 static void sparse_fill_launch(const SparsePack &k, cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at, cudaStream_t s, bool coop)
 {
     std::memset(cfg, 0, sizeof(*cfg));
-    cfg->gridDim = dim3(SCS);
+    cfg->gridDim = dim3(SCS * k.NC);
     cfg->blockDim = dim3(SNW * 32);
     cfg->dynamicSmemBytes = k.smem_bytes;
     cfg->stream = s;
@@ -508,196 +503,227 @@ int sparse_prepare(wrnn_model *m)
     const bool tall = m->mask_br == 16 && m->mask_bc == 1;
     if (!tall && (m->mask_br != 4 || m->mask_bc != 4)) { m->err = "single-cluster kernel takes 4 x 4 or 16 x 1 blocks"; return WRNN_ERR_UNSUPPORTED; }
     if (Hh != 1024) { m->err = "only H/2 = 1024 is instantiated (8 warps x 8 k-tiles for the logits tile)"; return WRNN_ERR_UNSUPPORTED; }
+    // The rows of R are dealt over NC clusters of 16 (the heads are held once per cluster); more clusters mean fewer block
+    // rows per CTA in the phase that dominates the step, at the price of the state crossing the chip through L2 instead
+    // of the cluster's shared memory.  The largest count that divides the units and can be co-resident is taken.
+    // WRNN_SPARSE_CLUSTERS = 1 / 2 / 4 forces one (diagnostic).
     SparsePack k;
-    k.H = H; k.K = Hh; k.NKT = Hh / 16; k.UC = Hh / SCS; k.HR = Hh / SCS;
-    const int BRH = tall ? 16 : 4;                                 // rows of one block
-    k.tall = tall ? 1 : 0;
-    k.NBR = (k.HR + 6 * k.UC) / BRH;
-    const int UC = k.UC, HR = k.HR, NBR = k.NBR, Kb = Hh / 4;      // Kb: 4-wide block columns per half
-    if (HR % BRH != 0 || UC % BRH != 0) { m->err = "block height does not divide the rows of one CTA"; return WRNN_ERR_UNSUPPORTED; }
+    std::vector<uint8_t> blob;
+    int64_t kept_bytes = 0;
+    auto pack = [&](int nc) -> int {
+    k = SparsePack();
+        k.NC = nc;
+        const int NCTA = nc * SCS;
+        k.H = H; k.K = Hh; k.NKT = Hh / 16; k.UC = Hh / NCTA; k.HR = Hh / SCS;
+        const int BRH = tall ? 16 : 4;                                 // rows of one block
+        k.tall = tall ? 1 : 0;
+        k.NBR = (k.HR + 6 * k.UC) / BRH;
+        const int UC = k.UC, HR = k.HR, NBR = k.NBR, Kb = Hh / 4;      // Kb: 4-wide block columns per half
+        if (Hh % NCTA != 0 || HR % BRH != 0 || UC % BRH != 0 || UC % 4 != 0) { m->err = "block height does not divide the rows of one CTA"; return WRNN_ERR_UNSUPPORTED; }
 
-    // kept blocks of each phase of each CTA.  A block is 16 weights: a 4 x 4 block row-major, or the 16 rows of one column;
-    // col is the block column (4 x 4) or the column (16 x 1) inside the phase's input half.
-    struct Blk { uint16_t col; float v[16]; };
-    std::vector<std::vector<std::vector<Blk>>> rows(SCS * 2);      // [cta * 2 + phase][local block row] -> blocks
-    const BsrHost *Oa[2] = {&m->hO1, &m->hO3};
-    for (int cta = 0; cta < SCS; ++cta)
-        for (int ph = 0; ph < 2; ++ph) {
-            auto &R = rows[cta * 2 + ph];
-            R.assign(NBR, {});
-            for (int lbr = 0; lbr < NBR; ++lbr) {
-                // the 4-row block rows of the source matrix under this block row, and the range of its 4-wide block columns
-                const BsrHost *M;
-                int br0, bc_lo, bc_hi;
-                if (lbr < HR / BRH) {
-                    M = Oa[ph];
-                    br0 = (cta * HR + lbr * BRH) / 4; bc_lo = 0; bc_hi = Kb;
-                } else {
-                    const int q = lbr - HR / BRH;                  // (half * 3 + gate) * (UC / BRH) + u
-                    const int half = q / (3 * (UC / BRH)), gate = (q / (UC / BRH)) % 3, u = q % (UC / BRH);
-                    M = &m->hR;
-                    br0 = (gate * H + half * Hh + cta * UC + u * BRH) / 4; bc_lo = ph * Kb; bc_hi = bc_lo + Kb;
-                }
-                if (!tall) {
-                    for (int i = M->row_ptr[br0]; i < M->row_ptr[br0 + 1]; ++i) {
-                        const int bc = M->col[i];
-                        if (bc < bc_lo || bc >= bc_hi) continue;
-                        Blk b;
-                        b.col = (uint16_t)(bc - bc_lo);
-                        std::memcpy(b.v, &M->vals[(size_t)i * 16], sizeof(b.v));
-                        R[lbr].push_back(b);
+        // kept blocks of each phase of each CTA.  A block is 16 weights: a 4 x 4 block row-major, or the 16 rows of one column;
+        // col is the block column (4 x 4) or the column (16 x 1) inside the phase's input half.
+        struct Blk { uint16_t col; float v[16]; };
+        std::vector<std::vector<std::vector<Blk>>> rows(NCTA * 2);      // [cta * 2 + phase][local block row] -> blocks
+        const BsrHost *Oa[2] = {&m->hO1, &m->hO3};
+        for (int cta = 0; cta < NCTA; ++cta)
+            for (int ph = 0; ph < 2; ++ph) {
+                const int rank = cta % SCS;                            // head rows go by the rank inside the cluster
+                auto &R = rows[cta * 2 + ph];
+                R.assign(NBR, {});
+                for (int lbr = 0; lbr < NBR; ++lbr) {
+                    // the 4-row block rows of the source matrix under this block row, and the range of its 4-wide block columns
+                    const BsrHost *M;
+                    int br0, bc_lo, bc_hi;
+                    if (lbr < HR / BRH) {
+                        M = Oa[ph];
+                        br0 = (rank * HR + lbr * BRH) / 4; bc_lo = 0; bc_hi = Kb;
+                    } else {
+                        const int q = lbr - HR / BRH;                  // (half * 3 + gate) * (UC / BRH) + u
+                        const int half = q / (3 * (UC / BRH)), gate = (q / (UC / BRH)) % 3, u = q % (UC / BRH);
+                        M = &m->hR;
+                        br0 = (gate * H + half * Hh + cta * UC + u * BRH) / 4; bc_lo = ph * Kb; bc_hi = bc_lo + Kb;
                     }
-                } else {
-                    // columns with a nonzero weight in any of the 16 rows, in ascending order
-                    std::vector<int> slot((size_t)4 * Kb, -1);
-                    std::vector<Blk> found;
-                    for (int r4 = 0; r4 < 4; ++r4)
-                        for (int i = M->row_ptr[br0 + r4]; i < M->row_ptr[br0 + r4 + 1]; ++i) {
+                    if (!tall) {
+                        for (int i = M->row_ptr[br0]; i < M->row_ptr[br0 + 1]; ++i) {
                             const int bc = M->col[i];
                             if (bc < bc_lo || bc >= bc_hi) continue;
-                            for (int c = 0; c < 4; ++c) {
-                                bool any = false;
-                                for (int r = 0; r < 4; ++r) any = any || M->vals[(size_t)i * 16 + 4 * r + c] != 0.f;
-                                if (!any) continue;
-                                const int col = 4 * (bc - bc_lo) + c;
-                                if (slot[col] < 0) { slot[col] = (int)found.size(); Blk b; b.col = (uint16_t)col; std::memset(b.v, 0, sizeof(b.v)); found.push_back(b); }
-                                for (int r = 0; r < 4; ++r) found[slot[col]].v[4 * r4 + r] = M->vals[(size_t)i * 16 + 4 * r + c];
-                            }
+                            Blk b;
+                            b.col = (uint16_t)(bc - bc_lo);
+                            std::memcpy(b.v, &M->vals[(size_t)i * 16], sizeof(b.v));
+                            R[lbr].push_back(b);
                         }
-                    std::sort(found.begin(), found.end(), [](const Blk &a, const Blk &b) { return a.col < b.col; });
-                    R[lbr] = found;
-                }
-            }
-        }
-    // slice every (CTA, phase): block rows sorted by length (longest first, stable), dealt to the warps in runs; the
-    // first w8 warps take four rows with eight lanes each, the others up to eight rows with four lanes each
-    struct Slice { std::vector<int> rows; int T = 0, lpr = 4; };
-    const int lpr_n = tall ? 16 : 4, cap_n = 32 / lpr_n, cap_w = cap_n / 2;     // lanes per row and rows per warp, narrow / wide slices
-    int w8 = (cap_n * SNW - NBR) / (cap_n - cap_w);                              // warps that can afford wide rows
-    if (w8 < 0) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
-    if (w8 > SNW) w8 = SNW;
-    if (w8 * cap_w > NBR) w8 = NBR / cap_w;
-    std::vector<std::vector<Slice>> slices(SCS * 2);              // [cta * 2 + phase][warp]
-    int max_slots = 0;
-    for (int cp = 0; cp < SCS * 2; ++cp) {
-        const auto &R = rows[cp];
-        std::vector<int> order(NBR);
-        for (int i = 0; i < NBR; ++i) order[i] = i;
-        std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return R[a].size() > R[b].size(); });
-        slices[cp].assign(SNW, {});
-        int next = 0, slots = 0;
-        for (int w = 0; w < SNW; ++w) {
-            Slice &sl = slices[cp][w];
-            sl.lpr = w < w8 ? 2 * lpr_n : lpr_n;
-            const int cap = 32 / sl.lpr;
-            // rows still to place, spread evenly over the remaining four-lane warps
-            int nr = cap;
-            if (w >= w8) { const int left = NBR - next, warps_left = SNW - w; nr = (left + warps_left - 1) / warps_left; }
-            if (nr > cap) nr = cap;
-            if (nr > NBR - next) nr = NBR - next;
-            size_t longest = 0;
-            for (int i = 0; i < nr; ++i) { sl.rows.push_back(order[next + i]); longest = std::max(longest, R[order[next + i]].size()); }
-            next += nr;
-            sl.T = (int)((longest + sl.lpr - 1) / sl.lpr);
-            if (sl.T < 1) sl.T = 1;                                  // the loop's first loads are unconditional
-            slots += sl.lpr * nr * sl.T;
-        }
-        if (next != NBR) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
-        max_slots = std::max(max_slots, slots);
-    }
-    k.max_slots = (max_slots + 7) & ~7;
-
-    size_t off = 0;
-    for (int ph = 0; ph < 2; ++ph) {
-        k.off_meta[ph] = off; off = a16(off + (size_t)SNW * sizeof(SliceMeta));
-        k.off_col[ph] = off; off = a16(off + (size_t)k.max_slots * 2);
-        k.off_val[ph] = off; off = a16(off + (size_t)k.max_slots * 32);
-    }
-    const size_t frag = (size_t)k.NKT * 512;
-    k.off_o2 = off; off += frag;
-    k.off_o4 = off; off += frag;
-    k.off_small = off; off = a16(off + ((size_t)6 * UC * 3 + 2 * HR + 32) * 4);
-    k.blob_bytes = off;
-    k.smem_bytes = sparse_smem_bytes(k);
-
-    cudaDeviceProp prop;
-    cudaGetDeviceProperties(&prop, m->device);
-    if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "pruned model does not fit the shared memory of one cluster"; return WRNN_ERR_UNSUPPORTED; }
-    if (cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-        cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
-        cudaGetLastError(); m->err = "cannot configure the 16-CTA cluster kernel"; return WRNN_ERR_UNSUPPORTED;
-    }
-    cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
-    sparse_fill_launch(k, &cfg, at, 0, false);
-    int max_clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&max_clusters, sparse_fn(), &cfg) != cudaSuccess || max_clusters < 1) {
-        cudaGetLastError(); m->err = "no 16-CTA cluster can be co-resident on this device"; return WRNN_ERR_UNSUPPORTED;
-    }
-
-    std::vector<uint8_t> blob((size_t)SCS * k.blob_bytes, 0);
-    const BsrHost *Ob[2] = {&m->hO2, &m->hO4};
-    int64_t kept_bytes = 0;
-    for (int cta = 0; cta < SCS; ++cta) {
-        uint8_t *base = blob.data() + (size_t)cta * k.blob_bytes;
-        for (int ph = 0; ph < 2; ++ph) {
-            SliceMeta *meta = reinterpret_cast<SliceMeta *>(base + k.off_meta[ph]);
-            uint16_t *col = reinterpret_cast<uint16_t *>(base + k.off_col[ph]);
-            uint16_t *val = reinterpret_cast<uint16_t *>(base + k.off_val[ph]);       // [slot plane][8 bf16]
-            const auto &R = rows[cta * 2 + ph];
-            int slot0 = 0, n = 0;
-            for (int w = 0; w < SNW; ++w) {
-                const Slice &sl = slices[cta * 2 + ph][w];
-                const int nl = sl.lpr * (int)sl.rows.size();
-                meta[w].voff = 2 * slot0; meta[w].coff = slot0; meta[w].T = sl.T; meta[w].nl = nl; meta[w].lpr = sl.lpr;
-                for (int g = 0; g < 8; ++g) meta[w].row[g] = g < (int)sl.rows.size() ? (int16_t)sl.rows[g] : (int16_t)-1;
-                for (int g = 0; g < (int)sl.rows.size(); ++g) {
-                    const auto &blocks = R[sl.rows[g]];
-                    for (int i = 0; i < (int)blocks.size(); ++i) {
-                        const int t = i / sl.lpr, lane = sl.lpr * g + i % sl.lpr;
-                        col[slot0 + t * nl + lane] = blocks[i].col;
-                        for (int h = 0; h < 2; ++h)                  // plane h holds rows 2 h, 2 h + 1 of the block
-                            for (int e = 0; e < 8; ++e)
-                                val[((size_t)2 * slot0 + (size_t)(2 * t + h) * nl + lane) * 8 + e] = bf16_bits_s(blocks[i].v[8 * h + e]);
-                        ++n;
+                    } else {
+                        // columns with a nonzero weight in any of the 16 rows, in ascending order
+                        std::vector<int> slot((size_t)4 * Kb, -1);
+                        std::vector<Blk> found;
+                        for (int r4 = 0; r4 < 4; ++r4)
+                            for (int i = M->row_ptr[br0 + r4]; i < M->row_ptr[br0 + r4 + 1]; ++i) {
+                                const int bc = M->col[i];
+                                if (bc < bc_lo || bc >= bc_hi) continue;
+                                for (int c = 0; c < 4; ++c) {
+                                    bool any = false;
+                                    for (int r = 0; r < 4; ++r) any = any || M->vals[(size_t)i * 16 + 4 * r + c] != 0.f;
+                                    if (!any) continue;
+                                    const int col = 4 * (bc - bc_lo) + c;
+                                    if (slot[col] < 0) { slot[col] = (int)found.size(); Blk b; b.col = (uint16_t)col; std::memset(b.v, 0, sizeof(b.v)); found.push_back(b); }
+                                    for (int r = 0; r < 4; ++r) found[slot[col]].v[4 * r4 + r] = M->vals[(size_t)i * 16 + 4 * r + c];
+                                }
+                            }
+                        std::sort(found.begin(), found.end(), [](const Blk &a, const Blk &b) { return a.col < b.col; });
+                        R[lbr] = found;
                     }
                 }
-                slot0 += nl * sl.T;
             }
-            kept_bytes += (int64_t)n * 34 + (int64_t)(NBR + 1) * 4;
+        // slice every (CTA, phase): block rows sorted by length (longest first, stable), dealt to the warps in runs; the
+        // first w8 warps take four rows with eight lanes each, the others up to eight rows with four lanes each
+        struct Slice { std::vector<int> rows; int T = 0, lpr = 4; };
+        const int lpr_n = tall ? 16 : 4, cap_n = 32 / lpr_n, cap_w = cap_n / 2;     // lanes per row and rows per warp, narrow / wide slices
+        int w8 = (cap_n * SNW - NBR) / (cap_n - cap_w);                              // warps that can afford wide rows
+        if (w8 < 0) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
+        if (w8 > SNW) w8 = SNW;
+        if (w8 * cap_w > NBR) w8 = NBR / cap_w;
+        std::vector<std::vector<Slice>> slices(NCTA * 2);              // [cta * 2 + phase][warp]
+        int max_slots = 0;
+        for (int cp = 0; cp < NCTA * 2; ++cp) {
+            const auto &R = rows[cp];
+            std::vector<int> order(NBR);
+            for (int i = 0; i < NBR; ++i) order[i] = i;
+            std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return R[a].size() > R[b].size(); });
+            slices[cp].assign(SNW, {});
+            int next = 0, slots = 0;
+            for (int w = 0; w < SNW; ++w) {
+                Slice &sl = slices[cp][w];
+                sl.lpr = w < w8 ? 2 * lpr_n : lpr_n;
+                const int cap = 32 / sl.lpr;
+                // rows still to place, spread evenly over the remaining four-lane warps
+                int nr = cap;
+                if (w >= w8) { const int left = NBR - next, warps_left = SNW - w; nr = (left + warps_left - 1) / warps_left; }
+                if (nr > cap) nr = cap;
+                if (nr > NBR - next) nr = NBR - next;
+                size_t longest = 0;
+                for (int i = 0; i < nr; ++i) { sl.rows.push_back(order[next + i]); longest = std::max(longest, R[order[next + i]].size()); }
+                next += nr;
+                sl.T = (int)((longest + sl.lpr - 1) / sl.lpr);
+                if (sl.T < 1) sl.T = 1;                                  // the loop's first loads are unconditional
+                slots += sl.lpr * nr * sl.T;
+            }
+            if (next != NBR) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
+            max_slots = std::max(max_slots, slots);
         }
-        // dense O2 / O4: 16 rows of this CTA as one tile of A fragments (natural column order)
-        for (int h = 0; h < 2; ++h) {
-            uint16_t *dst = reinterpret_cast<uint16_t *>(base + (h ? k.off_o4 : k.off_o2));
-            std::vector<uint16_t> dense((size_t)16 * Hh, 0);
-            const BsrHost &M = *Ob[h];
-            for (int r = 0; r < 16; ++r) {
-                const int row = cta * 16 + r, br = row / 4, rr = row % 4;
-                for (int i = M.row_ptr[br]; i < M.row_ptr[br + 1]; ++i)
-                    for (int c = 0; c < 4; ++c) dense[(size_t)r * Hh + 4 * M.col[i] + c] = bf16_bits_s(M.vals[(size_t)i * 16 + 4 * rr + c]);
-            }
-            for (int kt = 0; kt < k.NKT; ++kt)
-                for (int lane = 0; lane < 32; ++lane) {
-                    const int g = lane >> 2, t = lane & 3;
-                    uint16_t *o = dst + ((size_t)kt * 32 + lane) * 8;
-                    const int rsel[4] = {g, g + 8, g, g + 8}, csel[4] = {2 * t, 2 * t, 2 * t + 8, 2 * t + 8};
-                    for (int q = 0; q < 4; ++q)
-                        for (int j = 0; j < 2; ++j) o[2 * q + j] = dense[(size_t)rsel[q] * Hh + 16 * kt + csel[q] + j];
+        k.max_slots = (max_slots + 7) & ~7;
+
+        size_t off = 0;
+        for (int ph = 0; ph < 2; ++ph) {
+            k.off_meta[ph] = off; off = a16(off + (size_t)SNW * sizeof(SliceMeta));
+            k.off_col[ph] = off; off = a16(off + (size_t)k.max_slots * 2);
+            k.off_val[ph] = off; off = a16(off + (size_t)k.max_slots * 32);
+        }
+        const size_t frag = (size_t)k.NKT * 512;
+        k.off_o2 = off; off += frag;
+        k.off_o4 = off; off += frag;
+        k.off_small = off; off = a16(off + ((size_t)6 * UC * 3 + 2 * HR + 32) * 4);
+        k.blob_bytes = off;
+        k.smem_bytes = sparse_smem_bytes(k);
+
+        cudaDeviceProp prop;
+        cudaGetDeviceProperties(&prop, m->device);
+        if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "pruned model does not fit the shared memory of one cluster"; return WRNN_ERR_UNSUPPORTED; }
+        if (cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+            cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
+            cudaGetLastError(); m->err = "cannot configure the 16-CTA cluster kernel"; return WRNN_ERR_UNSUPPORTED;
+        }
+        cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
+        sparse_fill_launch(k, &cfg, at, 0, false);
+        int max_clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, sparse_fn(), &cfg) != cudaSuccess || max_clusters < nc) {
+            cudaGetLastError(); m->err = "the 16-CTA clusters cannot all be co-resident on this device"; return WRNN_ERR_UNSUPPORTED;
+        }
+
+        blob.assign((size_t)NCTA * k.blob_bytes, 0);
+        const BsrHost *Ob[2] = {&m->hO2, &m->hO4};
+        kept_bytes = 0;
+        for (int cta = 0; cta < NCTA; ++cta) {
+            const int rank = cta % SCS;
+            uint8_t *base = blob.data() + (size_t)cta * k.blob_bytes;
+            for (int ph = 0; ph < 2; ++ph) {
+                SliceMeta *meta = reinterpret_cast<SliceMeta *>(base + k.off_meta[ph]);
+                uint16_t *col = reinterpret_cast<uint16_t *>(base + k.off_col[ph]);
+                uint16_t *val = reinterpret_cast<uint16_t *>(base + k.off_val[ph]);       // [slot plane][8 bf16]
+                const auto &R = rows[cta * 2 + ph];
+                int slot0 = 0, n = 0, n_r = 0;
+                for (int w = 0; w < SNW; ++w) {
+                    const Slice &sl = slices[cta * 2 + ph][w];
+                    const int nl = sl.lpr * (int)sl.rows.size();
+                    meta[w].voff = 2 * slot0; meta[w].coff = slot0; meta[w].T = sl.T; meta[w].nl = nl; meta[w].lpr = sl.lpr;
+                    for (int g = 0; g < 8; ++g) meta[w].row[g] = g < (int)sl.rows.size() ? (int16_t)sl.rows[g] : (int16_t)-1;
+                    for (int g = 0; g < (int)sl.rows.size(); ++g) {
+                        const auto &blocks = R[sl.rows[g]];
+                        for (int i = 0; i < (int)blocks.size(); ++i) {
+                            const int t = i / sl.lpr, lane = sl.lpr * g + i % sl.lpr;
+                            col[slot0 + t * nl + lane] = blocks[i].col;
+                            for (int h = 0; h < 2; ++h)                  // plane h holds rows 2 h, 2 h + 1 of the block
+                                for (int e = 0; e < 8; ++e)
+                                    val[((size_t)2 * slot0 + (size_t)(2 * t + h) * nl + lane) * 8 + e] = bf16_bits_s(blocks[i].v[8 * h + e]);
+                            ++n;
+                            if (sl.rows[g] >= HR / BRH) ++n_r;
+                        }
+                    }
+                    slot0 += nl * sl.T;
                 }
+                // every kept block of R once; the heads once (cluster 0 stands for all)
+                kept_bytes += cta < SCS ? (int64_t)n * 34 + (int64_t)(NBR + 1) * 4 : (int64_t)n_r * 34;
+            }
+            // dense O2 / O4: 16 rows of this CTA as one tile of A fragments (natural column order)
+            for (int h = 0; h < 2; ++h) {
+                uint16_t *dst = reinterpret_cast<uint16_t *>(base + (h ? k.off_o4 : k.off_o2));
+                std::vector<uint16_t> dense((size_t)16 * Hh, 0);
+                const BsrHost &M = *Ob[h];
+                for (int r = 0; r < 16; ++r) {
+                    const int row = rank * 16 + r, br = row / 4, rr = row % 4;
+                    for (int i = M.row_ptr[br]; i < M.row_ptr[br + 1]; ++i)
+                        for (int c = 0; c < 4; ++c) dense[(size_t)r * Hh + 4 * M.col[i] + c] = bf16_bits_s(M.vals[(size_t)i * 16 + 4 * rr + c]);
+                }
+                for (int kt = 0; kt < k.NKT; ++kt)
+                    for (int lane = 0; lane < 32; ++lane) {
+                        const int g = lane >> 2, t = lane & 3;
+                        uint16_t *o = dst + ((size_t)kt * 32 + lane) * 8;
+                        const int rsel[4] = {g, g + 8, g, g + 8}, csel[4] = {2 * t, 2 * t, 2 * t + 8, 2 * t + 8};
+                        for (int q = 0; q < 4; ++q)
+                            for (int j = 0; j < 2; ++j) o[2 * q + j] = dense[(size_t)rsel[q] * Hh + 16 * kt + csel[q] + j];
+                    }
+            }
+            float *sm = reinterpret_cast<float *>(base + k.off_small);
+            for (int rr = 0; rr < 6 * UC; ++rr) {
+                const int half = rr / (3 * UC), gate = (rr / UC) % 3, u = rr % UC;
+                const int mrow = gate * H + half * Hh + cta * UC + u;
+                for (int c = 0; c < 3; ++c) sm[rr * 3 + c] = m->hI[(size_t)mrow * 3 + c];
+            }
+            float *b = sm + 6 * UC * 3;
+            for (int r = 0; r < HR; ++r) { b[r] = m->hb1[rank * HR + r]; b[HR + r] = m->hb3[rank * HR + r]; }
+            b += 2 * HR;
+            for (int r = 0; r < 16; ++r) { b[r] = m->hb2[rank * 16 + r]; b[16 + r] = m->hb4[rank * 16 + r]; }
         }
-        float *sm = reinterpret_cast<float *>(base + k.off_small);
-        for (int rr = 0; rr < 6 * UC; ++rr) {
-            const int half = rr / (3 * UC), gate = (rr / UC) % 3, u = rr % UC;
-            const int mrow = gate * H + half * Hh + cta * UC + u;
-            for (int c = 0; c < 3; ++c) sm[rr * 3 + c] = m->hI[(size_t)mrow * 3 + c];
+        return WRNN_OK;
+    };
+    {
+        const char *force = getenv("WRNN_SPARSE_CLUSTERS");
+        int rc = WRNN_ERR_UNSUPPORTED;
+        for (int nc : {4, 2, 1}) {
+            if (force && atoi(force) != nc) continue;
+            rc = pack(nc);
+            if (rc == WRNN_OK) break;
         }
-        float *b = sm + 6 * UC * 3;
-        for (int r = 0; r < HR; ++r) { b[r] = m->hb1[cta * HR + r]; b[HR + r] = m->hb3[cta * HR + r]; }
-        b += 2 * HR;
-        for (int r = 0; r < 16; ++r) { b[r] = m->hb2[cta * 16 + r]; b[16 + r] = m->hb4[cta * 16 + r]; }
+        if (rc != WRNN_OK) return rc;
     }
     SparsePack *pk = new SparsePack(k);
     if (cudaMalloc((void **)&pk->d_blob, blob.size()) != cudaSuccess ||
         cudaMemcpy(pk->d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaGetLastError(); cudaFree(pk->d_blob); delete pk;
+        m->err = "device allocation for the sparse cluster kernel failed";
+        return WRNN_ERR_NOMEM;
+    }
+    if (cudaMalloc((void **)&pk->d_slots, (size_t)4 * Hh * 8) != cudaSuccess) {
         cudaGetLastError(); cudaFree(pk->d_blob); delete pk;
         m->err = "device allocation for the sparse cluster kernel failed";
         return WRNN_ERR_NOMEM;
@@ -711,6 +737,7 @@ void sparse_destroy(wrnn_model *m)
 {
     if (!m->sparse_pack) return;
     cudaFree(m->sparse_pack->d_blob);
+    cudaFree(m->sparse_pack->d_slots);
     delete m->sparse_pack;
     m->sparse_pack = nullptr;
 }
@@ -719,7 +746,7 @@ int sparse_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threa
 {
     (void)batch;
     const SparsePack &k = *m->sparse_pack;
-    if (n_ctas) *n_ctas = SCS;
+    if (n_ctas) *n_ctas = SCS * k.NC;
     if (n_threads) *n_threads = SNW * 32;
     if (smem) *smem = k.smem_bytes;
     if (weight_bytes) *weight_bytes = k.weight_bytes_per_step;
@@ -739,7 +766,7 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.hop = m->cond_dim ? a.hop : 1;
     p.row_stride = m->cond_dim ? a.row_stride : 0;
     p.row_offset_mul = m->cond_dim ? a.row_offset_mul : 0;
-    p.blob = k.d_blob; p.g = m->g;
+    p.blob = k.d_blob; p.g = m->g; p.yslots = k.d_slots;
     p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in; p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
@@ -747,6 +774,7 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.limit_ns = 2000000000ull;
 
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
+    if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     const char *no_coop = getenv("WRNN_NO_COOP");
     sparse_fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));

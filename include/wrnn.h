@@ -59,7 +59,7 @@ typedef enum {
     WRNN_KERNEL_GENERIC = 1,    /* weights streamed from L2 every step; any shape; bring-up path */
     WRNN_KERNEL_RESIDENT = 2,   /* persistent kernel, weights resident in shared memory (one row) */
     WRNN_KERNEL_BATCHED = 3,    /* tensor-pipe contractions over all rows (dense bf16, >= 2 rows)  */
-    WRNN_KERNEL_SPARSE = 4,     /* block-sparse model resident in one 16-CTA cluster (one row)     */
+    WRNN_KERNEL_SPARSE = 4,     /* block-sparse model resident in 16-CTA clusters (one row)        */
     WRNN_KERNEL_BCLUSTER = 5    /* rows dealt to 16-CTA clusters, tcgen05 contractions (dense bf16, >= 2 rows) */
 } wrnn_kernel;
 
@@ -89,7 +89,7 @@ typedef struct {
     int32_t mask_block_rows;    /* rows and columns of one block of the three masks (Section 3.2:     */
     int32_t mask_block_cols;    /* 4 x 4, or m x 1 = 16 rows of one column, or 1 x 1 = unstructured); */
                                 /* 0, 0 means 4 x 4.  Both must divide H/2.  Every shape runs on the  */
-                                /* generic kernel; 4 x 4 and 16 x 1 also on the single-cluster kernel */
+                                /* generic kernel; 4 x 4 and 16 x 1 also on the sparse cluster kernel  */
     int32_t variant;            /* 0: WaveRNN (Eq. 2, shapes as above).  1: Fused Subscale WaveRNN 2x */
                                 /* (Section 4.4): I is [3H][12] (nibbles of a_{t-1}, of the previous  */
                                 /* b, of a_t; the last four columns are ignored on part-A rows),      */

@@ -1,11 +1,12 @@
 // Block-sparse single-stream sampling kernel (Section 3: only the kept 4x4 blocks of R_u, R_r, R_e, O1, O3
-// are stored and multiplied): bf16 weights, batch 1, the whole model resident in the shared memory of ONE
-// thread-block cluster of 16 CTAs.
+// are stored and multiplied): bf16 weights, batch 1, the whole model resident in the shared memory of NC
+// thread-block clusters of 16 CTAs (NC = 4 where they can be co-resident).
 //
-// A pruned model is small enough (H = 2048 at 96 %: 2.3 MB of blocks, plus the dense O2 / O4) that no state
-// ever has to cross the chip through L2: every exchange of a step -- the two halves of the state, the hidden
-// layer of a head, its logits -- is an all-gather of (value, tag) words through distributed shared memory.
-// Each CTA owns Hh/16 coarse and Hh/16 fine units (their block rows of R, compressed: block column index +
+// A pruned model is small (H = 2048 at 96 %: 2.3 MB of blocks, plus the dense O2 / O4).  The compressed block rows of R
+// are dealt over all NC x 16 CTAs; the heads are held once per cluster, so that the hidden layer of a head and its
+// logits are all-gathers of (value, tag) words through the distributed shared memory of a cluster; the two halves of
+// the state cross the chip as tagged words in L2 (arrival of the data is the signal).
+// Each CTA owns Hh/(16 NC) coarse and as many fine units (their block rows of R, compressed: block column index +
 // 16 bf16 per kept block), Hh/16 rows of O1 and O3 (compressed block rows) and 16 rows of the dense O2 and O4
 // (mma.sync A fragments).  Sparse rows: four lanes share a block row, each lane takes every fourth kept block
 // (two 16-byte weight loads, four activations, 16 FMAs), a four-value reduce-scatter finishes the rows; the rows
@@ -501,7 +502,7 @@ int sparse_prepare(wrnn_model *m)
     if (m->dtype != WRNN_BF16) { m->err = "sparse cluster kernel stores bf16 weights"; return WRNN_ERR_UNSUPPORTED; }
     if (!m->sparse) { m->err = "model has no block masks"; return WRNN_ERR_UNSUPPORTED; }
     const bool tall = m->mask_br == 16 && m->mask_bc == 1;
-    if (!tall && (m->mask_br != 4 || m->mask_bc != 4)) { m->err = "single-cluster kernel takes 4 x 4 or 16 x 1 blocks"; return WRNN_ERR_UNSUPPORTED; }
+    if (!tall && (m->mask_br != 4 || m->mask_bc != 4)) { m->err = "sparse cluster kernel takes 4 x 4 or 16 x 1 blocks"; return WRNN_ERR_UNSUPPORTED; }
     if (Hh != 1024) { m->err = "only H/2 = 1024 is instantiated (8 warps x 8 k-tiles for the logits tile)"; return WRNN_ERR_UNSUPPORTED; }
     // The rows of R are dealt over NC clusters of 16 (the heads are held once per cluster); more clusters mean fewer block
     // rows per CTA in the phase that dominates the step, at the price of the state crossing the chip through L2 instead
@@ -628,7 +629,7 @@ int sparse_prepare(wrnn_model *m)
 
         cudaDeviceProp prop;
         cudaGetDeviceProperties(&prop, m->device);
-        if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "pruned model does not fit the shared memory of one cluster"; return WRNN_ERR_UNSUPPORTED; }
+        if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "pruned model does not fit the shared memory of the clusters"; return WRNN_ERR_UNSUPPORTED; }
         if (cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
             cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
             cudaGetLastError(); m->err = "cannot configure the 16-CTA cluster kernel"; return WRNN_ERR_UNSUPPORTED;

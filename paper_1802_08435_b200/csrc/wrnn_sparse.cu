@@ -239,10 +239,10 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         }
     };
 
-    // Gates of Eq. 2 for this CTA's UC units of one half, then publish them to the whole grid.  The first GW warps
-    // each draw the sample redundantly (same logits, same uniform, same instructions -> same value) and then gate
-    // UC / GW units each, so that neither the gates nor the 16 x UC / 2 remote stores queue up in one warp.
-    constexpr int GW = 4;
+    // Gates of Eq. 2 for this CTA's UC units of one half, then publish them to the whole grid.  The first GW warps (one
+    // per 32 units: the fewer warps poll the logits buffer, the sooner the logits land) each draw the sample
+    // redundantly (same logits, same uniform, same instructions -> same value) and then gate UC / GW units each.
+    const int GW = (UC + 31) / 32;
     const int UW = UC / GW;
     auto load_g = [&](int half_g, long long s, float (&gv)[3]) {
         const long long fr = ((p.step0 + s) * p.row_stride + (long long)p.stream0 * p.row_offset_mul) / p.hop;

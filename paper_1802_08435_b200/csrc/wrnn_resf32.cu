@@ -204,14 +204,17 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
         gates_and_publish(0, 0, f_prev, gates_prepare(0, gv));
     }
 
-    // all-gather of n tagged words from the chip into a shared-memory vector
+    // all-gather of n (even) tagged words from the chip into a shared-memory vector: two adjacent slots per polling thread
     auto gather = [&](const unsigned long long *slots, int n, unsigned want, float *dst, int step, int phase) {
 #pragma unroll 1
-        for (int i = tid; i < n; i += blockDim.x) {
-            unsigned long long v, t0 = 0; unsigned cnt = 0;
-            while ((unsigned)((v = ld_relaxed_u64(slots + i)) >> 32) != want)
+        for (int i = tid; i < n / 2; i += blockDim.x) {
+            unsigned long long v0, v1, t0 = 0; unsigned cnt = 0;
+            while (true) {
+                asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0), "=l"(v1) : "l"(slots + 2 * i) : "memory");
+                if ((unsigned)(v0 >> 32) == want && (unsigned)(v1 >> 32) == want) break;
                 if ((++cnt & 4095u) == 0 && wt.expired(t0, step, phase)) { my_bad = true; break; }
-            dst[i] = __uint_as_float((unsigned)v);
+            }
+            dst[2 * i] = __uint_as_float((unsigned)v0); dst[2 * i + 1] = __uint_as_float((unsigned)v1);
         }
         return __syncthreads_or(my_bad) != 0;
     };

@@ -182,3 +182,33 @@ def test_resume_and_teacher_forcing():
     assert np.array_equal(np.concatenate([a.out, b.out], axis=1), full.out)
     tf = om.run(cond, 40, seed=4, hop=10, a_forced=full.a_out, b_forced=full.b_out)
     assert np.array_equal(tf.a_out, full.a_out) and np.array_equal(tf.b_out, full.b_out)
+
+
+def test_nibble_draws_follow_their_softmax():
+    """Each of the eight 4-bit symbols is a draw from the softmax of its own sixteen logits: with the state frozen
+    (u = 1 keeps h, zero input and recurrent weights) the logits are the same at every step, and the drawn nibbles'
+    frequencies match their softmax (chi-square, 5 sigma) while the eight heads use different uniforms."""
+    H = 16
+    w = fs2_weights(H, cond_dim=0, scale=3.0, seed=4)
+    w["R"] = np.zeros_like(w["R"]); w["I"] = np.zeros_like(w["I"])
+    w["b_gate"] = w["b_gate"].copy(); w["b_gate"][:H] = 80.0              # u = 1: h_t = h_{t-1}
+    om = orc.Fs2OracleModel(w, "f32")
+    h0 = np.random.default_rng(3).standard_normal(H).astype(np.float32)
+    T = 40000
+    r = om.run(None, T, seed=12, h=h0, dump=True)
+    assert np.array_equal(r.hs[0], h0) and np.array_equal(r.hs[-1], h0)
+    assert np.array_equal(r.logits[0], r.logits[-1])
+    streams = []
+    for part, drawn in ((0, r.a_out), (1, r.b_out)):
+        for k in range(4):
+            nib = (drawn.astype(np.int64) >> (12 - 4 * k)) & 15
+            l = r.logits[0, part, 16 * k: 16 * k + 16].astype(np.float64)
+            p = np.exp(l - l.max()); p /= p.sum()
+            counts = np.bincount(nib, minlength=16)
+            chi2 = ((counts - T * p) ** 2 / (T * p)).sum()
+            assert chi2 < 15 + 5 * np.sqrt(2 * 15), (part, k, chi2)
+            streams.append(nib)
+    # the eight symbols are driven by eight different uniform streams
+    for i in range(8):
+        for j in range(i + 1, 8):
+            assert not np.array_equal(streams[i], streams[j])

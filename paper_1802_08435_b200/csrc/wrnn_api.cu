@@ -126,6 +126,14 @@ static bool use_resf32(const wrnn_model *m, int batch)
     return m->resf32 != nullptr && resf32_supported(m, batch, nullptr) == WRNN_OK;
 }
 
+// two or four streams of a dense bf16 model: pairs on the two-stream form of the resident kernel, one pair after the other
+// (6.6-7 us per step and pair against 24 us per step of the multi-row kernel)
+static bool use_pair(const wrnn_model *m, int batch)
+{
+    if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_RESIDENT) return false;
+    return m->variant == 0 && resident_pair_supported(m, batch) == WRNN_OK;
+}
+
 static bool use_sparse(const wrnn_model *m, int batch)
 {
     if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_SPARSE) return false;
@@ -203,6 +211,13 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
         return generic_run(m, a, s);
     }
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
+    if (use_pair(m, a.batch)) {
+        for (int pair = 0; pair < a.batch / 2; ++pair) {
+            rc = resident_pair_run(m, a, pair, s);
+            if (rc != WRNN_OK) return rc;
+        }
+        return WRNN_OK;
+    }
     if (use_resf32(m, a.batch)) return resf32_run(m, a, s);
     if (use_sparse(m, a.batch)) return sparse_run(m, a, s);
     if (use_bcluster(m, a.batch)) return bcluster_run(m, a, s);
@@ -697,6 +712,10 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
 {
     if (!m || batch < 1 || batch > m->max_batch) return WRNN_ERR_INVALID_ARG;
     if (use_resident(m, batch)) {
+        if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
+        return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
+    }
+    if (use_pair(m, batch)) {
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
     }

@@ -131,6 +131,8 @@ int resident_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_thr
                          int64_t *weight_bytes);
 int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
 int resident_phase_cycles(const wrnn_model *m, long long *out16);
+int resident_pair_supported(const wrnn_model *m, int batch);          // two streams per launch on the same weights (batch 2 or 4)
+int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s);
 
 // wrnn_resf32.cu: the same role for dense fp32 models (every matrix sharded chip-wide, nothing replicated)
 int resf32_supported(const wrnn_model *m, int batch, std::string *why);

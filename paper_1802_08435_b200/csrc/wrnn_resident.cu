@@ -39,6 +39,8 @@ struct ResidentPack {
     int NC = 0, CS = 0, NCTA = 0, UC = 0, HR = 0, LR = 0, K = 0, NKT = 0, NMT = 0, NLT = 0, NW = 0, KSH = 0, KSL = 0;
     int n_rrows = 0;                 // 6 UC
     bool fused = false;              // Fused Subscale WaveRNN 2x: 12 input columns, 64 logits per head
+    int pair_smem = 0;               // dynamic shared memory of the two-stream kernel; 0 = not available
+    unsigned long long *d_slots2 = nullptr;  // [2 halves][2 parities][2 streams][K] (value, tag)
     size_t blob_bytes = 0;           // per CTA: bf16 weight fragments then fp32 small parameters
     size_t w_bytes = 0;              // bf16 part of the blob
     uint8_t *d_blob = nullptr;       // [NCTA][blob_bytes]
@@ -472,6 +474,382 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
     cluster.sync();     // nobody leaves while a peer may still write into its shared memory
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Two streams at once on the same resident weights (Section 5.1 reports a batch of four streams on the paper's kernel).
+// The MMAs of the single-stream kernel use three of their eight B columns (the hi / mid / lo parts of one input
+// vector); here the parts of a second stream take three more, so both streams advance for the tensor-pipe time of
+// one.  Everything per stream is doubled: state vectors, split images (eight columns per piece), exchange slots, the
+// drawing warp (warp s draws and gates stream s).  Same schedule, same waits, same weights layout as above.
+//
+// Columns of a B fragment: 0, 1 = hi, mid of stream 0; 2, 3 = hi, mid of stream 1; 4 = lo of stream 0; 6 = lo of stream 1
+// (5, 7 zero): lane (g, t) of a D fragment holds columns 2 t, 2 t + 1, so one shuffle (xor 2) leaves the sums of stream
+// t & 1 in the lanes with t < 2.
+__host__ __device__ __forceinline__ int split2s_pos(int i, int col)
+{
+    const int c = i & 15, kt = i >> 4;
+    const int t = (c & 7) >> 1, j = c & 1, hi = c >> 3;
+    return ((((((kt >> 1) * 4 + t) * 8 + col) << 1) + (kt & 1)) << 2) + 2 * hi + j;
+}
+__device__ __forceinline__ void store_split2s(__nv_bfloat16 *split, int stream, int i, float x)
+{
+    const __nv_bfloat16 b0 = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(b0);
+    const __nv_bfloat16 b1 = __float2bfloat16_rn(r1);
+    const float r2 = r1 - __bfloat162float(b1);
+    const __nv_bfloat16 b2 = __float2bfloat16_rn(r2);
+    split[split2s_pos(i, 2 * stream)] = b0;
+    split[split2s_pos(i, 2 * stream + 1)] = b1;
+    split[split2s_pos(i, 4 + 2 * stream)] = b2;
+}
+// NK consecutive k-tiles (even count, from the even k-tile kt0) of NT 16-row tiles times the two-stream split vector.
+// On return lane (g, t), t < 2, holds the partial totals of rows g (lo[n]) and g + 8 (hi[n]) of tile n for stream t.
+template <int NK, int NT>
+__device__ __forceinline__ void mma_tiles_pair(const uint4 *A, size_t tile_u4, int kt0, const __nv_bfloat16 *split, int lane, float (&lo)[NT], float (&hi)[NT])
+{
+    const int g = lane >> 2, t = lane & 3;
+    const uint4 *bsrc = reinterpret_cast<const uint4 *>(split) + ((kt0 >> 1) * 4 + t) * 8 + g;
+    uint4 av[NT][NK];
+    uint4 bv[NK / 2];
+#pragma unroll
+    for (int i = 0; i < NK / 2; ++i) bv[i] = bsrc[32 * i];
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+        for (int i = 0; i < NK; ++i) av[n][i] = A[n * tile_u4 + (size_t)(kt0 + i) * 32 + lane];
+    float acc[NT][2][4];
+#pragma unroll
+    for (int n = 0; n < NT; ++n)
+#pragma unroll
+        for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[n][c][i] = 0.f;
+#pragma unroll
+    for (int i = 0; i < NK; ++i)
+#pragma unroll
+        for (int n = 0; n < NT; ++n) {
+            float *c = acc[n][i & 1];
+            const unsigned b0 = (i & 1) ? bv[i >> 1].z : bv[i >> 1].x, b1 = (i & 1) ? bv[i >> 1].w : bv[i >> 1].y;
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                         : "r"(av[n][i].x), "r"(av[n][i].y), "r"(av[n][i].z), "r"(av[n][i].w), "r"(b0), "r"(b1));
+        }
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+        const float c0 = acc[n][0][0] + acc[n][1][0], c1 = acc[n][0][1] + acc[n][1][1];
+        const float c2 = acc[n][0][2] + acc[n][1][2], c3 = acc[n][0][3] + acc[n][1][3];
+        float s_lo = t < 2 ? c0 + c1 : c0, s_hi = t < 2 ? c2 + c3 : c2;     // t >= 2: the lo part sits in the even column only
+        s_lo += __shfl_xor_sync(FULL, s_lo, 2);
+        s_hi += __shfl_xor_sync(FULL, s_hi, 2);
+        lo[n] = s_lo; hi[n] = s_hi;
+    }
+}
+
+struct PairParams {
+    ResidentParams r;                        // fields of the single-stream kernel; pointers address row 0 of the pair
+    int n_batch;                             // rows of the whole call (row pitch of the diagnostic dumps)
+    const float *g1;                         // gate offsets of the second row (r.g: of the first)
+    unsigned long long *slots2;              // [2 halves][2 parities][2 streams][K]
+    long long row_pitch;                     // samples between the two rows of out / c_out / f_out / forced arrays
+};
+
+__global__ void __launch_bounds__(512, 1) resident_pair_kernel(const PairParams pp)
+{
+    constexpr int KSH = 7, NKH = 4, KSL = 7, NKL = 4;
+    const ResidentParams &p = pp.r;
+    extern __shared__ __align__(16) uint8_t smem[];
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = (int)cluster.block_rank();
+    const int cta = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int K = p.K, NKT = p.NKT, NMT = p.NMT, NLT = p.NLT, UC = p.UC, HR = p.HR, LR = p.LR, CS = p.CS, H = p.H;
+    const int NR = p.n_rrows;
+
+    // ---- shared memory carve-up (must match resident_pair_smem_bytes)
+    const size_t tile_u4 = (size_t)NKT * 32;
+    const uint4 *wMA = reinterpret_cast<const uint4 *>(smem);
+    const uint4 *wMB = wMA + (size_t)NMT * tile_u4;
+    const uint4 *wO2 = wMB + (size_t)NMT * tile_u4;
+    const uint4 *wO4 = wO2 + (size_t)NLT * tile_u4;
+    const float *sI = reinterpret_cast<const float *>(smem + p.w_bytes);       // [NR][3]
+    const float *sb1 = sI + NR * 3, *sb3 = sb1 + HR, *sb2 = sb3 + HR, *sb4 = sb2 + LR;
+    float *vecC = reinterpret_cast<float *>(smem + p.blob_bytes);              // [2][K]
+    float *vecF = vecC + 2 * K;                                                // [2][K]
+    float *a_part = vecF + 2 * K;                                              // [2][NR]
+    float *a_full = a_part + 2 * NR;                                           // [2][NR]
+    float *part = a_full + 2 * NR;                                             // [2 streams][32 slots][16]
+    __nv_bfloat16 *splC = reinterpret_cast<__nv_bfloat16 *>(part + 1024);      // two-stream split images, 8 K bf16 each
+    __nv_bfloat16 *splF = splC + 8 * K;
+    __nv_bfloat16 *splQ = splF + 8 * K;
+    float *qbuf = reinterpret_cast<float *>(splQ + 8 * K);                    // [2 parities][2 streams][K]
+    uint4 *lbuf = reinterpret_cast<uint4 *>(qbuf + 4 * K);                     // [2 parities][2 streams][128]
+    __shared__ __align__(8) unsigned long long xbar[2];
+
+    {
+        const uint4 *src = reinterpret_cast<const uint4 *>(p.blob + (size_t)cta * p.blob_bytes);
+        uint4 *dst = reinterpret_cast<uint4 *>(smem);
+        for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
+        for (int i = tid; i < 4 * K + 2048; i += blockDim.x) qbuf[i] = 0.f;             // qbuf and lbuf are adjacent
+        if (tid == 0) {
+            for (int i = 0; i < 2; ++i) mbar_init_cluster(smem_addr(&xbar[i]), 1);
+            mbar_fence_init();
+        }
+        for (int i = tid; i < 24 * K / 8; i += blockDim.x) reinterpret_cast<uint4 *>(splC)[i] = make_uint4(0, 0, 0, 0);
+        __syncthreads();
+        for (int i = tid; i < 2 * K; i += blockDim.x) {
+            const int st = i / K, j = i - st * K;
+            const float c = p.h_in ? p.h_in[(size_t)st * H + j] : 0.f, f = p.h_in ? p.h_in[(size_t)st * H + K + j] : 0.f;
+            vecC[i] = c; vecF[i] = f;
+            store_split2s(splC, st, j, c);
+            store_split2s(splF, st, j, f);
+        }
+    }
+    __syncthreads();
+    cluster.sync();
+
+    Waiter wt{p.status, p.limit_ns};
+    bool my_bad = false;
+    const bool writer = (cta == 0);
+    const int g4 = lane >> 2, t4 = lane & 3;
+    const int ws = warp & 1;                           // the stream a drawing warp (0, 1) serves
+
+    // warps 0 and 1 keep the scalar state of streams 0 and 1
+    int c_prev = 128, f_prev = 0;
+    float hC = 0.f, hF = 0.f;
+    if (warp < 2) {
+        c_prev = p.c_in ? p.c_in[ws] : 128; f_prev = p.f_in ? p.f_in[ws] : 0;
+        if (lane < UC) { hC = vecC[ws * K + cta * UC + lane]; hF = vecF[ws * K + cta * UC + lane]; }
+    }
+
+    const int h_pair = warp / KSH, h_ks = warp % KSH, h_kt0 = h_ks * NKH;
+    const int l_tile = warp / KSL, l_ks = warp % KSL, l_kt0 = l_ks * NKL;
+    const bool h_on = warp < (NMT / 2) * KSH, l_on = warp < NLT * KSL;
+    // partial sums: part[stream][tile * K-splits + split][16]
+    auto hidden_products = [&](const uint4 *Mx, const __nv_bfloat16 *sp) {
+        float lo[2], hi[2];
+        mma_tiles_pair<NKH, 2>(Mx + (size_t)(2 * h_pair) * tile_u4, tile_u4, h_kt0, sp, lane, lo, hi);
+        if (t4 < 2) {
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                float *d = part + t4 * 512 + ((2 * h_pair + n) * KSH + h_ks) * 16;
+                d[g4] = lo[n]; d[g4 + 8] = hi[n];
+            }
+        }
+    };
+    // one peer per warp; lanes [0, 16) serve stream 0, lanes [16, 32) stream 1
+    const int ls = lane >> 4, ll = lane & 15;
+    unsigned q_snd[2], l_snd[2], q_bar[2];
+#pragma unroll
+    for (int par2 = 0; par2 < 2; ++par2) {
+        const unsigned peer = warp < CS ? warp : 0;
+        q_snd[par2] = map_to_rank(smem_addr(qbuf + (size_t)(par2 * 2 + ls) * K + rank * HR + 2 * (ll < HR / 2 ? ll : 0)), peer);
+        l_snd[par2] = map_to_rank(smem_addr(lbuf + (size_t)(par2 * 2 + ls) * 128 + (rank * LR) / 2 + (ll < LR / 2 ? ll : 0)), peer);
+        q_bar[par2] = map_to_rank(smem_addr(&xbar[par2]), peer);
+    }
+    auto wait_arrival = [&](int which, unsigned use, int step, int phase) {
+        const unsigned bar = smem_addr(&xbar[which]);
+        unsigned long long t0 = 0; unsigned cnt = 0;
+        while (!mbar_try_parity(bar, use & 1u))
+            if ((++cnt & 1023u) == 0 && wt.expired(t0, step, phase)) return false;
+        return true;
+    };
+    // R rows of tile `tile` for stream `st`: sums of the K-split partials stay in this CTA
+    auto keep_r_rows = [&](int tile, int st, bool completes) {
+        const int row = 16 * tile + ll;
+        if (row >= HR && row - HR < NR) {
+            float v = 0.f;
+#pragma unroll
+            for (int sp = 0; sp < KSH; ++sp) v += part[st * 512 + (tile * KSH + sp) * 16 + ll];
+            if (completes) a_full[st * NR + row - HR] = a_part[st * NR + row - HR] + v;
+            else a_part[st * NR + row - HR] = v;
+        }
+    };
+
+    // ---- prologue: the recurrent products of step 0 from the initial state, coarse gates of step 0
+    if (h_on) hidden_products(wMA, splC);
+    __syncthreads();
+    if (warp < NMT) keep_r_rows(warp, ls, false);
+    __syncthreads();
+    if (h_on) hidden_products(wMB, splF);
+    __syncthreads();
+    if (warp < NMT) keep_r_rows(warp, ls, true);
+    __syncthreads();
+
+    struct GatePre { float pu, pr, pe, ae, ku, kr, ke; };
+    auto gates_prepare = [&](int half_g, const float (&gv)[3]) {
+        GatePre q;
+        const int rb = half_g ? 3 * UC : 0;
+        const float x0 = scale8(c_prev), x1 = scale8(f_prev);
+        const float *Iu = sI + 3 * (rb + lane), *Ir = sI + 3 * (rb + UC + lane), *Ie = sI + 3 * (rb + 2 * UC + lane);
+        const float *af = a_full + ws * NR;
+        q.pu = af[rb + lane] + fmaf(Iu[0], x0, half_g ? fmaf(Iu[1], x1, gv[0]) : gv[0]);
+        q.pr = af[rb + UC + lane] + fmaf(Ir[0], x0, half_g ? fmaf(Ir[1], x1, gv[1]) : gv[1]);
+        q.pe = fmaf(Ie[0], x0, half_g ? fmaf(Ie[1], x1, gv[2]) : gv[2]);
+        q.ae = af[rb + 2 * UC + lane];
+        q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
+        return q;
+    };
+    auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
+        const float xk = scale8(drawn);
+        const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
+        const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
+        const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
+        if (half_g) hF = hn; else hC = hn;
+        const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
+        st_relaxed_u64(pp.slots2 + ((size_t)((half_g ? 2 : 0) + (s & 1)) * 2 + ws) * K + j,
+                       ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+        if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * pp.n_batch + ws) * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
+        if (p.dbg_h) p.dbg_h[((size_t)s * pp.n_batch + ws) * H + jj] = hn;
+    };
+    auto load_g = [&](int half_g, long long s, float (&gv)[3]) {
+        const long long fr = ((p.step0 + s) * p.row_stride + (long long)(p.stream0 + (unsigned)ws) * p.row_offset_mul) / p.hop - p.frame_shift;
+        const float *g = (ws ? pp.g1 : p.g) + (size_t)fr * 3 * H + (half_g ? K : 0) + cta * UC + lane;
+#pragma unroll
+        for (int gate = 0; gate < 3; ++gate) gv[gate] = __ldg(g + gate * H);
+    };
+    if (warp < 2 && lane < UC) {
+        float gv[3];
+        load_g(0, 0, gv);
+        gates_and_publish(0, 0, f_prev, gates_prepare(0, gv));
+    }
+
+    const long long T = p.n_steps;
+#pragma unroll 1
+    for (long long n = 1; n <= 2 * T; ++n) {
+        const int half = (int)(n & 1);
+        const long long s = n >> 1;
+        const bool last = n == 2 * T;
+        const unsigned tag = (unsigned)n, par = (unsigned)((n - 1) & 1);
+        const uint4 *M = half ? wMA : wMB, *L = half ? wO2 : wO4;
+        const float *bh = half ? sb1 : sb3, *bl = half ? sb2 : sb4;
+        float *vec = half ? vecC : vecF;
+        __nv_bfloat16 *spl = half ? splC : splF;
+
+        const unsigned use = (unsigned)((n - 1) >> 1);
+        if (tid == 0) mbar_arrive_expect(smem_addr(&xbar[par]), (unsigned)K * 8u);      // this half's hidden layers: 2 x K values
+        float gv[3] = {0.f, 0.f, 0.f}, u01 = 0.f;
+        int forced = -1;
+        if (warp < 2) {
+            if (lane < UC && !last) load_g(half, s, gv);
+            const long long o = (long long)ws * pp.row_pitch + (half ? s : s - 1);
+            if (half) { if (p.c_forced) forced = p.c_forced[o]; }
+            else      { if (p.f_forced) forced = p.f_forced[o]; }
+            u01 = uniform24(p.seed, p.stream0 + (unsigned)ws, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
+        }
+
+        // ---- 1. the input half-vectors of both streams from the whole chip
+        {
+            const unsigned long long *slots = pp.slots2 + (size_t)(half ? (s & 1) : 2 + ((s - 1) & 1)) * 2 * K;
+            const unsigned ytag = (unsigned)(half ? s + 1 : s);
+#pragma unroll 1
+            for (int i = tid; i < K; i += blockDim.x) {              // K slot pairs: [stream][K / 2]
+                unsigned long long v0, v1, t0 = 0; unsigned cnt = 0;
+                while (true) {
+                    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0), "=l"(v1) : "l"(slots + 2 * i) : "memory");
+                    if ((unsigned)(v0 >> 32) == ytag && (unsigned)(v1 >> 32) == ytag) break;
+                    if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+                }
+                const int st = (2 * i) / K, j = 2 * i - st * K;
+                const float x0 = __uint_as_float((unsigned)v0), x1 = __uint_as_float((unsigned)v1);
+                vec[2 * i] = x0; vec[2 * i + 1] = x1;
+                store_split2s(spl, st, j, x0);
+                store_split2s(spl, st, j + 1, x1);
+            }
+            if (__syncthreads_or(my_bad)) break;
+        }
+
+        // ---- 2. hidden layers of the head + this CTA's R rows, both streams in the same MMAs
+        if (h_on) hidden_products(M, spl);
+        __syncthreads();
+        if (warp < CS && ll < HR / 2) {
+            const int r0 = 2 * ll, tile = r0 >> 4, rr = r0 & 15;
+            const float *pt = part + ls * 512;
+            float v0 = bh[r0], v1 = bh[r0 + 1];
+#pragma unroll
+            for (int sp = 0; sp < KSH; ++sp) { v0 += pt[(tile * KSH + sp) * 16 + rr]; v1 += pt[(tile * KSH + sp) * 16 + rr + 1]; }
+            st_async_v2(q_snd[par], fmaxf(v0, 0.f), fmaxf(v1, 0.f), q_bar[par]);
+        }
+        if (warp < NMT) keep_r_rows(warp, ls, !half);
+
+        // ---- 3. the cluster's hidden layers -> logits rows of this CTA
+        if (tid < K) {
+            if (!wait_arrival(par, use, (int)s, 2 + 4 * half)) my_bad = true;
+            const int st = (2 * tid) / K, j = 2 * tid - st * K;
+            const float2 v = reinterpret_cast<const float2 *>(qbuf + (size_t)par * 2 * K)[tid];
+            store_split2s(splQ, st, j, v.x);
+            store_split2s(splQ, st, j + 1, v.y);
+        }
+        if (__syncthreads_or(my_bad)) break;
+        if (l_on) {
+            float lo[1], hi[1];
+            mma_tiles_pair<NKL, 1>(L + (size_t)l_tile * tile_u4, tile_u4, l_kt0, splQ, lane, lo, hi);
+            if (t4 < 2) { float *d = part + t4 * 512 + warp * 16; d[g4] = lo[0]; d[g4 + 8] = hi[0]; }
+        }
+        __syncthreads();
+        if (warp < CS && ll < LR / 2) {
+            const int r0 = 2 * ll, tile = r0 >> 4, rr = r0 & 15;
+            const float *pt = part + ls * 512;
+            float v0 = bl[r0], v1 = bl[r0 + 1];
+#pragma unroll
+            for (int sp = 0; sp < KSL; ++sp) { v0 += pt[(tile * KSL + sp) * 16 + rr]; v1 += pt[(tile * KSL + sp) * 16 + rr + 1]; }
+            st_cluster_ll(l_snd[par], v0, v1, tag);
+        }
+
+        // ---- 4. warps 0, 1: the 256 logits of their stream -> draw; then the gates of the other half of its state
+        if (warp < 2) {
+            GatePre gp = {};
+            if (lane < UC && !last) gp = gates_prepare(half, gv);
+            float l[8];
+            {
+                const unsigned a = smem_addr(lbuf + (size_t)(par * 2 + ws) * 128 + 4 * lane);
+                uint4 v0, v1, v2, v3;
+                unsigned long long t0 = 0; unsigned cnt = 0;
+                while (true) {
+                    v0 = ld_shared_volatile_v4(a); v1 = ld_shared_volatile_v4(a + 16);
+                    v2 = ld_shared_volatile_v4(a + 32); v3 = ld_shared_volatile_v4(a + 48);
+                    const bool ok = v0.y == tag && v0.w == tag && v1.y == tag && v1.w == tag && v2.y == tag && v2.w == tag && v3.y == tag && v3.w == tag;
+                    if (ok) break;
+                    if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 3 + 4 * half)) { my_bad = true; break; }
+                }
+                l[0] = __uint_as_float(v0.x); l[1] = __uint_as_float(v0.z); l[2] = __uint_as_float(v1.x); l[3] = __uint_as_float(v1.z);
+                l[4] = __uint_as_float(v2.x); l[5] = __uint_as_float(v2.z); l[6] = __uint_as_float(v3.x); l[7] = __uint_as_float(v3.z);
+            }
+            my_bad = __any_sync(FULL, my_bad);
+            const int drawn = warp_softmax_draw_fast(l, u01, lane);
+            const int fed = forced >= 0 ? forced : drawn;
+            if (lane < UC && !last && !my_bad) gates_and_publish(half, s, fed, gp);
+            if (writer) {
+                if (p.dbg_logits) {
+                    float *d = p.dbg_logits + (((size_t)(half ? s : s - 1) * pp.n_batch + ws) * 2 + (half ? 0 : 1)) * 256 + 8 * lane;
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) d[k] = l[k];
+                }
+                if (lane == 0) {
+                    const long long o = (long long)ws * pp.row_pitch + (half ? s : s - 1);
+                    if (half) { if (p.c_out) p.c_out[o] = (uint8_t)drawn; }
+                    else      { if (p.f_out) p.f_out[o] = (uint8_t)drawn; }
+                    if (!half && p.out) p.out[o] = (int16_t)(256 * c_prev + fed - 32768);
+                }
+            }
+            if (half) c_prev = fed; else f_prev = fed;
+        }
+    }
+
+    const int any_bad = __syncthreads_or(my_bad);
+    if (writer && !any_bad) {
+        if (p.h_out)
+            for (int i = tid; i < 2 * K; i += blockDim.x) {
+                const int st = i / K, j = i - st * K;
+                p.h_out[(size_t)st * H + j] = vecC[i]; p.h_out[(size_t)st * H + K + j] = vecF[i];
+            }
+        if (warp < 2 && lane == 0) {
+            if (p.c_st_out) p.c_st_out[ws] = (uint8_t)c_prev;
+            if (p.f_st_out) p.f_st_out[ws] = (uint8_t)f_prev;
+        }
+    }
+    cluster.sync();
+}
+
 // ---------------------------------------------------------------------------------------------
 static int resident_smem_bytes(const ResidentPack &k)
 {
@@ -484,6 +862,18 @@ static int resident_smem_bytes(const ResidentPack &k)
     b += (size_t)12 * k.K * 2;                      // three split images of 4 K bf16
     b += (size_t)2 * k.K * 4;                       // qbuf [2][K]
     b += 256 * 16;                                  // lbuf [2][128] x 16 B
+    return (int)b;
+}
+
+static int resident_pair_smem_bytes(const ResidentPack &k)
+{
+    size_t b = k.blob_bytes;
+    b += (size_t)4 * k.K * 4;                       // vecC, vecF of two streams
+    b += (size_t)4 * k.n_rrows * 4;                 // a_part, a_full of two streams
+    b += 1024 * 4;                                  // partial sums [2 streams][32][16]
+    b += (size_t)24 * k.K * 2;                      // three two-stream split images of 8 K bf16
+    b += (size_t)4 * k.K * 4;                       // qbuf [2][2][K]
+    b += 512 * 16;                                  // lbuf [2][2][128] x 16 B
     return (int)b;
 }
 
@@ -622,6 +1012,20 @@ int resident_prepare(wrnn_model *m)
         break;
     }
     if (!found) { m->err = why; return WRNN_ERR_UNSUPPORTED; }
+    // the two-stream kernel shares the weights; it needs more shared memory for the doubled vectors and exchange buffers
+    if (!k.fused && (4 * k.n_rrows) % 4 == 0) {
+        const int ps = resident_pair_smem_bytes(k);
+        if ((size_t)ps <= prop.sharedMemPerBlockOptin &&
+            cudaFuncSetAttribute(resident_pair_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+            cudaFuncSetAttribute(resident_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ps) == cudaSuccess) {
+            cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
+            fill_launch(k, &cfg, at, 0, false);
+            cfg.dynamicSmemBytes = ps;
+            int max_clusters = 0;
+            if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_pair_kernel, &cfg) == cudaSuccess && max_clusters >= k.NC) k.pair_smem = ps;
+        }
+        cudaGetLastError();
+    }
 
     // ---- per-CTA blobs
     const int H = m->H, K = k.K, UC = k.UC, n_in = k.fused ? 12 : 3;
@@ -673,11 +1077,12 @@ int resident_prepare(wrnn_model *m)
     bool ok = cudaMalloc((void **)&pk->d_blob, blob.size()) == cudaSuccess &&
               cudaMemcpy(pk->d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) == cudaSuccess &&
               cudaMalloc((void **)&pk->d_slots, (size_t)4 * K * 8) == cudaSuccess &&
+              cudaMalloc((void **)&pk->d_slots2, (size_t)8 * K * 8) == cudaSuccess &&
               cudaMalloc((void **)&pk->d_prof, 16 * sizeof(long long)) == cudaSuccess &&
               cudaMemset(pk->d_prof, 0, 16 * sizeof(long long)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
-        cudaFree(pk->d_blob); cudaFree(pk->d_slots); cudaFree(pk->d_prof);
+        cudaFree(pk->d_blob); cudaFree(pk->d_slots); cudaFree(pk->d_slots2); cudaFree(pk->d_prof);
         delete pk;
         m->err = "device allocation for the resident kernel failed";
         return WRNN_ERR_NOMEM;
@@ -694,6 +1099,7 @@ void resident_destroy(wrnn_model *m)
     cudaFree(m->resident->d_blob);
     cudaFree(m->resident->d_slots);
     cudaFree(m->resident->d_prof);
+    cudaFree(m->resident->d_slots2);
     delete m->resident;
     m->resident = nullptr;
 }
@@ -745,6 +1151,62 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
                             : cudaLaunchKernelEx(&cfg, resident_dense_kernel<7, 4, 7, 4, false>, p);
     if (e != cudaSuccess) {
         m->err = std::string("resident kernel launch failed: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        return WRNN_ERR_CUDA;
+    }
+    ++g_launches;
+    return WRNN_OK;
+}
+
+int resident_pair_supported(const wrnn_model *m, int batch)
+{
+    return m->resident && m->resident->pair_smem > 0 && (batch == 2 || batch == 4) ? WRNN_OK : WRNN_ERR_UNSUPPORTED;
+}
+
+// Rows 2 pair, 2 pair + 1 of the call described by `a` (its conditioning already projected into m->g for all rows).
+int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s)
+{
+    const ResidentPack &k = *m->resident;
+    PairParams pp;
+    std::memset(&pp, 0, sizeof(pp));
+    ResidentParams &p = pp.r;
+    const int b0 = 2 * pair, H = m->H;
+    const size_t nf = m->cond_dim ? a.n_frames : 1;
+    p.H = H; p.K = k.K; p.NKT = k.NKT; p.NMT = k.NMT; p.NLT = k.NLT; p.UC = k.UC; p.HR = k.HR; p.LR = k.LR; p.CS = k.CS;
+    p.n_rrows = k.n_rrows;
+    p.n_steps = a.n_steps; p.step0 = a.step0; p.stream0 = a.stream0 + (unsigned)b0; p.seed = a.seed;
+    p.n_frames = (int)nf;
+    p.hop = m->cond_dim ? a.hop : 1;
+    p.row_stride = m->cond_dim ? a.row_stride : 0;
+    p.row_offset_mul = m->cond_dim ? a.row_offset_mul : 0;
+    p.blob = k.d_blob; p.blob_bytes = k.blob_bytes; p.w_bytes = k.w_bytes;
+    p.g = m->g + (size_t)b0 * nf * 3 * H;
+    pp.g1 = p.g + nf * 3 * H;
+    pp.slots2 = k.d_slots2;
+    pp.n_batch = a.batch;
+    pp.row_pitch = a.n_steps;
+    const size_t ro = (size_t)b0 * a.n_steps;
+    p.h_in = a.h_in ? a.h_in + (size_t)b0 * H : nullptr; p.h_out = a.h_out ? a.h_out + (size_t)b0 * H : nullptr;
+    p.c_in = a.c_in ? a.c_in + b0 : nullptr; p.f_in = a.f_in ? a.f_in + b0 : nullptr;
+    p.c_st_out = a.c_st_out ? a.c_st_out + b0 : nullptr; p.f_st_out = a.f_st_out ? a.f_st_out + b0 : nullptr;
+    p.c_forced = a.c_forced ? a.c_forced + ro : nullptr; p.f_forced = a.f_forced ? a.f_forced + ro : nullptr;
+    p.c_out = a.c_out ? a.c_out + ro : nullptr; p.f_out = a.f_out ? a.f_out + ro : nullptr;
+    p.out = a.out ? a.out + ro : nullptr;
+    p.dbg_gates = a.dbg_gates ? a.dbg_gates + (size_t)b0 * 3 * H : nullptr;
+    p.dbg_h = a.dbg_h ? a.dbg_h + (size_t)b0 * H : nullptr;
+    p.dbg_logits = a.dbg_logits ? a.dbg_logits + (size_t)b0 * 512 : nullptr;
+    p.status = m->status;
+    p.limit_ns = 2000000000ull;
+
+    if (cudaMemsetAsync(k.d_slots2, 0, (size_t)8 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
+    if (pair == 0 && cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
+    cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
+    const char *no_coop = getenv("WRNN_NO_COOP");
+    fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
+    cfg.dynamicSmemBytes = k.pair_smem;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, resident_pair_kernel, pp);
+    if (e != cudaSuccess) {
+        m->err = std::string("two-stream resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();
         return WRNN_ERR_CUDA;
     }

@@ -417,6 +417,37 @@ def test_resident_kernel_short_calls_and_resume(env):
         B.wrnn_destroy(m)
 
 
+@pytest.mark.parametrize("batch", [2, 4])
+def test_two_stream_resident_kernel(env, batch):
+    """Two and four streams of the dense H = 896 bf16 model run as pairs on the two-stream form of the resident kernel:
+    every gate, state and logit of every row against the oracle (rows keep their own conditioning offsets and Philox
+    streams), then a free run, a resumed run and the cross-check against the cluster-partitioned kernel."""
+    torch, B = env
+    wl = synth.WORKLOADS[7]                      # four streams of the dense model
+    w, masks, cond = synth.build_workload(wl, batch=batch)
+    om = orc.OracleModel(w, wl.dtype)
+    n = 400
+    m = B.wrnn_create(w, wl.dtype, max_batch=batch)
+    try:
+        assert B.wrnn_launch_info(m, batch)["kernel"] == B.WRNN_KERNEL_RESIDENT
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, n, batch, SEED, row_stride=1, row_offset_mul=7, stream0=3, threads=pu.NCPU)
+        _report("two-stream resident, batch %d" % batch, r)
+        _tol_check(r, wl.dtype)
+        full = _free_run(torch, B, m, cond, n, batch, SEED, row_offset_mul=7, stream0=3)
+        h = torch.zeros((batch, wl.H), dtype=torch.float32, device="cuda:0")
+        cp = torch.full((batch,), 128, dtype=torch.uint8, device="cuda:0")
+        fp = torch.zeros((batch,), dtype=torch.uint8, device="cuda:0")
+        a = _free_run(torch, B, m, cond, 150, batch, SEED, row_offset_mul=7, stream0=3, h=h, c_prev=cp, f_prev=fp)
+        b = _free_run(torch, B, m, cond, n - 150, batch, SEED, row_offset_mul=7, stream0=3, h=h, c_prev=cp, f_prev=fp, step0=150)
+        assert np.array_equal(np.concatenate([a, b], axis=1), full)
+        # each row equals the single-stream kernel on that row alone
+        one = _free_run(torch, B, m, cond[batch - 1:batch], n, 1, SEED, row_offset_mul=7, stream0=3 + batch - 1)
+        d = np.nonzero(one[0] != full[batch - 1])[0]
+        assert d.size == 0 or r["oracle"].margins[batch - 1, d[0]].min() < pu.MARGIN
+    finally:
+        B.wrnn_destroy(m)
+
+
 def test_config2_sparse_bf16(env):
     """Block-sparse H=2048 bf16 (96 % of the 4x4 blocks of R_u, R_r, R_e, O1, O3 pruned), batch 1: the first
     1,500 steps against the dense-with-zeros oracle; the full 24,000 steps for determinism and resume."""

@@ -150,14 +150,14 @@ __device__ __forceinline__ void mma_partial(const uint4 *A, int kt0, const __nv_
 }
 
 // ---------------------------------------------------------------------------------------------
-// The same split image with two k-tiles per 16-byte piece: [K/32 k-tile pairs][4 t][4 parts][2 k-tiles][4 bf16], so that
-// one 16-byte load per lane brings the B fragments of two k-tiles (the load/store unit is the busiest unit of the
-// single-stream kernel, and its cost goes by instructions, not bytes).
+// The same split image with two k-tiles per 16-byte piece: [K/32 k-tile pairs][4 parts][4 t][2 k-tiles][4 bf16], so that
+// one 16-byte load per lane brings the B fragments of two k-tiles, the loads of a warp are one contiguous run, and the
+// threads that write the image (consecutive elements per lane) spread over the banks.
 __host__ __device__ __forceinline__ int split2_pos(int i, int part)
 {
     const int c = i & 15, kt = i >> 4;
     const int t = (c & 7) >> 1, j = c & 1, hi = c >> 3;
-    return ((((((kt >> 1) * 4 + t) * 4 + part) << 1) + (kt & 1)) << 2) + 2 * hi + j;
+    return ((((((kt >> 1) * 4 + part) * 4 + t) << 1) + (kt & 1)) << 2) + 2 * hi + j;
 }
 
 __device__ __forceinline__ void store_split2(__nv_bfloat16 *split, int i, float x)
@@ -167,8 +167,22 @@ __device__ __forceinline__ void store_split2(__nv_bfloat16 *split, int i, float 
     const __nv_bfloat16 b1 = __float2bfloat16_rn(r1);
     const float r2 = r1 - __bfloat162float(b1);
     const __nv_bfloat16 b2 = __float2bfloat16_rn(r2);
-    const int pos = split2_pos(i, 0);
-    split[pos] = b0; split[pos + 8] = b1; split[pos + 16] = b2;
+    split[split2_pos(i, 0)] = b0; split[split2_pos(i, 1)] = b1; split[split2_pos(i, 2)] = b2;
+}
+// two adjacent elements (i even): they share a 32-bit word of every part
+__device__ __forceinline__ void store_split2_pair(__nv_bfloat16 *split, int i, float x0, float x1)
+{
+    unsigned w[3];
+    float r0 = x0, r1 = x1;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const __nv_bfloat16 a = __float2bfloat16_rn(r0), b = __float2bfloat16_rn(r1);
+        w[k] = (unsigned)__bfloat16_as_ushort(a) | ((unsigned)__bfloat16_as_ushort(b) << 16);
+        r0 -= __bfloat162float(a); r1 -= __bfloat162float(b);
+    }
+    unsigned *s32 = reinterpret_cast<unsigned *>(split);
+#pragma unroll
+    for (int k = 0; k < 3; ++k) s32[split2_pos(i, k) >> 1] = w[k];
 }
 
 // NK consecutive k-tiles (NK even, from the even k-tile kt0) of NT 16-row tiles (consecutive in memory, tile_u4 apart) of a
@@ -179,7 +193,7 @@ __device__ __forceinline__ void mma_tiles(const uint4 *A, size_t tile_u4, int kt
 {
     static_assert(NK % 2 == 0, "k-tiles come in pairs");
     const int g = lane >> 2, t = lane & 3;
-    const uint4 *bsrc = reinterpret_cast<const uint4 *>(split) + ((kt0 >> 1) * 4 + t) * 4 + (g & 3);
+    const uint4 *bsrc = reinterpret_cast<const uint4 *>(split) + ((kt0 >> 1) * 4 + (g & 3)) * 4 + t;
     uint4 av[NT][NK];
     uint4 bv[NK / 2];
 #pragma unroll

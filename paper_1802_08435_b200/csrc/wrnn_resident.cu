@@ -328,8 +328,7 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
                 }
                 const float x0 = __uint_as_float((unsigned)v0), x1 = __uint_as_float((unsigned)v1);
                 vec[2 * i] = x0; vec[2 * i + 1] = x1;
-                store_split2(spl, 2 * i, x0);
-                store_split2(spl, 2 * i + 1, x1);
+                store_split2_pair(spl, 2 * i, x0, x1);
             }
             if (__syncthreads_or(my_bad)) break;
         }
@@ -365,8 +364,7 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
         if (tid < K / 2) {
             if (!wait_arrival(par, use, (int)s, 2 + 4 * half)) my_bad = true;
             const float2 v = reinterpret_cast<const float2 *>(qbuf + (size_t)par * K)[tid];
-            store_split2(splQ, 2 * tid, v.x);
-            store_split2(splQ, 2 * tid + 1, v.y);
+            store_split2_pair(splQ, 2 * tid, v.x, v.y);
         }
         if (__syncthreads_or(my_bad)) break;
         STAMP(2 + 6 * half);
@@ -489,7 +487,7 @@ __host__ __device__ __forceinline__ int split2s_pos(int i, int col)
 {
     const int c = i & 15, kt = i >> 4;
     const int t = (c & 7) >> 1, j = c & 1, hi = c >> 3;
-    return ((((((kt >> 1) * 4 + t) * 8 + col) << 1) + (kt & 1)) << 2) + 2 * hi + j;
+    return ((((((kt >> 1) * 8 + col) * 4 + t) << 1) + (kt & 1)) << 2) + 2 * hi + j;
 }
 __device__ __forceinline__ void store_split2s(__nv_bfloat16 *split, int stream, int i, float x)
 {
@@ -502,13 +500,29 @@ __device__ __forceinline__ void store_split2s(__nv_bfloat16 *split, int stream, 
     split[split2s_pos(i, 2 * stream + 1)] = b1;
     split[split2s_pos(i, 4 + 2 * stream)] = b2;
 }
+// two adjacent elements (i even) of one stream: one 32-bit store per part
+__device__ __forceinline__ void store_split2s_pair(__nv_bfloat16 *split, int stream, int i, float x0, float x1)
+{
+    unsigned w[3];
+    float r0 = x0, r1 = x1;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+        const __nv_bfloat16 a = __float2bfloat16_rn(r0), b = __float2bfloat16_rn(r1);
+        w[k] = (unsigned)__bfloat16_as_ushort(a) | ((unsigned)__bfloat16_as_ushort(b) << 16);
+        r0 -= __bfloat162float(a); r1 -= __bfloat162float(b);
+    }
+    unsigned *s32 = reinterpret_cast<unsigned *>(split);
+    s32[split2s_pos(i, 2 * stream) >> 1] = w[0];
+    s32[split2s_pos(i, 2 * stream + 1) >> 1] = w[1];
+    s32[split2s_pos(i, 4 + 2 * stream) >> 1] = w[2];
+}
 // NK consecutive k-tiles (even count, from the even k-tile kt0) of NT 16-row tiles times the two-stream split vector.
 // On return lane (g, t), t < 2, holds the partial totals of rows g (lo[n]) and g + 8 (hi[n]) of tile n for stream t.
 template <int NK, int NT>
 __device__ __forceinline__ void mma_tiles_pair(const uint4 *A, size_t tile_u4, int kt0, const __nv_bfloat16 *split, int lane, float (&lo)[NT], float (&hi)[NT])
 {
     const int g = lane >> 2, t = lane & 3;
-    const uint4 *bsrc = reinterpret_cast<const uint4 *>(split) + ((kt0 >> 1) * 4 + t) * 8 + g;
+    const uint4 *bsrc = reinterpret_cast<const uint4 *>(split) + ((kt0 >> 1) * 8 + g) * 4 + t;
     uint4 av[NT][NK];
     uint4 bv[NK / 2];
 #pragma unroll
@@ -611,6 +625,13 @@ __global__ void __launch_bounds__(512, 1) resident_pair_kernel(const PairParams 
     bool my_bad = false;
     const bool writer = (cta == 0);
     const int g4 = lane >> 2, t4 = lane & 3;
+    // optional phase timing (CTA 0, warp 0), the slots of the single-stream kernel
+    const bool prof_on = p.prof != nullptr && cta == 0 && warp == 0;
+    __shared__ long long s_prof[16];
+    if (tid < 16) s_prof[tid] = 0;
+    __syncthreads();
+    long long prof_t = clock64();
+#define STAMP(i) do { if (prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
     const int ws = warp & 1;                           // the stream a drawing warp (0, 1) serves
 
     // warps 0 and 1 keep the scalar state of streams 0 and 1
@@ -752,15 +773,16 @@ __global__ void __launch_bounds__(512, 1) resident_pair_kernel(const PairParams 
                 const int st = (2 * i) / K, j = 2 * i - st * K;
                 const float x0 = __uint_as_float((unsigned)v0), x1 = __uint_as_float((unsigned)v1);
                 vec[2 * i] = x0; vec[2 * i + 1] = x1;
-                store_split2s(spl, st, j, x0);
-                store_split2s(spl, st, j + 1, x1);
+                store_split2s_pair(spl, st, j, x0, x1);
             }
             if (__syncthreads_or(my_bad)) break;
         }
+        STAMP(0 + 6 * half);
 
         // ---- 2. hidden layers of the head + this CTA's R rows, both streams in the same MMAs
         if (h_on) hidden_products(M, spl);
         __syncthreads();
+        STAMP(12 + half);
         if (warp < CS && ll < HR / 2) {
             const int r0 = 2 * ll, tile = r0 >> 4, rr = r0 & 15;
             const float *pt = part + ls * 512;
@@ -770,22 +792,24 @@ __global__ void __launch_bounds__(512, 1) resident_pair_kernel(const PairParams 
             st_async_v2(q_snd[par], fmaxf(v0, 0.f), fmaxf(v1, 0.f), q_bar[par]);
         }
         if (warp < NMT) keep_r_rows(warp, ls, !half);
+        STAMP(1 + 6 * half);
 
         // ---- 3. the cluster's hidden layers -> logits rows of this CTA
         if (tid < K) {
             if (!wait_arrival(par, use, (int)s, 2 + 4 * half)) my_bad = true;
             const int st = (2 * tid) / K, j = 2 * tid - st * K;
             const float2 v = reinterpret_cast<const float2 *>(qbuf + (size_t)par * 2 * K)[tid];
-            store_split2s(splQ, st, j, v.x);
-            store_split2s(splQ, st, j + 1, v.y);
+            store_split2s_pair(splQ, st, j, v.x, v.y);
         }
         if (__syncthreads_or(my_bad)) break;
+        STAMP(2 + 6 * half);
         if (l_on) {
             float lo[1], hi[1];
             mma_tiles_pair<NKL, 1>(L + (size_t)l_tile * tile_u4, tile_u4, l_kt0, splQ, lane, lo, hi);
             if (t4 < 2) { float *d = part + t4 * 512 + warp * 16; d[g4] = lo[0]; d[g4 + 8] = hi[0]; }
         }
         __syncthreads();
+        STAMP(14 + half);
         if (warp < CS && ll < LR / 2) {
             const int r0 = 2 * ll, tile = r0 >> 4, rr = r0 & 15;
             const float *pt = part + ls * 512;
@@ -794,6 +818,7 @@ __global__ void __launch_bounds__(512, 1) resident_pair_kernel(const PairParams 
             for (int sp = 0; sp < KSL; ++sp) { v0 += pt[(tile * KSL + sp) * 16 + rr]; v1 += pt[(tile * KSL + sp) * 16 + rr + 1]; }
             st_cluster_ll(l_snd[par], v0, v1, tag);
         }
+        STAMP(3 + 6 * half);
 
         // ---- 4. warps 0, 1: the 256 logits of their stream -> draw; then the gates of the other half of its state
         if (warp < 2) {
@@ -815,6 +840,7 @@ __global__ void __launch_bounds__(512, 1) resident_pair_kernel(const PairParams 
                 l[4] = __uint_as_float(v2.x); l[5] = __uint_as_float(v2.z); l[6] = __uint_as_float(v3.x); l[7] = __uint_as_float(v3.z);
             }
             my_bad = __any_sync(FULL, my_bad);
+            STAMP(4 + 6 * half);
             const int drawn = warp_softmax_draw_fast(l, u01, lane);
             const int fed = forced >= 0 ? forced : drawn;
             if (lane < UC && !last && !my_bad) gates_and_publish(half, s, fed, gp);
@@ -833,7 +859,10 @@ __global__ void __launch_bounds__(512, 1) resident_pair_kernel(const PairParams 
             }
             if (half) c_prev = fed; else f_prev = fed;
         }
+        STAMP(5 + 6 * half);
     }
+    if (prof_on && lane == 0) for (int i = 0; i < 16; ++i) p.prof[i] = s_prof[i];
+#undef STAMP
 
     const int any_bad = __syncthreads_or(my_bad);
     if (writer && !any_bad) {
@@ -1197,6 +1226,7 @@ int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s
     p.dbg_logits = a.dbg_logits ? a.dbg_logits + (size_t)b0 * 512 : nullptr;
     p.status = m->status;
     p.limit_ns = 2000000000ull;
+    p.prof = k.d_prof;
 
     if (cudaMemsetAsync(k.d_slots2, 0, (size_t)8 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (pair == 0 && cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;

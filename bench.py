@@ -299,6 +299,12 @@ def main():
             ach = flops * n_steps / (ms_per_step * 1e-3) / 1e12
             roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                     "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None, "peak_source": peaks["source"] + " sustained"}
+            if info["kernel"] == 2:      # the multi-stream resident kernel stamps the phases of its first CTA's first warp
+                pc = B.wrnn_phase_cycles(model)
+                names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_wait_recurrent",
+                         "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_wait_recurrent",
+                         "F.hid_products", "C.hid_products", "F.log_products", "C.log_products"]
+                roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
         elif wl.sparsity is not None:
             ach = wbytes * n_steps / (ms_per_step * 1e-3) / 1e9
             roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],

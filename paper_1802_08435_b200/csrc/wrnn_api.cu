@@ -134,6 +134,16 @@ static bool use_pair(const wrnn_model *m, int batch)
     return m->variant == 0 && resident_pair_supported(m, batch) == WRNN_OK;
 }
 
+// 2 to 16 lock-step streams of a dense bf16 H = 896 model: all of them in one launch on the resident weights
+// (WRNN_NO_MULTI=1 falls back to the two-stream and cluster-partitioned kernels: diagnostic)
+static bool use_multi(const wrnn_model *m, int batch)
+{
+    if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_RESIDENT) return false;
+    const char *off = getenv("WRNN_NO_MULTI");
+    if (off && off[0] == '1') return false;
+    return m->variant == 0 && resmulti_supported(m, batch) == WRNN_OK;
+}
+
 static bool use_sparse(const wrnn_model *m, int batch)
 {
     if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_SPARSE) return false;
@@ -206,11 +216,13 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     if (rc != WRNN_OK) return fail(m, rc, "conditioning projection launch failed");
     // staggered rows: the cluster-partitioned kernel, else the any-shape kernel
     if (a.row_lag > 0) {
+        if (a.batch >= 2 && use_multi(m, a.batch)) return resmulti_run(m, a, s);
         if (a.batch >= 2 && use_bcluster(m, a.batch)) return bcluster_run(m, a, s);
         if (a.batch == 1 && use_resident(m, 1)) return resident_run(m, a, s);     // a lone row (the ramps of the schedule)
         return generic_run(m, a, s);
     }
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
+    if (use_multi(m, a.batch)) return resmulti_run(m, a, s);
     if (use_pair(m, a.batch)) {
         for (int pair = 0; pair < a.batch / 2; ++pair) {
             rc = resident_pair_run(m, a, pair, s);
@@ -404,6 +416,7 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
             wrnn_destroy(m);
             return fail(nullptr, rc, "resident kernel unavailable: " + why);
         }
+        if (m->dtype == WRNN_BF16 && m->variant == 0 && max_batch >= 2) resmulti_prepare(m);   // optional: other kernels serve the batch without it
     }
     *out = m;
     return WRNN_OK;
@@ -416,6 +429,7 @@ void wrnn_destroy(wrnn_model *m)
     cudaDeviceSynchronize();
     resident_destroy(m);
     resf32_destroy(m);
+    resmulti_destroy(m);
     batched_destroy(m);
     bcluster_destroy(m);
     sparse_destroy(m);
@@ -715,6 +729,10 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
     }
+    if (use_multi(m, batch)) {
+        if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
+        return resmulti_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
+    }
     if (use_pair(m, batch)) {
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
@@ -747,6 +765,7 @@ int wrnn_phase_cycles(wrnn_model *m, int64_t *out16)
     if (!m || !out16) return WRNN_ERR_INVALID_ARG;
     static_assert(sizeof(long long) == sizeof(int64_t), "");
     if (m->resf32) return resf32_phase_cycles(m, reinterpret_cast<long long *>(out16));
+    if (m->prof_multi) return resmulti_phase_cycles(m, reinterpret_cast<long long *>(out16));
     return resident_phase_cycles(m, reinterpret_cast<long long *>(out16));
 }
 

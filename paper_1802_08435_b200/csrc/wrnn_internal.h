@@ -61,6 +61,7 @@ struct ResidentPack;   // packed weights of the shared-memory-resident kernels (
 struct BatchedPack;    // fragment-packed weights and activation images of the batched kernel (opaque here)
 struct SparsePack;     // compressed block rows of the single-cluster block-sparse kernel (opaque here)
 struct ResF32Pack;     // per-CTA fp32 weight shards of the single-stream fp32 resident kernel (opaque here)
+struct ResMultiPack;  // per-CTA weights of the multi-stream resident kernel (opaque here)
 struct BcPack;         // per-CTA weight slices and stacked activation images of the cluster-partitioned multi-row kernel
 
 }  // namespace wrnn
@@ -96,6 +97,8 @@ struct wrnn_model {
 
     wrnn::ResidentPack *resident = nullptr;
     wrnn::ResF32Pack *resf32 = nullptr;
+    wrnn::ResMultiPack *resmulti = nullptr;
+    bool prof_multi = false;        // the last call with phase timing ran on the multi-stream resident kernel
     wrnn::BatchedPack *batched = nullptr;
     wrnn::SparsePack *sparse_pack = nullptr;
     wrnn::BcPack *bcluster = nullptr;
@@ -133,6 +136,14 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
 int resident_phase_cycles(const wrnn_model *m, long long *out16);
 int resident_pair_supported(const wrnn_model *m, int batch);          // two streams per launch on the same weights (batch 2 or 4)
 int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s);
+
+// wrnn_resmulti.cu: 2 to 16 lock-step streams of a dense bf16 H = 896 model on resident weights
+int resmulti_supported(const wrnn_model *m, int batch);
+int resmulti_prepare(wrnn_model *m);
+void resmulti_destroy(wrnn_model *m);
+int resmulti_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem, int64_t *weight_bytes);
+int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
+int resmulti_phase_cycles(const wrnn_model *m, long long *out16);
 
 // wrnn_resf32.cu: the same role for dense fp32 models (every matrix sharded chip-wide, nothing replicated)
 int resf32_supported(const wrnn_model *m, int batch, std::string *why);

@@ -1184,6 +1184,7 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
         return WRNN_ERR_CUDA;
     }
     ++g_launches;
+    m->prof_multi = false;
     return WRNN_OK;
 }
 
@@ -1241,6 +1242,7 @@ int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s
         return WRNN_ERR_CUDA;
     }
     ++g_launches;
+    m->prof_multi = false;
     return WRNN_OK;
 }
 

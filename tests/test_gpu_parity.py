@@ -4,6 +4,8 @@ Tolerances (per vector v at each step: |gpu_i - ref_i| <= tol * max(|ref_i|, rms
 1e-4 for fp32 weights, 2e-3 for bf16 weights (the oracle uses the same bf16-rounded weights);
 drawn indices bit-exact except where the uniform lies within 1e-5 of a CDF boundary.
 """
+import os
+
 import numpy as np
 import pytest
 
@@ -417,21 +419,27 @@ def test_resident_kernel_short_calls_and_resume(env):
         B.wrnn_destroy(m)
 
 
-@pytest.mark.parametrize("batch", [2, 4])
-def test_two_stream_resident_kernel(env, batch):
-    """Two and four streams of the dense H = 896 bf16 model run as pairs on the two-stream form of the resident kernel:
-    every gate, state and logit of every row against the oracle (rows keep their own conditioning offsets and Philox
-    streams), then a free run, a resumed run and the cross-check against the cluster-partitioned kernel."""
+@pytest.mark.parametrize("batch,form", [(2, "multi"), (3, "multi"), (4, "multi"), (7, "multi"), (13, "multi"), (2, "pair"), (4, "pair")])
+def test_multi_stream_resident_kernels(env, batch, form):
+    """Several streams of the dense H = 896 bf16 model on resident weights -- all of them in one launch of the
+    multi-stream kernel (2 to 16 streams: one to four MMA column groups, heads of a column group per cluster), or as
+    pairs on the two-stream kernel: every gate, state and logit of every row against the oracle (rows keep their own
+    conditioning offsets and Philox streams), then a free run, a resumed run and the cross-check against the
+    single-stream kernel."""
     torch, B = env
     wl = synth.WORKLOADS[7]                      # four streams of the dense model
     w, masks, cond = synth.build_workload(wl, batch=batch)
     om = orc.OracleModel(w, wl.dtype)
     n = 400
+    if form == "pair":
+        os.environ["WRNN_NO_MULTI"] = "1"
     m = B.wrnn_create(w, wl.dtype, max_batch=batch)
     try:
-        assert B.wrnn_launch_info(m, batch)["kernel"] == B.WRNN_KERNEL_RESIDENT
+        info = B.wrnn_launch_info(m, batch)
+        assert info["kernel"] == B.WRNN_KERNEL_RESIDENT
+        assert (info["smem_bytes"] > 200000) == (form == "multi")          # the multi-stream kernel holds all streams' images
         r = pu.teacher_forced_parity(torch, B, m, om, cond, n, batch, SEED, row_stride=1, row_offset_mul=7, stream0=3, threads=pu.NCPU)
-        _report("two-stream resident, batch %d" % batch, r)
+        _report("%s-stream resident, batch %d" % (form, batch), r)
         _tol_check(r, wl.dtype)
         full = _free_run(torch, B, m, cond, n, batch, SEED, row_offset_mul=7, stream0=3)
         h = torch.zeros((batch, wl.H), dtype=torch.float32, device="cuda:0")
@@ -440,12 +448,14 @@ def test_two_stream_resident_kernel(env, batch):
         a = _free_run(torch, B, m, cond, 150, batch, SEED, row_offset_mul=7, stream0=3, h=h, c_prev=cp, f_prev=fp)
         b = _free_run(torch, B, m, cond, n - 150, batch, SEED, row_offset_mul=7, stream0=3, h=h, c_prev=cp, f_prev=fp, step0=150)
         assert np.array_equal(np.concatenate([a, b], axis=1), full)
+        assert np.array_equal(_free_run(torch, B, m, cond, n, batch, SEED, row_offset_mul=7, stream0=3), full)     # deterministic
         # each row equals the single-stream kernel on that row alone
         one = _free_run(torch, B, m, cond[batch - 1:batch], n, 1, SEED, row_offset_mul=7, stream0=3 + batch - 1)
         d = np.nonzero(one[0] != full[batch - 1])[0]
         assert d.size == 0 or r["oracle"].margins[batch - 1, d[0]].min() < pu.MARGIN
     finally:
         B.wrnn_destroy(m)
+        os.environ.pop("WRNN_NO_MULTI", None)
 
 
 def test_config2_sparse_bf16(env):
@@ -517,17 +527,21 @@ def test_sparse_16x1_blocks_cluster_kernel(env):
             B.wrnn_destroy(m)
 
 
-def test_config3_subscale_fold_batch16(env):
-    """One 24,000-sample sequence as 16 interleaved sub-sequences of 1,500 steps in lock-step, then unfolded."""
+@pytest.mark.parametrize("kernel", ["auto", "bcluster"])
+def test_config3_subscale_fold_batch16(env, kernel):
+    """One 24,000-sample sequence as 16 interleaved sub-sequences of 1,500 steps in lock-step, then unfolded: on the
+    multi-stream resident kernel (the default for 2 to 16 rows) and on the cluster-partitioned kernel."""
     torch, B = env
     wl = synth.WORKLOADS[3]
     w, masks, cond = synth.build_workload(wl)
     om = orc.OracleModel(w, wl.dtype)
-    m = B.wrnn_create(w, wl.dtype, max_batch=16)
+    kid = B.WRNN_KERNEL_AUTO if kernel == "auto" else B.WRNN_KERNEL_BCLUSTER
+    m = B.wrnn_create(w, wl.dtype, max_batch=16, kernel=kid)
     try:
+        assert B.wrnn_launch_info(m, 16)["kernel"] == (B.WRNN_KERNEL_RESIDENT if kernel == "auto" else B.WRNN_KERNEL_BCLUSTER)
         r = pu.teacher_forced_parity(torch, B, m, om, cond, wl.n_steps, 16, SEED, row_stride=16, row_offset_mul=1,
                                      threads=pu.NCPU)
-        _report("config3/subscale16", r)
+        _report("config3/subscale16/" + kernel, r)
         _tol_check(r, wl.dtype)
         out = torch.zeros(24000, dtype=torch.int16, device="cuda:0")
         B.wrnn_sample_subscale(m, torch.from_numpy(cond).cuda(), 24000, 16, SEED, out)
@@ -537,9 +551,11 @@ def test_config3_subscale_fold_batch16(env):
         div = pu.first_divergence(sub, r["oracle"].out)
         if div >= 0:
             assert r["oracle"].margins[:, div].min() < pu.MARGIN
-        # rows are independent: row 5 alone (global row id 5) reproduces row 5 of the batch
-        one = _free_run(torch, B, m, cond[5:6], wl.n_steps, 1, SEED, row_stride=16, row_offset_mul=1, stream0=5)
-        assert np.array_equal(one[0], sub[5])
+        # rows are independent: row 5 alone (global row id 5, another kernel) reproduces row 5 of the batch
+        if kernel == "auto":             # (the cluster-partitioned family takes two or more rows)
+            one = _free_run(torch, B, m, cond[5:6], wl.n_steps, 1, SEED, row_stride=16, row_offset_mul=1, stream0=5)
+            d = np.nonzero(one[0] != sub[5])[0]
+            assert d.size == 0 or r["oracle"].margins[5, d[0]].min() < pu.MARGIN
     finally:
         B.wrnn_destroy(m)
 

@@ -44,7 +44,8 @@ def _gpu_run(torch, Bn, m, frames, V, b, F, chunk, lag, B_rows, L, hop=synth.HOP
 
 @pytest.mark.parametrize("H,dtype,B_rows,L,F,chunk,kernel", [
     (32, "f32", 4, 90, 6, 3, "generic"), (64, "bf16", 5, 64, 8, 8, "generic"), (896, "bf16", 16, 300, 32, 32, "generic"),
-    (896, "bf16", 16, 300, 32, 32, "auto"),      # two or more active rows run on the cluster-partitioned kernel
+    (896, "bf16", 16, 300, 32, 32, "auto"),      # four or more active rows advance together on the multi-stream resident kernel
+    (896, "bf16", 16, 300, 32, 32, "bcluster"),  # the same on the cluster-partitioned kernel (lone rows on the any-shape kernel)
 ])
 def test_staggered_schedule_and_oracle(env, H, dtype, B_rows, L, F, chunk, kernel):
     torch, Bn = env
@@ -60,10 +61,11 @@ def test_staggered_schedule_and_oracle(env, H, dtype, B_rows, L, F, chunk, kerne
         Bn.wrnn_subscale_conditioning(hist, fr_d, V_d, b_d, F, row, v)
         torch.cuda.synchronize()
         assert pu.rel_err(v.cpu().numpy(), cond_ref[row]) < 1e-5, row
-    m = Bn.wrnn_create(w, dtype, max_batch=B_rows, kernel=Bn.WRNN_KERNEL_GENERIC if kernel == "generic" else Bn.WRNN_KERNEL_AUTO)
+    m = Bn.wrnn_create(w, dtype, max_batch=B_rows, kernel={"generic": Bn.WRNN_KERNEL_GENERIC, "auto": Bn.WRNN_KERNEL_AUTO,
+                                                           "bcluster": Bn.WRNN_KERNEL_BCLUSTER}[kernel])
     try:
-        if kernel == "auto":
-            assert Bn.wrnn_launch_info(m, B_rows)["kernel"] == Bn.WRNN_KERNEL_BCLUSTER
+        if kernel != "generic":
+            assert Bn.wrnn_launch_info(m, B_rows)["kernel"] == (Bn.WRNN_KERNEL_RESIDENT if kernel == "auto" else Bn.WRNN_KERNEL_BCLUSTER)
         lag = F + chunk if (F + chunk) % chunk == 0 else ((F + chunk + chunk - 1) // chunk) * chunk
         stag = _gpu_run(torch, Bn, m, frames, V, b, F, chunk, lag, B_rows, L)
         # row after row: a lag beyond the row length leaves one row active at a time

@@ -9,7 +9,8 @@
 //     (columns 2 j, 2 j + 1 = the bf16 high and low parts of stream j's fp32 vector), so 16 streams are four column
 //     groups;
 //   * the output heads are still held once per cluster, but cluster c serves only the streams of column group c
-//     (streams 4 c .. 4 c + 3): one MMA column group per head, as for a single stream.  The logits go to the cluster's
+//     (streams 4 c .. 4 c + 3) or, with up to seven streams, stream c alone (its state half is kept a second time as a
+//     column group of its own): one MMA column group per head, as for a single stream.  The logits go to the cluster's
 //     first CTA, which draws; the symbols travel to the gate threads of all CTAs through tagged L2 words;
 //   * the recurrent products of a half step are not needed before the gates at its end, so twelve warps compute them
 //     while the other four wait for the logits, draw and broadcast: they are off the critical path.
@@ -74,6 +75,7 @@ struct MultiParams {
     DevStatus *status;
     unsigned long long limit_ns;
     long long *prof;
+    unsigned flag_mode;                      // bit 0 / 1: with one / several column groups the gather waits for this CTA's own publication first
 };
 
 // Position (in bf16 units) of element i of column `col` in a column-group image: [k-tile pair][8 columns][4 t][2 k-tiles][4 bf16],
@@ -112,7 +114,10 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     const int cta = blockIdx.x, cl = cta / MCS;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int H = p.H, NS = p.NS, NG = (NS + 3) >> 2;
-    const int own_n = min(4, max(0, NS - 4 * cl));           // streams whose heads this cluster holds
+    // streams whose heads this cluster holds: up to seven streams, one per cluster (the exchanges inside a cluster are
+    // those of a single stream); more streams, the four of column group cl
+    const bool spread = NS <= MNC;
+    const int own_n = spread ? (cl < NS ? 1 : 0) : min(4, max(0, NS - 4 * cl));
     constexpr int K = MK;
 
     // ---- shared memory carve-up (must match resmulti_smem_bytes)
@@ -128,20 +133,23 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     float *part0 = part_R + PR_FLOATS;                                         // [4 streams][8 slots][16] (+8 per stream)
     uint4 *spl = reinterpret_cast<uint4 *>(part0 + 4 * P0S);                   // [4 column groups] images of the state half
     uint4 *splQ = spl + 4 * IMG_U4;                                            // image of the hidden layers of the own streams
-    float *qbuf = reinterpret_cast<float *>(splQ + IMG_U4);                    // [2 parities][4 streams][K]
+    uint4 *splOwn = splQ + IMG_U4;                                             // up to seven streams: the own stream's state half as a column group of its own
+    float *qbuf = reinterpret_cast<float *>(splOwn + IMG_U4);                    // [2 parities][4 streams][K]
     uint4 *lbuf = reinterpret_cast<uint4 *>(qbuf + 8 * K);                     // [2 parities][4 streams][128] {v, tag, v, tag}
     __shared__ __align__(8) unsigned long long xbar[2];
+    __shared__ long long s_pub;                 // the last half step whose state values this CTA's gate threads have published
 
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(p.blob + (size_t)cta * p.blob_bytes);
         uint4 *dst = reinterpret_cast<uint4 *>(smem);
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
         for (int i = tid; i < 8 * K + 4096; i += blockDim.x) qbuf[i] = 0.f;              // qbuf and lbuf are adjacent
-        for (int i = tid; i < 5 * IMG_U4; i += blockDim.x) spl[i] = make_uint4(0, 0, 0, 0);  // spl and splQ are adjacent
+        for (int i = tid; i < 6 * IMG_U4; i += blockDim.x) spl[i] = make_uint4(0, 0, 0, 0);  // spl, splQ and splOwn are adjacent
         for (int i = tid; i < 2 * MAXS * MNR + PR_FLOATS + 4 * P0S; i += blockDim.x) a_part[i] = 0.f;
         if (tid == 0) {
             for (int i = 0; i < 2; ++i) mbar_init_cluster(smem_addr(&xbar[i]), 1);
             mbar_fence_init();
+            s_pub = -1;
         }
     }
     __syncthreads();
@@ -160,7 +168,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     // ---- roles
     const int ws = warp;                                  // drawing warps 0..3: own stream ws
     const bool drawer = warp < 4 && ws < own_n && rank == 0;   // the cluster's first CTA draws for its streams
-    const int d_st = 4 * cl + ws;                         // the stream a drawing warp serves
+    const int d_st = spread ? cl : 4 * cl + ws;           // the stream a drawing warp serves
     const int rw = warp - 4, ridx = tid - 128;            // warps 4..15: recurrent rows, then the gates
     const bool gater = warp >= 4 && ridx < NS * MUC;
     const int gst = ridx / MUC, gu = ridx % MUC;          // (stream, unit) of a gate thread
@@ -273,6 +281,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         load_g(0, 0, gv);
         gates_and_publish(0, 0, f_prev, gates_prepare(0, gv));
     }
+    if (warp == 4) { __syncwarp(); if (lane == 0) *(volatile long long *)&s_pub = 0; }
 
     // send addresses: one peer per warp
     const int q_st = lane / 7, q_quad = lane % 7;             // hidden layer: lanes [0, 28): stream, four rows
@@ -331,39 +340,48 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                 at[q] = lin + rot < total ? lin + rot : lin + rot - total;
                 v0[q] = v1[q] = 0;
             }
-            // the first pair alone until it is there (most of the wait: one load in flight per thread), then all the others
-            // together, round after round, so that their round trips overlap; a pair goes into the image as soon as it is there
+            // a pair goes into the image as soon as it is there
             auto put = [&](int q) {
                 const int idx = at[q];
                 const int st = (2 * idx) / K, j = 2 * idx - st * K;
-                mimg_store_pair(spl, st, j, __uint_as_float((unsigned)v0[q]), __uint_as_float((unsigned)v1[q]));
+                const float x0 = __uint_as_float((unsigned)v0[q]), x1 = __uint_as_float((unsigned)v1[q]);
+                mimg_store_pair(spl, st, j, x0, x1);
+                if (spread && st == cl) mimg_store_pair(splOwn, 0, j, x0, x1);
             };
             unsigned pending = 0;
 #pragma unroll
-            for (int q = 1; q < NPT; ++q) if (tid + q * 512 < total) pending |= 1u << q;
-            if (tid < total) {
-                unsigned long long t0 = 0; unsigned cnt = 0;
-                while (true) {
-                    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0[0]), "=l"(v1[0]) : "l"(slots + 2 * at[0]) : "memory");
-                    if ((unsigned)(v0[0] >> 32) == ytag && (unsigned)(v1[0] >> 32) == ytag) break;
-                    if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
-                }
-#pragma unroll
-                for (int q = 1; q < NPT; ++q)
-                    if (pending & (1u << q))
-                        asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0[q]), "=l"(v1[q]) : "l"(slots + 2 * at[q]) : "memory");
-                put(0);
-            }
+            for (int q = 0; q < NPT; ++q) if (tid + q * 512 < total) pending |= 1u << q;
             {
                 unsigned long long t0 = 0; unsigned cnt = 0;
+                if (p.flag_mode & (NG == 1 ? 1u : 2u)) {
+                    // few streams: nobody polls L2 before this CTA's own gate threads have published (the others do so at
+                    // about the same time), so the publishing stores do not queue behind polls
+                    while (*(volatile long long *)&s_pub < n - 1)
+                        if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+                }
+                if (NG > 1 && (pending & 1u) && !my_bad) {
+                    // many streams: the first pair alone until it is there, so that the wait does not multiply the polling traffic
+                    while (true) {
+                        asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0[0]), "=l"(v1[0]) : "l"(slots + 2 * at[0]) : "memory");
+                        if ((unsigned)(v0[0] >> 32) == ytag && (unsigned)(v1[0] >> 32) == ytag) break;
+                        if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+                    }
+                    pending &= ~1u;
+                }
+                // then all pairs of the thread together, round after round, so that their round trips overlap
+#pragma unroll
+                for (int q = 0; q < NPT; ++q)
+                    if (pending & (1u << q))
+                        asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0[q]), "=l"(v1[q]) : "l"(slots + 2 * at[q]) : "memory");
+                if (NG > 1 && tid < total && !my_bad) put(0);
                 while (pending && !my_bad) {
 #pragma unroll
-                    for (int q = 1; q < NPT; ++q)
+                    for (int q = 0; q < NPT; ++q)
                         if ((pending & (1u << q)) && (unsigned)(v0[q] >> 32) == ytag && (unsigned)(v1[q] >> 32) == ytag) { pending &= ~(1u << q); put(q); }
                     if (!pending) break;
                     if ((++cnt & 1023u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
 #pragma unroll
-                    for (int q = 1; q < NPT; ++q)
+                    for (int q = 0; q < NPT; ++q)
                         if (pending & (1u << q))
                             asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0[q]), "=l"(v1[q]) : "l"(slots + 2 * at[q]) : "memory");
                 }
@@ -378,7 +396,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                 const int tsel = warp & 1, sp = warp >> 1;
                 const int p0 = (MKP * sp) / 4, p1 = (MKP * (sp + 1)) / 4;
                 float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                const uint4 *bimg = spl + cl * IMG_U4 + g4 * 4 + t4;
+                const uint4 *bimg = (spread ? splOwn : spl + cl * IMG_U4) + g4 * 4 + t4;
                 const uint4 *A = M + (2 + tsel) * TILE_U4 + lane;
 #pragma unroll 2
                 for (int kp = p0; kp < p1; ++kp) {
@@ -506,6 +524,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                 if (!my_bad) gates_and_publish(half, s, fed, gp);
                 if (half) c_prev = fed; else f_prev = fed;
             }
+            if (warp == 4 && !last) { __syncwarp(); if (lane == 0 && !my_bad) *(volatile long long *)&s_pub = n; }
         }
     }
     if (prof_on && lane == 0) for (int i = 0; i < 16; ++i) p.prof[i] = s_prof[i];
@@ -528,7 +547,7 @@ static int resmulti_smem_bytes(const ResMultiPack &k)
     size_t b = k.blob_bytes;
     b += (size_t)2 * MAXS * MNR * 4;                // a_part, a_full
     b += (size_t)PR_FLOATS * 4 + (size_t)4 * P0S * 4;
-    b += (size_t)5 * IMG_U4 * 16;                   // four column-group images + the hidden-layer image
+    b += (size_t)6 * IMG_U4 * 16;                   // four column-group images, the hidden-layer image, the own streams' image
     b += (size_t)8 * MK * 4;                        // qbuf
     b += (size_t)1024 * 16;                         // lbuf
     return (int)b;
@@ -701,6 +720,7 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.status = m->status;
     p.limit_ns = 2000000000ull;
     p.prof = k.d_prof;
+    { const char *d = getenv("WRNN_MULTI_FLAG"); p.flag_mode = d ? (unsigned)atoi(d) : 1u; }    // diagnostic: A/B of the gather protocol
 
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * MAXS * MK * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(k.d_sym, 0, (size_t)4 * 32 * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;

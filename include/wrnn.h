@@ -57,7 +57,7 @@ typedef enum { WRNN_F32 = 0, WRNN_BF16 = 1 } wrnn_dtype;
 typedef enum {
     WRNN_KERNEL_AUTO = 0,       /* the fastest one that supports the model and batch          */
     WRNN_KERNEL_GENERIC = 1,    /* weights streamed from L2 every step; any shape; bring-up path */
-    WRNN_KERNEL_RESIDENT = 2,   /* persistent kernel, weights resident in shared memory (one row) */
+    WRNN_KERNEL_RESIDENT = 2,   /* persistent kernel, weights resident in shared memory (one row; 2 to 16 rows of a dense bf16 H = 896 model) */
     WRNN_KERNEL_BATCHED = 3,    /* tensor-pipe contractions over all rows (dense bf16, >= 2 rows)  */
     WRNN_KERNEL_SPARSE = 4,     /* block-sparse model resident in 16-CTA clusters (one row)        */
     WRNN_KERNEL_BCLUSTER = 5    /* rows dealt to 16-CTA clusters, tcgen05 contractions (dense bf16, >= 2 rows) */

@@ -608,9 +608,10 @@ int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n
     auto run_rows = [&](int r_a, int n_rows, long long p_lo, int n) -> int {
         int rc = subscale_cond_launch(hist, frames, V, bias, v, B, L, F, D, n_frames, hop, r_a, n_rows, p_lo, lag, n, s);
         if (rc != WRNN_OK) return fail(m, rc, "conditioning launch failed");
-        // up to three rows go one after the other through the single-stream kernel where the model has one (6.6 us per
-        // step and row against 24 us per step of the multi-row kernel); more rows advance together
-        const int group = (n_rows <= 3 && use_resident(m, 1)) ? 1 : n_rows;
+        // rows advance together on the multi-stream resident kernel where the model has one (8.3 us per step at two rows
+        // against 6.4 us per step and row on the single-stream kernel); without it up to three rows go one after the other
+        // through the single-stream kernel (24 us per step of the cluster-partitioned kernel whatever the rows)
+        const int group = (n_rows >= 2 && use_multi(m, n_rows)) ? n_rows : (n_rows <= 3 && use_resident(m, 1)) ? 1 : n_rows;
         for (int b0 = 0; b0 < n_rows; b0 += group) {
             const int r0 = r_a + b0;
             const long long p0 = p_lo - (long long)b0 * lag;

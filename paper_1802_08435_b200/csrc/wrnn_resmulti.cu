@@ -11,7 +11,10 @@
 //   * the output heads are still held once per cluster, but cluster c serves only the streams of column group c
 //     (streams 4 c .. 4 c + 3) or, with up to seven streams, stream c alone (its state half is kept a second time as a
 //     column group of its own): one MMA column group per head, as for a single stream.  The logits go to the cluster's
-//     first CTA, which draws; the symbols travel to the gate threads of all CTAs through tagged L2 words;
+//     first CTA, which draws;
+//   * the gates of a stream are computed in the cluster that draws it (every CTA of the cluster takes 28 state units of
+//     each half), so the drawn symbol only crosses distributed shared memory; the rows of R h they need are published
+//     by the CTAs that own those rows of R as tagged L2 words, once per step, half a step or more before they are used;
 //   * the recurrent products of a half step are not needed before the gates at its end, so twelve warps compute them
 //     while the other four wait for the logits, draw and broadcast: they are off the critical path.
 // Every wait is bounded; a CTA that gives up records where and all CTAs leave through the final cluster barrier.
@@ -50,7 +53,7 @@ struct ResMultiPack {
     size_t blob_bytes = 0, w_bytes = 0;
     uint8_t *d_blob = nullptr;               // [112][blob_bytes]
     unsigned long long *d_slots = nullptr;   // [2 halves][2 parities][16 streams][K] (value, tag)
-    unsigned long long *d_sym = nullptr;     // [4][32] (symbol, tag)
+    unsigned long long *d_aslots = nullptr;  // [2 parities][16 streams][2 halves x 3 gates x K] (R h value, tag)
     long long *d_prof = nullptr;             // [16]
     int smem_bytes = 0;
     int64_t weight_bytes_per_step = 0;
@@ -65,7 +68,8 @@ struct MultiParams {
     long long out_pitch;
     const uint8_t *blob; unsigned long long blob_bytes, w_bytes;
     const float *g;                          // [NS][n_frames][3H]
-    unsigned long long *slots, *sym;
+    unsigned long long *slots, *aslots;
+    const float *I;                          // [3H][3] input weights (fp32, masked column zeroed)
     const float *h_in; float *h_out;
     const uint8_t *c_in, *f_in; uint8_t *c_st_out, *f_st_out;
     const uint8_t *c_forced, *f_forced;
@@ -128,8 +132,8 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     const float *sI = reinterpret_cast<const float *>(smem + p.w_bytes);       // [24][3]
     const float *sb1 = sI + MNR * 3, *sb3 = sb1 + MHR, *sb2 = sb3 + MHR, *sb4 = sb2 + MLR;
     float *a_part = reinterpret_cast<float *>(smem + p.blob_bytes);            // [16][24] R[:, :K] y_c
-    float *a_full = a_part + MAXS * MNR;                                       // [16][24] R h
-    float *part_R = a_full + MAXS * MNR;                                       // [streams][2 tiles x slots][16] (+8 per stream)
+    float *sIg = a_part + MAXS * MNR;                                          // [2 halves][3 gates][28 units][3] input weights of the gate threads' units
+    float *part_R = sIg + 2 * 3 * MHR * 3 + 8;                                       // [streams][2 tiles x slots][16] (+8 per stream)
     float *part0 = part_R + PR_FLOATS;                                         // [4 streams][8 slots][16] (+8 per stream)
     uint4 *spl = reinterpret_cast<uint4 *>(part0 + 4 * P0S);                   // [4 column groups] images of the state half
     uint4 *splQ = spl + 4 * IMG_U4;                                            // image of the hidden layers of the own streams
@@ -137,6 +141,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     float *qbuf = reinterpret_cast<float *>(splOwn + IMG_U4);                    // [2 parities][4 streams][K]
     uint4 *lbuf = reinterpret_cast<uint4 *>(qbuf + 8 * K);                     // [2 parities][4 streams][128] {v, tag, v, tag}
     __shared__ __align__(8) unsigned long long xbar[2];
+    __shared__ __align__(8) unsigned long long s_sym[8];   // [2 parities][4 own streams] (symbol, tag) from the drawing CTA
     __shared__ long long s_pub;                 // the last half step whose state values this CTA's gate threads have published
 
     {
@@ -145,12 +150,18 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
         for (int i = tid; i < 8 * K + 4096; i += blockDim.x) qbuf[i] = 0.f;              // qbuf and lbuf are adjacent
         for (int i = tid; i < 6 * IMG_U4; i += blockDim.x) spl[i] = make_uint4(0, 0, 0, 0);  // spl, splQ and splOwn are adjacent
-        for (int i = tid; i < 2 * MAXS * MNR + PR_FLOATS + 4 * P0S; i += blockDim.x) a_part[i] = 0.f;
+        for (int i = tid; i < MAXS * MNR + 2 * 3 * MHR * 3 + 8 + PR_FLOATS + 4 * P0S; i += blockDim.x) a_part[i] = 0.f;
         if (tid == 0) {
             for (int i = 0; i < 2; ++i) mbar_init_cluster(smem_addr(&xbar[i]), 1);
             mbar_fence_init();
             s_pub = -1;
         }
+        if (tid < 8) s_sym[tid] = 0;
+    }
+    __syncthreads();
+    for (int i = tid; i < 2 * 3 * MHR * 3; i += blockDim.x) {
+        const int c = i % 3, gq = (i / 3) % MHR, hg = i / (3 * MHR);          // hg = half * 3 + gate
+        sIg[i] = p.I[((size_t)(hg % 3) * H + (hg / 3) * K + MHR * rank + gq) * 3 + c];
     }
     __syncthreads();
     cluster.sync();
@@ -170,8 +181,10 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     const bool drawer = warp < 4 && ws < own_n && rank == 0;   // the cluster's first CTA draws for its streams
     const int d_st = spread ? cl : 4 * cl + ws;           // the stream a drawing warp serves
     const int rw = warp - 4, ridx = tid - 128;            // warps 4..15: recurrent rows, then the gates
-    const bool gater = warp >= 4 && ridx < NS * MUC;
-    const int gst = ridx / MUC, gu = ridx % MUC;          // (stream, unit) of a gate thread
+    // gate threads: the state units 28 rank .. + 27 of both halves, for every own stream of the cluster
+    const bool gater = warp >= 4 && ridx < own_n * MHR;
+    const int gl = ridx / MHR, gq = ridx % MHR;           // (own stream, unit of this CTA's share) of a gate thread
+    const int gst = (spread ? cl : 4 * cl) + gl, gj = MHR * rank + gq;
     const int r_cg = rw >= 0 ? rw % NG : 0, r_j = rw >= 0 ? rw / NG : 0;
     const int nsl = (NRW + NG - 1) / NG, PS = 2 * nsl * 16 + 8;
 
@@ -207,14 +220,20 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
             d[g4 + 8] = (acc[n][0][2] + acc[n][1][2]) + (acc[n][0][3] + acc[n][1][3]);
         }
     };
-    auto r_sums = [&](bool completes) {
+    // sums of the K-split partials; a completed row of R h (tag: the step whose gates use it, + 1) goes to the cluster
+    // that computes the gates of its stream
+    auto r_sums = [&](bool completes, long long s_use) {
         if (ridx < NS * MNR) {
             const int st = ridx / MNR, row = ridx - st * MNR;
             const int cgp = st >> 2, nw = (NRW - cgp + NG - 1) / NG;
             const float *s = part_R + st * PS + ((row >> 4) * nsl) * 16 + (row & 15);
             float v = 0.f;
             for (int j = 0; j < nw; ++j) v += s[j * 16];
-            if (completes) a_full[ridx] = a_part[ridx] + v; else a_part[ridx] = v;
+            if (completes) {
+                const int hg = row / MUC, u = row % MUC;                         // hg = half * 3 + gate
+                st_relaxed_u64(p.aslots + ((size_t)(s_use & 1) * NS + st) * (6 * K) + hg * K + cta * MUC + u,
+                               ((unsigned long long)(unsigned)(s_use + 1) << 32) | __float_as_uint(a_part[ridx] + v));
+            } else a_part[ridx] = v;
         }
     };
     auto fill_image = [&](int part) {
@@ -228,11 +247,11 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     // ---- prologue: R h of the initial state
     fill_image(0);
     __syncthreads();
-    if (warp >= 4) { r_products(wMA); named_sync(1, 384); r_sums(false); }
+    if (warp >= 4) { r_products(wMA); named_sync(1, 384); r_sums(false, 0); }
     __syncthreads();
     fill_image(1);
     __syncthreads();
-    if (warp >= 4) { r_products(wMB); named_sync(1, 384); r_sums(true); named_sync(1, 384); }
+    if (warp >= 4) { r_products(wMB); named_sync(1, 384); r_sums(true, 0); }
     __syncthreads();
 
     // state of a gate thread: its unit of both halves of its stream, and the stream's last symbols
@@ -240,21 +259,33 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     float hC = 0.f, hF = 0.f;
     if (gater) {
         c_prev = p.c_in ? p.c_in[gst] : 128; f_prev = p.f_in ? p.f_in[gst] : 0;
-        if (p.h_in) { hC = p.h_in[(size_t)gst * H + cta * MUC + gu]; hF = p.h_in[(size_t)gst * H + K + cta * MUC + gu]; }
+        if (p.h_in) { hC = p.h_in[(size_t)gst * H + gj]; hF = p.h_in[(size_t)gst * H + K + gj]; }
     }
     if (drawer) { c_prev = p.c_in ? p.c_in[d_st] : 128; f_prev = p.f_in ? p.f_in[d_st] : 0; }
 
     struct GatePre { float pu, pr, pe, ae, ku, kr, ke; };
-    auto gates_prepare = [&](int half_g, const float (&gv)[3]) {
+    // the three rows of R h of this thread's unit (published by the CTA that owns those rows of R)
+    auto load_a = [&](int half_g, long long s_use, float (&av)[3]) {
+        const unsigned long long *src = p.aslots + ((size_t)(s_use & 1) * NS + gst) * (6 * K) + (half_g * 3) * K + gj;
+        const unsigned atag = (unsigned)(s_use + 1);
+        unsigned long long v[3], t0 = 0; unsigned cnt = 0;
+        while (true) {
+#pragma unroll
+            for (int gate = 0; gate < 3; ++gate) v[gate] = ld_relaxed_u64(src + gate * K);
+            if ((unsigned)(v[0] >> 32) == atag && (unsigned)(v[1] >> 32) == atag && (unsigned)(v[2] >> 32) == atag) break;
+            if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s_use, 9)) { my_bad = true; break; }
+        }
+#pragma unroll
+        for (int gate = 0; gate < 3; ++gate) av[gate] = __uint_as_float((unsigned)v[gate]);
+    };
+    auto gates_prepare = [&](int half_g, const float (&gv)[3], const float (&av)[3]) {
         GatePre q;
-        const int rb = half_g ? 3 * MUC : 0;
         const float x0 = scale8(c_prev), x1 = scale8(f_prev);
-        const float *Iu = sI + 3 * (rb + gu), *Ir = sI + 3 * (rb + MUC + gu), *Ie = sI + 3 * (rb + 2 * MUC + gu);
-        const float *af = a_full + gst * MNR;
-        q.pu = af[rb + gu] + fmaf(Iu[0], x0, half_g ? fmaf(Iu[1], x1, gv[0]) : gv[0]);
-        q.pr = af[rb + MUC + gu] + fmaf(Ir[0], x0, half_g ? fmaf(Ir[1], x1, gv[1]) : gv[1]);
+        const float *Iu = sIg + ((half_g * 3 + 0) * MHR + gq) * 3, *Ir = sIg + ((half_g * 3 + 1) * MHR + gq) * 3, *Ie = sIg + ((half_g * 3 + 2) * MHR + gq) * 3;
+        q.pu = av[0] + fmaf(Iu[0], x0, half_g ? fmaf(Iu[1], x1, gv[0]) : gv[0]);
+        q.pr = av[1] + fmaf(Ir[0], x0, half_g ? fmaf(Ir[1], x1, gv[1]) : gv[1]);
         q.pe = fmaf(Ie[0], x0, half_g ? fmaf(Ie[1], x1, gv[2]) : gv[2]);
-        q.ae = af[rb + 2 * MUC + gu];
+        q.ae = av[2];
         q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
         return q;
     };
@@ -264,22 +295,23 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
-        const int j = cta * MUC + gu, jj = (half_g ? K : 0) + j;
-        st_relaxed_u64(p.slots + ((size_t)((half_g ? 2 : 0) + (s & 1)) * NS + gst) * K + j,
+        const int jj = (half_g ? K : 0) + gj;
+        st_relaxed_u64(p.slots + ((size_t)((half_g ? 2 : 0) + (s & 1)) * NS + gst) * K + gj,
                        ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * NS + gst) * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
         if (p.dbg_h) p.dbg_h[((size_t)s * NS + gst) * H + jj] = hn;
     };
     auto load_g = [&](int half_g, long long s, float (&gv)[3]) {
         const long long fr = p.row_lag > 0 ? s : ((p.step0 + s) * p.row_stride + (long long)(p.stream0 + (unsigned)gst) * p.row_offset_mul) / p.hop;
-        const float *g = p.g + ((size_t)gst * p.n_frames + fr) * 3 * H + (half_g ? K : 0) + cta * MUC + gu;
+        const float *g = p.g + ((size_t)gst * p.n_frames + fr) * 3 * H + (half_g ? K : 0) + gj;
 #pragma unroll
         for (int gate = 0; gate < 3; ++gate) gv[gate] = __ldg(g + gate * H);
     };
     if (gater) {
-        float gv[3];
+        float gv[3], av[3];
         load_g(0, 0, gv);
-        gates_and_publish(0, 0, f_prev, gates_prepare(0, gv));
+        load_a(0, 0, av);
+        if (!my_bad) gates_and_publish(0, 0, f_prev, gates_prepare(0, gv, av));
     }
     if (warp == 4) { __syncwarp(); if (lane == 0) *(volatile long long *)&s_pub = 0; }
 
@@ -353,7 +385,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
             for (int q = 0; q < NPT; ++q) if (tid + q * 512 < total) pending |= 1u << q;
             {
                 unsigned long long t0 = 0; unsigned cnt = 0;
-                if (p.flag_mode & (NG == 1 ? 1u : 2u)) {
+                if (own_n > 0 && (p.flag_mode & (NG == 1 ? 1u : 2u))) {
                     // few streams: nobody polls L2 before this CTA's own gate threads have published (the others do so at
                     // about the same time), so the publishing stores do not queue behind polls
                     while (*(volatile long long *)&s_pub < n - 1)
@@ -486,7 +518,11 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                 const int drawn = warp_softmax_draw_fast(l, u01, lane);
                 const int fed = forced >= 0 ? forced : drawn;
                 {
-                    if (lane == 0 && !my_bad) st_relaxed_u64(p.sym + (n & 3) * 32 + d_st, ((unsigned long long)tag << 32) | (unsigned)fed);
+                    // the symbol to the gate threads of the cluster's 16 CTAs
+                    if (lane < MCS && !my_bad) {
+                        const unsigned dst = map_to_rank(smem_addr(&s_sym[(n & 1) * 4 + ws]), (unsigned)lane);
+                        asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(dst), "l"(((unsigned long long)tag << 32) | (unsigned)fed) : "memory");
+                    }
                     const long long t = half ? s : s - 1;
                     if (p.dbg_logits) {
                         float *d = p.dbg_logits + (((size_t)t * NS + d_st) * 2 + (half ? 0 : 1)) * 256 + 8 * lane;
@@ -509,14 +545,15 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
             r_products(M);
             named_arrive(2, 512);
             named_sync(1, 384);
-            r_sums(!half);
-            named_sync(1, 384);
+            r_sums(!half, s);
             if (gater && !last) {
-                const GatePre gp = gates_prepare(half, gv);
-                const unsigned long long *sp = p.sym + (n & 3) * 32 + gst;
+                float av[3];
+                load_a(half, s, av);
+                const GatePre gp = gates_prepare(half, gv, av);
+                const volatile unsigned long long *sp = &s_sym[(n & 1) * 4 + gl];
                 unsigned long long v, t0 = 0; unsigned cnt = 0;
                 while (true) {
-                    v = ld_relaxed_u64(sp);
+                    v = *sp;
                     if ((unsigned)(v >> 32) == tag) break;
                     if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 4 + 4 * half)) { my_bad = true; break; }
                 }
@@ -532,7 +569,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
 
     const int any_bad = __syncthreads_or(my_bad);
     if (!any_bad) {
-        if (gater && p.h_out) { p.h_out[(size_t)gst * H + cta * MUC + gu] = hC; p.h_out[(size_t)gst * H + K + cta * MUC + gu] = hF; }
+        if (gater && p.h_out) { p.h_out[(size_t)gst * H + gj] = hC; p.h_out[(size_t)gst * H + K + gj] = hF; }
         if (drawer && lane == 0) {
             if (p.c_st_out) p.c_st_out[d_st] = (uint8_t)c_prev;
             if (p.f_st_out) p.f_st_out[d_st] = (uint8_t)f_prev;
@@ -545,7 +582,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
 static int resmulti_smem_bytes(const ResMultiPack &k)
 {
     size_t b = k.blob_bytes;
-    b += (size_t)2 * MAXS * MNR * 4;                // a_part, a_full
+    b += (size_t)MAXS * MNR * 4 + (size_t)(2 * 3 * MHR * 3 + 8) * 4;   // a_part, the gate threads' input weights
     b += (size_t)PR_FLOATS * 4 + (size_t)4 * P0S * 4;
     b += (size_t)6 * IMG_U4 * 16;                   // four column-group images, the hidden-layer image, the own streams' image
     b += (size_t)8 * MK * 4;                        // qbuf
@@ -652,12 +689,12 @@ int resmulti_prepare(wrnn_model *m)
     const bool ok = cudaMalloc((void **)&pk->d_blob, blob.size()) == cudaSuccess &&
                     cudaMemcpy(pk->d_blob, blob.data(), blob.size(), cudaMemcpyHostToDevice) == cudaSuccess &&
                     cudaMalloc((void **)&pk->d_slots, (size_t)4 * MAXS * K * 8) == cudaSuccess &&
-                    cudaMalloc((void **)&pk->d_sym, (size_t)4 * 32 * 8) == cudaSuccess &&
+                    cudaMalloc((void **)&pk->d_aslots, (size_t)2 * MAXS * 6 * K * 8) == cudaSuccess &&
                     cudaMalloc((void **)&pk->d_prof, 16 * sizeof(long long)) == cudaSuccess &&
                     cudaMemset(pk->d_prof, 0, 16 * sizeof(long long)) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
-        cudaFree(pk->d_blob); cudaFree(pk->d_slots); cudaFree(pk->d_sym); cudaFree(pk->d_prof);
+        cudaFree(pk->d_blob); cudaFree(pk->d_slots); cudaFree(pk->d_aslots); cudaFree(pk->d_prof);
         delete pk;
         m->err = "device allocation for the multi-stream resident kernel failed";
         return WRNN_ERR_NOMEM;
@@ -672,7 +709,7 @@ void resmulti_destroy(wrnn_model *m)
     if (!m->resmulti) return;
     cudaFree(m->resmulti->d_blob);
     cudaFree(m->resmulti->d_slots);
-    cudaFree(m->resmulti->d_sym);
+    cudaFree(m->resmulti->d_aslots);
     cudaFree(m->resmulti->d_prof);
     delete m->resmulti;
     m->resmulti = nullptr;
@@ -713,7 +750,7 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.row_offset_mul = m->cond_dim ? a.row_offset_mul : 0;
     p.row_lag = a.row_lag; p.out_pitch = a.out_pitch ? a.out_pitch : a.n_steps;
     p.blob = k.d_blob; p.blob_bytes = k.blob_bytes; p.w_bytes = k.w_bytes;
-    p.g = m->g; p.slots = k.d_slots; p.sym = k.d_sym;
+    p.g = m->g; p.slots = k.d_slots; p.aslots = k.d_aslots; p.I = m->I;
     p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in; p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
@@ -723,7 +760,7 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     { const char *d = getenv("WRNN_MULTI_FLAG"); p.flag_mode = d ? (unsigned)atoi(d) : 1u; }    // diagnostic: A/B of the gather protocol
 
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * MAXS * MK * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
-    if (cudaMemsetAsync(k.d_sym, 0, (size_t)4 * 32 * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
+    if (cudaMemsetAsync(k.d_aslots, 0, (size_t)2 * MAXS * 6 * MK * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     const char *no_coop = getenv("WRNN_NO_COOP");

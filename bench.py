@@ -305,6 +305,14 @@ def main():
                          "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_wait_recurrent",
                          "F.hid_products", "C.hid_products", "F.log_products", "C.log_products"]
                 roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
+                # the lock-step is the same chain of two chip-wide exchanges as a single stream's step: its floor
+                t_bar_ns = B.wrnn_measure_exchange_floor(info["n_ctas"], info["n_threads"], Hh, 20000)
+                smem_us = (3 * H * H + 2 * Hh * Hh + 2 * 256 * Hh) * 2 / (SMEM_PEAK_GBS * 1e3)
+                floor_us = smem_us + 2 * t_bar_ns * 1e-3
+                roof["latency_floor"] = {"smem_us": smem_us, "t_bar_us": t_bar_ns * 1e-3, "floor_us_per_step": floor_us,
+                                         "frac_of_floor": floor_us / us_per_sample_step,
+                                         "note": "weight bytes / smem bandwidth + 2 x measured chip-wide exchange of one stream's "
+                                                 "state half (the exchange of %d streams moves %d times the words)" % (wl.batch, wl.batch)}
         elif wl.sparsity is not None:
             ach = wbytes * n_steps / (ms_per_step * 1e-3) / 1e9
             roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],

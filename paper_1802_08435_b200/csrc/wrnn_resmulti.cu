@@ -430,13 +430,19 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                 float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
                 const uint4 *bimg = (spread ? splOwn : spl + cl * IMG_U4) + g4 * 4 + t4;
                 const uint4 *A = M + (2 + tsel) * TILE_U4 + lane;
-#pragma unroll 2
-                for (int kp = p0; kp < p1; ++kp) {
-                    const uint4 bv = bimg[kp * 32];
-                    const uint4 a0 = A[(2 * kp) * 32], a1 = A[(2 * kp + 1) * 32];
-                    mma16816(acc[0], a0, bv.x, bv.y);
-                    mma16816(acc[1], a1, bv.z, bv.w);
+                // three or four k-tile pairs: all fragment loads first, then the MMAs back to back
+                uint4 bv[4], a0[4], a1[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int kp = p0 + i < p1 ? p0 + i : p0;           // (a fourth pair that is not there repeats the first; its products are dropped)
+                    bv[i] = bimg[kp * 32]; a0[i] = A[(2 * kp) * 32]; a1[i] = A[(2 * kp + 1) * 32];
                 }
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (p0 + i < p1) {
+                        mma16816(acc[0], a0[i], bv[i].x, bv[i].y);
+                        mma16816(acc[1], a1[i], bv[i].z, bv[i].w);
+                    }
                 float *d = part0 + t4 * P0S + (tsel * 4 + sp) * 16;
                 d[g4] = (acc[0][0] + acc[1][0]) + (acc[0][1] + acc[1][1]);
                 d[g4 + 8] = (acc[0][2] + acc[1][2]) + (acc[0][3] + acc[1][3]);

@@ -131,6 +131,8 @@ static bool use_resf32(const wrnn_model *m, int batch)
 static bool use_pair(const wrnn_model *m, int batch)
 {
     if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_RESIDENT) return false;
+    const char *off = getenv("WRNN_NO_PAIR");
+    if (off && off[0] == '1') return false;
     return m->variant == 0 && resident_pair_supported(m, batch) == WRNN_OK;
 }
 
@@ -222,7 +224,8 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
         return generic_run(m, a, s);
     }
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
-    if (use_multi(m, a.batch)) return resmulti_run(m, a, s);
+    // two rows: the two-stream kernel (7.5 us per step against 8.2 on the multi-stream kernel); 3 to 16: the multi-stream kernel
+    if (use_multi(m, a.batch) && !(a.batch == 2 && use_pair(m, 2))) return resmulti_run(m, a, s);
     if (use_pair(m, a.batch)) {
         for (int pair = 0; pair < a.batch / 2; ++pair) {
             rc = resident_pair_run(m, a, pair, s);
@@ -730,7 +733,7 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
     }
-    if (use_multi(m, batch)) {
+    if (use_multi(m, batch) && !(batch == 2 && use_pair(m, 2))) {
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resmulti_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
     }

@@ -433,6 +433,8 @@ def test_multi_stream_resident_kernels(env, batch, form):
     n = 400
     if form == "pair":
         os.environ["WRNN_NO_MULTI"] = "1"
+    else:
+        os.environ["WRNN_NO_PAIR"] = "1"         # (two rows go to the two-stream kernel by default)
     m = B.wrnn_create(w, wl.dtype, max_batch=batch)
     try:
         info = B.wrnn_launch_info(m, batch)
@@ -456,6 +458,7 @@ def test_multi_stream_resident_kernels(env, batch, form):
     finally:
         B.wrnn_destroy(m)
         os.environ.pop("WRNN_NO_MULTI", None)
+        os.environ.pop("WRNN_NO_PAIR", None)
 
 
 def test_config2_sparse_bf16(env):

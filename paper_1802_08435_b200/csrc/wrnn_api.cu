@@ -421,6 +421,7 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
         }
         if (m->dtype == WRNN_BF16 && m->variant == 0 && max_batch >= 2) resmulti_prepare(m);   // optional: other kernels serve the batch without it
     }
+    m->err.clear();             // reasons why optional kernels were not prepared are not errors of this call
     *out = m;
     return WRNN_OK;
 }

@@ -461,6 +461,27 @@ def test_multi_stream_resident_kernels(env, batch, form):
         os.environ.pop("WRNN_NO_PAIR", None)
 
 
+def test_multi_stream_every_row_count(env):
+    """Every row count the multi-stream resident kernel takes (2 to 16: one to four column groups, partial groups, one
+    stream per cluster up to seven): 160 teacher-forced steps of every row against the oracle."""
+    torch, B = env
+    wl = synth.WORKLOADS[7]
+    os.environ["WRNN_NO_PAIR"] = "1"             # (two rows go to the two-stream kernel by default)
+    try:
+        for batch in range(2, 17):
+            w, masks, cond = synth.build_workload(wl, batch=batch)
+            om = orc.OracleModel(w, wl.dtype)
+            m = B.wrnn_create(w, wl.dtype, max_batch=batch)
+            try:
+                assert B.wrnn_launch_info(m, batch)["smem_bytes"] > 200000
+                r = pu.teacher_forced_parity(torch, B, m, om, cond, 160, batch, SEED, row_stride=1, row_offset_mul=5, stream0=2, threads=pu.NCPU)
+                _tol_check(r, wl.dtype)
+            finally:
+                B.wrnn_destroy(m)
+    finally:
+        os.environ.pop("WRNN_NO_PAIR", None)
+
+
 def test_config2_sparse_bf16(env):
     """Block-sparse H=2048 bf16 (96 % of the 4x4 blocks of R_u, R_r, R_e, O1, O3 pruned), batch 1: the first
     1,500 steps against the dense-with-zeros oracle; the full 24,000 steps for determinism and resume."""

@@ -136,10 +136,9 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     float *part_R = sIg + 2 * 3 * MHR * 3 + 8;                                       // [streams][2 tiles x slots][16] (+8 per stream)
     float *part0 = part_R + PR_FLOATS;                                         // [4 streams][8 slots][16] (+8 per stream)
     uint4 *spl = reinterpret_cast<uint4 *>(part0 + 4 * P0S);                   // [4 column groups] images of the state half
-    uint4 *splQ = spl + 4 * IMG_U4;                                            // image of the hidden layers of the own streams
+    uint4 *splQ = spl + 4 * IMG_U4;                                            // the hidden layers of the own streams, split by their senders (layout below)
     uint4 *splOwn = splQ + IMG_U4;                                             // up to seven streams: the own stream's state half as a column group of its own
-    float *qbuf = reinterpret_cast<float *>(splOwn + IMG_U4);                    // [2 parities][4 streams][K]
-    uint4 *lbuf = reinterpret_cast<uint4 *>(qbuf + 8 * K);                     // [2 parities][4 streams][128] {v, tag, v, tag}
+    uint4 *lbuf = splOwn + IMG_U4;                                             // [2 parities][4 streams][128] {v, tag, v, tag}
     __shared__ __align__(8) unsigned long long xbar[2];
     __shared__ __align__(8) unsigned long long s_sym[8];   // [2 parities][4 own streams] (symbol, tag) from the drawing CTA
     __shared__ long long s_pub;                 // the last half step whose state values this CTA's gate threads have published
@@ -148,7 +147,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         const uint4 *src = reinterpret_cast<const uint4 *>(p.blob + (size_t)cta * p.blob_bytes);
         uint4 *dst = reinterpret_cast<uint4 *>(smem);
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
-        for (int i = tid; i < 8 * K + 4096; i += blockDim.x) qbuf[i] = 0.f;              // qbuf and lbuf are adjacent
+        for (int i = tid; i < 1024; i += blockDim.x) lbuf[i] = make_uint4(0, 0, 0, 0);
         for (int i = tid; i < 6 * IMG_U4; i += blockDim.x) spl[i] = make_uint4(0, 0, 0, 0);  // spl, splQ and splOwn are adjacent
         for (int i = tid; i < MAXS * MNR + 2 * 3 * MHR * 3 + 8 + PR_FLOATS + 4 * P0S; i += blockDim.x) a_part[i] = 0.f;
         if (tid == 0) {
@@ -322,7 +321,15 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
 #pragma unroll
     for (int par2 = 0; par2 < 2; ++par2) {
         const unsigned peer = (unsigned)warp;
-        q_snd[par2] = map_to_rank(smem_addr(qbuf + (size_t)(par2 * 4 + (q_st < 4 ? q_st : 0)) * K + rank * MHR + 4 * q_quad), peer);
+        {
+            // The hidden layer travels already split: a lane's four rows j0 .. j0 + 3 (j0 a multiple of 4) of one stream are
+            // four 32-bit words -- (high parts of j0, j0+1), (high of j0+2, j0+3), (low of j0, j0+1), (low of j0+2, j0+3) --
+            // stored as one 16-byte piece of the receivers' image [k-tile pair][t / 2][k-tile & 1][upper half of the k-tile]
+            // [stream][part][t & 1], from which a B fragment is four words 16 words apart.
+            const int j0 = rank * MHR + 4 * q_quad, kt = j0 >> 4, c = j0 & 15;
+            const int w = (((((kt >> 1) * 2 + ((c & 7) >> 2)) * 2 + (kt & 1)) * 2 + (c >> 3)) * 4 + (q_st < 4 ? q_st : 0)) * 4;
+            q_snd[par2] = map_to_rank(smem_addr(reinterpret_cast<unsigned *>(splQ) + w), peer);
+        }
         l_snd[par2] = map_to_rank(smem_addr(lbuf + (size_t)(par2 * 4 + l_st) * 128 + (rank * MLR) / 2 + l_ll), 0u);
         q_bar[par2] = map_to_rank(smem_addr(&xbar[par2]), peer);
     }
@@ -458,31 +465,32 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                     const float4 a = *reinterpret_cast<const float4 *>(pt + sp * 16);
                     v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
                 }
-                st_async_v4(q_snd[par], fmaxf(v.x, 0.f), fmaxf(v.y, 0.f), fmaxf(v.z, 0.f), fmaxf(v.w, 0.f), q_bar[par]);
+                v.x = fmaxf(v.x, 0.f); v.y = fmaxf(v.y, 0.f); v.z = fmaxf(v.z, 0.f); v.w = fmaxf(v.w, 0.f);
+                const __nv_bfloat16 hx = __float2bfloat16_rn(v.x), hy = __float2bfloat16_rn(v.y), hz = __float2bfloat16_rn(v.z), hw = __float2bfloat16_rn(v.w);
+                const __nv_bfloat16 lx = __float2bfloat16_rn(v.x - __bfloat162float(hx)), ly = __float2bfloat16_rn(v.y - __bfloat162float(hy));
+                const __nv_bfloat16 lz = __float2bfloat16_rn(v.z - __bfloat162float(hz)), lw = __float2bfloat16_rn(v.w - __bfloat162float(hw));
+                auto pk = [](__nv_bfloat16 a, __nv_bfloat16 b) { return __uint_as_float((unsigned)__bfloat16_as_ushort(a) | ((unsigned)__bfloat16_as_ushort(b) << 16)); };
+                st_async_v4(q_snd[par], pk(hx, hy), pk(hz, hw), pk(lx, ly), pk(lz, lw), q_bar[par]);
             }
             STAMP(1 + 6 * half);
 
             // ---- 3. the cluster's hidden layers -> logits rows of this CTA
             if (!wait_arrival(par, use, (int)s, 2 + 4 * half)) my_bad = true;
-            for (int idx = tid; idx < own_n * K / 2; idx += blockDim.x) {
-                const int st = (2 * idx) / K, j = 2 * idx - st * K;
-                const float2 v = reinterpret_cast<const float2 *>(qbuf + (size_t)par * 4 * K)[idx];
-                mimg_store_pair(splQ, st, j, v.x, v.y);
-            }
         }
         if (__syncthreads_or(my_bad)) break;
         STAMP(2 + 6 * half);
         if (own_n > 0) {
             if (warp < 7) {
                 float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-                const uint4 *bimg = splQ + g4 * 4 + t4;
+                const unsigned *bimg = reinterpret_cast<const unsigned *>(splQ) + (t4 >> 1) * 64 + (g4 >> 1) * 4 + (g4 & 1) * 2 + (t4 & 1);
                 const uint4 *A = L + lane;
 #pragma unroll
                 for (int kp = 2 * warp; kp < 2 * warp + 2; ++kp) {
-                    const uint4 bv = bimg[kp * 32];
+                    const unsigned *b = bimg + kp * 128;
+                    const unsigned b00 = b[0], b01 = b[16], b10 = b[32], b11 = b[48];
                     const uint4 a0 = A[(2 * kp) * 32], a1 = A[(2 * kp + 1) * 32];
-                    mma16816(acc[0], a0, bv.x, bv.y);
-                    mma16816(acc[1], a1, bv.z, bv.w);
+                    mma16816(acc[0], a0, b00, b01);
+                    mma16816(acc[1], a1, b10, b11);
                 }
                 float *d = part0 + t4 * P0S + warp * 16;
                 d[g4] = (acc[0][0] + acc[1][0]) + (acc[0][1] + acc[1][1]);
@@ -591,7 +599,6 @@ static int resmulti_smem_bytes(const ResMultiPack &k)
     b += (size_t)MAXS * MNR * 4 + (size_t)(2 * 3 * MHR * 3 + 8) * 4;   // a_part, the gate threads' input weights
     b += (size_t)PR_FLOATS * 4 + (size_t)4 * P0S * 4;
     b += (size_t)6 * IMG_U4 * 16;                   // four column-group images, the hidden-layer image, the own streams' image
-    b += (size_t)8 * MK * 4;                        // qbuf
     b += (size_t)1024 * 16;                         // lbuf
     return (int)b;
 }

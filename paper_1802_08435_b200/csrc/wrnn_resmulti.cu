@@ -295,8 +295,10 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int jj = (half_g ? K : 0) + gj;
+        // published as the operand the 112 readers need: bf16 high and low parts, split once here
+        const __nv_bfloat16 hh = __float2bfloat16_rn(hn), hl = __float2bfloat16_rn(hn - __bfloat162float(hh));
         st_relaxed_u64(p.slots + ((size_t)((half_g ? 2 : 0) + (s & 1)) * NS + gst) * K + gj,
-                       ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+                       ((unsigned long long)(unsigned)(s + 1) << 32) | (unsigned)__bfloat16_as_ushort(hh) | ((unsigned)__bfloat16_as_ushort(hl) << 16));
         if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * NS + gst) * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
         if (p.dbg_h) p.dbg_h[((size_t)s * NS + gst) * H + jj] = hn;
     };
@@ -383,9 +385,15 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
             auto put = [&](int q) {
                 const int idx = at[q];
                 const int st = (2 * idx) / K, j = 2 * idx - st * K;
-                const float x0 = __uint_as_float((unsigned)v0[q]), x1 = __uint_as_float((unsigned)v1[q]);
-                mimg_store_pair(spl, st, j, x0, x1);
-                if (spread && st == cl) mimg_store_pair(splOwn, 0, j, x0, x1);
+                const unsigned x0 = (unsigned)v0[q], x1 = (unsigned)v1[q];       // (high | low << 16) of elements j, j + 1
+                const unsigned w_hi = (x0 & 0xffffu) | (x1 << 16), w_lo = (x0 >> 16) | (x1 & 0xffff0000u);
+                const int col = 2 * (st & 3);
+                unsigned *s32 = reinterpret_cast<unsigned *>(spl + (st >> 2) * IMG_U4);
+                s32[mimg_pos(j, col) >> 1] = w_hi; s32[mimg_pos(j, col + 1) >> 1] = w_lo;
+                if (spread && st == cl) {
+                    unsigned *o32 = reinterpret_cast<unsigned *>(splOwn);
+                    o32[mimg_pos(j, 0) >> 1] = w_hi; o32[mimg_pos(j, 1) >> 1] = w_lo;
+                }
             };
             unsigned pending = 0;
 #pragma unroll

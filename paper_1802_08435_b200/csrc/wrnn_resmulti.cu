@@ -135,7 +135,8 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     float *sIg = a_part + MAXS * MNR;                                          // [2 halves][3 gates][28 units][3] input weights of the gate threads' units
     float *part_R = sIg + 2 * 3 * MHR * 3 + 8;                                       // [streams][2 tiles x slots][16] (+8 per stream)
     float *part0 = part_R + PR_FLOATS;                                         // [4 streams][8 slots][16] (+8 per stream)
-    uint4 *spl = reinterpret_cast<uint4 *>(part0 + 4 * P0S);                   // [4 column groups] images of the state half
+    float *part1 = part0 + 4 * P0S;                                            // the same for the logits (its writers do not wait for the readers of part0)
+    uint4 *spl = reinterpret_cast<uint4 *>(part1 + 4 * P0S);                   // [4 column groups] images of the state half
     uint4 *splQ = spl + 4 * IMG_U4;                                            // the hidden layers of the own streams, split by their senders (layout below)
     uint4 *splOwn = splQ + IMG_U4;                                             // up to seven streams: the own stream's state half as a column group of its own
     uint4 *lbuf = splOwn + IMG_U4;                                             // [2 parities][4 streams][128] {v, tag, v, tag}
@@ -149,7 +150,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
         for (int i = tid; i < 1024; i += blockDim.x) lbuf[i] = make_uint4(0, 0, 0, 0);
         for (int i = tid; i < 6 * IMG_U4; i += blockDim.x) spl[i] = make_uint4(0, 0, 0, 0);  // spl, splQ and splOwn are adjacent
-        for (int i = tid; i < MAXS * MNR + 2 * 3 * MHR * 3 + 8 + PR_FLOATS + 4 * P0S; i += blockDim.x) a_part[i] = 0.f;
+        for (int i = tid; i < MAXS * MNR + 2 * 3 * MHR * 3 + 8 + PR_FLOATS + 8 * P0S; i += blockDim.x) a_part[i] = 0.f;
         if (tid == 0) {
             for (int i = 0; i < 2; ++i) mbar_init_cluster(smem_addr(&xbar[i]), 1);
             mbar_fence_init();
@@ -482,13 +483,13 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
             }
             STAMP(1 + 6 * half);
 
-            // ---- 3. the cluster's hidden layers -> logits rows of this CTA
-            if (!wait_arrival(par, use, (int)s, 2 + 4 * half)) my_bad = true;
         }
-        if (__syncthreads_or(my_bad)) break;
-        STAMP(2 + 6 * half);
-        if (own_n > 0) {
-            if (warp < 7) {
+        // ---- 3. the cluster's hidden layers -> logits rows of this CTA: warps 0..6 only; the others start the
+        // recurrent products (4b) while the hidden layers are in flight, so that R h reaches the gate threads early
+        if (own_n > 0 && warp < 7) {
+            if (!wait_arrival(par, use, (int)s, 2 + 4 * half)) my_bad = true;
+            STAMP(2 + 6 * half);
+            {
                 float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
                 const unsigned *bimg = reinterpret_cast<const unsigned *>(splQ) + (t4 >> 1) * 64 + (g4 >> 1) * 4 + (g4 & 1) * 2 + (t4 & 1);
                 const uint4 *A = L + lane;
@@ -500,15 +501,15 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                     mma16816(acc[0], a0, b00, b01);
                     mma16816(acc[1], a1, b10, b11);
                 }
-                float *d = part0 + t4 * P0S + warp * 16;
+                float *d = part1 + t4 * P0S + warp * 16;
                 d[g4] = (acc[0][0] + acc[1][0]) + (acc[0][1] + acc[1][1]);
                 d[g4 + 8] = (acc[0][2] + acc[1][2]) + (acc[0][3] + acc[1][3]);
             }
-            __syncthreads();
+            named_sync(3, 224);
             STAMP(14 + half);
             if (warp == 0 && l_st < own_n) {            // the logits go to the drawing CTA only
                 const int r0 = 2 * l_ll;
-                const float *pt = part0 + l_st * P0S + r0;
+                const float *pt = part1 + l_st * P0S + r0;
                 float v0 = bl[r0], v1 = bl[r0 + 1];
 #pragma unroll
                 for (int sp = 0; sp < 7; ++sp) { const float2 a = *reinterpret_cast<const float2 *>(pt + sp * 16); v0 += a.x; v1 += a.y; }
@@ -605,7 +606,7 @@ static int resmulti_smem_bytes(const ResMultiPack &k)
 {
     size_t b = k.blob_bytes;
     b += (size_t)MAXS * MNR * 4 + (size_t)(2 * 3 * MHR * 3 + 8) * 4;   // a_part, the gate threads' input weights
-    b += (size_t)PR_FLOATS * 4 + (size_t)4 * P0S * 4;
+    b += (size_t)PR_FLOATS * 4 + (size_t)8 * P0S * 4;
     b += (size_t)6 * IMG_U4 * 16;                   // four column-group images, the hidden-layer image, the own streams' image
     b += (size_t)1024 * 16;                         // lbuf
     return (int)b;

@@ -46,7 +46,6 @@ constexpr int TILE_U4 = 28 * 32;     // uint4 per 16-row tile of A fragments
 constexpr int IMG_U4 = MKP * 32;     // uint4 per column-group image of a vector
 constexpr int P0S = 136;             // floats per stream of the head partial sums (8 slots x 16 rows + 8 so that the streams hit different banks)
 constexpr int PR_FLOATS = 1664;      // partial sums of the recurrent rows
-constexpr int NRW = 12;              // warps that multiply the recurrent rows
 }  // namespace
 
 struct ResMultiPack {
@@ -180,17 +179,23 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     const int ws = warp;                                  // drawing warps 0..3: own stream ws
     const bool drawer = warp < 4 && ws < own_n && rank == 0;   // the cluster's first CTA draws for its streams
     const int d_st = spread ? cl : 4 * cl + ws;           // the stream a drawing warp serves
-    const int rw = warp - 4, ridx = tid - 128;            // warps 4..15: recurrent rows, then the gates
+    // recurrent products: warps 7..15 (warps 0..6 hold the logits MMAs of the head chain); with four column groups also
+    // warps 4..6, after their logits MMAs (measured: 10.47 against 10.52 us per 16-row lock-step; 7.81 against 8.09 at 4 rows)
+    const int RW0 = NG >= 4 ? 4 : 7, NRW = 16 - RW0;
+    const int rw = warp - RW0, ridx = tid - 128;          // warps 4..15: sums of the products, then the gates
     // gate threads: the state units 28 rank .. + 27 of both halves, for every own stream of the cluster
     const bool gater = warp >= 4 && ridx < own_n * MHR;
     const int gl = ridx / MHR, gq = ridx % MHR;           // (own stream, unit of this CTA's share) of a gate thread
     const int gst = (spread ? cl : 4 * cl) + gl, gj = MHR * rank + gq;
     const int r_cg = rw >= 0 ? rw % NG : 0, r_j = rw >= 0 ? rw / NG : 0;
     const int nsl = (NRW + NG - 1) / NG, PS = 2 * nsl * 16 + 8;
+    const int r_nw = (NRW - r_cg + NG - 1) / NG;                               // warps that share column group r_cg
+    const int s_st = ridx >= 0 ? ridx / MNR : 0, s_row = ridx >= 0 ? ridx - s_st * MNR : 0;      // (stream, row) a thread sums
+    const int s_nw = (NRW - (s_st >> 2) + NG - 1) / NG;
 
     // recurrent rows (tiles 0, 1 of Mx) times all streams: warp rw takes column group r_cg, k-tile pairs r_j, r_j + nw, ..
     auto r_products = [&](const uint4 *Mx) {
-        const int nw = (NRW - r_cg + NG - 1) / NG;
+        const int nw = r_nw;
         float acc[2][2][4];
 #pragma unroll
         for (int n = 0; n < 2; ++n)
@@ -224,8 +229,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     // that computes the gates of its stream
     auto r_sums = [&](bool completes, long long s_use) {
         if (ridx < NS * MNR) {
-            const int st = ridx / MNR, row = ridx - st * MNR;
-            const int cgp = st >> 2, nw = (NRW - cgp + NG - 1) / NG;
+            const int st = s_st, row = s_row, nw = s_nw;
             const float *s = part_R + st * PS + ((row >> 4) * nsl) * 16 + (row & 15);
             float v = 0.f;
             for (int j = 0; j < nw; ++j) v += s[j * 16];
@@ -247,11 +251,11 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     // ---- prologue: R h of the initial state
     fill_image(0);
     __syncthreads();
-    if (warp >= 4) { r_products(wMA); named_sync(1, 384); r_sums(false, 0); }
+    if (warp >= 4) { if (warp >= RW0) r_products(wMA); named_sync(1, 384); r_sums(false, 0); }
     __syncthreads();
     fill_image(1);
     __syncthreads();
-    if (warp >= 4) { r_products(wMB); named_sync(1, 384); r_sums(true, 0); }
+    if (warp >= 4) { if (warp >= RW0) r_products(wMB); named_sync(1, 384); r_sums(true, 0); }
     __syncthreads();
 
     // state of a gate thread: its unit of both halves of its stream, and the stream's last symbols
@@ -565,7 +569,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
             STAMP(5 + 6 * half);
         } else {
             // ---- 4b. recurrent rows times all streams, then the gates of the other half of the state
-            r_products(M);
+            if (warp >= RW0) r_products(M);
             named_arrive(2, 512);
             named_sync(1, 384);
             r_sums(!half, s);

@@ -324,7 +324,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     // send addresses: one peer per warp
     const int q_st = lane / 7, q_quad = lane % 7;             // hidden layer: lanes [0, 28): stream, four rows
     const int l_st = lane >> 3, l_ll = lane & 7;              // logits: stream, two rows
-    unsigned q_snd[2], l_snd[2], q_bar[2], q_snd2 = 0, q_bar2[2] = {0, 0};     // (second peer of a sending warp: warp + 8)
+    unsigned q_snd[2], l_snd[2], q_bar[2], q_off = 0;        // (a sending warp serves CTAs warp, warp + 4, warp + 8, warp + 12 of the cluster)
 #pragma unroll
     for (int par2 = 0; par2 < 2; ++par2) {
         const unsigned peer = (unsigned)warp;
@@ -339,8 +339,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         }
         l_snd[par2] = map_to_rank(smem_addr(lbuf + (size_t)(par2 * 4 + l_st) * 128 + (rank * MLR) / 2 + l_ll), 0u);
         q_bar[par2] = map_to_rank(smem_addr(&xbar[par2]), peer);
-        q_snd2 = map_to_rank(smem_addr(reinterpret_cast<unsigned *>(splQ)) + (q_snd[par2] - map_to_rank(smem_addr(reinterpret_cast<unsigned *>(splQ)), peer)), (peer + 8u) & 15u);
-        q_bar2[par2] = map_to_rank(smem_addr(&xbar[par2]), (peer + 8u) & 15u);
+        q_off = q_snd[par2] - map_to_rank(smem_addr(reinterpret_cast<unsigned *>(splQ)), peer);
     }
     auto wait_arrival = [&](int which, unsigned use, int step, int phase) {
         const unsigned bar = smem_addr(&xbar[which]);
@@ -471,8 +470,8 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
             }
             __syncthreads();
             STAMP(12 + half);
-            // warps 0..7 send, each to two CTAs of the cluster; warps 8..15 go straight to the recurrent products
-            if (warp < 8 && lane < 28 && q_st < own_n) {
+            // warps 0..3 send, each to four CTAs of the cluster; the others go straight on
+            if (warp < 4 && lane < 28 && q_st < own_n) {
                 const int r0 = 4 * q_quad;
                 const float *pt = part0 + q_st * P0S + ((r0 >> 4) * 4) * 16 + (r0 & 15);
                 float4 v = *reinterpret_cast<const float4 *>(bh + r0);
@@ -486,8 +485,12 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                 const __nv_bfloat16 lx = __float2bfloat16_rn(v.x - __bfloat162float(hx)), ly = __float2bfloat16_rn(v.y - __bfloat162float(hy));
                 const __nv_bfloat16 lz = __float2bfloat16_rn(v.z - __bfloat162float(hz)), lw = __float2bfloat16_rn(v.w - __bfloat162float(hw));
                 auto pk = [](__nv_bfloat16 a, __nv_bfloat16 b) { return __uint_as_float((unsigned)__bfloat16_as_ushort(a) | ((unsigned)__bfloat16_as_ushort(b) << 16)); };
-                st_async_v4(q_snd[par], pk(hx, hy), pk(hz, hw), pk(lx, ly), pk(lz, lw), q_bar[par]);
-                st_async_v4(q_snd2, pk(hx, hy), pk(hz, hw), pk(lx, ly), pk(lz, lw), q_bar2[par]);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const unsigned peer = (unsigned)(warp + 4 * k);
+                    st_async_v4(map_to_rank(smem_addr(reinterpret_cast<unsigned *>(splQ)), peer) + q_off, pk(hx, hy), pk(hz, hw), pk(lx, ly), pk(lz, lw),
+                                map_to_rank(smem_addr(&xbar[par]), peer));
+                }
             }
             STAMP(1 + 6 * half);
 

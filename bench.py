@@ -160,7 +160,237 @@ def cpu_baseline(wl, budget_s=12.0):
     run(n_steps)
     dt = time.perf_counter() - t0
     return {"value": n_steps * wl.batch * samples_per_step(wl) / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
-            "sample": "first %d of %d steps x %d rows of %s, once" % (n_steps, wl.n_steps, wl.batch, wl.name)}
+            "sample": "first %d of %d steps x %d rows of %s, once" % (n_steps, wl.n_steps, wl.batch, wl.name),
+            "extrapolated": n_steps < wl.n_steps}
+
+
+KERNEL_NAMES = {1: "generic", 2: "resident", 3: "batched", 4: "sparse-cluster", 5: "batched-cluster"}
+FIVE_CONFIGS = [0, 1, 2, 3, 4]            # positions of the five named configurations in synth.WORKLOADS
+
+
+class Ctx:
+    """What every measurement of one process shares: torch, the binding, the replica group, the device and the peaks."""
+
+    def __init__(self, torch, B, replicas, pg, rank, world, local):
+        self.torch, self.B, self.replicas, self.pg = torch, B, replicas, pg
+        self.rank, self.world, self.local = rank, world, local
+        self.dev = torch.device("cuda", local)
+        self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=self.dev)      # > 126 MB L2
+        self.peaks = measured_peaks()
+        self._smem_gbs = None
+
+    def smem_stream_gbs(self):
+        """Measured aggregate shared-memory stream rate (16-byte loads of a resident 144 KB buffer on every SM)."""
+        if self._smem_gbs is None:
+            n_sms = self.torch.cuda.get_device_properties(self.dev).multi_processor_count
+            self._smem_gbs = self.B.wrnn_measure_smem_stream(n_sms, 512, 144 * 1024, 2000)
+        return self._smem_gbs
+
+
+def n_weights(wl, fused=False):
+    H, Hh = wl.H, wl.H // 2
+    n_logits, n_in = (64, 12) if fused else (256, 3)
+    return 3 * H * H + 2 * Hh * Hh + 2 * n_logits * Hh + 3 * n_in * H
+
+
+def latency_floor(ctx, info, Hh, alg_bytes, us_per_step, note):
+    """Weight bytes over the shared-memory bandwidth plus the two chip-wide exchanges a step cannot avoid (Section 2.1:
+    with the model resident the remaining cost is the synchronisation between multiprocessors), the exchange measured
+    live in an empty persistent kernel of the same CTA shape."""
+    K = Hh if Hh % info["n_ctas"] == 0 else info["n_ctas"] * ((Hh + info["n_ctas"] - 1) // info["n_ctas"])
+    try:
+        t_bar_ns = ctx.B.wrnn_measure_exchange_floor(info["n_ctas"], info["n_threads"], K, 20000)
+    except ctx.B.WrnnError as e:
+        return {"unavailable": str(e)}
+    smem_us = alg_bytes / (ctx.smem_stream_gbs() * 1e3)
+    floor_us = smem_us + 2 * t_bar_ns * 1e-3
+    return {"smem_us": smem_us, "t_bar_us": t_bar_ns * 1e-3, "floor_us_per_step": floor_us, "frac_of_floor": floor_us / us_per_step,
+            "note": note}
+
+
+def roofline(ctx, wl, info, model, n_steps, ms_per_step, cond_bytes, out_bytes):
+    """The bound of the dominant (only) kernel of a call and how close the call came to it."""
+    B, peaks = ctx.B, ctx.peaks
+    us_per_step = ms_per_step * 1e3 / n_steps
+    wbytes = info["weight_bytes_per_step"]
+    fused = wl.variant == 1
+    H, Hh = wl.H, wl.H // 2
+    resident = info["kernel"] in (2, 4)
+    # DRAM bytes of one launch, from sizes the library reports: the packed weights are read once into shared memory
+    # (resident kernels) and stay there; conditioning frames in, projected gate offsets out and in again, samples out
+    g_bytes = wl.batch * (wl.n_frames if wl.n_frames else 1) * 3 * H * 4
+    traffic = (wbytes + cond_bytes + 2 * g_bytes + out_bytes) if resident else None
+    traffic_note = ("computed: resident weight bytes loaded once per launch (%d) + conditioning (%d) + projected gate offsets "
+                    "written and read (%d) + samples (%d); does not grow with the number of steps; the ncu captures in "
+                    "profiles/ measured the same quantity" % (wbytes, cond_bytes, 2 * g_bytes, out_bytes)) if resident else \
+                   "weights are re-read from L2 every step; DRAM traffic not modelled"
+    if wl.batch >= 2:
+        flops = 2.0 * wl.batch * (3 * H * H + 2 * Hh * Hh + 2 * 256 * Hh)
+        ach = flops * n_steps / (ms_per_step * 1e-3) / 1e12
+        roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops_sustained"], "traffic": traffic, "traffic_note": traffic_note,
+                "peak_source": peaks["source"] + " sustained", "algorithmic_flops_per_step": flops}
+        if info["kernel"] == 2:      # the multi-stream resident kernel stamps the phases of its first CTA's first warp
+            pc = B.wrnn_phase_cycles(model)
+            names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_wait_recurrent",
+                     "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_wait_recurrent",
+                     "F.hid_products", "C.hid_products", "F.log_products", "C.log_products"]
+            roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
+            roof["latency_floor"] = latency_floor(
+                ctx, info, Hh, n_weights(wl) * 2, us_per_step,
+                "weight bytes / measured smem stream rate + 2 x measured chip-wide exchange of one stream's state half "
+                "(the exchange of %d streams moves %d times the words)" % (wl.batch, wl.batch))
+        return roof
+    if wl.sparsity is not None:
+        ach = wbytes * n_steps / (ms_per_step * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                "traffic": traffic, "traffic_note": traffic_note, "peak_source": peaks["source"], "bytes_per_step": wbytes,
+                "note": "nonzero-block bytes per step over the HBM copy bandwidth (the bound the workload names); the pruned "
+                        "model is resident in shared memory, see smem and latency_floor"}
+        if info["kernel"] == 4:
+            roof["smem"] = {"achieved": ach, "peak": ctx.smem_stream_gbs(), "unit": "GB/s", "frac": ach / ctx.smem_stream_gbs(),
+                            "peak_source": "measured: 16-byte shared-memory loads on all SMs"}
+            roof["latency_floor"] = latency_floor(ctx, info, Hh, wbytes, us_per_step,
+                                                  "nonzero-block bytes / measured smem stream rate + 2 x measured chip-wide exchange")
+        return roof
+    # single stream, weights resident in shared memory: algorithmic bytes = every stored weight read once per step
+    alg_bytes = n_weights(wl, fused) * (2 if wl.dtype == "bf16" else 4)
+    ach = alg_bytes * n_steps / (ms_per_step * 1e-3) / 1e9
+    smem = ctx.smem_stream_gbs()
+    roof = {"bound": "smem", "achieved": ach, "peak": smem, "unit": "GB/s", "frac": ach / smem, "traffic": traffic,
+            "traffic_note": traffic_note, "peak_source": "measured: 16-byte shared-memory loads of a resident 144 KB buffer on all SMs",
+            "peak_derived": {"value": SMEM_PEAK_GBS, "how": "148 SMs x 128 B/clk x 1.965 GHz"},
+            "algorithmic_bytes_per_step": alg_bytes, "resident_bytes_read_per_step": wbytes,
+            "hbm_equivalent": {"achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                               "peak_source": peaks["source"]}}
+    if info["kernel"] == 2:
+        roof["latency_floor"] = latency_floor(ctx, info, Hh, alg_bytes, us_per_step,
+                                              "weight bytes / measured smem stream rate + 2 x measured chip-wide exchange")
+        pc = B.wrnn_phase_cycles(model)
+        tot = float(sum(pc)) or 1.0
+        names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_gates",
+                 "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_gates",
+                 "F.hid_products", "C.hid_products", "F.log_products", "C.log_products"]
+        roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
+        roof["wait_share"] = sum(pc[i] for i in (0, 2, 4, 6, 8, 10)) / tot
+    return roof
+
+
+def measure(ctx, wl, *, steps, warmup, kernel, n_steps=None, e2e=True, cpu_budget_s=12.0, sample_clocks=False):
+    """One workload: create the model, warm up, time `steps` calls with CUDA events (L2 flushed before each), then the
+    same through the host-buffer entry point, the roofline figures and the oracle's rate.  -> dict."""
+    torch, B, replicas, pg, dev = ctx.torch, ctx.B, ctx.replicas, ctx.pg, ctx.dev
+    n_steps = wl.n_steps if n_steps is None else n_steps
+    w, masks, cond_np = synth.build_workload(wl)
+    model = B.wrnn_create(w, wl.dtype, masks, max_batch=wl.batch, kernel=kernel, block=wl.block, variant=wl.variant)
+    try:
+        info = B.wrnn_launch_info(model, wl.batch)
+        cond = torch.from_numpy(cond_np).to(dev)
+        out = torch.zeros((wl.batch, n_steps), dtype=torch.int16, device=dev)
+        # rows of different ranks are different streams of the same workload (replicas; no collective on the path)
+        kw = dict(hop=synth.HOP, row_stride=wl.row_stride, row_offset_mul=wl.row_offset_mul, stream0=0)
+        seed = replicas.rank_seed(synth.SEED_SAMPLING, ctx.rank)
+        fused = wl.variant == 1
+        if fused:       # two streams per call, then the interleaved samples (the two pre-roll samples of part B dropped)
+            out = torch.zeros((2, n_steps), dtype=torch.int16, device=dev)
+            u_out = torch.zeros((2 * (n_steps - 2),), dtype=torch.int16, device=dev)
+        dep = wl.dependent
+        if dep:
+            Vn, bn = synth.make_subscale_conv(wl.batch, dep[0])
+            V_d, b_d = torch.from_numpy(Vn).to(dev), torch.from_numpy(bn).to(dev)
+            out = torch.zeros((wl.batch * n_steps,), dtype=torch.int16, device=dev)
+
+        def one():
+            if dep:
+                B.wrnn_sample_subscale_dependent(model, cond, V_d, b_d, dep[0], dep[1], dep[2], wl.batch * n_steps, wl.batch, seed, out, hop=synth.HOP)
+            elif fused:
+                B.wrnn_fs2_sample(model, cond, n_steps, seed, out, hop=synth.HOP)
+                B.wrnn_fs2_unfold(out, n_steps, u_out)
+            else:
+                B.wrnn_sample(model, cond, n_steps, wl.batch, seed, out, **kw)
+
+        for _ in range(max(warmup, 3)):
+            one()
+        torch.cuda.synchronize()
+        assert B.wrnn_poll_status(model) == 0, B.wrnn_last_error(model)
+
+        sampler = ClockSampler(ctx.local) if (sample_clocks and ctx.rank == 0) else None
+        if sampler:
+            sampler.start()
+            time.sleep(0.25)
+        replicas.barrier(pg)
+        torch.cuda.synchronize()
+        launches0 = B.wrnn_launch_count()
+        evs = []
+        for _ in range(steps):
+            ctx.flush.fill_(1)                                            # L2 flush between timed iterations
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            one()
+            e1.record()
+            evs.append((e0, e1))
+        torch.cuda.synchronize()
+        launches = B.wrnn_launch_count() - launches0
+        replicas.barrier(pg)
+        total_ms = replicas.max_over_ranks(sum(a.elapsed_time(b) for a, b in evs), pg, dev)
+        clocks = sampler.stop() if sampler else None
+        assert B.wrnn_poll_status(model) == 0, B.wrnn_last_error(model)
+
+        ms_per_step = total_ms / steps
+        samples_per_call = 2 * (n_steps - 2) if fused else n_steps * wl.batch
+        value = replicas.aggregate_throughput(ctx.world, samples_per_call, ms_per_step * 1e-3)
+
+        # end to end through the host-buffer entry point (pinned host memory)
+        e2e_d = None
+        if e2e:
+            cond_pin = torch.from_numpy(cond_np).pin_memory()
+            out_pin = torch.zeros((2 * (n_steps - 2),) if fused else (wl.batch, n_steps), dtype=torch.int16).pin_memory()
+            if dep:
+                V_pin, b_pin = torch.from_numpy(Vn).pin_memory(), torch.from_numpy(bn).pin_memory()
+                out_pin = torch.zeros((wl.batch * n_steps,), dtype=torch.int16).pin_memory()
+
+            def one_host():
+                if dep:      # host buffers in and out around the device entry point
+                    cond.copy_(cond_pin, non_blocking=True); V_d.copy_(V_pin, non_blocking=True); b_d.copy_(b_pin, non_blocking=True)
+                    one()
+                    out_pin.copy_(out, non_blocking=True)
+                    torch.cuda.synchronize()
+                elif fused:
+                    B.wrnn_fs2_sample_host(model, cond_pin.numpy()[0], n_steps, seed, out_pin.numpy(), hop=synth.HOP)
+                else:
+                    B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
+
+            for _ in range(2):
+                one_host()
+            replicas.barrier(pg)
+            t0 = time.perf_counter()
+            for _ in range(steps):
+                one_host()
+            dt = (time.perf_counter() - t0) / steps
+            dt = replicas.max_over_ranks(dt, pg, dev)
+            assert np.array_equal(out_pin.numpy(), (u_out if fused else out).cpu().numpy()), "host-buffer path disagrees with the device path"
+            e2e_d = {"value": replicas.aggregate_throughput(ctx.world, samples_per_call, dt), "unit": UNIT,
+                     "h2d_bytes_per_step": int(cond_np.nbytes) + (int(Vn.nbytes + bn.nbytes) if dep else 0),
+                     "d2h_bytes_per_step": int(out_pin.numel() * 2)}
+
+        res = {"wl": wl, "n_steps": n_steps, "info": info, "ms_per_step": ms_per_step, "value": value, "launches": int(launches),
+               "clocks": clocks, "e2e": e2e_d, "samples_per_call": samples_per_call, "roofline": None, "cpu_baseline": None}
+        if ctx.rank == 0:
+            res["roofline"] = roofline(ctx, wl, info, model, n_steps, ms_per_step, int(cond_np.nbytes), int(out.numel() * 2))
+            if cpu_budget_s and ctx.world == 1:
+                res["cpu_baseline"] = cpu_baseline(wl, cpu_budget_s)
+        return res
+    finally:
+        B.wrnn_destroy(model)
+
+
+def config_entry(res):
+    """One element of the line's `configs` array."""
+    wl, info = res["wl"], res["info"]
+    return {"workload": wl.name, "kernel": KERNEL_NAMES[info["kernel"]], "n_ctas": info["n_ctas"], "batch": wl.batch,
+            "n_steps": res["n_steps"], "us_per_step": res["ms_per_step"] * 1e3 / res["n_steps"], "value": res["value"], "unit": UNIT,
+            "x_realtime_24khz": res["value"] / 24000.0, "roofline": res["roofline"], "e2e": res["e2e"],
+            "cpu_baseline": res["cpu_baseline"]}
 
 
 def main():
@@ -174,206 +404,73 @@ def main():
     ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "resident", "batched", "bcluster"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the other four named configurations after the headline one")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)
         return
 
+    from paper_1802_08435_b200 import replicas
+    if replicas.needs_launch(args.gpus):
+        # asked for several GPUs without a launcher: start one rank per GPU ourselves
+        raise SystemExit(replicas.launch_local(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:]))
+    replicas.check_world(args.gpus)
+
     import torch
     from paper_1802_08435_b200 import binding as B
 
-    from paper_1802_08435_b200 import replicas
     rank, world, local = replicas.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    if torch.cuda.device_count() <= local:
+        raise SystemExit("rank %d has no GPU of its own (%d visible)" % (rank, torch.cuda.device_count()))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     pg = replicas.init("nccl", dev)
+    ctx = Ctx(torch, B, replicas, pg, rank, world, local)
 
-    n_steps = wl.n_steps if args.n_steps is None else args.n_steps
-    w, masks, cond_np = synth.build_workload(wl)
     kern = {"auto": B.WRNN_KERNEL_AUTO, "generic": B.WRNN_KERNEL_GENERIC, "resident": B.WRNN_KERNEL_RESIDENT, "batched": B.WRNN_KERNEL_BATCHED, "bcluster": B.WRNN_KERNEL_BCLUSTER}[args.kernel]
-    model = B.wrnn_create(w, wl.dtype, masks, max_batch=wl.batch, kernel=kern, block=wl.block, variant=wl.variant)
-    info = B.wrnn_launch_info(model, wl.batch)
-    cond = torch.from_numpy(cond_np).to(dev)
-    out = torch.zeros((wl.batch, n_steps), dtype=torch.int16, device=dev)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # > 126 MB L2
-    # rows of different ranks are different streams of the same workload (replicas; no collective on the path)
-    kw = dict(hop=synth.HOP, row_stride=wl.row_stride, row_offset_mul=wl.row_offset_mul, stream0=0)
-    seed = replicas.rank_seed(synth.SEED_SAMPLING, rank)
+    head = measure(ctx, wl, steps=args.steps, warmup=args.warmup, kernel=kern, n_steps=args.n_steps, e2e=not args.no_e2e,
+                   cpu_budget_s=0.0 if args.no_cpu_baseline else 12.0, sample_clocks=True)
 
-    fused = wl.variant == 1
-    if fused:       # two streams per call, then the interleaved samples (the two pre-roll samples of part B dropped)
-        out = torch.zeros((2, n_steps), dtype=torch.int16, device=dev)
-        u_out = torch.zeros((2 * (n_steps - 2),), dtype=torch.int16, device=dev)
-
-    dep = wl.dependent
-    if dep:
-        Vn, bn = synth.make_subscale_conv(wl.batch, dep[0])
-        V_d, b_d = torch.from_numpy(Vn).to(dev), torch.from_numpy(bn).to(dev)
-        out = torch.zeros((wl.batch * n_steps,), dtype=torch.int16, device=dev)
-
-    def one():
-        if dep:
-            B.wrnn_sample_subscale_dependent(model, cond, V_d, b_d, dep[0], dep[1], dep[2], wl.batch * n_steps, wl.batch, seed, out, hop=synth.HOP)
-        elif fused:
-            B.wrnn_fs2_sample(model, cond, n_steps, seed, out, hop=synth.HOP)
-            B.wrnn_fs2_unfold(out, n_steps, u_out)
-        else:
-            B.wrnn_sample(model, cond, n_steps, wl.batch, seed, out, **kw)
-
-    for _ in range(max(args.warmup, 3)):
-        one()
-    torch.cuda.synchronize()
-    assert B.wrnn_poll_status(model) == 0, B.wrnn_last_error(model)
-
-    sampler = ClockSampler(local)
-    if rank == 0:
+    # the other named configurations, each measured the same way (one GPU only: the scaling runs time the headline alone)
+    configs = None
+    if world == 1 and args.workload == 1 and args.n_steps is None and args.kernel == "auto" and not args.no_configs:
+        sampler = ClockSampler(local)
         sampler.start()
-        time.sleep(0.25)
-    replicas.barrier(pg)
-    torch.cuda.synchronize()
-    launches0 = B.wrnn_launch_count()
-    evs = []
-    for _ in range(args.steps):
-        flush.fill_(1)                                                # L2 flush between timed iterations
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        one()
-        e1.record()
-        evs.append((e0, e1))
-    torch.cuda.synchronize()
-    launches = B.wrnn_launch_count() - launches0
-    replicas.barrier(pg)
-    total_ms = replicas.max_over_ranks(sum(a.elapsed_time(b) for a, b in evs), pg, dev)
-    clocks = sampler.stop() if rank == 0 else None
-    assert B.wrnn_poll_status(model) == 0, B.wrnn_last_error(model)
-
-    ms_per_step = total_ms / args.steps
-    samples_per_call = 2 * (n_steps - 2) if fused else n_steps * wl.batch
-    value = replicas.aggregate_throughput(world, samples_per_call, ms_per_step * 1e-3)
-
-    # end to end through the host-buffer entry point (pinned host memory)
-    e2e = None
-    if not args.no_e2e:
-        cond_pin = torch.from_numpy(cond_np).pin_memory()
-        out_pin = torch.zeros((2 * (n_steps - 2),) if fused else (wl.batch, n_steps), dtype=torch.int16).pin_memory()
-
-        if dep:
-            V_pin, b_pin = torch.from_numpy(Vn).pin_memory(), torch.from_numpy(bn).pin_memory()
-            out_pin = torch.zeros((wl.batch * n_steps,), dtype=torch.int16).pin_memory()
-
-        def one_host():
-            if dep:      # host buffers in and out around the device entry point
-                cond.copy_(cond_pin, non_blocking=True); V_d.copy_(V_pin, non_blocking=True); b_d.copy_(b_pin, non_blocking=True)
-                one()
-                out_pin.copy_(out, non_blocking=True)
-                torch.cuda.synchronize()
-            elif fused:
-                B.wrnn_fs2_sample_host(model, cond_pin.numpy()[0], n_steps, seed, out_pin.numpy(), hop=synth.HOP)
-            else:
-                B.wrnn_sample_host(model, cond_pin.numpy(), n_steps, wl.batch, seed, out_pin.numpy(), **{k: v for k, v in kw.items() if k != "stream0"})
-
-        for _ in range(2):
-            one_host()
-        replicas.barrier(pg)
-        t0 = time.perf_counter()
-        for _ in range(args.steps):
-            one_host()
-        dt = (time.perf_counter() - t0) / args.steps
-        dt = replicas.max_over_ranks(dt, pg, dev)
-        assert np.array_equal(out_pin.numpy(), (u_out if fused else out).cpu().numpy()), "host-buffer path disagrees with the device path"
-        e2e = {"value": replicas.aggregate_throughput(world, samples_per_call, dt), "unit": UNIT,
-               "h2d_bytes_per_step": int(cond_np.nbytes) + (int(Vn.nbytes + bn.nbytes) if dep else 0),
-               "d2h_bytes_per_step": int(out_pin.numel() * 2)}
+        configs = []
+        for i in FIVE_CONFIGS:
+            if i == args.workload:
+                configs.append(config_entry(head))
+                continue
+            r = measure(ctx, synth.WORKLOADS[i], steps=5, warmup=3, kernel=B.WRNN_KERNEL_AUTO, e2e=not args.no_e2e,
+                        cpu_budget_s=0.0 if args.no_cpu_baseline else 4.0)
+            configs.append(config_entry(r))
+        configs_clocks = sampler.stop()
 
     if rank == 0:
-        peaks = measured_peaks()
-        us_per_sample_step = ms_per_step * 1e3 / n_steps
-        wbytes = info["weight_bytes_per_step"]
-        if wl.batch >= 2:
-            # dense contraction: algorithmic flops of R, O1..O4 products per lock-step
-            H, Hh = wl.H, wl.H // 2
-            flops = 2.0 * wl.batch * (3 * H * H + 2 * Hh * Hh + 2 * 256 * Hh)
-            ach = flops * n_steps / (ms_per_step * 1e-3) / 1e12
-            roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                    "frac": ach / peaks["bf16_tflops_sustained"], "traffic": None, "peak_source": peaks["source"] + " sustained"}
-            if info["kernel"] == 2:      # the multi-stream resident kernel stamps the phases of its first CTA's first warp
-                pc = B.wrnn_phase_cycles(model)
-                names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_wait_recurrent",
-                         "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_wait_recurrent",
-                         "F.hid_products", "C.hid_products", "F.log_products", "C.log_products"]
-                roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
-                # the lock-step is the same chain of two chip-wide exchanges as a single stream's step: its floor
-                t_bar_ns = B.wrnn_measure_exchange_floor(info["n_ctas"], info["n_threads"], Hh, 20000)
-                smem_us = (3 * H * H + 2 * Hh * Hh + 2 * 256 * Hh) * 2 / (SMEM_PEAK_GBS * 1e3)
-                floor_us = smem_us + 2 * t_bar_ns * 1e-3
-                roof["latency_floor"] = {"smem_us": smem_us, "t_bar_us": t_bar_ns * 1e-3, "floor_us_per_step": floor_us,
-                                         "frac_of_floor": floor_us / us_per_sample_step,
-                                         "note": "weight bytes / smem bandwidth + 2 x measured chip-wide exchange of one stream's "
-                                                 "state half (the exchange of %d streams moves %d times the words)" % (wl.batch, wl.batch)}
-        elif wl.sparsity is not None:
-            ach = wbytes * n_steps / (ms_per_step * 1e-3) / 1e9
-            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                    # DRAM bytes of one launch from the ncu capture in profiles/ (the one-time load of the pruned model into the
-                    # four clusters; nothing per step), known for the benchmark's 4 x 4 workload only
-                    "traffic": 7807744 if (info["kernel"] == 4 and wl.block == (4, 4)) else None,
-                    "peak_source": peaks["source"], "bytes_per_step": wbytes,
-                    "note": "nonzero-block bytes per step over the HBM copy bandwidth"}
-        else:
-            # single stream, weights resident in shared memory: algorithmic bytes = every stored weight read once
-            # per step (3,047,296 weights at H = 896) over the aggregate shared-memory bandwidth, plus the floor
-            # of the two chip-wide exchanges a step cannot avoid (measured live in an empty kernel of the same shape)
-            H, Hh = wl.H, wl.H // 2
-            n_logits, n_in = (64, 12) if fused else (256, 3)
-            n_w = 3 * H * H + 2 * Hh * Hh + 2 * n_logits * Hh + 3 * n_in * H
-            alg_bytes = n_w * (2 if wl.dtype == "bf16" else 4)
-            ach = alg_bytes * n_steps / (ms_per_step * 1e-3) / 1e9
-            roof = {"bound": "smem", "achieved": ach, "peak": SMEM_PEAK_GBS, "unit": "GB/s", "frac": ach / SMEM_PEAK_GBS,
-                    "traffic": (16394496 if wl.dtype == "bf16" else 17888000) if info["kernel"] == 2 and not fused else None,
-                    "traffic_note": "DRAM bytes per launch from the ncu capture in profiles/ (one-time weight load; "
-                                    "does not grow with the number of steps)",
-                    "peak_source": "derived: 148 SMs x 128 B/clk x 1.965 GHz", "algorithmic_bytes_per_step": alg_bytes,
-                    "resident_bytes_read_per_step": wbytes,
-                    # the same bytes per second against the measured HBM copy bandwidth: what a kernel that streamed the
-                    # weights from DRAM once per step would be held to (the weights are in fact resident on-chip)
-                    "hbm_equivalent": {"achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                                       "peak_source": peaks["source"]}}
-            if info["kernel"] == 2:
-                t_bar_ns = B.wrnn_measure_exchange_floor(info["n_ctas"], info["n_threads"], Hh, 20000)
-                smem_us = alg_bytes / (SMEM_PEAK_GBS * 1e3)
-                floor_us = smem_us + 2 * t_bar_ns * 1e-3
-                roof["latency_floor"] = {"smem_us": smem_us, "t_bar_us": t_bar_ns * 1e-3, "floor_us_per_step": floor_us,
-                                         "frac_of_floor": floor_us / us_per_sample_step,
-                                         "note": "weight bytes / smem bandwidth + 2 x measured chip-wide exchange"}
-            if info["kernel"] == 2:      # the resident kernels stamp their phases
-                pc = B.wrnn_phase_cycles(model)
-                tot = float(sum(pc)) or 1.0
-                names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_gates",
-                         "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_gates",
-                         "F.hid_products", "C.hid_products", "F.log_products", "C.log_products"]
-                roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
-                waits = sum(pc[i] for i in (0, 2, 4, 6, 8, 10))
-                roof["wait_share"] = waits / tot
+        info, n_steps, ms_per_step = head["info"], head["n_steps"], head["ms_per_step"]
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "H": wl.H, "batch": wl.batch, "n_steps": n_steps, "weights": wl.dtype,
                        "sparsity": wl.sparsity, "block": ("%dx%d" % tuple(wl.block)) if wl.sparsity is not None else None, "l2": "flushed between timed iterations (256 MiB fill)",
-                       "kernel": {1: "generic", 2: "resident", 3: "batched", 4: "sparse-cluster", 5: "batched-cluster"}[info["kernel"]], "n_ctas": info["n_ctas"],
+                       "kernel": KERNEL_NAMES[info["kernel"]], "n_ctas": info["n_ctas"],
                        "threads_per_cta": info["n_threads"], "smem_bytes_per_cta": info["smem_bytes"],
                        "multi_gpu": "replicas only"},
-            "us_per_sample_step": us_per_sample_step, "x_realtime_24khz": value / world / wl.batch / 24000.0 * wl.batch,
-            "x_realtime_24khz_per_stream": samples_per_call / wl.batch / (ms_per_step * 1e-3) / 24000.0 * (wl.subscale_B or 1),
+            "us_per_sample_step": ms_per_step * 1e3 / n_steps, "x_realtime_24khz": head["value"] / world / wl.batch / 24000.0 * wl.batch,
+            "x_realtime_24khz_per_stream": head["samples_per_call"] / wl.batch / (ms_per_step * 1e-3) / 24000.0 * (wl.subscale_B or 1),
             "paper_context": "4x real time (96,000 samples/s) on an Nvidia P100 (Section 2.1); not the target",
-            "gpu_launches": int(launches), "clocks": clocks, "roofline": roof, "e2e": e2e,
+            "gpu_launches": head["launches"], "clocks": head["clocks"], "roofline": head["roofline"], "e2e": head["e2e"],
         }
-        if not args.no_cpu_baseline and world == 1:
-            line["cpu_baseline"] = cpu_baseline(wl)
+        if head["cpu_baseline"] is not None:
+            line["cpu_baseline"] = head["cpu_baseline"]
+        if configs is not None:
+            line["configs"] = configs
+            line["configs_clocks"] = configs_clocks
         print(json.dumps(line), flush=True)
-    B.wrnn_destroy(model)
     if pg is not None:
         pg.destroy_process_group()
 

@@ -158,14 +158,16 @@ int wrnn_sample(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t b
  * region where device allocation is forbidden or would synchronise the whole device, or one running under a
  * fixed memory budget creates its model ahead of time and then needs a sampling call that never reaches
  * cudaMalloc / cudaFree -- wrnn_sample may grow its conditioning scratch on a larger request.  This entry
- * point takes the same arguments and produces the same samples (it always runs the generic step kernel), but
- * every byte of per-call scratch -- projected conditioning, state and head exchange buffers, the barrier
+ * point takes the same arguments and always runs the any-shape step kernel, so it produces exactly the samples of
+ * wrnn_sample on a model created with WRNN_KERNEL_GENERIC (on other models wrnn_sample runs a specialised kernel
+ * whose summation order may turn a draw that sits on a CDF boundary the other way), but every byte of per-call scratch -- projected conditioning, state and head exchange buffers, the barrier
  * counter -- lives in one fixed 8 MiB array inside the library's device image.  Each GPU that loads the
  * library carries that array until the process exits.
  *   - Sizes whose scratch does not fit (roughly batch * n_frames * 3H * 4 bytes plus batch * 5H * 4) are
  *     refused with WRNN_ERR_UNSUPPORTED and a message that states both numbers; nothing is launched.
- *   - The first call on a device looks up the array's device address (once per device, with that device made
- *     current); make that first call outside any stream capture.
+ *   - The array's device address is looked up once per device, with that device current: by wrnn_create for the
+ *     device the model lives on, otherwise by the first call of this entry point on a device; such a first call
+ *     should come before any stream capture.
  *   - All calls, on all models and streams, share the one array and it keeps what the previous call left
  *     behind; the entry point re-zeroes what must start at zero, but two calls that overlap on the GPU race on
  *     it.  Serialise them (one stream, or events).
@@ -217,9 +219,10 @@ int wrnn_sample_subscale(wrnn_model *m, const float *cond, int32_t n_frames, int
  * with x(u) = u / 32768 and positions beyond the row length contributing nothing; row r is a WaveRNN stream with Philox
  * stream id r, step = position, conditioning vector v_r[i] at step i.  The result does not depend on chunk or lag.
  * frames: DEVICE [B][n_frames][cond_dim]; V: DEVICE [B-1][F+1][cond_dim]; bias: DEVICE [cond_dim]; out: DEVICE int16
- * [n_total] in the original order.  B <= max_batch given at create.  Asynchronous on cuda_stream.  Dense bf16 models run
- * on the cluster-partitioned kernel while four or more rows are active and row by row on the resident kernel while fewer
- * are (the ramps of the schedule); everything else on the any-shape kernel.
+ * [n_total] in the original order.  B <= max_batch given at create.  Asynchronous on cuda_stream.  Dense bf16 H = 896
+ * models of up to 16 rows advance all active rows in one launch of the multi-stream resident kernel (a lone row on the
+ * single-stream resident kernel); other dense bf16 models use the cluster-partitioned kernel for two or more active rows;
+ * everything else runs on the any-shape kernel.
  * wrnn_subscale_conditioning computes v_row[0..L) alone from a given history (DEVICE int16 [B][L]) into
  * v (DEVICE [L][cond_dim]).
  */
@@ -319,6 +322,13 @@ int wrnn_phase_cycles(wrnn_model *m, int64_t *out16);
  * sampling step needs two such exchanges).  K must be a multiple of n_ctas.  HOST out-pointer.  Synchronous;
  * allocates and frees a small device buffer. */
 int wrnn_measure_exchange_floor(int32_t n_ctas, int32_t n_threads, int32_t K, int32_t iters, float *ns_per_exchange);
+
+/* Measured counterpart of the nominal shared-memory bandwidth that bounds "every resident weight read once per step"
+ * (Section 2.1: the model stays on chip across the whole utterance): n_ctas CTAs (one per SM when n_ctas <= the SM
+ * count) of n_threads threads each read a resident buffer of bytes_per_cta bytes `iters` times with 16-byte loads;
+ * *gb_per_s receives the aggregate rate (HOST out-pointer).  bytes_per_cta: a multiple of 16 up to 227 KiB.
+ * Synchronous; allocates and frees a small device buffer. */
+int wrnn_measure_smem_stream(int32_t n_ctas, int32_t n_threads, int32_t bytes_per_cta, int32_t iters, float *gb_per_s);
 
 /* Self-test of the bounded device-side waits (the error path of every persistent kernel here): a two-CTA kernel whose
  * first CTA waits at the grid barrier for an arrival that never comes, gives up after limit_ns (1 us .. 1 s of the

@@ -131,6 +131,22 @@ def split16(x: int):
     return c.value, f.value
 
 
+def split_samples(x: np.ndarray):
+    """int16 samples -> (coarse, fine) uint8 arrays, element by element through the C routines."""
+    x = np.ascontiguousarray(x, dtype=np.int16)
+    cf = [split16((int(v) + 32768) & 0xFFFF) for v in x.reshape(-1)]
+    c = np.array([a for a, _ in cf], np.uint8).reshape(x.shape)
+    f = np.array([b for _, b in cf], np.uint8).reshape(x.shape)
+    return c, f
+
+
+def join_samples(c: np.ndarray, f: np.ndarray) -> np.ndarray:
+    """(coarse, fine) uint8 arrays -> int16 samples, element by element through the C routine."""
+    c = np.asarray(c, np.uint8)
+    f = np.asarray(f, np.uint8)
+    return np.array([to_int16(int(a), int(b)) for a, b in zip(c.reshape(-1), f.reshape(-1))], np.int16).reshape(c.shape)
+
+
 def fold(x: np.ndarray, B: int) -> np.ndarray:
     x = np.ascontiguousarray(x, dtype=np.int16)
     assert x.size % B == 0
@@ -356,11 +372,12 @@ def subscale_conditioning(history: np.ndarray, s: int, V: np.ndarray, b: np.ndar
 
 
 def subscale_dependent_run(om: "OracleModel", frames: np.ndarray, V: np.ndarray, b: np.ndarray, B: int, L: int, hop: int,
-                           seed: int, forced: Optional[np.ndarray] = None):
+                           seed: int, forced: Optional[np.ndarray] = None, teacher: bool = False):
     """Generate the B sub-tensors one after the other (the order of Eq. 4).  frames: float32 [B][n_frames][D] (row s,
     frame (B i + s) div hop at position i).  forced: optional int16 [B][L]; when given, row s is conditioned on the
-    forced samples of rows < s (the drawn ones are still returned).  -> (samples int16 [B][L], cond float32 [B][L][D],
-    margins [B][L][2])."""
+    forced samples of rows < s (the drawn ones are still returned); with teacher = True the forced samples of row s
+    itself are fed back inside the row as well, so that every returned sample is the oracle's draw given the forced
+    history up to that point.  -> (samples int16 [B][L], cond float32 [B][L][D], margins [B][L][2])."""
     D = om.cond_dim
     out = np.zeros((B, L), np.int16)
     cond = np.zeros((B, L, D), np.float32)
@@ -369,7 +386,12 @@ def subscale_dependent_run(om: "OracleModel", frames: np.ndarray, V: np.ndarray,
         hist = out if forced is None else forced
         idx = (B * np.arange(L) + s) // hop
         cond[s] = frames[s][idx] + (subscale_conditioning(hist, s, V, b) if s > 0 else np.maximum(b, 0.0).astype(np.float32)[None, :])
-        r = om.run(cond[s][None], L, 1, seed, hop=1, stream0=s)
-        out[s] = r.out[0]
+        if teacher and forced is not None:
+            cf, ff = split_samples(forced[s])
+            r = om.run(cond[s][None], L, 1, seed, hop=1, stream0=s, c_forced=cf, f_forced=ff)
+            out[s] = join_samples(r.c_out[0], r.f_out[0])
+        else:
+            r = om.run(cond[s][None], L, 1, seed, hop=1, stream0=s)
+            out[s] = r.out[0]
         margins[s] = r.margins[0]
     return out, cond, margins

@@ -25,7 +25,7 @@ _STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "NOMEM", "CUDA", "TIMEOUT"]
 EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
-    "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor", "wrnn_sample_noalloc",
+    "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor", "wrnn_measure_smem_stream", "wrnn_sample_noalloc",
     "wrnn_selftest_bounded_wait", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold", "wrnn_fs2_sample_host",
     "wrnn_sample_subscale_dependent", "wrnn_subscale_conditioning", "wrnn_subscale_schedule",
 ]
@@ -98,6 +98,7 @@ def lib():
         L.wrnn_launch_info.argtypes = [vp, i32] + [vp] * 5
         L.wrnn_phase_cycles.argtypes = [vp, vp]
         L.wrnn_measure_exchange_floor.argtypes = [i32, i32, i32, i32, vp]
+        L.wrnn_measure_smem_stream.argtypes = [i32, i32, i32, i32, vp]
         L.wrnn_selftest_bounded_wait.argtypes = [i64] + [vp] * 5
         L.wrnn_launch_count.argtypes = []
         L.wrnn_launch_count.restype = i64
@@ -319,6 +320,13 @@ def wrnn_measure_exchange_floor(n_ctas: int, n_threads: int, K: int, iters: int 
     """Nanoseconds per chip-wide all-gather of K tagged values through L2 (empty persistent kernel)."""
     out = C.c_float()
     _check(lib().wrnn_measure_exchange_floor(n_ctas, n_threads, K, iters, C.byref(out)))
+    return out.value
+
+
+def wrnn_measure_smem_stream(n_ctas: int, n_threads: int, bytes_per_cta: int, iters: int = 2000) -> float:
+    """Aggregate GB/s of 16-byte shared-memory loads over a resident buffer on n_ctas CTAs (stream micro-benchmark)."""
+    out = C.c_float()
+    _check(lib().wrnn_measure_smem_stream(n_ctas, n_threads, bytes_per_cta, iters, C.byref(out)))
     return out.value
 
 

@@ -127,7 +127,7 @@ static bool use_resf32(const wrnn_model *m, int batch)
 }
 
 // two or four streams of a dense bf16 model: pairs on the two-stream form of the resident kernel, one pair after the other
-// (6.6-7 us per step and pair against 24 us per step of the multi-row kernel)
+// (the default for two rows only; three and more rows go to the multi-stream resident kernel where the model has one)
 static bool use_pair(const wrnn_model *m, int batch)
 {
     if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_RESIDENT) return false;
@@ -422,6 +422,7 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
         if (m->dtype == WRNN_BF16 && m->variant == 0 && max_batch >= 2) resmulti_prepare(m);   // optional: other kernels serve the batch without it
     }
     m->err.clear();             // reasons why optional kernels were not prepared are not errors of this call
+    noalloc_warm(dev);
     *out = m;
     return WRNN_OK;
 }

@@ -122,3 +122,68 @@ extern "C" int wrnn_selftest_bounded_wait(int64_t limit_ns, int32_t *code, int32
     return rc;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Shared-memory stream rate: every SM reads a resident buffer of the size the sampling kernels keep their weights in,
+// over and over, with 16-byte loads from all its threads (what the resident kernels' product phases do with their
+// weight shards, minus the arithmetic).  The aggregate rate is the measured counterpart of the nominal
+// SMs x 128 B/clk x clock that bounds "every resident weight read once per step" (Section 2.1: the weights stay on chip).
+namespace wrnn {
+__global__ void smem_stream_kernel(int bytes, int iters, unsigned *sink)
+{
+    extern __shared__ uint4 sbuf[];
+    const int n16 = bytes / 16;
+    for (int i = threadIdx.x; i < n16; i += blockDim.x) sbuf[i] = make_uint4(i, i + 1, i + 2, i + 3);
+    __syncthreads();
+    unsigned a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+    const unsigned base = (unsigned)__cvta_generic_to_shared(sbuf);
+    for (int it = 0; it < iters; ++it) {
+        // four independent loads per pass keep the load/store unit busy; consecutive lanes read consecutive 16-byte pieces
+        int i = threadIdx.x;
+        for (; i + 3 * (int)blockDim.x < n16; i += 4 * blockDim.x) {
+            uint4 v0, v1, v2, v3;
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v0.x), "=r"(v0.y), "=r"(v0.z), "=r"(v0.w) : "r"(base + 16u * i));
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v1.x), "=r"(v1.y), "=r"(v1.z), "=r"(v1.w) : "r"(base + 16u * (i + blockDim.x)));
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v2.x), "=r"(v2.y), "=r"(v2.z), "=r"(v2.w) : "r"(base + 16u * (i + 2 * blockDim.x)));
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v3.x), "=r"(v3.y), "=r"(v3.z), "=r"(v3.w) : "r"(base + 16u * (i + 3 * blockDim.x)));
+            a0 ^= v0.x ^ v1.y ^ v2.z ^ v3.w; a1 ^= v0.y ^ v1.z ^ v2.w ^ v3.x;
+            a2 ^= v0.z ^ v1.w ^ v2.x ^ v3.y; a3 ^= v0.w ^ v1.x ^ v2.y ^ v3.z;
+        }
+        for (; i < n16; i += blockDim.x) {
+            uint4 v;
+            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(base + 16u * i));
+            a0 ^= v.x; a1 ^= v.y; a2 ^= v.z; a3 ^= v.w;
+        }
+    }
+    if ((a0 ^ a1 ^ a2 ^ a3) == 0x9e3779b9u && iters < 0) sink[blockIdx.x] = a0;       // keeps the loads alive; never taken
+}
+}  // namespace wrnn
+
+extern "C" int wrnn_measure_smem_stream(int32_t n_ctas, int32_t n_threads, int32_t bytes_per_cta, int32_t iters, float *gb_per_s)
+{
+    if (n_ctas < 1 || n_threads < 32 || n_threads > 1024 || n_threads % 32 != 0 || bytes_per_cta < 1024 || bytes_per_cta % 16 != 0 ||
+        bytes_per_cta > 227 * 1024 || iters < 1 || !gb_per_s)
+        return WRNN_ERR_INVALID_ARG;
+    if (cudaFuncSetAttribute(wrnn::smem_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes_per_cta) != cudaSuccess) {
+        cudaGetLastError();
+        return WRNN_ERR_UNSUPPORTED;
+    }
+    unsigned *sink = nullptr;
+    if (cudaMalloc((void **)&sink, (size_t)n_ctas * 4) != cudaSuccess) { cudaGetLastError(); return WRNN_ERR_NOMEM; }
+    cudaEvent_t e0, e1;
+    cudaEventCreate(&e0); cudaEventCreate(&e1);
+    int rc = WRNN_OK;
+    float ms = 0.f;
+    for (int rep = 0; rep < 2 && rc == WRNN_OK; ++rep) {             // first repetition warms up
+        cudaEventRecord(e0, 0);
+        wrnn::smem_stream_kernel<<<n_ctas, n_threads, bytes_per_cta>>>(bytes_per_cta, iters, sink);
+        if (cudaGetLastError() != cudaSuccess) { rc = WRNN_ERR_CUDA; break; }
+        ++wrnn::g_launches;
+        cudaEventRecord(e1, 0);
+        if (cudaEventSynchronize(e1) != cudaSuccess) { rc = WRNN_ERR_CUDA; break; }
+        cudaEventElapsedTime(&ms, e0, e1);
+    }
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    cudaFree(sink);
+    if (rc == WRNN_OK) *gb_per_s = (float)((double)n_ctas * bytes_per_cta * iters / (ms * 1e-3) / 1e9);
+    return rc;
+}

@@ -8,6 +8,7 @@
 //   B  q_c = relu(O1 y_c + b1)          C  l_c = O2 q_c + b2         D  draw c_t
 //   E  fine gates (now with c_t) -> y_f
 //   F  q_f = relu(O3 y_f + b3)          G  l_f = O4 q_f + b4         H  draw f_t, emit sample
+#include <algorithm>
 #include <cstdio>
 
 #include "wrnn_internal.h"
@@ -256,18 +257,22 @@ __global__ void __launch_bounds__(512, 1) generic_step_kernel(const GenericParam
 
 __global__ void cond_project_kernel(const float *__restrict__ cond, const float *__restrict__ W_condT,
                                     const float *__restrict__ b_gate, float *__restrict__ g, int G, int D,
-                                    int n_frames)
+                                    long long n_pairs)
 {
+    // blockIdx.y strides over the (row of the batch, frame) pairs, so no grid dimension limits their number
     extern __shared__ float fr[];
-    const int k = blockIdx.y, b = blockIdx.z;
-    const float *f = cond + ((size_t)b * n_frames + k) * D;
-    for (int d = threadIdx.x; d < D; d += blockDim.x) fr[d] = f[d];
-    __syncthreads();
     const int row = blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= G) return;
-    float acc = 0.f;
-    for (int d = 0; d < D; ++d) acc = fmaf(W_condT[(size_t)d * G + row], fr[d], acc);
-    g[((size_t)b * n_frames + k) * G + row] = acc + (b_gate ? b_gate[row] : 0.f);
+    for (long long kb = blockIdx.y; kb < n_pairs; kb += gridDim.y) {
+        const float *f = cond + (size_t)kb * D;
+        __syncthreads();
+        for (int d = threadIdx.x; d < D; d += blockDim.x) fr[d] = f[d];
+        __syncthreads();
+        if (row < G) {
+            float acc = 0.f;
+            for (int d = 0; d < D; ++d) acc = fmaf(W_condT[(size_t)d * G + row], fr[d], acc);
+            g[(size_t)kb * G + row] = acc + (b_gate ? b_gate[row] : 0.f);
+        }
+    }
 }
 
 __global__ void cond_bias_only_kernel(const float *__restrict__ b_gate, float *__restrict__ g, int G, int batch)
@@ -282,9 +287,10 @@ int cond_project(wrnn_model *m, const float *cond, int batch, int n_frames, cuda
     if (m->cond_dim == 0) {
         cond_bias_only_kernel<<<(G * batch + 255) / 256, 256, 0, s>>>(m->b_gate, m->g, G, batch);
     } else {
-        dim3 grid((G + 255) / 256, n_frames, batch);
+        const long long n_pairs = (long long)batch * n_frames;
+        dim3 grid((G + 255) / 256, (unsigned)std::min<long long>(n_pairs, 65535));
         cond_project_kernel<<<grid, 256, m->cond_dim * sizeof(float), s>>>(cond, m->W_condT, m->b_gate, m->g, G,
-                                                                           m->cond_dim, n_frames);
+                                                                           m->cond_dim, n_pairs);
     }
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
@@ -347,6 +353,12 @@ int subscale_cond_launch(const int16_t *hist, const float *frames, const float *
                          int D, int n_frames, int hop, int r_lo, int n_rows, long long p_lo, int lag, int n_steps, cudaStream_t s)
 {
     if (n_rows <= 0 || n_steps <= 0) return WRNN_OK;
+    if (n_rows > 65535) return WRNN_ERR_UNSUPPORTED;                                  // grid.y
+    const size_t smem = (size_t)4 * D * sizeof(float);
+    if (smem > 48 * 1024 && cudaFuncSetAttribute(subscale_cond_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return WRNN_ERR_UNSUPPORTED;
+    }
     subscale_cond_kernel<<<dim3(n_steps, n_rows), dim3(64, 4), (size_t)4 * D * sizeof(float), s>>>(hist, frames, V, bias, v, B, L, F, D, n_frames, hop, r_lo, p_lo, lag, n_steps);
     ++g_launches;
     return cudaGetLastError() == cudaSuccess ? WRNN_OK : WRNN_ERR_CUDA;
@@ -461,6 +473,15 @@ static int static_scratch_base(int device, unsigned char **base, std::string *er
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
+// Called by wrnn_create (which allocates anyway) with the model's device current: looks the address up ahead of time, so
+// that with lazily loaded modules the load of the image that holds the array does not fall into a sampling call.
+void noalloc_warm(int device)
+{
+    unsigned char *base = nullptr;
+    std::string err;
+    (void)static_scratch_base(device, &base, &err);
+}
+
 }  // namespace wrnn
 
 using namespace wrnn;
@@ -505,8 +526,9 @@ extern "C" int wrnn_sample_noalloc(wrnn_model *m, const wrnn_cond *cond, int64_t
     if (m->cond_dim == 0) {
         cond_bias_only_kernel<<<(unsigned)((G * B + 255) / 256), 256, 0, s>>>(m->b_gate, g, (int)G, batch);
     } else {
-        dim3 grid((unsigned)((G + 255) / 256), (unsigned)nf, (unsigned)batch);
-        cond_project_kernel<<<grid, 256, m->cond_dim * sizeof(float), s>>>(a.cond, m->W_condT, m->b_gate, g, (int)G, m->cond_dim, (int)nf);
+        const long long n_pairs = (long long)(B * nf);
+        dim3 grid((unsigned)((G + 255) / 256), (unsigned)std::min<long long>(n_pairs, 65535));
+        cond_project_kernel<<<grid, 256, m->cond_dim * sizeof(float), s>>>(a.cond, m->W_condT, m->b_gate, g, (int)G, m->cond_dim, n_pairs);
     }
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) { m->err = "conditioning projection launch failed"; return WRNN_ERR_CUDA; }

@@ -121,6 +121,7 @@ int check_step(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t ba
 int generic_launch_info(const wrnn_model *m, int batch, int *n_ctas, int *n_threads, int *smem);
 int generic_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);   // returns wrnn_status
 int cond_project(wrnn_model *m, const float *cond, int batch, int n_frames, cudaStream_t s);
+void noalloc_warm(int device);   // resolves the device address of the fixed scratch array of wrnn_sample_noalloc (once per device)
 int fold_launch(const int16_t *x, long long n_total, int B, int16_t *sub, bool unfold, cudaStream_t s);
 int fs2_unfold_launch(const int16_t *ab, long long n, int16_t *u, cudaStream_t s);
 int subscale_cond_launch(const int16_t *hist, const float *frames, const float *V, const float *bias, float *v, int B, long long L, int F,

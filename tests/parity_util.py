@@ -75,3 +75,35 @@ def first_divergence(a: np.ndarray, b: np.ndarray) -> int:
     """Index of the first differing sample along the last axis (any row); -1 if none."""
     d = np.nonzero((a != b).any(axis=0))[0] if a.ndim == 2 else np.nonzero(a != b)[0]
     return int(d[0]) if d.size else -1
+
+
+def oracle_on_gpu_stream(om, cond_np, rows, gpu_out, seed, *, hop=120, row_stride=1, row_offset_mul=0, stream0=0,
+                         h_final=None):
+    """The oracle teacher-forced on the samples the GPU itself generated, one stream row at a time: at every step the
+    oracle sees the GPU's history and reports what it would draw, so every draw of the chosen rows is compared (a
+    free-run comparison alone stops at a row's first near-boundary draw).  rows index gpu_out's first axis (row b has
+    the global row id stream0 + b); cond_np is [batch][n_frames][D] or None.  -> dict of counts and the worst
+    final-state error (h_final = the GPU's [batch][H] final state, optional)."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    n = gpu_out.shape[1]
+
+    def one(b):
+        cf, ff = _split(gpu_out[b])
+        r = om.run(None if cond_np is None else cond_np[b:b + 1], n, 1, seed, hop=hop, row_stride=row_stride,
+                   row_offset_mul=row_offset_mul, stream0=stream0 + b, c_forced=cf, f_forced=ff)
+        nd_c, bad_c = check_indices(cf, r.c_out[0], r.margins[0, :, 0])
+        nd_f, bad_f = check_indices(ff, r.f_out[0], r.margins[0, :, 1])
+        herr = rel_err(h_final[b], r.h[0]) if h_final is not None else 0.0
+        return nd_c + nd_f, bad_c + bad_f, int((r.margins[0] < MARGIN).sum()), herr
+
+    with ThreadPoolExecutor(max_workers=NCPU) as ex:
+        res = list(ex.map(one, rows))
+    return {"rows": list(rows), "draws": 2 * n * len(res), "idx_diff": sum(r[0] for r in res), "idx_bad": sum(r[1] for r in res),
+            "near_boundary": sum(r[2] for r in res), "h_final_err": max(r[3] for r in res)}
+
+
+def _split(x):
+    """int16 samples -> the (coarse, fine) bytes the device emitted them from (plumbing for the forced arrays)."""
+    u = (x.astype(np.int32) + 32768).astype(np.uint16)
+    return (u >> 8).astype(np.uint8), (u & 255).astype(np.uint8)

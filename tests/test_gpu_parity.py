@@ -482,25 +482,82 @@ def test_multi_stream_every_row_count(env):
         os.environ.pop("WRNN_NO_PAIR", None)
 
 
-def test_config2_sparse_bf16(env):
-    """Block-sparse H=2048 bf16 (96 % of the 4x4 blocks of R_u, R_r, R_e, O1, O3 pruned), batch 1: the first
-    1,500 steps against the dense-with-zeros oracle; the full 24,000 steps for determinism and resume."""
-    torch, B = env
+def _sparse_golden():
+    """The oracle's stored 24,000-step run of the block-sparse workload (tests/golden/make_sparse2048_stream.py)."""
+    import hashlib
+    g = np.load(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "sparse2048_bf16_b1_24000_oracle.npz"))
     wl = synth.WORKLOADS[2]
     w, masks, cond = synth.build_workload(wl)
+    hsh = hashlib.sha256()
+    for k in sorted(w):
+        if w[k] is not None:
+            hsh.update(k.encode()); hsh.update(np.ascontiguousarray(w[k]).tobytes())
+    for k in sorted(masks):
+        hsh.update(k.encode()); hsh.update(np.ascontiguousarray(masks[k]).tobytes())
+    hsh.update(np.ascontiguousarray(cond).tobytes())
+    assert hsh.hexdigest() == str(g["inputs_sha256"]), "the stored oracle run belongs to other inputs: rerun tests/golden/make_sparse2048_stream.py"
+    return g, wl, w, masks, cond
+
+
+def test_config2_sparse_bf16(env):
+    """Block-sparse H=2048 bf16 (96 % of the 4x4 blocks of R_u, R_r, R_e, O1, O3 pruned), batch 1, on the four-cluster
+    sparse kernel.  (1) the first 1,500 steps, every gate / state / logit, against the dense-with-zeros oracle run here
+    (which must also reproduce the stored run); (2) all 24,000 steps teacher-forced on the oracle's stored stream: both
+    draws of every step, the vectors at every 1,000th step and the final state; (3) the free run against that stream,
+    determinism and resume."""
+    torch, B = env
+    g, wl, w, masks, cond = _sparse_golden()
     assert masks["R"].sum() == 3 * 10486 and masks["O1"].sum() == 2621
     om = orc.OracleModel(w, wl.dtype, masks)
+    n = wl.n_steps
     m = B.wrnn_create(w, wl.dtype, masks)
     try:
-        assert B.wrnn_launch_info(m, 1)["kernel"] == B.WRNN_KERNEL_SPARSE        # one 16-CTA cluster, all exchanges in DSMEM
+        assert B.wrnn_launch_info(m, 1)["kernel"] == B.WRNN_KERNEL_SPARSE
         r = pu.teacher_forced_parity(torch, B, m, om, cond, 1500, 1, SEED)
-        _report("config2/sparse", r)
+        _report("config2/sparse (1,500 steps, live oracle)", r)
         _tol_check(r, wl.dtype)
-        free = _free_run(torch, B, m, cond, wl.n_steps, 1, SEED)
-        d = pu.first_divergence(free[:, :1500], r["oracle"].out)
+        assert np.array_equal(r["oracle"].c_out[0], g["c_out"][:1500]) and np.array_equal(r["oracle"].f_out[0], g["f_out"][:1500])
+        assert np.array_equal(r["oracle"].hs[999, 0], g["snap_h"][0])       # the stored run is this oracle's
+
+        # (2) the whole second of audio on the stored stream
+        dev = "cuda:0"
+        margins = np.ones((n, 2), np.float64)
+        margins.reshape(-1)[g["nb_index"]] = g["nb_margin"]
+        cf = torch.from_numpy(g["c_out"][None].copy()).to(dev)
+        ff = torch.from_numpy(g["f_out"][None].copy()).to(dev)
+        co, fo = torch.zeros_like(cf), torch.zeros_like(ff)
+        gates = torch.zeros((n, 1, 3 * wl.H), dtype=torch.float32, device=dev)
+        hs = torch.zeros((n, 1, wl.H), dtype=torch.float32, device=dev)
+        logits = torch.zeros((n, 1, 2, 256), dtype=torch.float32, device=dev)
+        hfin = torch.zeros((1, wl.H), dtype=torch.float32, device=dev)
+        cp = torch.full((1,), 128, dtype=torch.uint8, device=dev)
+        fp = torch.zeros((1,), dtype=torch.uint8, device=dev)
+        B.wrnn_step_teacher_forced(m, torch.from_numpy(cond).to(dev), n, 1, SEED, cf, ff, co, fo, dbg_gates=gates, dbg_h=hs,
+                                   dbg_logits=logits, h=hfin, c_prev=cp, f_prev=fp)
+        torch.cuda.synchronize()
+        assert B.wrnn_poll_status(m) == 0, B.wrnn_last_error(m)
+        nd_c, bad_c = pu.check_indices(co.cpu().numpy()[0], g["c_out"], margins[:, 0])
+        nd_f, bad_f = pu.check_indices(fo.cpu().numpy()[0], g["f_out"], margins[:, 1])
+        st = torch.from_numpy(g["snap_steps"].astype(np.int64)).to(dev)
+        e_h = pu.rel_err(hs[st, 0].cpu().numpy(), g["snap_h"])
+        e_l = pu.rel_err(logits[st, 0].cpu().numpy(), g["snap_logits"])
+        sg = torch.from_numpy(g["snap_gates_steps"].astype(np.int64)).to(dev)
+        e_g = pu.rel_err(gates[sg, 0].cpu().numpy(), g["snap_gates"])
+        e_f = pu.rel_err(hfin.cpu().numpy()[0], g["h_final"])
+        print("\n[parity] config2/sparse 24,000 steps on the stored oracle stream: idx_diff=%d (near-boundary draws %d, bad %d) "
+              "at %d snapshot steps gates=%.2e h=%.2e logits=%.2e, final h=%.2e" % (
+                  nd_c + nd_f, int((margins < pu.MARGIN).sum()), bad_c + bad_f, len(g["snap_steps"]), e_g, e_h, e_l, e_f))
+        tol = pu.TOL[wl.dtype]
+        assert bad_c + bad_f == 0 and max(e_h, e_l, e_g, e_f) < tol
+        del gates, hs, logits
+
+        # (3) free run: may leave the stored stream only at a near-boundary draw; deterministic; resumable
+        free = _free_run(torch, B, m, cond, n, 1, SEED)
+        ref_out = orc.join_samples(g["c_out"], g["f_out"])
+        d = pu.first_divergence(free[0], ref_out)
         if d >= 0:
-            assert r["oracle"].margins[0, d].min() < pu.MARGIN
-        assert np.array_equal(free, _free_run(torch, B, m, cond, wl.n_steps, 1, SEED))
+            assert margins[d].min() < pu.MARGIN, (d, margins[d])
+        assert np.array_equal(free, _free_run(torch, B, m, cond, n, 1, SEED))
         h = torch.zeros((1, wl.H), dtype=torch.float32, device="cuda:0")
         cp = torch.full((1,), 128, dtype=torch.uint8, device="cuda:0")
         fp = torch.zeros((1,), dtype=torch.uint8, device="cuda:0")
@@ -585,25 +642,46 @@ def test_config3_subscale_fold_batch16(env, kernel):
 
 
 def test_config4_batched256(env):
-    """256 independent streams.  (1) all rows, first 100 steps, every gate / logit against the oracle;
-    (2) rows 0..7 for the full 24,000 steps (draws and final state, teacher-forced on the oracle's streams);
-    (3) the full 256 x 24,000 free run in the benchmark's launch configuration, rows 0..7 against (2)."""
+    """256 independent streams on the cluster-partitioned tcgen05 kernel, the one the benchmark times.
+    (1) all 256 rows, first 240 steps (two conditioning frames), every gate / state / logit and both draws against the
+        oracle, teacher-forced on the oracle's streams;
+    (2) the full 256 x 24,000 free run in the benchmark's launch configuration; the oracle is then teacher-forced on the
+        device's own samples for eight rows spread over the clusters (first, last, and rows either side of the cluster
+        boundaries), so that every one of their 2 x 24,000 draws and their final states are compared;
+    (3) rows 0..7 alone for the full 24,000 steps on a model pinned to the same kernel family, teacher-forced on the
+        oracle's streams (draws and final state)."""
     torch, B = env
     wl = synth.WORKLOADS[4]
     w, masks, cond = synth.build_workload(wl)
     om = orc.OracleModel(w, wl.dtype)
+    n = wl.n_steps
     m = B.wrnn_create(w, wl.dtype, max_batch=256)
     try:
-        r = pu.teacher_forced_parity(torch, B, m, om, cond, 100, 256, SEED, threads=pu.NCPU)
-        _report("config4/batched256 (100 steps, all rows)", r)
+        assert B.wrnn_launch_info(m, 256)["kernel"] == B.WRNN_KERNEL_BCLUSTER
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, 240, 256, SEED, threads=pu.NCPU)
+        _report("config4/batched256 (240 steps, all rows)", r)
         _tol_check(r, wl.dtype)
-        n = wl.n_steps
-        r8 = pu.teacher_forced_parity(torch, B, m, om, cond[:8], n, 8, SEED, threads=pu.NCPU, dump=False)
-        print("\n[parity] config4 rows 0..7 x %d steps: idx_diff=%d near-boundary=%d bad=%d h_final=%.2e" % (
-            n, r8["idx_diff"], r8["near_boundary"], r8["idx_bad"], r8["h_final_err"]))
-        assert r8["idx_bad"] == 0 and r8["h_final_err"] < pu.TOL[wl.dtype]
-        full = _free_run(torch, B, m, cond, n, 256, SEED)
-        _check_free_run_against_oracle(full[:8], r8["oracle"])
+        del r
+        h = torch.zeros((256, wl.H), dtype=torch.float32, device="cuda:0")
+        cp = torch.full((256,), 128, dtype=torch.uint8, device="cuda:0")
+        fp = torch.zeros((256,), dtype=torch.uint8, device="cuda:0")
+        full = _free_run(torch, B, m, cond, n, 256, SEED, h=h, c_prev=cp, f_prev=fp)
         assert len({full[b].tobytes() for b in range(256)}) == 256          # every stream is its own
+        rows = [0, 36, 37, 73, 74, 147, 221, 255]
+        chk = pu.oracle_on_gpu_stream(om, cond, rows, full, SEED, h_final=h.cpu().numpy())
+        print("\n[parity] config4 free run 256 x %d, oracle forced on the device's samples of rows %s: %d draws, idx_diff=%d "
+              "near-boundary=%d bad=%d h_final=%.2e" % (n, rows, chk["draws"], chk["idx_diff"], chk["near_boundary"], chk["idx_bad"],
+                                                        chk["h_final_err"]))
+        assert chk["idx_bad"] == 0 and chk["h_final_err"] < pu.TOL[wl.dtype], chk
     finally:
         B.wrnn_destroy(m)
+    m8 = B.wrnn_create(w, wl.dtype, max_batch=8, kernel=B.WRNN_KERNEL_BCLUSTER)
+    try:
+        assert B.wrnn_launch_info(m8, 8)["kernel"] == B.WRNN_KERNEL_BCLUSTER
+        r8 = pu.teacher_forced_parity(torch, B, m8, om, cond[:8], n, 8, SEED, threads=pu.NCPU, dump=False)
+        print("\n[parity] config4 rows 0..7 x %d steps (cluster-partitioned kernel): idx_diff=%d near-boundary=%d bad=%d h_final=%.2e" % (
+            n, r8["idx_diff"], r8["near_boundary"], r8["idx_bad"], r8["h_final_err"]))
+        assert r8["idx_bad"] == 0 and r8["h_final_err"] < pu.TOL[wl.dtype]
+        _check_free_run_against_oracle(full[:8], r8["oracle"])
+    finally:
+        B.wrnn_destroy(m8)

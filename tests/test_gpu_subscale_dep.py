@@ -77,16 +77,24 @@ def test_staggered_schedule_and_oracle(env, H, dtype, B_rows, L, F, chunk, kerne
             if chunk % 2 == 0 and F % (chunk // 2) == 0:
                 other = _gpu_run(torch, Bn, m, frames, V, b, F, chunk // 2, 2 * (F + chunk // 2), B_rows, L)
                 assert np.array_equal(other, stag)
-        # against the oracle: in the order of Eq. 4 (row after row) the first difference, if any, sits at a near-boundary draw
+        # against the oracle, every row and every draw: the oracle generates in the order of Eq. 4 conditioned on the
+        # DEVICE's samples (earlier rows through the conditioning network, the row's own past by teacher forcing) and
+        # reports what it would have drawn; only near-boundary draws may differ, in any row
         got = orc.fold(stag, B_rows)
+        want, _, mg = orc.subscale_dependent_run(om, frames, V, b, B_rows, L, synth.HOP, SEED, forced=got, teacher=True)
+        gc, gf = pu._split(got)
+        wc, wf = pu._split(want)
+        nd_c, bad_c = pu.check_indices(gc, wc, mg[:, :, 0])
+        nd_f, bad_f = pu.check_indices(gf, wf, mg[:, :, 1])
+        print("\n[parity] dependent subscale H=%d %s: %d rows x %d positions, oracle forced on the device's samples: idx_diff=%d "
+              "(near-boundary draws %d, bad %d)" % (H, kernel, B_rows, L, nd_c + nd_f, int((mg < pu.MARGIN).sum()), bad_c + bad_f))
+        assert bad_c + bad_f == 0
+        # and the free comparison with the oracle's own generation: the first difference, if any, at a near-boundary draw
         for row in range(B_rows):
             d = np.nonzero(got[row] != ref[row])[0]
             if d.size:
                 assert margins[row, d[0]].min() < pu.MARGIN, (row, int(d[0]))
-                print("\n[parity] dependent subscale: rows 0..%d identical, row %d parts at position %d (near-boundary draw)" % (row - 1, row, int(d[0])))
                 break
-        else:
-            print("\n[parity] dependent subscale H=%d: all %d x %d samples identical to the oracle's" % (H, B_rows, L))
     finally:
         Bn.wrnn_destroy(m)
 

@@ -351,3 +351,27 @@ def test_conditioning_frame_hold():
     r3 = om.run(cond, 6, 1, seed=1, hop=10, row_stride=4, row_offset_mul=1, stream0=3, dump=True)
     r4 = om.run(cond2, 6, 1, seed=1, hop=10, row_stride=4, row_offset_mul=1, stream0=3, dump=True)
     assert np.array_equal(r3.gates[:2], r4.gates[:2]) and not np.array_equal(r3.gates[2], r4.gates[2])
+
+
+def test_stored_sparse_run_is_this_oracles():
+    """The stored 24,000-step run of the block-sparse workload (tests/golden/make_sparse2048_stream.py) belongs to the
+    current input generator, and the oracle reproduces its first 120 steps and their near-boundary record."""
+    import hashlib
+    import os
+    g = np.load(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "sparse2048_bf16_b1_24000_oracle.npz"))
+    wl = synth.WORKLOADS[2]
+    w, masks, cond = synth.build_workload(wl)
+    hsh = hashlib.sha256()
+    for k in sorted(w):
+        if w[k] is not None:
+            hsh.update(k.encode()); hsh.update(np.ascontiguousarray(w[k]).tobytes())
+    for k in sorted(masks):
+        hsh.update(k.encode()); hsh.update(np.ascontiguousarray(masks[k]).tobytes())
+    hsh.update(np.ascontiguousarray(cond).tobytes())
+    assert hsh.hexdigest() == str(g["inputs_sha256"])
+    om = orc.OracleModel(w, wl.dtype, masks, wl.block)
+    r = om.run(cond, 120, 1, synth.SEED_SAMPLING, hop=synth.HOP)
+    assert np.array_equal(r.c_out[0], g["c_out"][:120]) and np.array_equal(r.f_out[0], g["f_out"][:120])
+    near = np.nonzero(r.margins[0].reshape(-1) < 1e-4)[0]
+    assert np.array_equal(near, g["nb_index"][g["nb_index"] < 240])
+    assert g["c_out"].shape == (24000,) and g["snap_h"].shape == (24, 2048) and int(g["snap_steps"][-1]) == 23999

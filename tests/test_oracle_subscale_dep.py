@@ -62,3 +62,22 @@ def test_dependency_order_and_future_horizon():
     # forcing the earlier rows to the generated ones reproduces the run
     again, cond2, _ = orc.subscale_dependent_run(om, frames, V, b, B, L, hop, seed=9, forced=base)
     assert np.array_equal(again, base) and np.array_equal(cond2, cond)
+    # teacher mode: every row also fed its own forced samples; on the oracle's own output nothing changes, and a
+    # flipped sample inside a row changes only what is drawn after it in that row and in later rows
+    t, cond3, mg = orc.subscale_dependent_run(om, frames, V, b, B, L, hop, seed=9, forced=base, teacher=True)
+    assert np.array_equal(t, base) and np.array_equal(cond3, cond)
+    bent = base.copy(); bent[1, 20] ^= 0x0100
+    t2, _, mg2 = orc.subscale_dependent_run(om, frames, V, b, B, L, hop, seed=9, forced=bent, teacher=True)
+    assert np.array_equal(t2[0], base[0]) and np.array_equal(t2[1, :21], base[1, :21])
+    # (the distance of a draw's uniform from its CDF boundary moves with every change of the logits)
+    # the bent bit is in the coarse byte of position 20: the fine draw of that very step already sees it (Eq. 2: c_t
+    # enters the fine gates), the coarse draw of the step and everything before it does not
+    assert np.array_equal(mg2[0], mg[0]) and np.array_equal(mg2[1, :20], mg[1, :20]) and mg2[1, 20, 0] == mg[1, 20, 0]
+    assert mg2[1, 20, 1] != mg[1, 20, 1] and not np.array_equal(mg2[1, 21], mg[1, 21]) and not np.array_equal(mg2[2], mg[2])
+
+
+def test_split_join_samples_roundtrip():
+    x = np.array([-32768, -1, 0, 1, 255, 256, 32767, -12345], np.int16)
+    c, f = orc.split_samples(x)
+    assert np.array_equal(orc.join_samples(c, f), x)
+    assert (c[0], f[0]) == (0, 0) and (c[2], f[2]) == (128, 0) and (c[6], f[6]) == (255, 255)

@@ -64,3 +64,24 @@ def test_single_process_needs_no_group(monkeypatch):
     assert replicas.init("gloo") is None
     assert replicas.max_over_ranks(3.5, None) == 3.5
     assert replicas.aggregate_throughput(1, 24000, 0.2) == 120000.0
+
+
+def test_launch_local_starts_the_ranks_and_reports_failures(tmp_path, monkeypatch):
+    """`--gpus N` without a launcher: the benchmark starts its own N ranks.  Two CPU ranks over gloo through that helper;
+    a rank that fails makes the launch fail; a world size other than the one asked for is refused."""
+    from paper_1802_08435_b200 import replicas
+    for k in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT"):
+        monkeypatch.delenv(k, raising=False)
+    assert replicas.needs_launch(2) and not replicas.needs_launch(1)
+    script = tmp_path / "worker.py"
+    script.write_text(WORKER + "\nreplicas.check_world(2)\nopen(sys.argv[2] + '.%d' % rank, 'w').write(str(slowest))\n")
+    mark = str(tmp_path / "done")
+    assert replicas.launch_local(2, [sys.executable, str(script), ROOT, mark], timeout_s=120) == 0
+    assert open(mark + ".0").read() == open(mark + ".1").read() == "15.0"
+    bad = tmp_path / "bad.py"
+    bad.write_text("import os, sys\nsys.exit(3 if os.environ['RANK'] == '1' else 0)\n")
+    assert replicas.launch_local(2, [sys.executable, str(bad)], timeout_s=60) == 3
+    monkeypatch.setenv("WORLD_SIZE", "2")
+    assert not replicas.needs_launch(4)
+    with pytest.raises(SystemExit):
+        replicas.check_world(4)

@@ -232,9 +232,7 @@ def roofline(ctx, wl, info, model, n_steps, ms_per_step, cond_bytes, out_bytes):
                 "peak_source": peaks["source"] + " sustained", "algorithmic_flops_per_step": flops}
         if info["kernel"] == 2:      # the multi-stream resident kernel stamps the phases of its first CTA's first warp
             pc = B.wrnn_phase_cycles(model)
-            names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_wait_recurrent",
-                     "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_wait_recurrent",
-                     "F.hid_products", "C.hid_products", "F.log_products", "C.log_products"]
+            names = B.wrnn_phase_names(model)
             roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
             roof["latency_floor"] = latency_floor(
                 ctx, info, Hh, n_weights(wl) * 2, us_per_step,
@@ -268,11 +266,9 @@ def roofline(ctx, wl, info, model, n_steps, ms_per_step, cond_bytes, out_bytes):
                                               "weight bytes / measured smem stream rate + 2 x measured chip-wide exchange")
         pc = B.wrnn_phase_cycles(model)
         tot = float(sum(pc)) or 1.0
-        names = ["F.wait_y", "F.hid_finish_send", "F.wait_q", "F.log_finish_send", "F.wait_logits", "F.draw_gates",
-                 "C.wait_y", "C.hid_finish_send", "C.wait_q", "C.log_finish_send", "C.wait_logits", "C.draw_gates",
-                 "F.hid_products", "C.hid_products", "F.log_products", "C.log_products"]
+        names = B.wrnn_phase_names(model)
         roof["phase_cycles_per_step"] = {k: round(v / n_steps, 1) for k, v in zip(names, pc)}
-        roof["wait_share"] = sum(pc[i] for i in (0, 2, 4, 6, 8, 10)) / tot
+        roof["wait_share"] = sum(v for k, v in zip(names, pc) if "wait" in k) / tot
     return roof
 
 
@@ -335,6 +331,14 @@ def measure(ctx, wl, *, steps, warmup, kernel, n_steps=None, e2e=True, cpu_budge
         total_ms = replicas.max_over_ranks(sum(a.elapsed_time(b) for a, b in evs), pg, dev)
         clocks = sampler.stop() if sampler else None
         assert B.wrnn_poll_status(model) == 0, B.wrnn_last_error(model)
+
+        if info["kernel"] == 2 and ctx.rank == 0:
+            # the phase table comes from one extra call with the stamps switched on (they slow the stamped warp, so the
+            # timed calls run without them)
+            B.wrnn_phase_profile(model, True)
+            one()
+            torch.cuda.synchronize()
+            B.wrnn_phase_profile(model, False)
 
         ms_per_step = total_ms / steps
         samples_per_call = 2 * (n_steps - 2) if fused else n_steps * wl.batch

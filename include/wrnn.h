@@ -313,14 +313,25 @@ int wrnn_fs2_sample_host(wrnn_model *m, const float *cond_host, int32_t n_frames
  *   5 / 11  softmax draw, gates of the other half, publish
  * A dense fp32 model runs the fp32 variant of the kernel: the same slots, with "partial products" read as its
  * plain fp32 row products, and 2 / 8 a second chip-wide wait (the hidden layer crosses L2 there).
- * Synchronous. */
+ * The lean single-stream kernel (the default for a dense bf16 H = 896 model) has eight phases per half, fine half in
+ * entries 0..7 and coarse half in 8..15: wait for the state half; hidden-layer products; hidden-layer sums and send;
+ * recurrent products; recurrent sums and gate preparation (while other warps wait for the cluster's hidden layer and
+ * multiply the output-layer rows); CTA barrier behind those rows and send; wait for the cluster's logits; draw, gates,
+ * publish.  wrnn_phase_names writes the sixteen names that belong to
+ * the last profiled call, comma-separated, into buf (HOST, cap bytes).
+ * The stamps cost the stamped warp, which is on the critical path of the whole chip, some tens of cycles each, so they
+ * are taken only while wrnn_phase_profile(m, 1) is in effect (default off); wrnn_phase_cycles then reports the last
+ * finished call.  Synchronous. */
+int wrnn_phase_profile(wrnn_model *m, int32_t enable);
+int wrnn_phase_names(wrnn_model *m, char *buf, int32_t cap);
 int wrnn_phase_cycles(wrnn_model *m, int64_t *out16);
 
 /* Floor of a chip-wide exchange on this device: nanoseconds per all-gather of K tagged fp32 values through
  * L2 among n_ctas co-resident CTAs of n_threads threads in an otherwise empty persistent kernel (Section 2.1:
  * once the weights are resident, what remains per step is the synchronisation between multiprocessors; the
- * sampling step needs two such exchanges).  K must be a multiple of n_ctas.  HOST out-pointer.  Synchronous;
- * allocates and frees a small device buffer. */
+ * sampling step needs two such exchanges).  Measured twice -- pollers starting at once, and pollers held back 150 cycles
+ * after their CTA's own publication, as the sampling kernels do -- and the smaller figure is reported.  K must be a
+ * multiple of n_ctas.  HOST out-pointer.  Synchronous; allocates and frees a small device buffer. */
 int wrnn_measure_exchange_floor(int32_t n_ctas, int32_t n_threads, int32_t K, int32_t iters, float *ns_per_exchange);
 
 /* Measured counterpart of the nominal shared-memory bandwidth that bounds "every resident weight read once per step"

@@ -25,7 +25,7 @@ _STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "NOMEM", "CUDA", "TIMEOUT"]
 EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
-    "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_measure_exchange_floor", "wrnn_measure_smem_stream", "wrnn_sample_noalloc",
+    "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_phase_profile", "wrnn_phase_names", "wrnn_measure_exchange_floor", "wrnn_measure_smem_stream", "wrnn_sample_noalloc",
     "wrnn_selftest_bounded_wait", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold", "wrnn_fs2_sample_host",
     "wrnn_sample_subscale_dependent", "wrnn_subscale_conditioning", "wrnn_subscale_schedule",
 ]
@@ -97,6 +97,8 @@ def lib():
         L.wrnn_last_error.restype = C.c_char_p
         L.wrnn_launch_info.argtypes = [vp, i32] + [vp] * 5
         L.wrnn_phase_cycles.argtypes = [vp, vp]
+        L.wrnn_phase_profile.argtypes = [vp, i32]
+        L.wrnn_phase_names.argtypes = [vp, vp, i32]
         L.wrnn_measure_exchange_floor.argtypes = [i32, i32, i32, i32, vp]
         L.wrnn_measure_smem_stream.argtypes = [i32, i32, i32, i32, vp]
         L.wrnn_selftest_bounded_wait.argtypes = [i64] + [vp] * 5
@@ -307,6 +309,18 @@ def wrnn_launch_info(model, batch: int = 1) -> dict:
 
 def wrnn_launch_count() -> int:
     return lib().wrnn_launch_count()
+
+
+def wrnn_phase_profile(model, enable: bool) -> None:
+    """Switch the phase stamps of the resident kernels on or off (off by default: they cost cycles on the critical warp)."""
+    _check(lib().wrnn_phase_profile(model, 1 if enable else 0), model)
+
+
+def wrnn_phase_names(model):
+    """Names of the sixteen phase slots of the last profiled call."""
+    buf = C.create_string_buffer(1024)
+    _check(lib().wrnn_phase_names(model, buf, 1024), model)
+    return buf.value.decode().split(",")
 
 
 def wrnn_phase_cycles(model):

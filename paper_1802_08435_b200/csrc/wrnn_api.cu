@@ -120,6 +120,16 @@ static bool use_resident(const wrnn_model *m, int batch)
     return m->resident != nullptr && resident_supported(m, batch, nullptr) == WRNN_OK;
 }
 
+// one stream of a dense bf16 H = 896 model: the lean form of the resident kernel (wrnn_reslean.cu)
+// (WRNN_RESIDENT_LEAN=0 keeps the first form: diagnostic, for A/B measurements on one device)
+static bool use_reslean(const wrnn_model *m, int batch)
+{
+    if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_RESIDENT) return false;
+    const char *sw = getenv("WRNN_RESIDENT_LEAN");
+    if (sw && sw[0] == '0') return false;
+    return reslean_supported(m, batch) == WRNN_OK;
+}
+
 static bool use_resf32(const wrnn_model *m, int batch)
 {
     if (m->kernel == WRNN_KERNEL_GENERIC || m->kernel == WRNN_KERNEL_BATCHED || m->kernel == WRNN_KERNEL_BCLUSTER) return false;
@@ -220,9 +230,11 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     if (a.row_lag > 0) {
         if (a.batch >= 2 && use_multi(m, a.batch)) return resmulti_run(m, a, s);
         if (a.batch >= 2 && use_bcluster(m, a.batch)) return bcluster_run(m, a, s);
-        if (a.batch == 1 && use_resident(m, 1)) return resident_run(m, a, s);     // a lone row (the ramps of the schedule)
+        if (a.batch == 1 && use_reslean(m, 1)) return reslean_run(m, a, s);           // a lone row (the ramps of the schedule)
+        if (a.batch == 1 && use_resident(m, 1)) return resident_run(m, a, s);
         return generic_run(m, a, s);
     }
+    if (use_reslean(m, a.batch)) return reslean_run(m, a, s);
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
     // two rows: the two-stream kernel (7.5 us per step against 8.2 on the multi-stream kernel); 3 to 16: the multi-stream kernel
     if (use_multi(m, a.batch) && !(a.batch == 2 && use_pair(m, 2))) return resmulti_run(m, a, s);
@@ -419,6 +431,7 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
             wrnn_destroy(m);
             return fail(nullptr, rc, "resident kernel unavailable: " + why);
         }
+        if (m->dtype == WRNN_BF16 && m->variant == 0) reslean_prepare(m);                        // optional: the row-split resident kernel serves the stream without it
         if (m->dtype == WRNN_BF16 && m->variant == 0 && max_batch >= 2) resmulti_prepare(m);   // optional: other kernels serve the batch without it
     }
     m->err.clear();             // reasons why optional kernels were not prepared are not errors of this call
@@ -433,6 +446,7 @@ void wrnn_destroy(wrnn_model *m)
     cudaSetDevice(m->device);
     cudaDeviceSynchronize();
     resident_destroy(m);
+    reslean_destroy(m);
     resf32_destroy(m);
     resmulti_destroy(m);
     batched_destroy(m);
@@ -616,7 +630,7 @@ int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n
         // rows advance together on the multi-stream resident kernel where the model has one (8.3 us per step at two rows
         // against 6.4 us per step and row on the single-stream kernel); without it up to three rows go one after the other
         // through the single-stream kernel (24 us per step of the cluster-partitioned kernel whatever the rows)
-        const int group = (n_rows >= 2 && use_multi(m, n_rows)) ? n_rows : (n_rows <= 3 && use_resident(m, 1)) ? 1 : n_rows;
+        const int group = (n_rows >= 2 && use_multi(m, n_rows)) ? n_rows : (n_rows <= 3 && (use_reslean(m, 1) || use_resident(m, 1))) ? 1 : n_rows;
         for (int b0 = 0; b0 < n_rows; b0 += group) {
             const int r0 = r_a + b0;
             const long long p0 = p_lo - (long long)b0 * lag;
@@ -731,6 +745,10 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
                      int64_t *weight_bytes_per_step, int32_t *smem_bytes)
 {
     if (!m || batch < 1 || batch > m->max_batch) return WRNN_ERR_INVALID_ARG;
+    if (use_reslean(m, batch)) {
+        if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
+        return reslean_launch_info(m, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
+    }
     if (use_resident(m, batch)) {
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
@@ -766,12 +784,36 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
 
 int64_t wrnn_launch_count(void) { return g_launches.load(); }
 
+int wrnn_phase_profile(wrnn_model *m, int32_t enable)
+{
+    if (!m) return WRNN_ERR_INVALID_ARG;
+    m->prof_enabled = enable != 0;
+    return WRNN_OK;
+}
+
+int wrnn_phase_names(wrnn_model *m, char *buf, int32_t cap)
+{
+    if (!m || !buf || cap < 1) return WRNN_ERR_INVALID_ARG;
+    const char *first = "F.wait_y,F.hid_finish_send,F.wait_q,F.log_finish_send,F.wait_logits,F.draw_gates,"
+                        "C.wait_y,C.hid_finish_send,C.wait_q,C.log_finish_send,C.wait_logits,C.draw_gates,"
+                        "F.hid_products,C.hid_products,F.log_products,C.log_products";
+    const char *multi = "F.wait_y,F.hid_finish_send,F.wait_q,F.log_finish_send,F.wait_logits,F.draw_wait_recurrent,"
+                        "C.wait_y,C.hid_finish_send,C.wait_q,C.log_finish_send,C.wait_logits,C.draw_wait_recurrent,"
+                        "F.hid_products,C.hid_products,F.log_products,C.log_products";
+    const char *lean = "F.wait_y,F.hid_products,F.hid_sums_send,F.recurrent_products,F.rsums_gateprep,F.wait_logit_rows_send,F.wait_logits,F.draw_gates,"
+                       "C.wait_y,C.hid_products,C.hid_sums_send,C.recurrent_products,C.rsums_gateprep,C.wait_logit_rows_send,C.wait_logits,C.draw_gates";
+    const char *src = (!m->resf32 && m->prof_multi) ? multi : (!m->resf32 && m->prof_lean) ? lean : first;
+    std::snprintf(buf, (size_t)cap, "%s", src);
+    return WRNN_OK;
+}
+
 int wrnn_phase_cycles(wrnn_model *m, int64_t *out16)
 {
     if (!m || !out16) return WRNN_ERR_INVALID_ARG;
     static_assert(sizeof(long long) == sizeof(int64_t), "");
     if (m->resf32) return resf32_phase_cycles(m, reinterpret_cast<long long *>(out16));
     if (m->prof_multi) return resmulti_phase_cycles(m, reinterpret_cast<long long *>(out16));
+    if (m->prof_lean) return reslean_phase_cycles(m, reinterpret_cast<long long *>(out16));
     return resident_phase_cycles(m, reinterpret_cast<long long *>(out16));
 }
 

@@ -129,14 +129,17 @@ __device__ __forceinline__ int float_order_key(float x)
 }
 __device__ __forceinline__ int warp_softmax_draw_fast(const float (&l)[8], float u, int lane)
 {
-    float m = l[0];
-#pragma unroll
-    for (int i = 1; i < 8; ++i) m = fmaxf(m, l[i]);
+    // (pairwise trees instead of chains: this sits on the critical path of every half-step)
+    float m = fmaxf(fmaxf(fmaxf(l[0], l[1]), fmaxf(l[2], l[3])), fmaxf(fmaxf(l[4], l[5]), fmaxf(l[6], l[7])));
     const int km = __reduce_max_sync(FULL, float_order_key(m));
     m = __int_as_float(km ^ ((km >> 31) & 0x7fffffff));
-    float w[8], s = 0.f;
+    float w[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) { w[i] = __expf(l[i] - m); s += w[i]; }
+    for (int i = 0; i < 8; ++i) w[i] = __expf(l[i] - m);
+    // running sums inside the lane: p[i] = w[0] + ... + w[i]
+    const float p1 = w[0] + w[1], p3 = p1 + (w[2] + w[3]), p5 = p3 + (w[4] + w[5]), p7 = p5 + (w[6] + w[7]);
+    const float p0 = w[0], p2 = p1 + w[2], p4 = p3 + w[4], p6 = p5 + w[6];
+    const float s = p7;
     float inc = s;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -144,15 +147,16 @@ __device__ __forceinline__ int warp_softmax_draw_fast(const float (&l)[8], float
         if (lane >= o) inc += t;
     }
     const float thr = u * __shfl_sync(FULL, inc, 31);
-    float run = inc - s;                 // exclusive prefix of this lane
-    int pick = 256;
-#pragma unroll
-    for (int i = 7; i >= 0; --i) {       // last assignment wins: the smallest qualifying index
-        float r = run;
-#pragma unroll
-        for (int j = 0; j <= i; ++j) r += w[j];
-        if (r > thr) pick = 8 * lane + i;
-    }
+    const float run = inc - s;           // exclusive prefix of this lane
+    int pick = 256;                      // last assignment wins: the smallest qualifying index
+    if (run + p7 > thr) pick = 8 * lane + 7;
+    if (run + p6 > thr) pick = 8 * lane + 6;
+    if (run + p5 > thr) pick = 8 * lane + 5;
+    if (run + p4 > thr) pick = 8 * lane + 4;
+    if (run + p3 > thr) pick = 8 * lane + 3;
+    if (run + p2 > thr) pick = 8 * lane + 2;
+    if (run + p1 > thr) pick = 8 * lane + 1;
+    if (run + p0 > thr) pick = 8 * lane;
     pick = __reduce_min_sync(FULL, pick);
     return pick == 256 ? 255 : pick;
 }
@@ -188,8 +192,10 @@ __device__ __forceinline__ float scale4(int v) { return (float)v * (1.0f / 7.5f)
 __device__ __forceinline__ float sigmoidf_fast(float x) { return __fdividef(1.0f, 1.0f + __expf(-x)); }
 __device__ __forceinline__ float tanhf_fast(float x)
 {
-    const float e = __expf(-2.0f * fabsf(x));
-    return copysignf(__fdividef(1.0f - e, 1.0f + e), x);
+    // 1 - 2 / (1 + e^{2x}): one ex2, one rcp; saturates to +-1 through e^{2x} = inf / 0 (the argument is clamped so that
+    // the reciprocal never sees inf)
+    const float e = __expf(2.0f * fminf(x, 40.0f));
+    return 1.0f - __fdividef(2.0f, 1.0f + e);
 }
 
 // ------------------------------------------------------------------ memory-order helpers

@@ -7,7 +7,10 @@
 
 namespace wrnn {
 
-__global__ void exchange_floor_kernel(unsigned long long *slots, int K, int U, int iters, int *err)
+// gap: cycles between a CTA's own publication and its first poll (0 = poll at once).  A poll that reaches L2 before the
+// words do costs a whole round trip before the same thread can look again, and early polls load the L2 slices the
+// publishing stores have to get through; the sampling kernels hold their pollers back the same way.
+__global__ void exchange_floor_kernel(unsigned long long *slots, int K, int U, int iters, int gap, int *err)
 {
     __shared__ float sh[2048];
     float acc = 0.f;
@@ -19,6 +22,7 @@ __global__ void exchange_floor_kernel(unsigned long long *slots, int K, int U, i
             asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(buf + blockIdx.x * U + threadIdx.x), "l"(v) : "memory");
         }
         bool bad = false;
+        if (gap > 0) { const long long c0 = clock64(); while (clock64() - c0 < gap) { } }
         for (int i = threadIdx.x; i < K; i += blockDim.x) {
             unsigned long long v;
             unsigned n = 0;
@@ -53,11 +57,14 @@ extern "C" int wrnn_measure_exchange_floor(int32_t n_ctas, int32_t n_threads, in
     cudaEvent_t e0, e1;
     cudaEventCreate(&e0); cudaEventCreate(&e1);
     int rc = WRNN_OK;
-    float ms = 0.f;
-    for (int rep = 0; rep < 2 && rc == WRNN_OK; ++rep) {             // first repetition warms up
+    float ms = 0.f, best_ms = 0.f;
+    // repetition 0 warms up; 1: pollers start at once; 2: pollers held back (the protocol of the sampling kernels); the
+    // smaller of the two is reported
+    for (int rep = 0; rep < 3 && rc == WRNN_OK; ++rep) {
+        int gap = rep == 2 ? 150 : 0;
         cudaMemset(slots, 0, (size_t)2 * K * 8);
         cudaMemset(err, 0, 4);
-        void *args[] = {(void *)&slots, (void *)&K, (void *)&U, (void *)&iters, (void *)&err};
+        void *args[] = {(void *)&slots, (void *)&K, (void *)&U, (void *)&iters, (void *)&gap, (void *)&err};
         cudaEventRecord(e0, 0);
         if (cudaLaunchCooperativeKernel((void *)exchange_floor_kernel, dim3(n_ctas), dim3(n_threads), args, 0, 0) != cudaSuccess) {
             cudaGetLastError(); rc = WRNN_ERR_CUDA; break;
@@ -66,13 +73,14 @@ extern "C" int wrnn_measure_exchange_floor(int32_t n_ctas, int32_t n_threads, in
         cudaEventRecord(e1, 0);
         if (cudaEventSynchronize(e1) != cudaSuccess) { rc = WRNN_ERR_CUDA; break; }
         cudaEventElapsedTime(&ms, e0, e1);
+        if (rep == 1 || (rep == 2 && ms < best_ms)) best_ms = ms;
         int herr = 0;
         cudaMemcpy(&herr, err, 4, cudaMemcpyDeviceToHost);
         if (herr) rc = WRNN_ERR_TIMEOUT;
     }
     cudaEventDestroy(e0); cudaEventDestroy(e1);
     cudaFree(slots); cudaFree(err);
-    if (rc == WRNN_OK) *ns_per_exchange = ms * 1e6f / (float)iters;
+    if (rc == WRNN_OK) *ns_per_exchange = best_ms * 1e6f / (float)iters;
     return rc;
 }
 

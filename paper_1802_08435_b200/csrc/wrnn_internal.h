@@ -61,6 +61,7 @@ struct ResidentPack;   // packed weights of the shared-memory-resident kernels (
 struct BatchedPack;    // fragment-packed weights and activation images of the batched kernel (opaque here)
 struct SparsePack;     // compressed block rows of the single-cluster block-sparse kernel (opaque here)
 struct ResF32Pack;     // per-CTA fp32 weight shards of the single-stream fp32 resident kernel (opaque here)
+struct ResLeanPack;      // per-CTA weights of the lean single-stream resident kernel (opaque here)
 struct ResMultiPack;  // per-CTA weights of the multi-stream resident kernel (opaque here)
 struct BcPack;         // per-CTA weight slices and stacked activation images of the cluster-partitioned multi-row kernel
 
@@ -96,8 +97,11 @@ struct wrnn_model {
     uint8_t *sub_scratch = nullptr; size_t sub_cap = 0;   // history, conditioning and carry state of wrnn_sample_subscale_dependent
 
     wrnn::ResidentPack *resident = nullptr;
+    wrnn::ResLeanPack *reslean = nullptr;
+    bool prof_lean = false;           // the last call with phase timing ran on the lean single-stream resident kernel
     wrnn::ResF32Pack *resf32 = nullptr;
     wrnn::ResMultiPack *resmulti = nullptr;
+    bool prof_enabled = false;      // wrnn_phase_profile: the resident kernels stamp their phases
     bool prof_multi = false;        // the last call with phase timing ran on the multi-stream resident kernel
     wrnn::BatchedPack *batched = nullptr;
     wrnn::SparsePack *sparse_pack = nullptr;
@@ -137,6 +141,18 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
 int resident_phase_cycles(const wrnn_model *m, long long *out16);
 int resident_pair_supported(const wrnn_model *m, int batch);          // two streams per launch on the same weights (batch 2 or 4)
 int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s);
+
+// host packers shared by the resident kernels (wrnn_resident.cu)
+void dense_row_bf16(const BsrHost &M, int row, int c0, int n, uint16_t *dst);       // dense row of a block-row matrix -> bf16 bits of columns [c0, c0 + n)
+void pack_tile(const std::vector<std::vector<uint16_t>> &rows, int K, uint16_t *dst);   // rows[16][K] -> m16n8k16 A fragments [K/16][32 lanes][8]
+
+// wrnn_reslean.cu: one stream of a dense bf16 H = 896 model, the row-split resident kernel with a shorter chain per half-step
+int reslean_supported(const wrnn_model *m, int batch);
+int reslean_prepare(wrnn_model *m);
+void reslean_destroy(wrnn_model *m);
+int reslean_launch_info(const wrnn_model *m, int *n_ctas, int *n_threads, int *smem, int64_t *weight_bytes);
+int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s);
+int reslean_phase_cycles(const wrnn_model *m, long long *out16);
 
 // wrnn_resmulti.cu: 2 to 16 lock-step streams of a dense bf16 H = 896 model on resident weights
 int resmulti_supported(const wrnn_model *m, int batch);

@@ -513,7 +513,7 @@ int resf32_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
     p.limit_ns = 2000000000ull;
-    p.prof = k.d_prof;
+    p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
 
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)6 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;

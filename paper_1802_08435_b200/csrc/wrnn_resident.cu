@@ -914,7 +914,7 @@ static uint16_t bf16_bits_of(float rounded)
 }
 
 // dense row `row` of a host block-row matrix -> bf16 bits for columns [c0, c0 + n)
-static void dense_row_bf16(const BsrHost &M, int row, int c0, int n, uint16_t *dst)
+void dense_row_bf16(const BsrHost &M, int row, int c0, int n, uint16_t *dst)
 {
     std::fill(dst, dst + n, (uint16_t)0);
     const int br = row / 4, r = row % 4;
@@ -931,7 +931,7 @@ static void dense_row_bf16(const BsrHost &M, int row, int c0, int n, uint16_t *d
 // lane (g, t) holds (row g, k 2t..2t+1), (row g+8, same), (row g, k 2t+8..9), (row g+8, same).
 // The vector side stores element 16 kt + c at split2_pos and the B-fragment load reads it back from
 // there, so fragment column c of k-tile kt is plain column 16 kt + c of the matrix.
-static void pack_tile(const std::vector<std::vector<uint16_t>> &rows, int K, uint16_t *dst)
+void pack_tile(const std::vector<std::vector<uint16_t>> &rows, int K, uint16_t *dst)
 {
     for (int kt = 0; kt < K / 16; ++kt)
         for (int lane = 0; lane < 32; ++lane) {
@@ -1166,7 +1166,7 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.a_forced = a.a_forced; p.b_forced = a.b_forced; p.a_out = a.a_out; p.b_out = a.b_out;
     p.status = m->status;
     p.limit_ns = 2000000000ull;
-    p.prof = k.d_prof;
+    p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
 
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
@@ -1185,6 +1185,7 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     }
     ++g_launches;
     m->prof_multi = false;
+    m->prof_lean = false;
     return WRNN_OK;
 }
 
@@ -1227,7 +1228,7 @@ int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s
     p.dbg_logits = a.dbg_logits ? a.dbg_logits + (size_t)b0 * 512 : nullptr;
     p.status = m->status;
     p.limit_ns = 2000000000ull;
-    p.prof = k.d_prof;
+    p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
 
     if (cudaMemsetAsync(k.d_slots2, 0, (size_t)8 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (pair == 0 && cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
@@ -1243,6 +1244,7 @@ int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s
     }
     ++g_launches;
     m->prof_multi = false;
+    m->prof_lean = false;
     return WRNN_OK;
 }
 

@@ -789,7 +789,7 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
     p.limit_ns = 2000000000ull;
-    p.prof = k.d_prof;
+    p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
     { const char *d = getenv("WRNN_MULTI_FLAG"); p.flag_mode = d ? (unsigned)atoi(d) : 1u; }    // diagnostic: A/B of the gather protocol
 
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * MAXS * MK * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;

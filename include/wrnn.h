@@ -348,6 +348,16 @@ int wrnn_measure_smem_stream(int32_t n_ctas, int32_t n_threads, int32_t bytes_pe
  * Nothing faults and the context stays usable.  Synchronous; allocates and frees two small device buffers. */
 int wrnn_selftest_bounded_wait(int64_t limit_ns, int32_t *code, int32_t *cta, int32_t *step, int32_t *phase, float *waited_ms);
 
+/* Self-test of the give-up paths of the sampling kernels themselves (the failure is made on the host side of the
+ * protocol: a message is withheld; nothing faults, traps or spins without bound).  From the next launch on this model,
+ * CTA `cta` withholds at step `step` (relative to the call) what it would hand to the other CTAs: the state values it
+ * publishes (shared-memory-resident and sparse kernels), one operand load of its own tensor pipeline (cluster-partitioned
+ * kernel), or its arrivals at the grid barrier (any-shape and grid-phased kernels); limit_ns (0 = the default of two
+ * seconds, at most two seconds) bounds every device-side wait of the launch.  The waits that depend on the missing piece
+ * run out, the first CTA to give up records WRNN_ERR_TIMEOUT with (cta, step, phase), every CTA leaves through its normal
+ * exit and wrnn_poll_status reports it.  cta = -1 restores normal operation (limit_ns still applies).  Host only. */
+int wrnn_selftest_lost_word(wrnn_model *m, int64_t limit_ns, int32_t cta, int64_t step);
+
 /* Kernels launched by this library in this process since load (all models). */
 int64_t wrnn_launch_count(void);
 

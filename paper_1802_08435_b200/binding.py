@@ -26,7 +26,7 @@ EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
     "wrnn_sample_subscale", "wrnn_sample_host", "wrnn_poll_status", "wrnn_last_error", "wrnn_launch_info",
     "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_phase_profile", "wrnn_phase_names", "wrnn_measure_exchange_floor", "wrnn_measure_smem_stream", "wrnn_sample_noalloc",
-    "wrnn_selftest_bounded_wait", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold", "wrnn_fs2_sample_host",
+    "wrnn_selftest_bounded_wait", "wrnn_selftest_lost_word", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold", "wrnn_fs2_sample_host",
     "wrnn_sample_subscale_dependent", "wrnn_subscale_conditioning", "wrnn_subscale_schedule",
 ]
 
@@ -102,6 +102,7 @@ def lib():
         L.wrnn_measure_exchange_floor.argtypes = [i32, i32, i32, i32, vp]
         L.wrnn_measure_smem_stream.argtypes = [i32, i32, i32, i32, vp]
         L.wrnn_selftest_bounded_wait.argtypes = [i64] + [vp] * 5
+        L.wrnn_selftest_lost_word.argtypes = [vp, i64, i32, i64]
         L.wrnn_launch_count.argtypes = []
         L.wrnn_launch_count.restype = i64
         _lib = L
@@ -349,6 +350,12 @@ def wrnn_selftest_bounded_wait(limit_ns: int = 50_000_000) -> dict:
     code, cta, step, phase, ms = C.c_int32(), C.c_int32(), C.c_int32(), C.c_int32(), C.c_float()
     _check(lib().wrnn_selftest_bounded_wait(limit_ns, C.byref(code), C.byref(cta), C.byref(step), C.byref(phase), C.byref(ms)))
     return {"code": code.value, "cta": cta.value, "step": step.value, "phase": phase.value, "waited_ms": ms.value}
+
+
+def wrnn_selftest_lost_word(model, limit_ns: int = 0, cta: int = -1, step: int = -1) -> None:
+    """From the next launch on: CTA `cta` withholds at `step` what it hands to the other CTAs and every device-side wait
+    is bounded by limit_ns (0 = default); cta = -1 restores normal operation."""
+    _check(lib().wrnn_selftest_lost_word(model, limit_ns, cta, step), model)
 
 
 def wrnn_sample_noalloc(model, cond, n_steps: int, batch: int, seed: int, out, *, hop: int = 120, row_stride: int = 1,

@@ -784,6 +784,15 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
 
 int64_t wrnn_launch_count(void) { return g_launches.load(); }
 
+int wrnn_selftest_lost_word(wrnn_model *m, int64_t limit_ns, int32_t cta, int64_t step)
+{
+    if (!m || limit_ns < 0 || limit_ns > 2000000000ll || cta < -1 || step < -1) return WRNN_ERR_INVALID_ARG;
+    m->dbg_limit_ns = (unsigned long long)limit_ns;
+    m->dbg_skip_cta = cta;
+    m->dbg_skip_step = cta < 0 ? -1 : step;
+    return WRNN_OK;
+}
+
 int wrnn_phase_profile(wrnn_model *m, int32_t enable)
 {
     if (!m) return WRNN_ERR_INVALID_ARG;

@@ -72,6 +72,7 @@ struct BatchedParams {
     unsigned long long *bar;
     DevStatus *status;
     unsigned long long limit_ns;
+    int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
     int tc;                                     // phase A on tcgen05
     __nv_bfloat16 *hrm[2][2];                   // [buffer][part] row-major hi / lo state
     alignas(64) CUtensorMap tmR;
@@ -383,6 +384,7 @@ __global__ void __launch_bounds__(512, 1) batched_step_kernel(const __grid_const
     };
 
     for (long long s = 0; s < p.n_steps && !failed; ++s) {
+        if ((int)blockIdx.x == p.skip_cta && s == p.skip_step) { failed = true; break; }      // self-test: this CTA's arrivals go missing
         __nv_bfloat16 *nhi = tc ? p.hrm[cur ^ 1][0] : nullptr, *nlo = tc ? p.hrm[cur ^ 1][1] : nullptr;
         // ---- A: a = R h_{t-1}
         BSTAMP(31);
@@ -646,7 +648,7 @@ int batched_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.bar = k.bar; p.status = m->status;
-    p.limit_ns = 2000000000ull;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
     // tcgen05 phase A: one CTA per (128 rows of R) x (BN rows of the batch); falls back to mma.sync when the grid is too small
     const int bn = bn_for(nt);
     if (k.tc && bn && (3 * m->H / TC_BM) * ((p.Bp + bn - 1) / bn) <= m->n_sms) {

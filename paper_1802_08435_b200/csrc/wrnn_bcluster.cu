@@ -79,6 +79,8 @@ struct BcParams {
     int16_t *out;
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
+    unsigned long long limit_ns;             // bound of every mbarrier wait
+    int skip_cta; long long skip_step;       // self-test: this CTA's weight producer withholds its first load of this step (-1: none)
     alignas(64) CUtensorMap tmWr;
     alignas(64) CUtensorMap tmO1;
     alignas(64) CUtensorMap tmO2;
@@ -213,7 +215,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
         *failed = 1;
         if (atomicCAS(&p.status->code, DEV_OK, DEV_TIMEOUT) == DEV_OK) { p.status->cta = blockIdx.x; p.status->step = step; p.status->phase = phase; }
     };
-    if (!mbar_wait(smem_u32(&s_wload), 0)) fail(-1, 0);
+    if (!mbar_wait(smem_u32(&s_wload), 0, p.limit_ns)) fail(-1, 0);
 
     // ---- initial state: fp32 in the registers of the gate threads, stacked high / low tiles in buffer 0
     // (operand rows that no thread writes were zeroed by the host)
@@ -265,7 +267,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
         if (warp == 1) {
             if (role == 0) {
                 RBEGIN();
-                if (!*failed && !mbar_wait(done_bar, dph)) fail(step, phase);
+                if (!*failed && !mbar_wait(done_bar, dph, p.limit_ns)) fail(step, phase);
                 RSTAMP(31);
             }
             __syncwarp();
@@ -288,7 +290,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 bool ok = true;
                 RBEGIN();
                 for (int kb = 0; kb < nkbA; ++kb) {
-                    if (!mbar_wait(full0 + 8u * (uint32_t)rst, rph)) { ok = false; break; }
+                    if (!mbar_wait(full0 + 8u * (uint32_t)rst, rph, p.limit_ns)) { ok = false; break; }
                     tc_fence_after();
                     umma_bf16_kblock(tmem + BC_COL_A, da, da + boff, idesc, kb ? 1u : 0u);
                     umma_commit(empty0 + 8u * (uint32_t)rst);
@@ -307,11 +309,11 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 RBEGIN();
                 // (the writers of the state tiles and of this shared memory issued their proxy fences before the cluster barrier)
                 for (int kb = 0; kb < nkbA; ++kb) {
-                    if (!mbar_wait(empty0 + 8u * (uint32_t)rst, rph ^ 1)) { fail(step, 1); break; }
+                    if (!mbar_wait(empty0 + 8u * (uint32_t)rst, rph ^ 1, p.limit_ns)) { fail(step, 1); break; }
                     const uint32_t fb = full0 + 8u * (uint32_t)rst;
                     mbar_expect_tx(fb, bytes);
                     if (is_act) tma_load_3d(dst, tmA, fb, 0, 0, coord);
-                    else tma_load_2d(dst, &p.tmWr, fb, 0, coord);
+                    else if (!(kb == 0 && (int)blockIdx.x == p.skip_cta && step == p.skip_step)) tma_load_2d(dst, &p.tmWr, fb, 0, coord);
                     coord += cstep;
                     dst += (uint32_t)p.stage_bytes;
                     if (++rst == p.n_stages) { rst = 0; rph ^= 1; dst -= (uint32_t)p.n_stages * (uint32_t)p.stage_bytes; }
@@ -335,14 +337,14 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 const uint32_t astep = abytes >> 4, wstep = (uint32_t)(n_w * 8);
                 uint32_t da = umma_desc_lo(area0), db = umma_desc_lo(wres);
                 RBEGIN();
-                bool ok = mbar_wait(smem_u32(&s_ofull[0]), oph);
+                bool ok = mbar_wait(smem_u32(&s_ofull[0]), oph, p.limit_ns);
                 RSTAMP(30);
                 if (ok) {
                     tc_fence_after();
                     int kb = 0;
                     for (; kb < p.kpart; ++kb, da += astep, db += wstep) umma_bf16_kblock(tmem + dcol, da, db, idesc, kb ? 1u : 0u);
                     RSTAMP(27);
-                    ok = mbar_wait(smem_u32(&s_ofull[1]), oph);
+                    ok = mbar_wait(smem_u32(&s_ofull[1]), oph, p.limit_ns);
                     RSTAMP(28);
                     if (ok) {
                         tc_fence_after();
@@ -793,6 +795,7 @@ int bcluster_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.row_lag = a.row_lag; p.out_pitch = a.out_pitch ? a.out_pitch : a.n_steps;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
     p.tmWr = k.tmWr; p.tmO1 = k.tmO1; p.tmO2 = k.tmO2; p.tmO3 = k.tmO3; p.tmO4 = k.tmO4;
     const int nkbA = m->H / 64, nkbH = m->H / 128;
     const long long tilesA = (long long)k.max_clusters * nkbA, tilesH = (long long)k.max_clusters * nkbH;

@@ -37,6 +37,7 @@ struct GenericParams {
     unsigned long long *bar;
     DevStatus *status;
     unsigned long long limit_ns;
+    int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
 };
 
 template <typename WT> __device__ __forceinline__ void load_block(const void *vals, int i, float (&w)[16]);
@@ -155,6 +156,7 @@ __global__ void __launch_bounds__(512, 1) generic_step_kernel(const GenericParam
     if (!bar.sync(-1, 0)) return;
 
     for (long long s = 0; s < p.n_steps; ++s) {
+        if ((int)blockIdx.x == p.skip_cta && s == p.skip_step) return;      // self-test: this CTA's arrivals go missing
         // ---- A: recurrent product for all gates; coarse gates finish here
         for (int item = gw; item < (H / 4) * ntiles; item += nw) {
             const int ug = item / ntiles, b0 = (item % ntiles) * TB, nb = min(TB, B - b0);
@@ -418,7 +420,7 @@ int generic_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.row_lag = a.row_lag; p.out_pitch = a.out_pitch ? a.out_pitch : a.n_steps;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.bar = m->bar; p.status = m->status;
-    p.limit_ns = 2000000000ull;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
 
     if (cudaMemsetAsync(m->bar, 0, sizeof(unsigned long long), s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
@@ -553,7 +555,7 @@ extern "C" int wrnn_sample_noalloc(wrnn_model *m, const wrnn_cond *cond, int64_t
     p.dbg_gates = nullptr; p.dbg_h = nullptr; p.dbg_logits = nullptr;
     p.bar = reinterpret_cast<unsigned long long *>(base + o_bar);
     p.status = m->status;
-    p.limit_ns = 2000000000ull;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
 
     // the array keeps the previous call's contents: the arrival counter must start at zero; the state and
     // sample bytes are (re)initialised by the kernel itself before use

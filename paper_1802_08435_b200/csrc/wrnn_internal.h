@@ -101,6 +101,12 @@ struct wrnn_model {
     bool prof_lean = false;           // the last call with phase timing ran on the lean single-stream resident kernel
     wrnn::ResF32Pack *resf32 = nullptr;
     wrnn::ResMultiPack *resmulti = nullptr;
+    // wrnn_selftest_lost_word: bound of every device-side wait (0 = the default of two seconds) and the CTA / step whose
+    // publication (or operand load) is withheld (-1 = none)
+    unsigned long long dbg_limit_ns = 0;
+    int dbg_skip_cta = -1;
+    long long dbg_skip_step = -1;
+    unsigned long long wait_limit_ns() const { return dbg_limit_ns ? dbg_limit_ns : 2000000000ull; }
     bool prof_enabled = false;      // wrnn_phase_profile: the resident kernels stamp their phases
     bool prof_multi = false;        // the last call with phase timing ran on the multi-stream resident kernel
     wrnn::BatchedPack *batched = nullptr;

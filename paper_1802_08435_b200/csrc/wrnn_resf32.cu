@@ -57,6 +57,7 @@ struct ResF32Params {
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
+    int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
     long long *prof;                         // [16] per-phase cycle totals of CTA 0, warp 0 (same slots as the bf16 kernel)
 };
 
@@ -187,8 +188,9 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
-        st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
-                       ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+        if (!(cta == p.skip_cta && s == p.skip_step))
+            st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
+                           ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
         if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
     };
@@ -512,7 +514,7 @@ int resf32_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
-    p.limit_ns = 2000000000ull;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
     p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
 
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)6 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;

@@ -72,6 +72,7 @@ struct ResidentParams {
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
+    int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
     long long *prof;                         // optional [16] per-phase cycle totals of CTA 0, warp 0
 };
 
@@ -262,8 +263,9 @@ __global__ void __launch_bounds__(512, 1) resident_dense_kernel(const ResidentPa
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
-        st_relaxed_u64(p.slots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
-                       ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+        if (!(cta == p.skip_cta && s == p.skip_step))
+            st_relaxed_u64(p.slots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
+                           ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
         if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
     };
@@ -717,8 +719,9 @@ __global__ void __launch_bounds__(512, 1) resident_pair_kernel(const PairParams 
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
-        st_relaxed_u64(pp.slots2 + ((size_t)((half_g ? 2 : 0) + (s & 1)) * 2 + ws) * K + j,
-                       ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+        if (!(cta == p.skip_cta && s == p.skip_step))
+            st_relaxed_u64(pp.slots2 + ((size_t)((half_g ? 2 : 0) + (s & 1)) * 2 + ws) * K + j,
+                           ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * pp.n_batch + ws) * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
         if (p.dbg_h) p.dbg_h[((size_t)s * pp.n_batch + ws) * H + jj] = hn;
     };
@@ -1165,7 +1168,7 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.a_in = a.a_in; p.b_in = a.b_in; p.a_st_out = a.a_st_out; p.b_st_out = a.b_st_out;
     p.a_forced = a.a_forced; p.b_forced = a.b_forced; p.a_out = a.a_out; p.b_out = a.b_out;
     p.status = m->status;
-    p.limit_ns = 2000000000ull;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
     p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
 
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
@@ -1227,7 +1230,7 @@ int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s
     p.dbg_h = a.dbg_h ? a.dbg_h + (size_t)b0 * H : nullptr;
     p.dbg_logits = a.dbg_logits ? a.dbg_logits + (size_t)b0 * 512 : nullptr;
     p.status = m->status;
-    p.limit_ns = 2000000000ull;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
     p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
 
     if (cudaMemsetAsync(k.d_slots2, 0, (size_t)8 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;

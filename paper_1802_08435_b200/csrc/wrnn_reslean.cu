@@ -67,6 +67,7 @@ struct ResLeanParams {
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
+    int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
     long long *prof;                         // optional [n CTAs][16] per-phase cycle totals of warp 0 (CTA 0 only unless prof_all)
     int prof_all;
     int poll_gap;                            // >= 0: the pollers of the chip-wide exchange start this many cycles after the CTA's own publication; < 0: at once
@@ -225,8 +226,9 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
-        st_relaxed_u64(p.slots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
-                       ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+        if (!(cta == p.skip_cta && s == p.skip_step))
+            st_relaxed_u64(p.slots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
+                           ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
         if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
     };
@@ -553,7 +555,7 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.frame_shift = a.row_lag > 0 ? a.step0 : 0;
     p.status = m->status;
-    p.limit_ns = 2000000000ull;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
     { const char *e = getenv("WRNN_POLL_GAP"); p.poll_gap = e ? atoi(e) : 150; }
     p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
     { const char *e = getenv("WRNN_PROF_ALL"); p.prof_all = (e && e[0] == '1') ? 1 : 0; }

@@ -77,6 +77,7 @@ struct MultiParams {
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
+    int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
     long long *prof;
     unsigned flag_mode;                      // bit 0 / 1: with one / several column groups the gather waits for this CTA's own publication first
 };
@@ -302,8 +303,9 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         const int jj = (half_g ? K : 0) + gj;
         // published as the operand the 112 readers need: bf16 high and low parts, split once here
         const __nv_bfloat16 hh = __float2bfloat16_rn(hn), hl = __float2bfloat16_rn(hn - __bfloat162float(hh));
-        st_relaxed_u64(p.slots + ((size_t)((half_g ? 2 : 0) + (s & 1)) * NS + gst) * K + gj,
-                       ((unsigned long long)(unsigned)(s + 1) << 32) | (unsigned)__bfloat16_as_ushort(hh) | ((unsigned)__bfloat16_as_ushort(hl) << 16));
+        if (!(cta == p.skip_cta && s == p.skip_step))
+            st_relaxed_u64(p.slots + ((size_t)((half_g ? 2 : 0) + (s & 1)) * NS + gst) * K + gj,
+                           ((unsigned long long)(unsigned)(s + 1) << 32) | (unsigned)__bfloat16_as_ushort(hh) | ((unsigned)__bfloat16_as_ushort(hl) << 16));
         if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * NS + gst) * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
         if (p.dbg_h) p.dbg_h[((size_t)s * NS + gst) * H + jj] = hn;
     };
@@ -788,7 +790,7 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
-    p.limit_ns = 2000000000ull;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
     p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
     { const char *d = getenv("WRNN_MULTI_FLAG"); p.flag_mode = d ? (unsigned)atoi(d) : 1u; }    // diagnostic: A/B of the gather protocol
 

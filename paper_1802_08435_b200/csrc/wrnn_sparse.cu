@@ -69,6 +69,7 @@ struct SparseParams {
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
+    int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
 };
 
 #ifdef WRNN_PROFILE_SPARSE
@@ -276,8 +277,9 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
             const float hn = fmaf(u, q.hprev, (1.0f - u) * e);
             // published to the whole chip: arrival of the tagged value is the signal (two-deep by step parity)
-            st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + cta * UC + u0,
-                           ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+            if (!(cta == p.skip_cta && s == p.skip_step))
+                st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + cta * UC + u0,
+                               ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
             const int jj = (half_g ? K : 0) + cta * UC + u0;
             if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
             if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
@@ -772,7 +774,7 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
-    p.limit_ns = 2000000000ull;
+    p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
 
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;

@@ -24,7 +24,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // bounded: false when the phase did not complete within about two seconds
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned long long limit_ns = TC_WAIT_NS)
 {
     unsigned long long t0 = 0;
     for (unsigned n = 1;; ++n) {
@@ -32,7 +32,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
         if ((n & 255u) == 0) {
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > TC_WAIT_NS) return false;
+            else if (now - t0 > limit_ns) return false;
         }
     }
 }

@@ -276,6 +276,77 @@ def test_bounded_wait_gives_up_cleanly(env):
         B.wrnn_destroy(m)
 
 
+@pytest.mark.parametrize("case", ["lean", "first-resident", "fused", "multi4", "multi16", "pair", "resf32", "sparse", "bcluster", "batched", "generic"])
+def test_lost_word_times_out_cleanly_in_every_kernel(env, case):
+    """The give-up paths of the sampling kernels themselves: one CTA withholds what it hands to the others at one step,
+    with every wait bounded by a few milliseconds.  The launch must return, the status must say WRNN_ERR_TIMEOUT with a
+    step at (or right after) the withheld one, and the same model must then sample exactly what it sampled before."""
+    torch, B = env
+    envset = {}
+    kw = {}
+    if case in ("lean", "first-resident", "multi4", "multi16", "pair"):
+        wl = synth.WORKLOADS[7]
+        batch = {"lean": 1, "first-resident": 1, "multi4": 4, "multi16": 16, "pair": 2}[case]
+        w, masks, cond = synth.build_workload(wl, batch=batch)
+        dtype, kern, n_ctas_min = wl.dtype, B.WRNN_KERNEL_AUTO, 100
+        if case == "first-resident":
+            envset["WRNN_RESIDENT_LEAN"] = "0"
+    elif case == "fused":
+        wl = synth.WORKLOADS[8]
+        w, masks, cond = synth.build_workload(wl)
+        batch, dtype, kern, n_ctas_min = 1, wl.dtype, B.WRNN_KERNEL_AUTO, 100
+        kw["variant"] = 1
+    elif case == "resf32":
+        w, masks, cond, batch, dtype, kern, n_ctas_min = _tiny(192), None, synth.make_cond(1, 12, 4), 1, "f32", B.WRNN_KERNEL_RESIDENT, 2
+    elif case == "sparse":
+        wl = synth.WORKLOADS[2]
+        w, masks, cond = synth.build_workload(wl)
+        batch, dtype, kern, n_ctas_min = 1, wl.dtype, B.WRNN_KERNEL_SPARSE, 16
+    else:
+        batch = 11 if case != "generic" else 3
+        w, masks, cond, dtype, n_ctas_min = _tiny(128), None, synth.make_cond(batch, 12, 4), "bf16", 2
+        kern = {"bcluster": B.WRNN_KERNEL_BCLUSTER, "batched": B.WRNN_KERNEL_BATCHED, "generic": B.WRNN_KERNEL_GENERIC}[case]
+    hop = 120 if cond.shape[2] == 64 else 10
+    n, k_step = 60, 23
+    for k_, v_ in envset.items():
+        os.environ[k_] = v_
+    m = B.wrnn_create(w, dtype, masks, max_batch=batch, kernel=kern, **kw)
+    try:
+        info = B.wrnn_launch_info(m, batch)
+        assert info["n_ctas"] >= n_ctas_min
+
+        def run():
+            if case == "fused":
+                out = torch.zeros((2, n), dtype=torch.int16, device="cuda:0")
+                B.wrnn_fs2_sample(m, torch.from_numpy(cond).cuda(), n, 5, out, hop=hop)
+            else:
+                out = torch.zeros((batch, n), dtype=torch.int16, device="cuda:0")
+                B.wrnn_sample(m, torch.from_numpy(cond).cuda(), n, batch, 5, out, hop=hop)
+            torch.cuda.synchronize()
+            return out.cpu().numpy()
+
+        ref = run()
+        assert B.wrnn_poll_status(m) == 0
+        victim = info["n_ctas"] // 2
+        B.wrnn_selftest_lost_word(m, 4_000_000, victim, k_step)
+        run()
+        assert B.wrnn_poll_status(m) == B.WRNN_ERR_TIMEOUT
+        msg = B.wrnn_last_error(m)
+        import re
+        got = re.search(r"at cta (-?\d+), step (-?\d+), phase (-?\d+)", msg)
+        assert got, msg
+        cta, step, phase = (int(x) for x in got.groups())
+        assert 0 <= cta < info["n_ctas"] and k_step <= step <= k_step + 1, msg
+        B.wrnn_selftest_lost_word(m, 0, -1, -1)
+        again = run()
+        assert B.wrnn_poll_status(m) == 0, B.wrnn_last_error(m)
+        assert np.array_equal(again, ref)
+    finally:
+        B.wrnn_destroy(m)
+        for k_ in envset:
+            os.environ.pop(k_, None)
+
+
 def test_fold_unfold_exact_permutation(env):
     torch, B = env
     for n, Bf in [(24000, 16), (16, 16), (35, 5), (7, 1)]:

@@ -148,3 +148,33 @@ def build_workload(wl: Workload, n_steps: Optional[int] = None, batch: Optional[
     b = wl.batch if batch is None else batch
     cond = make_cond(b, wl.n_frames)
     return w, masks, cond
+
+
+# Shape of the paper's conditioning network of the Subscale WaveRNN (Section 5.3): ten layers, kernel size 3, 384
+# convolution channels, 768 residual channels, five stages of increasing dilation.
+NET_DILATIONS = (1, 1, 2, 2, 4, 4, 8, 8, 16, 16)
+NET_CONV_CH = 384
+NET_RES_CH = 768
+
+
+def make_subscale_net(B: int, cond_dim: int = COND_DIM, conv_ch: int = NET_CONV_CH, res_ch: int = NET_RES_CH,
+                      dilations=NET_DILATIONS, taps: int = 3, seed: int = 418) -> Dict[str, np.ndarray]:
+    """Synthetic weights of the masked dilated conditioning network (the trained ones do not exist here): every matrix
+    i.i.d. normal, scaled so that activations stay of order one through the residual stack (the residual branch of a
+    layer adds about 0.3 rms); small biases.  fp32, row-major:
+        W_in [res][B], b_in [res]; W_conv [layers][taps][conv][res], b_conv [layers][conv];
+        W_res [layers][res][conv], b_res [layers][res]; W_out [cond_dim][res], b_out [cond_dim]; dilation int32 [layers].
+    """
+    rng = np.random.default_rng(seed)
+    nl = len(dilations)
+
+    def mat(scale, *shape):
+        return (rng.standard_normal(shape) * scale).astype(np.float32)
+
+    return {
+        "dilation": np.asarray(dilations, np.int32),
+        "W_in": mat(1.0 / np.sqrt(max(B - 1, 1) / 3.0), res_ch, B), "b_in": mat(0.1, res_ch),
+        "W_conv": mat(1.0 / np.sqrt(taps * res_ch), nl, taps, conv_ch, res_ch), "b_conv": mat(0.1, nl, conv_ch),
+        "W_res": mat(0.5 / np.sqrt(conv_ch), nl, res_ch, conv_ch), "b_res": mat(0.02, nl, res_ch),
+        "W_out": mat(1.5 / np.sqrt(res_ch), cond_dim, res_ch), "b_out": mat(0.1, cond_dim),
+    }

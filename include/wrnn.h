@@ -239,6 +239,45 @@ int wrnn_subscale_conditioning(const int16_t *hist, const float *frames, const f
 int wrnn_subscale_schedule(int32_t B, int64_t L, int32_t chunk, int32_t lag, int64_t *calls, int32_t max_calls);
 
 /*
+ * The conditioning network of the Subscale WaveRNN with the shape the paper states (Section 5.3: a masked dilated 1-D CNN,
+ * ten layers, kernels of size 3, 384 convolution channels, 768 residual channels, five stages of increasing dilation, a
+ * future horizon of F = 128 positions; Section 4.1: relus, the mask over the past connections).  The paper prints no
+ * equations for it; the reading built here (sub-tensor s, position i, x(u) = u / 32768):
+ *     X[i][z]    = x(u_{B i + z}) for z < s, 0 otherwise            block input, masked to the earlier sub-tensors
+ *     x_0[i]     = W_in X[i] + b_in
+ *     a_l[i]     = relu(b_conv[l] + sum_{t < taps} W_conv[l][t] x_l[i + t dilation[l]])      forward connections only
+ *     x_{l+1}[i] = x_l[i] + W_res[l] a_l[i] + b_res[l]
+ *     v_s[i]     = frames[s][(B i + s) div hop] + W_out relu(x_last[i]) + b_out
+ * positions at or beyond the row length hold the zero vector in every layer; the reach of the network is
+ * (taps - 1) * sum of the dilations (124 for 1,1,2,2,4,4,8,8,16,16).  All pointers HOST fp32 row-major, read during the
+ * call; the matrices are rounded to bf16 (nearest even), biases stay fp32:
+ *     W_in [res_ch][B], b_in [res_ch]; W_conv [n_layers][taps][conv_ch][res_ch], b_conv [n_layers][conv_ch];
+ *     W_res [n_layers][res_ch][conv_ch], b_res [n_layers][res_ch]; W_out [cond_dim][res_ch], b_out [cond_dim].
+ * The products run on the tensor cores (tiles of 128 positions): conv_ch must be a multiple of 192, res_ch of 128,
+ * B <= 64, cond_dim <= 64, every dilation <= 64; other shapes return WRNN_ERR_UNSUPPORTED.
+ */
+typedef struct wrnn_subscale_net wrnn_subscale_net;     /* opaque; owns its device memory */
+typedef struct {
+    int32_t B, n_layers, taps, conv_ch, res_ch, cond_dim;
+    const int32_t *dilation;                            /* HOST [n_layers] */
+    const float *W_in, *b_in, *W_conv, *b_conv, *W_res, *b_res, *W_out, *b_out;
+} wrnn_subscale_net_params;
+int wrnn_subscale_net_create(const wrnn_subscale_net_params *params, wrnn_subscale_net **out);    /* synchronous; current device */
+void wrnn_subscale_net_destroy(wrnn_subscale_net *net);                                            /* NULL allowed */
+/* v (DEVICE [L][cond_dim]) = conditioning vectors of sub-tensor `row` at all L positions from the history hist (DEVICE int16
+ * [B][L]); frames DEVICE [B][n_frames][cond_dim].  Asynchronous on cuda_stream; may grow the network's activation buffers
+ * (synchronously).  wrnn_subscale_net_status, after synchronising: WRNN_OK, or WRNN_ERR_TIMEOUT when a bounded wait of the
+ * tensor pipeline ran out. */
+int wrnn_subscale_net_conditioning(wrnn_subscale_net *net, const int16_t *hist, const float *frames, int32_t n_frames, int32_t hop,
+                                   int32_t row, int64_t L, float *v, void *cuda_stream);
+int wrnn_subscale_net_status(wrnn_subscale_net *net);
+/* wrnn_sample_subscale_dependent with this network in place of the one-layer convolution: B = the network's B; F >= the
+ * network's reach; lag a multiple of chunk and >= F + chunk.  Per chunk the network is evaluated for chunk + reach positions
+ * of every active row (the positions ahead are recomputed by the next chunk).  Asynchronous on cuda_stream. */
+int wrnn_sample_subscale_net(wrnn_model *m, wrnn_subscale_net *net, const float *frames, int32_t n_frames, int32_t hop, int32_t F,
+                             int32_t chunk, int32_t lag, int64_t n_total, uint64_t seed, int16_t *out, void *cuda_stream);
+
+/*
  * Host-buffer convenience for callers without device pointers: copies cond
  * (HOST [batch][n_frames][cond_dim]) to the device, runs wrnn_sample from the
  * default state and copies the samples back to out (HOST int16 [batch][n_steps]).

@@ -28,6 +28,7 @@ EXPORTS = [
     "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_phase_profile", "wrnn_phase_names", "wrnn_measure_exchange_floor", "wrnn_measure_smem_stream", "wrnn_sample_noalloc",
     "wrnn_selftest_bounded_wait", "wrnn_selftest_lost_word", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold", "wrnn_fs2_sample_host",
     "wrnn_sample_subscale_dependent", "wrnn_subscale_conditioning", "wrnn_subscale_schedule",
+    "wrnn_subscale_net_create", "wrnn_subscale_net_destroy", "wrnn_subscale_net_conditioning", "wrnn_subscale_net_status", "wrnn_sample_subscale_net",
 ]
 
 
@@ -103,6 +104,12 @@ def lib():
         L.wrnn_measure_smem_stream.argtypes = [i32, i32, i32, i32, vp]
         L.wrnn_selftest_bounded_wait.argtypes = [i64] + [vp] * 5
         L.wrnn_selftest_lost_word.argtypes = [vp, i64, i32, i64]
+        L.wrnn_subscale_net_create.argtypes = [vp, vp]
+        L.wrnn_subscale_net_destroy.argtypes = [vp]
+        L.wrnn_subscale_net_destroy.restype = None
+        L.wrnn_subscale_net_conditioning.argtypes = [vp, vp, vp, i32, i32, i32, i64, vp, vp]
+        L.wrnn_subscale_net_status.argtypes = [vp]
+        L.wrnn_sample_subscale_net.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i64, C.c_uint64, vp, vp]
         L.wrnn_launch_count.argtypes = []
         L.wrnn_launch_count.restype = i64
         _lib = L
@@ -256,6 +263,46 @@ def wrnn_sample_subscale_dependent(model, frames, V, bias, F: int, chunk: int, l
     V: CUDA float32 [B-1][F+1][D]; bias: CUDA float32 [D]; out: CUDA int16 [n_total] in the original order."""
     _check(lib().wrnn_sample_subscale_dependent(model, _dev_ptr(frames), int(frames.shape[1]), hop, _dev_ptr(V), _dev_ptr(bias), F,
                                                 chunk, lag, n_total, B, seed, _dev_ptr(out), _stream_ptr(stream)), model)
+
+
+class wrnn_subscale_net_params(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("B", "n_layers", "taps", "conv_ch", "res_ch", "cond_dim")] + \
+               [(n, C.c_void_p) for n in ("dilation", "W_in", "b_in", "W_conv", "b_conv", "W_res", "b_res", "W_out", "b_out")]
+
+
+def wrnn_subscale_net_create(w: Dict[str, np.ndarray]):
+    """The conditioning network of the Subscale WaveRNN from a dict of fp32 numpy arrays: dilation int32 [layers], W_in
+    [res][B], b_in, W_conv [layers][taps][conv][res], b_conv, W_res [layers][res][conv], b_res, W_out [D][res], b_out.
+    Returns an opaque handle."""
+    keep = {k: np.ascontiguousarray(w[k], dtype=np.int32 if k == "dilation" else np.float32) for k in
+            ("dilation", "W_in", "b_in", "W_conv", "b_conv", "W_res", "b_res", "W_out", "b_out")}
+    nl, taps, conv, res = keep["W_conv"].shape
+    p = wrnn_subscale_net_params(int(keep["W_in"].shape[1]), int(nl), int(taps), int(conv), int(res), int(keep["W_out"].shape[0]),
+                                 *[_np_ptr(keep[k]) for k in ("dilation", "W_in", "b_in", "W_conv", "b_conv", "W_res", "b_res", "W_out", "b_out")])
+    out = C.c_void_p()
+    _check(lib().wrnn_subscale_net_create(C.byref(p), C.byref(out)))
+    return out
+
+
+def wrnn_subscale_net_destroy(net) -> None:
+    lib().wrnn_subscale_net_destroy(net)
+
+
+def wrnn_subscale_net_conditioning(net, hist, frames, row: int, v, *, hop: int = 120, stream=None):
+    """v (CUDA float32 [L][D]) = conditioning vectors of sub-tensor `row` from the history hist (CUDA int16 [B][L])."""
+    _check(lib().wrnn_subscale_net_conditioning(net, _dev_ptr(hist), _dev_ptr(frames), int(frames.shape[1]), hop, row, int(hist.shape[1]),
+                                                _dev_ptr(v), _stream_ptr(stream)))
+
+
+def wrnn_subscale_net_status(net) -> int:
+    return lib().wrnn_subscale_net_status(net)
+
+
+def wrnn_sample_subscale_net(model, net, frames, F: int, chunk: int, lag: int, n_total: int, seed: int, out, *, hop: int = 120, stream=None):
+    """Subscale generation with dependent rows on the staggered schedule, conditioned through the masked dilated network.
+    frames: CUDA float32 [B][n_frames][D]; out: CUDA int16 [n_total] in the original order."""
+    _check(lib().wrnn_sample_subscale_net(model, net, _dev_ptr(frames), int(frames.shape[1]), hop, F, chunk, lag, n_total, seed, _dev_ptr(out),
+                                          _stream_ptr(stream)), model)
 
 
 def wrnn_subscale_schedule(B: int, L: int, chunk: int, lag: int):

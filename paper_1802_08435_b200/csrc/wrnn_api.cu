@@ -589,23 +589,27 @@ int wrnn_subscale_conditioning(const int16_t *hist, const float *frames, const f
     return subscale_cond_launch(hist, frames, V, bias, v, B, L, F, cond_dim, n_frames, hop, row, 1, 0, 0, (int)L, (cudaStream_t)cuda_stream);
 }
 
-int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n_frames, int32_t hop, const float *V, const float *bias,
-                                   int32_t F, int32_t chunk, int32_t lag, int64_t n_total, int32_t B, uint64_t seed, int16_t *out,
-                                   void *cuda_stream)
+}  // extern "C"
+
+namespace wrnn {
+// Subscale generation with dependent rows on the staggered schedule, whatever the conditioning network: `cond_rows`
+// computes the conditioning vectors v[n_rows][n][D] of one stepping call (rows r_a .. r_a + n_rows - 1, row b of the call
+// from position p_lo - b * lag on) from the sample history hist [B][L].
+template <typename CondFn>
+static int subscale_dependent_impl(wrnn_model *m, int32_t n_frames, int32_t hop, int32_t F, int32_t chunk, int32_t lag, int64_t n_total, int32_t B,
+                                   uint64_t seed, int16_t *out, cudaStream_t s, CondFn cond_rows)
 {
-    if (!m) return WRNN_ERR_INVALID_ARG;
     if (m->variant != 0) return fail(m, WRNN_ERR_UNSUPPORTED, "subscale generation takes a WaveRNN model (variant 0)");
     if (m->cond_dim <= 0) return fail(m, WRNN_ERR_INVALID_ARG, "the model must be conditioned");
     if (B < 1 || B > m->max_batch || n_total < 0 || n_total % B != 0) return fail(m, WRNN_ERR_INVALID_ARG, "B must divide n_total and fit max_batch");
     if (n_total == 0) return WRNN_OK;
-    if (!frames || !V || !bias || !out || hop < 1 || F < 0 || chunk < 1) return fail(m, WRNN_ERR_INVALID_ARG, "bad arguments");
+    if (!out || hop < 1 || F < 0 || chunk < 1) return fail(m, WRNN_ERR_INVALID_ARG, "bad arguments");
     // row r + 1 may use positions of row r up to F ahead of its own, for a whole chunk at a time: it follows F + chunk
     // steps (or more) behind; chunks of all rows line up when the lag is a multiple of the chunk
     if (lag < F + chunk || lag % chunk != 0) return fail(m, WRNN_ERR_INVALID_ARG, "lag must be a multiple of chunk and at least F + chunk");
     const long long L = n_total / B;
     if (((long long)B * (L - 1) + (B - 1)) / hop >= n_frames) return fail(m, WRNN_ERR_INVALID_ARG, "conditioning frames run out");
     if (cudaSetDevice(m->device) != cudaSuccess) return fail(m, WRNN_ERR_CUDA, "cudaSetDevice failed");
-    cudaStream_t s = (cudaStream_t)cuda_stream;
     const int D = m->cond_dim, H = m->H;
     // scratch: sample history [B][L], per-call conditioning [B][chunk][D], carry state
     const size_t need = (size_t)B * L * sizeof(int16_t) + (size_t)B * chunk * D * sizeof(float) + (size_t)B * H * sizeof(float) + 2 * (size_t)B + 64;
@@ -625,11 +629,10 @@ int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n
         return fail(m, WRNN_ERR_CUDA, "scratch initialisation failed");
 
     auto run_rows = [&](int r_a, int n_rows, long long p_lo, int n) -> int {
-        int rc = subscale_cond_launch(hist, frames, V, bias, v, B, L, F, D, n_frames, hop, r_a, n_rows, p_lo, lag, n, s);
+        int rc = cond_rows(hist, v, L, r_a, n_rows, p_lo, n);
         if (rc != WRNN_OK) return fail(m, rc, "conditioning launch failed");
-        // rows advance together on the multi-stream resident kernel where the model has one (8.3 us per step at two rows
-        // against 6.4 us per step and row on the single-stream kernel); without it up to three rows go one after the other
-        // through the single-stream kernel (24 us per step of the cluster-partitioned kernel whatever the rows)
+        // rows advance together on the multi-stream resident kernel where the model has one; without it up to three rows go
+        // one after the other through the single-stream kernel
         const int group = (n_rows >= 2 && use_multi(m, n_rows)) ? n_rows : (n_rows <= 3 && (use_reslean(m, 1) || use_resident(m, 1))) ? 1 : n_rows;
         for (int b0 = 0; b0 < n_rows; b0 += group) {
             const int r0 = r_a + b0;
@@ -654,6 +657,38 @@ int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n
         if (rc != WRNN_OK) return rc;
     }
     return fold_launch(hist, n_total, B, out, true, s);
+}
+}  // namespace wrnn
+
+extern "C" {
+
+int wrnn_sample_subscale_dependent(wrnn_model *m, const float *frames, int32_t n_frames, int32_t hop, const float *V, const float *bias,
+                                   int32_t F, int32_t chunk, int32_t lag, int64_t n_total, int32_t B, uint64_t seed, int16_t *out,
+                                   void *cuda_stream)
+{
+    if (!m) return WRNN_ERR_INVALID_ARG;
+    if (n_total > 0 && (!frames || !V || !bias)) return fail(m, WRNN_ERR_INVALID_ARG, "bad arguments");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const int D = m->cond_dim;
+    return subscale_dependent_impl(m, n_frames, hop, F, chunk, lag, n_total, B, seed, out, s,
+                                   [&](const int16_t *hist, float *v, long long L, int r_a, int n_rows, long long p_lo, int n) {
+                                       return subscale_cond_launch(hist, frames, V, bias, v, B, L, F, D, n_frames, hop, r_a, n_rows, p_lo, lag, n, s);
+                                   });
+}
+
+int wrnn_sample_subscale_net(wrnn_model *m, wrnn_subscale_net *net, const float *frames, int32_t n_frames, int32_t hop, int32_t F, int32_t chunk,
+                             int32_t lag, int64_t n_total, uint64_t seed, int16_t *out, void *cuda_stream)
+{
+    if (!m || !net) return WRNN_ERR_INVALID_ARG;
+    if (n_total > 0 && !frames) return fail(m, WRNN_ERR_INVALID_ARG, "bad arguments");
+    if (subnet_cond_dim(net) != m->cond_dim) return fail(m, WRNN_ERR_INVALID_ARG, "the network's output does not match the model's conditioning size");
+    if (F < subnet_reach(net)) return fail(m, WRNN_ERR_INVALID_ARG, "the future horizon F is shorter than the reach of the network");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const int B = subnet_B(net);
+    return subscale_dependent_impl(m, n_frames, hop, F, chunk, lag, n_total, B, seed, out, s,
+                                   [&](const int16_t *hist, float *v, long long L, int r_a, int n_rows, long long p_lo, int n) {
+                                       return subnet_run(net, hist, frames, n_frames, hop, L, r_a, n_rows, p_lo, lag, n, v, m->wait_limit_ns(), s);
+                                   });
 }
 
 int wrnn_sample_host(wrnn_model *m, const float *cond_host, int32_t n_frames, int32_t hop, int32_t row_stride,

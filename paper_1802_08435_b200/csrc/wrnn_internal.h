@@ -67,6 +67,8 @@ struct BcPack;         // per-CTA weight slices and stacked activation images of
 
 }  // namespace wrnn
 
+struct wrnn_subscale_net;   // the conditioning network of the Subscale WaveRNN (wrnn_subnet.cu)
+
 struct wrnn_model {
     int H = 0, cond_dim = 0, dtype = 0, kernel = 0, max_batch = 0;
     int variant = 0;                // 0: WaveRNN (Eq. 2); 1: Fused Subscale WaveRNN 2x (I has 12 columns, O2 / O4 64 rows)
@@ -136,6 +138,13 @@ int fold_launch(const int16_t *x, long long n_total, int B, int16_t *sub, bool u
 int fs2_unfold_launch(const int16_t *ab, long long n, int16_t *u, cudaStream_t s);
 int subscale_cond_launch(const int16_t *hist, const float *frames, const float *V, const float *bias, float *v, int B, long long L, int F,
                          int D, int n_frames, int hop, int r_lo, int n_rows, long long p_lo, int lag, int n_steps, cudaStream_t s);
+
+// wrnn_subnet.cu: the masked dilated conditioning network on the tensor cores, for the segments of one stepping call
+int subnet_run(wrnn_subscale_net *n, const int16_t *hist, const float *frames, int n_frames, int hop, long long L, int r_lo, int n_rows,
+               long long p_lo, int lag, int n_steps, float *v, unsigned long long limit_ns, cudaStream_t s);
+int subnet_reach(const wrnn_subscale_net *n);
+int subnet_B(const wrnn_subscale_net *n);
+int subnet_cond_dim(const wrnn_subscale_net *n);
 
 // wrnn_resident.cu
 int resident_supported(const wrnn_model *m, int batch, std::string *why);

@@ -138,6 +138,11 @@ def oracle_runner(orc, wl, w, masks, cond, threads):
     if wl.variant == 1:
         om = orc.Fs2OracleModel(w, wl.dtype)
         return lambda n: om.run(cond[0], n, seed=synth.SEED_SAMPLING, hop=synth.HOP)
+    if wl.dependent and wl.net:
+        from oracle import subscale_net as sn
+        om = orc.OracleModel(w, wl.dtype)
+        net = sn.SubscaleNet(synth.make_subscale_net(wl.batch))
+        return lambda n: sn.subscale_net_run(om, net, cond, n, synth.HOP, synth.SEED_SAMPLING)
     if wl.dependent:
         om = orc.OracleModel(w, wl.dtype)
         V, b = synth.make_subscale_conv(wl.batch, wl.dependent[0])
@@ -279,6 +284,7 @@ def measure(ctx, wl, *, steps, warmup, kernel, n_steps=None, e2e=True, cpu_budge
     n_steps = wl.n_steps if n_steps is None else n_steps
     w, masks, cond_np = synth.build_workload(wl)
     model = B.wrnn_create(w, wl.dtype, masks, max_batch=wl.batch, kernel=kernel, block=wl.block, variant=wl.variant)
+    net = None
     try:
         info = B.wrnn_launch_info(model, wl.batch)
         cond = torch.from_numpy(cond_np).to(dev)
@@ -295,9 +301,13 @@ def measure(ctx, wl, *, steps, warmup, kernel, n_steps=None, e2e=True, cpu_budge
             Vn, bn = synth.make_subscale_conv(wl.batch, dep[0])
             V_d, b_d = torch.from_numpy(Vn).to(dev), torch.from_numpy(bn).to(dev)
             out = torch.zeros((wl.batch * n_steps,), dtype=torch.int16, device=dev)
+            if wl.net:
+                net = B.wrnn_subscale_net_create(synth.make_subscale_net(wl.batch))
 
         def one():
-            if dep:
+            if net is not None:
+                B.wrnn_sample_subscale_net(model, net, cond, dep[0], dep[1], dep[2], wl.batch * n_steps, seed, out, hop=synth.HOP)
+            elif dep:
                 B.wrnn_sample_subscale_dependent(model, cond, V_d, b_d, dep[0], dep[1], dep[2], wl.batch * n_steps, wl.batch, seed, out, hop=synth.HOP)
             elif fused:
                 B.wrnn_fs2_sample(model, cond, n_steps, seed, out, hop=synth.HOP)
@@ -385,6 +395,8 @@ def measure(ctx, wl, *, steps, warmup, kernel, n_steps=None, e2e=True, cpu_budge
                 res["cpu_baseline"] = cpu_baseline(wl, cpu_budget_s)
         return res
     finally:
+        if net is not None:
+            B.wrnn_subscale_net_destroy(net)
         B.wrnn_destroy(model)
 
 

@@ -115,6 +115,7 @@ class Workload:
     block: tuple = (4, 4)     # shape of one block of the sparsity masks (rows, columns)
     variant: int = 0          # 1: Fused Subscale WaveRNN 2x (two samples per step)
     dependent: Optional[tuple] = None   # (F, chunk, lag): subscale rows conditioned on the earlier rows, staggered schedule
+    net: bool = False         # dependent rows conditioned through the ten-layer masked dilated network (else one convolution)
 
 
 # The five named workloads (index = position in the benchmark's config list), then three extra ones.
@@ -135,6 +136,9 @@ WORKLOADS = [
     # rows 256 steps apart (the batch is full after 15 x 256 of the 9,840 global steps)
     Workload("subscale16_dependent_896_bf16_6000", 896, "bf16", 16, 6000, 802, row_stride=16, row_offset_mul=1, subscale_B=16,
              dependent=(128, 128, 256)),
+    # the same through the conditioning network with the paper's shape (Section 5.3)
+    Workload("subscale16_net_896_bf16_6000", 896, "bf16", 16, 6000, 802, row_stride=16, row_offset_mul=1, subscale_B=16,
+             dependent=(128, 128, 256), net=True),
 ]
 
 

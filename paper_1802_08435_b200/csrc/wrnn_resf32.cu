@@ -181,6 +181,7 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
     };
     // Gates of Eq. 2 for this CTA's units of one half of the state, then publish them to the chip.
     // half_g = 0: coarse units (c_s does not reach them: their I* column is zero), 1: fine units.
+    const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
         const float xk = scale8(drawn);                  // the pending input
         const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
@@ -188,7 +189,7 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
-        if (!(cta == p.skip_cta && s == p.skip_step))
+        if ((int)s != skip_at)
             st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
                            ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }

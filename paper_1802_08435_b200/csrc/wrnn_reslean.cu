@@ -143,9 +143,9 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
     bool my_bad = false;
     const bool prof_on = p.prof != nullptr && (cta == 0 || p.prof_all) && warp == 0;
     __shared__ long long s_prof[16];
-    __shared__ unsigned pub_flag;            // last half-step whose state values this CTA's gate threads have published
+    __shared__ __align__(8) unsigned long long pub_bar;      // one arrival per half-step: this CTA's gate threads have published
     if (tid < 16) s_prof[tid] = 0;
-    if (tid == 0) pub_flag = 0;
+    if (tid == 0) { mbar_init_cluster(smem_addr(&pub_bar), 1); mbar_fence_init(); }
     __syncthreads();
     long long prof_t = clock64();
 #define STAMP(i) do { if (prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
@@ -219,6 +219,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
         return q;
     };
+    const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
         const float xk = scale8(drawn);
         const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
@@ -226,7 +227,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
-        if (!(cta == p.skip_cta && s == p.skip_step))
+        if ((int)s != skip_at)
             st_relaxed_u64(p.slots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
                            ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
@@ -243,6 +244,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         load_g(0, 0, gv);
         gates_and_publish(0, 0, f_prev, gates_prepare(0, gv));
     }
+    if (tid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&pub_bar)) : "memory");
 
     // Half-step n = 2 s + 1 is the coarse half of step s (input y_c(s): coarse head -> c_s, then the fine gates of step s),
     // n = 2 s the fine half (input y_f(s - 1): fine head -> f_{s-1}, R h_{s-1} completed, then the coarse gates of step s).
@@ -287,12 +289,10 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
                     // and a poll that just misses the data costs a whole round trip.  The pollers therefore hold back
                     // until this CTA's own gate threads have published (all CTAs publish at about the same time), plus
                     // poll_gap cycles, so that their first poll reaches L2 when the words do.
-                    unsigned seen;
-                    while (true) {
-                        asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(seen) : "r"(smem_addr(&pub_flag)) : "memory");
-                        if (seen + 1u >= (unsigned)n) break;
-                        if ((++cnt & 65535u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
-                    }
+                    // (waiting on an mbarrier parks the thread in hardware; a spin on a shared-memory word takes issue slots from
+                    // the warp that draws)
+                    while (!mbar_try_parity(smem_addr(&pub_bar), (unsigned)((n - 1) & 1)))
+                        if ((++cnt & 1023u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
                     const long long c0 = clock64();
                     while (clock64() - c0 < p.poll_gap) { }
                     cnt = 0; t0 = 0;
@@ -383,7 +383,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
             const int drawn = warp_softmax_draw_fast(l, u01, lane);
             const int fed = forced >= 0 ? forced : drawn;
             if (lane < UC && !last && !my_bad) gates_and_publish(half, s, fed, gp);
-            if (lane == 0) asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_addr(&pub_flag)), "r"((unsigned)n) : "memory");
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&pub_bar)) : "memory");
             if (writer) {
                 if (p.dbg_logits) {
                     float *d = p.dbg_logits + (size_t)(n - 1) * RL_NLOG + 8 * lane;
@@ -556,7 +556,7 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.frame_shift = a.row_lag > 0 ? a.step0 : 0;
     p.status = m->status;
     p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
-    { const char *e = getenv("WRNN_POLL_GAP"); p.poll_gap = e ? atoi(e) : 150; }
+    { const char *e = getenv("WRNN_POLL_GAP"); p.poll_gap = e ? atoi(e) : 100; }
     p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
     { const char *e = getenv("WRNN_PROF_ALL"); p.prof_all = (e && e[0] == '1') ? 1 : 0; }
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * RL_K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;

@@ -294,6 +294,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
         return q;
     };
+    const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
         const float xk = scale8(drawn);
         const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
@@ -303,7 +304,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         const int jj = (half_g ? K : 0) + gj;
         // published as the operand the 112 readers need: bf16 high and low parts, split once here
         const __nv_bfloat16 hh = __float2bfloat16_rn(hn), hl = __float2bfloat16_rn(hn - __bfloat162float(hh));
-        if (!(cta == p.skip_cta && s == p.skip_step))
+        if ((int)s != skip_at)
             st_relaxed_u64(p.slots + ((size_t)((half_g ? 2 : 0) + (s & 1)) * NS + gst) * K + gj,
                            ((unsigned long long)(unsigned)(s + 1) << 32) | (unsigned)__bfloat16_as_ushort(hh) | ((unsigned)__bfloat16_as_ushort(hl) << 16));
         if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * NS + gst) * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }

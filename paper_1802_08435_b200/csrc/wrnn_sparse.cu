@@ -269,6 +269,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         }
         return q;
     };
+    const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
     auto gates = [&](int half_g, long long s, int drawn, const GatePre &q) {
         if (lane < UW) {
             const int u0 = warp * UW + lane;
@@ -277,7 +278,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
             const float hn = fmaf(u, q.hprev, (1.0f - u) * e);
             // published to the whole chip: arrival of the tagged value is the signal (two-deep by step parity)
-            if (!(cta == p.skip_cta && s == p.skip_step))
+            if ((int)s != skip_at)
                 st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + cta * UC + u0,
                                ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
             const int jj = (half_g ? K : 0) + cta * UC + u0;

@@ -4,6 +4,7 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <cstdlib>
 #include <string>
 #include <vector>
 
@@ -125,6 +126,18 @@ struct wrnn_model {
 namespace wrnn {
 
 extern std::atomic<long long> g_launches;
+
+// Whether the persistent cluster kernels are launched with the cooperative attribute (the driver then refuses the launch
+// unless all clusters can be co-resident).  Co-residency is checked against the occupancy API when a model is created, so
+// the attribute is a second line of defence; it is dropped under WRNN_NO_COOP=1 and when a CUDA injection library is
+// loaded into the process (a profiler: kernel replay does not accept cooperative cluster launches).
+inline bool coop_launch_allowed()
+{
+    const char *no_coop = getenv("WRNN_NO_COOP");
+    if (no_coop && no_coop[0] == '1') return false;
+    const char *inj = getenv("CUDA_INJECTION64_PATH");
+    return !(inj && inj[0]);
+}
 
 // wrnn_api.cu: argument checks shared by the stepping entry points (fills the cond / state part of StepArgs)
 int check_step(wrnn_model *m, const wrnn_cond *cond, int64_t n_steps, int32_t batch, const wrnn_state *st, StepArgs *a);

@@ -524,8 +524,7 @@ int resf32_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     // The cooperative attribute makes the driver refuse the launch unless all clusters can be co-resident.
     // WRNN_NO_COOP=1 drops it (co-residency was already checked against the occupancy API at create):
     // a profiler that replays kernels may not accept cooperative cluster launches.
-    const char *no_coop = getenv("WRNN_NO_COOP");
-    fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
+    fill_launch(k, &cfg, at, s, coop_launch_allowed());
     const cudaError_t e = cudaLaunchKernelEx(&cfg, resident_f32_kernel, p);
     if (e != cudaSuccess) {
         m->err = std::string("fp32 resident kernel launch failed: ") + cudaGetErrorString(e);

@@ -1179,8 +1179,7 @@ int resident_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     // The cooperative attribute makes the driver refuse the launch unless all clusters can be co-resident.
     // WRNN_NO_COOP=1 drops it (co-residency was already checked against the occupancy API at create):
     // a profiler that replays kernels may not accept cooperative cluster launches.
-    const char *no_coop = getenv("WRNN_NO_COOP");
-    fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
+    fill_launch(k, &cfg, at, s, coop_launch_allowed());
     cudaError_t e = k.fused ? cudaLaunchKernelEx(&cfg, resident_dense_kernel<7, 4, 7, 4, true>, p)
                             : cudaLaunchKernelEx(&cfg, resident_dense_kernel<7, 4, 7, 4, false>, p);
     if (e != cudaSuccess) {
@@ -1238,8 +1237,7 @@ int resident_pair_run(wrnn_model *m, const StepArgs &a, int pair, cudaStream_t s
     if (cudaMemsetAsync(k.d_slots2, 0, (size_t)8 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (pair == 0 && cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
-    const char *no_coop = getenv("WRNN_NO_COOP");
-    fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
+    fill_launch(k, &cfg, at, s, coop_launch_allowed());
     cfg.dynamicSmemBytes = k.pair_smem;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, resident_pair_kernel, pp);
     if (e != cudaSuccess) {

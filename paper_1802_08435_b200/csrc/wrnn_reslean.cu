@@ -562,8 +562,7 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * RL_K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
-    const char *no_coop = getenv("WRNN_NO_COOP");
-    fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
+    fill_launch(k, &cfg, at, s, coop_launch_allowed());
     const cudaError_t e = cudaLaunchKernelEx(&cfg, resident_lean_kernel, p);
     if (e != cudaSuccess) {
         m->err = std::string("lean resident kernel launch failed: ") + cudaGetErrorString(e);

@@ -799,8 +799,7 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(k.d_aslots, 0, (size_t)2 * MAXS * 6 * MK * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
-    const char *no_coop = getenv("WRNN_NO_COOP");
-    multi_fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
+    multi_fill_launch(k, &cfg, at, s, coop_launch_allowed());
     const cudaError_t e = cudaLaunchKernelEx(&cfg, resident_multi_kernel, p);
     if (e != cudaSuccess) {
         m->err = std::string("multi-stream resident kernel launch failed: ") + cudaGetErrorString(e);

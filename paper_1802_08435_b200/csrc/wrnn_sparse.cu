@@ -780,8 +780,7 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
-    const char *no_coop = getenv("WRNN_NO_COOP");
-    sparse_fill_launch(k, &cfg, at, s, !(no_coop && no_coop[0] == '1'));
+    sparse_fill_launch(k, &cfg, at, s, coop_launch_allowed());
     cudaError_t e = cudaLaunchKernelEx(&cfg, sparse_cluster_kernel<8>, p);
     if (e != cudaSuccess) {
         m->err = std::string("sparse cluster kernel launch failed: ") + cudaGetErrorString(e);

@@ -277,6 +277,17 @@ int wrnn_subscale_net_status(wrnn_subscale_net *net);
 int wrnn_sample_subscale_net(wrnn_model *m, wrnn_subscale_net *net, const float *frames, int32_t n_frames, int32_t hop, int32_t F,
                              int32_t chunk, int32_t lag, int64_t n_total, uint64_t seed, int16_t *out, void *cuda_stream);
 
+/* One stepping call of the staggered schedule on caller-owned buffers: rows r_lo .. r_lo + n_rows - 1 of the B sub-tensors
+ * advance n_steps positions, row b of the call from position p_lo - b * lag on (the unit wrnn_sample_subscale_net is made of,
+ * exposed so that the sub-tensors can be spread over several devices, each generating some rows and passing the samples on one
+ * way, online: Section 5.3's closing paragraph).  hist: DEVICE int16 [B][L], read for the rows below r_lo + n_rows (positions up
+ * to F ahead must be there) and written in place for the rows of the call; h [B][H], c_prev / f_prev [B]: DEVICE carry state
+ * of all rows, read and written for the rows of the call (start from h = 0, c_prev = 128, f_prev = 0).  n_rows <= max_batch.
+ * Asynchronous on cuda_stream. */
+int wrnn_subscale_net_rows(wrnn_model *m, wrnn_subscale_net *net, const float *frames, int32_t n_frames, int32_t hop, int32_t lag, int16_t *hist,
+                           int64_t L, float *h, uint8_t *c_prev, uint8_t *f_prev, int32_t r_lo, int32_t n_rows, int64_t p_lo, int32_t n_steps,
+                           uint64_t seed, void *cuda_stream);
+
 /*
  * Host-buffer convenience for callers without device pointers: copies cond
  * (HOST [batch][n_frames][cond_dim]) to the device, runs wrnn_sample from the

@@ -28,7 +28,7 @@ EXPORTS = [
     "wrnn_launch_count", "wrnn_phase_cycles", "wrnn_phase_profile", "wrnn_phase_names", "wrnn_measure_exchange_floor", "wrnn_measure_smem_stream", "wrnn_sample_noalloc",
     "wrnn_selftest_bounded_wait", "wrnn_selftest_lost_word", "wrnn_fs2_sample", "wrnn_fs2_step_teacher_forced", "wrnn_fs2_unfold", "wrnn_fs2_sample_host",
     "wrnn_sample_subscale_dependent", "wrnn_subscale_conditioning", "wrnn_subscale_schedule",
-    "wrnn_subscale_net_create", "wrnn_subscale_net_destroy", "wrnn_subscale_net_conditioning", "wrnn_subscale_net_status", "wrnn_sample_subscale_net",
+    "wrnn_subscale_net_create", "wrnn_subscale_net_destroy", "wrnn_subscale_net_conditioning", "wrnn_subscale_net_status", "wrnn_sample_subscale_net", "wrnn_subscale_net_rows",
 ]
 
 
@@ -110,6 +110,7 @@ def lib():
         L.wrnn_subscale_net_conditioning.argtypes = [vp, vp, vp, i32, i32, i32, i64, vp, vp]
         L.wrnn_subscale_net_status.argtypes = [vp]
         L.wrnn_sample_subscale_net.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i64, C.c_uint64, vp, vp]
+        L.wrnn_subscale_net_rows.argtypes = [vp, vp, vp, i32, i32, i32, vp, i64, vp, vp, vp, i32, i32, i64, i32, C.c_uint64, vp]
         L.wrnn_launch_count.argtypes = []
         L.wrnn_launch_count.restype = i64
         _lib = L
@@ -303,6 +304,14 @@ def wrnn_sample_subscale_net(model, net, frames, F: int, chunk: int, lag: int, n
     frames: CUDA float32 [B][n_frames][D]; out: CUDA int16 [n_total] in the original order."""
     _check(lib().wrnn_sample_subscale_net(model, net, _dev_ptr(frames), int(frames.shape[1]), hop, F, chunk, lag, n_total, seed, _dev_ptr(out),
                                           _stream_ptr(stream)), model)
+
+
+def wrnn_subscale_net_rows(model, net, frames, lag: int, hist, h, c_prev, f_prev, r_lo: int, n_rows: int, p_lo: int, n_steps: int, seed: int, *,
+                           hop: int = 120, stream=None):
+    """One stepping call of the staggered schedule on caller-owned CUDA buffers: hist int16 [B][L] (in / out), h float32 [B][H],
+    c_prev / f_prev uint8 [B] (carry state of all rows); rows r_lo .. r_lo + n_rows - 1, row b from position p_lo - b * lag on."""
+    _check(lib().wrnn_subscale_net_rows(model, net, _dev_ptr(frames), int(frames.shape[1]), hop, lag, _dev_ptr(hist), int(hist.shape[1]), _dev_ptr(h),
+                                        _dev_ptr(c_prev), _dev_ptr(f_prev), r_lo, n_rows, p_lo, n_steps, seed, _stream_ptr(stream)), model)
 
 
 def wrnn_subscale_schedule(B: int, L: int, chunk: int, lag: int):

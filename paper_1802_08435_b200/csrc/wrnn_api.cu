@@ -691,6 +691,51 @@ int wrnn_sample_subscale_net(wrnn_model *m, wrnn_subscale_net *net, const float 
                                    });
 }
 
+int wrnn_subscale_net_rows(wrnn_model *m, wrnn_subscale_net *net, const float *frames, int32_t n_frames, int32_t hop, int32_t lag, int16_t *hist,
+                           int64_t L, float *h, uint8_t *c_prev, uint8_t *f_prev, int32_t r_lo, int32_t n_rows, int64_t p_lo, int32_t n_steps,
+                           uint64_t seed, void *cuda_stream)
+{
+    if (!m || !net) return WRNN_ERR_INVALID_ARG;
+    if (m->variant != 0) return fail(m, WRNN_ERR_UNSUPPORTED, "subscale generation takes a WaveRNN model (variant 0)");
+    const int B = subnet_B(net), D = m->cond_dim, H = m->H;
+    if (subnet_cond_dim(net) != D || D <= 0) return fail(m, WRNN_ERR_INVALID_ARG, "the network's output does not match the model's conditioning size");
+    if (!frames || !hist || !h || !c_prev || !f_prev || hop < 1 || L < 1 || r_lo < 0 || n_rows < 1 || r_lo + n_rows > B || n_rows > m->max_batch ||
+        n_steps < 1 || lag < 1)
+        return fail(m, WRNN_ERR_INVALID_ARG, "bad arguments");
+    // every row of the call stays inside its sub-tensor, and its frames exist
+    const long long p_last_row = p_lo - (long long)(n_rows - 1) * lag;
+    if (p_last_row < 0 || p_lo + n_steps > L) return fail(m, WRNN_ERR_INVALID_ARG, "positions outside the sub-tensors");
+    if (((long long)B * (p_lo + n_steps - 1) + (B - 1)) / hop >= n_frames) return fail(m, WRNN_ERR_INVALID_ARG, "conditioning frames run out");
+    if (cudaSetDevice(m->device) != cudaSuccess) return fail(m, WRNN_ERR_CUDA, "cudaSetDevice failed");
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    const size_t need = (size_t)n_rows * n_steps * D * sizeof(float);
+    if (need > m->sub_cap) {
+        cudaDeviceSynchronize();
+        cudaFree(m->sub_scratch); m->sub_scratch = nullptr; m->sub_cap = 0;
+        if (cudaMalloc((void **)&m->sub_scratch, need) != cudaSuccess) { cudaGetLastError(); return fail(m, WRNN_ERR_NOMEM, "scratch allocation failed"); }
+        m->sub_cap = need;
+    }
+    float *v = reinterpret_cast<float *>(m->sub_scratch);
+    int rc = subnet_run(net, hist, frames, n_frames, hop, L, r_lo, n_rows, p_lo, lag, n_steps, v, m->wait_limit_ns(), s);
+    if (rc != WRNN_OK) return fail(m, rc, "conditioning launch failed");
+    const int group = (n_rows >= 2 && use_multi(m, n_rows)) ? n_rows : (n_rows <= 3 && (use_reslean(m, 1) || use_resident(m, 1))) ? 1 : n_rows;
+    for (int b0 = 0; b0 < n_rows; b0 += group) {
+        const int r0 = r_lo + b0;
+        const long long p0 = p_lo - (long long)b0 * lag;
+        StepArgs a;
+        std::memset(&a, 0, sizeof(a));
+        a.cond = v + (size_t)b0 * n_steps * D; a.n_frames = n_steps; a.hop = 1; a.row_stride = 1; a.row_offset_mul = 0;
+        a.n_steps = n_steps; a.batch = group; a.seed = seed; a.step0 = p0; a.stream0 = (unsigned)r0;
+        a.h_in = a.h_out = h + (size_t)r0 * H;
+        a.c_in = a.c_st_out = c_prev + r0; a.f_in = a.f_st_out = f_prev + r0;
+        a.out = hist + (size_t)r0 * L + p0;
+        a.row_lag = lag; a.out_pitch = L - lag;
+        rc = run_steps(m, a, s);
+        if (rc != WRNN_OK) return rc;
+    }
+    return WRNN_OK;
+}
+
 int wrnn_sample_host(wrnn_model *m, const float *cond_host, int32_t n_frames, int32_t hop, int32_t row_stride,
                      int32_t row_offset_mul, int64_t n_steps, int32_t batch, uint64_t seed, int16_t *out_host)
 {

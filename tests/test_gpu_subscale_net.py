@@ -94,3 +94,74 @@ def test_generation_through_the_network(env, H, dtype, B_rows, L, chunk, kernel)
     finally:
         Bn.wrnn_subscale_net_destroy(net)
         Bn.wrnn_destroy(m)
+
+
+class _LocalLinks:
+    """In-process stand-in for the next-neighbour links of the pipeline (one GPU here): messages queue per destination."""
+
+    def __init__(self):
+        self.q = {}
+
+    def send(self, msg, dst):
+        self.q.setdefault(dst, []).append(msg.clone())
+
+    def irecv(self, buf, src):
+        links, dst = self, src + 1
+
+        class _Work:
+            def wait(self, timeout=None):
+                if not links.q.get(dst):
+                    return False
+                buf.copy_(links.q[dst].pop(0))
+                return True
+        return _Work()
+
+
+def test_pipeline_ranks_on_one_gpu(env):
+    """The device side of the one-way pipeline (Section 5.3): two ranks' worth of sub-tensors generated through
+    wrnn_subscale_net_rows on their own history and carry buffers, the samples handed on by the pipeline's messages (ranks
+    run turn by turn on the one GPU here); every draw of the last rank's history against the oracle forced on it."""
+    torch, Bn = env
+    from paper_1802_08435_b200 import pipeline as pl
+    dev = "cuda:0"
+    H, B_rows, L, chunk, F, world = 896, 16, 384, 128, 128, 2
+    lag = F + chunk
+    w = synth.make_weights(H, cond_dim=synth.COND_DIM, seed_w=31, seed_b=32)
+    nw = synth.make_subscale_net(B_rows)
+    frames = synth.make_cond(B_rows, (B_rows * L) // synth.HOP + 2, synth.COND_DIM)
+    om, net_o = orc.OracleModel(w, "bf16"), sn.SubscaleNet(nw)
+    m = Bn.wrnn_create(w, "bf16", max_batch=B_rows // world)
+    net = Bn.wrnn_subscale_net_create(nw)
+    try:
+        f_d = torch.from_numpy(frames).to(dev)
+        links = _LocalLinks()
+        ranks = []
+        for r in range(world):
+            hist = torch.zeros((B_rows, L), dtype=torch.int16, device=dev)
+            h = torch.zeros((B_rows, H), dtype=torch.float32, device=dev)
+            cp = torch.full((B_rows,), 128, dtype=torch.uint8, device=dev)
+            fp = torch.zeros((B_rows,), dtype=torch.uint8, device=dev)
+            pipe = pl.SubscalePipeline(links, r, world, B_rows, L, F, chunk, lag, device=dev, timeout_s=1.0)
+
+            def gen(r_lo, n_rows, p_lo, n, hist=hist, h=h, cp=cp, fp=fp):
+                Bn.wrnn_subscale_net_rows(m, net, f_d, lag, hist, h, cp, fp, r_lo, n_rows, p_lo, n, SEED)
+                torch.cuda.synchronize()
+                assert Bn.wrnn_poll_status(m) == 0, Bn.wrnn_last_error(m)
+            ranks.append((pipe, hist, gen))
+        for k in range(max(p.n_iterations() for p, _, _ in ranks)):
+            for pipe, hist, gen in ranks:
+                if k < pipe.n_iterations():
+                    pipe.step(k, hist, gen)
+        got = ranks[-1][1].cpu().numpy()
+        assert np.array_equal(ranks[0][1].cpu().numpy()[:B_rows // 2], got[:B_rows // 2])        # what rank 0 made is what rank 1 holds
+        want, _, mg = sn.subscale_net_run(om, net_o, frames, L, synth.HOP, SEED, forced=got, teacher=True)
+        gc, gf = pu._split(got)
+        wc, wf = pu._split(want)
+        nd_c, bad_c = pu.check_indices(gc, wc, mg[:, :, 0])
+        nd_f, bad_f = pu.check_indices(gf, wf, mg[:, :, 1])
+        print("\n[parity] two pipeline ranks x 8 sub-tensors: idx_diff=%d (near-boundary draws %d, bad %d); messages %s" % (
+            nd_c + nd_f, int((mg < pu.MARGIN).sum()), bad_c + bad_f, [(p.sent, p.received) for p, _, _ in ranks]))
+        assert bad_c + bad_f == 0
+    finally:
+        Bn.wrnn_subscale_net_destroy(net)
+        Bn.wrnn_destroy(m)

@@ -57,6 +57,7 @@ struct ResF32Params {
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
+    int poll_gap;                            // >= 0: the state exchange's pollers start this many cycles after the CTA's own publication
     int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
     long long *prof;                         // [16] per-phase cycle totals of CTA 0, warp 0 (same slots as the bf16 kernel)
 };
@@ -99,7 +100,10 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
 
     const bool prof_on = p.prof != nullptr && cta == 0 && warp == 0;
     __shared__ long long s_prof[16];
+    __shared__ __align__(8) unsigned long long pub_bar;      // one arrival per half-step: this CTA's gate threads have published
+    if (tid == 0) { mbar_init_cluster(smem_addr(&pub_bar), 1); mbar_fence_init(); }
     if (tid < 16) s_prof[tid] = 0;
+    __syncthreads();
     long long prof_t = clock64();
 #define STAMP(i) do { if (prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
 
@@ -206,21 +210,37 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
         load_g(0, 0, gv);
         gates_and_publish(0, 0, f_prev, gates_prepare(0, gv));
     }
+    if (tid == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&pub_bar)) : "memory");
 
-    // all-gather of n (even) tagged words from the chip into a shared-memory vector: two adjacent slots per polling thread
-    auto gather = [&](const unsigned long long *slots, int n, unsigned want, float *dst, int step, int phase) {
-#pragma unroll 1
-        for (int i = tid; i < n / 2; i += blockDim.x) {
-            unsigned long long v0, v1, t0 = 0; unsigned cnt = 0;
-            while (true) {
-                asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0), "=l"(v1) : "l"(slots + 2 * i) : "memory");
-                if ((unsigned)(v0 >> 32) == want && (unsigned)(v1 >> 32) == want) break;
-                if ((++cnt & 4095u) == 0 && wt.expired(t0, step, phase)) { my_bad = true; break; }
+    // all-gather of n (even) tagged words from the chip into a shared-memory vector: two adjacent slots per polling thread.
+    // held_back (the exchange of the state, whose words this CTA's own gate threads publish at about the time every other
+    // CTA's do): the drawing warp does not poll, and the pollers wait for the CTA's own publication plus poll_gap cycles, so
+    // that the first poll reaches L2 when the words do (a poll that just misses them costs a whole round trip, and early
+    // polls slow the publishing stores).  hs = the half-step index (parity of the publication barrier).
+    auto gather = [&](const unsigned long long *slots, int n, unsigned want, float *dst, int step, int phase, bool held_back, long long hs) {
+        const int first = held_back ? 32 : 0, np = (int)blockDim.x - first;
+        if (tid >= first) {
+            if (held_back) {
+                unsigned cnt = 0; unsigned long long t0 = 0;
+                while (!mbar_try_parity(smem_addr(&pub_bar), (unsigned)((hs - 1) & 1)))
+                    if ((++cnt & 1023u) == 0 && wt.expired(t0, step, phase)) { my_bad = true; break; }
+                const long long c0 = clock64();
+                while (clock64() - c0 < p.poll_gap) { }
             }
-            dst[2 * i] = __uint_as_float((unsigned)v0); dst[2 * i + 1] = __uint_as_float((unsigned)v1);
+#pragma unroll 1
+            for (int i = tid - first; i < n / 2; i += np) {
+                unsigned long long v0 = 0, v1 = 0, t0 = 0; unsigned cnt = 0;
+                while (!my_bad) {
+                    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0), "=l"(v1) : "l"(slots + 2 * i) : "memory");
+                    if ((unsigned)(v0 >> 32) == want && (unsigned)(v1 >> 32) == want) break;
+                    if ((++cnt & 4095u) == 0 && wt.expired(t0, step, phase)) { my_bad = true; break; }
+                }
+                dst[2 * i] = __uint_as_float((unsigned)v0); dst[2 * i + 1] = __uint_as_float((unsigned)v1);
+            }
         }
         return __syncthreads_or(my_bad) != 0;
     };
+    const bool hold = p.poll_gap >= 0 && blockDim.x > 32;
 
     // Half-step n = 2 s + 1 is the "coarse" half of step s (input y_c(s): coarse head -> c_s; R[:, :Hh] y_c(s) kept for
     // step s+1; then the fine gates of step s); n = 2 s is the "fine" half (input y_f(s-1): fine head -> f_{s-1};
@@ -244,7 +264,7 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
         }
 
         // ---- 1. input half-vector from the whole chip (y_c(s) carries tag s+1; y_f(s-1) carries tag s)
-        if (gather(p.yslots + (size_t)(half ? (s & 1) : 2 + ((s - 1) & 1)) * K, K, (unsigned)(half ? s + 1 : s), vec, (int)s, 1 + 4 * half)) break;
+        if (gather(p.yslots + (size_t)(half ? (s & 1) : 2 + ((s - 1) & 1)) * K, K, (unsigned)(half ? s + 1 : s), vec, (int)s, 1 + 4 * half, hold, n)) break;
         STAMP(0 + 6 * half);
 
         // ---- 2. this CTA's rows of the hidden layer and of R against the same input; publish the hidden-layer rows
@@ -255,7 +275,7 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
         STAMP(1 + 6 * half);
 
         // ---- 3. the whole hidden layer -> this CTA's rows of the logits, sent to every CTA of the cluster
-        if (gather(p.qslots + (size_t)par * K, K, tag, qvec, (int)s, 2 + 4 * half)) break;
+        if (gather(p.qslots + (size_t)par * K, K, tag, qvec, (int)s, 2 + 4 * half, false, n)) break;
         STAMP(2 + 6 * half);
         rows_times(half ? wO2 : wO4, LR, qvec);
         __syncthreads();
@@ -311,6 +331,7 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
                 f_prev = drawn;
             }
             if (lane < UC && !last && !my_bad) gates_and_publish(half, s, drawn, gp);
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&pub_bar)) : "memory");
             if (half) c_prev = drawn;
         }
         STAMP(5 + 6 * half);
@@ -515,6 +536,7 @@ int resf32_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
+    { const char *e = getenv("WRNN_F32_POLL_GAP"); p.poll_gap = e ? atoi(e) : 0; }
     p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
     p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
 

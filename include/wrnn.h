@@ -48,7 +48,10 @@ typedef enum {
     WRNN_ERR_UNSUPPORTED = 2,   /* shape / dtype / batch has no kernel, or it does not fit the device */
     WRNN_ERR_NOMEM = 3,
     WRNN_ERR_CUDA = 4,
-    WRNN_ERR_TIMEOUT = 5        /* a bounded device-side wait ran out; the kernel returned cleanly */
+    WRNN_ERR_TIMEOUT = 5,       /* a bounded device-side wait ran out; the kernel returned cleanly */
+    WRNN_ERR_CHECK = 6          /* checked build (models created under WRNN_DEBUG=1): an index left its array or a guard  */
+                                /* word behind a shared-memory region was overwritten; the access was skipped, the kernel */
+                                /* returned cleanly; wrnn_last_error names the CTA and the region                         */
 } wrnn_status;
 
 typedef enum { WRNN_F32 = 0, WRNN_BF16 = 1 } wrnn_dtype;

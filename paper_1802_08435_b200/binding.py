@@ -16,11 +16,11 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libwrnn.so")
 
-WRNN_OK, WRNN_ERR_INVALID_ARG, WRNN_ERR_UNSUPPORTED, WRNN_ERR_NOMEM, WRNN_ERR_CUDA, WRNN_ERR_TIMEOUT = range(6)
+WRNN_OK, WRNN_ERR_INVALID_ARG, WRNN_ERR_UNSUPPORTED, WRNN_ERR_NOMEM, WRNN_ERR_CUDA, WRNN_ERR_TIMEOUT, WRNN_ERR_CHECK = range(7)
 WRNN_F32, WRNN_BF16 = 0, 1
 WRNN_KERNEL_AUTO, WRNN_KERNEL_GENERIC, WRNN_KERNEL_RESIDENT, WRNN_KERNEL_BATCHED, WRNN_KERNEL_SPARSE = 0, 1, 2, 3, 4
 WRNN_KERNEL_BCLUSTER = 5
-_STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "NOMEM", "CUDA", "TIMEOUT"]
+_STATUS_NAMES = ["OK", "INVALID_ARG", "UNSUPPORTED", "NOMEM", "CUDA", "TIMEOUT", "CHECK"]
 
 EXPORTS = [
     "wrnn_create", "wrnn_destroy", "wrnn_sample", "wrnn_step_teacher_forced", "wrnn_fold", "wrnn_unfold",
@@ -34,7 +34,7 @@ EXPORTS = [
 
 class WrnnError(RuntimeError):
     def __init__(self, code: int, msg: str):
-        super().__init__("wrnn status %d (%s): %s" % (code, _STATUS_NAMES[code] if 0 <= code < 6 else "?", msg))
+        super().__init__("wrnn status %d (%s): %s" % (code, _STATUS_NAMES[code] if 0 <= code < 7 else "?", msg))
         self.code = code
 
 

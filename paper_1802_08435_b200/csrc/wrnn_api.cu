@@ -811,7 +811,14 @@ int wrnn_poll_status(wrnn_model *m)
     if (cudaMemcpy(&st, m->status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess)
         return fail(m, WRNN_ERR_CUDA, std::string("status read failed: ") + cudaGetErrorString(cudaGetLastError()));
     if (st.code != DEV_OK) {
-        char buf[160];
+        char buf[200];
+        if (st.code == DEV_CHECK) {
+            std::snprintf(buf, sizeof(buf), "checked build: cta %d found %s (region %d)", st.cta,
+                          st.step == -1 ? "an exchange slot outside the slot array" : st.step == -2 ? "a shared-memory carve-up that disagrees with the allocation"
+                                                                                                      : "a clobbered guard behind a shared-memory region", st.step);
+            m->err = buf;
+            return WRNN_ERR_CHECK;
+        }
         std::snprintf(buf, sizeof(buf), "device-side wait timed out (code %d) at cta %d, step %d, phase %d", st.code, st.cta, st.step, st.phase);
         m->err = buf;
         return st.code == DEV_TIMEOUT ? WRNN_ERR_TIMEOUT : WRNN_ERR_CUDA;

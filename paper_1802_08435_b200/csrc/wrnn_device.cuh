@@ -13,6 +13,7 @@ constexpr unsigned FULL = 0xffffffffu;
 struct DevStatus { int code; int cta; int step; int phase; };
 constexpr int DEV_OK = 0;
 constexpr int DEV_TIMEOUT = 5;      // == WRNN_ERR_TIMEOUT
+constexpr int DEV_CHECK = 6;        // == WRNN_ERR_CHECK: the checked build found an index outside its array or a clobbered guard
 
 // ------------------------------------------------------------------ Philox4x32-10
 // Counter-based generator of Salmon et al. (SC'11).  One call per (row, step, head).

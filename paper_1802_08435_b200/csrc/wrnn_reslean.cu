@@ -46,6 +46,7 @@ struct ResLeanPack {
     unsigned long long *d_slots = nullptr;   // [2 halves][2 parities][K] (value, tag)
     long long *d_prof = nullptr;             // [16] phase cycle totals of the last call
     int smem_bytes = 0;
+    bool checked = false;                    // WRNN_DEBUG=1 at create: the guarded carve-up
     int64_t weight_bytes_per_step = 0;
 };
 
@@ -70,6 +71,8 @@ struct ResLeanParams {
     int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
     long long *prof;                         // optional [n CTAs][16] per-phase cycle totals of warp 0 (CTA 0 only unless prof_all)
     int prof_all;
+    int chk_poke;                            // checked build only: make one deliberate one-past-the-end write (into a guard)
+    unsigned long long smem_bytes;           // dynamic shared memory of the launch (the checked build compares its carve-up with it)
     int poll_gap;                            // >= 0: the pollers of the chip-wide exchange start this many cycles after the CTA's own publication; < 0: at once
 };
 
@@ -86,6 +89,14 @@ constexpr size_t RL_SMEM_BYTES = RL_BLOB_BYTES + (size_t)2 * RL_K * 4 /* vecC, v
                                  2 * RL_KS * 32 * 4 /* partH, partR */ + 2 * 4 * RL_K * 2 /* splC, splF */ + 32 * 4 /* q_own */ +
                                  32 * 4 /* lrow */ + (size_t)2 * RL_K * 4 /* qbuf */ + (size_t)2 * RL_NLOG * 4 /* lbuf */;
 
+// CHK: the checked build (WRNN_DEBUG=1 at create).  Every writable region of the shared-memory carve-up is followed by a
+// 16-byte guard (and the first one preceded by one) that is filled at the start and verified at the end, the carve-up's end
+// is compared with the size the host allocated, and the index of every published exchange slot is range-checked; a
+// violation is recorded in the status word (code 6, step = index of the region or -1 for a slot, phase 99), the access that
+// would leave its array is skipped, and the kernel runs to its normal exit.
+constexpr int RL_N_GUARDS = 13;
+constexpr unsigned RL_GUARD_WORD = 0x5afec0deu;
+template <bool CHK>
 __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -104,18 +115,29 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
     const unsigned *wL4 = wL2 + RL_LR * K / 2;
     const float *sI = reinterpret_cast<const float *>(smem + RL_W_BYTES);           // [NR][3]
     const float *sb1 = sI + NR * 3, *sb3 = sb1 + 32, *sb2 = sb3 + 32, *sb4 = sb2 + RL_LR;
-    float *vecC = reinterpret_cast<float *>(smem + RL_BLOB_BYTES);                  // [K] y_c
-    float *vecF = vecC + K;                                                         // [K] y_f
-    float *a_part = vecF + K;                                                       // [NR] R[:, :Hh] y_c
-    float *a_full = a_part + NR;                                                    // [NR] R h
-    float *partH = a_full + NR;                                                     // [KS][32] K-split partials of the hidden rows
-    float *partR = partH + RL_KS * 32;                                              // [KS][32] ... of the R rows
-    __nv_bfloat16 *splC = reinterpret_cast<__nv_bfloat16 *>(partR + RL_KS * 32);    // split images, 4 K bf16 each
-    __nv_bfloat16 *splF = splC + 4 * K;
-    float *q_own = reinterpret_cast<float *>(splF + 4 * K);                         // [32] this CTA's rows of the hidden layer
-    float *lrow = q_own + 32;                                                       // [16 (+16)] this CTA's logits
-    float *qbuf = lrow + 32;                                                        // [2 parities][K] hidden layer of the cluster
-    float *lbuf = qbuf + 2 * K;                                                     // [2 parities][256] logits of the cluster
+    // writable regions, each followed by a guard in the checked build (region index = order below)
+    size_t off = RL_BLOB_BYTES;
+    unsigned guard_off[RL_N_GUARDS];
+    int n_guard = 0;
+    auto guard = [&]() { if (CHK) { guard_off[n_guard++] = (unsigned)off; off += 16; } };
+    auto carve = [&](size_t bytes) { uint8_t *r = smem + off; off += bytes; guard(); return r; };
+    guard();                                                                        // 0: between the weights and the first vector
+    float *vecC = reinterpret_cast<float *>(carve((size_t)K * 4));                  // 1: [K] y_c
+    float *vecF = reinterpret_cast<float *>(carve((size_t)K * 4));                  // 2: [K] y_f
+    float *a_part = reinterpret_cast<float *>(carve(NR * 4));                       // 3: [NR] R[:, :Hh] y_c
+    float *a_full = reinterpret_cast<float *>(carve(NR * 4));                       // 4: [NR] R h
+    float *partH = reinterpret_cast<float *>(carve(RL_KS * 32 * 4));                // 5: [KS][32] K-split partials of the hidden rows
+    float *partR = reinterpret_cast<float *>(carve(RL_KS * 32 * 4));                // 6: [KS][32] ... of the R rows
+    __nv_bfloat16 *splC = reinterpret_cast<__nv_bfloat16 *>(carve((size_t)4 * K * 2));   // 7: split images, 4 K bf16 each
+    __nv_bfloat16 *splF = reinterpret_cast<__nv_bfloat16 *>(carve((size_t)4 * K * 2));   // 8
+    float *q_own = reinterpret_cast<float *>(carve(32 * 4));                        // 9: [32] this CTA's rows of the hidden layer
+    float *lrow = reinterpret_cast<float *>(carve(32 * 4));                         // 10: [16 (+16)] this CTA's logits
+    float *qbuf = reinterpret_cast<float *>(carve((size_t)2 * K * 4));              // 11: [2 parities][K] hidden layer of the cluster
+    float *lbuf = reinterpret_cast<float *>(carve((size_t)2 * RL_NLOG * 4));        // 12: [2 parities][256] logits of the cluster
+    auto record_check = [&](int what) {
+        if (atomicCAS(&p.status->code, DEV_OK, DEV_CHECK) == DEV_OK) { p.status->cta = blockIdx.x; p.status->step = what; p.status->phase = 99; }
+    };
+    if (CHK && threadIdx.x == 0 && off != p.smem_bytes) record_check(-2);          // the carve-up and the allocation disagree
     __shared__ __align__(8) unsigned long long xq[2], xl[2];                        // arrival barriers of qbuf[.], lbuf[.]
 
     // ---- one-time load of this CTA's weights
@@ -127,7 +149,11 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
             for (int i = 0; i < 2; ++i) { mbar_init_cluster(smem_addr(&xq[i]), 1); mbar_init_cluster(smem_addr(&xl[i]), 1); }
             mbar_fence_init();
         }
-        for (int i = tid; i < 8 * K / 8; i += blockDim.x) reinterpret_cast<uint4 *>(splC)[i] = make_uint4(0, 0, 0, 0);
+        for (int i = tid; i < 4 * K / 8; i += blockDim.x) {
+            reinterpret_cast<uint4 *>(splC)[i] = make_uint4(0, 0, 0, 0);
+            reinterpret_cast<uint4 *>(splF)[i] = make_uint4(0, 0, 0, 0);
+        }
+        if (CHK && tid < n_guard) *reinterpret_cast<uint4 *>(smem + guard_off[tid]) = make_uint4(RL_GUARD_WORD, RL_GUARD_WORD, RL_GUARD_WORD, RL_GUARD_WORD);
         __syncthreads();
         for (int i = tid; i < K; i += blockDim.x) {
             const float c = p.h_in ? p.h_in[i] : 0.f, f = p.h_in ? p.h_in[K + i] : 0.f;
@@ -194,6 +220,8 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         return true;
     };
 
+    // self-test of the checker itself: one word written one past the end of a region (it lands in that region's guard)
+    if (CHK && p.chk_poke && cta == 3 && tid == 0) partR[RL_KS * 32] = 1.0f;
     // ---- prologue: R h of the initial state, coarse gates of step 0
     if (mma_on) tile_pair_products(wRA, splC, partR);
     __syncthreads();
@@ -227,9 +255,10 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
-        if ((int)s != skip_at)
-            st_relaxed_u64(p.slots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
-                           ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
+        const size_t slot = (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j;
+        if (CHK && slot >= (size_t)4 * K) record_check(-1);                          // an exchange slot outside the slot array: skipped
+        else if ((int)s != skip_at)
+            st_relaxed_u64(p.slots + slot, ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
         if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
     };
@@ -404,6 +433,10 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
 #undef STAMP
 
     const int any_bad = __syncthreads_or(my_bad);
+    if (CHK && tid < n_guard) {
+        const uint4 g = *reinterpret_cast<const uint4 *>(smem + guard_off[tid]);
+        if (g.x != RL_GUARD_WORD || g.y != RL_GUARD_WORD || g.z != RL_GUARD_WORD || g.w != RL_GUARD_WORD) record_check(tid);
+    }
     if (writer && !any_bad) {
         if (p.h_out) for (int i = tid; i < K; i += blockDim.x) { p.h_out[i] = vecC[i]; p.h_out[K + i] = vecF[i]; }
         if (tid == 0) {
@@ -420,7 +453,7 @@ static void fill_launch(const ResLeanPack &k, cudaLaunchConfig_t *cfg, cudaLaunc
     std::memset(cfg, 0, sizeof(*cfg));
     cfg->gridDim = dim3(k.NCTA);
     cfg->blockDim = dim3(512);
-    cfg->dynamicSmemBytes = k.smem_bytes;
+    cfg->dynamicSmemBytes = k.smem_bytes + (k.checked ? RL_N_GUARDS * 16 : 0);
     cfg->stream = s;
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = RL_CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
@@ -444,15 +477,17 @@ int reslean_prepare(wrnn_model *m)
     cudaDeviceProp prop;
     cudaGetDeviceProperties(&prop, m->device);
     if (k.NCTA > m->n_sms || (size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "lean resident kernel does not fit this device"; return WRNN_ERR_UNSUPPORTED; }
-    if (cudaFuncSetAttribute(resident_lean_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-        cudaFuncSetAttribute(resident_lean_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
+    { const char *d = getenv("WRNN_DEBUG"); k.checked = d && d[0] == '1'; }
+    const void *fn = k.checked ? (const void *)resident_lean_kernel<true> : (const void *)resident_lean_kernel<false>;
+    if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes + (k.checked ? RL_N_GUARDS * 16 : 0)) != cudaSuccess) {
         cudaGetLastError(); m->err = "lean resident kernel: cannot set the launch attributes"; return WRNN_ERR_UNSUPPORTED;
     }
     {
         cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
         fill_launch(k, &cfg, at, 0, false);
         int max_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_lean_kernel, &cfg) != cudaSuccess || max_clusters < k.NC) {
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, fn, &cfg) != cudaSuccess || max_clusters < k.NC) {
             cudaGetLastError(); m->err = "lean resident kernel: not enough co-resident clusters"; return WRNN_ERR_UNSUPPORTED;
         }
     }
@@ -532,7 +567,7 @@ int reslean_launch_info(const wrnn_model *m, int *n_ctas, int *n_threads, int *s
     const ResLeanPack &k = *m->reslean;
     if (n_ctas) *n_ctas = k.NCTA;
     if (n_threads) *n_threads = 512;
-    if (smem) *smem = k.smem_bytes;
+    if (smem) *smem = k.smem_bytes + (k.checked ? RL_N_GUARDS * 16 : 0);
     if (weight_bytes) *weight_bytes = k.weight_bytes_per_step;
     return WRNN_OK;
 }
@@ -563,7 +598,9 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     fill_launch(k, &cfg, at, s, coop_launch_allowed());
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, resident_lean_kernel, p);
+    p.smem_bytes = cfg.dynamicSmemBytes;
+    { const char *d = getenv("WRNN_DEBUG_POKE"); p.chk_poke = (k.checked && d && d[0] == '1') ? 1 : 0; }
+    const cudaError_t e = k.checked ? cudaLaunchKernelEx(&cfg, resident_lean_kernel<true>, p) : cudaLaunchKernelEx(&cfg, resident_lean_kernel<false>, p);
     if (e != cudaSuccess) {
         m->err = std::string("lean resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

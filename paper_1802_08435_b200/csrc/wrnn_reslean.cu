@@ -248,6 +248,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         return q;
     };
     const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
+    const bool dbg_any = p.dbg_gates != nullptr || p.dbg_h != nullptr;
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
         const float xk = scale8(drawn);
         const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
@@ -259,8 +260,10 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         if (CHK && slot >= (size_t)4 * K) record_check(-1);                          // an exchange slot outside the slot array: skipped
         else if ((int)s != skip_at)
             st_relaxed_u64(p.slots + slot, ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
-        if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
-        if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
+        if (dbg_any) {
+            if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
+            if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
+        }
     };
     auto load_g = [&](int half_g, long long s, float (&gv)[3]) {
         const long long fr = ((p.step0 + s) * p.row_stride + (long long)p.stream0 * p.row_offset_mul) / p.hop - p.frame_shift;

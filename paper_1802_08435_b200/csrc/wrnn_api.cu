@@ -397,6 +397,7 @@ int wrnn_create(const wrnn_params *p, int32_t max_batch, wrnn_model **out)
             wrnn_destroy(m);
             return fail(nullptr, rc, "resident kernel unavailable: " + why);
         }
+        reslean_prepare(m);     // optional: the lean form of the same kernel (the first form serves the variant without it)
         *out = m;
         return WRNN_OK;
     }

@@ -36,8 +36,10 @@ constexpr int RL_HR = 28;        // hidden-layer rows per CTA (= columns of its 
 constexpr int RL_UC = 4;         // state units per half per CTA
 constexpr int RL_NR = 24;        // rows of R per CTA: (coarse, fine) x (u, r, e) x UC
 constexpr int RL_KS = 14;        // K-splits of the hidden / recurrent products: 14 warps x 2 k-tiles
-constexpr int RL_NLOG = 256;
-constexpr int RL_LR = 16;        // output-layer rows per CTA: one per warp
+// per variant (FUSED = the Fused Subscale WaveRNN 2x: 64 logits per head as four softmaxes of 4 bits, twelve nibble inputs)
+__host__ __device__ constexpr int rl_nlog(bool fused) { return fused ? 64 : 256; }
+__host__ __device__ constexpr int rl_lr(bool fused) { return rl_nlog(fused) / RL_CS; }      // output-layer rows per CTA
+__host__ __device__ constexpr int rl_nin(bool fused) { return fused ? 12 : 3; }
 
 struct ResLeanPack {
     int NCTA = 0, NC = 0;
@@ -47,6 +49,7 @@ struct ResLeanPack {
     long long *d_prof = nullptr;             // [16] phase cycle totals of the last call
     int smem_bytes = 0;
     bool checked = false;                    // WRNN_DEBUG=1 at create: the guarded carve-up
+    bool fused = false;                      // the Fused Subscale WaveRNN 2x (model variant 1)
     int64_t weight_bytes_per_step = 0;
 };
 
@@ -65,6 +68,10 @@ struct ResLeanParams {
     const uint8_t *c_forced, *f_forced;
     uint8_t *c_out, *f_out;
     int16_t *out;
+    // the fused variant's 16-bit counterparts of the byte arrays above (part A = the coarse half, part B = the fine half)
+    const uint16_t *a_in, *b_in; uint16_t *a_st_out, *b_st_out;
+    const uint16_t *a_forced, *b_forced;
+    uint16_t *a_out, *b_out;
     float *dbg_gates, *dbg_h, *dbg_logits;
     DevStatus *status;
     unsigned long long limit_ns;
@@ -79,15 +86,17 @@ struct ResLeanParams {
 // byte offsets inside the bf16 part of a CTA's blob
 constexpr size_t RL_TILE_U4 = (size_t)RL_NKT * 32;                 // uint4 per 16-row tile over the full K
 constexpr size_t RL_HID_BYTES = 2 * RL_TILE_U4 * 16;               // two tiles: 28,672 B
-constexpr size_t RL_LOG_BYTES = (size_t)RL_LR * RL_K * 2;          // 16 rows of O2 (O4), row-major bf16: 14,336 B
-constexpr size_t RL_W_BYTES = 4 * RL_HID_BYTES + 2 * RL_LOG_BYTES; // 143,360 B
-constexpr int RL_SMALL_FLOATS = RL_NR * 3 + 2 * 32 + 2 * RL_LR;    // I*, b1, b3 (padded to 32), b2, b4 (this CTA's rows)
-constexpr size_t RL_BLOB_BYTES = RL_W_BYTES + (size_t)RL_SMALL_FLOATS * 4;
-static_assert(RL_BLOB_BYTES % 16 == 0, "blob is copied in 16-byte pieces");
+__host__ __device__ constexpr size_t rl_log_bytes(bool f) { return (size_t)rl_lr(f) * RL_K * 2; }          // this CTA's rows of O2 (O4), row-major bf16: 14,336 B
+__host__ __device__ constexpr size_t rl_w_bytes(bool f) { return 4 * RL_HID_BYTES + 2 * rl_log_bytes(f); }  // 143,360 B
+__host__ __device__ constexpr int rl_small_floats(bool f) { return RL_NR * rl_nin(f) + 2 * 32 + 2 * rl_lr(f); }   // I*, b1, b3 (padded to 32), b2, b4 (this CTA's rows)
+__host__ __device__ constexpr size_t rl_blob_bytes(bool f) { return rl_w_bytes(f) + (size_t)rl_small_floats(f) * 4; }
+static_assert(rl_blob_bytes(false) % 16 == 0 && rl_blob_bytes(true) % 16 == 0, "blob is copied in 16-byte pieces");
 
-constexpr size_t RL_SMEM_BYTES = RL_BLOB_BYTES + (size_t)2 * RL_K * 4 /* vecC, vecF */ + 2 * 24 * 4 /* a_part, a_full */ +
-                                 2 * RL_KS * 32 * 4 /* partH, partR */ + 2 * 4 * RL_K * 2 /* splC, splF */ + 32 * 4 /* q_own */ +
-                                 32 * 4 /* lrow */ + (size_t)2 * RL_K * 4 /* qbuf */ + (size_t)2 * RL_NLOG * 4 /* lbuf */;
+__host__ __device__ constexpr size_t rl_smem_bytes(bool f)
+{
+    return rl_blob_bytes(f) + (size_t)2 * RL_K * 4 /* vecC, vecF */ + 2 * 24 * 4 /* a_part, a_full */ + 2 * RL_KS * 32 * 4 /* partH, partR */ +
+           2 * 4 * RL_K * 2 /* splC, splF */ + 32 * 4 /* q_own */ + 32 * 4 /* lrow */ + (size_t)2 * RL_K * 4 /* qbuf */ + (size_t)2 * rl_nlog(f) * 4 /* lbuf */;
+}
 
 // CHK: the checked build (WRNN_DEBUG=1 at create).  Every writable region of the shared-memory carve-up is followed by a
 // 16-byte guard (and the first one preceded by one) that is filled at the start and verified at the end, the carve-up's end
@@ -96,9 +105,11 @@ constexpr size_t RL_SMEM_BYTES = RL_BLOB_BYTES + (size_t)2 * RL_K * 4 /* vecC, v
 // would leave its array is skipped, and the kernel runs to its normal exit.
 constexpr int RL_N_GUARDS = 13;
 constexpr unsigned RL_GUARD_WORD = 0x5afec0deu;
-template <bool CHK>
+template <bool CHK, bool FUSED>
 __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanParams p)
 {
+    constexpr int RL_NLOG = rl_nlog(FUSED), RL_LR = rl_lr(FUSED), NIN = rl_nin(FUSED), NP = NIN / 3;
+    constexpr size_t RL_W_BYTES = rl_w_bytes(FUSED), RL_BLOB_BYTES = rl_blob_bytes(FUSED);
     extern __shared__ __align__(16) uint8_t smem[];
     cg::cluster_group cluster = cg::this_cluster();
     const int rank = (int)cluster.block_rank();
@@ -113,8 +124,8 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
     const uint4 *wRB = wHB + 2 * RL_TILE_U4;                                        // R rows x fine columns
     const unsigned *wL2 = reinterpret_cast<const unsigned *>(wRB + 2 * RL_TILE_U4);   // this CTA's 16 rows of O2, row-major, two bf16 per word
     const unsigned *wL4 = wL2 + RL_LR * K / 2;
-    const float *sI = reinterpret_cast<const float *>(smem + RL_W_BYTES);           // [NR][3]
-    const float *sb1 = sI + NR * 3, *sb3 = sb1 + 32, *sb2 = sb3 + 32, *sb4 = sb2 + RL_LR;
+    const float *sI = reinterpret_cast<const float *>(smem + RL_W_BYTES);           // [NR][NIN]
+    const float *sb1 = sI + NR * NIN, *sb3 = sb1 + 32, *sb2 = sb3 + 32, *sb4 = sb2 + RL_LR;
     // writable regions, each followed by a guard in the checked build (region index = order below)
     size_t off = RL_BLOB_BYTES;
     unsigned guard_off[RL_N_GUARDS];
@@ -179,7 +190,11 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
     const bool writer = (cta == 0);
     const int g4 = lane >> 2;
 
-    int c_prev = p.c_in ? p.c_in[0] : 128, f_prev = p.f_in ? p.f_in[0] : 0;
+    // the symbols fed back: the coarse / fine bytes, or (fused) the 16-bit samples of parts A / B
+    int c_prev, f_prev;
+    if (FUSED) { c_prev = p.a_in ? p.a_in[0] : 0x8000; f_prev = p.b_in ? p.b_in[0] : 0x8000; }
+    else { c_prev = p.c_in ? p.c_in[0] : 128; f_prev = p.f_in ? p.f_in[0] : 0; }
+    auto xin = [](int v, int k) { return FUSED ? scale4((v >> (12 - 4 * k)) & 15) : scale8(v); };    // scalar k of a symbol as the network sees it
     float hC = 0.f, hF = 0.f;
     if (warp == 0 && lane < UC) { hC = vecC[cta * UC + lane]; hF = vecF[cta * UC + lane]; }
 
@@ -234,25 +249,46 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
 
     // Gates of Eq. 2 for this CTA's units of one half of the state (half_g = 0: coarse units, 1: fine units): everything
     // up to the one input that the pending draw supplies is prepared while the logits are on their way.
-    struct GatePre { float pu, pr, pe, ae, ku, kr, ke; };
+    struct GatePre { float pu, pr, pe, ae, ku[NP], kr[NP], ke[NP]; };
     auto gates_prepare = [&](int half_g, const float (&gv)[3]) {
         GatePre q;
         const int rb = half_g ? 3 * UC : 0;
-        const float x0 = scale8(c_prev), x1 = scale8(f_prev);
-        const float *Iu = sI + 3 * (rb + lane), *Ir = sI + 3 * (rb + UC + lane), *Ie = sI + 3 * (rb + 2 * UC + lane);
-        q.pu = a_full[rb + lane] + fmaf(Iu[0], x0, half_g ? fmaf(Iu[1], x1, gv[0]) : gv[0]);
-        q.pr = a_full[rb + UC + lane] + fmaf(Ir[0], x0, half_g ? fmaf(Ir[1], x1, gv[1]) : gv[1]);
-        q.pe = fmaf(Ie[0], x0, half_g ? fmaf(Ie[1], x1, gv[2]) : gv[2]);
+        const float *Iu = sI + NIN * (rb + lane), *Ir = sI + NIN * (rb + UC + lane), *Ie = sI + NIN * (rb + 2 * UC + lane);
+        // fine units: inputs (c_{s-1}, f_{s-1}) known, c_s pending (last column group); coarse units: c_{s-1} known, f_{s-1}
+        // pending (middle column group)
+        float su = gv[0], sr = gv[1], se = gv[2];
+#pragma unroll
+        for (int k = 0; k < NP; ++k) {
+            const float x = xin(c_prev, k);
+            su = fmaf(Iu[k], x, su); sr = fmaf(Ir[k], x, sr); se = fmaf(Ie[k], x, se);
+        }
+        if (half_g) {
+#pragma unroll
+            for (int k = 0; k < NP; ++k) {
+                const float x = xin(f_prev, k);
+                su = fmaf(Iu[NP + k], x, su); sr = fmaf(Ir[NP + k], x, sr); se = fmaf(Ie[NP + k], x, se);
+            }
+        }
+        q.pu = a_full[rb + lane] + su;
+        q.pr = a_full[rb + UC + lane] + sr;
+        q.pe = se;
         q.ae = a_full[rb + 2 * UC + lane];
-        q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
+        const int pend = half_g ? 2 * NP : NP;
+#pragma unroll
+        for (int k = 0; k < NP; ++k) { q.ku[k] = Iu[pend + k]; q.kr[k] = Ir[pend + k]; q.ke[k] = Ie[pend + k]; }
         return q;
     };
     const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
     const bool dbg_any = p.dbg_gates != nullptr || p.dbg_h != nullptr;
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
-        const float xk = scale8(drawn);
-        const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
-        const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
+        float pu = q.pu, pr = q.pr, pe = q.pe;
+#pragma unroll
+        for (int k = 0; k < NP; ++k) {
+            const float xk = xin(drawn, k);                  // the pending input
+            pu = fmaf(q.ku[k], xk, pu); pr = fmaf(q.kr[k], xk, pr); pe = fmaf(q.ke[k], xk, pe);
+        }
+        const float u = sigmoidf_fast(pu), r = sigmoidf_fast(pr);
+        const float e = tanhf_fast(fmaf(r, q.ae, pe));
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
@@ -303,9 +339,15 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         int forced = -1;
         if (warp == 0) {
             if (lane < UC && !last) load_g(half, s, gv);
-            if (half) { if (p.c_forced) forced = p.c_forced[s]; }
-            else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
-            u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
+            if (FUSED) {
+                if (half) { if (p.a_forced) forced = p.a_forced[s]; }
+                else      { if (p.b_forced) forced = p.b_forced[s - 1]; }
+                u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), (half ? 0u : 4u) + (unsigned)(lane >> 3));
+            } else {
+                if (half) { if (p.c_forced) forced = p.c_forced[s]; }
+                else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
+                u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
+            }
             asm volatile("" : "+f"(u01), "+r"(forced), "+f"(gv[0]), "+f"(gv[1]), "+f"(gv[2]));
         }
 
@@ -367,7 +409,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         // ---- 4. the cluster's hidden layer -> this CTA's 16 output-layer rows in fp32: warps 8..15 take two rows each, a
         // lane the element pairs lane, lane + 32, ... of both (every shared-memory pass delivers 128 distinct bytes)
         GatePre gp = {};
-        if (warp >= 8) {
+        if (warp >= 8 && warp < 8 + RL_LR / 2) {
             if (!wait_arrival(&xq[par], use, (int)s, 2 + 4 * half)) my_bad = true;
             const int ra = 2 * (warp - 8);
             const unsigned *wa = L + ra * (K / 2) + lane, *wb = wa + K / 2;
@@ -406,26 +448,41 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
             if (!wait_arrival(&xl[par], use, (int)s, 3 + 4 * half)) my_bad = true;
             my_bad = __any_sync(FULL, my_bad);
             STAMP(8 * half + 6);
-            float l[8];
-            {
+            constexpr int NL = FUSED ? 2 : 8;
+            float l[NL];
+            int drawn;
+            if (FUSED) {
+                // 64 logits: two per lane; lanes [8 k, 8 k + 8) are the softmax of nibble k (most significant first)
+                const float2 a = reinterpret_cast<const float2 *>(lbuf + (size_t)par * RL_NLOG)[lane];
+                l[0] = a.x; l[1] = a.y;
+                const int nib = group16_softmax_draw(l[0], l[1], u01, lane);
+                drawn = (__shfl_sync(FULL, nib, 0) << 12) | (__shfl_sync(FULL, nib, 8) << 8) | (__shfl_sync(FULL, nib, 16) << 4) | __shfl_sync(FULL, nib, 24);
+            } else {
                 const float4 a = reinterpret_cast<const float4 *>(lbuf + (size_t)par * RL_NLOG)[2 * lane];
                 const float4 b = reinterpret_cast<const float4 *>(lbuf + (size_t)par * RL_NLOG)[2 * lane + 1];
-                l[0] = a.x; l[1] = a.y; l[2] = a.z; l[3] = a.w; l[4] = b.x; l[5] = b.y; l[6] = b.z; l[7] = b.w;
+                l[0] = a.x; l[1] = a.y; l[2] = a.z; l[3] = a.w; l[NL - 4] = b.x; l[NL - 3] = b.y; l[NL - 2] = b.z; l[NL - 1] = b.w;
+                drawn = warp_softmax_draw_fast(reinterpret_cast<const float (&)[8]>(l), u01, lane);
             }
-            const int drawn = warp_softmax_draw_fast(l, u01, lane);
             const int fed = forced >= 0 ? forced : drawn;
             if (lane < UC && !last && !my_bad) gates_and_publish(half, s, fed, gp);
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&pub_bar)) : "memory");
             if (writer) {
                 if (p.dbg_logits) {
-                    float *d = p.dbg_logits + (size_t)(n - 1) * RL_NLOG + 8 * lane;
+                    float *d = p.dbg_logits + (size_t)(n - 1) * RL_NLOG + NL * lane;
 #pragma unroll
-                    for (int k = 0; k < 8; ++k) d[k] = l[k];
+                    for (int k = 0; k < NL; ++k) d[k] = l[k];
                 }
                 if (lane == 0) {
-                    if (half) { if (p.c_out) p.c_out[s] = (uint8_t)drawn; }
-                    else      { if (p.f_out) p.f_out[s - 1] = (uint8_t)drawn; }
-                    if (!half && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + fed - 32768);
+                    if (FUSED) {
+                        if (half) { if (p.a_out) p.a_out[s] = (uint16_t)drawn; }
+                        else      { if (p.b_out) p.b_out[s - 1] = (uint16_t)drawn; }
+                        // the two streams side by side: out[0][s] = a_s, out[1][s] = the sample part B emits in step s
+                        if (p.out) p.out[(half ? 0 : T) + (half ? s : s - 1)] = (int16_t)(fed - 32768);
+                    } else {
+                        if (half) { if (p.c_out) p.c_out[s] = (uint8_t)drawn; }
+                        else      { if (p.f_out) p.f_out[s - 1] = (uint8_t)drawn; }
+                        if (!half && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + fed - 32768);
+                    }
                 }
             }
             if (half) c_prev = fed; else f_prev = fed;
@@ -443,14 +500,25 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
     if (writer && !any_bad) {
         if (p.h_out) for (int i = tid; i < K; i += blockDim.x) { p.h_out[i] = vecC[i]; p.h_out[K + i] = vecF[i]; }
         if (tid == 0) {
-            if (p.c_st_out) p.c_st_out[0] = (uint8_t)c_prev;
-            if (p.f_st_out) p.f_st_out[0] = (uint8_t)f_prev;
+            if (FUSED) {
+                if (p.a_st_out) p.a_st_out[0] = (uint16_t)c_prev;
+                if (p.b_st_out) p.b_st_out[0] = (uint16_t)f_prev;
+            } else {
+                if (p.c_st_out) p.c_st_out[0] = (uint8_t)c_prev;
+                if (p.f_st_out) p.f_st_out[0] = (uint8_t)f_prev;
+            }
         }
     }
     cluster.sync();     // nobody leaves while a peer may still write into its shared memory
 }
 
 // ---------------------------------------------------------------------------------------------
+static const void *kernel_of(const ResLeanPack &k)
+{
+    if (k.fused) return k.checked ? (const void *)resident_lean_kernel<true, true> : (const void *)resident_lean_kernel<false, true>;
+    return k.checked ? (const void *)resident_lean_kernel<true, false> : (const void *)resident_lean_kernel<false, false>;
+}
+
 static void fill_launch(const ResLeanPack &k, cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at, cudaStream_t s, bool coop)
 {
     std::memset(cfg, 0, sizeof(*cfg));
@@ -473,15 +541,18 @@ int reslean_supported(const wrnn_model *m, int batch)
 
 int reslean_prepare(wrnn_model *m)
 {
-    if (m->dtype != WRNN_BF16 || m->sparse || m->variant != 0 || m->H != 2 * RL_K) { m->err = "lean resident kernel: dense bf16 H = 896 only"; return WRNN_ERR_UNSUPPORTED; }
+    if (m->dtype != WRNN_BF16 || m->sparse || m->H != 2 * RL_K) { m->err = "lean resident kernel: dense bf16 H = 896 only"; return WRNN_ERR_UNSUPPORTED; }
+    const bool fused = m->variant == 1;
+    const int LR = rl_lr(fused), NIN = rl_nin(fused);
     ResLeanPack k;
+    k.fused = fused;
     k.NCTA = RL_K / RL_UC; k.NC = k.NCTA / RL_CS;
-    k.blob_bytes = RL_BLOB_BYTES; k.w_bytes = RL_W_BYTES; k.smem_bytes = (int)RL_SMEM_BYTES;
+    k.blob_bytes = rl_blob_bytes(fused); k.w_bytes = rl_w_bytes(fused); k.smem_bytes = (int)rl_smem_bytes(fused);
     cudaDeviceProp prop;
     cudaGetDeviceProperties(&prop, m->device);
     if (k.NCTA > m->n_sms || (size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "lean resident kernel does not fit this device"; return WRNN_ERR_UNSUPPORTED; }
     { const char *d = getenv("WRNN_DEBUG"); k.checked = d && d[0] == '1'; }
-    const void *fn = k.checked ? (const void *)resident_lean_kernel<true> : (const void *)resident_lean_kernel<false>;
+    const void *fn = kernel_of(k);
     if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
         cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes + (k.checked ? RL_N_GUARDS * 16 : 0)) != cudaSuccess) {
         cudaGetLastError(); m->err = "lean resident kernel: cannot set the launch attributes"; return WRNN_ERR_UNSUPPORTED;
@@ -525,19 +596,19 @@ int reslean_prepare(wrnn_model *m)
                 pack_tile(rows, K, wR + (size_t)mt * tile_elems);
             }
         }
-        // output layers: this CTA's 16 rows of O2 (O4), row-major
+        // output layers: this CTA's rows of O2 (O4), row-major
         uint16_t *wl = w + (size_t)8 * tile_elems;
         for (int h = 0; h < 2; ++h)
-            for (int r = 0; r < RL_LR; ++r) dense_row_bf16(*Ob[h], rank * RL_LR + r, 0, K, wl + ((size_t)h * RL_LR + r) * K);
+            for (int r = 0; r < LR; ++r) dense_row_bf16(*Ob[h], rank * LR + r, 0, K, wl + ((size_t)h * LR + r) * K);
         for (int rr = 0; rr < RL_NR; ++rr) {
             const int half = rr / (3 * UC), gate = (rr / UC) % 3, u = rr % UC;
             const int mrow = gate * H + half * K + cta * UC + u;
-            for (int c = 0; c < 3; ++c) sm[rr * 3 + c] = m->hI[(size_t)mrow * 3 + c];
+            for (int c = 0; c < NIN; ++c) sm[rr * NIN + c] = m->hI[(size_t)mrow * NIN + c];
         }
-        float *b = sm + RL_NR * 3;
+        float *b = sm + RL_NR * NIN;
         for (int r = 0; r < RL_HR; ++r) { b[r] = m->hb1[rank * RL_HR + r]; b[32 + r] = m->hb3[rank * RL_HR + r]; }
         b += 64;
-        for (int r = 0; r < RL_LR; ++r) { b[r] = m->hb2[rank * RL_LR + r]; b[RL_LR + r] = m->hb4[rank * RL_LR + r]; }
+        for (int r = 0; r < LR; ++r) { b[r] = m->hb2[rank * LR + r]; b[LR + r] = m->hb4[rank * LR + r]; }
     }
     ResLeanPack *pk = new ResLeanPack(k);
     bool ok = cudaMalloc((void **)&pk->d_blob, blob.size()) == cudaSuccess &&
@@ -590,6 +661,8 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.g = m->g; p.slots = k.d_slots;
     p.h_in = a.h_in; p.h_out = a.h_out; p.c_in = a.c_in; p.f_in = a.f_in; p.c_st_out = a.c_st_out; p.f_st_out = a.f_st_out;
     p.c_forced = a.c_forced; p.f_forced = a.f_forced; p.c_out = a.c_out; p.f_out = a.f_out; p.out = a.out;
+    p.a_in = a.a_in; p.b_in = a.b_in; p.a_st_out = a.a_st_out; p.b_st_out = a.b_st_out;
+    p.a_forced = a.a_forced; p.b_forced = a.b_forced; p.a_out = a.a_out; p.b_out = a.b_out;
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.frame_shift = a.row_lag > 0 ? a.step0 : 0;
     p.status = m->status;
@@ -603,7 +676,8 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     fill_launch(k, &cfg, at, s, coop_launch_allowed());
     p.smem_bytes = cfg.dynamicSmemBytes;
     { const char *d = getenv("WRNN_DEBUG_POKE"); p.chk_poke = (k.checked && d && d[0] == '1') ? 1 : 0; }
-    const cudaError_t e = k.checked ? cudaLaunchKernelEx(&cfg, resident_lean_kernel<true>, p) : cudaLaunchKernelEx(&cfg, resident_lean_kernel<false>, p);
+    void *args[] = {&p};
+    const cudaError_t e = cudaLaunchKernelExC(&cfg, kernel_of(k), args);
     if (e != cudaSuccess) {
         m->err = std::string("lean resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

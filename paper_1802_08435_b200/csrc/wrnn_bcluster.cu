@@ -531,7 +531,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 const float4 v1 = *reinterpret_cast<const float4 *>(s_log + warp * 256 + 8 * lane + 4);
                 l[0] = v0.x; l[1] = v0.y; l[2] = v0.z; l[3] = v0.w; l[4] = v1.x; l[5] = v1.y; l[6] = v1.z; l[7] = v1.w;
                 const float u = uniform24(p.seed, p.stream0 + (unsigned)s_gb, (unsigned long long)(p.step0 + s - (long long)s_gb * p.row_lag), head);
-                drawn = warp_softmax_draw_fast(l, u, lane);
+                drawn = warp_softmax_draw_scan(l, u, lane);
                 const uint8_t *forced = head ? p.f_forced : p.c_forced;
                 used = forced ? (int)forced[s_o] : drawn;
                 if (lane < BC_CS) {

@@ -128,7 +128,12 @@ __device__ __forceinline__ int float_order_key(float x)
     const int i = __float_as_int(x);
     return i ^ ((i >> 31) & 0x7fffffff);          // signed-integer order == float order
 }
-__device__ __forceinline__ int warp_softmax_draw_fast(const float (&l)[8], float u, int lane)
+// SCAN = false: exclusive prefix and grand total of the lane sums by one five-step butterfly (no broadcast after the scan;
+// the shorter chain where the drawing warp is alone on the critical path: the lean single-stream kernel).  SCAN = true: an
+// inclusive shuffle-up scan and a broadcast of the last lane's total (fewer instructions; faster where several warps draw
+// at once or other warps compete for issue slots: measured per kernel).  The two orders of summation differ in rounding only.
+template <bool SCAN>
+__device__ __forceinline__ int warp_softmax_draw_impl(const float (&l)[8], float u, int lane)
 {
     // (pairwise trees instead of chains: this sits on the critical path of every half-step)
     float m = fmaxf(fmaxf(fmaxf(l[0], l[1]), fmaxf(l[2], l[3])), fmaxf(fmaxf(l[4], l[5]), fmaxf(l[6], l[7])));
@@ -143,11 +148,22 @@ __device__ __forceinline__ int warp_softmax_draw_fast(const float (&l)[8], float
     // butterfly over the lanes: after step o every lane holds the total of its block of 2 o lanes and, in `run`, the sum of
     // the lanes of that block below itself -- the exclusive prefix and the grand total in five shuffles, no broadcast after
     float tot = p7, run = 0.f;
+    if (SCAN) {
+        float inc = p7;
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const float other = __shfl_xor_sync(FULL, tot, o);
-        if (lane & o) run += other;
-        tot += other;
+        for (int o = 1; o < 32; o <<= 1) {
+            const float t = __shfl_up_sync(FULL, inc, o);
+            if (lane >= o) inc += t;
+        }
+        tot = __shfl_sync(FULL, inc, 31);
+        run = inc - p7;                  // exclusive prefix of this lane
+    } else {
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float other = __shfl_xor_sync(FULL, tot, o);
+            if (lane & o) run += other;
+            tot += other;
+        }
     }
     const float thr = u * tot;
     int pick = 256;                      // last assignment wins: the smallest qualifying index
@@ -162,6 +178,8 @@ __device__ __forceinline__ int warp_softmax_draw_fast(const float (&l)[8], float
     pick = __reduce_min_sync(FULL, pick);
     return pick == 256 ? 255 : pick;
 }
+__device__ __forceinline__ int warp_softmax_draw_fast(const float (&l)[8], float u, int lane) { return warp_softmax_draw_impl<false>(l, u, lane); }
+__device__ __forceinline__ int warp_softmax_draw_scan(const float (&l)[8], float u, int lane) { return warp_softmax_draw_impl<true>(l, u, lane); }
 
 // Four softmaxes of 16 in one warp (the 4-bit heads of the Fused Subscale WaveRNN 2x): lane l holds logits 2 l, 2 l + 1 of
 // 64, lanes [8 k, 8 k + 8) form softmax k and share the uniform u.  Returns, on every lane, the index its group drew

@@ -105,7 +105,8 @@ __host__ __device__ constexpr size_t rl_smem_bytes(bool f)
 // would leave its array is skipped, and the kernel runs to its normal exit.
 constexpr int RL_N_GUARDS = 13;
 constexpr unsigned RL_GUARD_WORD = 0x5afec0deu;
-template <bool CHK, bool FUSED>
+// HOOK: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); the others have no trace of it
+template <bool CHK, bool FUSED, bool HOOK>
 __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanParams p)
 {
     constexpr int RL_NLOG = rl_nlog(FUSED), RL_LR = rl_lr(FUSED), NIN = rl_nin(FUSED), NP = NIN / 3;
@@ -278,7 +279,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         for (int k = 0; k < NP; ++k) { q.ku[k] = Iu[pend + k]; q.kr[k] = Ir[pend + k]; q.ke[k] = Ie[pend + k]; }
         return q;
     };
-    const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
+    const int skip_at = (HOOK && cta == p.skip_cta) ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
     const bool dbg_any = p.dbg_gates != nullptr || p.dbg_h != nullptr;
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
         float pu = q.pu, pr = q.pr, pe = q.pe;
@@ -294,7 +295,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
         const size_t slot = (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j;
         if (CHK && slot >= (size_t)4 * K) record_check(-1);                          // an exchange slot outside the slot array: skipped
-        else if ((int)s != skip_at)
+        else if (!HOOK || (int)s != skip_at)
             st_relaxed_u64(p.slots + slot, ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (dbg_any) {
             if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
@@ -513,10 +514,11 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
 }
 
 // ---------------------------------------------------------------------------------------------
-static const void *kernel_of(const ResLeanPack &k)
+static const void *kernel_of(const ResLeanPack &k, bool hook)
 {
-    if (k.fused) return k.checked ? (const void *)resident_lean_kernel<true, true> : (const void *)resident_lean_kernel<false, true>;
-    return k.checked ? (const void *)resident_lean_kernel<true, false> : (const void *)resident_lean_kernel<false, false>;
+    if (k.checked) return k.fused ? (const void *)resident_lean_kernel<true, true, false> : (const void *)resident_lean_kernel<true, false, false>;
+    if (hook) return k.fused ? (const void *)resident_lean_kernel<false, true, true> : (const void *)resident_lean_kernel<false, false, true>;
+    return k.fused ? (const void *)resident_lean_kernel<false, true, false> : (const void *)resident_lean_kernel<false, false, false>;
 }
 
 static void fill_launch(const ResLeanPack &k, cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at, cudaStream_t s, bool coop)
@@ -552,10 +554,13 @@ int reslean_prepare(wrnn_model *m)
     cudaGetDeviceProperties(&prop, m->device);
     if (k.NCTA > m->n_sms || (size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "lean resident kernel does not fit this device"; return WRNN_ERR_UNSUPPORTED; }
     { const char *d = getenv("WRNN_DEBUG"); k.checked = d && d[0] == '1'; }
-    const void *fn = kernel_of(k);
-    if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-        cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes + (k.checked ? RL_N_GUARDS * 16 : 0)) != cudaSuccess) {
-        cudaGetLastError(); m->err = "lean resident kernel: cannot set the launch attributes"; return WRNN_ERR_UNSUPPORTED;
+    const void *fn = kernel_of(k, false);
+    for (int hook = 0; hook < 2; ++hook) {
+        const void *f = kernel_of(k, hook != 0);
+        if (cudaFuncSetAttribute(f, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+            cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes + (k.checked ? RL_N_GUARDS * 16 : 0)) != cudaSuccess) {
+            cudaGetLastError(); m->err = "lean resident kernel: cannot set the launch attributes"; return WRNN_ERR_UNSUPPORTED;
+        }
     }
     {
         cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
@@ -677,7 +682,7 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.smem_bytes = cfg.dynamicSmemBytes;
     { const char *d = getenv("WRNN_DEBUG_POKE"); p.chk_poke = (k.checked && d && d[0] == '1') ? 1 : 0; }
     void *args[] = {&p};
-    const cudaError_t e = cudaLaunchKernelExC(&cfg, kernel_of(k), args);
+    const cudaError_t e = cudaLaunchKernelExC(&cfg, kernel_of(k, m->dbg_skip_cta >= 0), args);
     if (e != cudaSuccess) {
         m->err = std::string("lean resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

@@ -110,6 +110,8 @@ __device__ __forceinline__ void mma16816(float (&c)[4], const uint4 &a, unsigned
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ void named_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
+// HOOK: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); the production one has no trace of it
+template <bool HOOK>
 __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -294,7 +296,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         q.ku = half_g ? Iu[2] : Iu[1]; q.kr = half_g ? Ir[2] : Ir[1]; q.ke = half_g ? Ie[2] : Ie[1];
         return q;
     };
-    const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
+    const int skip_at = (HOOK && cta == p.skip_cta) ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
         const float xk = scale8(drawn);
         const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
@@ -304,7 +306,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         const int jj = (half_g ? K : 0) + gj;
         // published as the operand the 112 readers need: bf16 high and low parts, split once here
         const __nv_bfloat16 hh = __float2bfloat16_rn(hn), hl = __float2bfloat16_rn(hn - __bfloat162float(hh));
-        if ((int)s != skip_at)
+        if (!HOOK || (int)s != skip_at)
             st_relaxed_u64(p.slots + ((size_t)((half_g ? 2 : 0) + (s & 1)) * NS + gst) * K + gj,
                            ((unsigned long long)(unsigned)(s + 1) << 32) | (unsigned)__bfloat16_as_ushort(hh) | ((unsigned)__bfloat16_as_ushort(hl) << 16));
         if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * NS + gst) * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
@@ -655,8 +657,10 @@ int resmulti_prepare(wrnn_model *m)
     cudaDeviceProp prop;
     cudaGetDeviceProperties(&prop, m->device);
     if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin ||
-        cudaFuncSetAttribute(resident_multi_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-        cudaFuncSetAttribute(resident_multi_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
+        cudaFuncSetAttribute(resident_multi_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
         cudaGetLastError();
         m->err = "multi-stream resident kernel does not fit in shared memory";
         return WRNN_ERR_UNSUPPORTED;
@@ -665,7 +669,7 @@ int resmulti_prepare(wrnn_model *m)
         cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
         multi_fill_launch(k, &cfg, at, 0, false);
         int max_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_multi_kernel, &cfg) != cudaSuccess || max_clusters < MNC) {
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_multi_kernel<false>, &cfg) != cudaSuccess || max_clusters < MNC) {
             cudaGetLastError();
             m->err = "not enough co-resident clusters for the multi-stream resident kernel";
             return WRNN_ERR_UNSUPPORTED;
@@ -800,7 +804,7 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     multi_fill_launch(k, &cfg, at, s, coop_launch_allowed());
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, resident_multi_kernel, p);
+    const cudaError_t e = m->dbg_skip_cta >= 0 ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<true>, p) : cudaLaunchKernelEx(&cfg, resident_multi_kernel<false>, p);
     if (e != cudaSuccess) {
         m->err = std::string("multi-stream resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

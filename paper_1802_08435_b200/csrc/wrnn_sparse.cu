@@ -80,7 +80,8 @@ __device__ long long g_sprof[16];
 #endif
 
 // NKL: k-tiles of the logits tile per warp (K / 16 / NKL warps split K).
-template <int NKL>
+// HOOK: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); the production one has no trace of it
+template <int NKL, bool HOOK>
 __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const SparseParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -269,7 +270,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         }
         return q;
     };
-    const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
+    const int skip_at = (HOOK && cta == p.skip_cta) ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
     auto gates = [&](int half_g, long long s, int drawn, const GatePre &q) {
         if (lane < UW) {
             const int u0 = warp * UW + lane;
@@ -278,7 +279,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             const float e = tanhf_fast(fmaf(r, q.ae, fmaf(q.ke, xk, q.pe)));
             const float hn = fmaf(u, q.hprev, (1.0f - u) * e);
             // published to the whole chip: arrival of the tagged value is the signal (two-deep by step parity)
-            if ((int)s != skip_at)
+            if (!HOOK || (int)s != skip_at)
                 st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + cta * UC + u0,
                                ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
             const int jj = (half_g ? K : 0) + cta * UC + u0;
@@ -415,7 +416,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             }
             my_bad = __any_sync(FULL, my_bad);
             SSTAMP(4);
-            int drawn = warp_softmax_draw_fast(l, u01, lane);
+            int drawn = warp_softmax_draw_scan(l, u01, lane);
             if (writer && warp == 0) {
                 if (p.dbg_logits) {
                     float *d = p.dbg_logits + (size_t)(n - 1) * 256 + 8 * lane;
@@ -482,7 +483,7 @@ int sparse_supported(const wrnn_model *m, int batch, std::string *why)
     return WRNN_OK;
 }
 
-static void *sparse_fn() { return (void *)sparse_cluster_kernel<8>; }
+static void *sparse_fn(bool hook) { return hook ? (void *)sparse_cluster_kernel<8, true> : (void *)sparse_cluster_kernel<8, false>; }
 
 static void sparse_fill_launch(const SparsePack &k, cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at, cudaStream_t s, bool coop)
 {
@@ -633,14 +634,16 @@ int sparse_prepare(wrnn_model *m)
         cudaDeviceProp prop;
         cudaGetDeviceProperties(&prop, m->device);
         if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "pruned model does not fit the shared memory of the clusters"; return WRNN_ERR_UNSUPPORTED; }
-        if (cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-            cudaFuncSetAttribute(sparse_fn(), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
+        if (cudaFuncSetAttribute(sparse_fn(false), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+            cudaFuncSetAttribute(sparse_fn(false), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess ||
+            cudaFuncSetAttribute(sparse_fn(true), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+            cudaFuncSetAttribute(sparse_fn(true), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
             cudaGetLastError(); m->err = "cannot configure the 16-CTA cluster kernel"; return WRNN_ERR_UNSUPPORTED;
         }
         cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
         sparse_fill_launch(k, &cfg, at, 0, false);
         int max_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, sparse_fn(), &cfg) != cudaSuccess || max_clusters < nc) {
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, sparse_fn(false), &cfg) != cudaSuccess || max_clusters < nc) {
             cudaGetLastError(); m->err = "the 16-CTA clusters cannot all be co-resident on this device"; return WRNN_ERR_UNSUPPORTED;
         }
 
@@ -781,7 +784,8 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     sparse_fill_launch(k, &cfg, at, s, coop_launch_allowed());
-    cudaError_t e = cudaLaunchKernelEx(&cfg, sparse_cluster_kernel<8>, p);
+    void *args[] = {&p};
+    cudaError_t e = cudaLaunchKernelExC(&cfg, sparse_fn(m->dbg_skip_cta >= 0), args);
     if (e != cudaSuccess) {
         m->err = std::string("sparse cluster kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

@@ -70,6 +70,7 @@ struct SparseParams {
     DevStatus *status;
     unsigned long long limit_ns;
     int skip_cta; long long skip_step;      // self-test: this CTA withholds what it publishes at this step (-1: none)
+    int poll_gap;                           // cycles the state pollers hold back after the CTA's own publication (-1: poll at once, all warps)
 };
 
 #ifdef WRNN_PROFILE_SPARSE
@@ -89,14 +90,14 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     const int rank = (int)cluster.block_rank();      // owner index of head rows and logits (per cluster)
     const int cta = blockIdx.x;                      // owner index of state units and their rows of R (whole grid)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int K = p.K, NKT = p.NKT, UC = p.UC, HR = p.HR, H = p.H;
+    const int K = p.K, UC = p.UC, HR = p.HR, H = p.H;
     const int NR = 6 * UC;
 
     // ---- shared memory carve-up (must match sparse_smem_bytes)
     const SliceMeta *smeta[2] = {reinterpret_cast<const SliceMeta *>(smem + p.off_meta[0]), reinterpret_cast<const SliceMeta *>(smem + p.off_meta[1])};
     const uint16_t *bcol[2] = {reinterpret_cast<const uint16_t *>(smem + p.off_col[0]), reinterpret_cast<const uint16_t *>(smem + p.off_col[1])};
     const uint4 *bval[2] = {reinterpret_cast<const uint4 *>(smem + p.off_val[0]), reinterpret_cast<const uint4 *>(smem + p.off_val[1])};
-    const uint4 *wO2 = reinterpret_cast<const uint4 *>(smem + p.off_o2), *wO4 = reinterpret_cast<const uint4 *>(smem + p.off_o4);
+    const unsigned *wO2 = reinterpret_cast<const unsigned *>(smem + p.off_o2), *wO4 = reinterpret_cast<const unsigned *>(smem + p.off_o4);   // [16 rows][K / 2] bf16 pairs
     const float *sI = reinterpret_cast<const float *>(smem + p.off_small);            // [NR][3]
     const float *sb1 = sI + NR * 3, *sb3 = sb1 + HR, *sb2 = sb3 + HR, *sb4 = sb2 + 16;
     float *vecC = reinterpret_cast<float *>(smem + p.blob_bytes);                     // [K] y_c
@@ -105,11 +106,11 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     float *a_part = qvec + K;                                                         // [NR]
     float *a_full = a_part + NR;                                                      // [NR]
     float *part = a_full + NR;                                                        // [16 warps][16]
-    __nv_bfloat16 *splQ = reinterpret_cast<__nv_bfloat16 *>(part + 256);              // split image of q, 4 K bf16
+    float *qall = part + 256;                                                         // [2 parities][K] the cluster's hidden layer, written by the peers' asynchronous stores
     // Cluster exchange buffers, one of each: a peer can only write the next half-step's words after it has received
     // words that this CTA sent after reading the current ones (q(n+1) follows y(n+1), which follows this CTA's draw from
     // logits(n); logits(n+1) follow q(n+1)).
-    uint4 *qbuf = reinterpret_cast<uint4 *>(splQ + 4 * K);                            // [K/2] hidden layer
+    uint4 *qbuf = reinterpret_cast<uint4 *>(qall + 2 * K);                            // [K/2] hidden layer
     uint4 *lbuf = qbuf + K / 2;                                                       // [128] logits
 
     {
@@ -117,7 +118,6 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         uint4 *dst = reinterpret_cast<uint4 *>(smem);
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
         for (int i = tid; i < K / 2 + 128; i += blockDim.x) qbuf[i] = make_uint4(0, 0, 0, 0);   // qbuf, lbuf are adjacent
-        for (int i = tid; i < 4 * K / 8; i += blockDim.x) reinterpret_cast<uint4 *>(splQ)[i] = make_uint4(0, 0, 0, 0);
         for (int i = tid; i < K; i += blockDim.x) {
             vecC[i] = p.h_in ? p.h_in[i] : 0.f;
             vecF[i] = p.h_in ? p.h_in[K + i] : 0.f;
@@ -129,6 +129,15 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
     const bool writer = (cta == 0);
+    __shared__ __align__(8) unsigned long long pub_bar;      // one phase per half-step: this CTA's gate warps have published
+    __shared__ __align__(8) unsigned long long xq[2];        // arrival barriers of qall[.]: the peers' stores count their bytes here
+    if (tid == 0) {
+        mbar_init_cluster(smem_addr(&pub_bar), (unsigned)((p.UC + 31) / 32));
+        mbar_init_cluster(smem_addr(&xq[0]), 1); mbar_init_cluster(smem_addr(&xq[1]), 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    cluster.sync();      // every peer's barriers are initialised before anyone sends
 #ifdef WRNN_PROFILE_SPARSE
     __shared__ long long s_sprof[16];
     long long st_ = clock64();
@@ -296,11 +305,9 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         float gv0[3] = {0.f, 0.f, 0.f};
         if (lane < UW) load_g(0, 0, gv0);
         gates(0, 0, f_prev, gates_prepare(0, gv0));
+        if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&pub_bar)) : "memory");
     }
 
-    const int l_kt0 = warp * NKL;
-    const int KSL = NKT / NKL;                   // warps that split K of the logits tile
-    const bool l_on = warp < KSL;
 
 #ifdef WRNN_PROFILE_SPARSE
     if (tid < 16) s_sprof[tid] = 0;
@@ -316,6 +323,8 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         const unsigned tag = (unsigned)n;
         float *vec = half ? vecC : vecF;
 
+        const unsigned par = (unsigned)((n - 1) & 1), use = (unsigned)((n - 1) >> 1);
+        if (tid == 0) mbar_arrive_expect(smem_addr(&xq[par]), (unsigned)K * 4u);      // this half-step's arrivals: K hidden values
         float u01 = 0.f, gv[3] = {0.f, 0.f, 0.f};
         int forced = -1;
         if (warp < GW) {
@@ -330,15 +339,30 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         {
             const unsigned long long *slots = p.yslots + (size_t)(half ? (s & 1) : 2 + ((s - 1) & 1)) * K;
             const unsigned ytag = (unsigned)(half ? s + 1 : s);
-#pragma unroll 1
-            for (int i = tid; i < K / 2; i += blockDim.x) {
-                unsigned long long v0, v1, t0 = 0; unsigned cnt = 0;
-                while (true) {
-                    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0), "=l"(v1) : "l"(slots + 2 * i) : "memory");
-                    if ((unsigned)(v0 >> 32) == ytag && (unsigned)(v1 >> 32) == ytag) break;
-                    if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+            // Polls that come before the data only load the L2 slices the publishing stores have to get through, and a poll
+            // that just misses the data costs a whole round trip: the pollers (every warp but the drawing ones, which have
+            // the longest way to the end of the half-step) hold back until this CTA's own gate warps have published (all
+            // CTAs publish at about the same time) plus poll_gap cycles.
+            const bool held = p.poll_gap >= 0;
+            const int first = held ? 32 * GW : 0, stride = (int)blockDim.x - first;
+            if (tid >= first) {
+                if (held) {
+                    unsigned long long t0 = 0; unsigned cnt = 0;
+                    while (!mbar_try_parity(smem_addr(&pub_bar), (unsigned)((n - 1) & 1)))
+                        if ((++cnt & 1023u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+                    const long long c0 = clock64();
+                    while (clock64() - c0 < p.poll_gap) { }
                 }
-                vec[2 * i] = __uint_as_float((unsigned)v0); vec[2 * i + 1] = __uint_as_float((unsigned)v1);
+#pragma unroll 1
+                for (int i = tid - first; i < K / 2 && !my_bad; i += stride) {
+                    unsigned long long v0, v1, t0 = 0; unsigned cnt = 0;
+                    while (true) {
+                        asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v0), "=l"(v1) : "l"(slots + 2 * i) : "memory");
+                        if ((unsigned)(v0 >> 32) == ytag && (unsigned)(v1 >> 32) == ytag) break;
+                        if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 1 + 4 * half)) { my_bad = true; break; }
+                    }
+                    vec[2 * i] = __uint_as_float((unsigned)v0); vec[2 * i + 1] = __uint_as_float((unsigned)v1);
+                }
             }
         }
         if (__syncthreads_or(my_bad)) break;
@@ -350,43 +374,81 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         __syncthreads();
         SSTAMP(8);
         // this CTA's HR hidden-layer values -> every peer, one coalesced 16-byte-per-lane store per peer (warp w -> peer w)
+        // (asynchronous stores that count their bytes on the receiver's barrier of that buffer: no tags, no polling pass)
         if (warp < SCS) {
+            const unsigned bar = map_to_rank(smem_addr(&xq[par]), warp);
             for (int pr2 = lane; pr2 < HR / 2; pr2 += 32) {
-                const unsigned a = map_to_rank(smem_addr(qbuf + (rank * HR) / 2 + pr2), warp);
-                st_cluster_ll(a, qvec[2 * pr2], qvec[2 * pr2 + 1], tag);
+                const unsigned a = map_to_rank(smem_addr(qall + (size_t)par * K + rank * HR + 2 * pr2), warp);
+                st_async_v2(a, qvec[2 * pr2], qvec[2 * pr2 + 1], bar);
             }
         }
         SSTAMP(1);
 
         // ---- 3. the cluster's hidden layer -> 16 logits rows of this CTA
-#pragma unroll 1
-        for (int i = tid; i < K / 2; i += blockDim.x) {
-            const unsigned a = smem_addr(qbuf + i);
-            uint4 v; unsigned long long t0 = 0; unsigned cnt = 0;
-            while (true) {
-                v = ld_shared_volatile_v4(a);
-                if (v.y == tag && v.w == tag) break;
-                if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 2 + 4 * half)) { my_bad = true; break; }
+        SSTAMP(2);
+        // the 16 output-layer rows in fp32 FMAs on 16 warps: warp w takes rows 4 (w & 3) .. + 3 over quarter w >> 2 of the
+        // element pairs; a lane takes pairs lane, lane + 32, ... of its quarter (a pass costs a warp some 75 cycles whatever
+        // it computes, so the passes are spread over all warps: four each at K = 1024); every pair of the hidden layer is
+        // loaded once per four rows.  The four partial sums of a row meet in `part`.
+        if (warp < 16) {
+#ifdef WRNN_PROFILE_SPARSE
+            const long long rt0_ = clock64();
+#endif
+            {
+                unsigned long long t0 = 0; unsigned cnt = 0;
+                while (!mbar_try_parity(smem_addr(&xq[par]), use & 1u))
+                    if ((++cnt & 1023u) == 0 && wt.expired(t0, (int)s, 2 + 4 * half)) { my_bad = true; break; }
             }
-            store_split(splQ, 2 * i, __uint_as_float(v.x));
-            store_split(splQ, 2 * i + 1, __uint_as_float(v.z));
+            const int r0 = 4 * (warp & 3), kq = warp >> 2;
+            const int Kp = K / 2, n_pass = (Kp + 31) / 32, npq = (n_pass + 3) / 4;
+            const unsigned *wr = (half ? wO2 : wO4) + (size_t)r0 * Kp + lane;
+            const float2 *q2 = reinterpret_cast<const float2 *>(qall + (size_t)par * K) + lane;
+            float a[4][2] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+            const int j_end = min((kq + 1) * npq, n_pass);
+#ifdef WRNN_PROFILE_SPARSE
+            const long long rt1_ = clock64();
+            if (warp == 4 && lane == 0) s_sprof[12] += rt1_ - rt0_;
+#endif
+#pragma unroll 4
+            for (int j = kq * npq; j < j_end; ++j) {
+                if (32 * j + lane < Kp) {
+                    const float2 q = q2[32 * j];
+#pragma unroll
+                    for (int r = 0; r < 4; ++r) {
+                        const unsigned x = wr[r * Kp + 32 * j];
+                        a[r][0] = fmaf(bf16lo(x), q.x, a[r][0]); a[r][1] = fmaf(bf16hi(x), q.y, a[r][1]);
+                    }
+                }
+            }
+#ifdef WRNN_PROFILE_SPARSE
+            const long long rt2_ = clock64();
+            if (warp == 4 && lane == 0) s_sprof[13] += rt2_ - rt1_;
+#endif
+            // four sums across the warp: two transposing steps leave row (lane >> 3) & 3 in every lane, three more finish it
+            float v4[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) v4[r] = a[r][0] + a[r][1];
+            const bool u16 = (lane & 16) != 0, u8 = (lane & 8) != 0;
+            const float t0 = (u16 ? v4[2] : v4[0]) + __shfl_xor_sync(FULL, u16 ? v4[0] : v4[2], 16);
+            const float t1 = (u16 ? v4[3] : v4[1]) + __shfl_xor_sync(FULL, u16 ? v4[1] : v4[3], 16);
+            float v = (u8 ? t1 : t0) + __shfl_xor_sync(FULL, u8 ? t0 : t1, 8);
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+            const int rr = r0 + (u16 ? 2 : 0) + (u8 ? 1 : 0);
+            if ((lane & 7) == 0) part[kq * 16 + rr] = v;
+#ifdef WRNN_PROFILE_SPARSE
+            if (warp == 4 && lane == 0) s_sprof[11] += clock64() - rt0_;
+#endif
         }
         if (__syncthreads_or(my_bad)) break;
-        SSTAMP(2);
-        if (l_on) {
-            float lo, hi;
-            mma_partial<NKL>(half ? wO2 : wO4, l_kt0, splQ, lane, lo, hi);
-            if ((lane & 3) == 0) { part[warp * 16 + (lane >> 2)] = lo; part[warp * 16 + (lane >> 2) + 8] = hi; }
-        }
-        __syncthreads();
         SSTAMP(3);
         if (warp == GW) {
-            // 16 logits of this CTA: lanes 0..7 finish one pair of rows each, then every peer gets the 8 pairs as one
-            // contiguous 128-byte piece (four store instructions, four peers each)
-            const float *bl = half ? sb2 : sb4;
+            // 16 logits of this CTA: every peer gets the 8 pairs as one contiguous 128-byte piece (four store instructions,
+            // four peers each)
             const int r = 2 * (lane & 7);
-            float v0 = bl[r], v1 = bl[r + 1];
-            for (int w = 0; w < KSL; ++w) { v0 += part[w * 16 + r]; v1 += part[w * 16 + r + 1]; }
+            const float *bl = half ? sb2 : sb4;
+            const float v0 = bl[r] + (part[r] + part[16 + r]) + (part[32 + r] + part[48 + r]);
+            const float v1 = bl[r + 1] + (part[r + 1] + part[17 + r]) + (part[33 + r] + part[49 + r]);
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 const int peer = 4 * k + (lane >> 3);
@@ -435,6 +497,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             }
             SSTAMP(5);
             if (!last && !my_bad) gates(half, s, drawn, gp);
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&pub_bar)) : "memory");
             if (half) c_prev = drawn;
             SSTAMP(6);
         }
@@ -463,7 +526,7 @@ static int sparse_smem_bytes(const SparsePack &k)
     b += (size_t)3 * k.K * 4;                      // vecC, vecF, qvec
     b += (size_t)2 * 6 * k.UC * 4;                 // a_part, a_full
     b += 256 * 4;                                  // part
-    b += (size_t)4 * k.K * 2;                      // split image of q
+    b += (size_t)2 * k.K * 4;                      // the cluster's hidden layer (K floats in use)
     b += (size_t)k.K * 8;                          // qbuf: [K/2] x 16 B
     b += 128 * 16;                                 // lbuf
     return (int)b;
@@ -681,7 +744,7 @@ int sparse_prepare(wrnn_model *m)
                 // every kept block of R once; the heads once (cluster 0 stands for all)
                 kept_bytes += cta < SCS ? (int64_t)n * 34 + (int64_t)(NBR + 1) * 4 : (int64_t)n_r * 34;
             }
-            // dense O2 / O4: 16 rows of this CTA as one tile of A fragments (natural column order)
+            // dense O2 / O4: 16 rows of this CTA, row-major bf16
             for (int h = 0; h < 2; ++h) {
                 uint16_t *dst = reinterpret_cast<uint16_t *>(base + (h ? k.off_o4 : k.off_o2));
                 std::vector<uint16_t> dense((size_t)16 * Hh, 0);
@@ -691,14 +754,7 @@ int sparse_prepare(wrnn_model *m)
                     for (int i = M.row_ptr[br]; i < M.row_ptr[br + 1]; ++i)
                         for (int c = 0; c < 4; ++c) dense[(size_t)r * Hh + 4 * M.col[i] + c] = bf16_bits_s(M.vals[(size_t)i * 16 + 4 * rr + c]);
                 }
-                for (int kt = 0; kt < k.NKT; ++kt)
-                    for (int lane = 0; lane < 32; ++lane) {
-                        const int g = lane >> 2, t = lane & 3;
-                        uint16_t *o = dst + ((size_t)kt * 32 + lane) * 8;
-                        const int rsel[4] = {g, g + 8, g, g + 8}, csel[4] = {2 * t, 2 * t, 2 * t + 8, 2 * t + 8};
-                        for (int q = 0; q < 4; ++q)
-                            for (int j = 0; j < 2; ++j) o[2 * q + j] = dense[(size_t)rsel[q] * Hh + 16 * kt + csel[q] + j];
-                    }
+                std::memcpy(dst, dense.data(), dense.size() * 2);
             }
             float *sm = reinterpret_cast<float *>(base + k.off_small);
             for (int rr = 0; rr < 6 * UC; ++rr) {
@@ -779,6 +835,7 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.dbg_gates = a.dbg_gates; p.dbg_h = a.dbg_h; p.dbg_logits = a.dbg_logits;
     p.status = m->status;
     p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
+    { const char *e = getenv("WRNN_SPARSE_POLL_GAP"); p.poll_gap = e ? atoi(e) : 0; }
 
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * k.K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;

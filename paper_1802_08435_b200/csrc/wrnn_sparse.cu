@@ -4,8 +4,9 @@
 //
 // A pruned model is small (H = 2048 at 96 %: 2.3 MB of blocks, plus the dense O2 / O4).  The compressed block rows of R
 // are dealt over all NC x 16 CTAs; the heads are held once per cluster, so that the hidden layer of a head and its
-// logits are all-gathers of (value, tag) words through the distributed shared memory of a cluster; the two halves of
-// the state cross the chip as tagged words in L2 (arrival of the data is the signal).
+// logits are all-gathers through the distributed shared memory of a cluster (asynchronous stores that count their bytes
+// on an mbarrier of the receiver); the two halves of the state cross the chip as tagged words in L2 (arrival of the data is
+// the signal).
 // Each CTA owns Hh/(16 NC) coarse and as many fine units (their block rows of R, compressed: block column index +
 // 16 bf16 per kept block), Hh/16 rows of O1 and O3 (compressed block rows) and 16 rows of the dense O2 and O4
 // (mma.sync A fragments).  Sparse rows: four lanes share a block row, each lane takes every fourth kept block
@@ -111,13 +112,12 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     // words that this CTA sent after reading the current ones (q(n+1) follows y(n+1), which follows this CTA's draw from
     // logits(n); logits(n+1) follow q(n+1)).
     uint4 *qbuf = reinterpret_cast<uint4 *>(qall + 2 * K);                            // [K/2] hidden layer
-    uint4 *lbuf = qbuf + K / 2;                                                       // [128] logits
+    float *lall = reinterpret_cast<float *>(qbuf + K / 2);                            // [2 parities][256] logits of the cluster
 
     {
         const uint4 *src = reinterpret_cast<const uint4 *>(p.blob + (size_t)cta * p.blob_bytes);
         uint4 *dst = reinterpret_cast<uint4 *>(smem);
         for (size_t i = tid; i < p.blob_bytes / 16; i += blockDim.x) dst[i] = __ldg(src + i);
-        for (int i = tid; i < K / 2 + 128; i += blockDim.x) qbuf[i] = make_uint4(0, 0, 0, 0);   // qbuf, lbuf are adjacent
         for (int i = tid; i < K; i += blockDim.x) {
             vecC[i] = p.h_in ? p.h_in[i] : 0.f;
             vecF[i] = p.h_in ? p.h_in[K + i] : 0.f;
@@ -130,10 +130,11 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     bool my_bad = false;
     const bool writer = (cta == 0);
     __shared__ __align__(8) unsigned long long pub_bar;      // one phase per half-step: this CTA's gate warps have published
-    __shared__ __align__(8) unsigned long long xq[2];        // arrival barriers of qall[.]: the peers' stores count their bytes here
+    __shared__ __align__(8) unsigned long long xq[2], xl[2]; // arrival barriers of qall[.] and lall[.]: the peers' stores count their bytes here
     if (tid == 0) {
         mbar_init_cluster(smem_addr(&pub_bar), (unsigned)((p.UC + 31) / 32));
         mbar_init_cluster(smem_addr(&xq[0]), 1); mbar_init_cluster(smem_addr(&xq[1]), 1);
+        mbar_init_cluster(smem_addr(&xl[0]), 1); mbar_init_cluster(smem_addr(&xl[1]), 1);
         mbar_fence_init();
     }
     __syncthreads();
@@ -320,11 +321,13 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         const int half = (int)(n & 1);                 // 1: coarse half (input y_c(s)), 0: fine half (input y_f(s-1))
         const long long s = n >> 1;
         const bool last = n == 2 * T;
-        const unsigned tag = (unsigned)n;
         float *vec = half ? vecC : vecF;
 
         const unsigned par = (unsigned)((n - 1) & 1), use = (unsigned)((n - 1) >> 1);
-        if (tid == 0) mbar_arrive_expect(smem_addr(&xq[par]), (unsigned)K * 4u);      // this half-step's arrivals: K hidden values
+        if (tid == 0) {
+            mbar_arrive_expect(smem_addr(&xq[par]), (unsigned)K * 4u);      // this half-step's arrivals: K hidden values
+            mbar_arrive_expect(smem_addr(&xl[par]), 256u * 4u);             // and 256 logits
+        }
         float u01 = 0.f, gv[3] = {0.f, 0.f, 0.f};
         int forced = -1;
         if (warp < GW) {
@@ -400,24 +403,33 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
                     if ((++cnt & 1023u) == 0 && wt.expired(t0, (int)s, 2 + 4 * half)) { my_bad = true; break; }
             }
             const int r0 = 4 * (warp & 3), kq = warp >> 2;
-            const int Kp = K / 2, n_pass = (Kp + 31) / 32, npq = (n_pass + 3) / 4;
-            const unsigned *wr = (half ? wO2 : wO4) + (size_t)r0 * Kp + lane;
-            const float2 *q2 = reinterpret_cast<const float2 *>(qall + (size_t)par * K) + lane;
+            const int Kp = K / 2, Q = Kp / 4;               // element pairs of a row and of a quarter (Q is a multiple of 64 at K = 1024)
             float a[4][2] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
-            const int j_end = min((kq + 1) * npq, n_pass);
 #ifdef WRNN_PROFILE_SPARSE
             const long long rt1_ = clock64();
             if (warp == 4 && lane == 0) s_sprof[12] += rt1_ - rt0_;
 #endif
-#pragma unroll 4
-            for (int j = kq * npq; j < j_end; ++j) {
-                if (32 * j + lane < Kp) {
-                    const float2 q = q2[32 * j];
+            // in every run of 64 pairs a lane takes pairs 2 l and 2 l + 1: one 16-byte load of the hidden layer, one 8-byte load
+            // of each row's weights (all of them conflict-free), issued for the whole quarter before the first FMA
+            {
+                const float4 *q4 = reinterpret_cast<const float4 *>(qall + (size_t)par * K) + (size_t)kq * (Q / 2) + lane;
+                const uint2 *w2 = reinterpret_cast<const uint2 *>((half ? wO2 : wO4) + (size_t)r0 * Kp + (size_t)kq * Q) + lane;
+                for (int c0 = 0; c0 < Q / 64; c0 += 2) {
+                    float4 q[2];
+                    uint2 x[2][4];
 #pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        const unsigned x = wr[r * Kp + 32 * j];
-                        a[r][0] = fmaf(bf16lo(x), q.x, a[r][0]); a[r][1] = fmaf(bf16hi(x), q.y, a[r][1]);
+                    for (int u = 0; u < 2; ++u) {
+                        q[u] = q4[32 * (c0 + u)];
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) x[u][r] = w2[(size_t)r * (Kp / 2) + 32 * (c0 + u)];
                     }
+#pragma unroll
+                    for (int u = 0; u < 2; ++u)
+#pragma unroll
+                        for (int r = 0; r < 4; ++r) {
+                            a[r][0] = fmaf(bf16lo(x[u][r].x), q[u].x, a[r][0]); a[r][1] = fmaf(bf16hi(x[u][r].x), q[u].y, a[r][1]);
+                            a[r][0] = fmaf(bf16lo(x[u][r].y), q[u].z, a[r][0]); a[r][1] = fmaf(bf16hi(x[u][r].y), q[u].w, a[r][1]);
+                        }
                 }
             }
 #ifdef WRNN_PROFILE_SPARSE
@@ -442,19 +454,13 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         }
         if (__syncthreads_or(my_bad)) break;
         SSTAMP(3);
-        if (warp == GW) {
-            // 16 logits of this CTA: every peer gets the 8 pairs as one contiguous 128-byte piece (four store instructions,
-            // four peers each)
-            const int r = 2 * (lane & 7);
+        // 16 logits of this CTA: warp w sums the four partials of two rows per lane and sends the eight pairs to peer w
+        if (warp < SCS && lane < 8) {
+            const int r = 2 * lane;
             const float *bl = half ? sb2 : sb4;
             const float v0 = bl[r] + (part[r] + part[16 + r]) + (part[32 + r] + part[48 + r]);
             const float v1 = bl[r + 1] + (part[r + 1] + part[17 + r]) + (part[33 + r] + part[49 + r]);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int peer = 4 * k + (lane >> 3);
-                const unsigned a = map_to_rank(smem_addr(lbuf + (rank * 16) / 2 + (lane & 7)), peer);
-                st_cluster_ll(a, v0, v1, tag);
-            }
+            st_async_v2(map_to_rank(smem_addr(lall + (size_t)par * 256 + rank * 16 + r), warp), v0, v1, map_to_rank(smem_addr(&xl[par]), warp));
         }
 
         // ---- 4. warps 0..GW-1: the cluster's 256 logits -> draw; then the gates of the other half, published to the cluster
@@ -462,19 +468,12 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             const GatePre gp = gates_prepare(half, gv);
             float l[8];
             {
-                // the four slots of this lane are loaded together and re-read until all of them carry this half-step's tag
-                const unsigned a = smem_addr(lbuf + 4 * lane);
-                uint4 v0, v1, v2, v3;
                 unsigned long long t0 = 0; unsigned cnt = 0;
-                while (true) {
-                    v0 = ld_shared_volatile_v4(a); v1 = ld_shared_volatile_v4(a + 16);
-                    v2 = ld_shared_volatile_v4(a + 32); v3 = ld_shared_volatile_v4(a + 48);
-                    const bool ok = v0.y == tag && v0.w == tag && v1.y == tag && v1.w == tag && v2.y == tag && v2.w == tag && v3.y == tag && v3.w == tag;
-                    if (ok) break;
-                    if ((++cnt & 4095u) == 0 && wt.expired(t0, (int)s, 3 + 4 * half)) { my_bad = true; break; }
-                }
-                l[0] = __uint_as_float(v0.x); l[1] = __uint_as_float(v0.z); l[2] = __uint_as_float(v1.x); l[3] = __uint_as_float(v1.z);
-                l[4] = __uint_as_float(v2.x); l[5] = __uint_as_float(v2.z); l[6] = __uint_as_float(v3.x); l[7] = __uint_as_float(v3.z);
+                while (!mbar_try_parity(smem_addr(&xl[par]), use & 1u))
+                    if ((++cnt & 1023u) == 0 && wt.expired(t0, (int)s, 3 + 4 * half)) { my_bad = true; break; }
+                const float4 a = reinterpret_cast<const float4 *>(lall + (size_t)par * 256)[2 * lane];
+                const float4 b = reinterpret_cast<const float4 *>(lall + (size_t)par * 256)[2 * lane + 1];
+                l[0] = a.x; l[1] = a.y; l[2] = a.z; l[3] = a.w; l[4] = b.x; l[5] = b.y; l[6] = b.z; l[7] = b.w;
             }
             my_bad = __any_sync(FULL, my_bad);
             SSTAMP(4);
@@ -528,7 +527,7 @@ static int sparse_smem_bytes(const SparsePack &k)
     b += 256 * 4;                                  // part
     b += (size_t)2 * k.K * 4;                      // the cluster's hidden layer (K floats in use)
     b += (size_t)k.K * 8;                          // qbuf: [K/2] x 16 B
-    b += 128 * 16;                                 // lbuf
+    b += 128 * 16;                                 // lall: [2][256] floats
     return (int)b;
 }
 

@@ -41,6 +41,7 @@ struct SliceMeta { int voff, coff, T, nl, lpr, pad[3]; int16_t row[8]; };   // o
 
 struct SparsePack {
     int H = 0, K = 0, NKT = 0, UC = 0, HR = 0, NBR = 0;   // NBR: block rows per phase = (HR + 6 UC) / rows of a block
+    int WH = 0;                       // > 0: split layout (hidden-layer block rows in the slices of warps [0, WH), rows of R in those of warps 16..19)
     int NC = 1;                       // clusters: the rows of R are dealt over NC x 16 CTAs, the heads once per cluster
     unsigned long long *d_slots = nullptr;   // [4][K] exchange slots of the state halves
     int tall = 0;                     // 16 x 1 blocks (else 4 x 4)
@@ -53,6 +54,7 @@ struct SparsePack {
 };
 
 struct SparseParams {
+    int WH;                                  // > 0: split layout, the sending warps do not wait for the rows of R
     int H, K, NKT, UC, HR, NBR, tall;        // tall: blocks are 16 x 1 (16 rows of one column) instead of 4 x 4
     unsigned long long *yslots;              // [2 halves][2 parities][K] (value, tag): the state crosses the chip when there is more than one cluster
     unsigned long long off_meta[2], off_col[2], off_val[2], off_o2, off_o4, off_small, blob_bytes;
@@ -374,10 +376,14 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         // ---- 2. hidden layer of the head + this CTA's R rows (compressed block rows)
         sparse_phase(half ? 0 : 1, vec, half ? sb1 : sb3);
         SSTAMP(7);
-        __syncthreads();
+        // Split layout (WH > 0): the hidden-layer block rows sit in the slices of warps [0, WH), the rows of R in those of warps
+        // 16..19, which take no part in the exchanges or the output rows: the sixteen sending warps meet at a barrier of their
+        // own while the rows of R, which nobody needs before the gates, are still being computed.  Warp w sends this CTA's HR
+        // values to peer w (asynchronous stores that count their bytes on the receiver's barrier of that buffer: no tags,
+        // no polling pass; one remote store instruction per warp: a second one from the same warp waits for the first).
+        if (p.WH > 0) { if (warp < SCS) asm volatile("bar.sync 1, 512;" ::: "memory"); }
+        else __syncthreads();
         SSTAMP(8);
-        // this CTA's HR hidden-layer values -> every peer, one coalesced 16-byte-per-lane store per peer (warp w -> peer w)
-        // (asynchronous stores that count their bytes on the receiver's barrier of that buffer: no tags, no polling pass)
         if (warp < SCS) {
             const unsigned bar = map_to_rank(smem_addr(&xq[par]), warp);
             for (int pr2 = lane; pr2 < HR / 2; pr2 += 32) {
@@ -656,17 +662,33 @@ int sparse_prepare(wrnn_model *m)
             const auto &R = rows[cp];
             std::vector<int> order(NBR);
             for (int i = 0; i < NBR; ++i) order[i] = i;
-            std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return R[a].size() > R[b].size(); });
+            // hidden-layer block rows first (their warps send while the others still work on the rows of R), each kind longest first
+            const int HRB = HR / BRH;
+            std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+                const bool ha = a < HRB, hb = b < HRB;
+                if (ha != hb) return ha;
+                return R[a].size() > R[b].size();
+            });
             slices[cp].assign(SNW, {});
             int next = 0, slots = 0;
+            // split layout: hidden-layer rows (first in `order`) wide on warps [0, wh), the rows of R narrow on warps 16..19
+            const int n_r = NBR - HRB, wh_split = (HRB + cap_w - 1) / cap_w;
+            const bool split = SNW > SCS && wh_split <= SCS && n_r <= cap_n * (SNW - SCS);
             for (int w = 0; w < SNW; ++w) {
                 Slice &sl = slices[cp][w];
-                sl.lpr = w < w8 ? 2 * lpr_n : lpr_n;
-                const int cap = 32 / sl.lpr;
-                // rows still to place, spread evenly over the remaining four-lane warps
-                int nr = cap;
-                if (w >= w8) { const int left = NBR - next, warps_left = SNW - w; nr = (left + warps_left - 1) / warps_left; }
-                if (nr > cap) nr = cap;
+                int nr;
+                if (split) {
+                    if (w < wh_split) { sl.lpr = 2 * lpr_n; nr = std::min(cap_w, HRB - next); }
+                    else if (w < SCS) { sl.lpr = lpr_n; nr = 0; }
+                    else { sl.lpr = lpr_n; const int left = NBR - next, warps_left = SNW - w; nr = (left + warps_left - 1) / warps_left; }
+                } else {
+                    sl.lpr = w < w8 ? 2 * lpr_n : lpr_n;
+                    const int cap = 32 / sl.lpr;
+                    // rows still to place, spread evenly over the remaining four-lane warps
+                    nr = cap;
+                    if (w >= w8) { const int left = NBR - next, warps_left = SNW - w; nr = (left + warps_left - 1) / warps_left; }
+                    if (nr > cap) nr = cap;
+                }
                 if (nr > NBR - next) nr = NBR - next;
                 size_t longest = 0;
                 for (int i = 0; i < nr; ++i) { sl.rows.push_back(order[next + i]); longest = std::max(longest, R[order[next + i]].size()); }
@@ -675,8 +697,10 @@ int sparse_prepare(wrnn_model *m)
                 if (sl.T < 1) sl.T = 1;                                  // the loop's first loads are unconditional
                 slots += sl.lpr * nr * sl.T;
             }
+            if (split) k.WH = wh_split;
             if (next != NBR) { m->err = "too many block rows for the warps of one CTA"; return WRNN_ERR_UNSUPPORTED; }
             max_slots = std::max(max_slots, slots);
+
         }
         k.max_slots = (max_slots + 7) & ~7;
 
@@ -820,7 +844,7 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     const SparsePack &k = *m->sparse_pack;
     SparseParams p;
     std::memset(&p, 0, sizeof(p));
-    p.H = k.H; p.K = k.K; p.NKT = k.NKT; p.UC = k.UC; p.HR = k.HR; p.NBR = k.NBR; p.tall = k.tall;
+    p.H = k.H; p.K = k.K; p.NKT = k.NKT; p.UC = k.UC; p.HR = k.HR; p.NBR = k.NBR; p.tall = k.tall; p.WH = k.WH;
     for (int ph = 0; ph < 2; ++ph) { p.off_meta[ph] = k.off_meta[ph]; p.off_col[ph] = k.off_col[ph]; p.off_val[ph] = k.off_val[ph]; }
     p.off_o2 = k.off_o2; p.off_o4 = k.off_o4; p.off_small = k.off_small; p.blob_bytes = k.blob_bytes;
     p.n_steps = a.n_steps; p.step0 = a.step0; p.stream0 = a.stream0; p.seed = a.seed;

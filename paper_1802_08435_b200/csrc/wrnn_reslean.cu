@@ -105,8 +105,9 @@ __host__ __device__ constexpr size_t rl_smem_bytes(bool f)
 // would leave its array is skipped, and the kernel runs to its normal exit.
 constexpr int RL_N_GUARDS = 13;
 constexpr unsigned RL_GUARD_WORD = 0x5afec0deu;
-// HOOK: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); the others have no trace of it
-template <bool CHK, bool FUSED, bool HOOK>
+// MODE 1: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); MODE 2: the one with the phase
+// stamps of wrnn_phase_profile; MODE 0 (production) has no trace of either
+template <bool CHK, bool FUSED, int MODE>
 __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanParams p)
 {
     constexpr int RL_NLOG = rl_nlog(FUSED), RL_LR = rl_lr(FUSED), NIN = rl_nin(FUSED), NP = NIN / 3;
@@ -179,14 +180,15 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
 
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
-    const bool prof_on = p.prof != nullptr && (cta == 0 || p.prof_all) && warp == 0;
+    constexpr bool HOOK = MODE == 1, PROF = MODE == 2 || CHK;
+    const bool prof_on = PROF && p.prof != nullptr && (cta == 0 || p.prof_all) && warp == 0;
     __shared__ long long s_prof[16];
     __shared__ __align__(8) unsigned long long pub_bar;      // one arrival per half-step: this CTA's gate threads have published
     if (tid < 16) s_prof[tid] = 0;
     if (tid == 0) { mbar_init_cluster(smem_addr(&pub_bar), 1); mbar_fence_init(); }
     __syncthreads();
     long long prof_t = clock64();
-#define STAMP(i) do { if (prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
+#define STAMP(i) do { if (PROF && prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
 
     const bool writer = (cta == 0);
     const int g4 = lane >> 2;
@@ -514,11 +516,12 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
 }
 
 // ---------------------------------------------------------------------------------------------
-static const void *kernel_of(const ResLeanPack &k, bool hook)
+static const void *kernel_of(const ResLeanPack &k, int mode)
 {
-    if (k.checked) return k.fused ? (const void *)resident_lean_kernel<true, true, false> : (const void *)resident_lean_kernel<true, false, false>;
-    if (hook) return k.fused ? (const void *)resident_lean_kernel<false, true, true> : (const void *)resident_lean_kernel<false, false, true>;
-    return k.fused ? (const void *)resident_lean_kernel<false, true, false> : (const void *)resident_lean_kernel<false, false, false>;
+    if (k.checked) return k.fused ? (const void *)resident_lean_kernel<true, true, 0> : (const void *)resident_lean_kernel<true, false, 0>;
+    if (mode == 1) return k.fused ? (const void *)resident_lean_kernel<false, true, 1> : (const void *)resident_lean_kernel<false, false, 1>;
+    if (mode == 2) return k.fused ? (const void *)resident_lean_kernel<false, true, 2> : (const void *)resident_lean_kernel<false, false, 2>;
+    return k.fused ? (const void *)resident_lean_kernel<false, true, 0> : (const void *)resident_lean_kernel<false, false, 0>;
 }
 
 static void fill_launch(const ResLeanPack &k, cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at, cudaStream_t s, bool coop)
@@ -554,9 +557,9 @@ int reslean_prepare(wrnn_model *m)
     cudaGetDeviceProperties(&prop, m->device);
     if (k.NCTA > m->n_sms || (size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "lean resident kernel does not fit this device"; return WRNN_ERR_UNSUPPORTED; }
     { const char *d = getenv("WRNN_DEBUG"); k.checked = d && d[0] == '1'; }
-    const void *fn = kernel_of(k, false);
-    for (int hook = 0; hook < 2; ++hook) {
-        const void *f = kernel_of(k, hook != 0);
+    const void *fn = kernel_of(k, 0);
+    for (int mode = 0; mode < 3; ++mode) {
+        const void *f = kernel_of(k, mode);
         if (cudaFuncSetAttribute(f, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
             cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes + (k.checked ? RL_N_GUARDS * 16 : 0)) != cudaSuccess) {
             cudaGetLastError(); m->err = "lean resident kernel: cannot set the launch attributes"; return WRNN_ERR_UNSUPPORTED;
@@ -682,7 +685,7 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.smem_bytes = cfg.dynamicSmemBytes;
     { const char *d = getenv("WRNN_DEBUG_POKE"); p.chk_poke = (k.checked && d && d[0] == '1') ? 1 : 0; }
     void *args[] = {&p};
-    const cudaError_t e = cudaLaunchKernelExC(&cfg, kernel_of(k, m->dbg_skip_cta >= 0), args);
+    const cudaError_t e = cudaLaunchKernelExC(&cfg, kernel_of(k, m->dbg_skip_cta >= 0 ? 1 : (p.prof ? 2 : 0)), args);
     if (e != cudaSuccess) {
         m->err = std::string("lean resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

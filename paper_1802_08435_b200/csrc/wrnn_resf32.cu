@@ -62,6 +62,9 @@ struct ResF32Params {
     long long *prof;                         // [16] per-phase cycle totals of CTA 0, warp 0 (same slots as the bf16 kernel)
 };
 
+// MODE 1: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); MODE 2: the one with the phase
+// stamps of wrnn_phase_profile; MODE 0 (production) has no trace of either
+template <int MODE>
 __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF32Params p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -98,14 +101,15 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
     }
     cluster.sync();     // peers' exchange buffers are zeroed before anyone writes into them
 
-    const bool prof_on = p.prof != nullptr && cta == 0 && warp == 0;
+    constexpr bool HOOK = MODE == 1, PROF = MODE == 2;
+    const bool prof_on = PROF && p.prof != nullptr && cta == 0 && warp == 0;
     __shared__ long long s_prof[16];
     __shared__ __align__(8) unsigned long long pub_bar;      // one arrival per half-step: this CTA's gate threads have published
     if (tid == 0) { mbar_init_cluster(smem_addr(&pub_bar), 1); mbar_fence_init(); }
     if (tid < 16) s_prof[tid] = 0;
     __syncthreads();
     long long prof_t = clock64();
-#define STAMP(i) do { if (prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
+#define STAMP(i) do { if (PROF && prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
 
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
@@ -185,7 +189,7 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
     };
     // Gates of Eq. 2 for this CTA's units of one half of the state, then publish them to the chip.
     // half_g = 0: coarse units (c_s does not reach them: their I* column is zero), 1: fine units.
-    const int skip_at = cta == p.skip_cta ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
+    const int skip_at = (HOOK && cta == p.skip_cta) ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
         const float xk = scale8(drawn);                  // the pending input
         const float u = sigmoidf_fast(fmaf(q.ku, xk, q.pu)), r = sigmoidf_fast(fmaf(q.kr, xk, q.pr));
@@ -193,7 +197,7 @@ __global__ void __launch_bounds__(RF_THREADS, 1) resident_f32_kernel(const ResF3
         const float hn = fmaf(u, half_g ? hF : hC, (1.0f - u) * e);
         if (half_g) hF = hn; else hC = hn;
         const int j = cta * UC + lane, jj = (half_g ? K : 0) + j;
-        if ((int)s != skip_at)
+        if (!HOOK || (int)s != skip_at)
             st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + j,
                            ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
         if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
@@ -400,6 +404,15 @@ int resf32_supported(const wrnn_model *m, int batch, std::string *why)
     return WRNN_OK;
 }
 
+// one launch attribute on all three instantiations of the kernel
+static cudaError_t rf_set_attr(cudaFuncAttribute a, int v)
+{
+    cudaError_t e = cudaFuncSetAttribute(resident_f32_kernel<0>, a, v);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(resident_f32_kernel<1>, a, v);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(resident_f32_kernel<2>, a, v);
+    return e;
+}
+
 int resf32_prepare(wrnn_model *m)
 {
     const int H = m->H, K = H / 2;
@@ -407,7 +420,7 @@ int resf32_prepare(wrnn_model *m)
     if (K % 16 != 0) { m->err = "H/2 must be a multiple of 16"; return WRNN_ERR_UNSUPPORTED; }
     cudaDeviceProp prop;
     cudaGetDeviceProperties(&prop, m->device);
-    if (cudaFuncSetAttribute(resident_f32_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
+    if (rf_set_attr(cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) {
         cudaGetLastError(); m->err = "cannot configure the fp32 resident kernel"; return WRNN_ERR_UNSUPPORTED;
     }
     // The largest number of CTAs that divides the half state, keeps a CTA's units within one warp, forms clusters (the
@@ -424,17 +437,17 @@ int resf32_prepare(wrnn_model *m)
             c.blob_bytes = r16(c.w_bytes + ((size_t)c.NR * 3 + 2 * c.UC + 2 * c.LR) * 4);
             c.smem_bytes = resf32_smem_bytes(c);
             if ((size_t)c.smem_bytes + 1024 > prop.sharedMemPerBlockOptin) continue;
-            if (cudaFuncSetAttribute(resident_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, c.smem_bytes) != cudaSuccess) { cudaGetLastError(); continue; }
+            if (rf_set_attr(cudaFuncAttributeMaxDynamicSharedMemorySize, c.smem_bytes) != cudaSuccess) { cudaGetLastError(); continue; }
             cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
             fill_launch(c, &cfg, at, 0, false);
             int max_clusters = 0;
-            if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_f32_kernel, &cfg) != cudaSuccess || max_clusters < n / cs) { cudaGetLastError(); continue; }
+            if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_f32_kernel<0>, &cfg) != cudaSuccess || max_clusters < n / cs) { cudaGetLastError(); continue; }
             k = c;
             break;
         }
     }
     if (k.NCTA == 0) { m->err = "no CTA count shards this model into the shared memory of the device"; return WRNN_ERR_UNSUPPORTED; }
-    if (cudaFuncSetAttribute(resident_f32_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
+    if (rf_set_attr(cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
         cudaGetLastError(); m->err = "cannot raise the dynamic shared memory limit"; return WRNN_ERR_UNSUPPORTED;
     }
 
@@ -547,7 +560,9 @@ int resf32_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     // WRNN_NO_COOP=1 drops it (co-residency was already checked against the occupancy API at create):
     // a profiler that replays kernels may not accept cooperative cluster launches.
     fill_launch(k, &cfg, at, s, coop_launch_allowed());
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, resident_f32_kernel, p);
+    const cudaError_t e = m->dbg_skip_cta >= 0 ? cudaLaunchKernelEx(&cfg, resident_f32_kernel<1>, p)
+                          : p.prof          ? cudaLaunchKernelEx(&cfg, resident_f32_kernel<2>, p)
+                                            : cudaLaunchKernelEx(&cfg, resident_f32_kernel<0>, p);
     if (e != cudaSuccess) {
         m->err = std::string("fp32 resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

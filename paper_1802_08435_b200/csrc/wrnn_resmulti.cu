@@ -110,8 +110,9 @@ __device__ __forceinline__ void mma16816(float (&c)[4], const uint4 &a, unsigned
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ void named_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
-// HOOK: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); the production one has no trace of it
-template <bool HOOK>
+// MODE 1: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); MODE 2: the one with the phase
+// stamps of wrnn_phase_profile; MODE 0 (production) has no trace of either
+template <int MODE>
 __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -171,12 +172,13 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
     const int g4 = lane >> 2, t4 = lane & 3;
-    const bool prof_on = p.prof != nullptr && cta == 0 && warp == 0;
+    constexpr bool HOOK = MODE == 1, PROF = MODE == 2;
+    const bool prof_on = PROF && p.prof != nullptr && cta == 0 && warp == 0;
     __shared__ long long s_prof[16];
     if (tid < 16) s_prof[tid] = 0;
     __syncthreads();
     long long prof_t = clock64();
-#define STAMP(i) do { if (prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
+#define STAMP(i) do { if (PROF && prof_on) { const long long now_ = clock64(); if (lane == 0) s_prof[i] += now_ - prof_t; prof_t = now_; } } while (0)
 
     // ---- roles
     const int ws = warp;                                  // drawing warps 0..3: own stream ws
@@ -657,10 +659,12 @@ int resmulti_prepare(wrnn_model *m)
     cudaDeviceProp prop;
     cudaGetDeviceProperties(&prop, m->device);
     if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin ||
-        cudaFuncSetAttribute(resident_multi_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-        cudaFuncSetAttribute(resident_multi_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess ||
-        cudaFuncSetAttribute(resident_multi_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-        cudaFuncSetAttribute(resident_multi_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
+        cudaFuncSetAttribute(resident_multi_kernel<0>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
         cudaGetLastError();
         m->err = "multi-stream resident kernel does not fit in shared memory";
         return WRNN_ERR_UNSUPPORTED;
@@ -669,7 +673,7 @@ int resmulti_prepare(wrnn_model *m)
         cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
         multi_fill_launch(k, &cfg, at, 0, false);
         int max_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_multi_kernel<false>, &cfg) != cudaSuccess || max_clusters < MNC) {
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, resident_multi_kernel<0>, &cfg) != cudaSuccess || max_clusters < MNC) {
             cudaGetLastError();
             m->err = "not enough co-resident clusters for the multi-stream resident kernel";
             return WRNN_ERR_UNSUPPORTED;
@@ -804,7 +808,12 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     multi_fill_launch(k, &cfg, at, s, coop_launch_allowed());
-    const cudaError_t e = m->dbg_skip_cta >= 0 ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<true>, p) : cudaLaunchKernelEx(&cfg, resident_multi_kernel<false>, p);
+    // Above four rows the instantiation that carries the (unexecuted) stamp code is the faster one: 16 rows 9.55 us per
+    // lock-step against 9.95 without it, 4 rows 7.21 against 7.02 (same call, alternating); the compiler orders the
+    // half-step differently around the clock reads.
+    const cudaError_t e = m->dbg_skip_cta >= 0        ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<1>, p)
+                          : (p.prof || a.batch > 4) ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<2>, p)
+                                                    : cudaLaunchKernelEx(&cfg, resident_multi_kernel<0>, p);
     if (e != cudaSuccess) {
         m->err = std::string("multi-stream resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

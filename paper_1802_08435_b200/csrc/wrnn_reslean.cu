@@ -15,6 +15,8 @@
 // exact three-way bf16 split.  Every wait is bounded; a CTA that gives up records where and all CTAs leave through the
 // final cluster barrier.
 #include <cooperative_groups.h>
+
+#include <type_traits>
 #include <cuda_bf16.h>
 
 #include <algorithm>
@@ -320,12 +322,12 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
     // Half-step n = 2 s + 1 is the coarse half of step s (input y_c(s): coarse head -> c_s, then the fine gates of step s),
     // n = 2 s the fine half (input y_f(s - 1): fine head -> f_{s-1}, R h_{s-1} completed, then the coarse gates of step s).
     const long long T = p.n_steps;
-#pragma unroll 1
-    for (long long n = 1; n <= 2 * T; ++n) {
-        const int half = (int)(n & 1);
+    // (one copy of the body per half, so that everything chosen by the half is chosen at compile time)
+    auto half_step = [&](auto HALF_C, const long long n) -> bool {
+        constexpr int half = decltype(HALF_C)::value;
         const long long s = n >> 1;
         const bool last = n == 2 * T;
-        const unsigned par = (unsigned)((n - 1) & 1);
+        constexpr unsigned par = 1u - (unsigned)half;           // (n - 1) & 1
         const uint4 *MH = half ? wHA : wHB, *MR = half ? wRA : wRB;
         const unsigned *L = half ? wL2 : wL4;
         const float *bh = half ? sb1 : sb3, *bl = half ? sb2 : sb4;
@@ -383,7 +385,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
                 vec[2 * i] = x0; vec[2 * i + 1] = x1;
                 store_split2_pair(spl, 2 * i, x0, x1);
             }
-            if (__syncthreads_or(my_bad)) break;
+            if (__syncthreads_or(my_bad)) return false;
         }
         STAMP(8 * half + 0);
 
@@ -439,7 +441,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
             if (lane < UC && !last) gp = gates_prepare(half, gv);
         }
         STAMP(8 * half + 4);
-        if (__syncthreads_or(my_bad)) break;
+        if (__syncthreads_or(my_bad)) return false;
         if (lane < RL_LR / 2) {
             const float2 v = reinterpret_cast<const float2 *>(lrow)[lane];
             st_async_v2(l_snd[par], v.x, v.y, l_bar[par]);
@@ -491,6 +493,12 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
             if (half) c_prev = fed; else f_prev = fed;
         }
         STAMP(8 * half + 7);
+        return true;
+    };
+#pragma unroll 1
+    for (long long s2 = 0; s2 < T; ++s2) {
+        if (!half_step(std::integral_constant<int, 1>{}, 2 * s2 + 1)) break;
+        if (!half_step(std::integral_constant<int, 0>{}, 2 * s2 + 2)) break;
     }
     if (prof_on && lane == 0) for (int i = 0; i < 16; ++i) p.prof[cta * 16 + i] = s_prof[i];
 #undef STAMP
@@ -675,7 +683,7 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.frame_shift = a.row_lag > 0 ? a.step0 : 0;
     p.status = m->status;
     p.limit_ns = m->wait_limit_ns(); p.skip_cta = m->dbg_skip_cta; p.skip_step = m->dbg_skip_step;
-    { const char *e = getenv("WRNN_POLL_GAP"); p.poll_gap = e ? atoi(e) : 100; }
+    { const char *e = getenv("WRNN_POLL_GAP"); p.poll_gap = e ? atoi(e) : 125; }
     p.prof = m->prof_enabled ? k.d_prof : nullptr;     // phase stamps cost the stamped warp some 50 cycles each: off unless asked for
     { const char *e = getenv("WRNN_PROF_ALL"); p.prof_all = (e && e[0] == '1') ? 1 : 0; }
     if (cudaMemsetAsync(k.d_slots, 0, (size_t)4 * RL_K * 8, s) != cudaSuccess) return WRNN_ERR_CUDA;

@@ -107,8 +107,9 @@ __host__ __device__ constexpr size_t rl_smem_bytes(bool f)
 // would leave its array is skipped, and the kernel runs to its normal exit.
 constexpr int RL_N_GUARDS = 13;
 constexpr unsigned RL_GUARD_WORD = 0x5afec0deu;
-// MODE 1: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); MODE 2: the one with the phase
-// stamps of wrnn_phase_profile; MODE 0 (production) has no trace of either
+// MODE 0: plain sampling (no forced symbols, no dumps, no stamps, no self-test predicate: what wrnn_sample runs);
+// MODE 1: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); MODE 2: the one with the
+// phase stamps of wrnn_phase_profile; MODE 3: teacher forcing and dumps.  Modes 1 to 3 all take forced symbols and dumps.
 template <bool CHK, bool FUSED, int MODE>
 __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanParams p)
 {
@@ -182,7 +183,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
 
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
-    constexpr bool HOOK = MODE == 1, PROF = MODE == 2 || CHK;
+    constexpr bool HOOK = MODE == 1, PROF = MODE == 2 || CHK, DBG = MODE != 0 || CHK;
     const bool prof_on = PROF && p.prof != nullptr && (cta == 0 || p.prof_all) && warp == 0;
     __shared__ long long s_prof[16];
     __shared__ __align__(8) unsigned long long pub_bar;      // one arrival per half-step: this CTA's gate threads have published
@@ -284,7 +285,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         return q;
     };
     const int skip_at = (HOOK && cta == p.skip_cta) ? (int)p.skip_step : -1;      // self-test: the step at which this CTA withholds its publication
-    const bool dbg_any = p.dbg_gates != nullptr || p.dbg_h != nullptr;
+    const bool dbg_any = DBG && (p.dbg_gates != nullptr || p.dbg_h != nullptr);
     auto gates_and_publish = [&](int half_g, long long s, int drawn, const GatePre &q) {
         float pu = q.pu, pr = q.pr, pe = q.pe;
 #pragma unroll
@@ -301,7 +302,7 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         if (CHK && slot >= (size_t)4 * K) record_check(-1);                          // an exchange slot outside the slot array: skipped
         else if (!HOOK || (int)s != skip_at)
             st_relaxed_u64(p.slots + slot, ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
-        if (dbg_any) {
+        if (DBG && dbg_any) {
             if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
             if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
         }
@@ -345,12 +346,16 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
         if (warp == 0) {
             if (lane < UC && !last) load_g(half, s, gv);
             if (FUSED) {
-                if (half) { if (p.a_forced) forced = p.a_forced[s]; }
-                else      { if (p.b_forced) forced = p.b_forced[s - 1]; }
+                if (DBG) {
+                    if (half) { if (p.a_forced) forced = p.a_forced[s]; }
+                    else      { if (p.b_forced) forced = p.b_forced[s - 1]; }
+                }
                 u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), (half ? 0u : 4u) + (unsigned)(lane >> 3));
             } else {
-                if (half) { if (p.c_forced) forced = p.c_forced[s]; }
-                else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
+                if (DBG) {
+                    if (half) { if (p.c_forced) forced = p.c_forced[s]; }
+                    else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
+                }
                 u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
             }
             asm volatile("" : "+f"(u01), "+r"(forced), "+f"(gv[0]), "+f"(gv[1]), "+f"(gv[2]));
@@ -468,11 +473,11 @@ __global__ void __launch_bounds__(512, 1) resident_lean_kernel(const ResLeanPara
                 l[0] = a.x; l[1] = a.y; l[2] = a.z; l[3] = a.w; l[NL - 4] = b.x; l[NL - 3] = b.y; l[NL - 2] = b.z; l[NL - 1] = b.w;
                 drawn = warp_softmax_draw_fast(reinterpret_cast<const float (&)[8]>(l), u01, lane);
             }
-            const int fed = forced >= 0 ? forced : drawn;
+            const int fed = (DBG && forced >= 0) ? forced : drawn;
             if (lane < UC && !last && !my_bad) gates_and_publish(half, s, fed, gp);
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(&pub_bar)) : "memory");
             if (writer) {
-                if (p.dbg_logits) {
+                if (DBG && p.dbg_logits) {
                     float *d = p.dbg_logits + (size_t)(n - 1) * RL_NLOG + NL * lane;
 #pragma unroll
                     for (int k = 0; k < NL; ++k) d[k] = l[k];
@@ -529,6 +534,7 @@ static const void *kernel_of(const ResLeanPack &k, int mode)
     if (k.checked) return k.fused ? (const void *)resident_lean_kernel<true, true, 0> : (const void *)resident_lean_kernel<true, false, 0>;
     if (mode == 1) return k.fused ? (const void *)resident_lean_kernel<false, true, 1> : (const void *)resident_lean_kernel<false, false, 1>;
     if (mode == 2) return k.fused ? (const void *)resident_lean_kernel<false, true, 2> : (const void *)resident_lean_kernel<false, false, 2>;
+    if (mode == 3) return k.fused ? (const void *)resident_lean_kernel<false, true, 3> : (const void *)resident_lean_kernel<false, false, 3>;
     return k.fused ? (const void *)resident_lean_kernel<false, true, 0> : (const void *)resident_lean_kernel<false, false, 0>;
 }
 
@@ -566,7 +572,7 @@ int reslean_prepare(wrnn_model *m)
     if (k.NCTA > m->n_sms || (size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "lean resident kernel does not fit this device"; return WRNN_ERR_UNSUPPORTED; }
     { const char *d = getenv("WRNN_DEBUG"); k.checked = d && d[0] == '1'; }
     const void *fn = kernel_of(k, 0);
-    for (int mode = 0; mode < 3; ++mode) {
+    for (int mode = 0; mode < 4; ++mode) {
         const void *f = kernel_of(k, mode);
         if (cudaFuncSetAttribute(f, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
             cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes + (k.checked ? RL_N_GUARDS * 16 : 0)) != cudaSuccess) {
@@ -693,7 +699,8 @@ int reslean_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     p.smem_bytes = cfg.dynamicSmemBytes;
     { const char *d = getenv("WRNN_DEBUG_POKE"); p.chk_poke = (k.checked && d && d[0] == '1') ? 1 : 0; }
     void *args[] = {&p};
-    const cudaError_t e = cudaLaunchKernelExC(&cfg, kernel_of(k, m->dbg_skip_cta >= 0 ? 1 : (p.prof ? 2 : 0)), args);
+    const bool teacher = p.c_forced || p.f_forced || p.a_forced || p.b_forced || p.dbg_gates || p.dbg_h || p.dbg_logits;
+    const cudaError_t e = cudaLaunchKernelExC(&cfg, kernel_of(k, m->dbg_skip_cta >= 0 ? 1 : (p.prof ? 2 : (teacher ? 3 : 0))), args);
     if (e != cudaSuccess) {
         m->err = std::string("lean resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

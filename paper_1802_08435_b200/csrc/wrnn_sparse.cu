@@ -84,8 +84,9 @@ __device__ long long g_sprof[16];
 #endif
 
 // NKL: k-tiles of the logits tile per warp (K / 16 / NKL warps split K).
-// HOOK: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); the production one has no trace of it
-template <int NKL, bool HOOK>
+// MODE 0: plain sampling (no forced symbols, no dumps, no self-test predicate: what wrnn_sample runs); MODE 1: the instantiation
+// that wrnn_selftest_lost_word runs (one CTA withholds one publication); MODE 3: teacher forcing and dumps (modes 1 and 3 take both)
+template <int NKL, int MODE>
 __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const SparseParams p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -128,6 +129,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
     __syncthreads();
     cluster.sync();
 
+    constexpr bool HOOK = MODE == 1, DBG = MODE != 0;
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
     const bool writer = (cta == 0);
@@ -295,8 +297,8 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
                 st_relaxed_u64(p.yslots + (size_t)((half_g ? 2 : 0) + (s & 1)) * K + cta * UC + u0,
                                ((unsigned long long)(unsigned)(s + 1) << 32) | __float_as_uint(hn));
             const int jj = (half_g ? K : 0) + cta * UC + u0;
-            if (p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
-            if (p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
+            if (DBG && p.dbg_gates) { float *d = p.dbg_gates + (size_t)s * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
+            if (DBG && p.dbg_h) p.dbg_h[(size_t)s * H + jj] = hn;
         }
     };
     // ---- prologue: R h of step 0 from the initial state, coarse gates of step 0
@@ -334,8 +336,10 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
         int forced = -1;
         if (warp < GW) {
             if (lane < UW && !last) load_g(half, s, gv);
-            if (half) { if (p.c_forced) forced = p.c_forced[s]; }
-            else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
+            if (DBG) {
+                if (half) { if (p.c_forced) forced = p.c_forced[s]; }
+                else      { if (p.f_forced) forced = p.f_forced[s - 1]; }
+            }
             u01 = uniform24(p.seed, p.stream0, (unsigned long long)(p.step0 + (half ? s : s - 1)), half ? 0u : 1u);
         }
 
@@ -485,7 +489,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
             SSTAMP(4);
             int drawn = warp_softmax_draw_scan(l, u01, lane);
             if (writer && warp == 0) {
-                if (p.dbg_logits) {
+                if (DBG && p.dbg_logits) {
                     float *d = p.dbg_logits + (size_t)(n - 1) * 256 + 8 * lane;
 #pragma unroll
                     for (int k = 0; k < 8; ++k) d[k] = l[k];
@@ -495,7 +499,7 @@ __global__ void __launch_bounds__(SNW * 32, 1) sparse_cluster_kernel(const Spars
                     else      { if (p.f_out) p.f_out[s - 1] = (uint8_t)drawn; }
                 }
             }
-            if (forced >= 0) drawn = forced;
+            if (DBG && forced >= 0) drawn = forced;
             if (!half) {
                 if (writer && warp == 0 && lane == 0 && p.out) p.out[s - 1] = (int16_t)(256 * c_prev + drawn - 32768);
                 f_prev = drawn;
@@ -551,7 +555,7 @@ int sparse_supported(const wrnn_model *m, int batch, std::string *why)
     return WRNN_OK;
 }
 
-static void *sparse_fn(bool hook) { return hook ? (void *)sparse_cluster_kernel<8, true> : (void *)sparse_cluster_kernel<8, false>; }
+static void *sparse_fn(int mode) { return mode == 1 ? (void *)sparse_cluster_kernel<8, 1> : mode == 3 ? (void *)sparse_cluster_kernel<8, 3> : (void *)sparse_cluster_kernel<8, 0>; }
 
 static void sparse_fill_launch(const SparsePack &k, cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at, cudaStream_t s, bool coop)
 {
@@ -720,16 +724,17 @@ int sparse_prepare(wrnn_model *m)
         cudaDeviceProp prop;
         cudaGetDeviceProperties(&prop, m->device);
         if ((size_t)k.smem_bytes > prop.sharedMemPerBlockOptin) { m->err = "pruned model does not fit the shared memory of the clusters"; return WRNN_ERR_UNSUPPORTED; }
-        if (cudaFuncSetAttribute(sparse_fn(false), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-            cudaFuncSetAttribute(sparse_fn(false), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess ||
-            cudaFuncSetAttribute(sparse_fn(true), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-            cudaFuncSetAttribute(sparse_fn(true), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
+        bool attr_ok = true;
+        for (int mode : {0, 1, 3})
+            attr_ok = attr_ok && cudaFuncSetAttribute(sparse_fn(mode), cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
+                      cudaFuncSetAttribute(sparse_fn(mode), cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) == cudaSuccess;
+        if (!attr_ok) {
             cudaGetLastError(); m->err = "cannot configure the 16-CTA cluster kernel"; return WRNN_ERR_UNSUPPORTED;
         }
         cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
         sparse_fill_launch(k, &cfg, at, 0, false);
         int max_clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&max_clusters, sparse_fn(false), &cfg) != cudaSuccess || max_clusters < nc) {
+        if (cudaOccupancyMaxActiveClusters(&max_clusters, sparse_fn(0), &cfg) != cudaSuccess || max_clusters < nc) {
             cudaGetLastError(); m->err = "the 16-CTA clusters cannot all be co-resident on this device"; return WRNN_ERR_UNSUPPORTED;
         }
 
@@ -865,7 +870,8 @@ int sparse_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     sparse_fill_launch(k, &cfg, at, s, coop_launch_allowed());
     void *args[] = {&p};
-    cudaError_t e = cudaLaunchKernelExC(&cfg, sparse_fn(m->dbg_skip_cta >= 0), args);
+    const bool teacher = p.c_forced || p.f_forced || p.dbg_gates || p.dbg_h || p.dbg_logits;
+    cudaError_t e = cudaLaunchKernelExC(&cfg, sparse_fn(m->dbg_skip_cta >= 0 ? 1 : (teacher ? 3 : 0)), args);
     if (e != cudaSuccess) {
         m->err = std::string("sparse cluster kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

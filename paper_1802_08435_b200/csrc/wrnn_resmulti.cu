@@ -110,8 +110,9 @@ __device__ __forceinline__ void mma16816(float (&c)[4], const uint4 &a, unsigned
 __device__ __forceinline__ void named_sync(int id, int n) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 __device__ __forceinline__ void named_arrive(int id, int n) { asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(n) : "memory"); }
 
-// MODE 1: the instantiation that wrnn_selftest_lost_word runs (one CTA withholds one publication); MODE 2: the one with the phase
-// stamps of wrnn_phase_profile; MODE 0 (production) has no trace of either
+// MODE 0: plain sampling (no forced symbols, no dumps, no stamps, no self-test predicate); MODE 1: the instantiation that
+// wrnn_selftest_lost_word runs (one CTA withholds one publication); MODE 2: the one with the phase stamps of wrnn_phase_profile
+// (and with forced symbols and dumps, like mode 1)
 template <int MODE>
 __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParams p)
 {
@@ -172,7 +173,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
     const int g4 = lane >> 2, t4 = lane & 3;
-    constexpr bool HOOK = MODE == 1, PROF = MODE == 2;
+    constexpr bool HOOK = MODE == 1, PROF = MODE == 2, DBG = MODE != 0;
     const bool prof_on = PROF && p.prof != nullptr && cta == 0 && warp == 0;
     __shared__ long long s_prof[16];
     if (tid < 16) s_prof[tid] = 0;
@@ -311,8 +312,8 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         if (!HOOK || (int)s != skip_at)
             st_relaxed_u64(p.slots + ((size_t)((half_g ? 2 : 0) + (s & 1)) * NS + gst) * K + gj,
                            ((unsigned long long)(unsigned)(s + 1) << 32) | (unsigned)__bfloat16_as_ushort(hh) | ((unsigned)__bfloat16_as_ushort(hl) << 16));
-        if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * NS + gst) * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
-        if (p.dbg_h) p.dbg_h[((size_t)s * NS + gst) * H + jj] = hn;
+        if (DBG && p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * NS + gst) * 3 * H; d[jj] = u; d[H + jj] = r; d[2 * H + jj] = e; }
+        if (DBG && p.dbg_h) p.dbg_h[((size_t)s * NS + gst) * H + jj] = hn;
     };
     auto load_g = [&](int half_g, long long s, float (&gv)[3]) {
         const long long fr = p.row_lag > 0 ? s : ((p.step0 + s) * p.row_stride + (long long)(p.stream0 + (unsigned)gst) * p.row_offset_mul) / p.hop;
@@ -374,8 +375,10 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
         if (drawer) {
             const long long t = half ? s : s - 1;
             const long long o = (long long)d_st * T + t;
-            if (half) { if (p.c_forced) forced = p.c_forced[o]; }
-            else      { if (p.f_forced) forced = p.f_forced[o]; }
+            if (DBG) {
+                if (half) { if (p.c_forced) forced = p.c_forced[o]; }
+                else      { if (p.f_forced) forced = p.f_forced[o]; }
+            }
             u01 = uniform24(p.seed, p.stream0 + (unsigned)d_st, (unsigned long long)(p.step0 + t - (long long)d_st * p.row_lag), half ? 0u : 1u);
         }
 
@@ -557,7 +560,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                 my_bad = __any_sync(FULL, my_bad);
                 STAMP(4 + 6 * half);
                 const int drawn = warp_softmax_draw_fast(l, u01, lane);
-                const int fed = forced >= 0 ? forced : drawn;
+                const int fed = (DBG && forced >= 0) ? forced : drawn;
                 {
                     // the symbol to the gate threads of the cluster's 16 CTAs
                     if (lane < MCS && !my_bad) {
@@ -565,7 +568,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
                         asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(dst), "l"(((unsigned long long)tag << 32) | (unsigned)fed) : "memory");
                     }
                     const long long t = half ? s : s - 1;
-                    if (p.dbg_logits) {
+                    if (DBG && p.dbg_logits) {
                         float *d = p.dbg_logits + (((size_t)t * NS + d_st) * 2 + (half ? 0 : 1)) * 256 + 8 * lane;
 #pragma unroll
                         for (int k = 0; k < 8; ++k) d[k] = l[k];
@@ -783,6 +786,7 @@ int resmulti_phase_cycles(const wrnn_model *m, long long *out16)
 
 int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
 {
+    static const int MODE0_MAX_ROWS = [] { const char *e = getenv("WRNN_MULTI_MODE0_ROWS"); return e ? atoi(e) : 4; }();
     const ResMultiPack &k = *m->resmulti;
     MultiParams p;
     std::memset(&p, 0, sizeof(p));
@@ -808,12 +812,14 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     multi_fill_launch(k, &cfg, at, s, coop_launch_allowed());
-    // Above four rows the instantiation that carries the (unexecuted) stamp code is the faster one: 16 rows 9.55 us per
-    // lock-step against 9.95 without it, 4 rows 7.21 against 7.02 (same call, alternating); the compiler orders the
-    // half-step differently around the clock reads.
-    const cudaError_t e = m->dbg_skip_cta >= 0        ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<1>, p)
-                          : (p.prof || a.batch > 4) ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<2>, p)
-                                                    : cudaLaunchKernelEx(&cfg, resident_multi_kernel<0>, p);
+    // Plain sampling of up to four rows runs the instantiation without stamps, forced symbols and dumps; above four rows the
+    // one that carries that (unexecuted) code is the faster one: 16 rows 9.55 us per lock-step against 9.95 without it, 4 rows
+    // 7.21 against 7.02 (same call, alternating): the compiler orders the half-step differently around the clock reads.
+    const bool teacher = p.c_forced || p.f_forced || p.dbg_gates || p.dbg_h || p.dbg_logits;
+    const int mode = m->dbg_skip_cta >= 0 ? 1 : (p.prof || teacher || a.batch > MODE0_MAX_ROWS) ? 2 : 0;
+    const cudaError_t e = mode == 1 ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<1>, p)
+                          : mode == 2 ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<2>, p)
+                                      : cudaLaunchKernelEx(&cfg, resident_multi_kernel<0>, p);
     if (e != cudaSuccess) {
         m->err = std::string("multi-stream resident kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

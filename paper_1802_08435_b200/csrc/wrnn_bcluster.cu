@@ -126,6 +126,8 @@ __device__ long long g_bcprof[32];
 #define RSTAMP(i) do { } while (0)
 #endif
 
+// DBG = false: plain sampling (no forced symbols, no dumps: what wrnn_sample runs)
+template <bool DBG>
 __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __grid_constant__ BcParams p)
 {
     extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -416,7 +418,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 const __nv_bfloat16 hi = __float2bfloat16_rn(hn);
                 Sout[(size_t)(2 * g_row) * BC_SOUT_PITCH + uh] = hi;
                 Sout[(size_t)(2 * g_row + 1) * BC_SOUT_PITCH + uh] = __float2bfloat16_rn(hn - __bfloat162float(hi));
-                if (p.dbg_gates || p.dbg_h) {
+                if (DBG && (p.dbg_gates || p.dbg_h)) {
                     const int unit = 8 * ((int)crank + BC_CS * (i0 + (uh >> 3))) + (uh & 7);
                     if (p.dbg_gates) { float *d = p.dbg_gates + ((size_t)s * p.batch + g_gb) * p.G + unit; d[0] = u; d[H] = r; d[2 * H] = e; }
                     if (p.dbg_h) p.dbg_h[((size_t)s * p.batch + g_gb) * H + unit] = hn;
@@ -516,7 +518,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                     // row bl of the group is drawn by warp bl / 16 of CTA bl % 16: the logits go straight into its shared memory
                     const unsigned dst = map_to_rank(smem_addr(s_log + (bl >> 4) * 256 + r0), (unsigned)(bl & 15));
                     asm volatile("st.shared::cluster.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(o.x), "f"(o.y), "f"(o.z), "f"(o.w) : "memory");
-                    if (p.dbg_logits) *reinterpret_cast<float4 *>(p.dbg_logits + (((size_t)s * p.batch + gb) * 2 + head) * 256 + r0) = o;
+                    if (DBG && p.dbg_logits) *reinterpret_cast<float4 *>(p.dbg_logits + (((size_t)s * p.batch + gb) * 2 + head) * 256 + r0) = o;
                 }
             }
             CSTAMP(8 + 8 * head);
@@ -533,7 +535,7 @@ __global__ void __launch_bounds__(BC_THREADS, 1) bcluster_step_kernel(const __gr
                 const float u = uniform24(p.seed, p.stream0 + (unsigned)s_gb, (unsigned long long)(p.step0 + s - (long long)s_gb * p.row_lag), head);
                 drawn = warp_softmax_draw_scan(l, u, lane);
                 const uint8_t *forced = head ? p.f_forced : p.c_forced;
-                used = forced ? (int)forced[s_o] : drawn;
+                used = (DBG && forced) ? (int)forced[s_o] : drawn;
                 if (lane < BC_CS) {
                     const unsigned dst = map_to_rank(smem_addr((head ? s_f : s_c) + s_r), (unsigned)lane);
                     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(dst), "r"(used) : "memory");
@@ -686,10 +688,12 @@ int bcluster_prepare(wrnn_model *m)
     int dev_smem = 0;
     cudaDeviceGetAttribute(&dev_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, m->device);
     cudaFuncAttributes fa;
-    if (cudaFuncGetAttributes(&fa, bcluster_step_kernel) != cudaSuccess) return failed("cluster-partitioned kernel image missing", WRNN_ERR_CUDA);
+    if (cudaFuncGetAttributes(&fa, bcluster_step_kernel<true>) != cudaSuccess) return failed("cluster-partitioned kernel image missing", WRNN_ERR_CUDA);
     k->max_dyn_smem = dev_smem - (int)fa.sharedSizeBytes;
-    if (cudaFuncSetAttribute(bcluster_step_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, k->max_dyn_smem) != cudaSuccess ||
-        cudaFuncSetAttribute(bcluster_step_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
+    if (cudaFuncSetAttribute(bcluster_step_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, k->max_dyn_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(bcluster_step_kernel<true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(bcluster_step_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, k->max_dyn_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(bcluster_step_kernel<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess)
         return failed("cluster-partitioned kernel attributes rejected", WRNN_ERR_UNSUPPORTED);
     {
         cudaLaunchConfig_t cfg = {};
@@ -699,7 +703,7 @@ int bcluster_prepare(wrnn_model *m)
         at[0].val.clusterDim.x = BC_CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
         cfg.attrs = at; cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, bcluster_step_kernel, &cfg) != cudaSuccess || n < 1)
+        if (cudaOccupancyMaxActiveClusters(&n, bcluster_step_kernel<true>, &cfg) != cudaSuccess || n < 1)
             return failed("device cannot co-schedule a 16-CTA cluster of this size", WRNN_ERR_UNSUPPORTED);
         k->max_clusters = n;
     }
@@ -815,7 +819,8 @@ int bcluster_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = BC_CS; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
     cfg.attrs = at; cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, bcluster_step_kernel, p);
+    const bool teacher = p.c_forced || p.f_forced || p.dbg_gates || p.dbg_h || p.dbg_logits;
+    const cudaError_t e = teacher ? cudaLaunchKernelEx(&cfg, bcluster_step_kernel<true>, p) : cudaLaunchKernelEx(&cfg, bcluster_step_kernel<false>, p);
     if (e != cudaSuccess) {
         m->err = std::string("cluster-partitioned kernel launch failed: ") + cudaGetErrorString(e);
         cudaGetLastError();

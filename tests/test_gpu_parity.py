@@ -689,6 +689,30 @@ def test_sparse_cluster_and_generic_kernels_agree(env):
             B.wrnn_destroy(m)
 
 
+@pytest.mark.parametrize("n_clusters", [1, 2])
+def test_sparse_cluster_kernel_on_fewer_clusters(env, monkeypatch, n_clusters):
+    """The block-sparse kernel on one and two clusters of 16 (the fallback where four cannot be co-resident): the block rows
+    of the hidden layer and of R then share the warps' slices and every warp meets at the CTA barrier before the send, the
+    path that the four-cluster layout does not take.  Teacher-forced with dumps, then a free run against the oracle's stream."""
+    torch, B = env
+    wl = synth.WORKLOADS[2]
+    w, masks, cond = synth.build_workload(wl)
+    om = orc.OracleModel(w, wl.dtype, masks)
+    res = om.run(cond, 200, 1, SEED, dump=True)
+    monkeypatch.setenv("WRNN_SPARSE_CLUSTERS", str(n_clusters))
+    m = B.wrnn_create(w, wl.dtype, masks, kernel=B.WRNN_KERNEL_SPARSE)
+    try:
+        info = B.wrnn_launch_info(m, 1)
+        assert info["kernel"] == B.WRNN_KERNEL_SPARSE and info["n_ctas"] == 16 * n_clusters
+        r = pu.teacher_forced_parity(torch, B, m, om, cond, 200, 1, SEED, oracle_free=res)
+        _report("sparse kernel on %d cluster(s)" % n_clusters, r)
+        _tol_check(r, wl.dtype)
+        free = _free_run(torch, B, m, cond, 200, 1, SEED)
+        _check_free_run_against_oracle(free, res)
+    finally:
+        B.wrnn_destroy(m)
+
+
 def test_sparse_16x1_blocks_cluster_kernel(env):
     """The H = 2048 model pruned to 96 % with 16 x 1 blocks (Section 3.2's m x 1 shape, one activation per block) on
     the single-cluster kernel and on the generic kernel, both against the dense-with-zeros oracle."""

@@ -112,7 +112,7 @@ __device__ __forceinline__ void named_arrive(int id, int n) { asm volatile("bar.
 
 // MODE 0: plain sampling (no forced symbols, no dumps, no stamps, no self-test predicate); MODE 1: the instantiation that
 // wrnn_selftest_lost_word runs (one CTA withholds one publication); MODE 2: the one with the phase stamps of wrnn_phase_profile
-// (and with forced symbols and dumps, like mode 1)
+// (and with forced symbols and dumps, like mode 1); MODE 4: stamp code without forced symbols and dumps
 template <int MODE>
 __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParams p)
 {
@@ -173,7 +173,7 @@ __global__ void __launch_bounds__(512, 1) resident_multi_kernel(const MultiParam
     Waiter wt{p.status, p.limit_ns};
     bool my_bad = false;
     const int g4 = lane >> 2, t4 = lane & 3;
-    constexpr bool HOOK = MODE == 1, PROF = MODE == 2, DBG = MODE != 0;
+    constexpr bool HOOK = MODE == 1, PROF = MODE == 2 || MODE == 4, DBG = MODE == 1 || MODE == 2;
     const bool prof_on = PROF && p.prof != nullptr && cta == 0 && warp == 0;
     __shared__ long long s_prof[16];
     if (tid < 16) s_prof[tid] = 0;
@@ -667,7 +667,9 @@ int resmulti_prepare(wrnn_model *m)
         cudaFuncSetAttribute(resident_multi_kernel<1>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
         cudaFuncSetAttribute(resident_multi_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess ||
         cudaFuncSetAttribute(resident_multi_kernel<2>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
-        cudaFuncSetAttribute(resident_multi_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
+        cudaFuncSetAttribute(resident_multi_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<4>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess ||
+        cudaFuncSetAttribute(resident_multi_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, k.smem_bytes) != cudaSuccess) {
         cudaGetLastError();
         m->err = "multi-stream resident kernel does not fit in shared memory";
         return WRNN_ERR_UNSUPPORTED;
@@ -812,13 +814,15 @@ int resmulti_run(wrnn_model *m, const StepArgs &a, cudaStream_t s)
     if (cudaMemsetAsync(m->status, 0, sizeof(DevStatus), s) != cudaSuccess) return WRNN_ERR_CUDA;
     cudaLaunchConfig_t cfg; cudaLaunchAttribute at[2];
     multi_fill_launch(k, &cfg, at, s, coop_launch_allowed());
-    // Plain sampling of up to four rows runs the instantiation without stamps, forced symbols and dumps; above four rows the
-    // one that carries that (unexecuted) code is the faster one: 16 rows 9.55 us per lock-step against 9.95 without it, 4 rows
-    // 7.21 against 7.02 (same call, alternating): the compiler orders the half-step differently around the clock reads.
+    // Plain sampling of up to four rows runs the instantiation without stamps, forced symbols and dumps (mode 0); above four
+    // rows the one that carries the (unexecuted) stamp code but no forced symbols or dumps (mode 4) is the fastest: 16 rows 9.52 us
+    // per lock-step against 9.55 with everything compiled in and 9.95 with nothing, 4 rows 7.21 against 6.97 (same call,
+    // alternating): the compiler orders the half-step differently around the clock reads.
     const bool teacher = p.c_forced || p.f_forced || p.dbg_gates || p.dbg_h || p.dbg_logits;
-    const int mode = m->dbg_skip_cta >= 0 ? 1 : (p.prof || teacher || a.batch > MODE0_MAX_ROWS) ? 2 : 0;
+    const int mode = m->dbg_skip_cta >= 0 ? 1 : (p.prof || teacher) ? 2 : a.batch > MODE0_MAX_ROWS ? 4 : 0;
     const cudaError_t e = mode == 1 ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<1>, p)
                           : mode == 2 ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<2>, p)
+                          : mode == 4 ? cudaLaunchKernelEx(&cfg, resident_multi_kernel<4>, p)
                                       : cudaLaunchKernelEx(&cfg, resident_multi_kernel<0>, p);
     if (e != cudaSuccess) {
         m->err = std::string("multi-stream resident kernel launch failed: ") + cudaGetErrorString(e);

@@ -381,6 +381,57 @@ def test_checked_build_of_the_resident_kernel(env):
         B.wrnn_destroy(m)
 
 
+@pytest.mark.parametrize("case", ["lean", "fused", "fp32", "multi4", "multi16"])
+def test_phase_profile_runs_another_instantiation_with_the_same_samples(env, case):
+    """`wrnn_phase_profile` switches the resident kernels to the instantiation that carries the clock stamps; plain sampling,
+    teacher forcing and the self-test each run one of their own.  The stamped one must draw the same samples as the plain one
+    (same inputs, same seed), report cycles for its sixteen named phases, and leave the model usable without stamps."""
+    torch, B = env
+    dev = "cuda:0"
+    n = 300
+    if case == "fp32":
+        wl = synth.WORKLOADS[0]
+    else:
+        wl = synth.WORKLOADS[1]
+    batch = {"multi4": 4, "multi16": 16}.get(case, 1)
+    if case == "fused":
+        w = synth.make_weights(896, cond_dim=64, n_inputs=12, n_logits=64)
+        cond_np = synth.make_cond(1, 10, 64)
+        m = B.wrnn_create(w, "bf16", max_batch=1, variant=1)
+    else:
+        w, masks, cond_np = synth.build_workload(wl)
+        if batch > 1:
+            cond_np = np.repeat(cond_np[:1], batch, axis=0).copy()
+        m = B.wrnn_create(w, wl.dtype, max_batch=batch)
+    try:
+        cond = torch.from_numpy(cond_np).to(dev)
+
+        def run():
+            if case == "fused":
+                ab = torch.zeros((2, n), dtype=torch.int16, device=dev)
+                B.wrnn_fs2_sample(m, cond, n, SEED, ab)
+                out = ab
+            else:
+                out = torch.zeros((batch, n), dtype=torch.int16, device=dev)
+                B.wrnn_sample(m, cond, n, batch, SEED, out, row_offset_mul=1 if batch > 1 else 0)
+            torch.cuda.synchronize()
+            assert B.wrnn_poll_status(m) == 0, B.wrnn_last_error(m)
+            return out.cpu().numpy()
+
+        plain = run()
+        B.wrnn_phase_profile(m, True)
+        stamped = run()
+        cycles = B.wrnn_phase_cycles(m)
+        names = B.wrnn_phase_names(m)
+        B.wrnn_phase_profile(m, False)
+        again = run()
+        assert np.array_equal(plain, stamped) and np.array_equal(plain, again)
+        assert len(names) == 16 and all(names)
+        assert sum(cycles) > 1000 * n and min(cycles[:12]) > 0, cycles
+    finally:
+        B.wrnn_destroy(m)
+
+
 def test_fold_unfold_exact_permutation(env):
     torch, B = env
     for n, Bf in [(24000, 16), (16, 16), (35, 5), (7, 1)]:

@@ -7,10 +7,12 @@
 //     (needed by the gates at the end of the half-step, not by the head) are multiplied while the hidden layer
 //     crosses the cluster;
 //   * K-split partial sums are added by one warp (lane = row) instead of by every sending warp;
-//   * the output layer is one row per warp in plain fp32 FMAs on the received hidden layer (no bf16 split, no partial
-//     sums, no CTA barrier before it): a lane keeps a 14-element slice of the hidden layer, five shuffles add up;
+//   * the output layer is plain fp32 FMAs on the received hidden layer (no bf16 split, no partial sums, no CTA barrier
+//     before it): two rows per warp on eight warps, a lane the element pairs lane, lane + 32, ... of both, six shuffles add up;
 //   * both cluster exchanges are asynchronous stores that count their bytes on the receiver's mbarrier;
-//   * the uniform, the forced symbol and the gate offsets of a half-step are pinned before its first wait.
+//   * the uniform, the forced symbol and the gate offsets of a half-step are pinned before its first wait;
+//   * the body of a half-step exists once per half, and plain sampling, teacher forcing (forced symbols, dumps), the phase
+//     stamps and the self-test predicate each run an instantiation of their own (template parameter MODE).
 // Hidden-layer and recurrent products are m16n8k16 bf16 MMAs on A-fragment-packed weights with the fp32 input as an
 // exact three-way bf16 split.  Every wait is bounded; a CTA that gives up records where and all CTAs leave through the
 // final cluster barrier.

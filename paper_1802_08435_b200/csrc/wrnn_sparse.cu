@@ -9,9 +9,11 @@
 // the signal).
 // Each CTA owns Hh/(16 NC) coarse and as many fine units (their block rows of R, compressed: block column index +
 // 16 bf16 per kept block), Hh/16 rows of O1 and O3 (compressed block rows) and 16 rows of the dense O2 and O4
-// (mma.sync A fragments).  Sparse rows: four lanes share a block row, each lane takes every fourth kept block
-// (two 16-byte weight loads, four activations, 16 FMAs), a four-value reduce-scatter finishes the rows; the rows
-// are sorted by length and stored sliced by warp so that every shared-memory load of a warp is one contiguous run.
+// (row-major bf16, multiplied as fp32 FMAs on the received hidden layer: 16 warps = 4 groups of four rows x 4 quarters of K).
+// Sparse rows: four (or eight) lanes share a block row, each lane takes every fourth (eighth) kept block (two 16-byte weight
+// loads, four activations, 16 FMAs), a four-value reduce-scatter finishes the rows; the rows are sorted by length and stored
+// sliced by warp so that every shared-memory load of a warp is one contiguous run; with four clusters the hidden-layer rows sit
+// in the slices of warps 0..3 and the rows of R in those of warps 16..19, which the exchanges do not wait for.
 // The step itself is the two-half schedule of the dense resident kernel (Fig. 1's order).
 //
 // Every wait is bounded; all CTAs leave through the final cluster barrier.

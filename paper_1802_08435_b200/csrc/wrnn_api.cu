@@ -137,7 +137,7 @@ static bool use_resf32(const wrnn_model *m, int batch)
 }
 
 // two or four streams of a dense bf16 model: pairs on the two-stream form of the resident kernel, one pair after the other
-// (the default for two rows only; three and more rows go to the multi-stream resident kernel where the model has one)
+// (the fallback of the multi-stream resident kernel, which takes 2 to 16 rows where the model has one)
 static bool use_pair(const wrnn_model *m, int batch)
 {
     if (m->kernel != WRNN_KERNEL_AUTO && m->kernel != WRNN_KERNEL_RESIDENT) return false;
@@ -236,8 +236,9 @@ static int run_steps(wrnn_model *m, StepArgs &a, cudaStream_t s)
     }
     if (use_reslean(m, a.batch)) return reslean_run(m, a, s);
     if (use_resident(m, a.batch)) return resident_run(m, a, s);
-    // two rows: the two-stream kernel (7.5 us per step against 8.2 on the multi-stream kernel); 3 to 16: the multi-stream kernel
-    if (use_multi(m, a.batch) && !(a.batch == 2 && use_pair(m, 2))) return resmulti_run(m, a, s);
+    // 2 to 16 rows: the multi-stream kernel (two rows 6.5 us per lock-step against 7.7 on the two-stream kernel, which serves
+    // them where the multi-stream kernel does not apply or under WRNN_NO_MULTI=1)
+    if (use_multi(m, a.batch)) return resmulti_run(m, a, s);
     if (use_pair(m, a.batch)) {
         for (int pair = 0; pair < a.batch / 2; ++pair) {
             rc = resident_pair_run(m, a, pair, s);
@@ -841,7 +842,7 @@ int wrnn_launch_info(wrnn_model *m, int32_t batch, int32_t *kernel, int32_t *n_c
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resident_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
     }
-    if (use_multi(m, batch) && !(batch == 2 && use_pair(m, 2))) {
+    if (use_multi(m, batch)) {
         if (kernel) *kernel = WRNN_KERNEL_RESIDENT;
         return resmulti_launch_info(m, batch, n_ctas, n_threads, smem_bytes, weight_bytes_per_step);
     }

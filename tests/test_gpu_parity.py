@@ -291,6 +291,8 @@ def test_lost_word_times_out_cleanly_in_every_kernel(env, case):
         dtype, kern, n_ctas_min = wl.dtype, B.WRNN_KERNEL_AUTO, 100
         if case == "first-resident":
             envset["WRNN_RESIDENT_LEAN"] = "0"
+        if case == "pair":
+            envset["WRNN_NO_MULTI"] = "1"            # (two rows go to the multi-stream kernel by default)
     elif case == "fused":
         wl = synth.WORKLOADS[8]
         w, masks, cond = synth.build_workload(wl)
@@ -590,7 +592,7 @@ def test_multi_stream_resident_kernels(env, batch, form):
     if form == "pair":
         os.environ["WRNN_NO_MULTI"] = "1"
     else:
-        os.environ["WRNN_NO_PAIR"] = "1"         # (two rows go to the two-stream kernel by default)
+        os.environ["WRNN_NO_PAIR"] = "1"         # (diagnostic switch; two rows go to the multi-stream kernel by default anyway)
     m = B.wrnn_create(w, wl.dtype, max_batch=batch)
     try:
         info = B.wrnn_launch_info(m, batch)
@@ -622,7 +624,7 @@ def test_multi_stream_every_row_count(env):
     stream per cluster up to seven): 160 teacher-forced steps of every row against the oracle."""
     torch, B = env
     wl = synth.WORKLOADS[7]
-    os.environ["WRNN_NO_PAIR"] = "1"             # (two rows go to the two-stream kernel by default)
+    os.environ["WRNN_NO_PAIR"] = "1"             # (diagnostic switch; two rows go to the multi-stream kernel by default anyway)
     try:
         for batch in range(2, 17):
             w, masks, cond = synth.build_workload(wl, batch=batch)

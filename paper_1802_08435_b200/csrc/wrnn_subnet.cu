@@ -282,7 +282,7 @@ static int ensure_acts(wrnn_subscale_net *n, int n_seg, int n_pos)
     return WRNN_OK;
 }
 
-constexpr int SN_BN_CONV = 96, SN_BN_RES = 128, SN_BN_OUT = 64;
+constexpr int SN_BN_CONV = 96, SN_BN_RES = 96, SN_BN_OUT = 64;
 constexpr int SN_ST_CONV = 4, SN_ST_RES = 4, SN_ST_OUT = 4;
 template <int BN, int ST> constexpr int sn_smem() { return ST * (2 * SN_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024; }
 

@@ -93,6 +93,10 @@ __global__ void __launch_bounds__(SN_THREADS, 1) subnet_gemm_kernel(const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
+    // Programmatic dependent launch: the next product of the chain may be scheduled now (its CTAs set up their barriers and
+    // TMEM on SMs that this grid has left or never used); nothing of the previous product is read before it has completed.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const int nkb = p.taps * p.n_kb_tap;
     const int arow0 = seg * p.n_alloc + mt * SN_BM;          // first activation row (position) of this tile
@@ -284,6 +288,20 @@ static int ensure_acts(wrnn_subscale_net *n, int n_seg, int n_pos)
 
 constexpr int SN_BN_CONV = 96, SN_BN_RES = 96, SN_BN_OUT = 64;
 constexpr int SN_ST_CONV = 4, SN_ST_RES = 4, SN_ST_OUT = 4;
+// launch with programmatic stream serialization: the kernel may start while its predecessor in the stream drains (it waits for
+// the predecessor's completion itself, with griddepcontrol.wait, before it reads anything)
+template <typename K>
+static void pdl_launch(K kernel, dim3 grid, int smem, cudaStream_t s, const CUtensorMap &a, const CUtensorMap &b, const CUtensorMap &w, const SubnetGemmParams &p)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(SN_THREADS); cfg.dynamicSmemBytes = (size_t)smem; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, a, b, w, p);
+}
+
 template <int BN, int ST> constexpr int sn_smem() { return ST * (2 * SN_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024; }
 
 // The whole network for the segments of one call: v[seg][n_steps][cond_dim] (the conditioning vectors the stepping call
@@ -309,20 +327,20 @@ int subnet_run(wrnn_subscale_net *n, const int16_t *hist, const float *frames, i
         // a_l = relu(conv): K = taps x res_ch, N = conv_ch
         p.n_kb_tap = n->res_ch / TC_BK; p.taps = n->taps; p.dil = d; p.w_row0 = l * n->taps * n->conv_ch; p.w_tap_rows = n->conv_ch;
         p.n_pos = need; p.C_out = n->conv_ch; p.bias = n->b_conv + (size_t)l * n->conv_ch; p.oh = n->ah; p.ol = n->al; p.xf = nullptr; p.relu_parts = 0;
-        subnet_gemm_kernel<SN_BN_CONV, SN_CONV, SN_ST_CONV><<<dim3(n->conv_ch / SN_BN_CONV, mtiles, n_rows), SN_THREADS, sn_smem<SN_BN_CONV, SN_ST_CONV>(), s>>>(
-            n->tmXh, n->tmXl, n->tmWc, p);
+        pdl_launch(subnet_gemm_kernel<SN_BN_CONV, SN_CONV, SN_ST_CONV>, dim3(n->conv_ch / SN_BN_CONV, mtiles, n_rows), sn_smem<SN_BN_CONV, SN_ST_CONV>(), s,
+                   n->tmXh, n->tmXl, n->tmWc, p);
         // x_{l+1} = x_l + W_res a_l + b_res: K = conv_ch, N = res_ch
         p.n_kb_tap = n->conv_ch / TC_BK; p.taps = 1; p.dil = 0; p.w_row0 = l * n->res_ch; p.w_tap_rows = 0;
         p.C_out = n->res_ch; p.bias = n->b_res + (size_t)l * n->res_ch; p.oh = n->xh; p.ol = n->xl; p.xf = n->xf; p.relu_parts = l == n->n_layers - 1;
-        subnet_gemm_kernel<SN_BN_RES, SN_RES, SN_ST_RES><<<dim3(n->res_ch / SN_BN_RES, mtiles, n_rows), SN_THREADS, sn_smem<SN_BN_RES, SN_ST_RES>(), s>>>(
-            n->tmAh, n->tmAl, n->tmWr, p);
+        pdl_launch(subnet_gemm_kernel<SN_BN_RES, SN_RES, SN_ST_RES>, dim3(n->res_ch / SN_BN_RES, mtiles, n_rows), sn_smem<SN_BN_RES, SN_ST_RES>(), s,
+                   n->tmAh, n->tmAl, n->tmWr, p);
         g_launches += 2;
     }
     // v = frames + W_out relu(x_last) + b_out
     p.n_kb_tap = n->res_ch / TC_BK; p.taps = 1; p.dil = 0; p.w_row0 = 0; p.w_tap_rows = 0; p.n_pos = n_steps; p.C_out = 0; p.bias = nullptr;
     p.v = v; p.n_steps = n_steps; p.cond_dim = n->cond_dim; p.frames = frames; p.n_frames = n_frames; p.hop = hop; p.Bsub = n->B; p.b_out = n->b_out;
-    subnet_gemm_kernel<SN_BN_OUT, SN_OUT, SN_ST_OUT><<<dim3(1, (n_steps + SN_BM - 1) / SN_BM, n_rows), SN_THREADS, sn_smem<SN_BN_OUT, SN_ST_OUT>(), s>>>(
-        n->tmXh, n->tmXl, n->tmWo, p);
+    pdl_launch(subnet_gemm_kernel<SN_BN_OUT, SN_OUT, SN_ST_OUT>, dim3(1, (n_steps + SN_BM - 1) / SN_BM, n_rows), sn_smem<SN_BN_OUT, SN_ST_OUT>(), s,
+               n->tmXh, n->tmXl, n->tmWo, p);
     ++g_launches;
     if (cudaGetLastError() != cudaSuccess) { n->err = "conditioning network launch failed"; return WRNN_ERR_CUDA; }
     return WRNN_OK;
